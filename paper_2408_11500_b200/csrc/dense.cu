@@ -1,0 +1,388 @@
+// Dense kernels of the layer: grouped (per-slice) row-panel GEMM with the fused epilogues of
+// Eq. 6-7, grouped weight gradients with a deterministic two-stage reduction, the cross-entropy
+// of Eq. 10 and the Adam update.  This file holds the CUDA-core (FFMA) implementations.
+#include "common.cuh"
+#include "kernels.cuh"
+
+namespace sgcn {
+namespace {
+
+__device__ __forceinline__ float ldf(const float* p) { return __ldg(p); }
+__device__ __forceinline__ float ldf(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+__device__ __forceinline__ void stf(float* p, float v) { *p = v; }
+__device__ __forceinline__ void stf(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
+
+// ------------------------------------------------------------------------------ grouped GEMM
+constexpr int GM = 128;   // rows per CTA
+constexpr int GK = 32;    // reduction slab
+
+template <typename TA, typename TC, int BN, int TM, int TN>
+__global__ void __launch_bounds__(256) gemm_kernel(const GemmArgs a) {
+    static_assert((GM / TM) * (BN / TN) == 256, "thread tiling must cover the CTA tile");
+    __shared__ float As[GK][GM + 4];
+    __shared__ float Bs[GK][BN];
+    const int g = blockIdx.z;
+    const int64_t row0 = (int64_t)blockIdx.x * GM;
+    const int n0 = blockIdx.y * BN;
+    const int tid = threadIdx.x;
+    const int tx = tid % (BN / TN), ty = tid / (BN / TN);
+    const TA* A = static_cast<const TA*>(a.A) + a.a_start[g];
+    const uint8_t* am = a.a_mask ? a.a_mask + a.a_start[g] : nullptr;
+    const float* B = a.B + (int64_t)g * a.b_gstride;
+    float acc[TM][TN];
+#pragma unroll
+    for (int i = 0; i < TM; ++i)
+#pragma unroll
+        for (int j = 0; j < TN; ++j) acc[i][j] = 0.f;
+
+    for (int k0 = 0; k0 < a.K; k0 += GK) {
+        // A slab: 128 rows x 32 k, one warp reads 32 consecutive k of a row
+        {
+            const int kk = tid & 31;
+            const int k = k0 + kk;
+#pragma unroll
+            for (int i = 0; i < GM / 8; ++i) {
+                const int r = (tid >> 5) + 8 * i;
+                const int64_t row = row0 + r;
+                float v = 0.f;
+                if (row < a.M && k < a.K) {
+                    v = ldf(A + row * a.lda + k);
+                    if (am) v *= (float)am[row * a.a_mask_ld + k];
+                }
+                As[kk][r] = v;
+            }
+        }
+        // B slab: 32 k x BN
+        for (int e = tid; e < GK * BN; e += 256) {
+            const int kk = e / BN, nn = e % BN;
+            const int k = k0 + kk, n = n0 + nn;
+            float v = 0.f;
+            if (k < a.K && n < a.N) v = a.b_trans ? __ldg(B + (int64_t)n * a.ldb + k) : __ldg(B + (int64_t)k * a.ldb + n);
+            Bs[kk][nn] = v;
+        }
+        __syncthreads();
+#pragma unroll 8
+        for (int kk = 0; kk < GK; ++kk) {
+            float av[TM], bv[TN];
+#pragma unroll
+            for (int i = 0; i < TM; i += 4) {
+                const float4 t = *reinterpret_cast<const float4*>(&As[kk][ty * TM + i]);
+                av[i] = t.x; av[i + 1] = t.y; av[i + 2] = t.z; av[i + 3] = t.w;
+            }
+#pragma unroll
+            for (int j = 0; j < TN; ++j) bv[j] = Bs[kk][tx * TN + j];
+#pragma unroll
+            for (int i = 0; i < TM; ++i)
+#pragma unroll
+                for (int j = 0; j < TN; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+
+    TC* C = static_cast<TC*>(a.C);
+    const int cs = a.c_start[g];
+#pragma unroll
+    for (int i = 0; i < TM; ++i) {
+        const int64_t row = row0 + ty * TM + i;
+        if (row >= a.M) continue;
+#pragma unroll
+        for (int j = 0; j < TN; ++j) {
+            const int n = n0 + tx * TN + j;
+            if (n >= a.N) continue;
+            const int col = cs + n;
+            float x = acc[i][j];
+            if (a.bias) x += __ldg(a.bias + g * a.N + n);
+            if (a.relu) {
+                if (a.mask_out) a.mask_out[row * a.mask_ld + col] = x > 0.f ? 1 : 0;
+                x = fmaxf(x, 0.f);
+            }
+            if (a.post1) x += __ldg(a.post1 + g * a.N + n);
+            if (a.post2) x += __ldg(a.post2 + g * a.N + n);
+            if (a.mul_pos) {
+                const float pv = a.mul_pos_dtype == SLICEGCN_F32
+                                     ? static_cast<const float*>(a.mul_pos)[row * a.mul_pos_ld + col]
+                                     : __bfloat162float(static_cast<const __nv_bfloat16*>(a.mul_pos)[row * a.mul_pos_ld + col]);
+                x = pv > 0.f ? x : 0.f;
+            }
+            if (a.accumulate) x += ldf(C + row * a.ldc + col);
+            stf(C + row * a.ldc + col, x);
+        }
+    }
+}
+
+template <typename TA, typename TC>
+slicegcn_status_t gemm_dispatch(const GemmArgs& a, cudaStream_t st) {
+    const unsigned gx = (unsigned)((a.M + GM - 1) / GM);
+    if (a.N <= 16) {
+        dim3 grid(gx, 1, a.groups);
+        gemm_kernel<TA, TC, 16, 4, 2><<<grid, 256, 0, st>>>(a);
+    } else if (a.N <= 32) {
+        dim3 grid(gx, 1, a.groups);
+        gemm_kernel<TA, TC, 32, 4, 4><<<grid, 256, 0, st>>>(a);
+    } else {
+        dim3 grid(gx, (a.N + 63) / 64, a.groups);
+        gemm_kernel<TA, TC, 64, 8, 4><<<grid, 256, 0, st>>>(a);
+    }
+    SGCN_LAUNCH_CHECK();
+    count_launch();
+    return SLICEGCN_OK;
+}
+
+// ------------------------------------------------------------------------------ weight gradient
+constexpr int WT = 64;    // tile of dW (k and n)
+constexpr int WR = 32;    // rows per smem slab
+
+template <typename TA>
+__global__ void __launch_bounds__(256) wgrad_partial_kernel(const WgradArgs a, float* scratch, int n_chunks,
+                                                            int64_t rows_per_chunk, int Kext) {
+    __shared__ float As[WR][WT];
+    __shared__ float Bs[WR][WT];
+    const int g = blockIdx.z;
+    const int tiles_n = (a.N + WT - 1) / WT;
+    const int k0 = (blockIdx.y / tiles_n) * WT, n0 = (blockIdx.y % tiles_n) * WT;
+    const int chunk = blockIdx.x;
+    const int64_t r_begin = chunk * rows_per_chunk;
+    const int64_t r_end = min(a.M, r_begin + rows_per_chunk);
+    const int tid = threadIdx.x;
+    const int tx = tid & 15, ty = tid >> 4;
+    const TA* A = static_cast<const TA*>(a.A) + a.a_start[g];
+    const float* B = a.B + a.b_start[g];
+    const uint8_t* bm = a.b_mask ? a.b_mask + a.b_start[g] : nullptr;
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+    for (int64_t rb = r_begin; rb < r_end; rb += WR) {
+        const int c = tid & 63;
+#pragma unroll
+        for (int i = 0; i < WR / 4; ++i) {
+            const int r = (tid >> 6) + 4 * i;
+            const int64_t row = rb + r;
+            float av = 0.f, bv = 0.f;
+            if (row < r_end) {
+                const int k = k0 + c, n = n0 + c;
+                if (k < a.K)
+                    av = ldf(A + row * a.lda + k);
+                else if (k == a.K && Kext > a.K)
+                    av = 1.f;   // the extra row of ones yields the bias gradient (column sums)
+                if (n < a.N) {
+                    bv = __ldg(B + row * a.ldb + n);
+                    if (bm) bv *= (float)bm[row * a.b_mask_ld + n];
+                }
+            }
+            As[r][c] = av;
+            Bs[r][c] = bv;
+        }
+        __syncthreads();
+#pragma unroll 8
+        for (int r = 0; r < WR; ++r) {
+            const float4 a4 = *reinterpret_cast<const float4*>(&As[r][ty * 4]);
+            const float4 b4 = *reinterpret_cast<const float4*>(&Bs[r][tx * 4]);
+            const float av[4] = {a4.x, a4.y, a4.z, a4.w};
+            const float bv[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+    float* out = scratch + ((int64_t)chunk * a.groups + g) * Kext * a.N;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int k = k0 + ty * 4 + i;
+        if (k >= Kext) continue;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int n = n0 + tx * 4 + j;
+            if (n < a.N) out[(int64_t)k * a.N + n] = acc[i][j];
+        }
+    }
+}
+
+__global__ void wgrad_reduce_kernel(const float* scratch, int n_chunks, int groups, int K, int Kext, int N, float* dW,
+                                    float* dbias, float* dbias2) {
+    const int64_t per = (int64_t)groups * Kext * N;
+    int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (i >= per) return;
+    float s = 0.f;
+    for (int c = 0; c < n_chunks; ++c) s += scratch[c * per + i];   // fixed order
+    const int g = (int)(i / ((int64_t)Kext * N));
+    const int rem = (int)(i % ((int64_t)Kext * N));
+    const int k = rem / N, n = rem % N;
+    if (k < K) {
+        if (dW) dW[((int64_t)g * K + k) * N + n] = s;
+    } else {
+        if (dbias) dbias[g * N + n] = s;
+        if (dbias2) dbias2[g * N + n] = s;
+    }
+}
+
+void wgrad_plan(int64_t M, int groups, int K, int N, bool bias, int* n_chunks, int64_t* rows_per_chunk, int* Kext) {
+    *Kext = K + (bias ? 1 : 0);
+    const int tiles = ((*Kext + WT - 1) / WT) * ((N + WT - 1) / WT) * groups;
+    int64_t want = (148 * 4 + tiles - 1) / tiles;
+    int64_t max_chunks = (M + 1023) / 1024;
+    if (want > max_chunks) want = max_chunks;
+    if (want < 1) want = 1;
+    int64_t rpc = (M + want - 1) / want;
+    rpc = (rpc + WR - 1) / WR * WR;
+    *rows_per_chunk = rpc;
+    *n_chunks = (int)((M + rpc - 1) / rpc);
+}
+
+// ------------------------------------------------------------------------------ small kernels
+__global__ void mask_mul_kernel(int64_t M, int N, const float* in, int64_t ld_in, const uint8_t* mask, int64_t ld_mask,
+                                float* out, int64_t ld_out) {
+    const int64_t total = M * N;
+    int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (; i < total; i += stride) {
+        const int64_t r = i / N;
+        const int c = (int)(i % N);
+        out[r * ld_out + c] = mask[r * ld_mask + c] ? in[r * ld_in + c] : 0.f;
+    }
+}
+
+// one warp per training row
+__global__ void softmax_ce_kernel(int C, const float* logits, const int32_t* labels, const int32_t* train_idx,
+                                  int64_t n_train, float inv_n, float* dlogits, float* row_loss) {
+    const int lane = threadIdx.x & 31;
+    const int64_t t = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
+    if (t >= n_train) return;
+    const int64_t r = train_idx ? train_idx[t] : t;
+    const float* z = logits + r * C;
+    float mx = -INFINITY;
+    for (int c = lane; c < C; c += 32) mx = fmaxf(mx, z[c]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    float s = 0.f;
+    for (int c = lane; c < C; c += 32) s += expf(z[c] - mx);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    const int y = labels[r];
+    const float lse = mx + logf(s);
+    if (lane == 0) row_loss[t] = lse - z[y];
+    const float inv_s = 1.f / s;
+    for (int c = lane; c < C; c += 32) {
+        float p = expf(z[c] - mx) * inv_s;
+        dlogits[r * C + c] = (p - (c == y ? 1.f : 0.f)) * inv_n;
+    }
+}
+
+// single CTA, fixed summation order: thread t sums elements t, t+1024, ...; then a tree in smem
+__global__ void __launch_bounds__(1024) mean_reduce_kernel(const float* v, int64_t n, float scale, float* out) {
+    __shared__ float sm[1024];
+    float s = 0.f;
+    for (int64_t i = threadIdx.x; i < n; i += 1024) s += v[i];
+    sm[threadIdx.x] = s;
+    __syncthreads();
+    for (int o = 512; o > 0; o >>= 1) {
+        if (threadIdx.x < o) sm[threadIdx.x] += sm[threadIdx.x + o];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) *out = sm[0] * scale;
+}
+
+__global__ void adam_kernel(int64_t count, float* theta, const float* grad, float* m1, float* m2, float lr, float b1,
+                            float b2, float eps, float wd, float c1, float c2) {
+    int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (i >= count) return;
+    const float th = theta[i];
+    const float g = grad[i] + wd * th;
+    const float m = b1 * m1[i] + (1.f - b1) * g;
+    const float v = b2 * m2[i] + (1.f - b2) * g * g;
+    m1[i] = m;
+    m2[i] = v;
+    theta[i] = th - lr * (m / c1) / (sqrtf(v / c2) + eps);
+}
+
+}  // namespace
+
+slicegcn_status_t gemm_run(const GemmArgs& a, cudaStream_t st) {
+    if (a.M < 1 || a.groups < 1 || a.groups > SLICEGCN_MAX_SLICES || a.N < 1 || a.K < 0)
+        SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "gemm: bad shape");
+    const bool abf = a.a_dtype == SLICEGCN_BF16, cbf = a.c_dtype == SLICEGCN_BF16;
+    if (!abf && !cbf) return gemm_dispatch<float, float>(a, st);
+    if (abf && cbf) return gemm_dispatch<__nv_bfloat16, __nv_bfloat16>(a, st);
+    if (abf && !cbf) return gemm_dispatch<__nv_bfloat16, float>(a, st);
+    return gemm_dispatch<float, __nv_bfloat16>(a, st);
+}
+
+int64_t wgrad_scratch_bytes(int64_t M, int groups, int K, int N) {
+    int64_t best = 0;
+    for (int bias = 0; bias < 2; ++bias) {
+        int n_chunks, Kext;
+        int64_t rpc;
+        wgrad_plan(M, groups, K, N, bias != 0, &n_chunks, &rpc, &Kext);
+        const int64_t b = (int64_t)n_chunks * groups * Kext * N * (int64_t)sizeof(float);
+        if (b > best) best = b;
+    }
+    return best;
+}
+
+slicegcn_status_t wgrad_run(const WgradArgs& a, void* scratch, int64_t scratch_bytes, cudaStream_t st) {
+    if (a.M < 1 || a.groups < 1 || a.groups > SLICEGCN_MAX_SLICES || a.N < 1 || a.K < 0)
+        SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "wgrad: bad shape");
+    const bool bias = a.dbias || a.dbias2;
+    if (a.K == 0 && !bias) return SLICEGCN_OK;
+    int n_chunks, Kext;
+    int64_t rpc;
+    wgrad_plan(a.M, a.groups, a.K, a.N, bias, &n_chunks, &rpc, &Kext);
+    const int64_t need = (int64_t)n_chunks * a.groups * Kext * a.N * (int64_t)sizeof(float);
+    if (!scratch || scratch_bytes < need)
+        SGCN_FAIL(SLICEGCN_ERR_ALLOC, "wgrad: scratch too small (%lld < %lld)", (long long)scratch_bytes, (long long)need);
+    dim3 grid(n_chunks, ((Kext + WT - 1) / WT) * ((a.N + WT - 1) / WT), a.groups);
+    if (a.a_dtype == SLICEGCN_BF16)
+        wgrad_partial_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(a, static_cast<float*>(scratch), n_chunks, rpc, Kext);
+    else
+        wgrad_partial_kernel<float><<<grid, 256, 0, st>>>(a, static_cast<float*>(scratch), n_chunks, rpc, Kext);
+    SGCN_LAUNCH_CHECK();
+    const int64_t per = (int64_t)a.groups * Kext * a.N;
+    wgrad_reduce_kernel<<<(unsigned)((per + 255) / 256), 256, 0, st>>>(static_cast<const float*>(scratch), n_chunks,
+                                                                      a.groups, a.K, Kext, a.N, a.dW, a.dbias, a.dbias2);
+    SGCN_LAUNCH_CHECK();
+    count_launch(2);
+    return SLICEGCN_OK;
+}
+
+slicegcn_status_t mask_mul_run(int64_t M, int N, const float* in, int64_t ld_in, const uint8_t* mask, int64_t ld_mask,
+                               float* out, int64_t ld_out, cudaStream_t st) {
+    int64_t blocks = (M * N + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    mask_mul_kernel<<<(unsigned)blocks, 256, 0, st>>>(M, N, in, ld_in, mask, ld_mask, out, ld_out);
+    SGCN_LAUNCH_CHECK();
+    count_launch();
+    return SLICEGCN_OK;
+}
+
+slicegcn_status_t softmax_ce_run(int64_t n, int C, const float* logits, const int32_t* labels, const int32_t* train_idx,
+                                 int64_t n_train, float* dlogits, float* row_loss, float* loss_out, cudaStream_t st) {
+    if (train_idx) SGCN_CUDA(cudaMemsetAsync(dlogits, 0, sizeof(float) * n * C, st));
+    const int64_t cnt = train_idx ? n_train : n;
+    if (cnt < 1) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "empty training set");
+    softmax_ce_kernel<<<(unsigned)((cnt + 7) / 8), 256, 0, st>>>(C, logits, labels, train_idx, cnt, 1.0f / (float)cnt,
+                                                                  dlogits, row_loss);
+    SGCN_LAUNCH_CHECK();
+    count_launch();
+    if (loss_out) {
+        mean_reduce_kernel<<<1, 1024, 0, st>>>(row_loss, cnt, 1.0f / (float)cnt, loss_out);
+        SGCN_LAUNCH_CHECK();
+        count_launch();
+    }
+    return SLICEGCN_OK;
+}
+
+slicegcn_status_t adam_run(int64_t count, float* theta, const float* grad, float* m1, float* m2, float lr, float beta1,
+                           float beta2, float eps, float weight_decay, int step, cudaStream_t st) {
+    const float c1 = (float)(1.0 - pow((double)beta1, (double)step));
+    const float c2 = (float)(1.0 - pow((double)beta2, (double)step));
+    adam_kernel<<<(unsigned)((count + 255) / 256), 256, 0, st>>>(count, theta, grad, m1, m2, lr, beta1, beta2, eps,
+                                                                  weight_decay, c1, c2);
+    SGCN_LAUNCH_CHECK();
+    count_launch();
+    return SLICEGCN_OK;
+}
+
+}  // namespace sgcn

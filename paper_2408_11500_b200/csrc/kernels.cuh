@@ -1,0 +1,94 @@
+// Internal launch interfaces shared by the translation units of the library.
+#pragma once
+
+#include "common.cuh"
+
+namespace sgcn {
+
+// ---- SpMM -------------------------------------------------------------------------------------
+// Optional fused epilogue of the aggregation (used by transform-first layers):
+//   y = dinv_i * acc + bias[col];  if relu: mask = (y > 0), y = max(y, 0);  if accumulate: y += Y_old
+struct SpmmEpilogue {
+    const float* bias = nullptr;
+    int relu = 0;
+    uint8_t* mask = nullptr;
+    int64_t mask_ld = 0;
+    int accumulate = 0;
+};
+int64_t spmm_partial_bytes(const slicegcn_graph* g, int width);
+slicegcn_status_t spmm_run(const slicegcn_graph* g, bool transpose, int in_dtype, int out_dtype, const void* X,
+                           int64_t ldx, void* Y, int64_t ldy, int width, const SpmmEpilogue* epi, void* ws,
+                           int64_t ws_bytes, cudaStream_t st);
+
+// ---- grouped row-panel GEMM  C_g = epilogue(A_g * B_g) ----------------------------------------
+// Group g (one slice) reads K columns of A starting at a_start[g], multiplies by its own K x N
+// block of B and writes N columns of C starting at c_start[g].  Epilogue, in this order:
+//   x = acc + bias[g][n];  if relu: (mask_out = x > 0), x = max(x, 0);  x += post1[g][n] + post2[g][n];
+//   if mul_pos: x *= (P[r, c] > 0);  if accumulate: x += C_old;  C = x
+struct GemmArgs {
+    int64_t M = 0;
+    int groups = 1, K = 0, N = 0;
+    const void* A = nullptr;
+    int64_t lda = 0;
+    int a_dtype = SLICEGCN_F32;
+    int a_start[SLICEGCN_MAX_SLICES] = {0};
+    const uint8_t* a_mask = nullptr;   // A element (r, col) is multiplied by a_mask[r*a_mask_ld + col]
+    int64_t a_mask_ld = 0;
+    const float* B = nullptr;          // group g: B + g*b_gstride; element (k, n) at k*ldb + n, or n*ldb + k if b_trans
+    int64_t b_gstride = 0;
+    int ldb = 0;
+    int b_trans = 0;
+    void* C = nullptr;
+    int64_t ldc = 0;
+    int c_dtype = SLICEGCN_F32;
+    int c_start[SLICEGCN_MAX_SLICES] = {0};
+    const float* bias = nullptr;       // [groups][N] (stride N), added before the activation
+    const float* post1 = nullptr;      // [groups][N], added after the activation
+    const float* post2 = nullptr;
+    int relu = 0;
+    uint8_t* mask_out = nullptr;       // mask_out[r*mask_ld + c] = pre-activation > 0 (c = column of C)
+    int64_t mask_ld = 0;
+    const void* mul_pos = nullptr;     // tensor P indexed like C (own dtype / leading dimension): x *= (P > 0)
+    int64_t mul_pos_ld = 0;
+    int mul_pos_dtype = SLICEGCN_F32;
+    int accumulate = 0;
+};
+slicegcn_status_t gemm_run(const GemmArgs& a, cudaStream_t st);
+
+// ---- grouped weight gradient  dW_g = A_g^T * B_g  (reduction over all rows) -------------------
+// A_g: K columns of A from a_start[g]; B_g: N columns of the fp32 matrix B from b_start[g], each
+// element optionally multiplied by b_mask (same column indexing as B).  dW [groups][K][N] and,
+// if dbias != NULL, dbias[groups][N] = column sums of (masked) B_g.  K may be 0 (bias only).
+// Two-stage deterministic reduction through `scratch`.
+struct WgradArgs {
+    int64_t M = 0;
+    int groups = 1, K = 0, N = 0;
+    const void* A = nullptr;
+    int64_t lda = 0;
+    int a_dtype = SLICEGCN_F32;
+    int a_start[SLICEGCN_MAX_SLICES] = {0};
+    const float* B = nullptr;
+    int64_t ldb = 0;
+    int b_start[SLICEGCN_MAX_SLICES] = {0};
+    const uint8_t* b_mask = nullptr;
+    int64_t b_mask_ld = 0;
+    float* dW = nullptr;       // may be NULL when K == 0
+    float* dbias = nullptr;    // may be NULL
+    float* dbias2 = nullptr;   // optional second copy of the column sums (slice-encoding gradient)
+};
+int64_t wgrad_scratch_bytes(int64_t M, int groups, int K, int N);
+slicegcn_status_t wgrad_run(const WgradArgs& a, void* scratch, int64_t scratch_bytes, cudaStream_t st);
+
+// ---- small kernels ----------------------------------------------------------------------------
+// out = in * mask (fp32, row-major with leading dimensions)
+slicegcn_status_t mask_mul_run(int64_t M, int N, const float* in, int64_t ld_in, const uint8_t* mask, int64_t ld_mask,
+                               float* out, int64_t ld_out, cudaStream_t st);
+// Softmax cross entropy (Eq. 10) over the training rows: writes dlogits = (softmax - onehot)/n_train
+// (rows outside the training set are zeroed) and the mean loss.  row_loss: scratch [n_train] floats.
+slicegcn_status_t softmax_ce_run(int64_t n, int C, const float* logits, const int32_t* labels, const int32_t* train_idx,
+                                 int64_t n_train, float* dlogits, float* row_loss, float* loss_out, cudaStream_t st);
+// Adam with bias correction; `step` is 1-based.
+slicegcn_status_t adam_run(int64_t count, float* theta, const float* grad, float* m1, float* m2, float lr, float beta1,
+                           float beta2, float eps, float weight_decay, int step, cudaStream_t st);
+
+}  // namespace sgcn

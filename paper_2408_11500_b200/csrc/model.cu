@@ -1,0 +1,904 @@
+// Host orchestration: slice strategy (Algorithm 1), one sliced layer forward / backward (Eq. 6-8),
+// the model's parameter layout and one training epoch (Algorithm 3).  Everything here is launch
+// sequencing on the caller's stream; all arithmetic on tensors happens in the kernels.
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "common.cuh"
+#include "kernels.cuh"
+
+namespace sgcn {
+namespace {
+
+inline int64_t align_up(int64_t v, int64_t a) { return (v + a - 1) / a * a; }
+inline int esize(int dtype) { return dtype == SLICEGCN_BF16 ? 2 : 4; }
+
+// Bump allocator over caller scratch; with base == nullptr it only measures.
+struct Bump {
+    char* base = nullptr;
+    int64_t off = 0;
+    void* take(int64_t bytes) {
+        off = align_up(off, 256);
+        void* p = base ? base + off : nullptr;
+        off += bytes;
+        return p;
+    }
+};
+
+slicegcn_status_t slice_strategy(int in_d, int p, double scale, int rule, int* starts, int* ends, int* slice_size) {
+    if (in_d < 1 || p < 1 || p > SLICEGCN_MAX_SLICES || !starts || !ends || !slice_size)
+        SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "slice_strategy: need in_d >= 1, 1 <= p <= %d, non-NULL outputs",
+                  SLICEGCN_MAX_SLICES);
+    int size;
+    if (rule == SLICEGCN_RULE_CEIL)
+        size = (in_d + p - 1) / p;
+    else if (rule == SLICEGCN_RULE_FLOOR_PLUS_1)
+        size = in_d / p + 1;
+    else
+        SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "slice_strategy: unknown rule %d", rule);
+    const double scaled = (double)size * scale;
+    if (!(scaled >= 1.0) || scaled > (double)in_d + 0.5) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "slice_strategy: scaled width outside [1, in_d]");
+    const int width = (int)scaled;   // truncation toward zero, as int() in the algorithm
+    if (width < 1 || width > in_d) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "slice_strategy: scaled width outside [1, in_d]");
+    for (int i = 0; i < p; ++i) {
+        int s = i * size, e = s + width;
+        if (e > in_d) {   // the last slice(s) are shifted left to end at in_d
+            s -= e - in_d;
+            e = in_d;
+        }
+        if (s < 0) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "slice_strategy: slice %d does not fit", i);
+        starts[i] = s;
+        ends[i] = e;
+    }
+    *slice_size = size;
+    return SLICEGCN_OK;
+}
+
+// ------------------------------------------------------------------------------------------ layer
+struct LayerPlan {
+    int p = 0, in_width = 0, in_cols = 0, h_s = 0, out_cols = 0;
+    int64_t in_ld = 0, out_ld = 0;
+    int dtype = 0, order = 0, esz = 4;
+    int in_starts[SLICEGCN_MAX_SLICES];
+    bool disjoint_cover = false;   // slices tile [0, in_cols) without overlap or gap
+    int zt_cols = 0;               // columns of the saved intermediate (Z: in_cols, T: out_cols)
+    int64_t zt_ld = 0, mask_ld = 0, zt_bytes = 0, mask_bytes = 0;
+    int64_t n = 0;
+};
+
+slicegcn_status_t make_plan(const slicegcn_graph* g, const slicegcn_layer_desc* d, LayerPlan* pl) {
+    if (!g || !d) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "layer: NULL graph or description");
+    if (d->num_slices < 1 || d->num_slices > SLICEGCN_MAX_SLICES || !d->in_starts || d->in_width < 1 || d->h_s < 1)
+        SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "layer: bad slice description");
+    if (d->dtype != SLICEGCN_F32 && d->dtype != SLICEGCN_BF16) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "layer: bad dtype");
+    if (!d->W_agg) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "layer: W_agg is NULL");
+    LayerPlan& L = *pl;
+    L.n = g->n;
+    L.p = d->num_slices;
+    L.in_width = d->in_width;
+    L.in_cols = d->in_cols;
+    L.h_s = d->h_s;
+    L.out_cols = L.p * L.h_s;
+    L.in_ld = d->in_ld;
+    L.out_ld = d->out_ld;
+    L.dtype = d->dtype;
+    L.esz = esize(d->dtype);
+    if (L.in_ld < L.in_cols || L.out_ld < L.out_cols) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "layer: leading dimension too small");
+    std::vector<int> cover(L.in_cols > 0 ? L.in_cols : 0, 0);
+    bool disjoint = true;
+    for (int i = 0; i < L.p; ++i) {
+        const int s = d->in_starts[i];
+        if (s < 0 || s + L.in_width > L.in_cols) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "layer: slice %d outside [0, in_cols)", i);
+        L.in_starts[i] = s;
+        for (int c = s; c < s + L.in_width; ++c)
+            if (cover[c]++) disjoint = false;
+    }
+    for (int c = 0; c < L.in_cols; ++c)
+        if (!cover[c]) disjoint = false;
+    L.disjoint_cover = disjoint;
+    L.order = d->order;
+    if (L.order == SLICEGCN_ORDER_AUTO) L.order = (L.in_cols <= L.out_cols) ? SLICEGCN_AGG_FIRST : SLICEGCN_XFORM_FIRST;
+    if (L.order != SLICEGCN_AGG_FIRST && L.order != SLICEGCN_XFORM_FIRST) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "layer: bad order");
+    L.zt_cols = L.order == SLICEGCN_AGG_FIRST ? L.in_cols : L.out_cols;
+    L.zt_ld = align_up(L.zt_cols, 8);
+    L.mask_ld = align_up(L.out_cols, 16);
+    L.zt_bytes = align_up(L.n * L.zt_ld * L.esz, 256);
+    L.mask_bytes = align_up(L.n * L.mask_ld, 256);
+    return SLICEGCN_OK;
+}
+
+int64_t layer_fwd_ws_bytes(const slicegcn_graph* g, const LayerPlan& L) {
+    Bump b;
+    b.take(spmm_partial_bytes(g, L.zt_cols));
+    return align_up(b.off, 256);
+}
+
+int64_t layer_wgrad_scratch(const LayerPlan& L) {
+    int64_t a = wgrad_scratch_bytes(L.n, L.p, L.in_width, L.h_s);
+    int64_t b = wgrad_scratch_bytes(L.n, L.p, 0, L.h_s);
+    return a > b ? a : b;
+}
+
+int64_t layer_bwd_ws_bytes(const slicegcn_graph* g, const LayerPlan& L) {
+    Bump b;
+    b.take(layer_wgrad_scratch(L));
+    b.take(spmm_partial_bytes(g, L.zt_cols));
+    if (L.order == SLICEGCN_AGG_FIRST) {
+        b.take(L.n * L.zt_ld * 4);
+    } else {
+        b.take(L.n * L.zt_ld * 4);
+        b.take(L.n * L.zt_ld * 4);
+    }
+    return align_up(b.off, 256);
+}
+
+// Runs a grouped GEMM either as one launch (groups in grid.z) or, when the groups' output
+// columns overlap, one group after the other.
+slicegcn_status_t gemm_groups(const GemmArgs& a, bool sequential, cudaStream_t st) {
+    if (!sequential || a.groups == 1) return gemm_run(a, st);
+    for (int g = 0; g < a.groups; ++g) {
+        GemmArgs s = a;
+        s.groups = 1;
+        s.a_start[0] = a.a_start[g];
+        s.c_start[0] = a.c_start[g];
+        s.B = a.B + (int64_t)g * a.b_gstride;
+        if (a.bias) s.bias = a.bias + g * a.N;
+        if (a.post1) s.post1 = a.post1 + g * a.N;
+        if (a.post2) s.post2 = a.post2 + g * a.N;
+        SGCN_TRY(gemm_run(s, st));
+    }
+    return SLICEGCN_OK;
+}
+
+slicegcn_status_t layer_forward_impl(const slicegcn_graph* g, const slicegcn_layer_desc* d, const LayerPlan& L,
+                                     const void* H_in, void* H_out, void* saved, void* ws, int64_t ws_bytes,
+                                     cudaStream_t st) {
+    char* zt = static_cast<char*>(saved);
+    uint8_t* mask = reinterpret_cast<uint8_t*>(zt + L.zt_bytes);
+    const int64_t part_bytes = spmm_partial_bytes(g, L.zt_cols);
+    if (ws_bytes < part_bytes) SGCN_FAIL(SLICEGCN_ERR_ALLOC, "layer_forward: workspace too small");
+    const bool has_post = d->W_self || d->b_self || d->E;
+
+    GemmArgs self;   // H_out = H_in W_self + b_self + E
+    self.M = L.n;
+    self.groups = L.p;
+    self.K = d->W_self ? L.in_width : 0;
+    self.N = L.h_s;
+    self.A = H_in;
+    self.lda = L.in_ld;
+    self.a_dtype = L.dtype;
+    self.B = d->W_self;
+    self.b_gstride = (int64_t)L.in_width * L.h_s;
+    self.ldb = L.h_s;
+    self.C = H_out;
+    self.ldc = L.out_ld;
+    self.c_dtype = L.dtype;
+    self.post1 = d->b_self;
+    self.post2 = d->E;
+    for (int i = 0; i < L.p; ++i) {
+        self.a_start[i] = L.in_starts[i];
+        self.c_start[i] = i * L.h_s;
+    }
+
+    if (L.order == SLICEGCN_AGG_FIRST) {
+        // Z = A_hat H_in over every input column once; slices then read their column ranges of Z
+        SGCN_TRY(spmm_run(g, false, L.dtype, L.dtype, H_in, L.in_ld, zt, L.zt_ld, L.in_cols, nullptr, ws, ws_bytes, st));
+        if (d->W_self) SGCN_TRY(gemm_run(self, st));
+        GemmArgs agg = self;   // H_out = ReLU(Z W_agg + b) (+ H_out | + b_self + E)
+        agg.K = L.in_width;
+        agg.A = zt;
+        agg.lda = L.zt_ld;
+        agg.B = d->W_agg;
+        agg.bias = d->b;
+        agg.relu = 1;
+        agg.mask_out = mask;
+        agg.mask_ld = L.mask_ld;
+        if (d->W_self) {
+            agg.post1 = agg.post2 = nullptr;
+            agg.accumulate = 1;
+        }
+        SGCN_TRY(gemm_run(agg, st));
+    } else {
+        GemmArgs tr = self;    // T = H_in W_agg
+        tr.K = L.in_width;
+        tr.B = d->W_agg;
+        tr.C = zt;
+        tr.ldc = L.zt_ld;
+        tr.post1 = tr.post2 = nullptr;
+        SGCN_TRY(gemm_run(tr, st));
+        if (has_post) SGCN_TRY(gemm_run(self, st));
+        SpmmEpilogue epi;      // H_out = ReLU(A_hat T + b) (+ H_out)
+        epi.bias = d->b;
+        epi.relu = 1;
+        epi.mask = mask;
+        epi.mask_ld = L.mask_ld;
+        epi.accumulate = has_post ? 1 : 0;
+        SGCN_TRY(spmm_run(g, false, L.dtype, L.dtype, zt, L.zt_ld, H_out, L.out_ld, L.out_cols, &epi, ws, ws_bytes, st));
+    }
+    return SLICEGCN_OK;
+}
+
+slicegcn_status_t layer_backward_impl(const slicegcn_graph* g, const slicegcn_layer_desc* d, const LayerPlan& L,
+                                      const void* H_in, const void* saved, const float* dH_out, int64_t dout_ld,
+                                      float* dH_in, int64_t din_ld, float* dW_agg, float* dW_self, float* db,
+                                      float* db_self, float* dE, void* ws, int64_t ws_bytes, cudaStream_t st) {
+    if (ws_bytes < layer_bwd_ws_bytes(g, L)) SGCN_FAIL(SLICEGCN_ERR_ALLOC, "layer_backward: workspace too small");
+    const char* zt = static_cast<const char*>(saved);
+    const uint8_t* mask = reinterpret_cast<const uint8_t*>(zt + L.zt_bytes);
+    Bump b;
+    b.base = static_cast<char*>(ws);
+    const int64_t wg_bytes = layer_wgrad_scratch(L);
+    void* wg = b.take(wg_bytes);
+    const int64_t part_bytes = spmm_partial_bytes(g, L.zt_cols);
+    void* part = b.take(part_bytes);
+    const bool seq = !L.disjoint_cover;
+
+    // self branch: dW_self = H_in^T dH, db_self = dE = colsum(dH)
+    if ((d->W_self && dW_self) || db_self || dE) {
+        WgradArgs w;
+        w.M = L.n;
+        w.groups = L.p;
+        w.K = (d->W_self && dW_self) ? L.in_width : 0;
+        w.N = L.h_s;
+        w.A = H_in;
+        w.lda = L.in_ld;
+        w.a_dtype = L.dtype;
+        w.B = dH_out;
+        w.ldb = dout_ld;
+        w.dW = dW_self;
+        w.dbias = db_self;
+        w.dbias2 = dE;
+        for (int i = 0; i < L.p; ++i) {
+            w.a_start[i] = L.in_starts[i];
+            w.b_start[i] = i * L.h_s;
+        }
+        SGCN_TRY(wgrad_run(w, wg, wg_bytes, st));
+    }
+
+    GemmArgs dself;   // dH_in (+)= dH W_self^T
+    dself.M = L.n;
+    dself.groups = L.p;
+    dself.K = L.h_s;
+    dself.N = L.in_width;
+    dself.A = dH_out;
+    dself.lda = dout_ld;
+    dself.a_dtype = SLICEGCN_F32;
+    dself.B = d->W_self;
+    dself.b_gstride = (int64_t)L.in_width * L.h_s;
+    dself.ldb = L.h_s;
+    dself.b_trans = 1;
+    dself.C = dH_in;
+    dself.ldc = din_ld;
+    dself.c_dtype = SLICEGCN_F32;
+    for (int i = 0; i < L.p; ++i) {
+        dself.a_start[i] = i * L.h_s;
+        dself.c_start[i] = L.in_starts[i];
+    }
+
+    if (L.order == SLICEGCN_AGG_FIRST) {
+        if (dW_agg || db) {   // dW_agg = Z^T (dH * mask), db = colsum(dH * mask)
+            WgradArgs w;
+            w.M = L.n;
+            w.groups = L.p;
+            w.K = dW_agg ? L.in_width : 0;
+            w.N = L.h_s;
+            w.A = zt;
+            w.lda = L.zt_ld;
+            w.a_dtype = L.dtype;
+            w.B = dH_out;
+            w.ldb = dout_ld;
+            w.b_mask = mask;
+            w.b_mask_ld = L.mask_ld;
+            w.dW = dW_agg;
+            w.dbias = db;
+            for (int i = 0; i < L.p; ++i) {
+                w.a_start[i] = L.in_starts[i];
+                w.b_start[i] = i * L.h_s;
+            }
+            SGCN_TRY(wgrad_run(w, wg, wg_bytes, st));
+        }
+        if (dH_in) {
+            float* dZ = static_cast<float*>(b.take(L.n * L.zt_ld * 4));
+            GemmArgs dz = dself;   // dZ = (dH * mask) W_agg^T
+            dz.a_mask = mask;
+            dz.a_mask_ld = L.mask_ld;
+            dz.B = d->W_agg;
+            dz.C = dZ;
+            dz.ldc = L.zt_ld;
+            if (seq) {
+                SGCN_CUDA(cudaMemsetAsync(dZ, 0, L.n * L.zt_ld * 4, st));
+                dz.accumulate = 1;
+            }
+            SGCN_TRY(gemm_groups(dz, seq, st));
+            SGCN_TRY(spmm_run(g, true, SLICEGCN_F32, SLICEGCN_F32, dZ, L.zt_ld, dH_in, din_ld, L.in_cols, nullptr, part,
+                              part_bytes, st));
+            if (d->W_self) {
+                dself.accumulate = 1;
+                SGCN_TRY(gemm_groups(dself, seq, st));
+            }
+        }
+    } else {
+        float* dM = static_cast<float*>(b.take(L.n * L.zt_ld * 4));
+        float* dT = static_cast<float*>(b.take(L.n * L.zt_ld * 4));
+        SGCN_TRY(mask_mul_run(L.n, L.out_cols, dH_out, dout_ld, mask, L.mask_ld, dM, L.zt_ld, st));
+        if (db) {
+            WgradArgs w;
+            w.M = L.n;
+            w.groups = L.p;
+            w.K = 0;
+            w.N = L.h_s;
+            w.B = dM;
+            w.ldb = L.zt_ld;
+            w.dbias = db;
+            for (int i = 0; i < L.p; ++i) w.b_start[i] = i * L.h_s;
+            SGCN_TRY(wgrad_run(w, wg, wg_bytes, st));
+        }
+        if (dW_agg || dH_in) {   // dT = A_hat^T dM
+            SGCN_TRY(spmm_run(g, true, SLICEGCN_F32, SLICEGCN_F32, dM, L.zt_ld, dT, L.zt_ld, L.out_cols, nullptr, part,
+                              part_bytes, st));
+        }
+        if (dW_agg) {
+            WgradArgs w;
+            w.M = L.n;
+            w.groups = L.p;
+            w.K = L.in_width;
+            w.N = L.h_s;
+            w.A = H_in;
+            w.lda = L.in_ld;
+            w.a_dtype = L.dtype;
+            w.B = dT;
+            w.ldb = L.zt_ld;
+            w.dW = dW_agg;
+            for (int i = 0; i < L.p; ++i) {
+                w.a_start[i] = L.in_starts[i];
+                w.b_start[i] = i * L.h_s;
+            }
+            SGCN_TRY(wgrad_run(w, wg, wg_bytes, st));
+        }
+        if (dH_in) {
+            GemmArgs dt = dself;   // dH_in = dT W_agg^T
+            dt.A = dT;
+            dt.lda = L.zt_ld;
+            dt.B = d->W_agg;
+            if (seq) {
+                SGCN_CUDA(cudaMemset2DAsync(dH_in, din_ld * 4, 0, (size_t)L.in_cols * 4, L.n, st));
+                dt.accumulate = 1;
+            }
+            SGCN_TRY(gemm_groups(dt, seq, st));
+            if (d->W_self) {
+                dself.accumulate = 1;
+                SGCN_TRY(gemm_groups(dself, seq, st));
+            }
+        }
+    }
+    return SLICEGCN_OK;
+}
+
+}  // namespace
+}  // namespace sgcn
+
+// ------------------------------------------------------------------------------------------ model
+struct slicegcn_model {
+    slicegcn_model_desc desc;
+    int starts[SLICEGCN_MAX_SLICES], ends[SLICEGCN_MAX_SLICES];
+    int slice_size = 0, slice_width = 0, h_s = 0;
+    struct Tensor {
+        std::string name;
+        int64_t offset;
+        int dims[3];
+    };
+    std::vector<Tensor> tensors;
+    int64_t param_count = 0, param_elems = 0;
+    // offsets into the flat parameter buffer (-1: absent)
+    int64_t ff_W1 = -1, ff_b1 = -1, ff_W2 = -1, ff_b2 = -1, E = -1, Wc1 = -1, bc1 = -1, Wc2 = -1, bc2 = -1;
+    std::vector<int64_t> W_agg, W_self, b, b_self;
+    std::vector<int> order;   // resolved per layer
+
+    int64_t add(const std::string& name, int d0, int d1, int d2) {
+        const int64_t off = param_elems;
+        tensors.push_back({name, off, {d0, d1, d2}});
+        const int64_t cnt = (int64_t)d0 * d1 * d2;
+        param_count += cnt;
+        param_elems = sgcn::align_up(off + cnt, 4);
+        return off;
+    }
+    int layer_in_width(int l) const { return l == 0 ? (desc.use_ff ? slice_size : slice_width) : h_s; }
+    int layer_in_cols(int l) const { return l == 0 ? (desc.use_ff ? slice_size : desc.in_d) : desc.num_slices * h_s; }
+    void layer_in_starts(int l, int* out) const {
+        for (int i = 0; i < desc.num_slices; ++i) out[i] = l == 0 ? (desc.use_ff ? 0 : starts[i]) : i * h_s;
+    }
+};
+
+namespace sgcn {
+namespace {
+
+struct EpochLayout {
+    // element leading dimensions
+    int64_t ld_h = 0, ld_x0 = 0, ld_ffact = 0, ld_cls = 0, ld_grad = 0;
+    int64_t total = 0;
+    // pointers (valid when built with a base)
+    void* ff_act = nullptr;
+    void* xff = nullptr;
+    std::vector<void*> H;        // H[l+1], l = 0..L-1
+    std::vector<void*> saved;
+    std::vector<int64_t> saved_bytes;
+    void* cls_act = nullptr;
+    float* logits = nullptr;
+    float* dlogits = nullptr;
+    float* row_loss = nullptr;
+    float* dA = nullptr;
+    float* dH[2] = {nullptr, nullptr};
+    float* dff = nullptr;
+    void* ws = nullptr;
+    int64_t ws_bytes = 0;
+};
+
+slicegcn_status_t layer_desc_for(const slicegcn_model* m, int l, const float* params, int64_t x_ld, int* starts_buf,
+                                 slicegcn_layer_desc* d) {
+    const slicegcn_model_desc& D = m->desc;
+    m->layer_in_starts(l, starts_buf);
+    d->num_slices = D.num_slices;
+    d->in_starts = starts_buf;
+    d->in_width = m->layer_in_width(l);
+    d->in_cols = m->layer_in_cols(l);
+    d->in_ld = l == 0 ? (D.use_ff ? align_up(m->slice_size, 8) : x_ld) : align_up((int64_t)D.num_slices * m->h_s, 8);
+    d->h_s = m->h_s;
+    d->out_ld = align_up((int64_t)D.num_slices * m->h_s, 8);
+    d->dtype = D.dtype;
+    d->order = m->order[l];
+    d->W_agg = params ? params + m->W_agg[l] : reinterpret_cast<const float*>(16);
+    d->W_self = D.use_self ? (params ? params + m->W_self[l] : reinterpret_cast<const float*>(16)) : nullptr;
+    d->b = params ? params + m->b[l] : nullptr;
+    d->b_self = D.use_b_self ? (params ? params + m->b_self[l] : reinterpret_cast<const float*>(16)) : nullptr;
+    d->E = (D.use_se && l == D.num_layers - 1) ? (params ? params + m->E : reinterpret_cast<const float*>(16)) : nullptr;
+    return SLICEGCN_OK;
+}
+
+slicegcn_status_t build_layout(const slicegcn_model* m, const slicegcn_graph* g, int64_t x_ld, char* base,
+                               EpochLayout* out) {
+    const slicegcn_model_desc& D = m->desc;
+    const int64_t n = g->n;
+    const int esz = esize(D.dtype);
+    const int p = D.num_slices, L = D.num_layers;
+    EpochLayout& E = *out;
+    Bump b;
+    b.base = base;
+    E.ld_h = align_up((int64_t)p * m->h_s, 8);
+    E.ld_cls = align_up(D.hidden, 8);
+    E.ld_ffact = align_up(D.in_d, 8);
+    E.ld_x0 = align_up(m->slice_size, 8);
+    int64_t gw = E.ld_h;
+    if (D.use_ff) gw = std::max(gw, std::max(E.ld_x0, E.ld_ffact));
+    E.ld_grad = gw;
+    if (D.use_ff) {
+        E.ff_act = b.take(n * E.ld_ffact * esz);
+        E.xff = b.take(n * E.ld_x0 * esz);
+    }
+    int64_t ws_need = 0;
+    E.H.resize(L);
+    E.saved.resize(L);
+    E.saved_bytes.resize(L);
+    for (int l = 0; l < L; ++l) {
+        int starts[SLICEGCN_MAX_SLICES];
+        slicegcn_layer_desc d;
+        layer_desc_for(m, l, nullptr, x_ld, starts, &d);
+        LayerPlan pl;
+        SGCN_TRY(make_plan(g, &d, &pl));
+        E.H[l] = b.take(n * E.ld_h * esz);
+        E.saved_bytes[l] = pl.zt_bytes + pl.mask_bytes;
+        E.saved[l] = b.take(E.saved_bytes[l]);
+        ws_need = std::max(ws_need, std::max(layer_fwd_ws_bytes(g, pl), layer_bwd_ws_bytes(g, pl)));
+    }
+    E.cls_act = b.take(n * E.ld_cls * esz);
+    E.logits = static_cast<float*>(b.take(n * (int64_t)D.num_classes * 4));
+    E.dlogits = static_cast<float*>(b.take(n * (int64_t)D.num_classes * 4));
+    E.row_loss = static_cast<float*>(b.take(n * 4));
+    E.dA = static_cast<float*>(b.take(n * E.ld_cls * 4));
+    E.dH[0] = static_cast<float*>(b.take(n * E.ld_grad * 4));
+    E.dH[1] = static_cast<float*>(b.take(n * E.ld_grad * 4));
+    // scratch of the dense heads (weight gradients)
+    ws_need = std::max(ws_need, wgrad_scratch_bytes(n, 1, D.hidden, D.num_classes));
+    ws_need = std::max(ws_need, wgrad_scratch_bytes(n, 1, p * m->h_s, D.hidden));
+    if (D.use_ff) {
+        ws_need = std::max(ws_need, wgrad_scratch_bytes(n, 1, D.in_d, m->slice_size));
+        ws_need = std::max(ws_need, wgrad_scratch_bytes(n, 1, D.in_d, D.in_d));
+    }
+    E.ws_bytes = align_up(ws_need, 256);
+    E.ws = b.take(E.ws_bytes);
+    E.total = align_up(b.off, 256);
+    return SLICEGCN_OK;
+}
+
+}  // namespace
+}  // namespace sgcn
+
+using namespace sgcn;
+
+extern "C" {
+
+slicegcn_status_t slicegcn_slice_strategy(int32_t in_d, int32_t p, double scale, int32_t rule, int32_t* starts,
+                                          int32_t* ends, int32_t* slice_size) {
+    return sgcn::slice_strategy(in_d, p, scale, rule, starts, ends, slice_size);
+}
+
+slicegcn_status_t slicegcn_layer_saved_bytes(const slicegcn_graph* g, const slicegcn_layer_desc* d, int64_t* bytes) {
+    if (!bytes) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "bytes is NULL");
+    LayerPlan pl;
+    SGCN_TRY(make_plan(g, d, &pl));
+    *bytes = pl.zt_bytes + pl.mask_bytes;
+    return SLICEGCN_OK;
+}
+
+slicegcn_status_t slicegcn_layer_workspace_bytes(const slicegcn_graph* g, const slicegcn_layer_desc* d, int64_t* bytes) {
+    if (!bytes) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "bytes is NULL");
+    LayerPlan pl;
+    SGCN_TRY(make_plan(g, d, &pl));
+    *bytes = std::max(layer_fwd_ws_bytes(g, pl), layer_bwd_ws_bytes(g, pl));
+    return SLICEGCN_OK;
+}
+
+slicegcn_status_t slicegcn_layer_forward(const slicegcn_graph* g, const slicegcn_layer_desc* d, const void* H_in,
+                                         void* H_out, void* saved, int64_t saved_bytes, void* workspace,
+                                         int64_t workspace_bytes, void* stream) {
+    LayerPlan pl;
+    SGCN_TRY(make_plan(g, d, &pl));
+    if (!H_in || !H_out || !saved) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "layer_forward: NULL tensor");
+    if (saved_bytes < pl.zt_bytes + pl.mask_bytes) SGCN_FAIL(SLICEGCN_ERR_ALLOC, "layer_forward: saved buffer too small");
+    if (workspace_bytes < layer_fwd_ws_bytes(g, pl) || (!workspace && layer_fwd_ws_bytes(g, pl) > 0))
+        SGCN_FAIL(SLICEGCN_ERR_ALLOC, "layer_forward: workspace too small");
+    return layer_forward_impl(g, d, pl, H_in, H_out, saved, workspace, workspace_bytes, (cudaStream_t)stream);
+}
+
+slicegcn_status_t slicegcn_layer_backward(const slicegcn_graph* g, const slicegcn_layer_desc* d, const void* H_in,
+                                          const void* saved, const float* dH_out, int64_t dout_ld, float* dH_in,
+                                          int64_t din_ld, float* dW_agg, float* dW_self, float* db, float* db_self,
+                                          float* dE, void* workspace, int64_t workspace_bytes, void* stream) {
+    LayerPlan pl;
+    SGCN_TRY(make_plan(g, d, &pl));
+    if (!H_in || !saved || !dH_out || !workspace) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "layer_backward: NULL tensor");
+    if (dout_ld < pl.out_cols || (dH_in && din_ld < pl.in_cols)) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "layer_backward: leading dimension too small");
+    return layer_backward_impl(g, d, pl, H_in, saved, dH_out, dout_ld, dH_in, din_ld, dW_agg, dW_self, db, db_self, dE,
+                               workspace, workspace_bytes, (cudaStream_t)stream);
+}
+
+slicegcn_status_t slicegcn_model_create(const slicegcn_model_desc* desc, slicegcn_model** out) {
+    if (!out) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "out is NULL");
+    *out = nullptr;
+    if (!desc) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "desc is NULL");
+    const slicegcn_model_desc& D = *desc;
+    if (D.in_d < 1 || D.hidden < 1 || D.num_layers < 1 || D.num_classes < 1 || D.num_slices < 1 ||
+        D.num_slices > SLICEGCN_MAX_SLICES)
+        SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "model: sizes must be positive and num_slices <= %d", SLICEGCN_MAX_SLICES);
+    if (D.dtype != SLICEGCN_F32 && D.dtype != SLICEGCN_BF16) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "model: bad dtype");
+    if (D.order != SLICEGCN_ORDER_AUTO && D.order != SLICEGCN_AGG_FIRST && D.order != SLICEGCN_XFORM_FIRST)
+        SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "model: bad order");
+    slicegcn_model* m = new (std::nothrow) slicegcn_model();
+    if (!m) SGCN_FAIL(SLICEGCN_ERR_ALLOC, "host allocation failed");
+    m->desc = D;
+    slicegcn_status_t s = sgcn::slice_strategy(D.in_d, D.num_slices, D.slice_size_scale, D.slice_rule, m->starts, m->ends,
+                                               &m->slice_size);
+    if (s != SLICEGCN_OK) {
+        delete m;
+        return s;
+    }
+    m->slice_width = m->ends[0] - m->starts[0];
+    m->h_s = (D.hidden + D.num_slices - 1) / D.num_slices;   // each layer scaled down in proportion to p
+    const int p = D.num_slices;
+    if (D.use_ff) {
+        m->ff_W1 = m->add("ff_W1", D.in_d, D.in_d, 1);
+        m->ff_b1 = m->add("ff_b1", D.in_d, 1, 1);
+        m->ff_W2 = m->add("ff_W2", D.in_d, m->slice_size, 1);
+        m->ff_b2 = m->add("ff_b2", m->slice_size, 1, 1);
+    }
+    for (int l = 0; l < D.num_layers; ++l) {
+        const int w_in = m->layer_in_width(l);
+        const std::string sfx = "." + std::to_string(l);
+        m->W_agg.push_back(m->add("W_agg" + sfx, p, w_in, m->h_s));
+        m->W_self.push_back(D.use_self ? m->add("W_self" + sfx, p, w_in, m->h_s) : -1);
+        m->b.push_back(m->add("b" + sfx, p, m->h_s, 1));
+        m->b_self.push_back(D.use_b_self ? m->add("b_self" + sfx, p, m->h_s, 1) : -1);
+        int order = D.order;
+        if (order == SLICEGCN_ORDER_AUTO)
+            order = m->layer_in_cols(l) <= p * m->h_s ? SLICEGCN_AGG_FIRST : SLICEGCN_XFORM_FIRST;
+        m->order.push_back(order);
+    }
+    if (D.use_se) m->E = m->add("E", p, m->h_s, 1);
+    m->Wc1 = m->add("Wc1", p * m->h_s, D.hidden, 1);
+    m->bc1 = m->add("bc1", D.hidden, 1, 1);
+    m->Wc2 = m->add("Wc2", D.hidden, D.num_classes, 1);
+    m->bc2 = m->add("bc2", D.num_classes, 1, 1);
+    *out = m;
+    return SLICEGCN_OK;
+}
+
+slicegcn_status_t slicegcn_model_destroy(slicegcn_model* m) {
+    delete m;
+    return SLICEGCN_OK;
+}
+
+slicegcn_status_t slicegcn_model_param_count(const slicegcn_model* m, int64_t* count) {
+    if (!m || !count) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "NULL argument");
+    *count = m->param_count;
+    return SLICEGCN_OK;
+}
+
+slicegcn_status_t slicegcn_model_param_elems(const slicegcn_model* m, int64_t* elems) {
+    if (!m || !elems) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "NULL argument");
+    *elems = m->param_elems;
+    return SLICEGCN_OK;
+}
+
+slicegcn_status_t slicegcn_model_num_tensors(const slicegcn_model* m, int32_t* count) {
+    if (!m || !count) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "NULL argument");
+    *count = (int32_t)m->tensors.size();
+    return SLICEGCN_OK;
+}
+
+slicegcn_status_t slicegcn_model_tensor_info(const slicegcn_model* m, int32_t t, char name[32], int64_t* offset,
+                                             int32_t dims[3]) {
+    if (!m || t < 0 || t >= (int32_t)m->tensors.size()) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "bad tensor index");
+    const auto& T = m->tensors[t];
+    if (name) {
+        std::strncpy(name, T.name.c_str(), 31);
+        name[31] = 0;
+    }
+    if (offset) *offset = T.offset;
+    if (dims)
+        for (int i = 0; i < 3; ++i) dims[i] = T.dims[i];
+    return SLICEGCN_OK;
+}
+
+slicegcn_status_t slicegcn_model_slices(const slicegcn_model* m, int32_t* starts, int32_t* ends, int32_t* slice_size,
+                                        int32_t* h_s) {
+    if (!m) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "model is NULL");
+    for (int i = 0; i < m->desc.num_slices; ++i) {
+        if (starts) starts[i] = m->starts[i];
+        if (ends) ends[i] = m->ends[i];
+    }
+    if (slice_size) *slice_size = m->slice_size;
+    if (h_s) *h_s = m->h_s;
+    return SLICEGCN_OK;
+}
+
+slicegcn_status_t slicegcn_model_layer_order(const slicegcn_model* m, int32_t layer, int32_t* order) {
+    if (!m || !order || layer < 0 || layer >= m->desc.num_layers) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "bad argument");
+    *order = m->order[layer];
+    return SLICEGCN_OK;
+}
+
+slicegcn_status_t slicegcn_train_workspace_bytes(const slicegcn_model* m, const slicegcn_graph* g, int64_t* bytes) {
+    if (!m || !g || !bytes) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "NULL argument");
+    EpochLayout E;
+    SGCN_TRY(build_layout(m, g, m->desc.in_d, nullptr, &E));
+    *bytes = E.total;
+    return SLICEGCN_OK;
+}
+
+slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_graph* g, const void* X, int64_t x_ld,
+                                       const int32_t* labels, const int32_t* train_idx, int64_t n_train, float* params,
+                                       float* grads, float* adam_m, float* adam_v, const slicegcn_opt_desc* opt,
+                                       float* logits_out, float* loss_out, void* workspace, int64_t workspace_bytes,
+                                       void* stream) {
+    if (!m || !g || !X || !labels || !params || !grads || !workspace)
+        SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "train_epoch: NULL argument");
+    const slicegcn_model_desc& D = m->desc;
+    if (x_ld < D.in_d) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "train_epoch: x_ld < in_d");
+    if (opt && (!adam_m || !adam_v)) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "train_epoch: optimiser state is NULL");
+    if (opt && (opt->total_epochs < 1 || opt->epoch < 0)) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "train_epoch: bad epoch");
+    if (train_idx && n_train < 1) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "train_epoch: empty training set");
+    cudaStream_t st = (cudaStream_t)stream;
+    const int64_t n = g->n;
+    const int p = D.num_slices, L = D.num_layers, C = D.num_classes;
+    EpochLayout E;
+    SGCN_TRY(build_layout(m, g, x_ld, static_cast<char*>(workspace), &E));
+    if (workspace_bytes < E.total)
+        SGCN_FAIL(SLICEGCN_ERR_ALLOC, "train_epoch: workspace too small (%lld < %lld)", (long long)workspace_bytes,
+                  (long long)E.total);
+    SGCN_CUDA(cudaMemsetAsync(grads, 0, sizeof(float) * m->param_elems, st));
+
+    // ---------------- forward
+    const void* h0 = X;
+    int64_t ld0 = x_ld;
+    if (D.use_ff) {   // X_ff = ReLU(X W1 + b1) W2 + b2  (Eq. 4 / Algorithm 3)
+        GemmArgs a;
+        a.M = n;
+        a.K = D.in_d;
+        a.N = D.in_d;
+        a.A = X;
+        a.lda = x_ld;
+        a.a_dtype = D.dtype;
+        a.B = params + m->ff_W1;
+        a.ldb = D.in_d;
+        a.bias = params + m->ff_b1;
+        a.relu = 1;
+        a.C = E.ff_act;
+        a.ldc = E.ld_ffact;
+        a.c_dtype = D.dtype;
+        SGCN_TRY(gemm_run(a, st));
+        GemmArgs c;
+        c.M = n;
+        c.K = D.in_d;
+        c.N = m->slice_size;
+        c.A = E.ff_act;
+        c.lda = E.ld_ffact;
+        c.a_dtype = D.dtype;
+        c.B = params + m->ff_W2;
+        c.ldb = m->slice_size;
+        c.bias = params + m->ff_b2;
+        c.C = E.xff;
+        c.ldc = E.ld_x0;
+        c.c_dtype = D.dtype;
+        SGCN_TRY(gemm_run(c, st));
+        h0 = E.xff;
+        ld0 = E.ld_x0;
+    }
+    std::vector<slicegcn_layer_desc> descs(L);
+    std::vector<LayerPlan> plans(L);
+    std::vector<std::vector<int>> starts(L, std::vector<int>(SLICEGCN_MAX_SLICES));
+    const void* hin = h0;
+    for (int l = 0; l < L; ++l) {
+        layer_desc_for(m, l, params, x_ld, starts[l].data(), &descs[l]);
+        if (l == 0) descs[l].in_ld = ld0;
+        SGCN_TRY(make_plan(g, &descs[l], &plans[l]));
+        SGCN_TRY(layer_forward_impl(g, &descs[l], plans[l], hin, E.H[l], E.saved[l], E.ws, E.ws_bytes, st));
+        hin = E.H[l];
+    }
+    const int HW = p * m->h_s;
+    float* logits = logits_out ? logits_out : E.logits;
+    {   // classifier (Eq. 9)
+        GemmArgs a;
+        a.M = n;
+        a.K = HW;
+        a.N = D.hidden;
+        a.A = hin;
+        a.lda = E.ld_h;
+        a.a_dtype = D.dtype;
+        a.B = params + m->Wc1;
+        a.ldb = D.hidden;
+        a.bias = params + m->bc1;
+        a.relu = 1;
+        a.C = E.cls_act;
+        a.ldc = E.ld_cls;
+        a.c_dtype = D.dtype;
+        SGCN_TRY(gemm_run(a, st));
+        GemmArgs c;
+        c.M = n;
+        c.K = D.hidden;
+        c.N = C;
+        c.A = E.cls_act;
+        c.lda = E.ld_cls;
+        c.a_dtype = D.dtype;
+        c.B = params + m->Wc2;
+        c.ldb = C;
+        c.bias = params + m->bc2;
+        c.C = logits;
+        c.ldc = C;
+        c.c_dtype = SLICEGCN_F32;
+        SGCN_TRY(gemm_run(c, st));
+    }
+    // ---------------- loss (Eq. 10) and its gradient
+    SGCN_TRY(softmax_ce_run(n, C, logits, labels, train_idx, n_train, E.dlogits, E.row_loss, loss_out, st));
+
+    // ---------------- backward
+    {
+        WgradArgs w;
+        w.M = n;
+        w.K = D.hidden;
+        w.N = C;
+        w.A = E.cls_act;
+        w.lda = E.ld_cls;
+        w.a_dtype = D.dtype;
+        w.B = E.dlogits;
+        w.ldb = C;
+        w.dW = grads + m->Wc2;
+        w.dbias = grads + m->bc2;
+        SGCN_TRY(wgrad_run(w, E.ws, E.ws_bytes, st));
+        GemmArgs a;   // dA = (dlogits Wc2^T) * (cls_act > 0)
+        a.M = n;
+        a.K = C;
+        a.N = D.hidden;
+        a.A = E.dlogits;
+        a.lda = C;
+        a.B = params + m->Wc2;
+        a.ldb = C;
+        a.b_trans = 1;
+        a.C = E.dA;
+        a.ldc = E.ld_cls;
+        a.mul_pos = E.cls_act;
+        a.mul_pos_ld = E.ld_cls;
+        a.mul_pos_dtype = D.dtype;
+        SGCN_TRY(gemm_run(a, st));
+        WgradArgs w1;
+        w1.M = n;
+        w1.K = HW;
+        w1.N = D.hidden;
+        w1.A = hin;
+        w1.lda = E.ld_h;
+        w1.a_dtype = D.dtype;
+        w1.B = E.dA;
+        w1.ldb = E.ld_cls;
+        w1.dW = grads + m->Wc1;
+        w1.dbias = grads + m->bc1;
+        SGCN_TRY(wgrad_run(w1, E.ws, E.ws_bytes, st));
+        GemmArgs h;   // dH = dA Wc1^T
+        h.M = n;
+        h.K = D.hidden;
+        h.N = HW;
+        h.A = E.dA;
+        h.lda = E.ld_cls;
+        h.B = params + m->Wc1;
+        h.ldb = D.hidden;
+        h.b_trans = 1;
+        h.C = E.dH[0];
+        h.ldc = E.ld_grad;
+        SGCN_TRY(gemm_run(h, st));
+    }
+    int cur = 0;
+    for (int l = L - 1; l >= 0; --l) {
+        const void* lin = l == 0 ? h0 : E.H[l - 1];
+        const bool need_din = l > 0 || D.use_ff;
+        SGCN_TRY(layer_backward_impl(g, &descs[l], plans[l], lin, E.saved[l], E.dH[cur], E.ld_grad,
+                                     need_din ? E.dH[cur ^ 1] : nullptr, E.ld_grad, grads + m->W_agg[l],
+                                     D.use_self ? grads + m->W_self[l] : nullptr, grads + m->b[l],
+                                     D.use_b_self ? grads + m->b_self[l] : nullptr,
+                                     (D.use_se && l == L - 1) ? grads + m->E : nullptr, E.ws, E.ws_bytes, st));
+        cur ^= 1;
+    }
+    if (D.use_ff) {   // backward of the fusion MLP from dX_ff (sum over slices already formed)
+        float* dxff = E.dH[cur];
+        WgradArgs w;
+        w.M = n;
+        w.K = D.in_d;
+        w.N = m->slice_size;
+        w.A = E.ff_act;
+        w.lda = E.ld_ffact;
+        w.a_dtype = D.dtype;
+        w.B = dxff;
+        w.ldb = E.ld_grad;
+        w.dW = grads + m->ff_W2;
+        w.dbias = grads + m->ff_b2;
+        SGCN_TRY(wgrad_run(w, E.ws, E.ws_bytes, st));
+        float* dact = E.dH[cur ^ 1];
+        GemmArgs a;
+        a.M = n;
+        a.K = m->slice_size;
+        a.N = D.in_d;
+        a.A = dxff;
+        a.lda = E.ld_grad;
+        a.B = params + m->ff_W2;
+        a.ldb = m->slice_size;
+        a.b_trans = 1;
+        a.C = dact;
+        a.ldc = E.ld_grad;
+        a.mul_pos = E.ff_act;
+        a.mul_pos_ld = E.ld_ffact;
+        a.mul_pos_dtype = D.dtype;
+        SGCN_TRY(gemm_run(a, st));
+        WgradArgs w1;
+        w1.M = n;
+        w1.K = D.in_d;
+        w1.N = D.in_d;
+        w1.A = X;
+        w1.lda = x_ld;
+        w1.a_dtype = D.dtype;
+        w1.B = dact;
+        w1.ldb = E.ld_grad;
+        w1.dW = grads + m->ff_W1;
+        w1.dbias = grads + m->ff_b1;
+        SGCN_TRY(wgrad_run(w1, E.ws, E.ws_bytes, st));
+    }
+    // ---------------- update: Adam, cosine-annealed learning rate, one step per epoch
+    if (opt) {
+        const double kPi = 3.14159265358979323846;
+        const double lr = opt->lr0 * 0.5 * (1.0 + std::cos(kPi * (double)opt->epoch / (double)opt->total_epochs));
+        SGCN_TRY(adam_run(m->param_elems, params, grads, adam_m, adam_v, (float)lr, (float)opt->beta1, (float)opt->beta2,
+                          (float)opt->eps, (float)opt->weight_decay, opt->epoch + 1, st));
+    }
+    return SLICEGCN_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,500 @@
+// Normalised sparse aggregation  Y = A_hat X  (Eq. 1 / Eq. 6 neighbor sum; A_hat^T X in backward).
+//
+// Row-parallel CSR kernel.  A group of L lanes owns one row; each lane keeps C 16-byte chunks of
+// the output row in registers, so one 128-bit load per lane per chunk covers a neighbor's slice
+// row.  Column indices are read coalesced (L at a time) together with the neighbor's 1/sqrt(deg)
+// and handed around with shuffles; U neighbors are gathered before the FMAs so several rows are in
+// flight per lane.  No per-edge value array exists:  A_hat_ij = dinv_i * dinv_j.
+// Rows longer than kLongRow are cut into kSegment-entry segments, one warp each, whose partial
+// rows are summed afterwards in segment order -- deterministic, no floating-point atomics.
+#include <vector>
+
+#include "common.cuh"
+#include "kernels.cuh"
+
+namespace sgcn {
+namespace {
+
+template <typename T>
+struct Vec;
+template <>
+struct Vec<float> {
+    static constexpr int V = 4;
+    static __device__ __forceinline__ void unpack(const uint4& r, float (&f)[4]) {
+        f[0] = __uint_as_float(r.x);
+        f[1] = __uint_as_float(r.y);
+        f[2] = __uint_as_float(r.z);
+        f[3] = __uint_as_float(r.w);
+    }
+    static __device__ __forceinline__ void store(float* p, const float (&f)[4]) {
+        *reinterpret_cast<float4*>(p) = make_float4(f[0], f[1], f[2], f[3]);
+    }
+};
+template <>
+struct Vec<__nv_bfloat16> {
+    static constexpr int V = 8;
+    static __device__ __forceinline__ void unpack(const uint4& r, float (&f)[8]) {
+        const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            f[2 * i] = __uint_as_float(w[i] << 16);
+            f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+        }
+    }
+    static __device__ __forceinline__ void store(__nv_bfloat16* p, const float (&f)[8]) {
+        uint4 r;
+        uint32_t* w = reinterpret_cast<uint32_t*>(&r);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+            w[i] = *reinterpret_cast<uint32_t*>(&h);
+        }
+        *reinterpret_cast<uint4*>(p) = r;
+    }
+};
+
+__device__ __forceinline__ float to_f(float v) { return v; }
+__device__ __forceinline__ float to_f(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T>
+__device__ __forceinline__ T from_f(float v);
+template <>
+__device__ __forceinline__ float from_f<float>(float v) { return v; }
+template <>
+__device__ __forceinline__ __nv_bfloat16 from_f<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+struct SpmmParams {
+    int64_t n;
+    const int32_t* rowptr;
+    const int32_t* colidx;
+    const float* dinv;
+    const void* X;
+    int64_t ldx;
+    void* Y;
+    int64_t ldy;
+    int32_t width;   // columns
+    int32_t nch;     // 16-byte chunks per row = ceil(width / V)
+    // long rows
+    int32_t n_long, n_seg;
+    const int32_t* long_rows;
+    const int32_t* seg_ptr;
+    const int32_t* seg_row;
+    float* partial;  // [n_seg][nch*V]
+    // epilogue (transform-first layers):  y = act(dinv_i*acc + bias) (+ previous y)
+    const float* bias;
+    uint8_t* mask;
+    int64_t mask_ld;
+    int32_t relu;
+    int32_t accumulate;
+};
+
+constexpr int kU = 4;   // neighbors gathered per lane before accumulating
+
+// Accumulate neighbors [base, base+cnt) of one row; lane `sl` of the group holds colidx[base+sl].
+template <typename TI, int L, int C>
+__device__ __forceinline__ void gather_block(const SpmmParams& p, unsigned gmask, int sl, int j, float dj, int cnt,
+                                             float (&acc)[C][Vec<TI>::V]) {
+    constexpr int V = Vec<TI>::V;
+    const TI* X = static_cast<const TI*>(p.X);
+    for (int t = 0; t < cnt; t += kU) {
+        uint4 raw[kU][C];
+        float dd[kU];
+#pragma unroll
+        for (int u = 0; u < kU; ++u) {
+            const int jj = __shfl_sync(gmask, j, (t + u) & (L - 1), L);
+            dd[u] = __shfl_sync(gmask, dj, (t + u) & (L - 1), L);
+            const bool live = (t + u) < cnt;
+            if (!live) dd[u] = 0.f;
+            const TI* xr = X + (int64_t)jj * p.ldx;
+#pragma unroll
+            for (int c = 0; c < C; ++c) {
+                const int chunk = sl + c * L;
+                if (live && chunk < p.nch)
+                    raw[u][c] = __ldg(reinterpret_cast<const uint4*>(xr + chunk * V));
+                else
+                    raw[u][c] = make_uint4(0, 0, 0, 0);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kU; ++u)
+#pragma unroll
+            for (int c = 0; c < C; ++c) {
+                float f[V];
+                Vec<TI>::unpack(raw[u][c], f);
+#pragma unroll
+                for (int e = 0; e < V; ++e) acc[c][e] = fmaf(dd[u], f[e], acc[c][e]);
+            }
+    }
+}
+
+template <typename TO, int V, bool EPI>
+__device__ __forceinline__ void finish_chunk(const SpmmParams& p, int64_t row, int chunk, float di, float (&o)[V]) {
+    TO* Y = static_cast<TO*>(p.Y) + row * p.ldy;
+    const int col0 = chunk * V;
+#pragma unroll
+    for (int e = 0; e < V; ++e) o[e] *= di;
+    if (EPI) {
+#pragma unroll
+        for (int e = 0; e < V; ++e) {
+            const int col = col0 + e;
+            if (col < p.width) {
+                float x = o[e] + (p.bias ? __ldg(p.bias + col) : 0.f);
+                if (p.relu) {
+                    if (p.mask) p.mask[row * p.mask_ld + col] = x > 0.f ? 1 : 0;
+                    x = fmaxf(x, 0.f);
+                }
+                if (p.accumulate) x += to_f(Y[col]);
+                o[e] = x;
+            }
+        }
+    }
+    if (col0 + V <= p.width && V == Vec<TO>::V) {
+        Vec<TO>::store(Y + col0, reinterpret_cast<float(&)[Vec<TO>::V]>(o));
+    } else {
+#pragma unroll
+        for (int e = 0; e < V; ++e)
+            if (col0 + e < p.width) Y[col0 + e] = from_f<TO>(o[e]);
+    }
+}
+
+template <typename TI, typename TO, int L, int C, bool EPI>
+__global__ void __launch_bounds__(256) spmm_rows_kernel(const SpmmParams p) {
+    constexpr int V = Vec<TI>::V;
+    constexpr int RPW = 32 / L;
+    const int lane = threadIdx.x & 31;
+    const int sub = lane / L, sl = lane % L;
+    const int64_t warp = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
+    const int64_t row = warp * RPW + sub;
+    if (row >= p.n) return;
+    const unsigned gmask = (L == 32) ? 0xffffffffu : (((1u << L) - 1u) << (sub * L));
+    const int start = __ldg(p.rowptr + row), end = __ldg(p.rowptr + row + 1);
+    if (end - start > kLongRow) return;   // long rows: segment kernels
+    float acc[C][V];
+#pragma unroll
+    for (int c = 0; c < C; ++c)
+#pragma unroll
+        for (int e = 0; e < V; ++e) acc[c][e] = 0.f;
+    for (int base = start; base < end; base += L) {
+        const int k = base + sl;
+        int j = 0;
+        float dj = 0.f;
+        if (k < end) {
+            j = __ldg(p.colidx + k);
+            dj = __ldg(p.dinv + j);
+        }
+        gather_block<TI, L, C>(p, gmask, sl, j, dj, min(L, end - base), acc);
+    }
+    const float di = __ldg(p.dinv + row);
+#pragma unroll
+    for (int c = 0; c < C; ++c) {
+        const int chunk = sl + c * L;
+        if (chunk < p.nch) finish_chunk<TO, V, EPI>(p, row, chunk, di, acc[c]);
+    }
+}
+
+// One warp per segment of a long row; the 32/L lane groups interleave over the segment's
+// neighbors and are combined with a butterfly (fixed order).
+template <typename TI, int L, int C>
+__global__ void __launch_bounds__(256) spmm_segment_kernel(const SpmmParams p) {
+    constexpr int V = Vec<TI>::V;
+    const int lane = threadIdx.x & 31;
+    const int sub = lane / L, sl = lane % L;
+    const int seg = (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5);
+    if (seg >= p.n_seg) return;
+    const unsigned gmask = (L == 32) ? 0xffffffffu : (((1u << L) - 1u) << (sub * L));
+    const int li = __ldg(p.seg_row + seg);
+    const int row = __ldg(p.long_rows + li);
+    const int start = __ldg(p.rowptr + row) + (seg - __ldg(p.seg_ptr + li)) * kSegment;
+    const int end = min(__ldg(p.rowptr + row + 1), start + kSegment);
+    float acc[C][V];
+#pragma unroll
+    for (int c = 0; c < C; ++c)
+#pragma unroll
+        for (int e = 0; e < V; ++e) acc[c][e] = 0.f;
+    for (int base = start + sub * L; base < end; base += 32) {
+        const int k = base + sl;
+        int j = 0;
+        float dj = 0.f;
+        if (k < end) {
+            j = __ldg(p.colidx + k);
+            dj = __ldg(p.dinv + j);
+        }
+        gather_block<TI, L, C>(p, gmask, sl, j, dj, min(L, end - base), acc);
+    }
+    __syncwarp();
+#pragma unroll
+    for (int off = L; off < 32; off <<= 1)
+#pragma unroll
+        for (int c = 0; c < C; ++c)
+#pragma unroll
+            for (int e = 0; e < V; ++e) acc[c][e] += __shfl_xor_sync(0xffffffffu, acc[c][e], off);
+    if (sub == 0) {
+        float* out = p.partial + (int64_t)seg * (p.nch * V);
+#pragma unroll
+        for (int c = 0; c < C; ++c) {
+            const int chunk = sl + c * L;
+            if (chunk < p.nch) {
+#pragma unroll
+                for (int e = 0; e < V; e += 4)
+                    *reinterpret_cast<float4*>(out + chunk * V + e) =
+                        make_float4(acc[c][e], acc[c][e + 1], acc[c][e + 2], acc[c][e + 3]);
+            }
+        }
+    }
+}
+
+// Sums the partial rows of each long row in segment order, then scales / applies the epilogue.
+template <typename TO, bool EPI>
+__global__ void __launch_bounds__(256) spmm_long_finish_kernel(const SpmmParams p, int pstride) {
+    const int lane = threadIdx.x & 31;
+    const int li = (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5);
+    if (li >= p.n_long) return;
+    const int64_t row = __ldg(p.long_rows + li);
+    const int s0 = __ldg(p.seg_ptr + li), s1 = __ldg(p.seg_ptr + li + 1);
+    const float di = __ldg(p.dinv + row);
+    TO* Y = static_cast<TO*>(p.Y) + row * p.ldy;
+    for (int col = lane; col < p.width; col += 32) {
+        float a = 0.f;
+        for (int s = s0; s < s1; ++s) a += p.partial[(int64_t)s * pstride + col];
+        float x = a * di;
+        if (EPI) {
+            x += p.bias ? __ldg(p.bias + col) : 0.f;
+            if (p.relu) {
+                if (p.mask) p.mask[row * p.mask_ld + col] = x > 0.f ? 1 : 0;
+                x = fmaxf(x, 0.f);
+            }
+            if (p.accumulate) x += to_f(Y[col]);
+        }
+        Y[col] = from_f<TO>(x);
+    }
+}
+
+// Fallback for operands that do not allow 128-bit access (odd leading dimension / alignment):
+// one warp per row, lanes over columns, scalar loads.  Handles long rows too (slow path).
+template <typename TI, typename TO, bool EPI>
+__global__ void __launch_bounds__(256) spmm_scalar_kernel(const SpmmParams p) {
+    const int lane = threadIdx.x & 31;
+    const int64_t row = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
+    if (row >= p.n) return;
+    const TI* X = static_cast<const TI*>(p.X);
+    TO* Y = static_cast<TO*>(p.Y) + row * p.ldy;
+    const int start = __ldg(p.rowptr + row), end = __ldg(p.rowptr + row + 1);
+    const float di = __ldg(p.dinv + row);
+    for (int col = lane; col < p.width; col += 32) {
+        float a = 0.f;
+        for (int k = start; k < end; ++k) {
+            const int j = __ldg(p.colidx + k);
+            a = fmaf(__ldg(p.dinv + j), to_f(X[(int64_t)j * p.ldx + col]), a);
+        }
+        float x = a * di;
+        if (EPI) {
+            x += p.bias ? __ldg(p.bias + col) : 0.f;
+            if (p.relu) {
+                if (p.mask) p.mask[row * p.mask_ld + col] = x > 0.f ? 1 : 0;
+                x = fmaxf(x, 0.f);
+            }
+            if (p.accumulate) x += to_f(Y[col]);
+        }
+        Y[col] = from_f<TO>(x);
+    }
+}
+
+template <typename TI, typename TO, int L, int C>
+slicegcn_status_t launch_lc(const SpmmParams& p, bool epi, cudaStream_t st) {
+    constexpr int RPW = 32 / L;
+    const int64_t warps = (p.n + RPW - 1) / RPW;
+    const int64_t blocks = (warps + 7) / 8;
+    if (epi)
+        spmm_rows_kernel<TI, TO, L, C, true><<<(unsigned)blocks, 256, 0, st>>>(p);
+    else
+        spmm_rows_kernel<TI, TO, L, C, false><<<(unsigned)blocks, 256, 0, st>>>(p);
+    SGCN_LAUNCH_CHECK();
+    count_launch();
+    if (p.n_seg > 0) {
+        spmm_segment_kernel<TI, L, C><<<(p.n_seg + 7) / 8, 256, 0, st>>>(p);
+        SGCN_LAUNCH_CHECK();
+        const int pstride = p.nch * Vec<TI>::V;
+        if (epi)
+            spmm_long_finish_kernel<TO, true><<<(p.n_long + 7) / 8, 256, 0, st>>>(p, pstride);
+        else
+            spmm_long_finish_kernel<TO, false><<<(p.n_long + 7) / 8, 256, 0, st>>>(p, pstride);
+        SGCN_LAUNCH_CHECK();
+        count_launch(2);
+    }
+    return SLICEGCN_OK;
+}
+
+template <typename TI, typename TO>
+slicegcn_status_t launch_vec(const SpmmParams& p, bool epi, cudaStream_t st) {
+    const int nch = p.nch;
+    if (nch <= 2) return launch_lc<TI, TO, 2, 1>(p, epi, st);
+    if (nch <= 4) return launch_lc<TI, TO, 4, 1>(p, epi, st);
+    if (nch <= 8) return launch_lc<TI, TO, 8, 1>(p, epi, st);
+    if (nch <= 16) return launch_lc<TI, TO, 16, 1>(p, epi, st);
+    if (nch <= 32) return launch_lc<TI, TO, 32, 1>(p, epi, st);
+    if (nch <= 64) return launch_lc<TI, TO, 32, 2>(p, epi, st);
+    if (nch <= 96) return launch_lc<TI, TO, 32, 3>(p, epi, st);
+    return launch_lc<TI, TO, 32, 4>(p, epi, st);
+}
+
+template <typename TI, typename TO>
+slicegcn_status_t launch_typed(SpmmParams p, bool vec_ok, bool epi, cudaStream_t st) {
+    constexpr int V = Vec<TI>::V;
+    if (!vec_ok) {
+        const int64_t blocks = (p.n + 7) / 8;
+        if (epi)
+            spmm_scalar_kernel<TI, TO, true><<<(unsigned)blocks, 256, 0, st>>>(p);
+        else
+            spmm_scalar_kernel<TI, TO, false><<<(unsigned)blocks, 256, 0, st>>>(p);
+        SGCN_LAUNCH_CHECK();
+        count_launch();
+        return SLICEGCN_OK;
+    }
+    // column blocks of at most 128 chunks (32 lanes x 4 chunks)
+    const int total = p.width;
+    const int block_cols = 128 * V;
+    const TI* X = static_cast<const TI*>(p.X);
+    TO* Y = static_cast<TO*>(p.Y);
+    for (int c0 = 0; c0 < total; c0 += block_cols) {
+        SpmmParams q = p;
+        q.width = min(block_cols, total - c0);
+        q.nch = (q.width + V - 1) / V;
+        q.X = X + c0;
+        q.Y = Y + c0;
+        if (q.bias) q.bias += c0;
+        if (q.mask) q.mask += c0;
+        SGCN_TRY((launch_vec<TI, TO>(q, epi, st)));
+    }
+    return SLICEGCN_OK;
+}
+
+}  // namespace
+
+// ---- instrumentation ---------------------------------------------------------------------------
+namespace {
+struct Profiler {
+    bool on = false;
+    std::vector<cudaEvent_t> ev;   // pairs
+    size_t used = 0;
+    int64_t calls = 0;
+    double bytes = 0.0;
+} g_prof;
+}  // namespace
+
+int64_t spmm_partial_bytes(const slicegcn_graph* g, int width) {
+    // enough for either dtype: chunks of 8 elements, at most 128 chunks per column block
+    int64_t w = width < 1024 ? width : 1024;
+    int64_t padded = (w + 7) / 8 * 8;
+    return (int64_t)g->max_segments() * padded * (int64_t)sizeof(float);
+}
+
+slicegcn_status_t spmm_run(const slicegcn_graph* g, bool transpose, int in_dtype, int out_dtype, const void* X,
+                           int64_t ldx, void* Y, int64_t ldy, int width, const SpmmEpilogue* epi, void* ws,
+                           int64_t ws_bytes, cudaStream_t st) {
+    if (!g || !X || !Y) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "spmm: NULL argument");
+    if (width < 1 || ldx < width || ldy < width) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "spmm: bad width / leading dimension");
+    if (in_dtype != out_dtype) SGCN_FAIL(SLICEGCN_ERR_UNSUPPORTED, "spmm: input and output dtype must match");
+    if (in_dtype != SLICEGCN_F32 && in_dtype != SLICEGCN_BF16) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "spmm: bad dtype");
+    const CsrView v = g->view(transpose);
+    SpmmParams p{};
+    p.n = g->n;
+    p.rowptr = v.rowptr;
+    p.colidx = v.colidx;
+    p.dinv = g->dinv;
+    p.X = X;
+    p.ldx = ldx;
+    p.Y = Y;
+    p.ldy = ldy;
+    p.width = width;
+    const int V = in_dtype == SLICEGCN_F32 ? 4 : 8;
+    const int64_t esz = in_dtype == SLICEGCN_F32 ? 4 : 2;
+    p.nch = (width + V - 1) / V;
+    const bool vec_ok = ((uintptr_t)X % 16 == 0) && ((uintptr_t)Y % 16 == 0) && (ldx * esz) % 16 == 0 &&
+                        (ldy * esz) % 16 == 0 && (int64_t)p.nch * V <= ldx;
+    if (vec_ok) {
+        p.n_long = v.n_long;
+        p.n_seg = v.n_seg;
+        p.long_rows = v.long_rows;
+        p.seg_ptr = v.seg_ptr;
+        p.seg_row = v.seg_row;
+        p.partial = static_cast<float*>(ws);
+        if (v.n_seg > 0 && (!ws || ws_bytes < spmm_partial_bytes(g, width)))
+            SGCN_FAIL(SLICEGCN_ERR_ALLOC, "spmm: workspace too small (%lld < %lld bytes)", (long long)ws_bytes,
+                      (long long)spmm_partial_bytes(g, width));
+    }
+    cudaEvent_t ev_stop = nullptr;
+    if (g_prof.on) {
+        if (g_prof.used + 2 > g_prof.ev.size()) {
+            for (int i = 0; i < 2; ++i) {
+                cudaEvent_t e;
+                SGCN_CUDA(cudaEventCreate(&e));
+                g_prof.ev.push_back(e);
+            }
+        }
+        SGCN_CUDA(cudaEventRecord(g_prof.ev[g_prof.used], st));
+        ev_stop = g_prof.ev[g_prof.used + 1];
+        g_prof.used += 2;
+        g_prof.calls += 1;
+        g_prof.bytes += 4.0 * (double)g->nnz + 4.0 * (double)(g->n + 1) + 4.0 * (double)g->n +
+                        2.0 * (double)g->n * (double)width * (double)esz;
+    }
+    bool has_epi = false;
+    if (epi) {
+        p.bias = epi->bias;
+        p.mask = epi->mask;
+        p.mask_ld = epi->mask_ld;
+        p.relu = epi->relu;
+        p.accumulate = epi->accumulate;
+        has_epi = true;
+    }
+    slicegcn_status_t rc = in_dtype == SLICEGCN_F32 ? launch_typed<float, float>(p, vec_ok, has_epi, st)
+                                                     : launch_typed<__nv_bfloat16, __nv_bfloat16>(p, vec_ok, has_epi, st);
+    if (ev_stop) SGCN_CUDA(cudaEventRecord(ev_stop, st));
+    return rc;
+}
+
+}  // namespace sgcn
+
+extern "C" {
+
+slicegcn_status_t slicegcn_profile_begin(void) {
+    using namespace sgcn;
+    g_prof.on = true;
+    g_prof.used = 0;
+    g_prof.calls = 0;
+    g_prof.bytes = 0.0;
+    reset_launches();
+    return SLICEGCN_OK;
+}
+
+slicegcn_status_t slicegcn_profile_end(double* spmm_ms, int64_t* spmm_calls, double* spmm_bytes,
+                                       int64_t* kernel_launches) {
+    using namespace sgcn;
+    g_prof.on = false;
+    SGCN_CUDA(cudaDeviceSynchronize());
+    double ms = 0.0;
+    for (size_t i = 0; i + 1 < g_prof.used; i += 2) {
+        float t = 0.f;
+        SGCN_CUDA(cudaEventElapsedTime(&t, g_prof.ev[i], g_prof.ev[i + 1]));
+        ms += t;
+    }
+    if (spmm_ms) *spmm_ms = ms;
+    if (spmm_calls) *spmm_calls = g_prof.calls;
+    if (spmm_bytes) *spmm_bytes = g_prof.bytes;
+    if (kernel_launches) *kernel_launches = launches();
+    return SLICEGCN_OK;
+}
+
+slicegcn_status_t slicegcn_spmm_workspace_bytes(const slicegcn_graph* g, int32_t width, int64_t* bytes) {
+    if (!g || !bytes || width < 1) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "spmm_workspace_bytes: bad argument");
+    *bytes = sgcn::spmm_partial_bytes(g, width);
+    return SLICEGCN_OK;
+}
+
+slicegcn_status_t slicegcn_spmm(const slicegcn_graph* g, int32_t transpose, int32_t in_dtype, int32_t out_dtype,
+                                const void* X, int64_t ldx, void* Y, int64_t ldy, int32_t width, void* workspace,
+                                int64_t workspace_bytes, void* stream) {
+    return sgcn::spmm_run(g, transpose != 0, in_dtype, out_dtype, X, ldx, Y, ldy, width, nullptr, workspace,
+                          workspace_bytes, (cudaStream_t)stream);
+}
+
+}  // extern "C"

@@ -1,0 +1,337 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle, element by element,
+on the same seeded inputs.  Index work must be bit-exact; fp32 tensors must agree to 1e-4 and
+bf16-stored ones to 2e-2 in max|a-b|/max|b| (logits and gradients)."""
+import numpy as np
+import pytest
+
+from oracle import slicegcn_oracle as orc
+from paper_2408_11500_b200 import synth
+
+from helpers import GpuProblem, oracle_desc, rel_inf, small_problem
+
+pytestmark = pytest.mark.gpu
+
+TOL_F32 = 1e-4
+TOL_BF16 = 2e-2
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2408_11500_b200 import binding
+    return binding
+
+
+@pytest.fixture(scope="module")
+def torch():
+    import torch
+    return torch
+
+
+# ------------------------------------------------------------------------------ graph construction
+
+@pytest.mark.parametrize("sym,loops", [(True, True), (True, False), (False, True), (False, False)])
+def test_graph_create_bit_exact(B, sym, loops):
+    rng = np.random.default_rng(5)
+    n, m = 3000, 20000
+    src = rng.integers(0, n, m).astype(np.int32); dst = rng.integers(0, n, m).astype(np.int32)
+    src[:50] = 7                                    # a hub row and repeated pairs
+    dst[50:60] = src[50:60]                         # input self-loops
+    src[100:200] = src[200:300]; dst[100:200] = dst[200:300]
+    og = orc.build_graph(n, src, dst, sym, loops)
+    flags = (B.SYMMETRIZE if sym else 0) | (B.ADD_SELF_LOOPS if loops else 0)
+    g = B.slicegcn_graph_create(n, src, dst, flags)
+    try:
+        info = B.slicegcn_graph_info(g)
+        ex = B.slicegcn_graph_export(g)
+        assert info["n"] == n and info["nnz"] == og.nnz and info["symmetric"] == og.symmetric
+        assert np.array_equal(ex["rowptr"], og.rowptr)
+        assert np.array_equal(ex["colidx"], og.colidx)
+        assert np.array_equal(ex["deg"], og.deg)
+        assert np.array_equal(ex["dinv"].view(np.uint32), orc.dinv_f32(og.deg).view(np.uint32))
+    finally:
+        B.slicegcn_graph_destroy(g)
+
+
+def test_graph_from_csr_device_input_and_errors(B, torch):
+    src, dst = synth.chung_lu_powerlaw(2000, 9000, 2.2, 300, seed=2)
+    og = orc.build_graph(2000, src, dst, True, True)
+    # CSR with unsorted columns, given on the device
+    rng = np.random.default_rng(0)
+    col = og.colidx.copy()
+    for i in range(0, 2000, 7):
+        s, e = og.rowptr[i], og.rowptr[i + 1]
+        col[s:e] = rng.permutation(col[s:e])
+    rp = torch.from_numpy(og.rowptr).cuda(); ci = torch.from_numpy(col).cuda()
+    g = B.slicegcn_graph_create_from_csr(2000, rp, ci, B.INPUT_ON_DEVICE)
+    ex = B.slicegcn_graph_export(g)
+    assert np.array_equal(ex["rowptr"], og.rowptr) and np.array_equal(ex["colidx"], og.colidx)
+    B.slicegcn_graph_destroy(g)
+    with pytest.raises(B.SliceGCNError) as e:
+        B.slicegcn_graph_create(10, np.array([0, 11], np.int32), np.array([1, 2], np.int32), 0)
+    assert e.value.status == B.ERR_OUT_OF_RANGE
+    with pytest.raises(B.SliceGCNError) as e:
+        B.slicegcn_graph_create(0, np.array([0], np.int32), np.array([0], np.int32), 0)
+    assert e.value.status == B.ERR_INVALID_ARG
+    with pytest.raises(B.SliceGCNError):
+        B.slicegcn_graph_create_from_csr(3, np.array([0, 2, 1, 3], np.int32), np.array([0, 1, 2], np.int32), 0)
+    # no edges at all, self-loops only: A_hat = I
+    g = B.slicegcn_graph_create(5, np.zeros(0, np.int32), np.zeros(0, np.int32), B.ADD_SELF_LOOPS)
+    ex = B.slicegcn_graph_export(g)
+    assert ex["rowptr"].tolist() == [0, 1, 2, 3, 4, 5] and ex["colidx"].tolist() == [0, 1, 2, 3, 4]
+    B.slicegcn_graph_destroy(g)
+
+
+# ------------------------------------------------------------------------------ SpMM
+
+def _gpu_spmm(B, torch, g, X, width, dtype, transpose=False, ld_pad=0):
+    n = X.shape[0]
+    dt = torch.float32 if dtype == B.F32 else torch.bfloat16
+    ld = width + ld_pad
+    xd = torch.zeros((n, ld), dtype=dt, device="cuda")
+    xd[:, :width] = torch.from_numpy(X).cuda().to(dt)
+    yd = torch.full((n, ld), float("nan"), dtype=dt, device="cuda")
+    wsb = B.slicegcn_spmm_workspace_bytes(g, width)
+    ws = torch.empty(max(wsb, 16), dtype=torch.uint8, device="cuda")
+    B.slicegcn_spmm(g, int(transpose), dtype, dtype, xd, ld, yd, ld, width, ws, wsb, torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    out = yd.float().cpu().numpy()
+    assert np.isnan(out[:, width:]).all() if ld_pad else True      # padding columns are left alone
+    return out[:, :width], xd[:, :width].float().cpu().numpy()
+
+
+@pytest.mark.parametrize("width,ld_pad", [(1, 0), (4, 0), (13, 3), (16, 0), (32, 0), (100, 4), (128, 0), (256, 0),
+                                          (300, 4), (512, 0), (602, 6), (1100, 4), (37, 0), (77, 1)])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_spmm_matches_oracle(B, torch, width, ld_pad, dtype):
+    n = 5000
+    src, dst = synth.chung_lu_powerlaw(n, 30000, 2.2, 1500, seed=1)      # several rows longer than 256
+    og = orc.build_graph(n, src, dst, True, True)
+    assert og.deg.max() > 600 and (og.deg > 256).sum() >= 3
+    g = B.slicegcn_graph_create(n, src, dst, B.SYMMETRIZE | B.ADD_SELF_LOOPS)
+    try:
+        assert B.slicegcn_graph_info(g)["n_segments"] > 0
+        X = synth.gaussian_features(n, width, seed=width)
+        dt = B.F32 if dtype == "f32" else B.BF16
+        got, x_used = _gpu_spmm(B, torch, g, X, width, dt, ld_pad=ld_pad)
+        want = orc.spmm(og, x_used.astype(np.float64))
+        if dtype == "f32":
+            assert rel_inf(got, want) <= 2e-6
+            assert np.abs(got - want).max() <= 1e-5 * max(1.0, np.abs(want).max())
+        else:   # one bf16 rounding of the fp32-accumulated result
+            assert np.all(np.abs(got - want) <= 2 ** -8 * np.abs(want) + 1e-5 * np.abs(want).max())
+    finally:
+        B.slicegcn_graph_destroy(g)
+
+
+def test_spmm_transposed_on_directed_graph(B, torch):
+    rng = np.random.default_rng(3)
+    n = 4000
+    src = rng.integers(0, n, 40000).astype(np.int32); dst = rng.integers(0, n, 40000).astype(np.int32)
+    dst[:900] = 11                                           # a long column -> long row of the transpose
+    og = orc.build_graph(n, src, dst, False, False)
+    g = B.slicegcn_graph_create(n, src, dst, 0)
+    try:
+        assert not B.slicegcn_graph_info(g)["symmetric"]
+        X = synth.gaussian_features(n, 64, seed=9)
+        got, _ = _gpu_spmm(B, torch, g, X, 64, B.F32, transpose=True)
+        assert rel_inf(got, orc.spmm(og, X.astype(np.float64), transpose=True)) <= 2e-6
+        got, _ = _gpu_spmm(B, torch, g, X, 64, B.F32, transpose=False)
+        assert rel_inf(got, orc.spmm(og, X.astype(np.float64))) <= 2e-6
+    finally:
+        B.slicegcn_graph_destroy(g)
+
+
+def test_spmm_is_deterministic_and_identity_holds(B, torch):
+    n = 20000
+    src, dst = synth.chung_lu_powerlaw(n, 150000, 2.2, 3000, seed=4)
+    g = B.slicegcn_graph_create(n, src, dst, B.SYMMETRIZE | B.ADD_SELF_LOOPS)
+    try:
+        deg = B.slicegcn_graph_export(g)["deg"]
+        v = np.sqrt(deg.astype(np.float64))
+        X = np.repeat(v[:, None], 32, axis=1).astype(np.float32)
+        a, _ = _gpu_spmm(B, torch, g, X, 32, B.F32)
+        b, _ = _gpu_spmm(B, torch, g, X, 32, B.F32)
+        assert np.array_equal(a, b)                          # no floating-point atomics anywhere
+        np.testing.assert_allclose(a, X, rtol=3e-6)          # A_hat sqrt(deg) = sqrt(deg)
+    finally:
+        B.slicegcn_graph_destroy(g)
+
+
+# ------------------------------------------------------------------------------ one layer
+
+@pytest.mark.parametrize("order", ["agg", "xform"])
+@pytest.mark.parametrize("case", ["plain_gcn", "sliced", "overlap_se_bself", "shared_input"])
+def test_layer_forward_backward(B, torch, order, case):
+    n = 1500
+    src, dst = synth.chung_lu_powerlaw(n, 7000, 2.2, 500, seed=6)
+    og = orc.build_graph(n, src, dst, True, True)
+    g = B.slicegcn_graph_create(n, src, dst, B.SYMMETRIZE | B.ADD_SELF_LOOPS)
+    rng = np.random.default_rng(1)
+    if case == "plain_gcn":
+        p, in_cols, starts, w_in, h_s, use_self, use_bs, use_e = 1, 45, [0], 45, 19, False, False, False
+    elif case == "sliced":
+        p, in_cols, starts, w_in, h_s, use_self, use_bs, use_e = 4, 48, [0, 12, 24, 36], 12, 8, True, False, False
+    elif case == "overlap_se_bself":
+        p, in_cols, starts, w_in, h_s, use_self, use_bs, use_e = 3, 10, [0, 4, 6], 4, 5, True, True, True
+    else:
+        p, in_cols, starts, w_in, h_s, use_self, use_bs, use_e = 3, 13, [0, 0, 0], 13, 6, True, False, True
+    in_ld, out_ld = in_cols + 3, p * h_s + 2
+    H = rng.standard_normal((n, in_cols)).astype(np.float32)
+    Wa = (rng.standard_normal((p, w_in, h_s)) * 0.3).astype(np.float32)
+    Ws = (rng.standard_normal((p, w_in, h_s)) * 0.3).astype(np.float32)
+    b = (rng.standard_normal((p, h_s)) * 0.2).astype(np.float32)
+    bs = (rng.standard_normal((p, h_s)) * 0.2).astype(np.float32)
+    E = (rng.standard_normal((p, h_s)) * 0.2).astype(np.float32)
+    dHo = rng.standard_normal((n, p * h_s)).astype(np.float32)
+    # ---- oracle, written out per slice from Eq. 6-7
+    H64 = H.astype(np.float64)
+    want_out = np.zeros((n, p * h_s)); dWa = np.zeros_like(Wa, np.float64); dWs = np.zeros_like(Ws, np.float64)
+    db = np.zeros((p, h_s)); dbs = np.zeros((p, h_s)); dHin = np.zeros((n, in_cols))
+    for i in range(p):
+        hin = H64[:, starts[i]:starts[i] + w_in]
+        z = orc.spmm(og, hin)
+        M = z @ Wa[i] + b[i]
+        o = np.maximum(M, 0)
+        if use_self: o = o + hin @ Ws[i]
+        if use_bs: o = o + bs[i]
+        if use_e: o = o + E[i]
+        want_out[:, i * h_s:(i + 1) * h_s] = o
+        d = dHo[:, i * h_s:(i + 1) * h_s].astype(np.float64)
+        dM = d * (M > 0)
+        dWa[i] = z.T @ dM; db[i] = dM.sum(0); dbs[i] = d.sum(0)
+        dh = orc.spmm(og, dM @ Wa[i].T.astype(np.float64), transpose=True)
+        if use_self:
+            dWs[i] = hin.T @ d
+            dh = dh + d @ Ws[i].T
+        dHin[:, starts[i]:starts[i] + w_in] += dh
+    # ---- CUDA path
+    cu = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    Hd = torch.zeros((n, in_ld), device="cuda"); Hd[:, :in_cols] = cu(H)
+    out = torch.full((n, out_ld), float("nan"), device="cuda")
+    Wad, Wsd, bd, bsd, Ed = cu(Wa), cu(Ws), cu(b), cu(bs), cu(E)
+    desc = B.make_layer_desc(p, starts, w_in, in_cols, in_ld, h_s, out_ld, B.F32,
+                             B.AGG_FIRST if order == "agg" else B.XFORM_FIRST, Wad, Wsd if use_self else None, bd,
+                             bsd if use_bs else None, Ed if use_e else None)
+    sb = B.slicegcn_layer_saved_bytes(g, desc); wb = B.slicegcn_layer_workspace_bytes(g, desc)
+    saved = torch.empty(sb, dtype=torch.uint8, device="cuda"); ws = torch.empty(max(wb, 16), dtype=torch.uint8, device="cuda")
+    st = torch.cuda.current_stream().cuda_stream
+    B.slicegcn_layer_forward(g, desc, Hd, out, saved, sb, ws, wb, st)
+    dHod = cu(dHo)
+    dHind = torch.full((n, in_ld), float("nan"), device="cuda")
+    gWa, gWs = torch.full_like(Wad, float("nan")), torch.full_like(Wsd, float("nan"))
+    gb, gbs, gE = torch.full_like(bd, float("nan")), torch.full_like(bd, float("nan")), torch.full_like(bd, float("nan"))
+    B.slicegcn_layer_backward(g, desc, Hd, saved, dHod, p * h_s, dHind, in_ld, gWa, gWs if use_self else None, gb,
+                              gbs if use_bs else None, gE if use_e else None, ws, wb, st)
+    torch.cuda.synchronize()
+    try:
+        assert rel_inf(out[:, :p * h_s].cpu().numpy(), want_out) <= TOL_F32
+        assert torch.isnan(out[:, p * h_s:]).all()
+        assert rel_inf(gWa.cpu().numpy(), dWa) <= TOL_F32
+        assert rel_inf(gb.cpu().numpy(), db) <= TOL_F32
+        assert rel_inf(dHind[:, :in_cols].cpu().numpy(), dHin) <= TOL_F32
+        if use_self: assert rel_inf(gWs.cpu().numpy(), dWs) <= TOL_F32
+        if use_bs: assert rel_inf(gbs.cpu().numpy(), dbs) <= TOL_F32
+        if use_e: assert rel_inf(gE.cpu().numpy(), dbs) <= TOL_F32
+    finally:
+        B.slicegcn_graph_destroy(g)
+
+
+# ------------------------------------------------------------------------------ whole epoch
+
+def _compare_epoch(gp, od, og, X, y, params, train_idx, tol, rnd=orc.identity, orders=None):
+    P = {k: v.astype(np.float64) for k, v in params.items()}
+    cache = orc.forward(od, og, X, P, y, train_idx, rnd=rnd, order=orders)
+    G = orc.backward(od, og, X, P, y, cache)
+    loss = gp.epoch(None)
+    errs = {"logits": rel_inf(gp.logits.cpu().numpy(), cache["logits"]), "loss": abs(loss - cache["loss"]) / abs(cache["loss"])}
+    got = gp.named_grads()
+    for k in P:
+        errs["d" + k] = rel_inf(got[k], G[k])
+    bad = {k: v for k, v in errs.items() if not v <= tol}
+    assert not bad, bad
+    return errs
+
+
+@pytest.mark.parametrize("kw", [
+    dict(p=4),
+    dict(p=1, use_self=False),
+    dict(p=3, in_d=10, hidden=6, use_se=True),
+    dict(p=3, in_d=10, hidden=7, use_ff=True, use_se=True),
+    dict(p=4, use_b_self=True, use_se=True, order=2),
+    dict(p=4, order=1, L=3),
+    dict(p=2, in_d=301, hidden=40, use_ff=True),
+])
+def test_epoch_gradients_fp32(B, kw):
+    kw = dict(kw)
+    order = kw.pop("order", 0)
+    src, dst, X, y, mk, od, params = small_problem(**kw)
+    mk["order"] = order
+    og = orc.build_graph(len(X), src, dst, True, True)
+    train_idx = np.arange(0, len(X), 3).astype(np.int32)
+    gp = GpuProblem(len(X), src, dst, X, y, params, train_idx=train_idx, **mk)
+    try:
+        orders = [{1: "agg", 2: "xform"}[B.slicegcn_model_layer_order(gp.m, l)] for l in range(mk["num_layers"])]
+        _compare_epoch(gp, od, og, X.astype(np.float64), y, params, train_idx, TOL_F32, orders=orders)
+    finally:
+        gp.close()
+
+
+def test_tiny_workload_ten_epochs_fp32(B):
+    """The tiny workload (2,708 nodes, 1,433 binary features, 4 overlapping slices, hidden 16):
+    ten training epochs, loss / logits / parameters tracked against the oracle."""
+    w = synth.WORKLOADS["tiny"]
+    src, dst = synth.make_graph(w, 0)
+    X = synth.make_features(w, 0); y = synth.uniform_labels(w["n"], w["classes"], 0)
+    mk = dict(in_d=w["in_d"], hidden=w["hidden"], num_layers=w["layers"], num_classes=w["classes"], num_slices=w["p"])
+    od = oracle_desc(**mk)
+    assert od.slices[-1] == (1074, 1433)
+    params = synth.init_params(orc.param_shapes(od), seed=0)
+    og = orc.build_graph(w["n"], src, dst, True, True)
+    gp = GpuProblem(w["n"], src, dst, X, y, params, **mk)
+    try:
+        P = {k: v.astype(np.float64) for k, v in params.items()}
+        st = {"m1": {}, "m2": {}}
+        orders = [{1: "agg", 2: "xform"}[B.slicegcn_model_layer_order(gp.m, l)] for l in range(2)]
+        for ep in range(10):
+            loss_o, logits_o, _ = orc.train_epoch(od, og, X.astype(np.float64), P, y, st, 0.01, ep, 10, order=orders)
+            loss_g = gp.epoch(B.make_opt_desc(lr0=0.01, epoch=ep, total_epochs=10))
+            assert abs(loss_g - loss_o) <= 1e-4 * abs(loss_o), (ep, loss_g, loss_o)
+            assert rel_inf(gp.logits.cpu().numpy(), logits_o) <= 5e-4, ep   # Adam amplifies rounding over epochs
+        got = gp.named_params()
+        for k in P:
+            assert rel_inf(got[k], P[k]) <= 2e-3, k
+    finally:
+        gp.close()
+
+
+def test_epoch_bf16_storage(B):
+    src, dst, X, y, mk, od, params = small_problem(n=3000, m_edges=15000, in_d=100, hidden=64, L=3, C=11, p=8,
+                                                   use_ff=True, use_se=True)
+    mk["dtype"] = B.BF16
+    Xr = orc.round_bf16(X)
+    og = orc.build_graph(len(X), src, dst, True, True)
+    gp = GpuProblem(len(X), src, dst, X, y, params, **mk)
+    try:
+        orders = [{1: "agg", 2: "xform"}[B.slicegcn_model_layer_order(gp.m, l)] for l in range(3)]
+        _compare_epoch(gp, od, og, Xr, y, params, None, TOL_BF16, rnd=orc.round_bf16, orders=orders)
+    finally:
+        gp.close()
+
+
+def test_citation_workload_full_size_fp32(B):
+    """The benchmark workload at full size (169,343 nodes, 3 layers, hidden 256, 8 slices), in the
+    launch configuration bench.py times: one epoch, every logit and gradient against the oracle."""
+    w = synth.WORKLOADS["citation"]
+    src, dst = synth.make_graph(w, 0)
+    X = synth.make_features(w, 0); y = synth.uniform_labels(w["n"], w["classes"], 0)
+    mk = dict(in_d=w["in_d"], hidden=w["hidden"], num_layers=w["layers"], num_classes=w["classes"], num_slices=w["p"])
+    od = oracle_desc(**mk)
+    params = synth.init_params(orc.param_shapes(od), seed=0)
+    og = orc.build_graph(w["n"], src, dst, True, True)
+    gp = GpuProblem(w["n"], src, dst, X, y, params, **mk)
+    try:
+        ex = B.slicegcn_graph_export(gp.g)
+        assert np.array_equal(ex["rowptr"], og.rowptr) and np.array_equal(ex["colidx"], og.colidx)
+        _compare_epoch(gp, od, og, X.astype(np.float64), y, params, None, TOL_F32)
+    finally:
+        gp.close()
