@@ -1,0 +1,306 @@
+#!/usr/bin/env python
+"""Benchmark: full-graph sliced-GCN training throughput (epochs/s) and SpMM bandwidth.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload citation] [--impl ours|reference]
+
+One "step" is one training epoch (Algorithm 3 of the paper: forward over every slice, loss,
+backward, one Adam update) on a seeded synthetic graph.  With N > 1 (launched under torchrun) every
+rank trains an independent replica: the single-GPU path has no sharding and no collectives, so
+`value` is the number of epochs all replicas finish per second (weak scaling).
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2408_11500_b200 import synth  # noqa: E402
+
+# dram__bytes_read.sum + dram__bytes_write.sum per SpMM launch from the ncu capture summarised under
+# profiles/ (None until a capture of that workload exists)
+NCU_SPMM_TRAFFIC_BYTES = {"citation": None}
+
+
+def measured_peak_gbs():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        return float(json.load(open(path))["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([t.strip() for t in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 6:
+                continue
+            try:
+                sm.append(float(r[0])); mx = float(r[1])
+            except ValueError:
+                continue
+            for nm, v in zip(names, r[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def scaled_workload(name: str, frac: float) -> dict:
+    w = dict(synth.WORKLOADS[name])
+    if frac < 1.0:
+        w["n"] = max(int(w["n"] * frac), 64)
+        w["m"] = max(int(w["m"] * frac), 64)
+        if "max_degree" in w:
+            w["max_degree"] = max(w["max_degree"] * frac, 16)
+    return w
+
+
+def model_kwargs(w: dict) -> dict:
+    return dict(in_d=w["in_d"], hidden=w["hidden"], num_layers=w["layers"], num_classes=w["classes"],
+                num_slices=w["p"], use_ff=w["use_ff"], use_se=w["use_se"])
+
+
+# ---------------------------------------------------------------------------------- oracle timing
+
+def oracle_epochs(w: dict, epochs: int, warm: int):
+    """Times the CPU oracle, as it stands, on workload w.  Returns (seconds per epoch list, threads)."""
+    from oracle import slicegcn_oracle as orc
+    src, dst = synth.make_graph(w, 0)
+    X = synth.make_features(w, 0).astype(np.float64)
+    y = synth.uniform_labels(w["n"], w["classes"], 0)
+    od = orc.ModelDesc(w["in_d"], w["hidden"], w["layers"], w["classes"], p=w["p"], use_ff=w["use_ff"], use_se=w["use_se"])
+    rnd = orc.round_bf16 if w["dtype"] == "bf16" else orc.identity
+    if w["dtype"] == "bf16":
+        X = orc.round_bf16(X)
+    P = {k: v.astype(np.float64) for k, v in synth.init_params(orc.param_shapes(od), 0).items()}
+    g = orc.build_graph(w["n"], src, dst, True, True)
+    st = {"m1": {}, "m2": {}}
+    times = []
+    for ep in range(warm + epochs):
+        t0 = time.perf_counter()
+        orc.train_epoch(od, g, X, P, y, st, 1e-3, ep, max(warm + epochs, 2), rnd=rnd)
+        if ep >= warm:
+            times.append(time.perf_counter() - t0)
+    return times, orc.max_threads()
+
+
+def run_reference(args, rank: int):
+    """--impl reference: the oracle on the host cores, on a bounded sample of the same workload."""
+    if rank != 0:
+        return
+    total_steps = args.steps + args.warmup
+    full_epoch_s = {"tiny": 0.4, "citation": 20.0, "social": 600.0, "copurchase": 900.0}[args.workload]
+    frac = 1.0
+    while frac > 1 / 64 and full_epoch_s * frac * total_steps > 200.0:
+        frac /= 2
+    w = scaled_workload(args.workload, frac)
+    times, threads = oracle_epochs(w, args.steps, args.warmup)
+    ms = 1e3 * sum(times) / len(times)
+    value = (1e3 / ms) * frac              # linear extrapolation to the full workload
+    sample = (f"{args.steps} epochs of the same generator at {frac:g} of the nodes and edges "
+              f"(n={w['n']}), epochs/s scaled by {frac:g}") if frac < 1 else f"{args.steps} full epochs"
+    line = {"impl": "reference", "metric": "full-graph GCN training throughput", "value": value, "unit": "epochs/s",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / frac,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload, "sample_fraction": frac},
+            "cpu_baseline": {"value": value, "unit": "epochs/s", "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": "epochs/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------- CUDA path
+
+def run_ours(args, rank: int, world: int, local_rank: int):
+    import torch
+    import torch.distributed as dist
+    from paper_2408_11500_b200 import binding as B
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    w = synth.WORKLOADS[args.workload]
+    src, dst = synth.make_graph(w, 0)
+    Xh = synth.make_features(w, 0)
+    yh = synth.uniform_labels(w["n"], w["classes"], 0)
+    n = w["n"]
+    dtype = B.BF16 if w["dtype"] == "bf16" else B.F32
+    tdt = torch.bfloat16 if dtype == B.BF16 else torch.float32
+    g = B.slicegcn_graph_create(n, src, dst, B.SYMMETRIZE | B.ADD_SELF_LOOPS)
+    info = B.slicegcn_graph_info(g)
+    m = B.slicegcn_model_create(dtype=dtype, **model_kwargs(w))
+    params0 = torch.from_numpy(B.pack_params(m, synth.init_params(B.named_param_shapes(m), 0))).to(dev)
+    params = params0.clone()
+    grads, m1, m2 = torch.zeros_like(params), torch.zeros_like(params), torch.zeros_like(params)
+    ws_bytes = B.slicegcn_train_workspace_bytes(m, g)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    X = torch.from_numpy(Xh).to(dev).to(tdt).contiguous()
+    y = torch.from_numpy(yh).to(dev)
+    loss = torch.zeros(1, dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream()
+    total_epochs = 500                        # the paper's schedule length (Table II); sets the cosine period
+
+    def epoch(ep, Xd, yd):
+        B.slicegcn_train_epoch(m, g, Xd, w["in_d"], yd, None, 0, params, grads, m1, m2,
+                               B.make_opt_desc(1e-3, ep, total_epochs), None, loss, ws, ws_bytes, stream.cuda_stream)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x: float) -> float:
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # ---- device-resident run
+    for ep in range(args.warmup):
+        epoch(ep, X, y)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    B.slicegcn_profile_begin()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for ep in range(args.steps):
+        epoch(args.warmup + ep, X, y)
+    e1.record(stream)
+    barrier()
+    prof = B.slicegcn_profile_end()
+    clocks = sampler.stop()
+    ms_total = max_over_ranks(e0.elapsed_time(e1))
+    final_loss = float(loss.item())
+
+    # ---- end to end: host buffers in, loss out, every step
+    Xp = (torch.from_numpy(Xh).to(tdt) if dtype == B.BF16 else torch.from_numpy(Xh)).pin_memory()
+    yp = torch.from_numpy(yh).pin_memory()
+    loss_host = torch.zeros(1, dtype=torch.float32).pin_memory()
+    Xd, yd = torch.empty_like(X), torch.empty_like(y)
+    params.copy_(params0); m1.zero_(); m2.zero_()
+
+    def e2e_step(ep):
+        Xd.copy_(Xp, non_blocking=True)
+        yd.copy_(yp, non_blocking=True)
+        epoch(ep, Xd, yd)
+        loss_host.copy_(loss, non_blocking=True)
+        stream.synchronize()                   # the caller reads the loss of this step
+
+    for ep in range(max(args.warmup, 1)):
+        e2e_step(ep)
+    barrier()
+    t0 = time.perf_counter()
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    f0.record(stream)
+    for ep in range(args.steps):
+        e2e_step(args.warmup + ep)
+    f1.record(stream)
+    barrier()
+    e2e_ms = max_over_ranks(max(f0.elapsed_time(f1), 1e3 * (time.perf_counter() - t0)))
+
+    value = world * args.steps / (ms_total / 1e3)
+    peak, peak_src = measured_peak_gbs()
+    spmm_avg_ms = prof["spmm_ms"] / max(prof["spmm_calls"], 1)
+    achieved = (prof["spmm_bytes"] / 1e9) / (prof["spmm_ms"] / 1e3) if prof["spmm_ms"] > 0 else 0.0
+    line = {
+        "metric": "full-graph GCN training throughput", "value": value, "unit": "epochs/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32" if dtype == B.F32 else "bf16", "data": "synthetic",
+        "config": {"workload": args.workload, "nodes": n, "nnz": info["nnz"], "in_d": w["in_d"], "hidden": w["hidden"],
+                   "layers": w["layers"], "classes": w["classes"], "num_slices": w["p"], "use_ff": w["use_ff"],
+                   "use_se": w["use_se"], "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "l2": "working set per epoch is larger than L2 (no flush needed)", "final_loss": final_loss},
+        "clocks": clocks,
+        "e2e": {"value": world * args.steps / (e2e_ms / 1e3), "unit": "epochs/s",
+                "h2d_bytes_per_step": Xp.numel() * Xp.element_size() + yp.numel() * 4, "d2h_bytes_per_step": 4},
+        "gpu_launches": int(prof["kernel_launches"]),
+        "roofline": {"bound": "hbm", "kernel": "spmm_rows_kernel (+ long-row segment kernels)",
+                     "achieved": achieved, "peak": peak, "peak_source": f"of {peak_src}", "unit": "GB/s",
+                     "frac": achieved / peak, "traffic": NCU_SPMM_TRAFFIC_BYTES.get(args.workload),
+                     "launches": int(prof["spmm_calls"]), "avg_ms": spmm_avg_ms,
+                     "algorithmic_bytes_per_launch": prof["spmm_bytes"] / max(prof["spmm_calls"], 1),
+                     "share_of_step": prof["spmm_ms"] / ms_total},
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cw = scaled_workload(args.workload, args.cpu_fraction)
+        times, threads = oracle_epochs(cw, 1, 0)
+        v = args.cpu_fraction / times[0]
+        sample = ("1 full epoch of the same workload" if args.cpu_fraction >= 1 else
+                  f"1 epoch of the same generator at {args.cpu_fraction:g} of the nodes and edges, scaled")
+        line["cpu_baseline"] = {"value": v, "unit": "epochs/s", "cores": threads, "kind": "oracle", "sample": sample}
+    B.slicegcn_model_destroy(m)
+    B.slicegcn_graph_destroy(g)
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="citation", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--cpu-fraction", type=float, default=1.0, help="size of the oracle's timed sample")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+    else:
+        run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

@@ -367,9 +367,14 @@ def forward(m: ModelDesc, g: Graph, x: np.ndarray, params: Dict[str, np.ndarray]
 
 
 def backward(m: ModelDesc, g: Graph, x: np.ndarray, params: Dict[str, np.ndarray], labels: np.ndarray,
-             cache: Dict[str, object], threads: int = 0) -> Dict[str, np.ndarray]:
+             cache: Dict[str, object], threads: int = 0, relu_margin: float = 0.0) -> Dict[str, np.ndarray]:
     """Reverse-mode gradient of the mean cross-entropy w.r.t. every parameter
-    (storage rounding treated as identity).  ReLU'(0) = 0."""
+    (storage rounding treated as identity).  ReLU'(0) = 0.
+
+    relu_margin (default 0 = the definition) moves the ReLU decision threshold to
+    relu_margin * max|pre-activation| of each ReLU: a positive / negative margin switches every
+    pre-activation that is within rounding noise of zero off / on.  Tests use the two results to
+    bound the effect of sign decisions that fp32 and fp64 arithmetic may take differently."""
     P = {k: np.asarray(v, dtype=np.float64) for k, v in params.items()}
     x = np.asarray(x, dtype=np.float64)
     idx = cache["train_idx"]
@@ -383,7 +388,11 @@ def backward(m: ModelDesc, g: Graph, x: np.ndarray, params: Dict[str, np.ndarray
     dlog[idx] = sm / idx.size
     G["Wc2"] = cache["cls_act"].T @ dlog
     G["bc2"] = dlog.sum(axis=0)
-    da = (dlog @ P["Wc2"].T) * (cache["cls_pre"] > 0)
+    def on(pre, scale=None):
+        sc = np.abs(pre).max() if scale is None else scale
+        return pre > relu_margin * sc
+
+    da = (dlog @ P["Wc2"].T) * on(cache["cls_pre"])
     hL = cache[f"H{m.num_layers}"]
     G["Wc1"] = hL.T @ da
     G["bc1"] = da.sum(axis=0)
@@ -395,10 +404,11 @@ def backward(m: ModelDesc, g: Graph, x: np.ndarray, params: Dict[str, np.ndarray
         dprev = np.zeros_like(hprev)
         if m.use_se and l == m.num_layers - 1:
             G["E"] = np.stack([dh[:, i * m.h_s:(i + 1) * m.h_s].sum(axis=0) for i in range(m.p)])
+        m_scale = max(np.abs(c[f"M.{l}.{i}"]).max() for i in range(m.p))
         for i, (s, e) in enumerate(ranges):
             dhi = dh[:, i * m.h_s:(i + 1) * m.h_s]
             hin = hprev[:, s:e]
-            dm = dhi * (c[f"M.{l}.{i}"] > 0)
+            dm = dhi * on(c[f"M.{l}.{i}"], m_scale)
             G[f"b.{l}.{i}"] = dm.sum(axis=0)
             if m.use_b_self:
                 G[f"b_self.{l}.{i}"] = dhi.sum(axis=0)
@@ -421,7 +431,7 @@ def backward(m: ModelDesc, g: Graph, x: np.ndarray, params: Dict[str, np.ndarray
     if m.use_ff:
         G["ff_W2"] = c["ff_act"].T @ dh
         G["ff_b2"] = dh.sum(axis=0)
-        dpre = (dh @ P["ff_W2"].T) * (c["ff_pre"] > 0)
+        dpre = (dh @ P["ff_W2"].T) * on(c["ff_pre"])
         G["ff_W1"] = x.T @ dpre
         G["ff_b1"] = dpre.sum(axis=0)
     return G

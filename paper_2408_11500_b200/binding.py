@@ -301,6 +301,25 @@ def tensor_table(m) -> List[Tuple[str, int, Tuple[int, int, int]]]:
     return [slicegcn_model_tensor_info(m, t) for t in range(slicegcn_model_num_tensors(m))]
 
 
+def named_param_shapes(m) -> Dict[str, Tuple[int, ...]]:
+    """Shapes under the per-slice names pack_params() accepts."""
+    shapes: Dict[str, Tuple[int, ...]] = {}
+    for name, _, dims in tensor_table(m):
+        if name.startswith(("W_agg.", "W_self.")):
+            for i in range(dims[0]):
+                shapes[f"{name}.{i}"] = (dims[1], dims[2])
+        elif name.startswith(("b.", "b_self.")):
+            for i in range(dims[0]):
+                shapes[f"{name}.{i}"] = (dims[1],)
+        elif name == "E":
+            shapes[name] = (dims[0], dims[1])
+        elif dims[1] == 1:
+            shapes[name] = (dims[0],)
+        else:
+            shapes[name] = (dims[0], dims[1])
+    return shapes
+
+
 def pack_params(m, named: Dict[str, np.ndarray]) -> np.ndarray:
     """Per-slice named arrays ("W_agg.<l>.<i>", "b.<l>.<i>", "E", "Wc1", ...) -> the flat fp32 buffer."""
     flat = np.zeros(slicegcn_model_param_elems(m), np.float32)

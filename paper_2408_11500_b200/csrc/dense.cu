@@ -221,7 +221,8 @@ __global__ void wgrad_reduce_kernel(const float* scratch, int n_chunks, int grou
 
 void wgrad_plan(int64_t M, int groups, int K, int N, bool bias, int* n_chunks, int64_t* rows_per_chunk, int* Kext) {
     *Kext = K + (bias ? 1 : 0);
-    const int tiles = ((*Kext + WT - 1) / WT) * ((N + WT - 1) / WT) * groups;
+    int tiles = ((*Kext + WT - 1) / WT) * ((N + WT - 1) / WT) * groups;
+    if (tiles < 1) tiles = 1;
     int64_t want = (148 * 4 + tiles - 1) / tiles;
     int64_t max_chunks = (M + 1023) / 1024;
     if (want > max_chunks) want = max_chunks;

@@ -238,16 +238,34 @@ def test_layer_forward_backward(B, torch, order, case):
 
 # ------------------------------------------------------------------------------ whole epoch
 
-def _compare_epoch(gp, od, og, X, y, params, train_idx, tol, rnd=orc.identity, orders=None):
+def _compare_epoch(gp, od, og, X, y, params, train_idx, tol, rnd=orc.identity, orders=None, relu_margin=0.0):
+    """Logits, loss and every gradient against the oracle, per tensor in max|a-b|/max|b|.
+    With relu_margin > 0 (full-size runs): of ~10^8 ReLU pre-activations a handful lie within fp32
+    rounding noise of zero, and the fp32 kernel may take their sign differently from the fp64
+    oracle.  One such unit moves a weight-gradient entry by one summand of its sum over nodes,
+    i.e. by ~1/sqrt(n) of its size, which is above 1e-4 at these sizes.  Each tensor may therefore
+    also differ by twice the largest change the oracle's own gradient shows when every borderline
+    unit is switched off versus on.  Logits, loss and the gradients above the last ReLU (Wc2, bc2)
+    do not depend on any such decision and keep the plain tolerance."""
     P = {k: v.astype(np.float64) for k, v in params.items()}
     cache = orc.forward(od, og, X, P, y, train_idx, rnd=rnd, order=orders)
     G = orc.backward(od, og, X, P, y, cache)
+    spread = None
+    if relu_margin > 0:
+        lo = orc.backward(od, og, X, P, y, cache, relu_margin=relu_margin)
+        hi = orc.backward(od, og, X, P, y, cache, relu_margin=-relu_margin)
+        spread = {k: np.abs(hi[k] - lo[k]) for k in P}
     loss = gp.epoch(None)
     errs = {"logits": rel_inf(gp.logits.cpu().numpy(), cache["logits"]), "loss": abs(loss - cache["loss"]) / abs(cache["loss"])}
+    bad = {k: v for k, v in errs.items() if not v <= tol}
     got = gp.named_grads()
     for k in P:
         errs["d" + k] = rel_inf(got[k], G[k])
-    bad = {k: v for k, v in errs.items() if not v <= tol}
+        allowed = tol
+        if spread is not None and k not in ("Wc2", "bc2"):
+            allowed += 2.0 * spread[k].max() / np.abs(G[k]).max()
+        if not errs["d" + k] <= allowed:
+            bad["d" + k] = (errs["d" + k], allowed)
     assert not bad, bad
     return errs
 
@@ -332,6 +350,9 @@ def test_citation_workload_full_size_fp32(B):
     try:
         ex = B.slicegcn_graph_export(gp.g)
         assert np.array_equal(ex["rowptr"], og.rowptr) and np.array_equal(ex["colidx"], og.colidx)
-        _compare_epoch(gp, od, og, X.astype(np.float64), y, params, None, TOL_F32)
+        errs = _compare_epoch(gp, od, og, X.astype(np.float64), y, params, None, TOL_F32, relu_margin=1e-6)
+        # most tensors are not visibly touched by a borderline unit and meet the plain 1e-4 bound
+        assert sum(v <= TOL_F32 for v in errs.values()) >= 0.75 * len(errs)
+        assert max(errs.values()) <= 1e-3
     finally:
         gp.close()
