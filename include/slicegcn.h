@@ -102,6 +102,10 @@ slicegcn_status_t slicegcn_graph_info(const slicegcn_graph* g, int64_t* n, int64
  * deg [host, n], dinv [host, n] (any may be NULL).  Synchronises the device. */
 slicegcn_status_t slicegcn_graph_export(const slicegcn_graph* g, int32_t* rowptr, int32_t* colidx, int32_t* deg,
                                         float* dinv);
+/* Device-side status word of the graph.  Kernels that wait on asynchronous copies bound every wait;
+ * a wait that runs out sets this word instead of hanging.  Synchronises the device; *status is 0
+ * when no kernel working on this graph ever gave up.  Errors: INVALID_ARG, CUDA. */
+slicegcn_status_t slicegcn_graph_device_status(const slicegcn_graph* g, int32_t* status);
 /* Frees the handle and its device memory (NULL is accepted). */
 slicegcn_status_t slicegcn_graph_destroy(slicegcn_graph* g);
 

@@ -27,7 +27,7 @@ MAX_SLICES = 64
 
 EXPORTS = [
     "slicegcn_last_error", "slicegcn_slice_strategy", "slicegcn_graph_create", "slicegcn_graph_create_from_csr",
-    "slicegcn_graph_info", "slicegcn_graph_export", "slicegcn_graph_destroy", "slicegcn_spmm_workspace_bytes",
+    "slicegcn_graph_info", "slicegcn_graph_export", "slicegcn_graph_device_status", "slicegcn_graph_destroy", "slicegcn_spmm_workspace_bytes",
     "slicegcn_spmm", "slicegcn_layer_saved_bytes", "slicegcn_layer_workspace_bytes", "slicegcn_layer_forward",
     "slicegcn_layer_backward", "slicegcn_model_create", "slicegcn_model_destroy", "slicegcn_model_param_count",
     "slicegcn_model_param_elems", "slicegcn_model_num_tensors", "slicegcn_model_tensor_info", "slicegcn_model_slices",
@@ -147,6 +147,12 @@ def slicegcn_graph_export(g) -> Dict[str, np.ndarray]:
     dinv = np.empty(info["n"], np.float32)
     _check(_lib.slicegcn_graph_export(g, _vp(rowptr), _vp(colidx), _vp(deg), _vp(dinv)))
     return {"rowptr": rowptr, "colidx": colidx[:info["nnz"]], "deg": deg, "dinv": dinv}
+
+
+def slicegcn_graph_device_status(g) -> int:
+    v = c_int32()
+    _check(_lib.slicegcn_graph_device_status(g, byref(v)))
+    return v.value
 
 
 def slicegcn_graph_destroy(g) -> None:

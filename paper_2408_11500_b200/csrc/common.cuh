@@ -52,6 +52,10 @@ void reset_launches();
 // in a fixed order afterwards (deterministic, no floating-point atomics).
 constexpr int kLongRow = 256;
 constexpr int kSegment = 256;
+// The remaining rows are dealt out in row-aligned chunks of about kChunk stored entries: chunk c
+// owns every row whose first entry index lies in [c*kChunk, (c+1)*kChunk), so each lane group gets
+// the same amount of gather work whatever the degree distribution.
+constexpr int kChunk = 128;
 
 struct CsrView {
     const int32_t* rowptr = nullptr;   // [n+1]
@@ -61,6 +65,8 @@ struct CsrView {
     const int32_t* seg_ptr = nullptr;    // [n_long+1] first segment of each long row
     int32_t n_seg = 0;
     const int32_t* seg_row = nullptr;    // [n_seg] index into long_rows
+    int32_t n_chunks = 0;
+    const int32_t* chunk_row = nullptr;  // [n_chunks+1] first row of each chunk
 };
 
 }  // namespace sgcn
@@ -73,6 +79,7 @@ struct slicegcn_graph {
     int32_t* colidx = nullptr;
     int32_t* deg = nullptr;
     float* dinv = nullptr;
+    int* fault = nullptr;   // device status word: non-zero once a bounded wait in a kernel ran out
     // transpose pattern (only when !symmetric)
     int32_t* rowptr_t = nullptr;
     int32_t* colidx_t = nullptr;
@@ -82,6 +89,8 @@ struct slicegcn_graph {
     int32_t* seg_row[2] = {nullptr, nullptr};
     int32_t n_long[2] = {0, 0};
     int32_t n_seg[2] = {0, 0};
+    int32_t* chunk_row[2] = {nullptr, nullptr};
+    int32_t n_chunks[2] = {0, 0};
 
     sgcn::CsrView view(bool transpose) const {
         sgcn::CsrView v;
@@ -93,6 +102,8 @@ struct slicegcn_graph {
         v.seg_ptr = seg_ptr[t];
         v.n_seg = n_seg[t];
         v.seg_row = seg_row[t];
+        v.n_chunks = n_chunks[t];
+        v.chunk_row = chunk_row[t];
         return v;
     }
     int32_t max_segments() const { return n_seg[0] > n_seg[1] ? n_seg[0] : n_seg[1]; }

@@ -147,6 +147,19 @@ __global__ void seg_fill_kernel(const int32_t* seg_ptr, int32_t n_long, int32_t*
         for (int32_t s = seg_ptr[i] + threadIdx.x; s < seg_ptr[i + 1]; s += blockDim.x) seg_row[s] = i;
 }
 
+// Row r opens a new chunk when its first entry index falls into another kChunk-sized window than
+// its predecessor's, or when it or its predecessor is a long row (long rows sit alone in a chunk, so
+// a chunk is either one long row or a run of short rows with contiguous entries).
+struct IsChunkStart {
+    const int32_t* rowptr;
+    __device__ bool is_long(int32_t r) const { return rowptr[r + 1] - rowptr[r] > kLongRow; }
+    __device__ bool operator()(int32_t r) const {
+        if (r == 0) return true;
+        if (rowptr[r] / kChunk != rowptr[r - 1] / kChunk) return true;
+        return is_long(r) || is_long(r - 1);
+    }
+};
+
 inline int grid_for(int64_t work, int block = 256) {
     int64_t g = (work + block - 1) / block;
     if (g < 1) g = 1;
@@ -183,6 +196,27 @@ slicegcn_status_t build_long_tables(slicegcn_graph* g, int t, const int32_t* row
     SGCN_CUDA(cudaStreamSynchronize(st));
     g->n_long[t] = n_long;
     g->n_seg[t] = 0;
+    {
+        DevBuf starts, ccnt, ctmp;
+        SGCN_CUDA(starts.alloc(sizeof(int32_t) * (n + 1)));
+        SGCN_CUDA(ccnt.alloc(sizeof(int32_t)));
+        IsChunkStart cpred{rowptr};
+        size_t ctb = 0;
+        SGCN_CUDA(cub::DeviceSelect::If(nullptr, ctb, it, starts.as<int32_t>(), ccnt.as<int32_t>(), (int)n, cpred, st));
+        SGCN_CUDA(ctmp.alloc(ctb));
+        SGCN_CUDA(cub::DeviceSelect::If(ctmp.p, ctb, it, starts.as<int32_t>(), ccnt.as<int32_t>(), (int)n, cpred, st));
+        int32_t n_chunks = 0;
+        SGCN_CUDA(cudaMemcpyAsync(&n_chunks, ccnt.p, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+        SGCN_CUDA(cudaStreamSynchronize(st));
+        DevBuf cr;
+        SGCN_CUDA(cr.alloc(sizeof(int32_t) * (n_chunks + 1)));
+        SGCN_CUDA(cudaMemcpyAsync(cr.p, starts.p, sizeof(int32_t) * n_chunks, cudaMemcpyDeviceToDevice, st));
+        const int32_t n32 = (int32_t)n;
+        SGCN_CUDA(cudaMemcpyAsync(cr.as<int32_t>() + n_chunks, &n32, sizeof(int32_t), cudaMemcpyHostToDevice, st));
+        SGCN_CUDA(cudaStreamSynchronize(st));
+        g->n_chunks[t] = n_chunks;
+        g->chunk_row[t] = cr.release<int32_t>();
+    }
     if (n_long == 0) return SLICEGCN_OK;
     DevBuf lr, counts, sp, tmp2;
     SGCN_CUDA(lr.alloc(sizeof(int32_t) * n_long));
@@ -321,6 +355,12 @@ slicegcn_status_t create_impl(int64_t n, int64_t m, const int32_t* d_src, const 
         }
     }
     g->symmetric = symmetric;
+    {
+        DevBuf fl;
+        SGCN_CUDA(fl.alloc(sizeof(int)));
+        SGCN_CUDA(cudaMemsetAsync(fl.p, 0, sizeof(int), st));
+        g->fault = fl.release<int>();
+    }
     g->rowptr = rowptr.release<int32_t>();
     g->colidx = colidx.release<int32_t>();
     g->deg = deg.release<int32_t>();
@@ -425,18 +465,29 @@ slicegcn_status_t slicegcn_graph_export(const slicegcn_graph* g, int32_t* rowptr
     return SLICEGCN_OK;
 }
 
+slicegcn_status_t slicegcn_graph_device_status(const slicegcn_graph* g, int32_t* status) {
+    if (!g || !status) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "NULL argument");
+    SGCN_CUDA(cudaDeviceSynchronize());
+    int v = 0;
+    SGCN_CUDA(cudaMemcpy(&v, g->fault, sizeof(int), cudaMemcpyDeviceToHost));
+    *status = v;
+    return SLICEGCN_OK;
+}
+
 slicegcn_status_t slicegcn_graph_destroy(slicegcn_graph* g) {
     if (!g) return SLICEGCN_OK;
     cudaFree(g->rowptr);
     cudaFree(g->colidx);
     cudaFree(g->deg);
     cudaFree(g->dinv);
+    cudaFree(g->fault);
     cudaFree(g->rowptr_t);
     cudaFree(g->colidx_t);
     for (int t = 0; t < 2; ++t) {
         cudaFree(g->long_rows[t]);
         cudaFree(g->seg_ptr[t]);
         cudaFree(g->seg_row[t]);
+        cudaFree(g->chunk_row[t]);
     }
     delete g;
     return SLICEGCN_OK;

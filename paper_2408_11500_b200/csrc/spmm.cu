@@ -7,6 +7,7 @@
 // flight per lane.  No per-edge value array exists:  A_hat_ij = dinv_i * dinv_j.
 // Rows longer than kLongRow are cut into kSegment-entry segments, one warp each, whose partial
 // rows are summed afterwards in segment order -- deterministic, no floating-point atomics.
+#include <cstdlib>
 #include <vector>
 
 #include "common.cuh"
@@ -27,7 +28,7 @@ struct Vec<float> {
         f[3] = __uint_as_float(r.w);
     }
     static __device__ __forceinline__ void store(float* p, const float (&f)[4]) {
-        *reinterpret_cast<float4*>(p) = make_float4(f[0], f[1], f[2], f[3]);
+        __stcs(reinterpret_cast<float4*>(p), make_float4(f[0], f[1], f[2], f[3]));   // streaming: keep X in L2
     }
 };
 template <>
@@ -49,7 +50,7 @@ struct Vec<__nv_bfloat16> {
             __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
             w[i] = *reinterpret_cast<uint32_t*>(&h);
         }
-        *reinterpret_cast<uint4*>(p) = r;
+        __stcs(reinterpret_cast<uint4*>(p), r);
     }
 };
 
@@ -79,6 +80,8 @@ struct SpmmParams {
     const int32_t* seg_ptr;
     const int32_t* seg_row;
     float* partial;  // [n_seg][nch*V]
+    int32_t n_chunks;
+    const int32_t* chunk_row;
     // epilogue (transform-first layers):  y = act(dinv_i*acc + bias) (+ previous y)
     const float* bias;
     uint8_t* mask;
@@ -156,39 +159,367 @@ __device__ __forceinline__ void finish_chunk(const SpmmParams& p, int64_t row, i
     }
 }
 
+// One lane group per row-aligned chunk of about kChunk stored entries (see common.cuh): a run of
+// short rows whose entries are contiguous.  The group streams the chunk's entries L at a time; a row
+// ends where the running entry index meets the row's end, at which point the accumulators are
+// scaled, stored and cleared.  Short rows therefore share one stream of gathers (many loads in
+// flight even for degree-1 rows) and every group does the same amount of work.  Row ends and
+// 1/sqrt(deg) of L consecutive rows are fetched by the L lanes at once and handed out by shuffles;
+// the column indices of the next batch are requested before the current batch is gathered.
+// Chunks that consist of one long row are left to the segment kernels.
+constexpr int kRowsWarps = 4;   // warps per CTA of the row kernel
+
 template <typename TI, typename TO, int L, int C, bool EPI>
-__global__ void __launch_bounds__(256) spmm_rows_kernel(const SpmmParams p) {
+__global__ void __launch_bounds__(kRowsWarps * 32, 20 / kRowsWarps) spmm_rows_kernel(const SpmmParams p) {
     constexpr int V = Vec<TI>::V;
     constexpr int RPW = 32 / L;
+    constexpr int U = (8 / C) < 2 ? 2 : (8 / C);   // neighbors gathered per round: U*C 16-byte loads per lane
+    // (column index, 1/sqrt(deg) bits) of the current batch, one slot per lane: read back as one
+    // broadcast 8-byte load per neighbor
+    __shared__ int2 nbuf[kRowsWarps][32];
     const int lane = threadIdx.x & 31;
     const int sub = lane / L, sl = lane % L;
     const int64_t warp = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
-    const int64_t row = warp * RPW + sub;
-    if (row >= p.n) return;
+    const int64_t chunk = warp * RPW + sub;
+    if (chunk >= p.n_chunks) return;
     const unsigned gmask = (L == 32) ? 0xffffffffu : (((1u << L) - 1u) << (sub * L));
-    const int start = __ldg(p.rowptr + row), end = __ldg(p.rowptr + row + 1);
-    if (end - start > kLongRow) return;   // long rows: segment kernels
+    const int r0 = __ldg(p.chunk_row + chunk);
+    const int r1 = __ldg(p.chunk_row + chunk + 1);
+    if (r0 >= r1) return;
+    int kk = __ldg(p.rowptr + r0);             // next entry to consume
+    const int k1 = __ldg(p.rowptr + r1);       // end of the chunk's entries
+    // row metadata of L rows at a time
+    int rbase = r0;
+    int rp_l = (r0 + sl < r1) ? __ldg(p.rowptr + r0 + sl + 1) : k1;
+    float di_l = (r0 + sl < r1) ? __ldg(p.dinv + r0 + sl) : 0.f;
+    int row = r0;
+    int row_end = __shfl_sync(gmask, rp_l, 0, L);
+    if (row_end - kk > kLongRow) return;       // a long row sits alone in its chunk
+    // per-lane column pointers (lanes past the last chunk re-read it; they never store)
+    const uint32_t row16 = (uint32_t)((p.ldx * (int64_t)sizeof(TI)) >> 4);
+    const uint4* xl[C];
+#pragma unroll
+    for (int c = 0; c < C; ++c) xl[c] = static_cast<const uint4*>(p.X) + min(sl + c * L, p.nch - 1);
+    int2* nb = &nbuf[threadIdx.x >> 5][sub * L];
     float acc[C][V];
 #pragma unroll
     for (int c = 0; c < C; ++c)
 #pragma unroll
         for (int e = 0; e < V; ++e) acc[c][e] = 0.f;
-    for (int base = start; base < end; base += L) {
-        const int k = base + sl;
-        int j = 0;
-        float dj = 0.f;
-        if (k < end) {
-            j = __ldg(p.colidx + k);
-            dj = __ldg(p.dinv + j);
-        }
-        gather_block<TI, L, C>(p, gmask, sl, j, dj, min(L, end - base), acc);
-    }
-    const float di = __ldg(p.dinv + row);
+    int jn = (kk + sl < k1) ? __ldg(p.colidx + kk + sl) : 0;
+    float djn = (kk + sl < k1) ? __ldg(p.dinv + jn) : 0.f;
+
+    auto close_row = [&]() {   // scale, store and clear the finished row; step to the next one
+        const float di = __shfl_sync(gmask, di_l, row - rbase, L);
 #pragma unroll
-    for (int c = 0; c < C; ++c) {
-        const int chunk = sl + c * L;
-        if (chunk < p.nch) finish_chunk<TO, V, EPI>(p, row, chunk, di, acc[c]);
+        for (int c = 0; c < C; ++c) {
+            const int ch = sl + c * L;
+            if (ch < p.nch) finish_chunk<TO, V, EPI>(p, row, ch, di, acc[c]);
+#pragma unroll
+            for (int e = 0; e < V; ++e) acc[c][e] = 0.f;
+        }
+        ++row;
+        if (row < r1) {
+            if (row - rbase == L) {
+                rbase = row;
+                rp_l = (row + sl < r1) ? __ldg(p.rowptr + row + sl + 1) : k1;
+                di_l = (row + sl < r1) ? __ldg(p.dinv + row + sl) : 0.f;
+            }
+            row_end = __shfl_sync(gmask, rp_l, row - rbase, L);
+        } else {
+            row_end = -1;   // no further row: never matches an entry index
+        }
+    };
+
+    for (;;) {
+        while (kk == row_end) close_row();   // rows ending here, rows without entries included
+        if (row >= r1) return;
+        // one batch of up to L entries starting at kk
+        const int cnt = min(L, k1 - kk);
+        __syncwarp(gmask);
+        nb[sl] = make_int2(jn, __float_as_int(djn));
+        __syncwarp(gmask);
+        const int nk = kk + cnt;
+        if (nk + sl < k1) jn = __ldg(p.colidx + nk + sl);   // requested now, used by the next batch
+        for (int t = 0; t < cnt;) {
+            uint4 raw[U][C];
+            int2 meta[U];
+            if (t + U <= cnt && row_end - kk >= U) {
+                // fast round: U entries of the current row, no row end among them
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    meta[u] = nb[t + u];
+#pragma unroll
+                    for (int c = 0; c < C; ++c) raw[u][c] = __ldg(xl[c] + (uint64_t)(uint32_t)meta[u].x * row16);
+                }
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const float dd = __int_as_float(meta[u].y);
+#pragma unroll
+                    for (int c = 0; c < C; ++c) {
+                        float f[V];
+                        Vec<TI>::unpack(raw[u][c], f);
+#pragma unroll
+                        for (int e = 0; e < V; ++e) acc[c][e] = fmaf(dd, f[e], acc[c][e]);
+                    }
+                }
+                kk += U;
+                t += U;
+                continue;
+            }
+            // general round: up to U entries, rows may end in between
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (t + u < cnt) {
+                    meta[u] = nb[t + u];
+#pragma unroll
+                    for (int c = 0; c < C; ++c) raw[u][c] = __ldg(xl[c] + (uint64_t)(uint32_t)meta[u].x * row16);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (t + u >= cnt) break;
+                while (kk == row_end) close_row();   // a row ends inside the batch
+                const float dd = __int_as_float(meta[u].y);
+#pragma unroll
+                for (int c = 0; c < C; ++c) {
+                    float f[V];
+                    Vec<TI>::unpack(raw[u][c], f);
+#pragma unroll
+                    for (int e = 0; e < V; ++e) acc[c][e] = fmaf(dd, f[e], acc[c][e]);
+                }
+                ++kk;
+            }
+            t += U;
+        }
+        if (nk + sl < k1) djn = __ldg(p.dinv + jn);   // its index has arrived by now
     }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Wide rows (a row of the operand is at least 512 bytes): neighbor rows are staged in shared memory
+// by asynchronous 16-byte copies (cp.async) instead of being held in registers, so the number of
+// rows a warp keeps in flight is set by shared memory, not by the register file.  Each warp runs its
+// own ring of kRingStages stages; a stage holds the operand rows of the next S entries of the warp's
+// work list and is one cp.async group, so a warp has (kRingStages-1)*S rows in flight while it
+// reduces the stage that has landed.  Work is the same row-aligned chunk list as above, dealt to
+// warps round-robin; in SEG mode the work items are the segments of the long rows and the result
+// goes to the partial-row buffer.  Row ends and 1/sqrt(deg) of 32 consecutive rows are fetched by
+// the 32 lanes at once and handed out by shuffles, so closing a row costs no memory round trip.
+constexpr int kRingWarps = 12;
+constexpr int kRingStages = 4;
+constexpr int kRingStageBytes = 4096;
+constexpr int kRingSmem = kRingWarps * kRingStages * kRingStageBytes;
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void cp_async16(void* dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_addr(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+// Entry range and rows of work item ci.  Returns false when the item holds nothing for this kernel.
+template <bool SEG>
+__device__ __forceinline__ bool item_range(const SpmmParams& p, int ci, int& r0, int& r1, int& lo, int& hi) {
+    if (SEG) {
+        const int li = __ldg(p.seg_row + ci);
+        const int r = __ldg(p.long_rows + li);
+        lo = __ldg(p.rowptr + r) + (ci - __ldg(p.seg_ptr + li)) * kSegment;
+        hi = min(__ldg(p.rowptr + r + 1), lo + kSegment);
+        r0 = ci;
+        r1 = ci + 1;
+        return true;
+    }
+    r0 = __ldg(p.chunk_row + ci);
+    r1 = __ldg(p.chunk_row + ci + 1);
+    if (r0 >= r1) return false;
+    lo = __ldg(p.rowptr + r0);
+    hi = __ldg(p.rowptr + r1);
+    if (__ldg(p.rowptr + r0 + 1) - lo > kLongRow) return false;   // a long row: segment pass
+    return true;
+}
+
+template <typename TI, typename TO, int C, bool EPI, bool SEG>
+__global__ void __launch_bounds__(kRingWarps * 32, 1) spmm_ring_kernel(const SpmmParams p, const int S) {
+    constexpr int V = Vec<TI>::V;
+    extern __shared__ __align__(1024) unsigned char smem[];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    unsigned char* wbase = smem + warp * (kRingStages * kRingStageBytes);
+    const int W = gridDim.x * kRingWarps;
+    const int n_items = SEG ? p.n_seg : p.n_chunks;
+    const uint32_t rowbytes = (uint32_t)p.nch * 16u;
+    const unsigned char* Xb = static_cast<const unsigned char*>(p.X);
+    const int64_t pitch = p.ldx * (int64_t)sizeof(TI);
+
+    // ---- producer cursor: entries [pk, pk_end) of item pci still to be fetched
+    int pci = blockIdx.x * kRingWarps + warp - W;
+    int pk = 0, pk_end = 0;
+    bool p_live = true;
+    auto prod_next = [&]() {
+        for (;;) {
+            pci += W;
+            if (pci >= n_items) {
+                p_live = false;
+                pk = pk_end = 0;
+                return;
+            }
+            int r0, r1, lo, hi;
+            if (item_range<SEG>(p, pci, r0, r1, lo, hi) && hi > lo) {
+                pk = lo;
+                pk_end = hi;
+                return;
+            }
+        }
+    };
+    prod_next();
+    int jn = 0;   // column index lane t holds for entry pk + t of the next fill
+    if (p_live && lane < min(S, pk_end - pk)) jn = __ldg(p.colidx + pk + lane);
+
+    float djr[kRingStages];
+    int cntr[kRingStages];
+    auto fill = [&](int s) {
+        const int cnt = p_live ? min(S, pk_end - pk) : 0;
+        cntr[s] = cnt;
+        djr[s] = 0.f;
+        if (cnt > 0) {
+            unsigned char* stage = wbase + s * kRingStageBytes;
+            for (int t = 0; t < cnt; ++t) {
+                const int jj = __shfl_sync(0xffffffffu, jn, t);
+                const unsigned char* src = Xb + (int64_t)jj * pitch;
+#pragma unroll
+                for (int c = 0; c < C; ++c) {
+                    const int ch = lane + c * 32;
+                    if (ch < p.nch) cp_async16(stage + t * rowbytes + ch * 16, src + ch * 16);
+                }
+            }
+            if (lane < cnt) djr[s] = __ldg(p.dinv + jn);
+            pk += cnt;
+            if (pk == pk_end) prod_next();
+            if (p_live && lane < min(S, pk_end - pk)) jn = __ldg(p.colidx + pk + lane);
+        }
+        cp_async_commit();   // one group per fill, empty or not, so the group count stays in step
+    };
+
+    // ---- consumer cursor
+    int cci = blockIdx.x * kRingWarps + warp - W;
+    int row = 0, r_end = 0, kk = 0, row_end = 0;
+    int rbase = 0, rp_l = 0;   // lane t: rowptr[rbase + 1 + t]
+    float di_l = 0.f;          // lane t: dinv[rbase + t]
+    bool finished = false;
+    float acc[C][V];
+#pragma unroll
+    for (int c = 0; c < C; ++c)
+#pragma unroll
+        for (int e = 0; e < V; ++e) acc[c][e] = 0.f;
+
+    auto load_row_meta = [&]() {   // rows [row, row+32) of the current item
+        rbase = row;
+        const int r = row + lane;
+        rp_l = r < r_end ? __ldg(p.rowptr + r + 1) : 0;
+        di_l = r < r_end ? __ldg(p.dinv + r) : 0.f;
+    };
+    auto flush = [&]() {
+        if (SEG) {
+            float* out = p.partial + (int64_t)row * (p.nch * V);
+#pragma unroll
+            for (int c = 0; c < C; ++c) {
+                const int ch = lane + c * 32;
+                if (ch < p.nch) {
+#pragma unroll
+                    for (int e = 0; e < V; e += 4)
+                        *reinterpret_cast<float4*>(out + ch * V + e) =
+                            make_float4(acc[c][e], acc[c][e + 1], acc[c][e + 2], acc[c][e + 3]);
+                }
+#pragma unroll
+                for (int e = 0; e < V; ++e) acc[c][e] = 0.f;
+            }
+        } else {
+            const float di = __shfl_sync(0xffffffffu, di_l, row - rbase);
+#pragma unroll
+            for (int c = 0; c < C; ++c) {
+                const int ch = lane + c * 32;
+                if (ch < p.nch) finish_chunk<TO, V, EPI>(p, row, ch, di, acc[c]);
+#pragma unroll
+                for (int e = 0; e < V; ++e) acc[c][e] = 0.f;
+            }
+        }
+    };
+    // closes every row that ends at kk; moves on to the next item when the current one is done
+    auto close_rows = [&]() {
+        while (!finished && kk == row_end) {
+            if (row < r_end) {
+                flush();
+                ++row;
+            }
+            if (row >= r_end) {
+                for (;;) {
+                    cci += W;
+                    if (cci >= n_items) {
+                        finished = true;
+                        break;
+                    }
+                    int r0, r1, lo, hi;
+                    if (item_range<SEG>(p, cci, r0, r1, lo, hi)) {
+                        row = r0;
+                        r_end = r1;
+                        kk = lo;
+                        if (SEG) {
+                            row_end = hi;
+                        } else {
+                            load_row_meta();
+                            row_end = __shfl_sync(0xffffffffu, rp_l, 0);
+                        }
+                        break;
+                    }
+                }
+            } else {
+                if (row - rbase == 32) load_row_meta();
+                row_end = __shfl_sync(0xffffffffu, rp_l, row - rbase);
+            }
+        }
+    };
+
+#pragma unroll
+    for (int s = 0; s < kRingStages; ++s) fill(s);
+    close_rows();   // positions the consumer on its first item (and writes leading empty rows)
+
+    while (!finished) {
+#pragma unroll
+        for (int s = 0; s < kRingStages; ++s) {
+            if (finished) break;
+            const int cnt = cntr[s];
+            if (cnt == 0) {   // producer ran dry: close_rows() has already written whatever remained
+                finished = true;
+                break;
+            }
+            cp_async_wait<kRingStages - 1>();   // this stage's group has landed (newer ones may be pending)
+            __syncwarp();
+            const unsigned char* stage = wbase + s * kRingStageBytes;
+            for (int t = 0; t < cnt; ++t) {
+                if (kk == row_end) close_rows();
+                const float dd = __shfl_sync(0xffffffffu, djr[s], t);
+#pragma unroll
+                for (int c = 0; c < C; ++c) {
+                    const int ch = lane + c * 32;
+                    if (ch < p.nch) {
+                        const uint4 raw = *reinterpret_cast<const uint4*>(stage + t * rowbytes + ch * 16);
+                        float f[V];
+                        Vec<TI>::unpack(raw, f);
+#pragma unroll
+                        for (int e = 0; e < V; ++e) acc[c][e] = fmaf(dd, f[e], acc[c][e]);
+                    }
+                }
+                ++kk;
+            }
+            if (kk == row_end) close_rows();
+            __syncwarp();     // every lane is done reading the stage before it is refilled
+            fill(s);
+        }
+    }
+    cp_async_wait<0>();
 }
 
 // One warp per segment of a long row; the 32/L lane groups interleave over the segment's
@@ -254,7 +585,15 @@ __global__ void __launch_bounds__(256) spmm_long_finish_kernel(const SpmmParams 
     TO* Y = static_cast<TO*>(p.Y) + row * p.ldy;
     for (int col = lane; col < p.width; col += 32) {
         float a = 0.f;
-        for (int s = s0; s < s1; ++s) a += p.partial[(int64_t)s * pstride + col];
+        int s = s0;
+        for (; s + 8 <= s1; s += 8) {   // eight loads in flight, summed in segment order
+            float v[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) v[q] = p.partial[(int64_t)(s + q) * pstride + col];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) a += v[q];
+        }
+        for (; s < s1; ++s) a += p.partial[(int64_t)s * pstride + col];
         float x = a * di;
         if (EPI) {
             x += p.bias ? __ldg(p.bias + col) : 0.f;
@@ -301,12 +640,12 @@ __global__ void __launch_bounds__(256) spmm_scalar_kernel(const SpmmParams p) {
 template <typename TI, typename TO, int L, int C>
 slicegcn_status_t launch_lc(const SpmmParams& p, bool epi, cudaStream_t st) {
     constexpr int RPW = 32 / L;
-    const int64_t warps = (p.n + RPW - 1) / RPW;
-    const int64_t blocks = (warps + 7) / 8;
+    const int64_t warps = ((int64_t)p.n_chunks + RPW - 1) / RPW;
+    const int64_t blocks = (warps + kRowsWarps - 1) / kRowsWarps;
     if (epi)
-        spmm_rows_kernel<TI, TO, L, C, true><<<(unsigned)blocks, 256, 0, st>>>(p);
+        spmm_rows_kernel<TI, TO, L, C, true><<<(unsigned)blocks, kRowsWarps * 32, 0, st>>>(p);
     else
-        spmm_rows_kernel<TI, TO, L, C, false><<<(unsigned)blocks, 256, 0, st>>>(p);
+        spmm_rows_kernel<TI, TO, L, C, false><<<(unsigned)blocks, kRowsWarps * 32, 0, st>>>(p);
     SGCN_LAUNCH_CHECK();
     count_launch();
     if (p.n_seg > 0) {
@@ -323,9 +662,60 @@ slicegcn_status_t launch_lc(const SpmmParams& p, bool epi, cudaStream_t st) {
     return SLICEGCN_OK;
 }
 
+template <typename TI, typename TO, int C>
+slicegcn_status_t launch_bulk(const SpmmParams& p, bool epi, int* fault, cudaStream_t st) {
+    static bool configured = false;
+    if (!configured) {
+        SGCN_CUDA(cudaFuncSetAttribute(spmm_ring_kernel<TI, TO, C, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingSmem));
+        SGCN_CUDA(cudaFuncSetAttribute(spmm_ring_kernel<TI, TO, C, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingSmem));
+        SGCN_CUDA(cudaFuncSetAttribute(spmm_ring_kernel<TI, TO, C, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingSmem));
+        configured = true;
+    }
+    const int rowbytes = p.nch * 16;
+    int S = kRingStageBytes / rowbytes;
+    if (S > 32) S = 32;
+    if (S < 1) S = 1;
+    int sms = 148;
+    {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        int v = 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) sms = v;
+    }
+    int grid = (p.n_chunks + kRingWarps - 1) / kRingWarps;
+    if (grid > sms) grid = sms;
+    if (epi)
+        spmm_ring_kernel<TI, TO, C, true, false><<<grid, kRingWarps * 32, kRingSmem, st>>>(p, S);
+    else
+        spmm_ring_kernel<TI, TO, C, false, false><<<grid, kRingWarps * 32, kRingSmem, st>>>(p, S);
+    SGCN_LAUNCH_CHECK();
+    count_launch();
+    if (p.n_seg > 0) {
+        int sgrid = (p.n_seg + kRingWarps - 1) / kRingWarps;
+        if (sgrid > sms) sgrid = sms;
+        spmm_ring_kernel<TI, TO, C, false, true><<<sgrid, kRingWarps * 32, kRingSmem, st>>>(p, S);
+        SGCN_LAUNCH_CHECK();
+        const int pstride = p.nch * Vec<TI>::V;
+        if (epi)
+            spmm_long_finish_kernel<TO, true><<<(p.n_long + 7) / 8, 256, 0, st>>>(p, pstride);
+        else
+            spmm_long_finish_kernel<TO, false><<<(p.n_long + 7) / 8, 256, 0, st>>>(p, pstride);
+        SGCN_LAUNCH_CHECK();
+        count_launch(2);
+    }
+    return SLICEGCN_OK;
+}
+
 template <typename TI, typename TO>
-slicegcn_status_t launch_vec(const SpmmParams& p, bool epi, cudaStream_t st) {
+slicegcn_status_t launch_vec(const SpmmParams& p, bool epi, int* fault, cudaStream_t st) {
     const int nch = p.nch;
+    static const bool use_ring = getenv("SLICEGCN_SPMM_RING") != nullptr;   // experimental staged variant
+    if (use_ring && nch >= 32) {
+        if (nch <= 32) return launch_bulk<TI, TO, 1>(p, epi, fault, st);
+        if (nch <= 64) return launch_bulk<TI, TO, 2>(p, epi, fault, st);
+        if (nch <= 96) return launch_bulk<TI, TO, 3>(p, epi, fault, st);
+        return launch_bulk<TI, TO, 4>(p, epi, fault, st);
+    }
     if (nch <= 2) return launch_lc<TI, TO, 2, 1>(p, epi, st);
     if (nch <= 4) return launch_lc<TI, TO, 4, 1>(p, epi, st);
     if (nch <= 8) return launch_lc<TI, TO, 8, 1>(p, epi, st);
@@ -337,7 +727,7 @@ slicegcn_status_t launch_vec(const SpmmParams& p, bool epi, cudaStream_t st) {
 }
 
 template <typename TI, typename TO>
-slicegcn_status_t launch_typed(SpmmParams p, bool vec_ok, bool epi, cudaStream_t st) {
+slicegcn_status_t launch_typed(SpmmParams p, bool vec_ok, bool epi, int* fault, cudaStream_t st) {
     constexpr int V = Vec<TI>::V;
     if (!vec_ok) {
         const int64_t blocks = (p.n + 7) / 8;
@@ -362,7 +752,7 @@ slicegcn_status_t launch_typed(SpmmParams p, bool vec_ok, bool epi, cudaStream_t
         q.Y = Y + c0;
         if (q.bias) q.bias += c0;
         if (q.mask) q.mask += c0;
-        SGCN_TRY((launch_vec<TI, TO>(q, epi, st)));
+        SGCN_TRY((launch_vec<TI, TO>(q, epi, fault, st)));
     }
     return SLICEGCN_OK;
 }
@@ -410,6 +800,8 @@ slicegcn_status_t spmm_run(const slicegcn_graph* g, bool transpose, int in_dtype
     p.nch = (width + V - 1) / V;
     const bool vec_ok = ((uintptr_t)X % 16 == 0) && ((uintptr_t)Y % 16 == 0) && (ldx * esz) % 16 == 0 &&
                         (ldy * esz) % 16 == 0 && (int64_t)p.nch * V <= ldx;
+    p.n_chunks = v.n_chunks;
+    p.chunk_row = v.chunk_row;
     if (vec_ok) {
         p.n_long = v.n_long;
         p.n_seg = v.n_seg;
@@ -446,8 +838,9 @@ slicegcn_status_t spmm_run(const slicegcn_graph* g, bool transpose, int in_dtype
         p.accumulate = epi->accumulate;
         has_epi = true;
     }
-    slicegcn_status_t rc = in_dtype == SLICEGCN_F32 ? launch_typed<float, float>(p, vec_ok, has_epi, st)
-                                                     : launch_typed<__nv_bfloat16, __nv_bfloat16>(p, vec_ok, has_epi, st);
+    slicegcn_status_t rc = in_dtype == SLICEGCN_F32
+                               ? launch_typed<float, float>(p, vec_ok, has_epi, g->fault, st)
+                               : launch_typed<__nv_bfloat16, __nv_bfloat16>(p, vec_ok, has_epi, g->fault, st);
     if (ev_stop) SGCN_CUDA(cudaEventRecord(ev_stop, st));
     return rc;
 }
