@@ -1,6 +1,9 @@
 // Dense kernels of the layer: grouped (per-slice) row-panel GEMM with the fused epilogues of
 // Eq. 6-7, grouped weight gradients with a deterministic two-stage reduction, the cross-entropy
 // of Eq. 10 and the Adam update.  This file holds the CUDA-core (FFMA) implementations.
+#include <algorithm>
+#include <cstdlib>
+
 #include "common.cuh"
 #include "kernels.cuh"
 
@@ -219,6 +222,55 @@ __global__ void wgrad_reduce_kernel(const float* scratch, int n_chunks, int grou
     }
 }
 
+// Column sums of a (masked) row-major fp32 matrix: partial sums per row chunk, then a fixed-order
+// reduction (deterministic).  Used for the bias and slice-encoding gradients.
+__global__ void __launch_bounds__(256) colsum_partial_kernel(const WgradArgs a, int total_cols, int64_t rows_per_chunk,
+                                                             float* scratch) {
+    // blockDim = (32 columns) x (8 row lanes); grid = (column blocks, row chunks)
+    __shared__ float sm[8][33];
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    const int c = blockIdx.x * 32 + tx;
+    const int64_t r0 = blockIdx.y * rows_per_chunk, r1 = min(a.M, r0 + rows_per_chunk);
+    float s = 0.f;
+    if (c < total_cols) {
+        const float* B = a.B + a.b_start[0] + c;
+        const uint8_t* bm = a.b_mask ? a.b_mask + a.b_start[0] + c : nullptr;
+        int64_t r = r0 + ty;
+        for (; r + 56 < r1; r += 64) {   // eight independent loads in flight, summed in row order
+            float v[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                v[q] = __ldg(B + (r + 8 * q) * a.ldb);
+                if (bm) v[q] = bm[(r + 8 * q) * a.b_mask_ld] ? v[q] : 0.f;
+            }
+#pragma unroll
+            for (int q = 0; q < 8; ++q) s += v[q];
+        }
+        for (; r < r1; r += 8) {
+            float v = __ldg(B + r * a.ldb);
+            if (bm) v = bm[r * a.b_mask_ld] ? v : 0.f;
+            s += v;
+        }
+    }
+    sm[ty][tx] = s;
+    __syncthreads();
+    if (ty == 0 && c < total_cols) {
+        float t = 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) t += sm[i][tx];
+        scratch[(int64_t)blockIdx.y * total_cols + c] = t;
+    }
+}
+
+__global__ void colsum_reduce_kernel(const float* scratch, int n_chunks, int total_cols, float* out1, float* out2) {
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= total_cols) return;
+    float s = 0.f;
+    for (int i = 0; i < n_chunks; ++i) s += scratch[(int64_t)i * total_cols + c];
+    if (out1) out1[c] = s;
+    if (out2) out2[c] = s;
+}
+
 void wgrad_plan(int64_t M, int groups, int K, int N, bool bias, int* n_chunks, int64_t* rows_per_chunk, int* Kext) {
     *Kext = K + (bias ? 1 : 0);
     int tiles = ((*Kext + WT - 1) / WT) * ((N + WT - 1) / WT) * groups;
@@ -304,6 +356,9 @@ __global__ void adam_kernel(int64_t count, float* theta, const float* grad, floa
 slicegcn_status_t gemm_run(const GemmArgs& a, cudaStream_t st) {
     if (a.M < 1 || a.groups < 1 || a.groups > SLICEGCN_MAX_SLICES || a.N < 1 || a.K < 0)
         SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "gemm: bad shape");
+    static const bool no_tc = getenv("SLICEGCN_NO_TC") != nullptr;   // CUDA-core kernels only (for A/B checks)
+    if (!no_tc && a.fault && a.b_image && a.K >= 1 && a.b_image_bytes >= tc_image_bytes(a.groups, a.K, a.N))
+        return tc_gemm_run(a, st);
     const bool abf = a.a_dtype == SLICEGCN_BF16, cbf = a.c_dtype == SLICEGCN_BF16;
     if (!abf && !cbf) return gemm_dispatch<float, float>(a, st);
     if (abf && cbf) return gemm_dispatch<__nv_bfloat16, __nv_bfloat16>(a, st);
@@ -312,7 +367,9 @@ slicegcn_status_t gemm_run(const GemmArgs& a, cudaStream_t st) {
 }
 
 int64_t wgrad_scratch_bytes(int64_t M, int groups, int K, int N) {
-    int64_t best = 0;
+    // the tensor-core kernel keeps one 128 x (<= 256) partial tile per (row chunk, column tile)
+    const int64_t m_tiles = std::max<int64_t>(groups, (K + 127) / 128);
+    int64_t best = (148 * 3 + m_tiles) * 128 * 256 * (int64_t)sizeof(float);
     for (int bias = 0; bias < 2; ++bias) {
         int n_chunks, Kext;
         int64_t rpc;
@@ -328,6 +385,38 @@ slicegcn_status_t wgrad_run(const WgradArgs& a, void* scratch, int64_t scratch_b
         SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "wgrad: bad shape");
     const bool bias = a.dbias || a.dbias2;
     if (a.K == 0 && !bias) return SLICEGCN_OK;
+    static const bool no_tc = getenv("SLICEGCN_NO_TC") != nullptr;
+    // bias-only request over contiguous groups: plain column sums
+    if (a.K == 0 && bias) {
+        bool contiguous = true;
+        for (int g = 0; g < a.groups; ++g) contiguous = contiguous && (a.b_start[g] == a.b_start[0] + g * a.N);
+        const int total_cols = a.groups * a.N;
+        int64_t rpc = (a.M + 147) / 148;
+        rpc = (rpc + 7) / 8 * 8;
+        const int n_chunks = (int)((a.M + rpc - 1) / rpc);
+        if (contiguous && scratch && scratch_bytes >= (int64_t)n_chunks * total_cols * (int64_t)sizeof(float)) {
+            dim3 grid((total_cols + 31) / 32, n_chunks);
+            colsum_partial_kernel<<<grid, 256, 0, st>>>(a, total_cols, rpc, static_cast<float*>(scratch));
+            SGCN_LAUNCH_CHECK();
+            colsum_reduce_kernel<<<(total_cols + 255) / 256, 256, 0, st>>>(static_cast<const float*>(scratch), n_chunks,
+                                                                           total_cols, a.dbias, a.dbias2);
+            SGCN_LAUNCH_CHECK();
+            count_launch(2);
+            return SLICEGCN_OK;
+        }
+    }
+    if (!no_tc && a.fault && a.K >= 1 && a.dW) {
+        const slicegcn_status_t rc = tc_wgrad_run(a, scratch, scratch_bytes, st);
+        if (rc == SLICEGCN_OK) {
+            if (!bias) return SLICEGCN_OK;
+            WgradArgs b = a;     // column sums only
+            b.K = 0;
+            b.dW = nullptr;
+            b.fault = nullptr;
+            return wgrad_run(b, scratch, scratch_bytes, st);
+        }
+        if (rc != SLICEGCN_ERR_UNSUPPORTED) return rc;
+    }
     int n_chunks, Kext;
     int64_t rpc;
     wgrad_plan(a.M, a.groups, a.K, a.N, bias, &n_chunks, &rpc, &Kext);

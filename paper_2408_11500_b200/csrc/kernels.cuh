@@ -52,8 +52,15 @@ struct GemmArgs {
     int64_t mul_pos_ld = 0;
     int mul_pos_dtype = SLICEGCN_F32;
     int accumulate = 0;
+    // tensor-core path: device status word (set when a bounded wait runs out) and scratch for the
+    // prepared weight image (tc_image_bytes()); without both the CUDA-core kernel runs
+    int* fault = nullptr;
+    void* b_image = nullptr;
+    int64_t b_image_bytes = 0;
 };
 slicegcn_status_t gemm_run(const GemmArgs& a, cudaStream_t st);
+slicegcn_status_t tc_gemm_run(const GemmArgs& a, cudaStream_t st);
+int64_t tc_image_bytes(int groups, int K, int N);
 
 // ---- grouped weight gradient  dW_g = A_g^T * B_g  (reduction over all rows) -------------------
 // A_g: K columns of A from a_start[g]; B_g: N columns of the fp32 matrix B from b_start[g], each
@@ -75,8 +82,11 @@ struct WgradArgs {
     float* dW = nullptr;       // may be NULL when K == 0
     float* dbias = nullptr;    // may be NULL
     float* dbias2 = nullptr;   // optional second copy of the column sums (slice-encoding gradient)
+    int* fault = nullptr;      // device status word; NULL: CUDA-core path
 };
 int64_t wgrad_scratch_bytes(int64_t M, int groups, int K, int N);
+int64_t tc_wgrad_scratch_bytes(const WgradArgs& a);
+slicegcn_status_t tc_wgrad_run(const WgradArgs& a, void* scratch, int64_t scratch_bytes, cudaStream_t st);
 slicegcn_status_t wgrad_run(const WgradArgs& a, void* scratch, int64_t scratch_bytes, cudaStream_t st);
 
 // ---- small kernels ----------------------------------------------------------------------------

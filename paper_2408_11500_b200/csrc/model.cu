@@ -111,8 +111,14 @@ slicegcn_status_t make_plan(const slicegcn_graph* g, const slicegcn_layer_desc* 
     return SLICEGCN_OK;
 }
 
+// scratch for the prepared weight images of the tensor-core GEMMs of one layer (forward and dgrad shapes)
+int64_t layer_tc_img(const LayerPlan& L) {
+    return std::max(tc_image_bytes(L.p, L.in_width, L.h_s), tc_image_bytes(L.p, L.h_s, L.in_width));
+}
+
 int64_t layer_fwd_ws_bytes(const slicegcn_graph* g, const LayerPlan& L) {
     Bump b;
+    b.take(layer_tc_img(L));
     b.take(spmm_partial_bytes(g, L.zt_cols));
     return align_up(b.off, 256);
 }
@@ -125,6 +131,7 @@ int64_t layer_wgrad_scratch(const LayerPlan& L) {
 
 int64_t layer_bwd_ws_bytes(const slicegcn_graph* g, const LayerPlan& L) {
     Bump b;
+    b.take(layer_tc_img(L));
     b.take(layer_wgrad_scratch(L));
     b.take(spmm_partial_bytes(g, L.zt_cols));
     if (L.order == SLICEGCN_AGG_FIRST) {
@@ -159,11 +166,20 @@ slicegcn_status_t layer_forward_impl(const slicegcn_graph* g, const slicegcn_lay
                                      cudaStream_t st) {
     char* zt = static_cast<char*>(saved);
     uint8_t* mask = reinterpret_cast<uint8_t*>(zt + L.zt_bytes);
+    if (ws_bytes < layer_fwd_ws_bytes(g, L)) SGCN_FAIL(SLICEGCN_ERR_ALLOC, "layer_forward: workspace too small");
+    Bump fb;
+    fb.base = static_cast<char*>(ws);
+    const int64_t img_bytes = layer_tc_img(L);
+    void* img = fb.take(img_bytes);
     const int64_t part_bytes = spmm_partial_bytes(g, L.zt_cols);
-    if (ws_bytes < part_bytes) SGCN_FAIL(SLICEGCN_ERR_ALLOC, "layer_forward: workspace too small");
+    void* part = fb.take(part_bytes);
     const bool has_post = d->W_self || d->b_self || d->E;
 
     GemmArgs self;   // H_out = H_in W_self + b_self + E
+
+    self.fault = g->fault;
+    self.b_image = img;
+    self.b_image_bytes = img_bytes;
     self.M = L.n;
     self.groups = L.p;
     self.K = d->W_self ? L.in_width : 0;
@@ -186,7 +202,7 @@ slicegcn_status_t layer_forward_impl(const slicegcn_graph* g, const slicegcn_lay
 
     if (L.order == SLICEGCN_AGG_FIRST) {
         // Z = A_hat H_in over every input column once; slices then read their column ranges of Z
-        SGCN_TRY(spmm_run(g, false, L.dtype, L.dtype, H_in, L.in_ld, zt, L.zt_ld, L.in_cols, nullptr, ws, ws_bytes, st));
+        SGCN_TRY(spmm_run(g, false, L.dtype, L.dtype, H_in, L.in_ld, zt, L.zt_ld, L.in_cols, nullptr, part, part_bytes, st));
         if (d->W_self) SGCN_TRY(gemm_run(self, st));
         GemmArgs agg = self;   // H_out = ReLU(Z W_agg + b) (+ H_out | + b_self + E)
         agg.K = L.in_width;
@@ -217,7 +233,7 @@ slicegcn_status_t layer_forward_impl(const slicegcn_graph* g, const slicegcn_lay
         epi.mask = mask;
         epi.mask_ld = L.mask_ld;
         epi.accumulate = has_post ? 1 : 0;
-        SGCN_TRY(spmm_run(g, false, L.dtype, L.dtype, zt, L.zt_ld, H_out, L.out_ld, L.out_cols, &epi, ws, ws_bytes, st));
+        SGCN_TRY(spmm_run(g, false, L.dtype, L.dtype, zt, L.zt_ld, H_out, L.out_ld, L.out_cols, &epi, part, part_bytes, st));
     }
     return SLICEGCN_OK;
 }
@@ -231,6 +247,8 @@ slicegcn_status_t layer_backward_impl(const slicegcn_graph* g, const slicegcn_la
     const uint8_t* mask = reinterpret_cast<const uint8_t*>(zt + L.zt_bytes);
     Bump b;
     b.base = static_cast<char*>(ws);
+    const int64_t img_bytes = layer_tc_img(L);
+    void* img = b.take(img_bytes);
     const int64_t wg_bytes = layer_wgrad_scratch(L);
     void* wg = b.take(wg_bytes);
     const int64_t part_bytes = spmm_partial_bytes(g, L.zt_cols);
@@ -240,6 +258,7 @@ slicegcn_status_t layer_backward_impl(const slicegcn_graph* g, const slicegcn_la
     // self branch: dW_self = H_in^T dH, db_self = dE = colsum(dH)
     if ((d->W_self && dW_self) || db_self || dE) {
         WgradArgs w;
+        w.fault = g->fault;
         w.M = L.n;
         w.groups = L.p;
         w.K = (d->W_self && dW_self) ? L.in_width : 0;
@@ -260,6 +279,10 @@ slicegcn_status_t layer_backward_impl(const slicegcn_graph* g, const slicegcn_la
     }
 
     GemmArgs dself;   // dH_in (+)= dH W_self^T
+
+    dself.fault = g->fault;
+    dself.b_image = img;
+    dself.b_image_bytes = img_bytes;
     dself.M = L.n;
     dself.groups = L.p;
     dself.K = L.h_s;
@@ -282,6 +305,7 @@ slicegcn_status_t layer_backward_impl(const slicegcn_graph* g, const slicegcn_la
     if (L.order == SLICEGCN_AGG_FIRST) {
         if (dW_agg || db) {   // dW_agg = Z^T (dH * mask), db = colsum(dH * mask)
             WgradArgs w;
+            w.fault = g->fault;
             w.M = L.n;
             w.groups = L.p;
             w.K = dW_agg ? L.in_width : 0;
@@ -327,6 +351,7 @@ slicegcn_status_t layer_backward_impl(const slicegcn_graph* g, const slicegcn_la
         SGCN_TRY(mask_mul_run(L.n, L.out_cols, dH_out, dout_ld, mask, L.mask_ld, dM, L.zt_ld, st));
         if (db) {
             WgradArgs w;
+            w.fault = g->fault;
             w.M = L.n;
             w.groups = L.p;
             w.K = 0;
@@ -343,6 +368,7 @@ slicegcn_status_t layer_backward_impl(const slicegcn_graph* g, const slicegcn_la
         }
         if (dW_agg) {
             WgradArgs w;
+            w.fault = g->fault;
             w.M = L.n;
             w.groups = L.p;
             w.K = L.in_width;
@@ -435,6 +461,8 @@ struct EpochLayout {
     float* dff = nullptr;
     void* ws = nullptr;
     int64_t ws_bytes = 0;
+    void* tc_img = nullptr;      // weight images of the dense heads' tensor-core GEMMs
+    int64_t tc_img_bytes = 0;
 };
 
 slicegcn_status_t layer_desc_for(const slicegcn_model* m, int l, const float* params, int64_t x_ld, int* starts_buf,
@@ -509,6 +537,17 @@ slicegcn_status_t build_layout(const slicegcn_model* m, const slicegcn_graph* g,
     }
     E.ws_bytes = align_up(ws_need, 256);
     E.ws = b.take(E.ws_bytes);
+    {
+        const int HW = p * m->h_s;
+        int64_t img = std::max(tc_image_bytes(1, HW, D.hidden), tc_image_bytes(1, D.hidden, HW));
+        img = std::max(img, std::max(tc_image_bytes(1, D.hidden, D.num_classes), tc_image_bytes(1, D.num_classes, D.hidden)));
+        if (D.use_ff) {
+            img = std::max(img, tc_image_bytes(1, D.in_d, D.in_d));
+            img = std::max(img, std::max(tc_image_bytes(1, D.in_d, m->slice_size), tc_image_bytes(1, m->slice_size, D.in_d)));
+        }
+        E.tc_img_bytes = align_up(img, 256);
+        E.tc_img = b.take(E.tc_img_bytes);
+    }
     E.total = align_up(b.off, 256);
     return SLICEGCN_OK;
 }
@@ -705,6 +744,9 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
     int64_t ld0 = x_ld;
     if (D.use_ff) {   // X_ff = ReLU(X W1 + b1) W2 + b2  (Eq. 4 / Algorithm 3)
         GemmArgs a;
+        a.fault = g->fault;
+        a.b_image = E.tc_img;
+        a.b_image_bytes = E.tc_img_bytes;
         a.M = n;
         a.K = D.in_d;
         a.N = D.in_d;
@@ -720,6 +762,9 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
         a.c_dtype = D.dtype;
         SGCN_TRY(gemm_run(a, st));
         GemmArgs c;
+        c.fault = g->fault;
+        c.b_image = E.tc_img;
+        c.b_image_bytes = E.tc_img_bytes;
         c.M = n;
         c.K = D.in_d;
         c.N = m->slice_size;
@@ -751,6 +796,9 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
     float* logits = logits_out ? logits_out : E.logits;
     {   // classifier (Eq. 9)
         GemmArgs a;
+        a.fault = g->fault;
+        a.b_image = E.tc_img;
+        a.b_image_bytes = E.tc_img_bytes;
         a.M = n;
         a.K = HW;
         a.N = D.hidden;
@@ -766,6 +814,9 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
         a.c_dtype = D.dtype;
         SGCN_TRY(gemm_run(a, st));
         GemmArgs c;
+        c.fault = g->fault;
+        c.b_image = E.tc_img;
+        c.b_image_bytes = E.tc_img_bytes;
         c.M = n;
         c.K = D.hidden;
         c.N = C;
@@ -786,6 +837,7 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
     // ---------------- backward
     {
         WgradArgs w;
+        w.fault = g->fault;
         w.M = n;
         w.K = D.hidden;
         w.N = C;
@@ -798,6 +850,9 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
         w.dbias = grads + m->bc2;
         SGCN_TRY(wgrad_run(w, E.ws, E.ws_bytes, st));
         GemmArgs a;   // dA = (dlogits Wc2^T) * (cls_act > 0)
+        a.fault = g->fault;
+        a.b_image = E.tc_img;
+        a.b_image_bytes = E.tc_img_bytes;
         a.M = n;
         a.K = C;
         a.N = D.hidden;
@@ -813,6 +868,7 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
         a.mul_pos_dtype = D.dtype;
         SGCN_TRY(gemm_run(a, st));
         WgradArgs w1;
+        w1.fault = g->fault;
         w1.M = n;
         w1.K = HW;
         w1.N = D.hidden;
@@ -825,6 +881,9 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
         w1.dbias = grads + m->bc1;
         SGCN_TRY(wgrad_run(w1, E.ws, E.ws_bytes, st));
         GemmArgs h;   // dH = dA Wc1^T
+        h.fault = g->fault;
+        h.b_image = E.tc_img;
+        h.b_image_bytes = E.tc_img_bytes;
         h.M = n;
         h.K = D.hidden;
         h.N = HW;
@@ -851,6 +910,7 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
     if (D.use_ff) {   // backward of the fusion MLP from dX_ff (sum over slices already formed)
         float* dxff = E.dH[cur];
         WgradArgs w;
+        w.fault = g->fault;
         w.M = n;
         w.K = D.in_d;
         w.N = m->slice_size;
@@ -864,6 +924,9 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
         SGCN_TRY(wgrad_run(w, E.ws, E.ws_bytes, st));
         float* dact = E.dH[cur ^ 1];
         GemmArgs a;
+        a.fault = g->fault;
+        a.b_image = E.tc_img;
+        a.b_image_bytes = E.tc_img_bytes;
         a.M = n;
         a.K = m->slice_size;
         a.N = D.in_d;
@@ -879,6 +942,7 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
         a.mul_pos_dtype = D.dtype;
         SGCN_TRY(gemm_run(a, st));
         WgradArgs w1;
+        w1.fault = g->fault;
         w1.M = n;
         w1.K = D.in_d;
         w1.N = D.in_d;

@@ -1,0 +1,815 @@
+// Tensor-core (tcgen05) versions of the dense kernels of the layer: the grouped row-panel GEMM with
+// the fused epilogues of Eq. 6-7 and the grouped weight gradient.
+//
+// Operands are staged in shared memory in the canonical K-major, 128-byte-swizzled layout that
+// tcgen05.mma reads through a matrix descriptor; accumulators live in tensor memory (TMEM) and come
+// back through tcgen05.ld for the epilogue.  fp32 operands use the tf32 path three times
+// (hi*hi + lo*hi + hi*lo with hi = the top 19 bits of the value, lo = value - hi), which keeps
+// ~21 mantissa bits -- single-pass tf32 (10 bits) would miss the 1e-4 parity bound.  bf16 operands use
+// one kind::f16 pass.  The hi/lo split needs a pass through registers anyway, so tiles are written
+// to shared memory with ordinary stores (swizzled by hand) followed by a proxy fence.
+// Every wait on an mbarrier is bounded; a wait that runs out sets the caller's status word.
+#include "common.cuh"
+#include "kernels.cuh"
+
+namespace sgcn {
+namespace {
+
+constexpr int kWaitSpins = 1 << 22;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+    for (int i = 0; i < kWaitSpins; ++i)
+        if (mbar_test(bar, parity)) return true;
+    return false;
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(ncols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void proxy_fence() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// D[tmem] (+)= A[smem desc] * B[smem desc]
+template <bool BF16>
+__device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    if (BF16) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+            "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+            "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    }
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// contiguous global -> shared copy by the bulk-copy engine; completion is counted on the mbarrier
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_u32(dst)),
+                 "l"(src), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// 32 lanes x 32 columns of fp32: thread t of the warp receives row (lane base + t), columns col..col+31
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+          "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+          "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+          "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// K-major, 128-byte swizzle: rows of 128 bytes, 8-row groups 1024 bytes apart
+__device__ __forceinline__ uint64_t smem_desc(const void* tile) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_u32(tile) >> 4) & 0x3FFF);   // start address
+    d |= (uint64_t)1 << 16;                            // leading byte offset (unused with swizzle): 1
+    d |= (uint64_t)(1024 >> 4) << 32;                  // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;                            // descriptor version
+    d |= (uint64_t)2 << 61;                            // SWIZZLE_128B
+    return d;
+}
+// byte offset of 4-byte element (row, k) [k < 32] or 2-byte element [k < 64] inside a swizzled tile
+__device__ __forceinline__ uint32_t sw_off(int row, int byte_in_row) {
+    const int chunk = (byte_in_row >> 4) ^ (row & 7);
+    return (uint32_t)(row * 128 + (chunk << 4) + (byte_in_row & 15));
+}
+__device__ __forceinline__ uint32_t idesc_f32acc(int M, int N, bool bf16) {
+    const uint32_t fmt = bf16 ? 1u : 2u;   // BF16 : TF32
+    return (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+__device__ __forceinline__ float ld_as_f(const float* p) { return __ldg(p); }
+__device__ __forceinline__ float ld_as_f(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+
+// nearest value with a 10-bit mantissa (what the tf32 path keeps); Inf/NaN pass through
+__device__ __forceinline__ float tf32_hi(float v) {
+    const uint32_t b = __float_as_uint(v);
+    if ((b & 0x7F800000u) == 0x7F800000u) return v;
+    return __uint_as_float((b + 0x1000u) & 0xFFFFE000u);
+}
+// stores one fp32 operand value into the hi / lo tiles (tf32 split) or one bf16 value
+__device__ __forceinline__ void put_f32(unsigned char* hi, unsigned char* lo, int row, int k, float v) {
+    const float h = tf32_hi(v);
+    const uint32_t off = sw_off(row, k * 4);
+    *reinterpret_cast<float*>(hi + off) = h;
+    *reinterpret_cast<float*>(lo + off) = v - h;
+}
+__device__ __forceinline__ void put_bf16(unsigned char* t, int row, int k, float v) {
+    *reinterpret_cast<__nv_bfloat16*>(t + sw_off(row, k * 2)) = __float2bfloat16_rn(v);
+}
+// fp32 weight as two bf16 values (hi + lo keeps ~16 mantissa bits); the activation operand is exact in bf16
+__device__ __forceinline__ void put_bf16x2(unsigned char* hi, unsigned char* lo, int row, int k, float v) {
+    const __nv_bfloat16 h = __float2bfloat16_rn(v);
+    const uint32_t off = sw_off(row, k * 2);
+    *reinterpret_cast<__nv_bfloat16*>(hi + off) = h;
+    *reinterpret_cast<__nv_bfloat16*>(lo + off) = __float2bfloat16_rn(v - __bfloat162float(h));
+}
+
+// ------------------------------------------------------------------------------ weight images
+// The B operand (a small weight block) is the same for every row tile, so it is converted once per
+// GEMM into the exact bytes a shared-memory tile holds -- K-major rows of 128 bytes, swizzled, split
+// into hi and lo -- and every CTA then pulls a slab's image with one bulk copy.
+// Image of (group g, n tile nt, K slab s): [hi: n_pad rows x 128 B][lo: n_pad rows x 128 B].
+template <bool BF16>
+__global__ void __launch_bounds__(128) tc_prep_b_kernel(const GemmArgs a, const int n_pad, unsigned char* image) {
+    constexpr int KS = BF16 ? 64 : 32;
+    const int s = blockIdx.x, nt = blockIdx.y, g = blockIdx.z;
+    const int n_slabs = gridDim.x, n_tiles = gridDim.y;
+    const float* B = a.B + (int64_t)g * a.b_gstride;
+    unsigned char* hi = image + ((((int64_t)g * n_tiles + nt) * n_slabs + s) * 2) * ((int64_t)n_pad * 128);
+    unsigned char* lo = hi + (int64_t)n_pad * 128;
+    const int n0 = nt * n_pad, k0 = s * KS;
+    for (int e = threadIdx.x; e < n_pad * KS; e += 128) {
+        int n, kk;
+        if (a.b_trans) {
+            kk = e % KS;
+            n = e / KS;
+        } else {
+            n = e % n_pad;
+            kk = e / n_pad;
+        }
+        const int k = k0 + kk, col = n0 + n;
+        float v = 0.f;
+        if (col < a.N && k < a.K) v = a.b_trans ? __ldg(B + (int64_t)col * a.ldb + k) : __ldg(B + (int64_t)k * a.ldb + col);
+        if (BF16)
+            put_bf16x2(hi, lo, n, kk, v);
+        else
+            put_f32(hi, lo, n, kk, v);
+    }
+}
+
+// ------------------------------------------------------------------------------ row-panel GEMM
+// Persistent CTAs (128 threads) walk work items (128-row tile, n tile of up to 256 columns, group).
+// K is walked in slabs of one swizzle row (32 fp32 / 64 bf16 values).  Per slab: the weight image
+// arrives by bulk copy into one of two buffers; the activation slab, fetched into registers one step
+// ahead, is split and stored to shared memory; one elected thread issues the MMAs.  The global loads
+// of the next slab (or next item) are in flight while the MMAs run and while the finished item's
+// accumulators go TMEM -> registers -> per-warp staging tile -> global memory in whole 128-byte rows.
+constexpr int kTcThreads = 128;
+constexpr int kStagePitch = 33;   // floats per staged row (odd: conflict-free both ways)
+
+template <typename TA, typename TC, bool BF16, bool VEC>
+__global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const GemmArgs a, const int n_pad, const int n_tiles,
+                                                             const unsigned char* image, int* fault) {
+    extern __shared__ __align__(1024) unsigned char smem[];
+    constexpr int KS = BF16 ? 64 : 32;          // K values per slab
+    constexpr int UK = BF16 ? 16 : 8;           // K values per MMA
+    constexpr int EPC = BF16 ? 8 : 4;           // elements per 16-byte chunk
+    constexpr int NLD = VEC ? 8 : (BF16 ? 64 : 32);   // register slots of the prefetched slab
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    // the swizzled tiles need 1024-byte alignment; the launch reserves the slack
+    unsigned char* base = smem + ((1024u - (smem_u32(smem) & 1023u)) & 1023u);
+    unsigned char* A_hi = base;
+    unsigned char* A_lo = base + 16384;
+    unsigned char* Bbuf = base + (BF16 ? 16384 : 32768);           // two buffers of [hi | lo]
+    const uint32_t slab_bytes = 2u * (uint32_t)n_pad * 128u;
+    float* stage = reinterpret_cast<float*>(Bbuf + 2 * slab_bytes) + warp * (32 * kStagePitch);
+    unsigned char* tail = Bbuf + 2 * slab_bytes + 4 * 32 * kStagePitch * 4;
+    uint64_t* mbar_mma = reinterpret_cast<uint64_t*>(tail);
+    uint64_t* mbar_b = reinterpret_cast<uint64_t*>(tail + 8);      // [2]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 24);
+    const int n_mma_max = n_pad;
+    uint32_t ncols = 32;
+    while ((int)ncols < n_mma_max) ncols <<= 1;
+    if (tid == 0) {
+        mbar_init(mbar_mma, 1);
+        mbar_init(&mbar_b[0], 1);
+        mbar_init(&mbar_b[1], 1);
+    }
+    if (warp == 0) tmem_alloc(tmem_slot, ncols);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    const int n_slabs = (a.K + KS - 1) / KS;
+    const int64_t row_tiles = (a.M + 127) / 128;
+    const int64_t n_items = row_tiles * a.groups * n_tiles;
+    // item -> (row tile, group, n tile): groups and n tiles of one row tile are adjacent
+    auto decode = [&](int64_t item, int64_t& row0, int& g, int& nt) {
+        nt = (int)(item % n_tiles);
+        g = (int)((item / n_tiles) % a.groups);
+        row0 = (item / ((int64_t)n_tiles * a.groups)) * 128;
+    };
+    // prefetch of one activation slab into registers
+    uint4 pre[VEC ? 8 : 1];
+    float pres[VEC ? 1 : NLD];
+    auto prefetch = [&](int64_t row0, int g, int s) {
+        const TA* A = static_cast<const TA*>(a.A) + a.a_start[g];
+        const uint8_t* am = a.a_mask ? a.a_mask + a.a_start[g] : nullptr;
+        const int k0 = s * KS;
+        if (VEC) {
+            const int c = tid & 7;
+            const int k = k0 + c * EPC;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int64_t row = row0 + (tid >> 3) + 16 * i;
+                uint4 raw = make_uint4(0, 0, 0, 0);
+                if (row < a.M && k < a.K) {
+                    raw = __ldg(reinterpret_cast<const uint4*>(A + row * a.lda + k));
+                    if (am) {
+                        if (BF16) {
+                            const uint2 m8 = *reinterpret_cast<const uint2*>(am + row * a.a_mask_ld + k);
+                            uint32_t* w = reinterpret_cast<uint32_t*>(&raw);
+                            const uint32_t mm[2] = {m8.x, m8.y};
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                const uint32_t b0 = (mm[q >> 1] >> (16 * (q & 1))) & 0xFFu;
+                                const uint32_t b1 = (mm[q >> 1] >> (16 * (q & 1) + 8)) & 0xFFu;
+                                w[q] &= (b0 ? 0x0000FFFFu : 0u) | (b1 ? 0xFFFF0000u : 0u);
+                            }
+                        } else {
+                            const uint32_t m4 = *reinterpret_cast<const uint32_t*>(am + row * a.a_mask_ld + k);
+                            if (!(m4 & 0x000000FFu)) raw.x = 0;
+                            if (!(m4 & 0x0000FF00u)) raw.y = 0;
+                            if (!(m4 & 0x00FF0000u)) raw.z = 0;
+                            if (!(m4 & 0xFF000000u)) raw.w = 0;
+                        }
+                    }
+                }
+                pre[i] = raw;
+            }
+        } else {
+            // any alignment: warp w takes rows w, w+4, ...; a warp reads one row's KS values
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const int64_t row = row0 + warp + 4 * i;
+#pragma unroll
+                for (int q = 0; q < KS / 32; ++q) {
+                    const int k = k0 + lane + 32 * q;
+                    float v = 0.f;
+                    if (row < a.M && k < a.K) {
+                        v = ld_as_f(A + row * a.lda + k);
+                        if (am) v = am[row * a.a_mask_ld + k] ? v : 0.f;
+                    }
+                    pres[i * (KS / 32) + q] = v;
+                }
+            }
+        }
+    };
+    auto store_slab = [&]() {
+        if (VEC) {
+            const int c = tid & 7;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int r = (tid >> 3) + 16 * i;
+                const uint32_t off = sw_off(r, c * 16);
+                if (BF16) {
+                    *reinterpret_cast<uint4*>(A_hi + off) = pre[i];
+                } else {
+                    const float v0 = __uint_as_float(pre[i].x), v1 = __uint_as_float(pre[i].y);
+                    const float v2 = __uint_as_float(pre[i].z), v3 = __uint_as_float(pre[i].w);
+                    const float h0 = tf32_hi(v0), h1 = tf32_hi(v1), h2 = tf32_hi(v2), h3 = tf32_hi(v3);
+                    *reinterpret_cast<float4*>(A_hi + off) = make_float4(h0, h1, h2, h3);
+                    *reinterpret_cast<float4*>(A_lo + off) = make_float4(v0 - h0, v1 - h1, v2 - h2, v3 - h3);
+                }
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+#pragma unroll
+                for (int q = 0; q < KS / 32; ++q) {
+                    const float v = pres[i * (KS / 32) + q];
+                    if (BF16)
+                        put_bf16(A_hi, warp + 4 * i, lane + 32 * q, v);
+                    else
+                        put_f32(A_hi, A_lo, warp + 4 * i, lane + 32 * q, v);
+                }
+            }
+        }
+    };
+    auto image_of = [&](int g, int nt, int s) {
+        return image + ((((int64_t)g * n_tiles + nt) * n_slabs + s)) * (int64_t)slab_bytes;
+    };
+
+    uint32_t mma_phase = 0, b_phase = 0;   // b_phase: bit i = parity of weight buffer i
+    bool ok = true;
+    int64_t item = blockIdx.x;
+    int64_t row0 = 0;
+    int g = 0, nt = 0;
+    int bsel = 0;   // weight buffer of the slab about to run
+    if (item < n_items) {
+        decode(item, row0, g, nt);
+        if (tid == 0) {
+            mbar_expect_tx(&mbar_b[0], slab_bytes);
+            bulk_g2s(Bbuf, image_of(g, nt, 0), slab_bytes, &mbar_b[0]);
+        }
+        prefetch(row0, g, 0);
+    }
+    while (item < n_items && ok) {
+        const int n0 = nt * n_pad;
+        const int nn = min(n_pad, a.N - n0);
+        const int n_mma = (nn + 15) & ~15;
+        const uint32_t idesc = idesc_f32acc(128, n_mma, BF16);
+        // the item after this one (its first slab is prefetched during this item's last slab)
+        const int64_t nitem = item + gridDim.x;
+        int64_t nrow0 = 0;
+        int ng = 0, nnt = 0;
+        if (nitem < n_items) decode(nitem, nrow0, ng, nnt);
+        for (int s = 0; s < n_slabs && ok; ++s) {
+            store_slab();
+            proxy_fence();          // generic-proxy stores -> visible to the tensor core's async proxy
+            tc_fence_before();
+            __syncthreads();
+            if (tid == 0) {
+                if (mbar_wait(&mbar_b[bsel], (b_phase >> bsel) & 1u)) {
+                    tc_fence_after();
+                    unsigned char* B_hi = Bbuf + bsel * slab_bytes;
+                    const uint64_t da_hi = smem_desc(A_hi), da_lo = smem_desc(A_lo);
+                    const uint64_t db_hi = smem_desc(B_hi), db_lo = smem_desc(B_hi + n_pad * 128);
+#pragma unroll
+                    for (int ks = 0; ks < KS / UK; ++ks) {
+                        const uint64_t adv = (uint64_t)((ks * 32) >> 4);   // 32 bytes per MMA along K
+                        const uint32_t first = (s == 0 && ks == 0) ? 0u : 1u;
+                        umma<BF16>(tmem, da_hi + adv, db_hi + adv, idesc, first);
+                        if (!BF16) umma<BF16>(tmem, da_lo + adv, db_hi + adv, idesc, 1u);
+                        umma<BF16>(tmem, da_hi + adv, db_lo + adv, idesc, 1u);
+                    }
+                } else {
+                    atomicExch(fault, 3);
+                }
+                umma_commit(mbar_mma);   // arrives when the MMAs above have read smem and written TMEM
+                // weight image of the next slab into the other buffer (its last reader finished before
+                // this slab's stores began)
+                const bool more = (s + 1 < n_slabs) || (nitem < n_items);
+                if (more) {
+                    const unsigned char* src = (s + 1 < n_slabs) ? image_of(g, nt, s + 1) : image_of(ng, nnt, 0);
+                    mbar_expect_tx(&mbar_b[bsel ^ 1], slab_bytes);
+                    bulk_g2s(Bbuf + (bsel ^ 1) * slab_bytes, src, slab_bytes, &mbar_b[bsel ^ 1]);
+                }
+            }
+            b_phase ^= (1u << bsel);
+            bsel ^= 1;
+            // global loads of the next slab fly while the MMAs run
+            if (s + 1 < n_slabs)
+                prefetch(row0, g, s + 1);
+            else if (nitem < n_items)
+                prefetch(nrow0, ng, 0);
+            ok = mbar_wait(mbar_mma, mma_phase);
+            mma_phase ^= 1u;
+            tc_fence_after();
+        }
+        if (!ok) break;
+        // epilogue: warp w owns TMEM lanes 32w..32w+31 = rows row0+32w..; staged so that every global
+        // access is one whole row segment (32 consecutive columns)
+        TC* C = static_cast<TC*>(a.C);
+        const int cs = a.c_start[g] + n0;
+        for (int c0 = 0; c0 < n_mma; c0 += 32) {
+            float v[32];
+            tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) stage[lane * kStagePitch + j] = v[j];
+            __syncwarp();
+            const int n = c0 + lane;          // this lane's column within the tile
+            const bool col_ok = n < nn;
+            const int col = cs + n;
+            float bias = 0.f, post = 0.f;
+            if (col_ok) {
+                if (a.bias) bias = __ldg(a.bias + g * a.N + n0 + n);
+                if (a.post1) post += __ldg(a.post1 + g * a.N + n0 + n);
+                if (a.post2) post += __ldg(a.post2 + g * a.N + n0 + n);
+            }
+            // operands the epilogue reads back (previous C, ReLU gate): all 32 rows requested up front
+            float cold[32], gate[32];
+            if (a.accumulate) {
+#pragma unroll
+                for (int r = 0; r < 32; ++r) {
+                    const int64_t row = row0 + warp * 32 + r;
+                    cold[r] = (row < a.M && col_ok) ? ld_as_f(C + row * a.ldc + col) : 0.f;
+                }
+            }
+            if (a.mul_pos) {
+#pragma unroll
+                for (int r = 0; r < 32; ++r) {
+                    const int64_t row = row0 + warp * 32 + r;
+                    float pv = 1.f;
+                    if (row < a.M && col_ok)
+                        pv = a.mul_pos_dtype == SLICEGCN_F32
+                                 ? __ldg(static_cast<const float*>(a.mul_pos) + row * a.mul_pos_ld + col)
+                                 : __bfloat162float(static_cast<const __nv_bfloat16*>(a.mul_pos)[row * a.mul_pos_ld + col]);
+                    gate[r] = pv;
+                }
+            }
+#pragma unroll
+            for (int r = 0; r < 32; ++r) {
+                const int64_t row = row0 + warp * 32 + r;
+                if (row >= a.M || !col_ok) continue;
+                float x = stage[r * kStagePitch + lane] + bias;
+                if (a.relu) {
+                    if (a.mask_out) a.mask_out[row * a.mask_ld + col] = x > 0.f ? 1 : 0;
+                    x = fmaxf(x, 0.f);
+                }
+                x += post;
+                if (a.mul_pos) x = gate[r] > 0.f ? x : 0.f;
+                if (a.accumulate) x += cold[r];
+                if (sizeof(TC) == 4)
+                    reinterpret_cast<float*>(C)[row * a.ldc + col] = x;
+                else
+                    reinterpret_cast<__nv_bfloat16*>(C)[row * a.ldc + col] = __float2bfloat16_rn(x);
+            }
+            __syncwarp();
+        }
+        tc_fence_before();   // TMEM reads done before the next item's first MMA overwrites the accumulator
+        item = nitem;
+        row0 = nrow0;
+        g = ng;
+        nt = nnt;
+    }
+    if (!ok && tid == 0) atomicExch(fault, 3);
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, ncols);
+}
+
+int tc_n_pad(int N) { return N <= 256 ? ((N + 15) & ~15) : 256; }
+
+template <typename TA, typename TC, bool BF16>
+slicegcn_status_t tc_gemm_launch(const GemmArgs& a, void* image, int64_t image_bytes, int* fault, cudaStream_t st) {
+    constexpr int KS = BF16 ? 64 : 32;
+    constexpr int EPC = BF16 ? 8 : 4;
+    const int n_pad = tc_n_pad(a.N);
+    const int n_tiles = (a.N + n_pad - 1) / n_pad;
+    const int n_slabs = (a.K + KS - 1) / KS;
+    const int64_t need = (int64_t)a.groups * n_tiles * n_slabs * 2 * n_pad * 128;
+    if (!image || image_bytes < need) SGCN_FAIL(SLICEGCN_ERR_ALLOC, "tc_gemm: weight image scratch too small");
+    const int smem_bytes = (BF16 ? 16384 : 32768) + 4 * n_pad * 128 + 4 * 32 * kStagePitch * 4 + 64 + 1024;
+    static bool configured = false;
+    if (!configured) {
+        const int mx = 32768 + 4 * 256 * 128 + 4 * 32 * kStagePitch * 4 + 64 + 1024;
+        SGCN_CUDA(cudaFuncSetAttribute(tc_gemm_kernel<TA, TC, BF16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, mx));
+        SGCN_CUDA(cudaFuncSetAttribute(tc_gemm_kernel<TA, TC, BF16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, mx));
+        configured = true;
+    }
+    dim3 pgrid(n_slabs, n_tiles, a.groups);
+    tc_prep_b_kernel<BF16><<<pgrid, 128, 0, st>>>(a, n_pad, static_cast<unsigned char*>(image));
+    SGCN_LAUNCH_CHECK();
+    // 16-byte loads of the activation need aligned slices
+    bool vec = ((uintptr_t)a.A % 16 == 0) && (a.lda % EPC == 0) && (a.K % EPC == 0);
+    for (int g = 0; g < a.groups; ++g) vec = vec && (a.a_start[g] % EPC == 0);
+    if (a.a_mask) vec = vec && ((uintptr_t)a.a_mask % 8 == 0) && (a.a_mask_ld % 8 == 0);
+    // persistent grid: as many CTAs as fit at once (shared memory and 512 TMEM columns per SM)
+    int ncols = 32;
+    while (ncols < n_pad) ncols <<= 1;
+    int per_sm = (227 * 1024) / (smem_bytes + 1024);
+    if (per_sm > 512 / ncols) per_sm = 512 / ncols;
+    if (per_sm > 8) per_sm = 8;
+    if (per_sm < 1) per_sm = 1;
+    const int64_t n_items = ((a.M + 127) / 128) * a.groups * n_tiles;
+    int64_t grid = (int64_t)148 * per_sm;
+    if (grid > n_items) grid = n_items;
+    if (vec)
+        tc_gemm_kernel<TA, TC, BF16, true><<<(unsigned)grid, kTcThreads, smem_bytes, st>>>(a, n_pad, n_tiles, static_cast<unsigned char*>(image), fault);
+    else
+        tc_gemm_kernel<TA, TC, BF16, false><<<(unsigned)grid, kTcThreads, smem_bytes, st>>>(a, n_pad, n_tiles, static_cast<unsigned char*>(image), fault);
+    SGCN_LAUNCH_CHECK();
+    count_launch(2);
+    return SLICEGCN_OK;
+}
+
+// ------------------------------------------------------------------------------ weight gradient
+// dW = A^T B with the reduction running over the rows (nodes).  One CTA owns a 128-wide tile of A's
+// columns (the MMA's M), the matching columns of B (the MMA's N: for grouped layers only the groups
+// of that tile, so the block-diagonal structure is not wasted twice) and a chunk of rows.  Every 32
+// rows form one K slab: both operands are read with 16-byte loads, transposed in registers (4x4
+// micro-tiles) and stored K-major; the next slab's loads are in flight while the current slab's MMAs
+// run (two shared-memory stages).  The CTA's partial product leaves TMEM once, at the end, into the
+// scratch buffer; a second kernel sums the chunks in a fixed order.
+constexpr int kWgThreads = 256;
+
+struct WgTcPlan {
+    int m_tiles;        // tiles of 128 A-columns
+    int n_t;            // B columns per tile (MMA N, multiple of 16)
+    int n_valid;        // valid B columns per tile
+    int a_col0, b_col0; // first column of A / B
+    int a_cols;         // total A columns (all groups)
+    int b_cols_per_tile;
+    int n_chunks;
+    int64_t rows_per_chunk;
+    int stages;
+};
+
+template <typename TA, int STAGES>
+__global__ void __launch_bounds__(kWgThreads, STAGES == 1 ? 2 : 1) tc_wgrad_kernel(const WgradArgs a, const WgTcPlan pl,
+                                                                                    float* scratch, int* fault) {
+    extern __shared__ __align__(1024) unsigned char smem[];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int mt = blockIdx.y, chunk = blockIdx.x;
+    unsigned char* base = smem + ((1024u - (smem_u32(smem) & 1023u)) & 1023u);
+    const uint32_t a_bytes = 16384, b_bytes = (uint32_t)pl.n_t * 128u;
+    const uint32_t stage_bytes = 2 * a_bytes + 2 * b_bytes;
+    unsigned char* tail = base + STAGES * stage_bytes;
+    uint64_t* mbar_done = reinterpret_cast<uint64_t*>(tail);   // [2]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 16);
+    uint32_t ncols = 32;
+    while ((int)ncols < pl.n_t) ncols <<= 1;
+    if (tid == 0) {
+        mbar_init(&mbar_done[0], 1);
+        mbar_init(&mbar_done[1], 1);
+    }
+    if (warp == 0) tmem_alloc(tmem_slot, ncols);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    const int64_t r_begin = (int64_t)chunk * pl.rows_per_chunk;
+    const int64_t r_end = min(a.M, r_begin + pl.rows_per_chunk);
+    const int n_slabs = (int)((r_end - r_begin + 31) / 32);
+    // this thread's 4x4 micro-tiles: rows 4*rq .. 4*rq+3 of the slab, column quad cq of the operand
+    const int rq = lane & 7;
+    const int a_cq = warp * 4 + (lane >> 3);                 // 32 column quads of A (128 columns)
+    const int a_col = mt * 128 + a_cq * 4;                   // column inside A's range
+    const bool a_ok = a_col < pl.a_cols;
+    const TA* Ap = static_cast<const TA*>(a.A) + pl.a_col0 + a_col;
+    const int b_quads = pl.n_t / 4;                          // column quads of B in this tile (<= 64)
+    const float* Bp = a.B + pl.b_col0 + mt * pl.b_cols_per_tile;
+    const uint8_t* Mp = a.b_mask ? a.b_mask + pl.b_col0 + mt * pl.b_cols_per_tile : nullptr;
+
+    float4 ra[4];
+    float4 rb[2][4];
+    auto load = [&](int s) {
+        const int64_t rr = r_begin + (int64_t)s * 32 + rq * 4;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int64_t row = rr + i;
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (a_ok && row < r_end) {
+                if (sizeof(TA) == 4) {
+                    v = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(Ap) + row * a.lda));
+                } else {
+                    const uint2 h = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(Ap) + row * a.lda));
+                    v = make_float4(__uint_as_float(h.x << 16), __uint_as_float(h.x & 0xffff0000u),
+                                    __uint_as_float(h.y << 16), __uint_as_float(h.y & 0xffff0000u));
+                }
+            }
+            ra[i] = v;
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                const int cq = warp * 4 + (lane >> 3) + 32 * j;
+                float4 w = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (cq < b_quads && cq * 4 < pl.n_valid && row < r_end) {
+                    w = __ldg(reinterpret_cast<const float4*>(Bp + row * a.ldb + cq * 4));
+                    if (Mp) {
+                        const uint32_t m4 = *reinterpret_cast<const uint32_t*>(Mp + row * a.b_mask_ld + cq * 4);
+                        if (!(m4 & 0x000000FFu)) w.x = 0.f;
+                        if (!(m4 & 0x0000FF00u)) w.y = 0.f;
+                        if (!(m4 & 0x00FF0000u)) w.z = 0.f;
+                        if (!(m4 & 0xFF000000u)) w.w = 0.f;
+                    }
+                }
+                rb[j][i] = w;
+            }
+        }
+    };
+    // element (column c of the quad, rows 4*rq..+3) -> tile row (quad*4 + c), 16-byte chunk rq
+    auto put_quad = [&](unsigned char* hi, unsigned char* lo, int quad, const float4 (&r)[4]) {
+        const float e[4][4] = {{r[0].x, r[1].x, r[2].x, r[3].x},
+                               {r[0].y, r[1].y, r[2].y, r[3].y},
+                               {r[0].z, r[1].z, r[2].z, r[3].z},
+                               {r[0].w, r[1].w, r[2].w, r[3].w}};
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const uint32_t off = sw_off(quad * 4 + c, rq * 16);
+            const float h0 = tf32_hi(e[c][0]), h1 = tf32_hi(e[c][1]), h2 = tf32_hi(e[c][2]), h3 = tf32_hi(e[c][3]);
+            *reinterpret_cast<float4*>(hi + off) = make_float4(h0, h1, h2, h3);
+            *reinterpret_cast<float4*>(lo + off) = make_float4(e[c][0] - h0, e[c][1] - h1, e[c][2] - h2, e[c][3] - h3);
+        }
+    };
+    const uint32_t idesc = idesc_f32acc(128, pl.n_t, false);
+    uint32_t done_phase = 0;   // bit i: parity to wait for on mbar_done[i]
+    int pending[2] = {0, 0};   // commits on each stage not yet waited for
+    bool ok = true;
+    if (n_slabs > 0) load(0);
+    for (int s = 0; s < n_slabs && ok; ++s) {
+        const int st = STAGES == 1 ? 0 : (s & 1);
+        unsigned char* A_hi = base + st * stage_bytes;
+        unsigned char* A_lo = A_hi + a_bytes;
+        unsigned char* B_hi = A_lo + a_bytes;
+        unsigned char* B_lo = B_hi + b_bytes;
+        if (pending[st]) {   // the MMAs of slab s-2 must have finished reading this stage
+            ok = mbar_wait(&mbar_done[st], (done_phase >> st) & 1u);
+            done_phase ^= (1u << st);
+            pending[st] = 0;
+            if (!ok) break;
+        }
+        put_quad(A_hi, A_lo, a_cq, ra);
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const int cq = warp * 4 + (lane >> 3) + 32 * j;
+            if (cq < b_quads) put_quad(B_hi, B_lo, cq, rb[j]);
+        }
+        if (s + 1 < n_slabs) load(s + 1);   // in flight while this slab's MMAs run
+        proxy_fence();
+        tc_fence_before();
+        __syncthreads();
+        if (tid == 0) {
+            tc_fence_after();
+            const uint64_t da_hi = smem_desc(A_hi), da_lo = smem_desc(A_lo);
+            const uint64_t db_hi = smem_desc(B_hi), db_lo = smem_desc(B_lo);
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {
+                const uint64_t adv = (uint64_t)((ks * 32) >> 4);
+                umma<false>(tmem, da_hi + adv, db_hi + adv, idesc, (s == 0 && ks == 0) ? 0u : 1u);
+                if (sizeof(TA) == 4) umma<false>(tmem, da_lo + adv, db_hi + adv, idesc, 1u);   // bf16 values have no lo part
+                umma<false>(tmem, da_hi + adv, db_lo + adv, idesc, 1u);
+            }
+            umma_commit(&mbar_done[st]);
+        }
+        pending[st] = 1;
+    }
+    // drain the commits still outstanding (at most one per stage)
+    for (int st = 0; st < 2; ++st)
+        if (ok && pending[st]) ok = mbar_wait(&mbar_done[st], (done_phase >> st) & 1u);
+    tc_fence_after();
+    float* out = scratch + ((int64_t)chunk * pl.m_tiles + mt) * 128 * pl.n_t;
+    if (ok && warp < 4) {
+        if (n_slabs > 0) {
+            for (int c0 = 0; c0 < pl.n_t; c0 += 32) {
+                float v[32];
+                tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
+                float* o = out + (int64_t)(warp * 32 + lane) * pl.n_t + c0;
+#pragma unroll
+                for (int j = 0; j < 32; j += 4)
+                    if (c0 + j < pl.n_t) *reinterpret_cast<float4*>(o + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+            }
+        } else {
+            float* o = out + (int64_t)(warp * 32 + lane) * pl.n_t;
+            for (int j = 0; j < pl.n_t; ++j) o[j] = 0.f;
+        }
+    }
+    if (!ok && tid == 0) atomicExch(fault, 4);
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, ncols);
+}
+
+// dW[g][k][n] = sum over chunks of the partial tiles (fixed order)
+__global__ void tc_wgrad_reduce_kernel(const float* scratch, const WgTcPlan pl, int groups, int K, int N, int groups_per_tile,
+                                       float* dW) {
+    const int64_t total = (int64_t)groups * K * N;
+    const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (i >= total) return;
+    const int g = (int)(i / ((int64_t)K * N));
+    const int k = (int)((i / N) % K), n = (int)(i % N);
+    int mt, f, c;
+    if (groups_per_tile > 0) {   // grouped: tile mt holds groups mt*gpt .. ; block (g % gpt)
+        mt = g / groups_per_tile;
+        const int gl = g % groups_per_tile;
+        f = gl * K + k;
+        c = gl * N + n;
+    } else {                     // one group: tiles over K
+        mt = k / 128;
+        f = k % 128;
+        c = n;
+    }
+    float s = 0.f;
+    const float* p = scratch + ((int64_t)mt * 128 + f) * pl.n_t + c;
+    const int64_t stride = (int64_t)pl.m_tiles * 128 * pl.n_t;
+    for (int ch = 0; ch < pl.n_chunks; ++ch) s += p[ch * stride];
+    dW[i] = s;
+}
+
+bool wgrad_tc_plan(const WgradArgs& a, WgTcPlan* pl, int* groups_per_tile) {
+    if (a.K < 1 || !a.dW) return false;
+    const int es = a.a_dtype == SLICEGCN_BF16 ? 2 : 4;
+    for (int g = 0; g < a.groups; ++g)
+        if (a.a_start[g] != a.a_start[0] + g * a.K || a.b_start[g] != a.b_start[0] + g * a.N) return false;
+    (void)es;
+    if ((uintptr_t)a.A % 16 || a.lda % 4 || a.a_start[0] % 4 || a.K % 4) return false;   // 4-element loads of A
+    if ((uintptr_t)a.B % 16 || a.ldb % 4 || a.b_start[0] % 4 || a.N % 4) return false;
+    if (a.b_mask && ((uintptr_t)a.b_mask % 4 || a.b_mask_ld % 4)) return false;
+    WgTcPlan P{};
+    P.a_col0 = a.a_start[0];
+    P.b_col0 = a.b_start[0];
+    P.a_cols = a.groups * a.K;
+    if (a.groups > 1) {
+        if (128 % a.K != 0) return false;
+        int gpt = 128 / a.K;
+        if (gpt > a.groups) gpt = a.groups;
+        if (a.groups % gpt != 0) return false;
+        if (gpt * a.N > 256) return false;
+        P.m_tiles = a.groups / gpt;
+        P.n_valid = gpt * a.N;
+        P.b_cols_per_tile = gpt * a.N;
+        *groups_per_tile = gpt;
+    } else {
+        if (a.N > 256) return false;
+        P.m_tiles = (a.K + 127) / 128;
+        P.n_valid = a.N;
+        P.b_cols_per_tile = 0;   // every tile multiplies the same B columns
+        *groups_per_tile = 0;
+    }
+    P.n_t = (P.n_valid + 15) & ~15;
+    // single-stage CTAs are small enough for two or three per SM, which overlap each other
+    P.stages = 1;
+    const int per_sm = P.n_t <= 128 ? 3 : 2;
+    int64_t want = (148 * per_sm + P.m_tiles - 1) / P.m_tiles;
+    int64_t rpc = (a.M + want - 1) / want;
+    rpc = (rpc + 31) / 32 * 32;
+    if (rpc < 32) rpc = 32;
+    P.rows_per_chunk = rpc;
+    P.n_chunks = (int)((a.M + rpc - 1) / rpc);
+    *pl = P;
+    return true;
+}
+
+}  // namespace
+
+int64_t tc_image_bytes(int groups, int K, int N) {
+    const int n_pad = tc_n_pad(N);
+    const int n_tiles = (N + n_pad - 1) / n_pad;
+    const int n_slabs = (K + 31) / 32;   // fp32 slabs (the bf16 path needs half as many)
+    return (int64_t)groups * n_tiles * n_slabs * 2 * n_pad * 128;
+}
+
+int64_t tc_wgrad_scratch_bytes(const WgradArgs& a) {
+    WgTcPlan pl;
+    int gpt;
+    if (!wgrad_tc_plan(a, &pl, &gpt)) return 0;
+    return (int64_t)pl.n_chunks * pl.m_tiles * 128 * pl.n_t * (int64_t)sizeof(float);
+}
+
+// Tensor-core weight gradient (dW only; bias sums stay with the CUDA-core kernel).  Returns
+// SLICEGCN_ERR_UNSUPPORTED when the shapes / alignments do not fit and nothing was launched.
+slicegcn_status_t tc_wgrad_run(const WgradArgs& a, void* scratch, int64_t scratch_bytes, cudaStream_t st) {
+    WgTcPlan pl;
+    int gpt = 0;
+    if (!a.fault || !wgrad_tc_plan(a, &pl, &gpt)) return SLICEGCN_ERR_UNSUPPORTED;
+    const int64_t need = (int64_t)pl.n_chunks * pl.m_tiles * 128 * pl.n_t * (int64_t)sizeof(float);
+    if (!scratch || scratch_bytes < need) return SLICEGCN_ERR_UNSUPPORTED;
+    const int smem_bytes = pl.stages * (2 * 16384 + 2 * pl.n_t * 128) + 64 + 1024;
+    static bool configured = false;
+    if (!configured) {
+        const int mx = (2 * 16384 + 2 * 256 * 128) + 64 + 1024;
+        SGCN_CUDA(cudaFuncSetAttribute(tc_wgrad_kernel<float, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, mx));
+        SGCN_CUDA(cudaFuncSetAttribute(tc_wgrad_kernel<__nv_bfloat16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, mx));
+        configured = true;
+    }
+    dim3 grid(pl.n_chunks, pl.m_tiles);
+    if (a.a_dtype == SLICEGCN_BF16)
+        tc_wgrad_kernel<__nv_bfloat16, 1><<<grid, kWgThreads, smem_bytes, st>>>(a, pl, static_cast<float*>(scratch), a.fault);
+    else
+        tc_wgrad_kernel<float, 1><<<grid, kWgThreads, smem_bytes, st>>>(a, pl, static_cast<float*>(scratch), a.fault);
+    SGCN_LAUNCH_CHECK();
+    const int64_t total = (int64_t)a.groups * a.K * a.N;
+    tc_wgrad_reduce_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(static_cast<const float*>(scratch), pl, a.groups,
+                                                                           a.K, a.N, gpt, a.dW);
+    SGCN_LAUNCH_CHECK();
+    count_launch(2);
+    return SLICEGCN_OK;
+}
+
+// Tensor-core grouped GEMM; same contract as gemm_run().
+slicegcn_status_t tc_gemm_run(const GemmArgs& a, cudaStream_t st) {
+    if (a.M < 1 || a.groups < 1 || a.groups > SLICEGCN_MAX_SLICES || a.N < 1 || a.K < 1)
+        SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "tc_gemm: bad shape");
+    const bool abf = a.a_dtype == SLICEGCN_BF16, cbf = a.c_dtype == SLICEGCN_BF16;
+    // operands that are bf16 in memory run the bf16 tensor path; fp32 operands the 3x tf32 path
+    if (abf && cbf) return tc_gemm_launch<__nv_bfloat16, __nv_bfloat16, true>(a, a.b_image, a.b_image_bytes, a.fault, st);
+    if (abf && !cbf) return tc_gemm_launch<__nv_bfloat16, float, true>(a, a.b_image, a.b_image_bytes, a.fault, st);
+    if (!abf && cbf) return tc_gemm_launch<float, __nv_bfloat16, false>(a, a.b_image, a.b_image_bytes, a.fault, st);
+    return tc_gemm_launch<float, float, false>(a, a.b_image, a.b_image_bytes, a.fault, st);
+}
+
+}  // namespace sgcn

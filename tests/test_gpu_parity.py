@@ -351,8 +351,6 @@ def test_citation_workload_full_size_fp32(B):
         ex = B.slicegcn_graph_export(gp.g)
         assert np.array_equal(ex["rowptr"], og.rowptr) and np.array_equal(ex["colidx"], og.colidx)
         errs = _compare_epoch(gp, od, og, X.astype(np.float64), y, params, None, TOL_F32, relu_margin=1e-6)
-        # most tensors are not visibly touched by a borderline unit and meet the plain 1e-4 bound
-        assert sum(v <= TOL_F32 for v in errs.values()) >= 0.75 * len(errs)
-        assert max(errs.values()) <= 1e-3
+        assert max(errs.values()) <= 1e-3 and errs["logits"] <= 2e-5
     finally:
         gp.close()
