@@ -298,6 +298,25 @@ __global__ void mask_mul_kernel(int64_t M, int N, const float* in, int64_t ld_in
     }
 }
 
+// same, four columns per thread (all leading dimensions and N multiples of 4, 16-byte aligned rows)
+__global__ void mask_mul4_kernel(int64_t M, int N4, const float4* in, int64_t ld_in4, const uint32_t* mask, int64_t ld_mask4,
+                                 float4* out, int64_t ld_out4) {
+    const int64_t total = M * N4;
+    int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (; i < total; i += stride) {
+        const int64_t r = i / N4;
+        const int c = (int)(i - r * N4);
+        float4 v = __ldg(in + r * ld_in4 + c);
+        const uint32_t m = __ldg(mask + r * ld_mask4 + c);
+        if (!(m & 0x000000FFu)) v.x = 0.f;
+        if (!(m & 0x0000FF00u)) v.y = 0.f;
+        if (!(m & 0x00FF0000u)) v.z = 0.f;
+        if (!(m & 0xFF000000u)) v.w = 0.f;
+        out[r * ld_out4 + c] = v;
+    }
+}
+
 // one warp per training row
 __global__ void softmax_ce_kernel(int C, const float* logits, const int32_t* labels, const int32_t* train_idx,
                                   int64_t n_train, float inv_n, float* dlogits, float* row_loss) {
@@ -441,7 +460,14 @@ slicegcn_status_t mask_mul_run(int64_t M, int N, const float* in, int64_t ld_in,
                                float* out, int64_t ld_out, cudaStream_t st) {
     int64_t blocks = (M * N + 255) / 256;
     if (blocks > 148 * 16) blocks = 148 * 16;
-    mask_mul_kernel<<<(unsigned)blocks, 256, 0, st>>>(M, N, in, ld_in, mask, ld_mask, out, ld_out);
+    const bool vec = N % 4 == 0 && ld_in % 4 == 0 && ld_out % 4 == 0 && ld_mask % 4 == 0 && (uintptr_t)in % 16 == 0 &&
+                     (uintptr_t)out % 16 == 0 && (uintptr_t)mask % 4 == 0;
+    if (vec)
+        mask_mul4_kernel<<<(unsigned)blocks, 256, 0, st>>>(M, N / 4, reinterpret_cast<const float4*>(in), ld_in / 4,
+                                                           reinterpret_cast<const uint32_t*>(mask), ld_mask / 4,
+                                                           reinterpret_cast<float4*>(out), ld_out / 4);
+    else
+        mask_mul_kernel<<<(unsigned)blocks, 256, 0, st>>>(M, N, in, ld_in, mask, ld_mask, out, ld_out);
     SGCN_LAUNCH_CHECK();
     count_launch();
     return SLICEGCN_OK;

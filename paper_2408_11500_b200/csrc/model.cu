@@ -134,12 +134,8 @@ int64_t layer_bwd_ws_bytes(const slicegcn_graph* g, const LayerPlan& L) {
     b.take(layer_tc_img(L));
     b.take(layer_wgrad_scratch(L));
     b.take(spmm_partial_bytes(g, L.zt_cols));
-    if (L.order == SLICEGCN_AGG_FIRST) {
-        b.take(L.n * L.zt_ld * 4);
-    } else {
-        b.take(L.n * L.zt_ld * 4);
-        b.take(L.n * L.zt_ld * 4);
-    }
+    b.take(L.n * align_up(L.out_cols, 8) * 4);   // dM = dH * mask
+    b.take(L.n * L.zt_ld * 4);                   // dZ (aggregate-first) or dT (transform-first)
     return align_up(b.off, 256);
 }
 
@@ -303,7 +299,11 @@ slicegcn_status_t layer_backward_impl(const slicegcn_graph* g, const slicegcn_la
     }
 
     if (L.order == SLICEGCN_AGG_FIRST) {
-        if (dW_agg || db) {   // dW_agg = Z^T (dH * mask), db = colsum(dH * mask)
+        // dM = dH * mask, materialised once: it feeds the weight gradient, the bias gradient and dZ
+        const int64_t dm_ld = align_up(L.out_cols, 8);
+        float* dM = static_cast<float*>(b.take(L.n * dm_ld * 4));
+        SGCN_TRY(mask_mul_run(L.n, L.out_cols, dH_out, dout_ld, mask, L.mask_ld, dM, dm_ld, st));
+        if (dW_agg || db) {   // dW_agg = Z^T dM, db = colsum(dM)
             WgradArgs w;
             w.fault = g->fault;
             w.M = L.n;
@@ -313,10 +313,8 @@ slicegcn_status_t layer_backward_impl(const slicegcn_graph* g, const slicegcn_la
             w.A = zt;
             w.lda = L.zt_ld;
             w.a_dtype = L.dtype;
-            w.B = dH_out;
-            w.ldb = dout_ld;
-            w.b_mask = mask;
-            w.b_mask_ld = L.mask_ld;
+            w.B = dM;
+            w.ldb = dm_ld;
             w.dW = dW_agg;
             w.dbias = db;
             for (int i = 0; i < L.p; ++i) {
@@ -327,9 +325,9 @@ slicegcn_status_t layer_backward_impl(const slicegcn_graph* g, const slicegcn_la
         }
         if (dH_in) {
             float* dZ = static_cast<float*>(b.take(L.n * L.zt_ld * 4));
-            GemmArgs dz = dself;   // dZ = (dH * mask) W_agg^T
-            dz.a_mask = mask;
-            dz.a_mask_ld = L.mask_ld;
+            GemmArgs dz = dself;   // dZ = dM W_agg^T
+            dz.A = dM;
+            dz.lda = dm_ld;
             dz.B = d->W_agg;
             dz.C = dZ;
             dz.ldc = L.zt_ld;

@@ -9,6 +9,8 @@
 // one kind::f16 pass.  The hi/lo split needs a pass through registers anyway, so tiles are written
 // to shared memory with ordinary stores (swizzled by hand) followed by a proxy fence.
 // Every wait on an mbarrier is bounded; a wait that runs out sets the caller's status word.
+#include <cstdlib>
+
 #include "common.cuh"
 #include "kernels.cuh"
 
@@ -461,6 +463,268 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const GemmArgs a, c
     if (warp == 0) tmem_dealloc(tmem, ncols);
 }
 
+// ------------------------------------------------------------------------------ row-panel GEMM, warp-specialised
+// The same contract as tc_gemm_kernel, for 16-byte-aligned, unmasked operands.  One persistent CTA per
+// SM, nine warps in three roles connected by mbarriers (every wait is bounded):
+//   warps 0-3  producers: stream the activation slab of up to D-1 future steps into the stage ring
+//              with cp.async (16-byte chunks, written straight into the swizzled tile), and, for the
+//              step that has landed, split each fp32 chunk into its tf32 hi part (in place) and lo
+//              part; thread 0 also requests the step's weight image by bulk copy into the same stage;
+//   warp  4    MMA: one thread waits for a full stage, issues the tcgen05.mma chain into one of two
+//              TMEM accumulators and commits -- to the stage's "free" barrier after every slab, to
+//              the accumulator's "full" barrier after an item's last slab;
+//   warps 5-8  epilogue: drain a finished accumulator (tcgen05.ld), hand it back, then apply the
+//              fused epilogue and write whole 128-byte row segments.
+// Loads, MMAs and the epilogue of neighbouring items therefore overlap inside one CTA, and the
+// bytes in flight are set by the ring depth, not by the register file.
+constexpr int kWsThreads = 288;
+
+template <typename TA, typename TC, bool BF16>
+__global__ void __launch_bounds__(kWsThreads, 1) tc_gemm_ws_kernel(const GemmArgs a, const int n_pad, const int n_tiles,
+                                                                   const int D, const unsigned char* image, int* fault) {
+    extern __shared__ __align__(1024) unsigned char smem[];
+    constexpr int KS = BF16 ? 64 : 32;
+    constexpr int UK = BF16 ? 16 : 8;
+    constexpr int EPC = BF16 ? 8 : 4;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    unsigned char* base = smem + ((1024u - (smem_u32(smem) & 1023u)) & 1023u);
+    const uint32_t slab_bytes = 2u * (uint32_t)n_pad * 128u;                  // weight image [hi | lo]
+    const uint32_t a_bytes = BF16 ? 16384u : 32768u;                          // activation tile(s) of a stage
+    const uint32_t stage_bytes = a_bytes + slab_bytes;
+    float* stage_out = reinterpret_cast<float*>(base + (uint32_t)D * stage_bytes);   // 4 x 32 x kStagePitch floats
+    unsigned char* tail = reinterpret_cast<unsigned char*>(stage_out) + 4 * 32 * kStagePitch * 4;
+    uint64_t* full = reinterpret_cast<uint64_t*>(tail);            // [D]   128 producer arrivals + weight bytes
+    uint64_t* freeb = full + 8;                                     // [D]   MMAs of the stage have completed
+    uint64_t* tfull = freeb + 8;                                    // [2]   accumulator complete
+    uint64_t* tfree = tfull + 2;                                    // [2]   accumulator drained (128 arrivals)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tfree + 2);
+    uint32_t acc_cols = 32;
+    while ((int)acc_cols < n_pad) acc_cols <<= 1;
+    const uint32_t ncols = 2 * acc_cols;
+    if (tid == 0) {
+        for (int i = 0; i < D; ++i) {
+            mbar_init(&full[i], 129);
+            mbar_init(&freeb[i], 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&tfull[i], 1);
+            mbar_init(&tfree[i], 128);
+        }
+    }
+    if (warp == 4) tmem_alloc(tmem_slot, ncols);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    const int n_slabs = (a.K + KS - 1) / KS;
+    const int64_t row_tiles = (a.M + 127) / 128;
+    const int64_t n_items = row_tiles * a.groups * n_tiles;
+    const int64_t my_items = n_items > blockIdx.x ? (n_items - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+    const int64_t my_steps = my_items * n_slabs;
+    auto decode = [&](int64_t local_item, int64_t& row0, int& g, int& nt) {
+        const int64_t item = blockIdx.x + local_item * gridDim.x;
+        nt = (int)(item % n_tiles);
+        g = (int)((item / n_tiles) % a.groups);
+        row0 = (item / ((int64_t)n_tiles * a.groups)) * 128;
+    };
+
+    if (warp < 4) {
+        // ------------------------------------------------------------ producers
+        const int c = tid & 7;          // 16-byte chunk of the 128-byte row
+        const int rbase = tid >> 3;     // rows rbase + 16 i
+        const int L = D - 1;            // steps requested ahead of the one being finished
+        auto issue = [&](int64_t j) {   // requests step j's activation slab (and weight image)
+            const int st = (int)(j % D);
+            const int64_t use = j / D;
+            bool okw = true;
+            if (use >= 1) okw = mbar_wait(&freeb[st], (uint32_t)((use - 1) & 1));
+            if (!okw) {
+                if (lane == 0) atomicExch(fault, 5);
+                return false;
+            }
+            int64_t row0;
+            int g, nt;
+            decode(j / n_slabs, row0, g, nt);
+            const int s = (int)(j % n_slabs);
+            unsigned char* stg = base + (uint32_t)st * stage_bytes;
+            if (tid == 0) {
+                mbar_expect_tx(&full[st], slab_bytes);
+                bulk_g2s(stg + a_bytes, image + ((((int64_t)g * n_tiles + nt) * n_slabs + s)) * (int64_t)slab_bytes, slab_bytes,
+                         &full[st]);
+            }
+            const TA* A = static_cast<const TA*>(a.A) + a.a_start[g];
+            const int k = s * KS + c * EPC;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int r = rbase + 16 * i;
+                const int64_t row = row0 + r;
+                const bool in = row < a.M && k < a.K;
+                const TA* src = in ? (A + row * a.lda + k) : static_cast<const TA*>(a.A);
+                const uint32_t dst = smem_u32(stg + sw_off(r, c * 16));
+                const int sz = in ? 16 : 0;   // zero-fill outside the matrix
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(sz) : "memory");
+            }
+            return true;
+        };
+        bool okp = true;
+        for (int64_t j = 0; j < L && okp; ++j) {   // exactly L groups, empty past the end, so the count below holds
+            if (j < my_steps) okp = issue(j);
+            asm volatile("cp.async.commit_group;" ::: "memory");
+        }
+        for (int64_t j = 0; j < my_steps && okp; ++j) {
+            if (j + L < my_steps) okp = issue(j + L);
+            asm volatile("cp.async.commit_group;" ::: "memory");   // one group per step, empty or not
+            if (!okp) break;
+            // step j's chunks (this thread's own copies) have landed once at most L newer groups are pending
+            if (D == 2) asm volatile("cp.async.wait_group 1;" ::: "memory");
+            else if (D == 3) asm volatile("cp.async.wait_group 2;" ::: "memory");
+            else asm volatile("cp.async.wait_group 3;" ::: "memory");
+            const int st = (int)(j % D);
+            unsigned char* stg = base + (uint32_t)st * stage_bytes;
+            if (!BF16) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const uint32_t off = sw_off(rbase + 16 * i, c * 16);
+                    const float4 v = *reinterpret_cast<const float4*>(stg + off);
+                    const float h0 = tf32_hi(v.x), h1 = tf32_hi(v.y), h2 = tf32_hi(v.z), h3 = tf32_hi(v.w);
+                    *reinterpret_cast<float4*>(stg + off) = make_float4(h0, h1, h2, h3);
+                    *reinterpret_cast<float4*>(stg + 16384 + off) = make_float4(v.x - h0, v.y - h1, v.z - h2, v.w - h3);
+                }
+            }
+            proxy_fence();
+            asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&full[st])) : "memory");
+        }
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+    } else if (warp == 4) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            bool okm = true;
+            for (int64_t it = 0; it < my_items && okm; ++it) {
+                const int acc = (int)(it & 1);
+                const int64_t use = it >> 1;
+                if (use >= 1) okm = mbar_wait(&tfree[acc], (uint32_t)((use - 1) & 1));
+                if (!okm) break;
+                tc_fence_after();
+                int64_t row0;
+                int g, nt;
+                decode(it, row0, g, nt);
+                const int nn = min(n_pad, a.N - nt * n_pad);
+                const int n_mma = (nn + 15) & ~15;
+                const uint32_t idesc = idesc_f32acc(128, n_mma, BF16);
+                const uint32_t d_tmem = tmem + (uint32_t)acc * acc_cols;
+                for (int s = 0; s < n_slabs && okm; ++s) {
+                    const int64_t j = it * n_slabs + s;
+                    const int st = (int)(j % D);
+                    okm = mbar_wait(&full[st], (uint32_t)((j / D) & 1));
+                    if (!okm) break;
+                    tc_fence_after();
+                    unsigned char* stg = base + (uint32_t)st * stage_bytes;
+                    const uint64_t da_hi = smem_desc(stg), da_lo = smem_desc(stg + 16384);
+                    const uint64_t db_hi = smem_desc(stg + a_bytes), db_lo = smem_desc(stg + a_bytes + n_pad * 128);
+#pragma unroll
+                    for (int ks = 0; ks < KS / UK; ++ks) {
+                        const uint64_t adv = (uint64_t)((ks * 32) >> 4);
+                        umma<BF16>(d_tmem, da_hi + adv, db_hi + adv, idesc, (s == 0 && ks == 0) ? 0u : 1u);
+                        if (!BF16) umma<BF16>(d_tmem, da_lo + adv, db_hi + adv, idesc, 1u);
+                        umma<BF16>(d_tmem, da_hi + adv, db_lo + adv, idesc, 1u);
+                    }
+                    umma_commit(&freeb[st]);
+                }
+                if (okm) umma_commit(&tfull[acc]);
+            }
+            if (!okm) atomicExch(fault, 6);
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue
+        const int q = warp & 3;                       // TMEM lane quarter this warp may read
+        float* stage = stage_out + q * (32 * kStagePitch);
+        TC* C = static_cast<TC*>(a.C);
+        bool oke = true;
+        for (int64_t it = 0; it < my_items && oke; ++it) {
+            const int acc = (int)(it & 1);
+            oke = mbar_wait(&tfull[acc], (uint32_t)((it >> 1) & 1));
+            if (!oke) break;
+            tc_fence_after();
+            int64_t row0;
+            int g, nt;
+            decode(it, row0, g, nt);
+            const int n0 = nt * n_pad;
+            const int nn = min(n_pad, a.N - n0);
+            const int n_mma = (nn + 15) & ~15;
+            const int cs = a.c_start[g] + n0;
+            const uint32_t d_tmem = tmem + (uint32_t)acc * acc_cols + ((uint32_t)(q * 32) << 16);
+            for (int c0 = 0; c0 < n_mma; c0 += 32) {
+                float v[32];
+                tmem_ld32(d_tmem + (uint32_t)c0, v);
+                if (c0 + 32 >= n_mma) {   // last read of this accumulator: hand it back to the MMA warp
+                    tc_fence_before();
+                    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&tfree[acc])) : "memory");
+                }
+#pragma unroll
+                for (int j = 0; j < 32; ++j) stage[lane * kStagePitch + j] = v[j];
+                __syncwarp();
+                const int n = c0 + lane;
+                const bool col_ok = n < nn;
+                const int col = cs + n;
+                float bias = 0.f, post = 0.f;
+                if (col_ok) {
+                    if (a.bias) bias = __ldg(a.bias + g * a.N + n0 + n);
+                    if (a.post1) post += __ldg(a.post1 + g * a.N + n0 + n);
+                    if (a.post2) post += __ldg(a.post2 + g * a.N + n0 + n);
+                }
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    float cold[16], gate[16];
+                    if (a.accumulate) {
+#pragma unroll
+                        for (int r = 0; r < 16; ++r) {
+                            const int64_t row = row0 + q * 32 + half * 16 + r;
+                            cold[r] = (row < a.M && col_ok) ? ld_as_f(C + row * a.ldc + col) : 0.f;
+                        }
+                    }
+                    if (a.mul_pos) {
+#pragma unroll
+                        for (int r = 0; r < 16; ++r) {
+                            const int64_t row = row0 + q * 32 + half * 16 + r;
+                            float pv = 1.f;
+                            if (row < a.M && col_ok)
+                                pv = a.mul_pos_dtype == SLICEGCN_F32
+                                         ? __ldg(static_cast<const float*>(a.mul_pos) + row * a.mul_pos_ld + col)
+                                         : __bfloat162float(static_cast<const __nv_bfloat16*>(a.mul_pos)[row * a.mul_pos_ld + col]);
+                            gate[r] = pv;
+                        }
+                    }
+#pragma unroll
+                    for (int r = 0; r < 16; ++r) {
+                        const int rr = half * 16 + r;
+                        const int64_t row = row0 + q * 32 + rr;
+                        if (row >= a.M || !col_ok) continue;
+                        float x = stage[rr * kStagePitch + lane] + bias;
+                        if (a.relu) {
+                            if (a.mask_out) a.mask_out[row * a.mask_ld + col] = x > 0.f ? 1 : 0;
+                            x = fmaxf(x, 0.f);
+                        }
+                        x += post;
+                        if (a.mul_pos) x = gate[r] > 0.f ? x : 0.f;
+                        if (a.accumulate) x += cold[r];
+                        if (sizeof(TC) == 4)
+                            reinterpret_cast<float*>(C)[row * a.ldc + col] = x;
+                        else
+                            reinterpret_cast<__nv_bfloat16*>(C)[row * a.ldc + col] = __float2bfloat16_rn(x);
+                    }
+                }
+                __syncwarp();
+            }
+        }
+        if (!oke && lane == 0) atomicExch(fault, 7);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 4) tmem_dealloc(tmem, ncols);
+}
+
 int tc_n_pad(int N) { return N <= 256 ? ((N + 15) & ~15) : 256; }
 
 template <typename TA, typename TC, bool BF16>
@@ -487,6 +751,30 @@ slicegcn_status_t tc_gemm_launch(const GemmArgs& a, void* image, int64_t image_b
     bool vec = ((uintptr_t)a.A % 16 == 0) && (a.lda % EPC == 0) && (a.K % EPC == 0);
     for (int g = 0; g < a.groups; ++g) vec = vec && (a.a_start[g] % EPC == 0);
     if (a.a_mask) vec = vec && ((uintptr_t)a.a_mask % 8 == 0) && (a.a_mask_ld % 8 == 0);
+    static const bool no_ws = getenv("SLICEGCN_NO_WS") != nullptr;
+    if (vec && !a.a_mask && !no_ws) {
+        // warp-specialised kernel: one CTA per SM, ring depth from what fits in shared memory
+        const int a_bytes = BF16 ? 16384 : 32768;
+        const int stage_b = a_bytes + 2 * n_pad * 128;
+        const int fixed = 4 * 32 * kStagePitch * 4 + 256 + 1024;
+        int D = (220 * 1024 - fixed) / stage_b;
+        if (D > 4) D = 4;
+        if (D >= 2) {
+            const int ws_smem = D * stage_b + fixed;
+            static bool ws_configured = false;
+            if (!ws_configured) {
+                SGCN_CUDA(cudaFuncSetAttribute(tc_gemm_ws_kernel<TA, TC, BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
+                ws_configured = true;
+            }
+            const int64_t items = ((a.M + 127) / 128) * a.groups * n_tiles;
+            int64_t wgrid = 148;
+            if (wgrid > items) wgrid = items;
+            tc_gemm_ws_kernel<TA, TC, BF16><<<(unsigned)wgrid, kWsThreads, ws_smem, st>>>(a, n_pad, n_tiles, D, static_cast<unsigned char*>(image), fault);
+            SGCN_LAUNCH_CHECK();
+            count_launch(2);
+            return SLICEGCN_OK;
+        }
+    }
     // persistent grid: as many CTAs as fit at once (shared memory and 512 TMEM columns per SM)
     int ncols = 32;
     while (ncols < n_pad) ncols <<= 1;
