@@ -35,9 +35,25 @@ __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
+__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;   // may suspend the thread for a short, hardware-bounded time before returning
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up (returns false) after kWaitSpins attempts or about two seconds.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
-    for (int i = 0; i < kWaitSpins; ++i)
-        if (mbar_test(bar, parity)) return true;
+    if (mbar_test(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (int i = 0; i < kWaitSpins; ++i) {
+        if (mbar_try(bar, parity)) return true;
+        if (clock64() - t0 > 4000000000LL) break;
+    }
     return false;
 }
 
@@ -122,11 +138,10 @@ __device__ __forceinline__ uint32_t idesc_f32acc(int M, int N, bool bf16) {
 __device__ __forceinline__ float ld_as_f(const float* p) { return __ldg(p); }
 __device__ __forceinline__ float ld_as_f(const __nv_bfloat16* p) { return __bfloat162float(*p); }
 
-// nearest value with a 10-bit mantissa (what the tf32 path keeps); Inf/NaN pass through
+// nearest value with a 10-bit mantissa (what the tf32 path keeps)
 __device__ __forceinline__ float tf32_hi(float v) {
-    const uint32_t b = __float_as_uint(v);
-    if ((b & 0x7F800000u) == 0x7F800000u) return v;
-    return __uint_as_float((b + 0x1000u) & 0xFFFFE000u);
+    // round half up in magnitude on the 13 dropped bits; Inf stays Inf, NaN stays NaN
+    return __uint_as_float((__float_as_uint(v) + 0x1000u) & 0xFFFFE000u);
 }
 // stores one fp32 operand value into the hi / lo tiles (tf32 split) or one bf16 value
 __device__ __forceinline__ void put_f32(unsigned char* hi, unsigned char* lo, int row, int k, float v) {
@@ -187,7 +202,7 @@ __global__ void __launch_bounds__(128) tc_prep_b_kernel(const GemmArgs a, const 
 // of the next slab (or next item) are in flight while the MMAs run and while the finished item's
 // accumulators go TMEM -> registers -> per-warp staging tile -> global memory in whole 128-byte rows.
 constexpr int kTcThreads = 128;
-constexpr int kStagePitch = 33;   // floats per staged row (odd: conflict-free both ways)
+constexpr int kStagePitch = 36;   // floats per staged row: 16-byte aligned rows, few bank conflicts either way
 
 template <typename TA, typename TC, bool BF16, bool VEC>
 __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const GemmArgs a, const int n_pad, const int n_tiles,
@@ -524,17 +539,25 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_gemm_ws_kernel(const GemmArg
     const int64_t my_items = n_items > blockIdx.x ? (n_items - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
     const int64_t my_steps = my_items * n_slabs;
     auto decode = [&](int64_t local_item, int64_t& row0, int& g, int& nt) {
-        const int64_t item = blockIdx.x + local_item * gridDim.x;
-        nt = (int)(item % n_tiles);
-        g = (int)((item / n_tiles) % a.groups);
-        row0 = (item / ((int64_t)n_tiles * a.groups)) * 128;
+        const uint32_t item = (uint32_t)(blockIdx.x + local_item * gridDim.x);   // host keeps the item count < 2^31
+        const uint32_t per_row = (uint32_t)(n_tiles * a.groups);
+        const uint32_t rt = item / per_row, rem = item - rt * per_row;
+        g = (int)(rem / (uint32_t)n_tiles);
+        nt = (int)(rem - (uint32_t)g * (uint32_t)n_tiles);
+        row0 = (int64_t)rt * 128;
     };
 
     if (warp < 4) {
         // ------------------------------------------------------------ producers
         const int c = tid & 7;          // 16-byte chunk of the 128-byte row
         const int rbase = tid >> 3;     // rows rbase + 16 i
-        const int L = D - 1;            // steps requested ahead of the one being finished
+        uint32_t offs[8];               // swizzled byte offsets of this thread's eight chunks
+#pragma unroll
+        for (int i = 0; i < 8; ++i) offs[i] = sw_off(rbase + 16 * i, c * 16);
+        const int64_t row_step = 16 * a.lda;
+        // steps requested ahead of the one being finished; with D >= 3 the stage a new request goes to
+        // was last used two steps back, so the producer never waits for the MMAs it has just fed
+        const int L = D >= 3 ? D - 2 : 1;
         auto issue = [&](int64_t j) {   // requests step j's activation slab (and weight image)
             const int st = (int)(j % D);
             const int64_t use = j / D;
@@ -554,17 +577,17 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_gemm_ws_kernel(const GemmArg
                 bulk_g2s(stg + a_bytes, image + ((((int64_t)g * n_tiles + nt) * n_slabs + s)) * (int64_t)slab_bytes, slab_bytes,
                          &full[st]);
             }
-            const TA* A = static_cast<const TA*>(a.A) + a.a_start[g];
             const int k = s * KS + c * EPC;
+            const TA* src0 = static_cast<const TA*>(a.A) + a.a_start[g] + (row0 + rbase) * a.lda + k;
+            const uint32_t dst0 = smem_u32(stg);
+            const int rows_left = (int)min((int64_t)128, a.M - row0) - rbase;   // rows rbase + 16 i < rows of the tile
+            const bool k_in = k < a.K;
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-                const int r = rbase + 16 * i;
-                const int64_t row = row0 + r;
-                const bool in = row < a.M && k < a.K;
-                const TA* src = in ? (A + row * a.lda + k) : static_cast<const TA*>(a.A);
-                const uint32_t dst = smem_u32(stg + sw_off(r, c * 16));
+                const bool in = k_in && 16 * i < rows_left;
+                const TA* src = in ? (src0 + i * row_step) : static_cast<const TA*>(a.A);
                 const int sz = in ? 16 : 0;   // zero-fill outside the matrix
-                asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(sz) : "memory");
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst0 + offs[i]), "l"(src), "r"(sz) : "memory");
             }
             return true;
         };
@@ -574,27 +597,24 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_gemm_ws_kernel(const GemmArg
             asm volatile("cp.async.commit_group;" ::: "memory");
         }
         for (int64_t j = 0; j < my_steps && okp; ++j) {
-            if (j + L < my_steps) okp = issue(j + L);
-            asm volatile("cp.async.commit_group;" ::: "memory");   // one group per step, empty or not
-            if (!okp) break;
-            // step j's chunks (this thread's own copies) have landed once at most L newer groups are pending
-            if (D == 2) asm volatile("cp.async.wait_group 1;" ::: "memory");
-            else if (D == 3) asm volatile("cp.async.wait_group 2;" ::: "memory");
-            else asm volatile("cp.async.wait_group 3;" ::: "memory");
+            // L + j groups so far: step j (this thread's own copies) has landed once at most L-1 are pending
+            if (L == 2) asm volatile("cp.async.wait_group 1;" ::: "memory");
+            else asm volatile("cp.async.wait_group 0;" ::: "memory");
             const int st = (int)(j % D);
             unsigned char* stg = base + (uint32_t)st * stage_bytes;
             if (!BF16) {
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
-                    const uint32_t off = sw_off(rbase + 16 * i, c * 16);
-                    const float4 v = *reinterpret_cast<const float4*>(stg + off);
+                    const float4 v = *reinterpret_cast<const float4*>(stg + offs[i]);
                     const float h0 = tf32_hi(v.x), h1 = tf32_hi(v.y), h2 = tf32_hi(v.z), h3 = tf32_hi(v.w);
-                    *reinterpret_cast<float4*>(stg + off) = make_float4(h0, h1, h2, h3);
-                    *reinterpret_cast<float4*>(stg + 16384 + off) = make_float4(v.x - h0, v.y - h1, v.z - h2, v.w - h3);
+                    *reinterpret_cast<float4*>(stg + offs[i]) = make_float4(h0, h1, h2, h3);
+                    *reinterpret_cast<float4*>(stg + 16384 + offs[i]) = make_float4(v.x - h0, v.y - h1, v.z - h2, v.w - h3);
                 }
             }
             proxy_fence();
             asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&full[st])) : "memory");
+            if (j + L < my_steps) okp = issue(j + L);
+            asm volatile("cp.async.commit_group;" ::: "memory");   // one group per step, empty or not
         }
         asm volatile("cp.async.wait_group 0;" ::: "memory");
     } else if (warp == 4) {
@@ -638,9 +658,12 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_gemm_ws_kernel(const GemmArg
         }
     } else {
         // ------------------------------------------------------------ epilogue
+        // lane: column quad cq (4 consecutive columns) of rows sub, sub+4, ...: every global access of a
+        // warp covers four whole 128-byte row segments
         const int q = warp & 3;                       // TMEM lane quarter this warp may read
         float* stage = stage_out + q * (32 * kStagePitch);
-        TC* C = static_cast<TC*>(a.C);
+        const int cq = lane & 7, sub = lane >> 3;
+        unsigned char* Cb = static_cast<unsigned char*>(a.C);
         bool oke = true;
         for (int64_t it = 0; it < my_items && oke; ++it) {
             const int acc = (int)(it & 1);
@@ -655,6 +678,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_gemm_ws_kernel(const GemmArg
             const int n_mma = (nn + 15) & ~15;
             const int cs = a.c_start[g] + n0;
             const uint32_t d_tmem = tmem + (uint32_t)acc * acc_cols + ((uint32_t)(q * 32) << 16);
+            const int rows_here = (int)min((int64_t)32, a.M - (row0 + q * 32));   // valid rows of this warp's quarter
             for (int c0 = 0; c0 < n_mma; c0 += 32) {
                 float v[32];
                 tmem_ld32(d_tmem + (uint32_t)c0, v);
@@ -663,56 +687,89 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_gemm_ws_kernel(const GemmArg
                     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&tfree[acc])) : "memory");
                 }
 #pragma unroll
-                for (int j = 0; j < 32; ++j) stage[lane * kStagePitch + j] = v[j];
+                for (int j = 0; j < 32; j += 4)
+                    *reinterpret_cast<float4*>(stage + lane * kStagePitch + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
                 __syncwarp();
-                const int n = c0 + lane;
-                const bool col_ok = n < nn;
+                const int n = c0 + cq * 4;            // first of this lane's four columns within the tile
+                const bool col_ok = n < nn;           // nn is a multiple of 4 on this path
                 const int col = cs + n;
-                float bias = 0.f, post = 0.f;
+                float4 bias = make_float4(0.f, 0.f, 0.f, 0.f), post = bias;
                 if (col_ok) {
-                    if (a.bias) bias = __ldg(a.bias + g * a.N + n0 + n);
-                    if (a.post1) post += __ldg(a.post1 + g * a.N + n0 + n);
-                    if (a.post2) post += __ldg(a.post2 + g * a.N + n0 + n);
+                    if (a.bias) bias = __ldg(reinterpret_cast<const float4*>(a.bias + g * a.N + n0 + n));
+                    if (a.post1) post = __ldg(reinterpret_cast<const float4*>(a.post1 + g * a.N + n0 + n));
+                    if (a.post2) {
+                        const float4 p2 = __ldg(reinterpret_cast<const float4*>(a.post2 + g * a.N + n0 + n));
+                        post = make_float4(post.x + p2.x, post.y + p2.y, post.z + p2.z, post.w + p2.w);
+                    }
+                }
+                const int64_t rfirst = row0 + q * 32 + sub;
+                float4 cold[8], gate[8];
+                if (a.accumulate) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        cold[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (col_ok && 4 * i + sub < rows_here) {
+                            if (sizeof(TC) == 4) {
+                                cold[i] = *reinterpret_cast<const float4*>(Cb + ((rfirst + 4 * i) * a.ldc + col) * 4);
+                            } else {
+                                const uint2 h = *reinterpret_cast<const uint2*>(Cb + ((rfirst + 4 * i) * a.ldc + col) * 2);
+                                cold[i] = make_float4(__uint_as_float(h.x << 16), __uint_as_float(h.x & 0xffff0000u),
+                                                      __uint_as_float(h.y << 16), __uint_as_float(h.y & 0xffff0000u));
+                            }
+                        }
+                    }
+                }
+                if (a.mul_pos) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        gate[i] = make_float4(1.f, 1.f, 1.f, 1.f);
+                        if (col_ok && 4 * i + sub < rows_here) {
+                            if (a.mul_pos_dtype == SLICEGCN_F32) {
+                                gate[i] = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(a.mul_pos) +
+                                                                                (rfirst + 4 * i) * a.mul_pos_ld + col));
+                            } else {
+                                const uint2 h = __ldg(reinterpret_cast<const uint2*>(
+                                    static_cast<const __nv_bfloat16*>(a.mul_pos) + (rfirst + 4 * i) * a.mul_pos_ld + col));
+                                gate[i] = make_float4(__uint_as_float(h.x << 16), __uint_as_float(h.x & 0xffff0000u),
+                                                      __uint_as_float(h.y << 16), __uint_as_float(h.y & 0xffff0000u));
+                            }
+                        }
+                    }
                 }
 #pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    float cold[16], gate[16];
-                    if (a.accumulate) {
-#pragma unroll
-                        for (int r = 0; r < 16; ++r) {
-                            const int64_t row = row0 + q * 32 + half * 16 + r;
-                            cold[r] = (row < a.M && col_ok) ? ld_as_f(C + row * a.ldc + col) : 0.f;
+                for (int i = 0; i < 8; ++i) {
+                    const int rr = 4 * i + sub;
+                    if (!col_ok || rr >= rows_here) continue;
+                    const int64_t row = rfirst + 4 * i;
+                    const float4 t = *reinterpret_cast<const float4*>(stage + rr * kStagePitch + cq * 4);
+                    float x[4] = {t.x + bias.x, t.y + bias.y, t.z + bias.z, t.w + bias.w};
+                    if (a.relu) {
+                        if (a.mask_out) {
+                            const uint32_t m = (x[0] > 0.f ? 1u : 0u) | (x[1] > 0.f ? 0x100u : 0u) | (x[2] > 0.f ? 0x10000u : 0u) |
+                                               (x[3] > 0.f ? 0x1000000u : 0u);
+                            *reinterpret_cast<uint32_t*>(a.mask_out + row * a.mask_ld + col) = m;
                         }
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) x[e] = fmaxf(x[e], 0.f);
                     }
+                    x[0] += post.x; x[1] += post.y; x[2] += post.z; x[3] += post.w;
                     if (a.mul_pos) {
-#pragma unroll
-                        for (int r = 0; r < 16; ++r) {
-                            const int64_t row = row0 + q * 32 + half * 16 + r;
-                            float pv = 1.f;
-                            if (row < a.M && col_ok)
-                                pv = a.mul_pos_dtype == SLICEGCN_F32
-                                         ? __ldg(static_cast<const float*>(a.mul_pos) + row * a.mul_pos_ld + col)
-                                         : __bfloat162float(static_cast<const __nv_bfloat16*>(a.mul_pos)[row * a.mul_pos_ld + col]);
-                            gate[r] = pv;
-                        }
+                        x[0] = gate[i].x > 0.f ? x[0] : 0.f;
+                        x[1] = gate[i].y > 0.f ? x[1] : 0.f;
+                        x[2] = gate[i].z > 0.f ? x[2] : 0.f;
+                        x[3] = gate[i].w > 0.f ? x[3] : 0.f;
                     }
-#pragma unroll
-                    for (int r = 0; r < 16; ++r) {
-                        const int rr = half * 16 + r;
-                        const int64_t row = row0 + q * 32 + rr;
-                        if (row >= a.M || !col_ok) continue;
-                        float x = stage[rr * kStagePitch + lane] + bias;
-                        if (a.relu) {
-                            if (a.mask_out) a.mask_out[row * a.mask_ld + col] = x > 0.f ? 1 : 0;
-                            x = fmaxf(x, 0.f);
-                        }
-                        x += post;
-                        if (a.mul_pos) x = gate[r] > 0.f ? x : 0.f;
-                        if (a.accumulate) x += cold[r];
-                        if (sizeof(TC) == 4)
-                            reinterpret_cast<float*>(C)[row * a.ldc + col] = x;
-                        else
-                            reinterpret_cast<__nv_bfloat16*>(C)[row * a.ldc + col] = __float2bfloat16_rn(x);
+                    if (a.accumulate) {
+                        x[0] += cold[i].x; x[1] += cold[i].y; x[2] += cold[i].z; x[3] += cold[i].w;
+                    }
+                    if (sizeof(TC) == 4) {
+                        *reinterpret_cast<float4*>(Cb + (row * a.ldc + col) * 4) = make_float4(x[0], x[1], x[2], x[3]);
+                    } else {
+                        const __nv_bfloat162 lo2 = __floats2bfloat162_rn(x[0], x[1]), hi2 = __floats2bfloat162_rn(x[2], x[3]);
+                        uint2 pk;
+                        pk.x = *reinterpret_cast<const uint32_t*>(&lo2);
+                        pk.y = *reinterpret_cast<const uint32_t*>(&hi2);
+                        *reinterpret_cast<uint2*>(Cb + (row * a.ldc + col) * 2) = pk;
                     }
                 }
                 __syncwarp();
@@ -752,7 +809,18 @@ slicegcn_status_t tc_gemm_launch(const GemmArgs& a, void* image, int64_t image_b
     for (int g = 0; g < a.groups; ++g) vec = vec && (a.a_start[g] % EPC == 0);
     if (a.a_mask) vec = vec && ((uintptr_t)a.a_mask % 8 == 0) && (a.a_mask_ld % 8 == 0);
     static const bool no_ws = getenv("SLICEGCN_NO_WS") != nullptr;
-    if (vec && !a.a_mask && !no_ws) {
+    // the warp-specialised kernel also writes (and re-reads) C, the ReLU mask and the gate in 4-element pieces
+    const int ces = sizeof(TC);
+    bool cvec = (a.N % 4 == 0) && (a.ldc % 4 == 0) && ((uintptr_t)a.C % 16 == 0);
+    for (int g = 0; g < a.groups; ++g) cvec = cvec && (a.c_start[g] % 4 == 0);
+    if (a.mask_out) cvec = cvec && (a.mask_ld % 4 == 0) && ((uintptr_t)a.mask_out % 4 == 0);
+    if (a.mul_pos) cvec = cvec && (a.mul_pos_ld % 4 == 0) && ((uintptr_t)a.mul_pos % 16 == 0);
+    if (a.bias) cvec = cvec && ((uintptr_t)a.bias % 16 == 0);
+    if (a.post1) cvec = cvec && ((uintptr_t)a.post1 % 16 == 0);
+    if (a.post2) cvec = cvec && ((uintptr_t)a.post2 % 16 == 0);
+    (void)ces;
+    const int64_t all_items = ((a.M + 127) / 128) * a.groups * n_tiles;
+    if (vec && cvec && !a.a_mask && !no_ws && all_items < ((int64_t)1 << 31)) {
         // warp-specialised kernel: one CTA per SM, ring depth from what fits in shared memory
         const int a_bytes = BF16 ? 16384 : 32768;
         const int stage_b = a_bytes + 2 * n_pad * 128;
