@@ -169,13 +169,14 @@ __device__ __forceinline__ void put_bf16x2(unsigned char* hi, unsigned char* lo,
 template <bool BF16>
 __global__ void __launch_bounds__(128) tc_prep_b_kernel(const GemmArgs a, const int n_pad, unsigned char* image) {
     constexpr int KS = BF16 ? 64 : 32;
-    const int s = blockIdx.x, nt = blockIdx.y, g = blockIdx.z;
-    const int n_slabs = gridDim.x, n_tiles = gridDim.y;
+    const int s = blockIdx.x / 4, part = blockIdx.x % 4, nt = blockIdx.y, g = blockIdx.z;
+    const int n_slabs = gridDim.x / 4, n_tiles = gridDim.y;
     const float* B = a.B + (int64_t)g * a.b_gstride;
     unsigned char* hi = image + ((((int64_t)g * n_tiles + nt) * n_slabs + s) * 2) * ((int64_t)n_pad * 128);
     unsigned char* lo = hi + (int64_t)n_pad * 128;
     const int n0 = nt * n_pad, k0 = s * KS;
-    for (int e = threadIdx.x; e < n_pad * KS; e += 128) {
+    const int per = (n_pad * KS + 3) / 4;   // this block's quarter of the tile's elements
+    for (int e = part * per + threadIdx.x; e < min((part + 1) * per, n_pad * KS); e += 128) {
         int n, kk;
         if (a.b_trans) {
             kk = e % KS;
@@ -801,7 +802,7 @@ slicegcn_status_t tc_gemm_launch(const GemmArgs& a, void* image, int64_t image_b
         SGCN_CUDA(cudaFuncSetAttribute(tc_gemm_kernel<TA, TC, BF16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, mx));
         configured = true;
     }
-    dim3 pgrid(n_slabs, n_tiles, a.groups);
+    dim3 pgrid(n_slabs * 4, n_tiles, a.groups);
     tc_prep_b_kernel<BF16><<<pgrid, 128, 0, st>>>(a, n_pad, static_cast<unsigned char*>(image));
     SGCN_LAUNCH_CHECK();
     // 16-byte loads of the activation need aligned slices
@@ -1062,7 +1063,15 @@ __global__ void tc_wgrad_reduce_kernel(const float* scratch, const WgTcPlan pl, 
     float s = 0.f;
     const float* p = scratch + ((int64_t)mt * 128 + f) * pl.n_t + c;
     const int64_t stride = (int64_t)pl.m_tiles * 128 * pl.n_t;
-    for (int ch = 0; ch < pl.n_chunks; ++ch) s += p[ch * stride];
+    int ch = 0;
+    for (; ch + 8 <= pl.n_chunks; ch += 8) {   // eight loads in flight, summed in chunk order
+        float v[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) v[q] = __ldg(p + (ch + q) * stride);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) s += v[q];
+    }
+    for (; ch < pl.n_chunks; ++ch) s += __ldg(p + ch * stride);
     dW[i] = s;
 }
 
