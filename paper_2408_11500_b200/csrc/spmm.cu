@@ -7,7 +7,6 @@
 // flight per lane.  No per-edge value array exists:  A_hat_ij = dinv_i * dinv_j.
 // Rows longer than kLongRow are cut into kSegment-entry segments, one warp each, whose partial
 // rows are summed afterwards in segment order -- deterministic, no floating-point atomics.
-#include <cstdlib>
 #include <vector>
 
 #include "common.cuh"
@@ -170,7 +169,7 @@ __device__ __forceinline__ void finish_chunk(const SpmmParams& p, int64_t row, i
 constexpr int kRowsWarps = 4;   // warps per CTA of the row kernel
 
 template <typename TI, typename TO, int L, int C, bool EPI>
-__global__ void __launch_bounds__(kRowsWarps * 32, 20 / kRowsWarps) spmm_rows_kernel(const SpmmParams p) {
+__device__ __forceinline__ void spmm_rows_block(const SpmmParams& p, const int64_t vblock) {
     constexpr int V = Vec<TI>::V;
     constexpr int RPW = 32 / L;
     constexpr int U = (8 / C) < 2 ? 2 : (8 / C);   // neighbors gathered per round: U*C 16-byte loads per lane
@@ -179,7 +178,7 @@ __global__ void __launch_bounds__(kRowsWarps * 32, 20 / kRowsWarps) spmm_rows_ke
     __shared__ int2 nbuf[kRowsWarps][32];
     const int lane = threadIdx.x & 31;
     const int sub = lane / L, sl = lane % L;
-    const int64_t warp = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
+    const int64_t warp = (vblock * (int64_t)blockDim.x + threadIdx.x) >> 5;
     const int64_t chunk = warp * RPW + sub;
     if (chunk >= p.n_chunks) return;
     const unsigned gmask = (L == 32) ? 0xffffffffu : (((1u << L) - 1u) << (sub * L));
@@ -296,240 +295,14 @@ __global__ void __launch_bounds__(kRowsWarps * 32, 20 / kRowsWarps) spmm_rows_ke
     }
 }
 
-// ---------------------------------------------------------------------------------------------
-// Wide rows (a row of the operand is at least 512 bytes): neighbor rows are staged in shared memory
-// by asynchronous 16-byte copies (cp.async) instead of being held in registers, so the number of
-// rows a warp keeps in flight is set by shared memory, not by the register file.  Each warp runs its
-// own ring of kRingStages stages; a stage holds the operand rows of the next S entries of the warp's
-// work list and is one cp.async group, so a warp has (kRingStages-1)*S rows in flight while it
-// reduces the stage that has landed.  Work is the same row-aligned chunk list as above, dealt to
-// warps round-robin; in SEG mode the work items are the segments of the long rows and the result
-// goes to the partial-row buffer.  Row ends and 1/sqrt(deg) of 32 consecutive rows are fetched by
-// the 32 lanes at once and handed out by shuffles, so closing a row costs no memory round trip.
-constexpr int kRingWarps = 12;
-constexpr int kRingStages = 4;
-constexpr int kRingStageBytes = 4096;
-constexpr int kRingSmem = kRingWarps * kRingStages * kRingStageBytes;
-
-__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void cp_async16(void* dst, const void* src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_addr(dst)), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() {
-    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
-}
-
-// Entry range and rows of work item ci.  Returns false when the item holds nothing for this kernel.
-template <bool SEG>
-__device__ __forceinline__ bool item_range(const SpmmParams& p, int ci, int& r0, int& r1, int& lo, int& hi) {
-    if (SEG) {
-        const int li = __ldg(p.seg_row + ci);
-        const int r = __ldg(p.long_rows + li);
-        lo = __ldg(p.rowptr + r) + (ci - __ldg(p.seg_ptr + li)) * kSegment;
-        hi = min(__ldg(p.rowptr + r + 1), lo + kSegment);
-        r0 = ci;
-        r1 = ci + 1;
-        return true;
-    }
-    r0 = __ldg(p.chunk_row + ci);
-    r1 = __ldg(p.chunk_row + ci + 1);
-    if (r0 >= r1) return false;
-    lo = __ldg(p.rowptr + r0);
-    hi = __ldg(p.rowptr + r1);
-    if (__ldg(p.rowptr + r0 + 1) - lo > kLongRow) return false;   // a long row: segment pass
-    return true;
-}
-
-template <typename TI, typename TO, int C, bool EPI, bool SEG>
-__global__ void __launch_bounds__(kRingWarps * 32, 1) spmm_ring_kernel(const SpmmParams p, const int S) {
-    constexpr int V = Vec<TI>::V;
-    extern __shared__ __align__(1024) unsigned char smem[];
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    unsigned char* wbase = smem + warp * (kRingStages * kRingStageBytes);
-    const int W = gridDim.x * kRingWarps;
-    const int n_items = SEG ? p.n_seg : p.n_chunks;
-    const uint32_t rowbytes = (uint32_t)p.nch * 16u;
-    const unsigned char* Xb = static_cast<const unsigned char*>(p.X);
-    const int64_t pitch = p.ldx * (int64_t)sizeof(TI);
-
-    // ---- producer cursor: entries [pk, pk_end) of item pci still to be fetched
-    int pci = blockIdx.x * kRingWarps + warp - W;
-    int pk = 0, pk_end = 0;
-    bool p_live = true;
-    auto prod_next = [&]() {
-        for (;;) {
-            pci += W;
-            if (pci >= n_items) {
-                p_live = false;
-                pk = pk_end = 0;
-                return;
-            }
-            int r0, r1, lo, hi;
-            if (item_range<SEG>(p, pci, r0, r1, lo, hi) && hi > lo) {
-                pk = lo;
-                pk_end = hi;
-                return;
-            }
-        }
-    };
-    prod_next();
-    int jn = 0;   // column index lane t holds for entry pk + t of the next fill
-    if (p_live && lane < min(S, pk_end - pk)) jn = __ldg(p.colidx + pk + lane);
-
-    float djr[kRingStages];
-    int cntr[kRingStages];
-    auto fill = [&](int s) {
-        const int cnt = p_live ? min(S, pk_end - pk) : 0;
-        cntr[s] = cnt;
-        djr[s] = 0.f;
-        if (cnt > 0) {
-            unsigned char* stage = wbase + s * kRingStageBytes;
-            for (int t = 0; t < cnt; ++t) {
-                const int jj = __shfl_sync(0xffffffffu, jn, t);
-                const unsigned char* src = Xb + (int64_t)jj * pitch;
-#pragma unroll
-                for (int c = 0; c < C; ++c) {
-                    const int ch = lane + c * 32;
-                    if (ch < p.nch) cp_async16(stage + t * rowbytes + ch * 16, src + ch * 16);
-                }
-            }
-            if (lane < cnt) djr[s] = __ldg(p.dinv + jn);
-            pk += cnt;
-            if (pk == pk_end) prod_next();
-            if (p_live && lane < min(S, pk_end - pk)) jn = __ldg(p.colidx + pk + lane);
-        }
-        cp_async_commit();   // one group per fill, empty or not, so the group count stays in step
-    };
-
-    // ---- consumer cursor
-    int cci = blockIdx.x * kRingWarps + warp - W;
-    int row = 0, r_end = 0, kk = 0, row_end = 0;
-    int rbase = 0, rp_l = 0;   // lane t: rowptr[rbase + 1 + t]
-    float di_l = 0.f;          // lane t: dinv[rbase + t]
-    bool finished = false;
-    float acc[C][V];
-#pragma unroll
-    for (int c = 0; c < C; ++c)
-#pragma unroll
-        for (int e = 0; e < V; ++e) acc[c][e] = 0.f;
-
-    auto load_row_meta = [&]() {   // rows [row, row+32) of the current item
-        rbase = row;
-        const int r = row + lane;
-        rp_l = r < r_end ? __ldg(p.rowptr + r + 1) : 0;
-        di_l = r < r_end ? __ldg(p.dinv + r) : 0.f;
-    };
-    auto flush = [&]() {
-        if (SEG) {
-            float* out = p.partial + (int64_t)row * (p.nch * V);
-#pragma unroll
-            for (int c = 0; c < C; ++c) {
-                const int ch = lane + c * 32;
-                if (ch < p.nch) {
-#pragma unroll
-                    for (int e = 0; e < V; e += 4)
-                        *reinterpret_cast<float4*>(out + ch * V + e) =
-                            make_float4(acc[c][e], acc[c][e + 1], acc[c][e + 2], acc[c][e + 3]);
-                }
-#pragma unroll
-                for (int e = 0; e < V; ++e) acc[c][e] = 0.f;
-            }
-        } else {
-            const float di = __shfl_sync(0xffffffffu, di_l, row - rbase);
-#pragma unroll
-            for (int c = 0; c < C; ++c) {
-                const int ch = lane + c * 32;
-                if (ch < p.nch) finish_chunk<TO, V, EPI>(p, row, ch, di, acc[c]);
-#pragma unroll
-                for (int e = 0; e < V; ++e) acc[c][e] = 0.f;
-            }
-        }
-    };
-    // closes every row that ends at kk; moves on to the next item when the current one is done
-    auto close_rows = [&]() {
-        while (!finished && kk == row_end) {
-            if (row < r_end) {
-                flush();
-                ++row;
-            }
-            if (row >= r_end) {
-                for (;;) {
-                    cci += W;
-                    if (cci >= n_items) {
-                        finished = true;
-                        break;
-                    }
-                    int r0, r1, lo, hi;
-                    if (item_range<SEG>(p, cci, r0, r1, lo, hi)) {
-                        row = r0;
-                        r_end = r1;
-                        kk = lo;
-                        if (SEG) {
-                            row_end = hi;
-                        } else {
-                            load_row_meta();
-                            row_end = __shfl_sync(0xffffffffu, rp_l, 0);
-                        }
-                        break;
-                    }
-                }
-            } else {
-                if (row - rbase == 32) load_row_meta();
-                row_end = __shfl_sync(0xffffffffu, rp_l, row - rbase);
-            }
-        }
-    };
-
-#pragma unroll
-    for (int s = 0; s < kRingStages; ++s) fill(s);
-    close_rows();   // positions the consumer on its first item (and writes leading empty rows)
-
-    while (!finished) {
-#pragma unroll
-        for (int s = 0; s < kRingStages; ++s) {
-            if (finished) break;
-            const int cnt = cntr[s];
-            if (cnt == 0) {   // producer ran dry: close_rows() has already written whatever remained
-                finished = true;
-                break;
-            }
-            cp_async_wait<kRingStages - 1>();   // this stage's group has landed (newer ones may be pending)
-            __syncwarp();
-            const unsigned char* stage = wbase + s * kRingStageBytes;
-            for (int t = 0; t < cnt; ++t) {
-                if (kk == row_end) close_rows();
-                const float dd = __shfl_sync(0xffffffffu, djr[s], t);
-#pragma unroll
-                for (int c = 0; c < C; ++c) {
-                    const int ch = lane + c * 32;
-                    if (ch < p.nch) {
-                        const uint4 raw = *reinterpret_cast<const uint4*>(stage + t * rowbytes + ch * 16);
-                        float f[V];
-                        Vec<TI>::unpack(raw, f);
-#pragma unroll
-                        for (int e = 0; e < V; ++e) acc[c][e] = fmaf(dd, f[e], acc[c][e]);
-                    }
-                }
-                ++kk;
-            }
-            if (kk == row_end) close_rows();
-            __syncwarp();     // every lane is done reading the stage before it is refilled
-            fill(s);
-        }
-    }
-    cp_async_wait<0>();
-}
-
 // One warp per segment of a long row; the 32/L lane groups interleave over the segment's
 // neighbors and are combined with a butterfly (fixed order).
 template <typename TI, int L, int C>
-__global__ void __launch_bounds__(256) spmm_segment_kernel(const SpmmParams p) {
+__device__ __forceinline__ void spmm_segment_block(const SpmmParams& p, const int64_t vblock) {
     constexpr int V = Vec<TI>::V;
     const int lane = threadIdx.x & 31;
     const int sub = lane / L, sl = lane % L;
-    const int seg = (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5);
+    const int seg = (int)((vblock * (int64_t)blockDim.x + threadIdx.x) >> 5);
     if (seg >= p.n_seg) return;
     const unsigned gmask = (L == 32) ? 0xffffffffu : (((1u << L) - 1u) << (sub * L));
     const int li = __ldg(p.seg_row + seg);
@@ -571,6 +344,16 @@ __global__ void __launch_bounds__(256) spmm_segment_kernel(const SpmmParams p) {
             }
         }
     }
+}
+
+// One launch for both kinds of work: the first seg_blocks CTAs reduce the segments of the long rows
+// (they are the heaviest items, so they start first), the others the row chunks.
+template <typename TI, typename TO, int L, int C, bool EPI>
+__global__ void __launch_bounds__(kRowsWarps * 32, 20 / kRowsWarps) spmm_rows_kernel(const SpmmParams p, const int seg_blocks) {
+    if ((int)blockIdx.x < seg_blocks)
+        spmm_segment_block<TI, L, C>(p, blockIdx.x);
+    else
+        spmm_rows_block<TI, TO, L, C, EPI>(p, (int64_t)blockIdx.x - seg_blocks);
 }
 
 // Sums the partial rows of each long row in segment order, then scales / applies the epilogue.
@@ -642,66 +425,21 @@ slicegcn_status_t launch_lc(const SpmmParams& p, bool epi, cudaStream_t st) {
     constexpr int RPW = 32 / L;
     const int64_t warps = ((int64_t)p.n_chunks + RPW - 1) / RPW;
     const int64_t blocks = (warps + kRowsWarps - 1) / kRowsWarps;
+    const int seg_blocks = (p.n_seg + kRowsWarps - 1) / kRowsWarps;
     if (epi)
-        spmm_rows_kernel<TI, TO, L, C, true><<<(unsigned)blocks, kRowsWarps * 32, 0, st>>>(p);
+        spmm_rows_kernel<TI, TO, L, C, true><<<(unsigned)(blocks + seg_blocks), kRowsWarps * 32, 0, st>>>(p, seg_blocks);
     else
-        spmm_rows_kernel<TI, TO, L, C, false><<<(unsigned)blocks, kRowsWarps * 32, 0, st>>>(p);
+        spmm_rows_kernel<TI, TO, L, C, false><<<(unsigned)(blocks + seg_blocks), kRowsWarps * 32, 0, st>>>(p, seg_blocks);
     SGCN_LAUNCH_CHECK();
     count_launch();
     if (p.n_seg > 0) {
-        spmm_segment_kernel<TI, L, C><<<(p.n_seg + 7) / 8, 256, 0, st>>>(p);
-        SGCN_LAUNCH_CHECK();
         const int pstride = p.nch * Vec<TI>::V;
         if (epi)
             spmm_long_finish_kernel<TO, true><<<(p.n_long + 7) / 8, 256, 0, st>>>(p, pstride);
         else
             spmm_long_finish_kernel<TO, false><<<(p.n_long + 7) / 8, 256, 0, st>>>(p, pstride);
         SGCN_LAUNCH_CHECK();
-        count_launch(2);
-    }
-    return SLICEGCN_OK;
-}
-
-template <typename TI, typename TO, int C>
-slicegcn_status_t launch_bulk(const SpmmParams& p, bool epi, int* fault, cudaStream_t st) {
-    static bool configured = false;
-    if (!configured) {
-        SGCN_CUDA(cudaFuncSetAttribute(spmm_ring_kernel<TI, TO, C, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingSmem));
-        SGCN_CUDA(cudaFuncSetAttribute(spmm_ring_kernel<TI, TO, C, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingSmem));
-        SGCN_CUDA(cudaFuncSetAttribute(spmm_ring_kernel<TI, TO, C, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingSmem));
-        configured = true;
-    }
-    const int rowbytes = p.nch * 16;
-    int S = kRingStageBytes / rowbytes;
-    if (S > 32) S = 32;
-    if (S < 1) S = 1;
-    int sms = 148;
-    {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        int v = 0;
-        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) sms = v;
-    }
-    int grid = (p.n_chunks + kRingWarps - 1) / kRingWarps;
-    if (grid > sms) grid = sms;
-    if (epi)
-        spmm_ring_kernel<TI, TO, C, true, false><<<grid, kRingWarps * 32, kRingSmem, st>>>(p, S);
-    else
-        spmm_ring_kernel<TI, TO, C, false, false><<<grid, kRingWarps * 32, kRingSmem, st>>>(p, S);
-    SGCN_LAUNCH_CHECK();
-    count_launch();
-    if (p.n_seg > 0) {
-        int sgrid = (p.n_seg + kRingWarps - 1) / kRingWarps;
-        if (sgrid > sms) sgrid = sms;
-        spmm_ring_kernel<TI, TO, C, false, true><<<sgrid, kRingWarps * 32, kRingSmem, st>>>(p, S);
-        SGCN_LAUNCH_CHECK();
-        const int pstride = p.nch * Vec<TI>::V;
-        if (epi)
-            spmm_long_finish_kernel<TO, true><<<(p.n_long + 7) / 8, 256, 0, st>>>(p, pstride);
-        else
-            spmm_long_finish_kernel<TO, false><<<(p.n_long + 7) / 8, 256, 0, st>>>(p, pstride);
-        SGCN_LAUNCH_CHECK();
-        count_launch(2);
+        count_launch();
     }
     return SLICEGCN_OK;
 }
@@ -709,13 +447,7 @@ slicegcn_status_t launch_bulk(const SpmmParams& p, bool epi, int* fault, cudaStr
 template <typename TI, typename TO>
 slicegcn_status_t launch_vec(const SpmmParams& p, bool epi, int* fault, cudaStream_t st) {
     const int nch = p.nch;
-    static const bool use_ring = getenv("SLICEGCN_SPMM_RING") != nullptr;   // experimental staged variant
-    if (use_ring && nch >= 32) {
-        if (nch <= 32) return launch_bulk<TI, TO, 1>(p, epi, fault, st);
-        if (nch <= 64) return launch_bulk<TI, TO, 2>(p, epi, fault, st);
-        if (nch <= 96) return launch_bulk<TI, TO, 3>(p, epi, fault, st);
-        return launch_bulk<TI, TO, 4>(p, epi, fault, st);
-    }
+    (void)fault;
     if (nch <= 2) return launch_lc<TI, TO, 2, 1>(p, epi, st);
     if (nch <= 4) return launch_lc<TI, TO, 4, 1>(p, epi, st);
     if (nch <= 8) return launch_lc<TI, TO, 8, 1>(p, epi, st);
