@@ -29,7 +29,7 @@ from paper_2408_11500_b200 import synth  # noqa: E402
 
 # dram__bytes_read.sum + dram__bytes_write.sum per SpMM launch from the ncu capture summarised under
 # profiles/ (None until a capture of that workload exists)
-NCU_SPMM_TRAFFIC_BYTES = {"citation": None}
+NCU_SPMM_TRAFFIC_BYTES = {"citation": 943e6}   # width-256 launches (4 of the 5 per epoch)
 
 
 def measured_peak_gbs():
@@ -46,6 +46,7 @@ class ClockSampler:
 
     def __init__(self, index: int):
         self.index, self.rows, self.proc = index, [], None
+        self.t0 = self.t1 = None          # the timed region; only samples taken inside it are used
 
     def start(self):
         try:
@@ -59,7 +60,13 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append([t.strip() for t in line.split(",")])
+            self.rows.append((time.time(), [t.strip() for t in line.split(",")]))
+
+    def mark_begin(self):
+        self.t0 = time.time()
+
+    def mark_end(self):
+        self.t1 = time.time()
 
     def stop(self):
         if self.proc is None:
@@ -71,7 +78,8 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, reasons = [], None, set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
+        inside = [r for (t, r) in self.rows if self.t0 is not None and self.t0 <= t <= (self.t1 or t) + 0.15]
+        for r in (inside if inside else [r for (_, r) in self.rows[-3:]]):
             if len(r) < 6:
                 continue
             try:
@@ -201,11 +209,12 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         return float(t.item())
 
     # ---- device-resident run
+    sampler = ClockSampler(local_rank)
+    sampler.start()
     for ep in range(args.warmup):
         epoch(ep, X, y)
     barrier()
-    sampler = ClockSampler(local_rank)
-    sampler.start()
+    sampler.mark_begin()
     B.slicegcn_profile_begin()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
@@ -213,6 +222,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         epoch(args.warmup + ep, X, y)
     e1.record(stream)
     barrier()
+    sampler.mark_end()
     prof = B.slicegcn_profile_end()
     clocks = sampler.stop()
     ms_total = max_over_ranks(e0.elapsed_time(e1))
@@ -285,7 +295,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="citation", choices=sorted(synth.WORKLOADS))
