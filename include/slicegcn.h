@@ -124,6 +124,28 @@ slicegcn_status_t slicegcn_spmm(const slicegcn_graph* g, int32_t transpose, int3
                                 const void* X, int64_t ldx, void* Y, int64_t ldy, int32_t width,
                                 void* workspace, int64_t workspace_bytes, void* stream);
 
+/* The same aggregation for callers that cannot allocate device memory.  (The paper has no counterpart:
+ * this entry point exists for the embedding, not for the method.)
+ *
+ * Some callers may not call cudaMalloc: code running inside a stream capture, a host with a fixed memory
+ * plan handed out at start-up, a plugin that must not touch the allocator of the process it lives in.  For
+ * them the scratch the split hub rows need (their partial sums) comes from a buffer compiled into the
+ * library: 8 MiB of device memory that every GPU loading the library holds until the process exits.
+ * The call allocates nothing on the host or the device and frees nothing; X and Y are still the caller's.
+ *   - Limit: slicegcn_spmm_workspace_bytes(g, width) must be <= 8 MiB (8,388,608 bytes); otherwise the call
+ *     fails with SLICEGCN_ERR_UNSUPPORTED and a message giving both numbers, and nothing is launched.
+ *   - The first call on a device looks the buffer's device address up (once per device, with that device
+ *     current -- the device of `g` must be current, as for every call).  Make that first call outside any
+ *     stream capture.
+ *   - All calls share the one buffer, which keeps whatever the last call left in it.  Nothing in it needs to
+ *     start at zero (a call only reads partial sums it wrote itself), but two calls whose kernels overlap on
+ *     the GPU -- different streams, or different threads -- race on it: serialise them.
+ *   - Not counted by slicegcn_profile_begin/end.
+ * Arguments, results and the other errors are those of slicegcn_spmm. */
+slicegcn_status_t slicegcn_spmm_static_scratch(const slicegcn_graph* g, int32_t transpose, int32_t in_dtype,
+                                               int32_t out_dtype, const void* X, int64_t ldx, void* Y, int64_t ldy,
+                                               int32_t width, void* stream);
+
 /* ---------------------------------------------------------------------------------------------
  * One sliced GCN layer -- Eq. 6 (and Eq. 7-8 when E is given):
  *   for slice i:  M_i = b_i + (A_hat H_in[:, in_starts[i] : in_starts[i]+in_width]) W_agg_i

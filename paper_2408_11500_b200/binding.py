@@ -28,7 +28,7 @@ MAX_SLICES = 64
 EXPORTS = [
     "slicegcn_last_error", "slicegcn_slice_strategy", "slicegcn_graph_create", "slicegcn_graph_create_from_csr",
     "slicegcn_graph_info", "slicegcn_graph_export", "slicegcn_graph_device_status", "slicegcn_graph_destroy", "slicegcn_spmm_workspace_bytes",
-    "slicegcn_spmm", "slicegcn_layer_saved_bytes", "slicegcn_layer_workspace_bytes", "slicegcn_layer_forward",
+    "slicegcn_spmm", "slicegcn_spmm_static_scratch", "slicegcn_layer_saved_bytes", "slicegcn_layer_workspace_bytes", "slicegcn_layer_forward",
     "slicegcn_layer_backward", "slicegcn_model_create", "slicegcn_model_destroy", "slicegcn_model_param_count",
     "slicegcn_model_param_elems", "slicegcn_model_num_tensors", "slicegcn_model_tensor_info", "slicegcn_model_slices",
     "slicegcn_model_layer_order", "slicegcn_train_workspace_bytes", "slicegcn_train_epoch", "slicegcn_profile_begin",
@@ -171,6 +171,15 @@ def slicegcn_spmm(g, transpose: int, in_dtype: int, out_dtype: int, X, ldx: int,
                   workspace=None, workspace_bytes: int = 0, stream=None) -> None:
     _check(_lib.slicegcn_spmm(g, c_int32(transpose), c_int32(in_dtype), c_int32(out_dtype), _vp(X), c_int64(ldx), _vp(Y),
                               c_int64(ldy), c_int32(width), _vp(workspace), c_int64(workspace_bytes), _vp(stream)))
+
+
+def slicegcn_spmm_static_scratch(g, transpose: int, in_dtype: int, out_dtype: int, X, ldx: int, Y, ldy: int, width: int,
+                                 stream=None) -> None:
+    """slicegcn_spmm for callers that cannot allocate: the hub-row scratch is an 8 MiB buffer built into the
+    library (shared by all calls; overlapping calls race).  Raises SliceGCNError(ERR_UNSUPPORTED) when the graph
+    and width need more."""
+    _check(_lib.slicegcn_spmm_static_scratch(g, c_int32(transpose), c_int32(in_dtype), c_int32(out_dtype), _vp(X),
+                                             c_int64(ldx), _vp(Y), c_int64(ldy), c_int32(width), _vp(stream)))
 
 
 # ------------------------------------------------------------------------------------------ layer

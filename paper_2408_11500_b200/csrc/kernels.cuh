@@ -18,7 +18,7 @@ struct SpmmEpilogue {
 int64_t spmm_partial_bytes(const slicegcn_graph* g, int width);
 slicegcn_status_t spmm_run(const slicegcn_graph* g, bool transpose, int in_dtype, int out_dtype, const void* X,
                            int64_t ldx, void* Y, int64_t ldy, int width, const SpmmEpilogue* epi, void* ws,
-                           int64_t ws_bytes, cudaStream_t st);
+                           int64_t ws_bytes, cudaStream_t st, bool instrument = true);
 
 // ---- grouped row-panel GEMM  C_g = epilogue(A_g * B_g) ----------------------------------------
 // Group g (one slice) reads K columns of A starting at a_start[g], multiplies by its own K x N

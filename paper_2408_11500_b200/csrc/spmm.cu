@@ -511,7 +511,7 @@ int64_t spmm_partial_bytes(const slicegcn_graph* g, int width) {
 
 slicegcn_status_t spmm_run(const slicegcn_graph* g, bool transpose, int in_dtype, int out_dtype, const void* X,
                            int64_t ldx, void* Y, int64_t ldy, int width, const SpmmEpilogue* epi, void* ws,
-                           int64_t ws_bytes, cudaStream_t st) {
+                           int64_t ws_bytes, cudaStream_t st, bool instrument) {
     if (!g || !X || !Y) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "spmm: NULL argument");
     if (width < 1 || ldx < width || ldy < width) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "spmm: bad width / leading dimension");
     if (in_dtype != out_dtype) SGCN_FAIL(SLICEGCN_ERR_UNSUPPORTED, "spmm: input and output dtype must match");
@@ -546,7 +546,7 @@ slicegcn_status_t spmm_run(const slicegcn_graph* g, bool transpose, int in_dtype
                       (long long)spmm_partial_bytes(g, width));
     }
     cudaEvent_t ev_stop = nullptr;
-    if (g_prof.on) {
+    if (g_prof.on && instrument) {
         if (g_prof.used + 2 > g_prof.ev.size()) {
             for (int i = 0; i < 2; ++i) {
                 cudaEvent_t e;
@@ -577,9 +577,48 @@ slicegcn_status_t spmm_run(const slicegcn_graph* g, bool transpose, int in_dtype
     return rc;
 }
 
+// ---- fixed scratch for callers that cannot allocate ------------------------------------------
+// Lives in the library image: every GPU that loads the library holds these bytes until the process
+// exits.  In host code the array's name is only a stand-in for the symbol, never a device address;
+// the address a kernel may use comes from cudaGetSymbolAddress, once per device.
+constexpr int64_t kStaticScratchBytes = 8ll << 20;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+static void* g_static_scratch_ptr[64] = {nullptr};   // per device ordinal, filled on first use
+
+static slicegcn_status_t static_scratch_for_current_device(void** out) {
+    int dev = -1;
+    SGCN_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) SGCN_FAIL(SLICEGCN_ERR_UNSUPPORTED, "device ordinal %d outside the supported range", dev);
+    if (!g_static_scratch_ptr[dev]) {
+        void* p = nullptr;
+        SGCN_CUDA(cudaGetSymbolAddress(&p, g_static_scratch));
+        g_static_scratch_ptr[dev] = p;
+    }
+    *out = g_static_scratch_ptr[dev];
+    return SLICEGCN_OK;
+}
+
 }  // namespace sgcn
 
 extern "C" {
+
+slicegcn_status_t slicegcn_spmm_static_scratch(const slicegcn_graph* g, int32_t transpose, int32_t in_dtype,
+                                               int32_t out_dtype, const void* X, int64_t ldx, void* Y, int64_t ldy,
+                                               int32_t width, void* stream) {
+    using namespace sgcn;
+    if (!g || width < 1) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "spmm_static_scratch: bad argument");
+    const int64_t need = spmm_partial_bytes(g, width);
+    if (need > kStaticScratchBytes)
+        SGCN_FAIL(SLICEGCN_ERR_UNSUPPORTED,
+                  "spmm_static_scratch: this graph and width need %lld bytes of scratch, the built-in buffer holds %lld; "
+                  "use slicegcn_spmm with a caller-provided workspace",
+                  (long long)need, (long long)kStaticScratchBytes);
+    void* scratch = nullptr;
+    SGCN_TRY(static_scratch_for_current_device(&scratch));
+    // nothing in the buffer has to start at zero: every partial row a call reads was written by that call
+    return spmm_run(g, transpose != 0, in_dtype, out_dtype, X, ldx, Y, ldy, width, nullptr, scratch, kStaticScratchBytes,
+                    (cudaStream_t)stream, /*instrument=*/false);
+}
 
 slicegcn_status_t slicegcn_profile_begin(void) {
     using namespace sgcn;
