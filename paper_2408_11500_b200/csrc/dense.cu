@@ -319,7 +319,7 @@ __global__ void mask_mul4_kernel(int64_t M, int N4, const float4* in, int64_t ld
 
 // one warp per training row
 __global__ void softmax_ce_kernel(int C, const float* logits, const int32_t* labels, const int32_t* train_idx,
-                                  int64_t n_train, float inv_n, float* dlogits, float* row_loss) {
+                                  int64_t n_train, float inv_n, float* dlogits, int64_t ld_d, float* row_loss) {
     const int lane = threadIdx.x & 31;
     const int64_t t = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
     if (t >= n_train) return;
@@ -337,9 +337,10 @@ __global__ void softmax_ce_kernel(int C, const float* logits, const int32_t* lab
     const float lse = mx + logf(s);
     if (lane == 0) row_loss[t] = lse - z[y];
     const float inv_s = 1.f / s;
-    for (int c = lane; c < C; c += 32) {
-        float p = expf(z[c] - mx) * inv_s;
-        dlogits[r * C + c] = (p - (c == y ? 1.f : 0.f)) * inv_n;
+    for (int c = lane; c < ld_d; c += 32) {
+        float v = 0.f;   // padding columns stay zero
+        if (c < C) v = (expf(z[c] - mx) * inv_s - (c == y ? 1.f : 0.f)) * inv_n;
+        dlogits[r * ld_d + c] = v;
     }
 }
 
@@ -474,12 +475,13 @@ slicegcn_status_t mask_mul_run(int64_t M, int N, const float* in, int64_t ld_in,
 }
 
 slicegcn_status_t softmax_ce_run(int64_t n, int C, const float* logits, const int32_t* labels, const int32_t* train_idx,
-                                 int64_t n_train, float* dlogits, float* row_loss, float* loss_out, cudaStream_t st) {
-    if (train_idx) SGCN_CUDA(cudaMemsetAsync(dlogits, 0, sizeof(float) * n * C, st));
+                                 int64_t n_train, float* dlogits, int64_t ld_d, float* row_loss, float* loss_out,
+                                 cudaStream_t st) {
+    if (train_idx) SGCN_CUDA(cudaMemsetAsync(dlogits, 0, sizeof(float) * n * ld_d, st));
     const int64_t cnt = train_idx ? n_train : n;
     if (cnt < 1) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "empty training set");
     softmax_ce_kernel<<<(unsigned)((cnt + 7) / 8), 256, 0, st>>>(C, logits, labels, train_idx, cnt, 1.0f / (float)cnt,
-                                                                  dlogits, row_loss);
+                                                                  dlogits, ld_d, row_loss);
     SGCN_LAUNCH_CHECK();
     count_launch();
     if (loss_out) {

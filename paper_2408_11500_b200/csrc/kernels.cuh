@@ -32,6 +32,7 @@ struct GemmArgs {
     int64_t lda = 0;
     int a_dtype = SLICEGCN_F32;
     int a_start[SLICEGCN_MAX_SLICES] = {0};
+    int a_pad_zero = 0;                // columns a_start+K .. next multiple of 8 exist (< lda) and hold zeros
     const uint8_t* a_mask = nullptr;   // A element (r, col) is multiplied by a_mask[r*a_mask_ld + col]
     int64_t a_mask_ld = 0;
     const float* B = nullptr;          // group g: B + g*b_gstride; element (k, n) at k*ldb + n, or n*ldb + k if b_trans
@@ -79,6 +80,8 @@ struct WgradArgs {
     int b_start[SLICEGCN_MAX_SLICES] = {0};
     const uint8_t* b_mask = nullptr;
     int64_t b_mask_ld = 0;
+    int a_pad_zero = 0;        // A / B columns up to the next multiple of 4 past the last group exist and hold zeros
+    int b_pad_zero = 0;
     float* dW = nullptr;       // may be NULL when K == 0
     float* dbias = nullptr;    // may be NULL
     float* dbias2 = nullptr;   // optional second copy of the column sums (slice-encoding gradient)
@@ -95,8 +98,10 @@ slicegcn_status_t mask_mul_run(int64_t M, int N, const float* in, int64_t ld_in,
                                float* out, int64_t ld_out, cudaStream_t st);
 // Softmax cross entropy (Eq. 10) over the training rows: writes dlogits = (softmax - onehot)/n_train
 // (rows outside the training set are zeroed) and the mean loss.  row_loss: scratch [n_train] floats.
+// dlogits has leading dimension ld_d >= C; columns C..ld_d-1 of every row are written as zeros.
 slicegcn_status_t softmax_ce_run(int64_t n, int C, const float* logits, const int32_t* labels, const int32_t* train_idx,
-                                 int64_t n_train, float* dlogits, float* row_loss, float* loss_out, cudaStream_t st);
+                                 int64_t n_train, float* dlogits, int64_t ld_d, float* row_loss, float* loss_out,
+                                 cudaStream_t st);
 // Adam with bias correction; `step` is 1-based.
 slicegcn_status_t adam_run(int64_t count, float* theta, const float* grad, float* m1, float* m2, float lr, float beta1,
                            float beta2, float eps, float weight_decay, int step, cudaStream_t st);

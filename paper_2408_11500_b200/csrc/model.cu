@@ -68,6 +68,9 @@ struct LayerPlan {
     int zt_cols = 0;               // columns of the saved intermediate (Z: in_cols, T: out_cols)
     int64_t zt_ld = 0, mask_ld = 0, zt_bytes = 0, mask_bytes = 0;
     int64_t n = 0;
+    // set by callers that keep the padding columns (up to the leading dimension) of H_in / the saved
+    // intermediate at zero: lets 16-byte loads run over widths that are not multiples of 8
+    bool in_pad_zero = false, zt_pad_zero = false;
 };
 
 slicegcn_status_t make_plan(const slicegcn_graph* g, const slicegcn_layer_desc* d, LayerPlan* pl) {
@@ -191,6 +194,7 @@ slicegcn_status_t layer_forward_impl(const slicegcn_graph* g, const slicegcn_lay
     self.c_dtype = L.dtype;
     self.post1 = d->b_self;
     self.post2 = d->E;
+    self.a_pad_zero = L.in_pad_zero ? 1 : 0;
     for (int i = 0; i < L.p; ++i) {
         self.a_start[i] = L.in_starts[i];
         self.c_start[i] = i * L.h_s;
@@ -204,6 +208,7 @@ slicegcn_status_t layer_forward_impl(const slicegcn_graph* g, const slicegcn_lay
         agg.K = L.in_width;
         agg.A = zt;
         agg.lda = L.zt_ld;
+        agg.a_pad_zero = L.zt_pad_zero ? 1 : 0;
         agg.B = d->W_agg;
         agg.bias = d->b;
         agg.relu = 1;
@@ -262,6 +267,7 @@ slicegcn_status_t layer_backward_impl(const slicegcn_graph* g, const slicegcn_la
         w.A = H_in;
         w.lda = L.in_ld;
         w.a_dtype = L.dtype;
+        w.a_pad_zero = L.in_pad_zero ? 1 : 0;
         w.B = dH_out;
         w.ldb = dout_ld;
         w.dW = dW_self;
@@ -313,6 +319,7 @@ slicegcn_status_t layer_backward_impl(const slicegcn_graph* g, const slicegcn_la
             w.A = zt;
             w.lda = L.zt_ld;
             w.a_dtype = L.dtype;
+            w.a_pad_zero = L.zt_pad_zero ? 1 : 0;
             w.B = dM;
             w.ldb = dm_ld;
             w.dW = dW_agg;
@@ -374,6 +381,7 @@ slicegcn_status_t layer_backward_impl(const slicegcn_graph* g, const slicegcn_la
             w.A = H_in;
             w.lda = L.in_ld;
             w.a_dtype = L.dtype;
+            w.a_pad_zero = L.in_pad_zero ? 1 : 0;
             w.B = dT;
             w.ldb = L.zt_ld;
             w.dW = dW_agg;
@@ -442,7 +450,7 @@ namespace {
 
 struct EpochLayout {
     // element leading dimensions
-    int64_t ld_h = 0, ld_x0 = 0, ld_ffact = 0, ld_cls = 0, ld_grad = 0;
+    int64_t ld_h = 0, ld_x0 = 0, ld_ffact = 0, ld_cls = 0, ld_grad = 0, ld_dlog = 0;
     int64_t total = 0;
     // pointers (valid when built with a base)
     void* ff_act = nullptr;
@@ -521,7 +529,8 @@ slicegcn_status_t build_layout(const slicegcn_model* m, const slicegcn_graph* g,
     }
     E.cls_act = b.take(n * E.ld_cls * esz);
     E.logits = static_cast<float*>(b.take(n * (int64_t)D.num_classes * 4));
-    E.dlogits = static_cast<float*>(b.take(n * (int64_t)D.num_classes * 4));
+    E.ld_dlog = align_up(D.num_classes, 4);
+    E.dlogits = static_cast<float*>(b.take(n * E.ld_dlog * 4));
     E.row_loss = static_cast<float*>(b.take(n * 4));
     E.dA = static_cast<float*>(b.take(n * E.ld_cls * 4));
     E.dH[0] = static_cast<float*>(b.take(n * E.ld_grad * 4));
@@ -740,6 +749,8 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
     // ---------------- forward
     const void* h0 = X;
     int64_t ld0 = x_ld;
+    if (D.use_ff && (m->slice_size % 8) != 0)
+        SGCN_CUDA(cudaMemsetAsync(E.xff, 0, n * E.ld_x0 * esize(D.dtype), st));
     if (D.use_ff) {   // X_ff = ReLU(X W1 + b1) W2 + b2  (Eq. 4 / Algorithm 3)
         GemmArgs a;
         a.fault = g->fault;
@@ -787,6 +798,15 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
         layer_desc_for(m, l, params, x_ld, starts[l].data(), &descs[l]);
         if (l == 0) descs[l].in_ld = ld0;
         SGCN_TRY(make_plan(g, &descs[l], &plans[l]));
+        if (l == 0 && D.use_ff && (m->slice_size % 8) != 0) {
+            // the fused input is narrower than its leading dimension: keep the padding columns of X_ff and of
+            // the saved intermediate at zero (both buffers are fully rewritten below, padding excluded)
+            plans[l].in_pad_zero = true;
+            if (plans[l].order == SLICEGCN_AGG_FIRST) {
+                plans[l].zt_pad_zero = true;
+                SGCN_CUDA(cudaMemsetAsync(E.saved[l], 0, plans[l].zt_bytes, st));
+            }
+        }
         SGCN_TRY(layer_forward_impl(g, &descs[l], plans[l], hin, E.H[l], E.saved[l], E.ws, E.ws_bytes, st));
         hin = E.H[l];
     }
@@ -830,7 +850,7 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
         SGCN_TRY(gemm_run(c, st));
     }
     // ---------------- loss (Eq. 10) and its gradient
-    SGCN_TRY(softmax_ce_run(n, C, logits, labels, train_idx, n_train, E.dlogits, E.row_loss, loss_out, st));
+    SGCN_TRY(softmax_ce_run(n, C, logits, labels, train_idx, n_train, E.dlogits, E.ld_dlog, E.row_loss, loss_out, st));
 
     // ---------------- backward
     {
@@ -843,7 +863,8 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
         w.lda = E.ld_cls;
         w.a_dtype = D.dtype;
         w.B = E.dlogits;
-        w.ldb = C;
+        w.ldb = E.ld_dlog;
+        w.b_pad_zero = 1;
         w.dW = grads + m->Wc2;
         w.dbias = grads + m->bc2;
         SGCN_TRY(wgrad_run(w, E.ws, E.ws_bytes, st));
@@ -855,7 +876,8 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
         a.K = C;
         a.N = D.hidden;
         a.A = E.dlogits;
-        a.lda = C;
+        a.lda = E.ld_dlog;
+        a.a_pad_zero = 1;
         a.B = params + m->Wc2;
         a.ldb = C;
         a.b_trans = 1;

@@ -806,7 +806,7 @@ slicegcn_status_t tc_gemm_launch(const GemmArgs& a, void* image, int64_t image_b
     tc_prep_b_kernel<BF16><<<pgrid, 128, 0, st>>>(a, n_pad, static_cast<unsigned char*>(image));
     SGCN_LAUNCH_CHECK();
     // 16-byte loads of the activation need aligned slices
-    bool vec = ((uintptr_t)a.A % 16 == 0) && (a.lda % EPC == 0) && (a.K % EPC == 0);
+    bool vec = ((uintptr_t)a.A % 16 == 0) && (a.lda % EPC == 0) && (a.K % EPC == 0 || a.a_pad_zero);
     for (int g = 0; g < a.groups; ++g) vec = vec && (a.a_start[g] % EPC == 0);
     if (a.a_mask) vec = vec && ((uintptr_t)a.a_mask % 8 == 0) && (a.a_mask_ld % 8 == 0);
     static const bool no_ws = getenv("SLICEGCN_NO_WS") != nullptr;
@@ -1055,6 +1055,10 @@ __global__ void tc_wgrad_reduce_kernel(const float* scratch, const WgTcPlan pl, 
         const int gl = g % groups_per_tile;
         f = gl * K + k;
         c = gl * N + n;
+    } else if (groups_per_tile < 0) {   // all groups share A: tiles over K, group g in columns g*N ..
+        mt = k / 128;
+        f = k % 128;
+        c = g * N + n;
     } else {                     // one group: tiles over K
         mt = k / 128;
         f = k % 128;
@@ -1077,18 +1081,30 @@ __global__ void tc_wgrad_reduce_kernel(const float* scratch, const WgTcPlan pl, 
 
 bool wgrad_tc_plan(const WgradArgs& a, WgTcPlan* pl, int* groups_per_tile) {
     if (a.K < 1 || !a.dW) return false;
-    const int es = a.a_dtype == SLICEGCN_BF16 ? 2 : 4;
-    for (int g = 0; g < a.groups; ++g)
-        if (a.a_start[g] != a.a_start[0] + g * a.K || a.b_start[g] != a.b_start[0] + g * a.N) return false;
-    (void)es;
-    if ((uintptr_t)a.A % 16 || a.lda % 4 || a.a_start[0] % 4 || a.K % 4) return false;   // 4-element loads of A
-    if ((uintptr_t)a.B % 16 || a.ldb % 4 || a.b_start[0] % 4 || a.N % 4) return false;
+    bool shared_a = a.groups > 1;   // every group reads the same A columns (fused input feeding all slices)
+    for (int g = 0; g < a.groups; ++g) shared_a = shared_a && (a.a_start[g] == a.a_start[0]);
+    for (int g = 0; g < a.groups; ++g) {
+        if (!shared_a && a.a_start[g] != a.a_start[0] + g * a.K) return false;
+        if (a.b_start[g] != a.b_start[0] + g * a.N) return false;
+    }
+    // 4-element loads: aligned starts; widths either multiples of 4 or followed by zero padding
+    if ((uintptr_t)a.A % 16 || a.lda % 4 || a.a_start[0] % 4) return false;
+    if ((uintptr_t)a.B % 16 || a.ldb % 4 || a.b_start[0] % 4) return false;
+    const bool a_single = a.groups == 1 || shared_a;
+    if (a.K % 4 && !(a.a_pad_zero && a_single)) return false;
+    if (a.N % 4 && !(a.b_pad_zero && a.groups == 1)) return false;
     if (a.b_mask && ((uintptr_t)a.b_mask % 4 || a.b_mask_ld % 4)) return false;
     WgTcPlan P{};
     P.a_col0 = a.a_start[0];
     P.b_col0 = a.b_start[0];
-    P.a_cols = a.groups * a.K;
-    if (a.groups > 1) {
+    P.a_cols = shared_a ? a.K : a.groups * a.K;
+    if (shared_a) {
+        if (a.groups * a.N > 256) return false;
+        P.m_tiles = (a.K + 127) / 128;
+        P.n_valid = a.groups * a.N;
+        P.b_cols_per_tile = 0;
+        *groups_per_tile = -1;   // reduce: row k of tile k/128, column g*N + n
+    } else if (a.groups > 1) {
         if (128 % a.K != 0) return false;
         int gpt = 128 / a.K;
         if (gpt > a.groups) gpt = a.groups;
