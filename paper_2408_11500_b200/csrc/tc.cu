@@ -1041,6 +1041,200 @@ __global__ void __launch_bounds__(kWgThreads, STAGES == 1 ? 2 : 1) tc_wgrad_kern
     if (warp == 0) tmem_dealloc(tmem, ncols);
 }
 
+// ------------------------------------------------------------------------------ weight gradient, warp-specialised
+// Same product, for unmasked fp32 operands.  Both operands of dW = A^T B are read in their natural
+// row-major form: a slab of 32 rows is, for the MMA, a K=32 slice whose M (resp. N) index runs along
+// the contiguous columns -- the "MN-major" operand form -- so the slab goes from global memory into
+// the swizzled tile by cp.async without any transposition, and the producers only split it into hi
+// and lo parts in place.  One CTA per SM: 4 producer warps keep a ring of D stages filled, one thread
+// of warp 4 issues the MMAs (one accumulation chain per CTA), warps 5-8 write the partial tile out at
+// the end.  Tile layout (the one MN-major tf32 operands must use, "128-byte swizzle with 32-byte
+// base"): atoms of 4 K-rows x 128 bytes (32 columns), the 32-byte chunk index XORed with the K-row;
+// atom (K atom ka, column block mb) at ((ka * blocks + mb) * 512) bytes.
+__device__ __forceinline__ uint64_t smem_desc_mn(const void* tile, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_u32(tile) >> 4) & 0x3FFF);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;   // between column blocks (MN direction)
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;   // between 8-row K blocks
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)1 << 61;                             // SWIZZLE_128B with 32-byte base
+    return d;
+}
+
+template <bool WIDE>   // WIDE: more than 32 column quads in the B tile
+__global__ void __launch_bounds__(kWsThreads, 1) tc_wgrad_ws_kernel(const WgradArgs a, const WgTcPlan pl, const int D,
+                                                                    float* scratch, int* fault) {
+    extern __shared__ __align__(1024) unsigned char smem[];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int mt = blockIdx.y, chunk = blockIdx.x;
+    unsigned char* base = smem + ((1024u - (smem_u32(smem) & 1023u)) & 1023u);
+    const int nbk = (pl.n_t + 31) / 32;                      // column blocks of the B tile
+    const uint32_t b_bytes = 4u * (uint32_t)nbk * 1024u;     // one B tile (hi or lo)
+    const uint32_t stage_bytes = 32768u + 2u * b_bytes;      // A hi | A lo | B hi | B lo
+    unsigned char* tail = base + (uint32_t)D * stage_bytes;
+    uint64_t* full = reinterpret_cast<uint64_t*>(tail);      // [D] 128 producer arrivals
+    uint64_t* freeb = full + 4;                              // [D] MMAs of the stage completed
+    uint64_t* tfull = freeb + 4;                             // accumulator complete
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tfull + 1);
+    uint32_t ncols = 32;
+    while ((int)ncols < pl.n_t) ncols <<= 1;
+    if (tid == 0) {
+        for (int i = 0; i < D; ++i) {
+            mbar_init(&full[i], 128);
+            mbar_init(&freeb[i], 1);
+        }
+        mbar_init(tfull, 1);
+    }
+    if (warp == 4) tmem_alloc(tmem_slot, ncols);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    const int64_t r_begin = (int64_t)chunk * pl.rows_per_chunk;
+    const int64_t r_end = min(a.M, r_begin + pl.rows_per_chunk);
+    const int n_slabs = r_end > r_begin ? (int)((r_end - r_begin + 31) / 32) : 0;
+
+    if (warp < 4) {
+        // ------------------------------------------------------------ producers
+        // A: thread t copies 16-byte column chunk (t % 32) of rows t/32 + 4 i; B: chunk (t % 32) of the same
+        // rows, or (WIDE) chunk (t % 64) of rows t/64 + 2 i
+        const int acc_c = tid & 31, a_r0 = tid >> 5;
+        const int b_cc = WIDE ? (tid & 63) : (tid & 31), b_r0 = WIDE ? (tid >> 6) : (tid >> 5);
+        constexpr int BI = WIDE ? 16 : 8, BSTEP = WIDE ? 2 : 4;
+        const int a_col = mt * 128 + acc_c * 4;
+        const bool a_ok = a_col < pl.a_cols;
+        const int nq = pl.n_t / 4;
+        const bool b_ok = b_cc < nq && b_cc * 4 < pl.n_valid;
+        const float* Ap = static_cast<const float*>(a.A) + pl.a_col0 + a_col;
+        const float* Bp = a.B + pl.b_col0 + mt * pl.b_cols_per_tile + b_cc * 4;
+        // (row r of the slab, 16-byte column chunk cc) -> byte offset inside the tile
+        auto a_off = [&](int r) {
+            return (uint32_t)((((r >> 2) * 4 + (acc_c >> 3)) << 9) + ((r & 3) << 7) + (((((acc_c & 7) >> 1) ^ (r & 3))) << 5) + ((acc_c & 1) << 4));
+        };
+        auto b_off = [&](int r) {
+            return (uint32_t)((((r >> 2) * nbk + (b_cc >> 3)) << 9) + ((r & 3) << 7) + (((((b_cc & 7) >> 1) ^ (r & 3))) << 5) + ((b_cc & 1) << 4));
+        };
+        const int L = D >= 3 ? D - 1 : 1;
+        auto issue = [&](int j) {
+            const int st = j % D;
+            const int use = j / D;
+            if (use >= 1 && !mbar_wait(&freeb[st], (uint32_t)((use - 1) & 1))) {
+                if (lane == 0) atomicExch(fault, 8);
+                return false;
+            }
+            unsigned char* stg = base + (uint32_t)st * stage_bytes;
+            const uint32_t dA = smem_u32(stg), dB = smem_u32(stg + 32768);
+            const int64_t rr = r_begin + (int64_t)j * 32;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int r = a_r0 + 4 * i;
+                const bool in = a_ok && rr + r < r_end;
+                const float* src = in ? Ap + (rr + r) * a.lda : static_cast<const float*>(a.A);
+                const int sz = in ? 16 : 0;
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dA + a_off(r)), "l"(src), "r"(sz) : "memory");
+            }
+            if (b_cc < nq) {
+#pragma unroll
+                for (int i = 0; i < BI; ++i) {
+                    const int r = b_r0 + BSTEP * i;
+                    const bool in = b_ok && rr + r < r_end;
+                    const float* src = in ? Bp + (rr + r) * a.ldb : a.B;
+                    const int sz = in ? 16 : 0;
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dB + b_off(r)), "l"(src), "r"(sz) : "memory");
+                }
+            }
+            return true;
+        };
+        bool okp = true;
+        for (int j = 0; j < L && okp; ++j) {
+            if (j < n_slabs) okp = issue(j);
+            asm volatile("cp.async.commit_group;" ::: "memory");
+        }
+        for (int j = 0; j < n_slabs && okp; ++j) {
+            if (L == 2) asm volatile("cp.async.wait_group 1;" ::: "memory");
+            else asm volatile("cp.async.wait_group 0;" ::: "memory");
+            const int st = j % D;
+            unsigned char* stg = base + (uint32_t)st * stage_bytes;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const uint32_t off = a_off(a_r0 + 4 * i);
+                const float4 v = *reinterpret_cast<const float4*>(stg + off);
+                const float h0 = tf32_hi(v.x), h1 = tf32_hi(v.y), h2 = tf32_hi(v.z), h3 = tf32_hi(v.w);
+                *reinterpret_cast<float4*>(stg + off) = make_float4(h0, h1, h2, h3);
+                *reinterpret_cast<float4*>(stg + 16384 + off) = make_float4(v.x - h0, v.y - h1, v.z - h2, v.w - h3);
+            }
+            if (b_cc < nq) {
+#pragma unroll
+                for (int i = 0; i < BI; ++i) {
+                    const uint32_t off = b_off(b_r0 + BSTEP * i);
+                    const float4 v = *reinterpret_cast<const float4*>(stg + 32768 + off);
+                    const float h0 = tf32_hi(v.x), h1 = tf32_hi(v.y), h2 = tf32_hi(v.z), h3 = tf32_hi(v.w);
+                    *reinterpret_cast<float4*>(stg + 32768 + off) = make_float4(h0, h1, h2, h3);
+                    *reinterpret_cast<float4*>(stg + 32768 + b_bytes + off) = make_float4(v.x - h0, v.y - h1, v.z - h2, v.w - h3);
+                }
+            }
+            proxy_fence();
+            asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&full[st])) : "memory");
+            if (j + L < n_slabs) okp = issue(j + L);
+            asm volatile("cp.async.commit_group;" ::: "memory");
+        }
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+    } else if (warp == 4) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            // M = 128 A-columns, N = n_t B-columns, both operands MN-major
+            const uint32_t idesc = idesc_f32acc(128, pl.n_t, false) | (1u << 15) | (1u << 16);
+            bool okm = true;
+            for (int j = 0; j < n_slabs && okm; ++j) {
+                const int st = j % D;
+                okm = mbar_wait(&full[st], (uint32_t)((j / D) & 1));
+                if (!okm) break;
+                tc_fence_after();
+                unsigned char* stg = base + (uint32_t)st * stage_bytes;
+#pragma unroll
+                for (int kb = 0; kb < 4; ++kb) {
+                    // one MMA covers 8 K-rows = two K atoms; column blocks are 512 bytes apart
+                    const uint64_t da_hi = smem_desc_mn(stg + kb * 4096, 512, 2048);
+                    const uint64_t da_lo = smem_desc_mn(stg + 16384 + kb * 4096, 512, 2048);
+                    const uint64_t db_hi = smem_desc_mn(stg + 32768 + kb * nbk * 1024, 512, nbk * 512);
+                    const uint64_t db_lo = smem_desc_mn(stg + 32768 + b_bytes + kb * nbk * 1024, 512, nbk * 512);
+                    umma<false>(tmem, da_hi, db_hi, idesc, (j == 0 && kb == 0) ? 0u : 1u);
+                    umma<false>(tmem, da_lo, db_hi, idesc, 1u);
+                    umma<false>(tmem, da_hi, db_lo, idesc, 1u);
+                }
+                umma_commit(&freeb[st]);
+            }
+            if (okm) umma_commit(tfull);
+            else atomicExch(fault, 9);
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue: partial tile -> scratch
+        const int q = warp & 3;
+        float* out = scratch + ((int64_t)chunk * pl.m_tiles + mt) * 128 * pl.n_t + (int64_t)(q * 32 + lane) * pl.n_t;
+        if (n_slabs > 0) {
+            if (mbar_wait(tfull, 0)) {
+                tc_fence_after();
+                for (int c0 = 0; c0 < pl.n_t; c0 += 32) {
+                    float v[32];
+                    tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
+#pragma unroll
+                    for (int j = 0; j < 32; j += 4)
+                        if (c0 + j < pl.n_t) *reinterpret_cast<float4*>(out + c0 + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                }
+            } else if (lane == 0) {
+                atomicExch(fault, 10);
+            }
+        } else {
+            for (int j = 0; j < pl.n_t; ++j) out[j] = 0.f;
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 4) tmem_dealloc(tmem, ncols);
+}
+
 // dW[g][k][n] = sum over chunks of the partial tiles (fixed order)
 __global__ void tc_wgrad_reduce_kernel(const float* scratch, const WgTcPlan pl, int groups, int K, int N, int groups_per_tile,
                                        float* dW) {
@@ -1079,7 +1273,7 @@ __global__ void tc_wgrad_reduce_kernel(const float* scratch, const WgTcPlan pl, 
     dW[i] = s;
 }
 
-bool wgrad_tc_plan(const WgradArgs& a, WgTcPlan* pl, int* groups_per_tile) {
+bool wgrad_tc_plan(const WgradArgs& a, WgTcPlan* pl, int* groups_per_tile, int force_per_sm = 0) {
     if (a.K < 1 || !a.dW) return false;
     bool shared_a = a.groups > 1;   // every group reads the same A columns (fused input feeding all slices)
     for (int g = 0; g < a.groups; ++g) shared_a = shared_a && (a.a_start[g] == a.a_start[0]);
@@ -1124,7 +1318,7 @@ bool wgrad_tc_plan(const WgradArgs& a, WgTcPlan* pl, int* groups_per_tile) {
     P.n_t = (P.n_valid + 15) & ~15;
     // single-stage CTAs are small enough for two or three per SM, which overlap each other
     P.stages = 1;
-    const int per_sm = P.n_t <= 128 ? 3 : 2;
+    const int per_sm = force_per_sm > 0 ? force_per_sm : (P.n_t <= 128 ? 3 : 2);
     int64_t want = (148 * per_sm + P.m_tiles - 1) / P.m_tiles;
     int64_t rpc = (a.M + want - 1) / want;
     rpc = (rpc + 31) / 32 * 32;
@@ -1157,6 +1351,40 @@ slicegcn_status_t tc_wgrad_run(const WgradArgs& a, void* scratch, int64_t scratc
     WgTcPlan pl;
     int gpt = 0;
     if (!a.fault || !wgrad_tc_plan(a, &pl, &gpt)) return SLICEGCN_ERR_UNSUPPORTED;
+    static const bool no_ws = getenv("SLICEGCN_NO_WS") != nullptr;
+    if (!no_ws && a.a_dtype == SLICEGCN_F32 && !a.b_mask) {
+        // warp-specialised variant: one CTA per SM
+        WgTcPlan pw;
+        int gw = 0;
+        if (wgrad_tc_plan(a, &pw, &gw, 1)) {
+            const int nbk = (pw.n_t + 31) / 32;
+            const int stage_b = 32768 + 2 * 4 * nbk * 1024;
+            int D = (220 * 1024) / stage_b;
+            if (D > 3) D = 3;
+            const int64_t need_w = (int64_t)pw.n_chunks * pw.m_tiles * 128 * pw.n_t * (int64_t)sizeof(float);
+            if (D >= 2 && scratch && scratch_bytes >= need_w) {
+                const int ws_smem = D * stage_b + 256 + 1024;
+                static bool ws_configured = false;
+                if (!ws_configured) {
+                    SGCN_CUDA(cudaFuncSetAttribute(tc_wgrad_ws_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
+                    SGCN_CUDA(cudaFuncSetAttribute(tc_wgrad_ws_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
+                    ws_configured = true;
+                }
+                dim3 wgrid(pw.n_chunks, pw.m_tiles);
+                if (pw.n_t / 4 > 32)
+                    tc_wgrad_ws_kernel<true><<<wgrid, kWsThreads, ws_smem, st>>>(a, pw, D, static_cast<float*>(scratch), a.fault);
+                else
+                    tc_wgrad_ws_kernel<false><<<wgrid, kWsThreads, ws_smem, st>>>(a, pw, D, static_cast<float*>(scratch), a.fault);
+                SGCN_LAUNCH_CHECK();
+                const int64_t total_w = (int64_t)a.groups * a.K * a.N;
+                tc_wgrad_reduce_kernel<<<(unsigned)((total_w + 255) / 256), 256, 0, st>>>(static_cast<const float*>(scratch), pw,
+                                                                                         a.groups, a.K, a.N, gw, a.dW);
+                SGCN_LAUNCH_CHECK();
+                count_launch(2);
+                return SLICEGCN_OK;
+            }
+        }
+    }
     const int64_t need = (int64_t)pl.n_chunks * pl.m_tiles * 128 * pl.n_t * (int64_t)sizeof(float);
     if (!scratch || scratch_bytes < need) return SLICEGCN_ERR_UNSUPPORTED;
     const int smem_bytes = pl.stages * (2 * 16384 + 2 * pl.n_t * 128) + 64 + 1024;
