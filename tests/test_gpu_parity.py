@@ -354,3 +354,58 @@ def test_citation_workload_full_size_fp32(B):
         assert max(errs.values()) <= 1e-3 and errs["logits"] <= 2e-5
     finally:
         gp.close()
+
+
+# ------------------------------------------------------------------------------ other workload shapes
+
+def test_social_shape_transform_first_fp32(B):
+    """Dense-social shape at reduced size: 602 input features in 4 slices of 151 (last one overlapping),
+    transform-first first layer, hidden 256, high mean degree (most rows are split into segments)."""
+    n = 4000
+    src, dst = synth.chung_lu_lognormal(n, 400000, 1.0, seed=3)
+    X = synth.gaussian_features(n, 602, seed=3); y = synth.uniform_labels(n, 41, seed=3)
+    mk = dict(in_d=602, hidden=256, num_layers=2, num_classes=41, num_slices=4)
+    od = oracle_desc(**mk)
+    assert od.slices == [(0, 151), (151, 302), (302, 453), (451, 602)]
+    params = synth.init_params(orc.param_shapes(od), seed=3, bias_scale=0.1)
+    og = orc.build_graph(n, src, dst, True, True)
+    assert np.median(og.deg) > 100
+    gp = GpuProblem(n, src, dst, X, y, params, **mk)
+    try:
+        assert [B.slicegcn_model_layer_order(gp.m, l) for l in range(2)] == [B.XFORM_FIRST, B.AGG_FIRST]
+        # ~3 M ReLU units: a borderline sign decision is likely, so the oracle's own spread is allowed for
+        errs = _compare_epoch(gp, od, og, X.astype(np.float64), y, params, None, TOL_F32, orders=["xform", "agg"],
+                              relu_margin=1e-6)
+        assert max(errs.values()) <= 2e-3 and errs["logits"] <= 2e-5
+        assert B.slicegcn_graph_device_status(gp.g) == 0
+    finally:
+        gp.close()
+
+
+@pytest.mark.parametrize("relabel", [False, True])
+@pytest.mark.parametrize("dtype,width", [("f32", 16), ("f32", 64), ("f32", 512), ("bf16", 32), ("bf16", 256)])
+def test_rmat_sweep_sampled_rows_and_identity(B, torch, relabel, dtype, width):
+    """SpMM sweep on an R-MAT graph (a, b, c = 0.57, 0.19, 0.19; edge factor 16): exact oracle values on a
+    seeded sample of rows that includes the 100 longest, and A_hat sqrt(deg) = sqrt(deg) on every row."""
+    n, src, dst = synth.rmat(16, 16, seed=2, relabel=relabel)
+    og = orc.build_graph(n, src, dst, True, True)
+    g = B.slicegcn_graph_create(n, src, dst, B.SYMMETRIZE | B.ADD_SELF_LOOPS)
+    try:
+        ex = B.slicegcn_graph_export(g)
+        assert np.array_equal(ex["rowptr"], og.rowptr) and np.array_equal(ex["colidx"], og.colidx)
+        dt = B.F32 if dtype == "f32" else B.BF16
+        X = synth.gaussian_features(n, width, seed=5)
+        got, x_used = _gpu_spmm(B, torch, g, X, width, dt)
+        rows = np.unique(np.concatenate([np.argsort(og.deg)[-100:], np.random.default_rng(0).integers(0, n, 4000)]))
+        want = orc.spmm(og, x_used.astype(np.float64), rows=rows.astype(np.int64))
+        if dtype == "f32":
+            assert rel_inf(got[rows], want) <= 2e-6
+        else:
+            assert np.all(np.abs(got[rows] - want) <= 2 ** -8 * np.abs(want) + 1e-5 * np.abs(want).max())
+        if dtype == "f32":
+            v = np.sqrt(og.deg.astype(np.float64))
+            Xv = np.repeat(v[:, None], width, axis=1).astype(np.float32)
+            idn, _ = _gpu_spmm(B, torch, g, Xv, width, dt)
+            np.testing.assert_allclose(idn, Xv, rtol=5e-6)
+    finally:
+        B.slicegcn_graph_destroy(g)
