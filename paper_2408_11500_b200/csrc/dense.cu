@@ -377,6 +377,10 @@ slicegcn_status_t gemm_run(const GemmArgs& a, cudaStream_t st) {
     if (a.M < 1 || a.groups < 1 || a.groups > SLICEGCN_MAX_SLICES || a.N < 1 || a.K < 0)
         SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "gemm: bad shape");
     static const bool no_tc = getenv("SLICEGCN_NO_TC") != nullptr;   // CUDA-core kernels only (for A/B checks)
+    if (a.A2) {   // two products in one pass: tensor-core path only, the caller splits it otherwise
+        if (no_tc || !a.fault || !a.b_image || a.K < 1) return SLICEGCN_ERR_UNSUPPORTED;
+        return tc_gemm_run(a, st);
+    }
     if (!no_tc && a.fault && a.b_image && a.K >= 1 && a.b_image_bytes >= tc_image_bytes(a.groups, a.K, a.N))
         return tc_gemm_run(a, st);
     const bool abf = a.a_dtype == SLICEGCN_BF16, cbf = a.c_dtype == SLICEGCN_BF16;

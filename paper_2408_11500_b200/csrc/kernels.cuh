@@ -58,6 +58,16 @@ struct GemmArgs {
     int* fault = nullptr;
     void* b_image = nullptr;
     int64_t b_image_bytes = 0;
+    // optional second product added after the activation:  C = epilogue(A B) + A2 B2  (the self term of
+    // Eq. 6 next to the aggregation term).  Same dtype, group count, N and b_trans as the first product.
+    // Only the warp-specialised tensor-core kernel takes it; gemm_run() reports UNSUPPORTED otherwise.
+    const void* A2 = nullptr;
+    int64_t lda2 = 0;
+    int a2_start[SLICEGCN_MAX_SLICES] = {0};
+    int a2_pad_zero = 0;
+    const float* B2 = nullptr;
+    int64_t b2_gstride = 0;
+    int K2 = 0;
 };
 slicegcn_status_t gemm_run(const GemmArgs& a, cudaStream_t st);
 slicegcn_status_t tc_gemm_run(const GemmArgs& a, cudaStream_t st);

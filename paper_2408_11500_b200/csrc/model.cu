@@ -116,7 +116,8 @@ slicegcn_status_t make_plan(const slicegcn_graph* g, const slicegcn_layer_desc* 
 
 // scratch for the prepared weight images of the tensor-core GEMMs of one layer (forward and dgrad shapes)
 int64_t layer_tc_img(const LayerPlan& L) {
-    return std::max(tc_image_bytes(L.p, L.in_width, L.h_s), tc_image_bytes(L.p, L.h_s, L.in_width));
+    // forward may run the aggregation and self products in one pass: two images
+    return std::max(2 * tc_image_bytes(L.p, L.in_width, L.h_s), tc_image_bytes(L.p, L.h_s, L.in_width));
 }
 
 int64_t layer_fwd_ws_bytes(const slicegcn_graph* g, const LayerPlan& L) {
@@ -203,7 +204,30 @@ slicegcn_status_t layer_forward_impl(const slicegcn_graph* g, const slicegcn_lay
     if (L.order == SLICEGCN_AGG_FIRST) {
         // Z = A_hat H_in over every input column once; slices then read their column ranges of Z
         SGCN_TRY(spmm_run(g, false, L.dtype, L.dtype, H_in, L.in_ld, zt, L.zt_ld, L.in_cols, nullptr, part, part_bytes, st));
-        if (d->W_self) SGCN_TRY(gemm_run(self, st));
+        if (d->W_self) {
+            // one pass: H_out = ReLU(Z W_agg + b) + H_in W_self + b_self + E (two accumulators)
+            GemmArgs both = self;
+            both.K = L.in_width;
+            both.A = zt;
+            both.lda = L.zt_ld;
+            both.a_pad_zero = L.zt_pad_zero ? 1 : 0;
+            both.B = d->W_agg;
+            both.bias = d->b;
+            both.relu = 1;
+            both.mask_out = mask;
+            both.mask_ld = L.mask_ld;
+            both.A2 = H_in;
+            both.lda2 = L.in_ld;
+            both.a2_pad_zero = L.in_pad_zero ? 1 : 0;
+            both.B2 = d->W_self;
+            both.b2_gstride = self.b_gstride;
+            both.K2 = L.in_width;
+            for (int i = 0; i < L.p; ++i) both.a2_start[i] = L.in_starts[i];
+            const slicegcn_status_t rc = gemm_run(both, st);
+            if (rc == SLICEGCN_OK) return SLICEGCN_OK;
+            if (rc != SLICEGCN_ERR_UNSUPPORTED) return rc;
+            SGCN_TRY(gemm_run(self, st));
+        }
         GemmArgs agg = self;   // H_out = ReLU(Z W_agg + b) (+ H_out | + b_self + E)
         agg.K = L.in_width;
         agg.A = zt;

@@ -497,7 +497,8 @@ constexpr int kWsThreads = 288;
 
 template <typename TA, typename TC, bool BF16>
 __global__ void __launch_bounds__(kWsThreads, 1) tc_gemm_ws_kernel(const GemmArgs a, const int n_pad, const int n_tiles,
-                                                                   const int D, const unsigned char* image, int* fault) {
+                                                                   const int D, const unsigned char* image,
+                                                                   const unsigned char* image2, int* fault) {
     extern __shared__ __align__(1024) unsigned char smem[];
     constexpr int KS = BF16 ? 64 : 32;
     constexpr int UK = BF16 ? 16 : 8;
@@ -507,15 +508,17 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_gemm_ws_kernel(const GemmArg
     const uint32_t slab_bytes = 2u * (uint32_t)n_pad * 128u;                  // weight image [hi | lo]
     const uint32_t a_bytes = BF16 ? 16384u : 32768u;                          // activation tile(s) of a stage
     const uint32_t stage_bytes = a_bytes + slab_bytes;
-    float* stage_out = reinterpret_cast<float*>(base + (uint32_t)D * stage_bytes);   // 4 x 32 x kStagePitch floats
-    unsigned char* tail = reinterpret_cast<unsigned char*>(stage_out) + 4 * 32 * kStagePitch * 4;
+    const bool fused = a.A2 != nullptr;     // second product: its accumulator sits next to the first
+    float* stage_out = reinterpret_cast<float*>(base + (uint32_t)D * stage_bytes);   // 4 (8 if fused) x 32 x kStagePitch floats
+    unsigned char* tail = reinterpret_cast<unsigned char*>(stage_out) + (fused ? 8 : 4) * 32 * kStagePitch * 4;
     uint64_t* full = reinterpret_cast<uint64_t*>(tail);            // [D]   128 producer arrivals + weight bytes
     uint64_t* freeb = full + 8;                                     // [D]   MMAs of the stage have completed
     uint64_t* tfull = freeb + 8;                                    // [2]   accumulator complete
     uint64_t* tfree = tfull + 2;                                    // [2]   accumulator drained (128 arrivals)
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tfree + 2);
-    uint32_t acc_cols = 32;
-    while ((int)acc_cols < n_pad) acc_cols <<= 1;
+    uint32_t half_cols = 32;
+    while ((int)half_cols < n_pad) half_cols <<= 1;
+    const uint32_t acc_cols = fused ? 2 * half_cols : half_cols;
     const uint32_t ncols = 2 * acc_cols;
     if (tid == 0) {
         for (int i = 0; i < D; ++i) {
@@ -534,7 +537,9 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_gemm_ws_kernel(const GemmArg
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
-    const int n_slabs = (a.K + KS - 1) / KS;
+    const int ns1 = (a.K + KS - 1) / KS;                     // K slabs of the first product
+    const int ns2 = fused ? (a.K2 + KS - 1) / KS : 0;        // and of the second
+    const int n_slabs = ns1 + ns2;
     const int64_t row_tiles = (a.M + 127) / 128;
     const int64_t n_items = row_tiles * a.groups * n_tiles;
     const int64_t my_items = n_items > blockIdx.x ? (n_items - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
@@ -555,7 +560,6 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_gemm_ws_kernel(const GemmArg
         uint32_t offs[8];               // swizzled byte offsets of this thread's eight chunks
 #pragma unroll
         for (int i = 0; i < 8; ++i) offs[i] = sw_off(rbase + 16 * i, c * 16);
-        const int64_t row_step = 16 * a.lda;
         // steps requested ahead of the one being finished; with D >= 3 the stage a new request goes to
         // was last used two steps back, so the producer never waits for the MMAs it has just fed
         const int L = D >= 3 ? D - 2 : 1;
@@ -571,18 +575,24 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_gemm_ws_kernel(const GemmArg
             int64_t row0;
             int g, nt;
             decode(j / n_slabs, row0, g, nt);
-            const int s = (int)(j % n_slabs);
+            int s = (int)(j % n_slabs);
+            const bool second = s >= ns1;     // this step belongs to the second product
+            if (second) s -= ns1;
             unsigned char* stg = base + (uint32_t)st * stage_bytes;
             if (tid == 0) {
+                const unsigned char* img = second ? image2 + ((((int64_t)g * n_tiles + nt) * ns2 + s)) * (int64_t)slab_bytes
+                                                  : image + ((((int64_t)g * n_tiles + nt) * ns1 + s)) * (int64_t)slab_bytes;
                 mbar_expect_tx(&full[st], slab_bytes);
-                bulk_g2s(stg + a_bytes, image + ((((int64_t)g * n_tiles + nt) * n_slabs + s)) * (int64_t)slab_bytes, slab_bytes,
-                         &full[st]);
+                bulk_g2s(stg + a_bytes, img, slab_bytes, &full[st]);
             }
             const int k = s * KS + c * EPC;
-            const TA* src0 = static_cast<const TA*>(a.A) + a.a_start[g] + (row0 + rbase) * a.lda + k;
+            const int64_t ld = second ? a.lda2 : a.lda;
+            const TA* src0 = (second ? static_cast<const TA*>(a.A2) + a.a2_start[g] : static_cast<const TA*>(a.A) + a.a_start[g]) +
+                             (row0 + rbase) * ld + k;
+            const int64_t row_step = 16 * ld;
             const uint32_t dst0 = smem_u32(stg);
             const int rows_left = (int)min((int64_t)128, a.M - row0) - rbase;   // rows rbase + 16 i < rows of the tile
-            const bool k_in = k < a.K;
+            const bool k_in = k < (second ? a.K2 : a.K);
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 const bool in = k_in && 16 * i < rows_left;
@@ -634,8 +644,9 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_gemm_ws_kernel(const GemmArg
                 const int nn = min(n_pad, a.N - nt * n_pad);
                 const int n_mma = (nn + 15) & ~15;
                 const uint32_t idesc = idesc_f32acc(128, n_mma, BF16);
-                const uint32_t d_tmem = tmem + (uint32_t)acc * acc_cols;
+                const uint32_t d_tmem0 = tmem + (uint32_t)acc * acc_cols;
                 for (int s = 0; s < n_slabs && okm; ++s) {
+                    const uint32_t d_tmem = d_tmem0 + (s >= ns1 ? half_cols : 0u);   // second product: own columns
                     const int64_t j = it * n_slabs + s;
                     const int st = (int)(j % D);
                     okm = mbar_wait(&full[st], (uint32_t)((j / D) & 1));
@@ -647,7 +658,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_gemm_ws_kernel(const GemmArg
 #pragma unroll
                     for (int ks = 0; ks < KS / UK; ++ks) {
                         const uint64_t adv = (uint64_t)((ks * 32) >> 4);
-                        umma<BF16>(d_tmem, da_hi + adv, db_hi + adv, idesc, (s == 0 && ks == 0) ? 0u : 1u);
+                        umma<BF16>(d_tmem, da_hi + adv, db_hi + adv, idesc, ((s == 0 || s == ns1) && ks == 0) ? 0u : 1u);
                         if (!BF16) umma<BF16>(d_tmem, da_lo + adv, db_hi + adv, idesc, 1u);
                         umma<BF16>(d_tmem, da_hi + adv, db_lo + adv, idesc, 1u);
                     }
@@ -663,6 +674,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_gemm_ws_kernel(const GemmArg
         // warp covers four whole 128-byte row segments
         const int q = warp & 3;                       // TMEM lane quarter this warp may read
         float* stage = stage_out + q * (32 * kStagePitch);
+        float* stage2 = stage_out + (4 + q) * (32 * kStagePitch);   // only there (and used) when fused
         const int cq = lane & 7, sub = lane >> 3;
         unsigned char* Cb = static_cast<unsigned char*>(a.C);
         bool oke = true;
@@ -682,6 +694,12 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_gemm_ws_kernel(const GemmArg
             const int rows_here = (int)min((int64_t)32, a.M - (row0 + q * 32));   // valid rows of this warp's quarter
             for (int c0 = 0; c0 < n_mma; c0 += 32) {
                 float v[32];
+                if (fused) {   // the second product's columns first, into the second staging tile
+                    tmem_ld32(d_tmem + half_cols + (uint32_t)c0, v);
+#pragma unroll
+                    for (int j = 0; j < 32; j += 4)
+                        *reinterpret_cast<float4*>(stage2 + lane * kStagePitch + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                }
                 tmem_ld32(d_tmem + (uint32_t)c0, v);
                 if (c0 + 32 >= n_mma) {   // last read of this accumulator: hand it back to the MMA warp
                     tc_fence_before();
@@ -763,6 +781,10 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_gemm_ws_kernel(const GemmArg
                     if (a.accumulate) {
                         x[0] += cold[i].x; x[1] += cold[i].y; x[2] += cold[i].z; x[3] += cold[i].w;
                     }
+                    if (fused) {
+                        const float4 t2 = *reinterpret_cast<const float4*>(stage2 + rr * kStagePitch + cq * 4);
+                        x[0] += t2.x; x[1] += t2.y; x[2] += t2.z; x[3] += t2.w;
+                    }
                     if (sizeof(TC) == 4) {
                         *reinterpret_cast<float4*>(Cb + (row * a.ldc + col) * 4) = make_float4(x[0], x[1], x[2], x[3]);
                     } else {
@@ -793,7 +815,30 @@ slicegcn_status_t tc_gemm_launch(const GemmArgs& a, void* image, int64_t image_b
     const int n_tiles = (a.N + n_pad - 1) / n_pad;
     const int n_slabs = (a.K + KS - 1) / KS;
     const int64_t need = (int64_t)a.groups * n_tiles * n_slabs * 2 * n_pad * 128;
-    if (!image || image_bytes < need) SGCN_FAIL(SLICEGCN_ERR_ALLOC, "tc_gemm: weight image scratch too small");
+    const bool fused = a.A2 != nullptr;
+    const int n_slabs2 = fused ? (a.K2 + KS - 1) / KS : 0;
+    const int64_t need2 = (int64_t)a.groups * n_tiles * n_slabs2 * 2 * n_pad * 128;
+    if (!image || image_bytes < need + need2) {
+        if (fused) return SLICEGCN_ERR_UNSUPPORTED;   // the caller falls back to two separate products
+        SGCN_FAIL(SLICEGCN_ERR_ALLOC, "tc_gemm: weight image scratch too small");
+    }
+    unsigned char* image2 = static_cast<unsigned char*>(image) + need;
+    if (fused) {
+        // everything the fused form needs is checked before anything is launched
+        bool ok2 = ((uintptr_t)a.A % 16 == 0) && (a.lda % EPC == 0) && (a.K % EPC == 0 || a.a_pad_zero) &&
+                   ((uintptr_t)a.A2 % 16 == 0) && (a.lda2 % EPC == 0) && (a.K2 % EPC == 0 || a.a2_pad_zero) && a.K2 >= 1 &&
+                   !a.a_mask && !a.accumulate && n_pad <= 128 && a.N % 4 == 0 && a.ldc % 4 == 0 && ((uintptr_t)a.C % 16 == 0) &&
+                   getenv("SLICEGCN_NO_WS") == nullptr;
+        for (int g = 0; g < a.groups; ++g) ok2 = ok2 && a.a_start[g] % EPC == 0 && a.a2_start[g] % EPC == 0 && a.c_start[g] % 4 == 0;
+        if (a.mask_out) ok2 = ok2 && (a.mask_ld % 4 == 0) && ((uintptr_t)a.mask_out % 4 == 0);
+        if (a.mul_pos) ok2 = false;
+        if (a.bias) ok2 = ok2 && ((uintptr_t)a.bias % 16 == 0);
+        if (a.post1) ok2 = ok2 && ((uintptr_t)a.post1 % 16 == 0);
+        if (a.post2) ok2 = ok2 && ((uintptr_t)a.post2 % 16 == 0);
+        const int stage_b2 = (BF16 ? 16384 : 32768) + 2 * n_pad * 128;
+        ok2 = ok2 && (220 * 1024 - (8 * 32 * kStagePitch * 4 + 256 + 1024)) / stage_b2 >= 2;
+        if (!ok2) return SLICEGCN_ERR_UNSUPPORTED;
+    }
     const int smem_bytes = (BF16 ? 16384 : 32768) + 4 * n_pad * 128 + 4 * 32 * kStagePitch * 4 + 64 + 1024;
     static bool configured = false;
     if (!configured) {
@@ -805,6 +850,15 @@ slicegcn_status_t tc_gemm_launch(const GemmArgs& a, void* image, int64_t image_b
     dim3 pgrid(n_slabs * 4, n_tiles, a.groups);
     tc_prep_b_kernel<BF16><<<pgrid, 128, 0, st>>>(a, n_pad, static_cast<unsigned char*>(image));
     SGCN_LAUNCH_CHECK();
+    if (fused) {
+        GemmArgs b2 = a;
+        b2.B = a.B2;
+        b2.b_gstride = a.b2_gstride;
+        b2.K = a.K2;
+        dim3 pgrid2(n_slabs2 * 4, n_tiles, a.groups);
+        tc_prep_b_kernel<BF16><<<pgrid2, 128, 0, st>>>(b2, n_pad, image2);
+        SGCN_LAUNCH_CHECK();
+    }
     // 16-byte loads of the activation need aligned slices
     bool vec = ((uintptr_t)a.A % 16 == 0) && (a.lda % EPC == 0) && (a.K % EPC == 0 || a.a_pad_zero);
     for (int g = 0; g < a.groups; ++g) vec = vec && (a.a_start[g] % EPC == 0);
@@ -825,7 +879,7 @@ slicegcn_status_t tc_gemm_launch(const GemmArgs& a, void* image, int64_t image_b
         // warp-specialised kernel: one CTA per SM, ring depth from what fits in shared memory
         const int a_bytes = BF16 ? 16384 : 32768;
         const int stage_b = a_bytes + 2 * n_pad * 128;
-        const int fixed = 4 * 32 * kStagePitch * 4 + 256 + 1024;
+        const int fixed = (fused ? 8 : 4) * 32 * kStagePitch * 4 + 256 + 1024;
         int D = (220 * 1024 - fixed) / stage_b;
         if (D > 4) D = 4;
         if (D >= 2) {
@@ -838,12 +892,13 @@ slicegcn_status_t tc_gemm_launch(const GemmArgs& a, void* image, int64_t image_b
             const int64_t items = ((a.M + 127) / 128) * a.groups * n_tiles;
             int64_t wgrid = 148;
             if (wgrid > items) wgrid = items;
-            tc_gemm_ws_kernel<TA, TC, BF16><<<(unsigned)wgrid, kWsThreads, ws_smem, st>>>(a, n_pad, n_tiles, D, static_cast<unsigned char*>(image), fault);
+            tc_gemm_ws_kernel<TA, TC, BF16><<<(unsigned)wgrid, kWsThreads, ws_smem, st>>>(a, n_pad, n_tiles, D, static_cast<unsigned char*>(image), image2, fault);
             SGCN_LAUNCH_CHECK();
-            count_launch(2);
+            count_launch(fused ? 3 : 2);
             return SLICEGCN_OK;
         }
     }
+    if (fused) return SLICEGCN_ERR_UNSUPPORTED;   // not reachable: the fused form was vetted above
     // persistent grid: as many CTAs as fit at once (shared memory and 512 TMEM columns per SM)
     int ncols = 32;
     while (ncols < n_pad) ncols <<= 1;
