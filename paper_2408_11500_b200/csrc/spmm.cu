@@ -309,20 +309,75 @@ __device__ __forceinline__ void spmm_segment_block(const SpmmParams& p, const in
     const int row = __ldg(p.long_rows + li);
     const int start = __ldg(p.rowptr + row) + (seg - __ldg(p.seg_ptr + li)) * kSegment;
     const int end = min(__ldg(p.rowptr + row + 1), start + kSegment);
+    constexpr int U = (8 / C) < 2 ? 2 : (8 / C);   // neighbors gathered per round
+    __shared__ int2 nbuf[kRowsWarps][32];          // (column index, 1/sqrt(deg) bits) of the current batch
+    int2* nb = &nbuf[threadIdx.x >> 5][sub * L];
+    const uint32_t row16 = (uint32_t)((p.ldx * (int64_t)sizeof(TI)) >> 4);
+    const uint4* xl[C];
+#pragma unroll
+    for (int c = 0; c < C; ++c) xl[c] = static_cast<const uint4*>(p.X) + min(sl + c * L, p.nch - 1);
     float acc[C][V];
 #pragma unroll
     for (int c = 0; c < C; ++c)
 #pragma unroll
         for (int e = 0; e < V; ++e) acc[c][e] = 0.f;
-    for (int base = start + sub * L; base < end; base += 32) {
-        const int k = base + sl;
-        int j = 0;
-        float dj = 0.f;
-        if (k < end) {
-            j = __ldg(p.colidx + k);
-            dj = __ldg(p.dinv + j);
+    int base = start + sub * L;
+    int jn = (base + sl < end) ? __ldg(p.colidx + base + sl) : 0;
+    float djn = (base + sl < end) ? __ldg(p.dinv + jn) : 0.f;
+    for (; base < end; base += 32) {
+        const int cnt = min(L, end - base);
+        __syncwarp(gmask);
+        nb[sl] = make_int2(jn, __float_as_int(djn));
+        __syncwarp(gmask);
+        const int nbase = base + 32;
+        if (nbase + sl < end) jn = __ldg(p.colidx + nbase + sl);   // requested now, used by the next batch
+        int t = 0;
+        for (; t + U <= cnt; t += U) {   // no row ends inside a segment: plain rounds
+            uint4 raw[U][C];
+            int2 meta[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                meta[u] = nb[t + u];
+#pragma unroll
+                for (int c = 0; c < C; ++c) raw[u][c] = __ldg(xl[c] + (uint64_t)(uint32_t)meta[u].x * row16);
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const float dd = __int_as_float(meta[u].y);
+#pragma unroll
+                for (int c = 0; c < C; ++c) {
+                    float f[V];
+                    Vec<TI>::unpack(raw[u][c], f);
+#pragma unroll
+                    for (int e = 0; e < V; ++e) acc[c][e] = fmaf(dd, f[e], acc[c][e]);
+                }
+            }
         }
-        gather_block<TI, L, C>(p, gmask, sl, j, dj, min(L, end - base), acc);
+        if (t < cnt) {                   // ragged end of the row's last segment
+            uint4 raw[U][C];
+            int2 meta[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (t + u < cnt) {
+                    meta[u] = nb[t + u];
+#pragma unroll
+                    for (int c = 0; c < C; ++c) raw[u][c] = __ldg(xl[c] + (uint64_t)(uint32_t)meta[u].x * row16);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (t + u >= cnt) break;
+                const float dd = __int_as_float(meta[u].y);
+#pragma unroll
+                for (int c = 0; c < C; ++c) {
+                    float f[V];
+                    Vec<TI>::unpack(raw[u][c], f);
+#pragma unroll
+                    for (int e = 0; e < V; ++e) acc[c][e] = fmaf(dd, f[e], acc[c][e]);
+                }
+            }
+        }
+        if (nbase + sl < end) djn = __ldg(p.dinv + jn);   // its index has arrived by now
     }
     __syncwarp();
 #pragma unroll
