@@ -50,7 +50,7 @@ void reset_launches();
 // Rows with more than kLongRow stored entries are split into segments of kSegment entries; each
 // segment is reduced by one warp into a partial row, and the partial rows of a long row are summed
 // in a fixed order afterwards (deterministic, no floating-point atomics).
-constexpr int kLongRow = 256;
+constexpr int kLongRow = 64;
 constexpr int kSegment = 256;
 // The remaining rows are dealt out in row-aligned chunks of about kChunk stored entries: chunk c
 // owns every row whose first entry index lies in [c*kChunk, (c+1)*kChunk), so each lane group gets

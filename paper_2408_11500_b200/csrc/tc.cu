@@ -494,6 +494,7 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const GemmArgs a, c
 // Loads, MMAs and the epilogue of neighbouring items therefore overlap inside one CTA, and the
 // bytes in flight are set by the ring depth, not by the register file.
 constexpr int kWsThreads = 288;
+constexpr int kWsVecFloats = 1024;   // bias / post vectors up to this many floats are staged in shared memory
 
 template <typename TA, typename TC, bool BF16>
 __global__ void __launch_bounds__(kWsThreads, 1) tc_gemm_ws_kernel(const GemmArgs a, const int n_pad, const int n_tiles,
@@ -544,13 +545,40 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_gemm_ws_kernel(const GemmArg
     const int64_t n_items = row_tiles * a.groups * n_tiles;
     const int64_t my_items = n_items > blockIdx.x ? (n_items - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
     const int64_t my_steps = my_items * n_slabs;
-    auto decode = [&](int64_t local_item, int64_t& row0, int& g, int& nt) {
-        const uint32_t item = (uint32_t)(blockIdx.x + local_item * gridDim.x);   // host keeps the item count < 2^31
-        const uint32_t per_row = (uint32_t)(n_tiles * a.groups);
-        const uint32_t rt = item / per_row, rem = item - rt * per_row;
-        g = (int)(rem / (uint32_t)n_tiles);
-        nt = (int)(rem - (uint32_t)g * (uint32_t)n_tiles);
-        row0 = (int64_t)rt * 128;
+    // Cursor over this CTA's items (item = blockIdx.x + i * gridDim.x; the host keeps the item count
+    // below 2^31): row tile, group and column tile follow by additions -- nothing on the per-step
+    // paths divides.
+    struct ItemCursor {
+        uint32_t rt, rem, dq, dr, per_row;
+        int n_tiles, g, nt;
+        __device__ void init(uint32_t first, uint32_t stride, int groups, int n_tiles_) {
+            n_tiles = n_tiles_;
+            per_row = (uint32_t)(n_tiles * groups);
+            rt = first / per_row;
+            rem = first - rt * per_row;
+            dq = stride / per_row;
+            dr = stride - dq * per_row;
+            split();
+        }
+        __device__ void split() {
+            if (n_tiles == 1) {
+                g = (int)rem;
+                nt = 0;
+            } else {
+                g = (int)(rem / (uint32_t)n_tiles);
+                nt = (int)(rem - (uint32_t)g * (uint32_t)n_tiles);
+            }
+        }
+        __device__ void next() {
+            rem += dr;
+            rt += dq;
+            if (rem >= per_row) {
+                rem -= per_row;
+                ++rt;
+            }
+            split();
+        }
+        __device__ int64_t row0() const { return (int64_t)rt * 128; }
     };
 
     if (warp < 4) {
@@ -563,19 +591,30 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_gemm_ws_kernel(const GemmArg
         // steps requested ahead of the one being finished; with D >= 3 the stage a new request goes to
         // was last used two steps back, so the producer never waits for the MMAs it has just fed
         const int L = D >= 3 ? D - 2 : 1;
-        auto issue = [&](int64_t j) {   // requests step j's activation slab (and weight image)
-            const int st = (int)(j % D);
-            const int64_t use = j / D;
+        // issue cursor: the step whose loads are requested next -> (stage, ring pass) and (item, slab)
+        int i_st = 0, i_s = 0;
+        uint32_t i_pass = 0;
+        ItemCursor i_it;
+        i_it.init(blockIdx.x, gridDim.x, a.groups, n_tiles);
+        auto issue = [&]() {   // requests the next step's activation slab (and weight image)
+            const int st = i_st;
             bool okw = true;
-            if (use >= 1) okw = mbar_wait(&freeb[st], (uint32_t)((use - 1) & 1));
+            if (i_pass >= 1) okw = mbar_wait(&freeb[st], (i_pass - 1) & 1);
             if (!okw) {
                 if (lane == 0) atomicExch(fault, 5);
                 return false;
             }
-            int64_t row0;
-            int g, nt;
-            decode(j / n_slabs, row0, g, nt);
-            int s = (int)(j % n_slabs);
+            const int64_t row0 = i_it.row0();
+            const int g = i_it.g, nt = i_it.nt;
+            int s = i_s;
+            if (++i_st == D) {
+                i_st = 0;
+                ++i_pass;
+            }
+            if (++i_s == n_slabs) {
+                i_s = 0;
+                i_it.next();
+            }
             const bool second = s >= ns1;     // this step belongs to the second product
             if (second) s -= ns1;
             unsigned char* stg = base + (uint32_t)st * stage_bytes;
@@ -604,14 +643,14 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_gemm_ws_kernel(const GemmArg
         };
         bool okp = true;
         for (int64_t j = 0; j < L && okp; ++j) {   // exactly L groups, empty past the end, so the count below holds
-            if (j < my_steps) okp = issue(j);
+            if (j < my_steps) okp = issue();
             asm volatile("cp.async.commit_group;" ::: "memory");
         }
+        int st = 0;   // stage of the step being finished
         for (int64_t j = 0; j < my_steps && okp; ++j) {
             // L + j groups so far: step j (this thread's own copies) has landed once at most L-1 are pending
             if (L == 2) asm volatile("cp.async.wait_group 1;" ::: "memory");
             else asm volatile("cp.async.wait_group 0;" ::: "memory");
-            const int st = (int)(j % D);
             unsigned char* stg = base + (uint32_t)st * stage_bytes;
             if (!BF16) {
 #pragma unroll
@@ -624,7 +663,8 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_gemm_ws_kernel(const GemmArg
             }
             proxy_fence();
             asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&full[st])) : "memory");
-            if (j + L < my_steps) okp = issue(j + L);
+            if (++st == D) st = 0;
+            if (j + L < my_steps) okp = issue();
             asm volatile("cp.async.commit_group;" ::: "memory");   // one group per step, empty or not
         }
         asm volatile("cp.async.wait_group 0;" ::: "memory");
@@ -632,24 +672,25 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_gemm_ws_kernel(const GemmArg
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             bool okm = true;
+            ItemCursor m_it;
+            m_it.init(blockIdx.x, gridDim.x, a.groups, n_tiles);
+            int st = 0;
+            uint32_t pass = 0;
             for (int64_t it = 0; it < my_items && okm; ++it) {
                 const int acc = (int)(it & 1);
                 const int64_t use = it >> 1;
                 if (use >= 1) okm = mbar_wait(&tfree[acc], (uint32_t)((use - 1) & 1));
                 if (!okm) break;
                 tc_fence_after();
-                int64_t row0;
-                int g, nt;
-                decode(it, row0, g, nt);
+                const int nt = m_it.nt;
+                m_it.next();
                 const int nn = min(n_pad, a.N - nt * n_pad);
                 const int n_mma = (nn + 15) & ~15;
                 const uint32_t idesc = idesc_f32acc(128, n_mma, BF16);
                 const uint32_t d_tmem0 = tmem + (uint32_t)acc * acc_cols;
                 for (int s = 0; s < n_slabs && okm; ++s) {
                     const uint32_t d_tmem = d_tmem0 + (s >= ns1 ? half_cols : 0u);   // second product: own columns
-                    const int64_t j = it * n_slabs + s;
-                    const int st = (int)(j % D);
-                    okm = mbar_wait(&full[st], (uint32_t)((j / D) & 1));
+                    okm = mbar_wait(&full[st], pass & 1);
                     if (!okm) break;
                     tc_fence_after();
                     unsigned char* stg = base + (uint32_t)st * stage_bytes;
@@ -663,6 +704,10 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_gemm_ws_kernel(const GemmArg
                         umma<BF16>(d_tmem, da_hi + adv, db_lo + adv, idesc, 1u);
                     }
                     umma_commit(&freeb[st]);
+                    if (++st == D) {
+                        st = 0;
+                        ++pass;
+                    }
                 }
                 if (okm) umma_commit(&tfull[acc]);
             }
@@ -677,15 +722,31 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_gemm_ws_kernel(const GemmArg
         float* stage2 = stage_out + (4 + q) * (32 * kStagePitch);   // only there (and used) when fused
         const int cq = lane & 7, sub = lane >> 3;
         unsigned char* Cb = static_cast<unsigned char*>(a.C);
+        // bias and post-activation vectors of all groups, staged once (a load from global memory per
+        // item would sit on the critical path of every tile)
+        float* sbias = reinterpret_cast<float*>(tail + 256);
+        float* spost = sbias + kWsVecFloats;
+        const bool vec_staged = a.groups * a.N <= kWsVecFloats;
+        if (vec_staged) {
+            for (int i = tid - 160; i < a.groups * a.N; i += 128) {
+                sbias[i] = a.bias ? __ldg(a.bias + i) : 0.f;
+                float pv = a.post1 ? __ldg(a.post1 + i) : 0.f;
+                if (a.post2) pv += __ldg(a.post2 + i);
+                spost[i] = pv;
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+        }
         bool oke = true;
+        ItemCursor e_it;
+        e_it.init(blockIdx.x, gridDim.x, a.groups, n_tiles);
         for (int64_t it = 0; it < my_items && oke; ++it) {
             const int acc = (int)(it & 1);
             oke = mbar_wait(&tfull[acc], (uint32_t)((it >> 1) & 1));
             if (!oke) break;
             tc_fence_after();
-            int64_t row0;
-            int g, nt;
-            decode(it, row0, g, nt);
+            const int64_t row0 = e_it.row0();
+            const int g = e_it.g, nt = e_it.nt;
+            e_it.next();
             const int n0 = nt * n_pad;
             const int nn = min(n_pad, a.N - n0);
             const int n_mma = (nn + 15) & ~15;
@@ -713,7 +774,10 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_gemm_ws_kernel(const GemmArg
                 const bool col_ok = n < nn;           // nn is a multiple of 4 on this path
                 const int col = cs + n;
                 float4 bias = make_float4(0.f, 0.f, 0.f, 0.f), post = bias;
-                if (col_ok) {
+                if (col_ok && vec_staged) {
+                    bias = *reinterpret_cast<const float4*>(sbias + g * a.N + n0 + n);
+                    post = *reinterpret_cast<const float4*>(spost + g * a.N + n0 + n);
+                } else if (col_ok) {
                     if (a.bias) bias = __ldg(reinterpret_cast<const float4*>(a.bias + g * a.N + n0 + n));
                     if (a.post1) post = __ldg(reinterpret_cast<const float4*>(a.post1 + g * a.N + n0 + n));
                     if (a.post2) {
@@ -836,7 +900,7 @@ slicegcn_status_t tc_gemm_launch(const GemmArgs& a, void* image, int64_t image_b
         if (a.post1) ok2 = ok2 && ((uintptr_t)a.post1 % 16 == 0);
         if (a.post2) ok2 = ok2 && ((uintptr_t)a.post2 % 16 == 0);
         const int stage_b2 = (BF16 ? 16384 : 32768) + 2 * n_pad * 128;
-        ok2 = ok2 && (220 * 1024 - (8 * 32 * kStagePitch * 4 + 256 + 1024)) / stage_b2 >= 2;
+        ok2 = ok2 && (220 * 1024 - (8 * 32 * kStagePitch * 4 + 256 + 1024 + 2 * kWsVecFloats * 4)) / stage_b2 >= 2;
         if (!ok2) return SLICEGCN_ERR_UNSUPPORTED;
     }
     const int smem_bytes = (BF16 ? 16384 : 32768) + 4 * n_pad * 128 + 4 * 32 * kStagePitch * 4 + 64 + 1024;
@@ -879,7 +943,7 @@ slicegcn_status_t tc_gemm_launch(const GemmArgs& a, void* image, int64_t image_b
         // warp-specialised kernel: one CTA per SM, ring depth from what fits in shared memory
         const int a_bytes = BF16 ? 16384 : 32768;
         const int stage_b = a_bytes + 2 * n_pad * 128;
-        const int fixed = (fused ? 8 : 4) * 32 * kStagePitch * 4 + 256 + 1024;
+        const int fixed = (fused ? 8 : 4) * 32 * kStagePitch * 4 + 256 + 1024 + 2 * kWsVecFloats * 4;
         int D = (220 * 1024 - fixed) / stage_b;
         if (D > 4) D = 4;
         if (D >= 2) {
@@ -1172,12 +1236,17 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_wgrad_ws_kernel(const WgradA
             return (uint32_t)((((r >> 2) * nbk + (b_cc >> 3)) << 9) + ((r & 3) << 7) + (((((b_cc & 7) >> 1) ^ (r & 3))) << 5) + ((b_cc & 1) << 4));
         };
         const int L = D >= 3 ? D - 1 : 1;
+        int i_st = 0;            // issue cursor: stage and ring pass of the slab requested next
+        uint32_t i_pass = 0;
         auto issue = [&](int j) {
-            const int st = j % D;
-            const int use = j / D;
-            if (use >= 1 && !mbar_wait(&freeb[st], (uint32_t)((use - 1) & 1))) {
+            const int st = i_st;
+            if (i_pass >= 1 && !mbar_wait(&freeb[st], (i_pass - 1) & 1)) {
                 if (lane == 0) atomicExch(fault, 8);
                 return false;
+            }
+            if (++i_st == D) {
+                i_st = 0;
+                ++i_pass;
             }
             unsigned char* stg = base + (uint32_t)st * stage_bytes;
             const uint32_t dA = smem_u32(stg), dB = smem_u32(stg + 32768);
@@ -1207,10 +1276,10 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_wgrad_ws_kernel(const WgradA
             if (j < n_slabs) okp = issue(j);
             asm volatile("cp.async.commit_group;" ::: "memory");
         }
+        int st = 0;
         for (int j = 0; j < n_slabs && okp; ++j) {
             if (L == 2) asm volatile("cp.async.wait_group 1;" ::: "memory");
             else asm volatile("cp.async.wait_group 0;" ::: "memory");
-            const int st = j % D;
             unsigned char* stg = base + (uint32_t)st * stage_bytes;
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
@@ -1232,6 +1301,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_wgrad_ws_kernel(const WgradA
             }
             proxy_fence();
             asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&full[st])) : "memory");
+            if (++st == D) st = 0;
             if (j + L < n_slabs) okp = issue(j + L);
             asm volatile("cp.async.commit_group;" ::: "memory");
         }
@@ -1242,9 +1312,10 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_wgrad_ws_kernel(const WgradA
             // M = 128 A-columns, N = n_t B-columns, both operands MN-major
             const uint32_t idesc = idesc_f32acc(128, pl.n_t, false) | (1u << 15) | (1u << 16);
             bool okm = true;
+            int st = 0;
+            uint32_t pass = 0;
             for (int j = 0; j < n_slabs && okm; ++j) {
-                const int st = j % D;
-                okm = mbar_wait(&full[st], (uint32_t)((j / D) & 1));
+                okm = mbar_wait(&full[st], pass & 1);
                 if (!okm) break;
                 tc_fence_after();
                 unsigned char* stg = base + (uint32_t)st * stage_bytes;
@@ -1260,6 +1331,10 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_wgrad_ws_kernel(const WgradA
                     umma<false>(tmem, da_hi, db_lo, idesc, 1u);
                 }
                 umma_commit(&freeb[st]);
+                if (++st == D) {
+                    st = 0;
+                    ++pass;
+                }
             }
             if (okm) umma_commit(tfull);
             else atomicExch(fault, 9);
