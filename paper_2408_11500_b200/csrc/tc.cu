@@ -10,6 +10,7 @@
 // to shared memory with ordinary stores (swizzled by hand) followed by a proxy fence.
 // Every wait on an mbarrier is bounded; a wait that runs out sets the caller's status word.
 #include <cstdlib>
+#include <type_traits>
 
 #include "common.cuh"
 #include "kernels.cuh"
@@ -113,6 +114,63 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// The same load without the wait, so that several can be in flight; tmem_ld_wait() before the values are used.
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+          "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+          "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+          "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// 32 lanes x 32 columns, registers -> TMEM: thread t of the warp writes row (lane base + t), columns col..col+31
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};" ::"r"(taddr),
+        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]),
+        "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]),
+        "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]),
+        "r"(r[31])
+        : "memory");
+}
+// 32 lanes x 16 columns from r[OFF..OFF+15]
+template <int OFF>
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(taddr),
+        "r"(r[OFF + 0]), "r"(r[OFF + 1]), "r"(r[OFF + 2]), "r"(r[OFF + 3]), "r"(r[OFF + 4]), "r"(r[OFF + 5]), "r"(r[OFF + 6]),
+        "r"(r[OFF + 7]), "r"(r[OFF + 8]), "r"(r[OFF + 9]), "r"(r[OFF + 10]), "r"(r[OFF + 11]), "r"(r[OFF + 12]), "r"(r[OFF + 13]),
+        "r"(r[OFF + 14]), "r"(r[OFF + 15])
+        : "memory");
+}
+// 32 lanes x 16 columns of fp32, added onto x[OFF..OFF+15]
+template <int OFF>
+__device__ __forceinline__ void tmem_ld16_add(uint32_t taddr, float (&x)[32]) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+          "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) x[OFF + i] += __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+// D[tmem] (+)= A[tmem] * B[smem desc], tf32: A's row i sits in TMEM lane i, its K values in consecutive columns
+__device__ __forceinline__ void umma_ts_tf32(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
 }
 
 // K-major, 128-byte swizzle: rows of 128 bytes, 8-row groups 1024 bytes apart
@@ -479,6 +537,43 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const GemmArgs a, c
     if (warp == 0) tmem_dealloc(tmem, ncols);
 }
 
+// Cursor over a CTA's work items (item = first + i * stride; the host keeps the item count below
+// 2^31): row tile, group and column tile follow by additions, so nothing on the per-step paths of
+// the persistent kernels divides.
+struct ItemCursor {
+    uint32_t rt, rem, dq, dr, per_row;
+    int n_tiles, g, nt;
+    __device__ void init(uint32_t first, uint32_t stride, int groups, int n_tiles_) {
+        n_tiles = n_tiles_;
+        per_row = (uint32_t)(n_tiles * groups);
+        rt = first / per_row;
+        rem = first - rt * per_row;
+        dq = stride / per_row;
+        dr = stride - dq * per_row;
+        split();
+    }
+    __device__ void split() {
+        if (n_tiles == 1) {
+            g = (int)rem;
+            nt = 0;
+        } else {
+            g = (int)(rem / (uint32_t)n_tiles);
+            nt = (int)(rem - (uint32_t)g * (uint32_t)n_tiles);
+        }
+    }
+    __device__ void next() {
+        rem += dr;
+        rt += dq;
+        if (rem >= per_row) {
+            rem -= per_row;
+            ++rt;
+        }
+        split();
+    }
+    __device__ int64_t row0() const { return (int64_t)rt * 128; }
+};
+
+
 // ------------------------------------------------------------------------------ row-panel GEMM, warp-specialised
 // The same contract as tc_gemm_kernel, for 16-byte-aligned, unmasked operands.  One persistent CTA per
 // SM, nine warps in three roles connected by mbarriers (every wait is bounded):
@@ -545,42 +640,6 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_gemm_ws_kernel(const GemmArg
     const int64_t n_items = row_tiles * a.groups * n_tiles;
     const int64_t my_items = n_items > blockIdx.x ? (n_items - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
     const int64_t my_steps = my_items * n_slabs;
-    // Cursor over this CTA's items (item = blockIdx.x + i * gridDim.x; the host keeps the item count
-    // below 2^31): row tile, group and column tile follow by additions -- nothing on the per-step
-    // paths divides.
-    struct ItemCursor {
-        uint32_t rt, rem, dq, dr, per_row;
-        int n_tiles, g, nt;
-        __device__ void init(uint32_t first, uint32_t stride, int groups, int n_tiles_) {
-            n_tiles = n_tiles_;
-            per_row = (uint32_t)(n_tiles * groups);
-            rt = first / per_row;
-            rem = first - rt * per_row;
-            dq = stride / per_row;
-            dr = stride - dq * per_row;
-            split();
-        }
-        __device__ void split() {
-            if (n_tiles == 1) {
-                g = (int)rem;
-                nt = 0;
-            } else {
-                g = (int)(rem / (uint32_t)n_tiles);
-                nt = (int)(rem - (uint32_t)g * (uint32_t)n_tiles);
-            }
-        }
-        __device__ void next() {
-            rem += dr;
-            rt += dq;
-            if (rem >= per_row) {
-                rem -= per_row;
-                ++rt;
-            }
-            split();
-        }
-        __device__ int64_t row0() const { return (int64_t)rt * 128; }
-    };
-
     if (warp < 4) {
         // ------------------------------------------------------------ producers
         const int c = tid & 7;          // 16-byte chunk of the 128-byte row
@@ -869,6 +928,384 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_gemm_ws_kernel(const GemmArg
     if (warp == 4) tmem_dealloc(tmem, ncols);
 }
 
+// ------------------------------------------------------------------------------ row-panel GEMM, activation operand in TMEM
+// The kernel for the sliced layers proper: fp32 operands, narrow outputs per group (n_pad <= 64, or
+// <= 32 with the fused second product).  What limits the kernel above on these shapes is shared
+// memory traffic -- every activation byte is written by the copy, read and written twice by the
+// hi/lo split and read three times by the MMAs -- so here the activation operand never returns to
+// shared memory:
+//   warps 0-3   producers.  Warp w owns rows 32w..32w+31 of every tile.  It keeps a private ring of
+//               kTsRing raw slabs filled with cp.async (no barrier: nobody else touches its rows),
+//               reads the landed slab one row per lane, splits it in registers and writes hi and lo
+//               into a TMEM stage with tcgen05.st (row = TMEM lane, K along the columns -- the form
+//               the MMA takes its A operand in).  Thread 0 also requests the step's weight image.
+//   warp 4      MMA issuer.  Per K slab two chains instead of three: A_hi x [B_hi | B_lo] (the image
+//               holds hi and lo back to back, so they form one operand of 2 n_pad rows) into
+//               accumulator columns [0, 2 n_pad), then A_lo x B_hi onto columns [0, n_pad).
+//   warps 5-12  epilogue, two groups of four that take alternate items (one per accumulator):
+//               the halves (and the second product) are summed in registers in the row-per-lane
+//               form, bias / ReLU / post are applied there, and only the finished tile (plus the
+//               ReLU mask bytes) goes through a per-warp staging tile to be written in whole
+//               128-byte row segments.
+// TMEM columns: [accumulator 0][accumulator 1] (accw each) then kTsStages x 64 (A hi | A lo).
+constexpr int kTsThreads = 416;
+constexpr int kTsRing = 6;     // raw slabs per producer warp (kTsRing - 1 in flight)
+constexpr int kTsStages = 3;   // TMEM operand stages (with their weight images in shared memory)
+constexpr int kTsMaskPitch = 48;
+
+__global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArgs a, const int n_pad, const int n_tiles,
+                                                                   const unsigned char* image, const unsigned char* image2,
+                                                                   int* fault) {
+    extern __shared__ __align__(1024) unsigned char smem[];
+    constexpr int R = kTsRing, S = kTsStages;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    unsigned char* base = smem + ((1024u - (smem_u32(smem) & 1023u)) & 1023u);
+    const uint32_t slab_bytes = 2u * (uint32_t)n_pad * 128u;                  // weight image [hi | lo]
+    const bool fused = a.A2 != nullptr;
+    unsigned char* wring = base;                                              // [S] weight images
+    unsigned char* raw = wring + (uint32_t)S * slab_bytes;                    // [4 warps][R] x 4096 B
+    float* stage_out = reinterpret_cast<float*>(raw + 4 * R * 4096);          // [8 warps] 32 x kStagePitch floats
+    unsigned char* stage_mask = reinterpret_cast<unsigned char*>(stage_out + 8 * 32 * kStagePitch);   // [8] 32 x kTsMaskPitch
+    float* sbias = reinterpret_cast<float*>(stage_mask + 8 * 32 * kTsMaskPitch);
+    float* spost = sbias + kWsVecFloats + 64;
+    uint64_t* afull = reinterpret_cast<uint64_t*>(spost + kWsVecFloats + 64);   // [S] 128 producer arrivals + weight bytes
+    uint64_t* afree = afull + S;                                              // [S] MMAs of the stage have completed
+    uint64_t* tfull = afree + S;                                              // [2] accumulator complete
+    uint64_t* tfree = tfull + 2;                                              // [2] accumulator drained (128 arrivals)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tfree + 2);
+    const uint32_t prodw = 2u * (uint32_t)n_pad;            // columns of one product: [hi*hi + lo*hi | hi*lo]
+    const uint32_t accw = fused ? 2 * prodw : prodw;        // columns of one accumulator
+    const uint32_t a_col0 = 2 * accw;                       // first column of the operand stages
+    if (tid == 0) {
+        for (int i = 0; i < S; ++i) {
+            mbar_init(&afull[i], 129);
+            mbar_init(&afree[i], 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&tfull[i], 1);
+            mbar_init(&tfree[i], 128);
+        }
+    }
+    if (warp == 4) tmem_alloc(tmem_slot, 512);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    const int ns1 = (a.K + 31) / 32;                         // K slabs of the first product
+    const int ns2 = fused ? (a.K2 + 31) / 32 : 0;            // and of the second
+    const int n_slabs = ns1 + ns2;
+    const int64_t row_tiles = (a.M + 127) / 128;
+    const int64_t n_items = row_tiles * a.groups * n_tiles;
+    const int64_t my_items = n_items > blockIdx.x ? (n_items - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+    const int64_t my_steps = my_items * n_slabs;
+
+    if (warp < 4) {
+        // ------------------------------------------------------------ producers
+        unsigned char* myraw = raw + warp * (R * 4096);
+        const int c = lane & 7, r0 = lane >> 3;   // copy: 16-byte chunk c of rows r0 + 4 i of the warp's 32 rows
+        uint32_t woff[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) woff[i] = (uint32_t)((r0 + 4 * i) * 128 + ((c ^ ((r0 + 4 * i) & 7)) << 4));
+        const uint32_t roff = (uint32_t)(lane * 128);   // split: lane reads row `lane`, chunk cc at (cc ^ (lane & 7)) * 16
+        // cursor of the step whose loads are requested next, and of the step being converted
+        int i_rs = 0, i_s = 0;
+        ItemCursor i_it;
+        i_it.init(blockIdx.x, gridDim.x, a.groups, n_tiles);
+        auto issue = [&]() {
+            const int64_t row0 = i_it.row0();
+            const int g = i_it.g;
+            int s = i_s;
+            unsigned char* slot = myraw + i_rs * 4096;
+            if (++i_rs == R) i_rs = 0;
+            if (++i_s == n_slabs) {
+                i_s = 0;
+                i_it.next();
+            }
+            const bool second = s >= ns1;
+            if (second) s -= ns1;
+            const int k = s * 32 + c * 4;
+            const int64_t ld = second ? a.lda2 : a.lda;
+            const float* src0 = (second ? static_cast<const float*>(a.A2) + a.a2_start[g] : static_cast<const float*>(a.A) + a.a_start[g]) +
+                                (row0 + 32 * warp + r0) * ld + k;
+            const int64_t row_step = 4 * ld;
+            const uint32_t dst0 = smem_u32(slot);
+            const int rows_left = (int)min((int64_t)128, a.M - row0) - 32 * warp - r0;   // rows r0 + 4 i below this exist
+            const bool k_in = k < (second ? a.K2 : a.K);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const bool in = k_in && 4 * i < rows_left;
+                const float* src = in ? (src0 + i * row_step) : static_cast<const float*>(a.A);
+                const int sz = in ? 16 : 0;   // zero-fill outside the matrix
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst0 + woff[i]), "l"(src), "r"(sz) : "memory");
+            }
+        };
+        for (int j = 0; j < R - 1; ++j) {   // exactly R-1 groups, empty past the end, so the count below holds
+            if (j < my_steps) issue();
+            asm volatile("cp.async.commit_group;" ::: "memory");
+        }
+        int rs = 0, ts = 0, c_s = 0;
+        uint32_t pass = 0;
+        ItemCursor c_it;
+        c_it.init(blockIdx.x, gridDim.x, a.groups, n_tiles);
+        bool okp = true;
+        for (int64_t j = 0; j < my_steps; ++j) {
+            // R-1+j groups so far; step j has landed once at most R-2 are pending
+            asm volatile("cp.async.wait_group %0;" ::"n"(R - 2) : "memory");
+            __syncwarp();   // every lane's copies of step j are in, every lane is done reading step j-1
+            if (j + R - 1 < my_steps) issue();   // into the slot step j-1 was read from
+            asm volatile("cp.async.commit_group;" ::: "memory");   // one group per step, empty or not
+            if (pass >= 1) okp = mbar_wait(&afree[ts], (pass - 1) & 1);
+            if (!okp) break;
+            if (tid == 0) {
+                int s = c_s;
+                const bool second = s >= ns1;
+                if (second) s -= ns1;
+                const int g = c_it.g, nt = c_it.nt;
+                const unsigned char* img = second ? image2 + ((((int64_t)g * n_tiles + nt) * ns2 + s)) * (int64_t)slab_bytes
+                                                  : image + ((((int64_t)g * n_tiles + nt) * ns1 + s)) * (int64_t)slab_bytes;
+                mbar_expect_tx(&afull[ts], slab_bytes);
+                bulk_g2s(wring + (uint32_t)ts * slab_bytes, img, slab_bytes, &afull[ts]);
+                if (++c_s == n_slabs) {
+                    c_s = 0;
+                    c_it.next();
+                }
+            }
+            __syncwarp();
+            tc_fence_after();
+            const unsigned char* slot = myraw + rs * 4096 + roff;
+            const uint32_t t_hi = tmem + ((uint32_t)(32 * warp) << 16) + a_col0 + (uint32_t)ts * 64u;
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {   // 16 K values at a time keeps the register count down
+                uint32_t h[32];                      // [0,16): hi of K 16 half..; [16,32): lo of the same
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc) {
+                    const int ch = half * 4 + cc;
+                    const float4 v = *reinterpret_cast<const float4*>(slot + ((ch ^ (lane & 7)) << 4));
+                    const float h0 = tf32_hi(v.x), h1 = tf32_hi(v.y), h2 = tf32_hi(v.z), h3 = tf32_hi(v.w);
+                    h[4 * cc + 0] = __float_as_uint(h0);
+                    h[4 * cc + 1] = __float_as_uint(h1);
+                    h[4 * cc + 2] = __float_as_uint(h2);
+                    h[4 * cc + 3] = __float_as_uint(h3);
+                    h[16 + 4 * cc + 0] = __float_as_uint(v.x - h0);
+                    h[16 + 4 * cc + 1] = __float_as_uint(v.y - h1);
+                    h[16 + 4 * cc + 2] = __float_as_uint(v.z - h2);
+                    h[16 + 4 * cc + 3] = __float_as_uint(v.w - h3);
+                }
+                tmem_st16<0>(t_hi + 16u * half, h);
+                tmem_st16<16>(t_hi + 32u + 16u * half, h);
+            }
+            tmem_st_wait();
+            tc_fence_before();
+            asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&afull[ts])) : "memory");
+            if (++rs == R) rs = 0;
+            if (++ts == S) {
+                ts = 0;
+                ++pass;
+            }
+        }
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        if (!okp && lane == 0) atomicExch(fault, 5);
+    } else if (warp == 4) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            bool okm = true;
+            const uint32_t idesc_wide = idesc_f32acc(128, 2 * n_pad, false);   // A_hi x [B_hi | B_lo]
+            const uint32_t idesc_hi = idesc_f32acc(128, n_pad, false);         // A_lo x B_hi
+            int ts = 0;
+            uint32_t pass = 0;
+            for (int64_t it = 0; it < my_items && okm; ++it) {
+                const int acc = (int)(it & 1);
+                const int64_t use = it >> 1;
+                if (use >= 1) okm = mbar_wait(&tfree[acc], (uint32_t)((use - 1) & 1));
+                if (!okm) break;
+                tc_fence_after();
+                const uint32_t d_tmem0 = tmem + (uint32_t)acc * accw;
+                for (int s = 0; s < n_slabs && okm; ++s) {
+                    const uint32_t d_tmem = d_tmem0 + (s >= ns1 ? prodw : 0u);   // second product: own columns
+                    okm = mbar_wait(&afull[ts], pass & 1);
+                    if (!okm) break;
+                    tc_fence_after();
+                    const uint32_t a_hi = tmem + a_col0 + (uint32_t)ts * 64u, a_lo = a_hi + 32u;
+                    const uint64_t db = smem_desc(wring + (uint32_t)ts * slab_bytes);
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks)
+                        umma_ts_tf32(d_tmem, a_hi + 8u * ks, db + (uint64_t)((ks * 32) >> 4), idesc_wide,
+                                     ((s == 0 || s == ns1) && ks == 0) ? 0u : 1u);
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks)
+                        umma_ts_tf32(d_tmem, a_lo + 8u * ks, db + (uint64_t)((ks * 32) >> 4), idesc_hi, 1u);
+                    umma_commit(&afree[ts]);
+                    if (++ts == S) {
+                        ts = 0;
+                        ++pass;
+                    }
+                }
+                if (okm) umma_commit(&tfull[acc]);
+            }
+            if (!okm) atomicExch(fault, 6);
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue
+        // Group e takes items e, e+2, ... (accumulator e).  Phase 1, one row per lane: sum the partial
+        // accumulators, apply bias / ReLU / post, park the tile (and the mask bytes) in the warp's
+        // staging tiles.  Phase 2, lane = (column quad cq, row sub): gate, add the old C, store -- every
+        // global access of a warp covers four whole 128-byte row segments.
+        const int ew = warp - 5;                      // 0..7
+        const int e = ew >> 2;                        // group = accumulator
+        const int q = warp & 3;                       // TMEM lane quarter this warp may read
+        float* stage = stage_out + ew * (32 * kStagePitch);
+        unsigned char* mstage = stage_mask + ew * (32 * kTsMaskPitch);
+        const int cq = lane & 7, sub = lane >> 3;
+        float* Cf = static_cast<float*>(a.C);
+        const bool wmask = a.relu && a.mask_out;
+        for (int i = tid - 160; i < a.groups * a.N; i += 256) {
+            sbias[i] = a.bias ? __ldg(a.bias + i) : 0.f;
+            float pv = a.post1 ? __ldg(a.post1 + i) : 0.f;
+            if (a.post2) pv += __ldg(a.post2 + i);
+            spost[i] = pv;
+        }
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        bool oke = true;
+        ItemCursor e_it;
+        e_it.init(blockIdx.x + (uint32_t)e * gridDim.x, 2 * gridDim.x, a.groups, n_tiles);
+        for (int64_t it = e; it < my_items && oke; it += 2) {
+            const int64_t row0 = e_it.row0();
+            const int g = e_it.g, nt = e_it.nt;
+            e_it.next();
+            const int n0 = nt * n_pad;
+            const int nn = min(n_pad, a.N - n0);
+            const int cs = a.c_start[g] + n0;
+            const int rows_here = (int)min((int64_t)32, a.M - (row0 + q * 32));   // valid rows of this warp's quarter
+            const int64_t rfirst = row0 + q * 32 + sub;
+            if (a.mul_pos && it + 2 < my_items && cq == 0) {
+                // the group's next item: ask for the lines of the gate it will read
+                const int64_t nrow = e_it.row0() + q * 32 + sub;
+                const int ncol0 = a.c_start[e_it.g] + e_it.nt * n_pad;
+                const int nnn = min(n_pad, a.N - e_it.nt * n_pad);
+                for (int i = 0; i < 8; ++i) {
+                    if (nrow + 4 * i >= a.M) break;
+                    for (int cc = 0; cc < nnn; cc += 32) {
+                        asm volatile("prefetch.global.L2 [%0];" ::"l"(static_cast<const char*>(a.mul_pos) +
+                                                                          ((nrow + 4 * i) * a.mul_pos_ld + ncol0 + cc) *
+                                                                              (a.mul_pos_dtype == SLICEGCN_F32 ? 4 : 2)));
+                    }
+                }
+            }
+            oke = mbar_wait(&tfull[e], (uint32_t)((it >> 1) & 1));
+            if (!oke) break;
+            tc_fence_after();
+            const uint32_t d_tmem = tmem + (uint32_t)e * accw + ((uint32_t)(q * 32) << 16);
+            for (int c0 = 0; c0 < nn; c0 += 32) {
+                const int n = c0 + cq * 4;            // first of this lane's four columns in phase 2
+                const bool col_ok = n < nn;           // nn is a multiple of 4 on this path
+                const int col = cs + n;
+                // ---- phase 1
+                float x[32];
+                tmem_ld32(d_tmem + (uint32_t)c0, x);
+                tmem_ld16_add<0>(d_tmem + (uint32_t)(n_pad + c0), x);
+                tmem_ld16_add<16>(d_tmem + (uint32_t)(n_pad + c0 + 16), x);
+                const float* bvec = sbias + g * a.N + n0 + c0;
+                const float* pvec = spost + g * a.N + n0 + c0;
+                uint32_t mbits = 0;
+#pragma unroll
+                for (int j = 0; j < 32; j += 4) {
+                    const float4 b4 = *reinterpret_cast<const float4*>(bvec + j);
+                    const float4 p4 = *reinterpret_cast<const float4*>(pvec + j);
+                    x[j] += b4.x; x[j + 1] += b4.y; x[j + 2] += b4.z; x[j + 3] += b4.w;
+                    if (a.relu) {
+#pragma unroll
+                        for (int t = 0; t < 4; ++t) {
+                            mbits |= (x[j + t] > 0.f ? 1u : 0u) << (j + t);
+                            x[j + t] = fmaxf(x[j + t], 0.f);
+                        }
+                    }
+                    x[j] += p4.x; x[j + 1] += p4.y; x[j + 2] += p4.z; x[j + 3] += p4.w;
+                }
+                if (fused) {
+                    tmem_ld16_add<0>(d_tmem + prodw + (uint32_t)c0, x);
+                    tmem_ld16_add<16>(d_tmem + prodw + (uint32_t)(c0 + 16), x);
+                    tmem_ld16_add<0>(d_tmem + prodw + (uint32_t)(n_pad + c0), x);
+                    tmem_ld16_add<16>(d_tmem + prodw + (uint32_t)(n_pad + c0 + 16), x);
+                }
+                if (c0 + 32 >= nn) {   // last read of this accumulator: hand it back to the MMA warp
+                    tc_fence_before();
+                    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&tfree[e])) : "memory");
+                }
+#pragma unroll
+                for (int j = 0; j < 32; j += 4)
+                    *reinterpret_cast<float4*>(stage + lane * kStagePitch + j) = make_float4(x[j], x[j + 1], x[j + 2], x[j + 3]);
+                if (wmask) {
+#pragma unroll
+                    for (int j = 0; j < 32; j += 16) {
+                        uint4 mb;
+                        mb.x = ((mbits >> (j + 0)) & 1u) | (((mbits >> (j + 1)) & 1u) << 8) | (((mbits >> (j + 2)) & 1u) << 16) | (((mbits >> (j + 3)) & 1u) << 24);
+                        mb.y = ((mbits >> (j + 4)) & 1u) | (((mbits >> (j + 5)) & 1u) << 8) | (((mbits >> (j + 6)) & 1u) << 16) | (((mbits >> (j + 7)) & 1u) << 24);
+                        mb.z = ((mbits >> (j + 8)) & 1u) | (((mbits >> (j + 9)) & 1u) << 8) | (((mbits >> (j + 10)) & 1u) << 16) | (((mbits >> (j + 11)) & 1u) << 24);
+                        mb.w = ((mbits >> (j + 12)) & 1u) | (((mbits >> (j + 13)) & 1u) << 8) | (((mbits >> (j + 14)) & 1u) << 16) | (((mbits >> (j + 15)) & 1u) << 24);
+                        *reinterpret_cast<uint4*>(mstage + lane * kTsMaskPitch + j) = mb;
+                    }
+                }
+                __syncwarp();
+                // ---- phase 2, four rows at a time (the lines of the gate values were requested into L2 an
+                // item earlier)
+#pragma unroll 1
+                for (int hh = 0; hh < 8; hh += 4) {
+                    float4 gate[4];
+                    if (a.mul_pos) {
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            gate[i] = make_float4(1.f, 1.f, 1.f, 1.f);
+                            if (col_ok && 4 * (hh + i) + sub < rows_here) {
+                                if (a.mul_pos_dtype == SLICEGCN_F32) {
+                                    gate[i] = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(a.mul_pos) +
+                                                                                    (rfirst + 4 * (hh + i)) * a.mul_pos_ld + col));
+                                } else {
+                                    const uint2 hq = __ldg(reinterpret_cast<const uint2*>(
+                                        static_cast<const __nv_bfloat16*>(a.mul_pos) + (rfirst + 4 * (hh + i)) * a.mul_pos_ld + col));
+                                    gate[i] = make_float4(__uint_as_float(hq.x << 16), __uint_as_float(hq.x & 0xffff0000u),
+                                                          __uint_as_float(hq.y << 16), __uint_as_float(hq.y & 0xffff0000u));
+                                }
+                            }
+                        }
+                    }
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int rr = 4 * (hh + i) + sub;
+                        if (!col_ok || rr >= rows_here) continue;
+                        const int64_t row = rfirst + 4 * (hh + i);
+                        float4 t = *reinterpret_cast<const float4*>(stage + rr * kStagePitch + cq * 4);
+                        if (wmask)
+                            *reinterpret_cast<uint32_t*>(a.mask_out + row * a.mask_ld + col) =
+                                *reinterpret_cast<const uint32_t*>(mstage + rr * kTsMaskPitch + cq * 4);
+                        if (a.mul_pos) {
+                            t.x = gate[i].x > 0.f ? t.x : 0.f;
+                            t.y = gate[i].y > 0.f ? t.y : 0.f;
+                            t.z = gate[i].z > 0.f ? t.z : 0.f;
+                            t.w = gate[i].w > 0.f ? t.w : 0.f;
+                        }
+                        if (a.accumulate) {
+                            // C += t at the L2: every element receives exactly one addition per launch, so the
+                            // result does not depend on the order, and the old value never travels to the SM
+                            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(Cf + row * a.ldc + col), "f"(t.x),
+                                         "f"(t.y), "f"(t.z), "f"(t.w)
+                                         : "memory");
+                        } else {
+                            *reinterpret_cast<float4*>(Cf + row * a.ldc + col) = t;
+                        }
+                    }
+                }
+                __syncwarp();
+            }
+        }
+        if (!oke && lane == 0) atomicExch(fault, 7);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 4) tmem_dealloc(tmem, 512);
+}
+
 int tc_n_pad(int N) { return N <= 256 ? ((N + 15) & ~15) : 256; }
 
 template <typename TA, typename TC, bool BF16>
@@ -939,6 +1376,26 @@ slicegcn_status_t tc_gemm_launch(const GemmArgs& a, void* image, int64_t image_b
     if (a.post2) cvec = cvec && ((uintptr_t)a.post2 % 16 == 0);
     (void)ces;
     const int64_t all_items = ((a.M + 127) / 128) * a.groups * n_tiles;
+    if constexpr (!BF16 && std::is_same<TA, float>::value && std::is_same<TC, float>::value) {
+        // narrow fp32 outputs (the sliced layers): the kernel that keeps the activation operand in TMEM
+        static const bool no_ts = getenv("SLICEGCN_NO_TS") != nullptr;
+        if (vec && cvec && !a.a_mask && !no_ws && !no_ts && n_pad <= (fused ? 32 : 64) && a.groups * a.N <= kWsVecFloats &&
+            all_items < ((int64_t)1 << 31)) {
+            const int ts_smem = kTsStages * 2 * n_pad * 128 + 4 * kTsRing * 4096 + 8 * 32 * kStagePitch * 4 + 8 * 32 * kTsMaskPitch +
+                                2 * (kWsVecFloats + 64) * 4 + 256 + 1024;
+            static bool ts_configured = false;
+            if (!ts_configured) {
+                SGCN_CUDA(cudaFuncSetAttribute(tc_gemm_ts_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
+                ts_configured = true;
+            }
+            int64_t tgrid = 148;
+            if (tgrid > all_items) tgrid = all_items;
+            tc_gemm_ts_kernel<<<(unsigned)tgrid, kTsThreads, ts_smem, st>>>(a, n_pad, n_tiles, static_cast<unsigned char*>(image), image2, fault);
+            SGCN_LAUNCH_CHECK();
+            count_launch(fused ? 3 : 2);
+            return SLICEGCN_OK;
+        }
+    }
     if (vec && cvec && !a.a_mask && !no_ws && all_items < ((int64_t)1 << 31)) {
         // warp-specialised kernel: one CTA per SM, ring depth from what fits in shared memory
         const int a_bytes = BF16 ? 16384 : 32768;
