@@ -9,6 +9,9 @@
 // one kind::f16 pass.  The hi/lo split needs a pass through registers anyway, so tiles are written
 // to shared memory with ordinary stores (swizzled by hand) followed by a proxy fence.
 // Every wait on an mbarrier is bounded; a wait that runs out sets the caller's status word.
+#include <cuda.h>
+
+#include <algorithm>
 #include <cstdlib>
 #include <type_traits>
 
@@ -171,6 +174,16 @@ __device__ __forceinline__ void umma_ts_tf32(uint32_t d_tmem, uint32_t a_tmem, u
         "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
         "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
         : "memory");
+}
+
+// One box of a 2-D tensor map, global -> shared, by the tensor copy engine; completion (bytes) is
+// counted on the mbarrier.  x (the contiguous coordinate) times the element size must be a multiple
+// of 16 bytes; rows or columns outside the tensor arrive as zeros.
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+                     smem_u32(dst)),
+                 "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
+                 : "memory");
 }
 
 // K-major, 128-byte swizzle: rows of 128 bytes, 8-row groups 1024 bytes apart
@@ -934,28 +947,32 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_gemm_ws_kernel(const GemmArg
 // memory traffic -- every activation byte is written by the copy, read and written twice by the
 // hi/lo split and read three times by the MMAs -- so here the activation operand never returns to
 // shared memory:
-//   warps 0-3   producers.  Warp w owns rows 32w..32w+31 of every tile.  It keeps a private ring of
-//               kTsRing raw slabs filled with cp.async (no barrier: nobody else touches its rows),
-//               reads the landed slab one row per lane, splits it in registers and writes hi and lo
-//               into a TMEM stage with tcgen05.st (row = TMEM lane, K along the columns -- the form
-//               the MMA takes its A operand in).  Thread 0 also requests the step's weight image.
+//   warp 5      loader.  One thread keeps a ring of kTsRing raw slabs (128 rows x 32 values, 128-byte
+//               swizzle) filled, one tensor copy (TMA) per step; rows past the matrix arrive as zeros.
+//   warps 0-3   producers.  Warp w owns rows 32w..32w+31 of every tile: it reads the landed slab one
+//               row per lane, splits it in registers and writes hi and lo into a TMEM stage with
+//               tcgen05.st (row = TMEM lane, K along the columns -- the form the MMA takes its A
+//               operand in).  Thread 0 also requests the step's weight image.  A K slab that runs past
+//               a group's K columns brings the neighbouring columns along; the weight image holds zeros
+//               there, so they do not contribute.
 //   warp 4      MMA issuer.  Per K slab two chains instead of three: A_hi x [B_hi | B_lo] (the image
 //               holds hi and lo back to back, so they form one operand of 2 n_pad rows) into
 //               accumulator columns [0, 2 n_pad), then A_lo x B_hi onto columns [0, n_pad).
-//   warps 5-12  epilogue, two groups of four that take alternate items (one per accumulator):
+//   warps 8-15  epilogue, two groups of four that take alternate items (one per accumulator):
 //               the halves (and the second product) are summed in registers in the row-per-lane
 //               form, bias / ReLU / post are applied there, and only the finished tile (plus the
 //               ReLU mask bytes) goes through a per-warp staging tile to be written in whole
 //               128-byte row segments.
 // TMEM columns: [accumulator 0][accumulator 1] (accw each) then kTsStages x 64 (A hi | A lo).
-constexpr int kTsThreads = 416;
-constexpr int kTsRing = 6;     // raw slabs per producer warp (kTsRing - 1 in flight)
+constexpr int kTsThreads = 512;
+constexpr int kTsRing = 6;     // raw slabs in flight or being read
 constexpr int kTsStages = 3;   // TMEM operand stages (with their weight images in shared memory)
 constexpr int kTsMaskPitch = 48;
 
 __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArgs a, const int n_pad, const int n_tiles,
                                                                    const unsigned char* image, const unsigned char* image2,
-                                                                   int* fault) {
+                                                                   int* fault, const __grid_constant__ CUtensorMap map_a,
+                                                                   const __grid_constant__ CUtensorMap map_a2) {
     extern __shared__ __align__(1024) unsigned char smem[];
     constexpr int R = kTsRing, S = kTsStages;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -963,8 +980,8 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
     const uint32_t slab_bytes = 2u * (uint32_t)n_pad * 128u;                  // weight image [hi | lo]
     const bool fused = a.A2 != nullptr;
     unsigned char* wring = base;                                              // [S] weight images
-    unsigned char* raw = wring + (uint32_t)S * slab_bytes;                    // [4 warps][R] x 4096 B
-    float* stage_out = reinterpret_cast<float*>(raw + 4 * R * 4096);          // [8 warps] 32 x kStagePitch floats
+    unsigned char* raw = wring + (uint32_t)S * slab_bytes;                    // [R] raw activation slabs, 128 rows x 128 B, swizzled
+    float* stage_out = reinterpret_cast<float*>(raw + R * 16384);             // [8 warps] 32 x kStagePitch floats
     unsigned char* stage_mask = reinterpret_cast<unsigned char*>(stage_out + 8 * 32 * kStagePitch);   // [8] 32 x kTsMaskPitch
     float* sbias = reinterpret_cast<float*>(stage_mask + 8 * 32 * kTsMaskPitch);
     float* spost = sbias + kWsVecFloats + 64;
@@ -972,7 +989,9 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
     uint64_t* afree = afull + S;                                              // [S] MMAs of the stage have completed
     uint64_t* tfull = afree + S;                                              // [2] accumulator complete
     uint64_t* tfree = tfull + 2;                                              // [2] accumulator drained (128 arrivals)
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tfree + 2);
+    uint64_t* rfull = tfree + 2;                                              // [R] raw slab landed (bytes)
+    uint64_t* rfree = rfull + R;                                              // [R] raw slab read by the four producer warps
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(rfree + R);
     const uint32_t prodw = 2u * (uint32_t)n_pad;            // columns of one product: [hi*hi + lo*hi | hi*lo]
     const uint32_t accw = fused ? 2 * prodw : prodw;        // columns of one accumulator
     const uint32_t a_col0 = 2 * accw;                       // first column of the operand stages
@@ -984,6 +1003,10 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
         for (int i = 0; i < 2; ++i) {
             mbar_init(&tfull[i], 1);
             mbar_init(&tfree[i], 128);
+        }
+        for (int i = 0; i < R; ++i) {
+            mbar_init(&rfull[i], 1);
+            mbar_init(&rfree[i], 4);
         }
     }
     if (warp == 4) tmem_alloc(tmem_slot, 512);
@@ -1003,60 +1026,16 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
 
     if (warp < 4) {
         // ------------------------------------------------------------ producers
-        unsigned char* myraw = raw + warp * (R * 4096);
-        const int c = lane & 7, r0 = lane >> 3;   // copy: 16-byte chunk c of rows r0 + 4 i of the warp's 32 rows
-        uint32_t woff[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) woff[i] = (uint32_t)((r0 + 4 * i) * 128 + ((c ^ ((r0 + 4 * i) & 7)) << 4));
-        const uint32_t roff = (uint32_t)(lane * 128);   // split: lane reads row `lane`, chunk cc at (cc ^ (lane & 7)) * 16
-        // cursor of the step whose loads are requested next, and of the step being converted
-        int i_rs = 0, i_s = 0;
-        ItemCursor i_it;
-        i_it.init(blockIdx.x, gridDim.x, a.groups, n_tiles);
-        auto issue = [&]() {
-            const int64_t row0 = i_it.row0();
-            const int g = i_it.g;
-            int s = i_s;
-            unsigned char* slot = myraw + i_rs * 4096;
-            if (++i_rs == R) i_rs = 0;
-            if (++i_s == n_slabs) {
-                i_s = 0;
-                i_it.next();
-            }
-            const bool second = s >= ns1;
-            if (second) s -= ns1;
-            const int k = s * 32 + c * 4;
-            const int64_t ld = second ? a.lda2 : a.lda;
-            const float* src0 = (second ? static_cast<const float*>(a.A2) + a.a2_start[g] : static_cast<const float*>(a.A) + a.a_start[g]) +
-                                (row0 + 32 * warp + r0) * ld + k;
-            const int64_t row_step = 4 * ld;
-            const uint32_t dst0 = smem_u32(slot);
-            const int rows_left = (int)min((int64_t)128, a.M - row0) - 32 * warp - r0;   // rows r0 + 4 i below this exist
-            const bool k_in = k < (second ? a.K2 : a.K);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const bool in = k_in && 4 * i < rows_left;
-                const float* src = in ? (src0 + i * row_step) : static_cast<const float*>(a.A);
-                const int sz = in ? 16 : 0;   // zero-fill outside the matrix
-                asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst0 + woff[i]), "l"(src), "r"(sz) : "memory");
-            }
-        };
-        for (int j = 0; j < R - 1; ++j) {   // exactly R-1 groups, empty past the end, so the count below holds
-            if (j < my_steps) issue();
-            asm volatile("cp.async.commit_group;" ::: "memory");
-        }
+        // lane reads row 32 warp + lane of the landed slab: 16-byte chunk cc sits at (cc ^ (row & 7)) * 16
+        const uint32_t roff = (uint32_t)((32 * warp + lane) * 128);
         int rs = 0, ts = 0, c_s = 0;
-        uint32_t pass = 0;
+        uint32_t pass = 0, rpass = 0;
         ItemCursor c_it;
         c_it.init(blockIdx.x, gridDim.x, a.groups, n_tiles);
         bool okp = true;
         for (int64_t j = 0; j < my_steps; ++j) {
-            // R-1+j groups so far; step j has landed once at most R-2 are pending
-            asm volatile("cp.async.wait_group %0;" ::"n"(R - 2) : "memory");
-            __syncwarp();   // every lane's copies of step j are in, every lane is done reading step j-1
-            if (j + R - 1 < my_steps) issue();   // into the slot step j-1 was read from
-            asm volatile("cp.async.commit_group;" ::: "memory");   // one group per step, empty or not
-            if (pass >= 1) okp = mbar_wait(&afree[ts], (pass - 1) & 1);
+            okp = mbar_wait(&rfull[rs], rpass & 1);
+            if (okp && pass >= 1) okp = mbar_wait(&afree[ts], (pass - 1) & 1);
             if (!okp) break;
             if (tid == 0) {
                 int s = c_s;
@@ -1074,7 +1053,7 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
             }
             __syncwarp();
             tc_fence_after();
-            const unsigned char* slot = myraw + rs * 4096 + roff;
+            const unsigned char* slot = raw + rs * 16384 + roff;
             const uint32_t t_hi = tmem + ((uint32_t)(32 * warp) << 16) + a_col0 + (uint32_t)ts * 64u;
 #pragma unroll
             for (int half = 0; half < 2; ++half) {   // 16 K values at a time keeps the register count down
@@ -1093,20 +1072,55 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
                     h[16 + 4 * cc + 2] = __float_as_uint(v.z - h2);
                     h[16 + 4 * cc + 3] = __float_as_uint(v.w - h3);
                 }
+                if (half == 1) {   // the slab is in registers: hand the slot back to the loader
+                    __syncwarp();
+                    if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&rfree[rs])) : "memory");
+                    __syncwarp();
+                }
                 tmem_st16<0>(t_hi + 16u * half, h);
                 tmem_st16<16>(t_hi + 32u + 16u * half, h);
             }
             tmem_st_wait();
             tc_fence_before();
             asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&afull[ts])) : "memory");
-            if (++rs == R) rs = 0;
+            if (++rs == R) {
+                rs = 0;
+                ++rpass;
+            }
             if (++ts == S) {
                 ts = 0;
                 ++pass;
             }
         }
-        asm volatile("cp.async.wait_group 0;" ::: "memory");
         if (!okp && lane == 0) atomicExch(fault, 5);
+    } else if (warp == 5) {
+        // ------------------------------------------------------------ loader: one tensor copy per step
+        if (lane == 0) {
+            int rs = 0, l_s = 0;
+            uint32_t rpass = 0;
+            ItemCursor l_it;
+            l_it.init(blockIdx.x, gridDim.x, a.groups, n_tiles);
+            for (int64_t j = 0; j < my_steps; ++j) {
+                if (rpass >= 1 && !mbar_wait(&rfree[rs], (rpass - 1) & 1)) {
+                    atomicExch(fault, 8);
+                    break;
+                }
+                int s = l_s;
+                const bool second = s >= ns1;
+                if (second) s -= ns1;
+                const int x = (second ? a.a2_start[l_it.g] : a.a_start[l_it.g]) + s * 32;
+                mbar_expect_tx(&rfull[rs], 16384u);
+                tma_load_2d(raw + rs * 16384, second ? &map_a2 : &map_a, x, (int)l_it.row0(), &rfull[rs]);
+                if (++l_s == n_slabs) {
+                    l_s = 0;
+                    l_it.next();
+                }
+                if (++rs == R) {
+                    rs = 0;
+                    ++rpass;
+                }
+            }
+        }
     } else if (warp == 4) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
@@ -1146,13 +1160,13 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
             }
             if (!okm) atomicExch(fault, 6);
         }
-    } else {
+    } else if (warp >= 8) {
         // ------------------------------------------------------------ epilogue
         // Group e takes items e, e+2, ... (accumulator e).  Phase 1, one row per lane: sum the partial
         // accumulators, apply bias / ReLU / post, park the tile (and the mask bytes) in the warp's
         // staging tiles.  Phase 2, lane = (column quad cq, row sub): gate, add the old C, store -- every
         // global access of a warp covers four whole 128-byte row segments.
-        const int ew = warp - 5;                      // 0..7
+        const int ew = warp - 8;                      // 0..7
         const int e = ew >> 2;                        // group = accumulator
         const int q = warp & 3;                       // TMEM lane quarter this warp may read
         float* stage = stage_out + ew * (32 * kStagePitch);
@@ -1160,7 +1174,7 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
         const int cq = lane & 7, sub = lane >> 3;
         float* Cf = static_cast<float*>(a.C);
         const bool wmask = a.relu && a.mask_out;
-        for (int i = tid - 160; i < a.groups * a.N; i += 256) {
+        for (int i = tid - 256; i < a.groups * a.N; i += 256) {
             sbias[i] = a.bias ? __ldg(a.bias + i) : 0.f;
             float pv = a.post1 ? __ldg(a.post1 + i) : 0.f;
             if (a.post2) pv += __ldg(a.post2 + i);
@@ -1306,6 +1320,29 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
     if (warp == 4) tmem_dealloc(tmem, 512);
 }
 
+// Tensor map over a row-major fp32 matrix for boxes of 128 rows x 32 columns (one activation slab),
+// written to shared memory with the 128-byte swizzle.  `cols` bounds the columns a box may read
+// (beyond it: zeros).  The encoder is a driver entry point, looked up once; false if unavailable.
+typedef CUresult (*TensorMapEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                      const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                      CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+bool make_slab_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int64_t ld) {
+    static TensorMapEncodeFn encode = [] {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult q = cudaDriverEntryPointSymbolNotFound;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess)
+            fn = nullptr;
+        return reinterpret_cast<TensorMapEncodeFn>(fn);
+    }();
+    if (!encode || rows < 1 || cols < 1) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)ld * sizeof(float)};
+    const cuuint32_t box[2] = {32, 128};
+    const cuuint32_t estr[2] = {1, 1};
+    return encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 int tc_n_pad(int N) { return N <= 256 ? ((N + 15) & ~15) : 256; }
 
 template <typename TA, typename TC, bool BF16>
@@ -1380,7 +1417,18 @@ slicegcn_status_t tc_gemm_launch(const GemmArgs& a, void* image, int64_t image_b
         // narrow fp32 outputs (the sliced layers): the kernel that keeps the activation operand in TMEM
         static const bool no_ts = getenv("SLICEGCN_NO_TS") != nullptr;
         if (vec && cvec && !a.a_mask && !no_ws && !no_ts && n_pad <= (fused ? 32 : 64) && a.groups * a.N <= kWsVecFloats &&
-            all_items < ((int64_t)1 << 31)) {
+            all_items < ((int64_t)1 << 31) && a.M < ((int64_t)1 << 31)) {
+            // columns the slabs may touch: up to the end of the last group (the rest reads as zeros)
+            int cols1 = 0, cols2 = 0;
+            for (int g = 0; g < a.groups; ++g) {
+                cols1 = std::max(cols1, a.a_start[g] + a.K);
+                if (fused) cols2 = std::max(cols2, a.a2_start[g] + a.K2);
+            }
+            CUtensorMap map_a, map_a2;
+            bool maps_ok = make_slab_map(&map_a, a.A, a.M, std::min<int64_t>(cols1, a.lda), a.lda);
+            if (maps_ok && fused) maps_ok = make_slab_map(&map_a2, a.A2, a.M, std::min<int64_t>(cols2, a.lda2), a.lda2);
+            if (maps_ok && !fused) map_a2 = map_a;
+            if (maps_ok) {
             const int ts_smem = kTsStages * 2 * n_pad * 128 + 4 * kTsRing * 4096 + 8 * 32 * kStagePitch * 4 + 8 * 32 * kTsMaskPitch +
                                 2 * (kWsVecFloats + 64) * 4 + 256 + 1024;
             static bool ts_configured = false;
@@ -1390,10 +1438,12 @@ slicegcn_status_t tc_gemm_launch(const GemmArgs& a, void* image, int64_t image_b
             }
             int64_t tgrid = 148;
             if (tgrid > all_items) tgrid = all_items;
-            tc_gemm_ts_kernel<<<(unsigned)tgrid, kTsThreads, ts_smem, st>>>(a, n_pad, n_tiles, static_cast<unsigned char*>(image), image2, fault);
+            tc_gemm_ts_kernel<<<(unsigned)tgrid, kTsThreads, ts_smem, st>>>(a, n_pad, n_tiles, static_cast<unsigned char*>(image), image2, fault,
+                                                                            map_a, map_a2);
             SGCN_LAUNCH_CHECK();
             count_launch(fused ? 3 : 2);
             return SLICEGCN_OK;
+            }
         }
     }
     if (vec && cvec && !a.a_mask && !no_ws && all_items < ((int64_t)1 << 31)) {
