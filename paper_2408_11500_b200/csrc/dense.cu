@@ -430,9 +430,10 @@ slicegcn_status_t wgrad_run(const WgradArgs& a, void* scratch, int64_t scratch_b
         }
     }
     if (!no_tc && a.fault && a.K >= 1 && a.dW) {
-        const slicegcn_status_t rc = tc_wgrad_run(a, scratch, scratch_bytes, st);
+        bool bias_done = false;
+        const slicegcn_status_t rc = tc_wgrad_run(a, scratch, scratch_bytes, st, &bias_done);
         if (rc == SLICEGCN_OK) {
-            if (!bias) return SLICEGCN_OK;
+            if (!bias || bias_done) return SLICEGCN_OK;
             WgradArgs b = a;     // column sums only
             b.K = 0;
             b.dW = nullptr;

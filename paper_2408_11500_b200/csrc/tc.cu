@@ -1320,13 +1320,14 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
     if (warp == 4) tmem_dealloc(tmem, 512);
 }
 
-// Tensor map over a row-major fp32 matrix for boxes of 128 rows x 32 columns (one activation slab),
-// written to shared memory with the 128-byte swizzle.  `cols` bounds the columns a box may read
+// Tensor map over a row-major fp32 matrix for boxes of box_rows x box_cols values (default: one
+// activation slab of 128 rows x 32 columns), written to shared memory with the 128-byte swizzle or plain.  `cols` bounds the columns a box may read
 // (beyond it: zeros).  The encoder is a driver entry point, looked up once; false if unavailable.
 typedef CUresult (*TensorMapEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                       const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                       CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-bool make_slab_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int64_t ld) {
+bool make_slab_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int64_t ld, int box_cols = 32, int box_rows = 128,
+                   bool swizzle128 = true) {
     static TensorMapEncodeFn encode = [] {
         void* fn = nullptr;
         cudaDriverEntryPointQueryResult q = cudaDriverEntryPointSymbolNotFound;
@@ -1337,10 +1338,10 @@ bool make_slab_map(CUtensorMap* map, const void* base, int64_t rows, int64_t col
     if (!encode || rows < 1 || cols < 1) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
     const cuuint64_t strides[1] = {(cuuint64_t)ld * sizeof(float)};
-    const cuuint32_t box[2] = {32, 128};
+    const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
     return encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+                  swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 int tc_n_pad(int N) { return N <= 256 ? ((N + 15) & ~15) : 256; }
@@ -1872,6 +1873,242 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_wgrad_ws_kernel(const WgradA
     if (warp == 4) tmem_dealloc(tmem, ncols);
 }
 
+// ------------------------------------------------------------------------------ weight gradient, A^T operand in TMEM
+// dW = A^T B for fp32 operands and B tiles of at most 128 columns (the sliced layers).  Same tiling and
+// partial-sum scratch as the kernels above; what changes is the path of the operands, along the lines
+// of the TS GEMM:
+//   warp 5     loader: per slab of 32 rows one tensor copy of the A tile (32 x 128 values) and one of
+//              the B tile (32 x n_t), unswizzled, into a ring of kWtRing raw slots; rows past the end
+//              of the matrix and columns past its width arrive as zeros.
+//   warps 0-3  producers: lane m of warp w reads column 32w + m of the raw A slab (32 values down the
+//              rows -- consecutive lanes, consecutive words), splits them and writes hi and lo into a
+//              TMEM stage with tcgen05.st: A^T in the K-major form, M index = TMEM lane.  The B slab is
+//              split into the MN-major operand tile ("128-byte swizzle, 32-byte base"; per K atom the
+//              hi column blocks are followed by the lo column blocks, so [hi | lo] is one operand of
+//              2 n_t columns).  The producers also keep the column sums of B (the bias gradient) and,
+//              after the last slab, drain the accumulator into the scratch tile.
+//   warp 4     MMA issuer: per 8 rows A_hi x [B_hi | B_lo] and A_lo x B_hi.
+// TMEM columns: accumulator [hi*hi + lo*hi | hi*lo] (64 nbk), then kWtStages x 64 (A hi | A lo).
+constexpr int kWtThreads = 192;
+constexpr int kWtRing = 4;
+constexpr int kWtStages = 2;
+
+__global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradArgs a, const WgTcPlan pl, float* scratch, float* colsum,
+                                                                    int* fault, const __grid_constant__ CUtensorMap map_a,
+                                                                    const __grid_constant__ CUtensorMap map_b) {
+    extern __shared__ __align__(1024) unsigned char smem[];
+    constexpr int R = kWtRing, S = kWtStages;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int mt = blockIdx.y, chunk = blockIdx.x;
+    unsigned char* base = smem + ((1024u - (smem_u32(smem) & 1023u)) & 1023u);
+    const int nbk = (pl.n_t + 31) / 32;                      // column blocks of the B tile
+    const uint32_t b_raw_bytes = 32u * (uint32_t)pl.n_t * 4u;
+    const uint32_t slot_bytes = 16384u + ((b_raw_bytes + 1023u) & ~1023u);   // raw A | raw B
+    const uint32_t op_bytes = (uint32_t)nbk * 8192u;         // B operand stage: 8 K atoms x (nbk hi + nbk lo) x 512 B
+    unsigned char* ops = base;                               // [S]
+    unsigned char* raw = ops + S * op_bytes;                 // [R]
+    float* csum_s = reinterpret_cast<float*>(raw + R * slot_bytes);   // [4][128] column-sum partials
+    uint64_t* afull = reinterpret_cast<uint64_t*>(csum_s + 4 * 128);  // [S] 128 producer arrivals
+    uint64_t* afree = afull + S;                             // [S] MMAs of the stage completed
+    uint64_t* rfull = afree + S;                             // [R] raw slab landed
+    uint64_t* rfree = rfull + R;                             // [R] raw slab read by the four producer warps
+    uint64_t* tfull = rfree + R;                             // accumulator complete
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tfull + 1);
+    const uint32_t accw = 64u * (uint32_t)nbk;               // accumulator columns
+    if (tid == 0) {
+        for (int i = 0; i < S; ++i) {
+            mbar_init(&afull[i], 128);
+            mbar_init(&afree[i], 1);
+        }
+        for (int i = 0; i < R; ++i) {
+            mbar_init(&rfull[i], 1);
+            mbar_init(&rfree[i], 4);
+        }
+        mbar_init(tfull, 1);
+    }
+    if (warp == 4) tmem_alloc(tmem_slot, 512);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    const int64_t r_begin = (int64_t)chunk * pl.rows_per_chunk;
+    const int64_t r_end = min(a.M, r_begin + pl.rows_per_chunk);
+    const int n_slabs = r_end > r_begin ? (int)((r_end - r_begin + 31) / 32) : 0;
+
+    if (warp < 4) {
+        // ------------------------------------------------------------ producers (and, at the end, epilogue)
+        const int b_cc = tid & 31, b_r0 = tid >> 5;          // B: 16-byte column chunk b_cc of rows b_r0 + 4 i
+        const int nq = pl.n_t / 4;
+        const bool b_mine = b_cc < nq;
+        float4 csum = make_float4(0.f, 0.f, 0.f, 0.f);
+        int rs = 0, ts = 0;
+        uint32_t pass = 0, rpass = 0;
+        bool okp = true;
+        for (int j = 0; j < n_slabs; ++j) {
+            okp = mbar_wait(&rfull[rs], rpass & 1);
+            if (okp && pass >= 1) okp = mbar_wait(&afree[ts], (pass - 1) & 1);
+            if (!okp) break;
+            tc_fence_after();
+            const unsigned char* slot = raw + rs * slot_bytes;
+            // ---- A: column 32 warp + lane, 32 values down the rows
+            const float* acol = reinterpret_cast<const float*>(slot) + 32 * warp + lane;
+            const uint32_t t_hi = tmem + ((uint32_t)(32 * warp) << 16) + accw + (uint32_t)ts * 64u;
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                uint32_t h[32];   // [0,16): hi of rows 16 half ..; [16,32): lo of the same
+#pragma unroll
+                for (int k = 0; k < 16; ++k) {
+                    const float v = acol[(16 * half + k) * 128];
+                    const float hv = tf32_hi(v);
+                    h[k] = __float_as_uint(hv);
+                    h[16 + k] = __float_as_uint(v - hv);
+                }
+                tmem_st16<0>(t_hi + 16u * half, h);
+                tmem_st16<16>(t_hi + 32u + 16u * half, h);
+            }
+            // ---- B: split into the operand tile
+            if (b_mine) {
+                const unsigned char* braw = slot + 16384 + b_cc * 16;
+                unsigned char* op = ops + ts * op_bytes;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int r = b_r0 + 4 * i;
+                    const float4 v = *reinterpret_cast<const float4*>(braw + r * (pl.n_t * 4));
+                    const float h0 = tf32_hi(v.x), h1 = tf32_hi(v.y), h2 = tf32_hi(v.z), h3 = tf32_hi(v.w);
+                    const uint32_t off = (uint32_t)((((r >> 2) * 2 * nbk + (b_cc >> 3)) << 9) + ((r & 3) << 7) +
+                                                    (((((b_cc & 7) >> 1) ^ (r & 3))) << 5) + ((b_cc & 1) << 4));
+                    *reinterpret_cast<float4*>(op + off) = make_float4(h0, h1, h2, h3);
+                    *reinterpret_cast<float4*>(op + off + nbk * 512) = make_float4(v.x - h0, v.y - h1, v.z - h2, v.w - h3);
+                    csum.x += v.x; csum.y += v.y; csum.z += v.z; csum.w += v.w;
+                }
+            }
+            __syncwarp();
+            if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&rfree[rs])) : "memory");
+            tmem_st_wait();
+            tc_fence_before();
+            proxy_fence();
+            asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&afull[ts])) : "memory");
+            if (++rs == R) {
+                rs = 0;
+                ++rpass;
+            }
+            if (++ts == S) {
+                ts = 0;
+                ++pass;
+            }
+        }
+        if (!okp && lane == 0) atomicExch(fault, 8);
+        // column sums of this chunk's rows: four row groups per column chunk, added in a fixed order
+        if (colsum && (pl.b_cols_per_tile > 0 || mt == 0)) {
+            if (b_mine) *reinterpret_cast<float4*>(csum_s + b_r0 * 128 + b_cc * 4) = csum;
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (tid < pl.n_t) {
+                const float sum = ((csum_s[tid] + csum_s[128 + tid]) + csum_s[256 + tid]) + csum_s[384 + tid];
+                colsum[((int64_t)chunk * pl.m_tiles + mt) * pl.n_t + tid] = tid < pl.n_valid ? sum : 0.f;
+            }
+        }
+        // epilogue: partial tile -> scratch (row = A column 32 warp + lane of the tile)
+        float* out = scratch + ((int64_t)chunk * pl.m_tiles + mt) * 128 * pl.n_t + (int64_t)(warp * 32 + lane) * pl.n_t;
+        if (n_slabs > 0 && okp) {
+            if (mbar_wait(tfull, 0)) {
+                tc_fence_after();
+                const uint32_t d_tmem = tmem + ((uint32_t)(warp * 32) << 16);
+                for (int c0 = 0; c0 < pl.n_t; c0 += 16) {
+                    float x[32];
+#pragma unroll
+                    for (int jx = 0; jx < 16; ++jx) x[jx] = 0.f;
+                    tmem_ld16_add<0>(d_tmem + (uint32_t)c0, x);
+                    tmem_ld16_add<0>(d_tmem + (uint32_t)(32 * nbk + c0), x);
+#pragma unroll
+                    for (int jx = 0; jx < 16; jx += 4)
+                        *reinterpret_cast<float4*>(out + c0 + jx) = make_float4(x[jx], x[jx + 1], x[jx + 2], x[jx + 3]);
+                }
+            } else if (lane == 0) {
+                atomicExch(fault, 10);
+            }
+        } else if (n_slabs == 0) {
+            for (int jx = 0; jx < pl.n_t; ++jx) out[jx] = 0.f;
+        }
+    } else if (warp == 4) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            // M = 128 A-columns (K-major, from TMEM), N = B-columns (MN-major, from shared memory)
+            const uint32_t idesc_wide = idesc_f32acc(128, 64 * nbk, false) | (1u << 16);
+            const uint32_t idesc_hi = idesc_f32acc(128, 32 * nbk, false) | (1u << 16);
+            bool okm = true;
+            int ts = 0;
+            uint32_t pass = 0;
+            for (int j = 0; j < n_slabs && okm; ++j) {
+                okm = mbar_wait(&afull[ts], pass & 1);
+                if (!okm) break;
+                tc_fence_after();
+                const unsigned char* op = ops + ts * op_bytes;
+                const uint32_t a_hi = tmem + accw + (uint32_t)ts * 64u, a_lo = a_hi + 32u;
+#pragma unroll
+                for (int kb = 0; kb < 4; ++kb) {
+                    // one MMA covers 8 rows = two K atoms; column blocks are 512 bytes apart
+                    const uint64_t db = smem_desc_mn(op + kb * 2 * (2 * nbk * 512), 512, 2 * nbk * 512);
+                    umma_ts_tf32(tmem, a_hi + 8u * kb, db, idesc_wide, (j == 0 && kb == 0) ? 0u : 1u);
+                    umma_ts_tf32(tmem, a_lo + 8u * kb, db, idesc_hi, 1u);
+                }
+                umma_commit(&afree[ts]);
+                if (++ts == S) {
+                    ts = 0;
+                    ++pass;
+                }
+            }
+            if (okm) umma_commit(tfull);
+            else atomicExch(fault, 9);
+        }
+    } else {
+        // ------------------------------------------------------------ loader
+        if (lane == 0) {
+            int rs = 0;
+            uint32_t rpass = 0;
+            const int ax = pl.a_col0 + mt * 128, bx = pl.b_col0 + mt * pl.b_cols_per_tile;
+            for (int j = 0; j < n_slabs; ++j) {
+                if (rpass >= 1 && !mbar_wait(&rfree[rs], (rpass - 1) & 1)) {
+                    atomicExch(fault, 11);
+                    break;
+                }
+                unsigned char* slot = raw + rs * slot_bytes;
+                const int y = (int)(r_begin + (int64_t)j * 32);
+                mbar_expect_tx(&rfull[rs], 16384u + b_raw_bytes);
+                tma_load_2d(slot, &map_a, ax, y, &rfull[rs]);
+                tma_load_2d(slot + 16384, &map_b, bx, y, &rfull[rs]);
+                if (++rs == R) {
+                    rs = 0;
+                    ++rpass;
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 4) tmem_dealloc(tmem, 512);
+}
+
+// dbias[g][n] = sum over chunks of the column-sum partials (fixed order); same tile mapping as the dW reduce
+__global__ void tc_wgrad_bias_reduce_kernel(const float* colsum, const WgTcPlan pl, int groups, int N, int groups_per_tile, float* dbias,
+                                            float* dbias2) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= groups * N) return;
+    const int g = i / N, n = i % N;
+    int mt = 0, c = n;
+    if (groups_per_tile > 0) {
+        mt = g / groups_per_tile;
+        c = (g % groups_per_tile) * N + n;
+    } else if (groups_per_tile < 0) {
+        c = g * N + n;
+    }
+    float s = 0.f;
+    for (int ch = 0; ch < pl.n_chunks; ++ch) s += __ldg(colsum + ((int64_t)ch * pl.m_tiles + mt) * pl.n_t + c);
+    if (dbias) dbias[i] = s;
+    if (dbias2) dbias2[i] = s;
+}
+
 // dW[g][k][n] = sum over chunks of the partial tiles (fixed order)
 __global__ void tc_wgrad_reduce_kernel(const float* scratch, const WgTcPlan pl, int groups, int K, int N, int groups_per_tile,
                                        float* dW) {
@@ -1984,9 +2221,10 @@ int64_t tc_wgrad_scratch_bytes(const WgradArgs& a) {
 
 // Tensor-core weight gradient (dW only; bias sums stay with the CUDA-core kernel).  Returns
 // SLICEGCN_ERR_UNSUPPORTED when the shapes / alignments do not fit and nothing was launched.
-slicegcn_status_t tc_wgrad_run(const WgradArgs& a, void* scratch, int64_t scratch_bytes, cudaStream_t st) {
+slicegcn_status_t tc_wgrad_run(const WgradArgs& a, void* scratch, int64_t scratch_bytes, cudaStream_t st, bool* bias_done) {
     WgTcPlan pl;
     int gpt = 0;
+    if (bias_done) *bias_done = false;
     if (!a.fault || !wgrad_tc_plan(a, &pl, &gpt)) return SLICEGCN_ERR_UNSUPPORTED;
     static const bool no_ws = getenv("SLICEGCN_NO_WS") != nullptr;
     if (!no_ws && a.a_dtype == SLICEGCN_F32 && !a.b_mask) {
@@ -1995,6 +2233,41 @@ slicegcn_status_t tc_wgrad_run(const WgradArgs& a, void* scratch, int64_t scratc
         int gw = 0;
         if (wgrad_tc_plan(a, &pw, &gw, 1)) {
             const int nbk = (pw.n_t + 31) / 32;
+            static const bool no_ts = getenv("SLICEGCN_NO_TS") != nullptr;
+            const int64_t need_ts = (int64_t)pw.n_chunks * pw.m_tiles * 128 * pw.n_t * (int64_t)sizeof(float);
+            const int64_t need_cs = (int64_t)pw.n_chunks * pw.m_tiles * pw.n_t * (int64_t)sizeof(float);
+            if (!no_ts && nbk <= 4 && scratch && scratch_bytes >= need_ts && a.M < ((int64_t)1 << 31)) {
+                // B tiles of at most 128 columns: the kernel that keeps A^T in TMEM (and sums B's columns on the way)
+                const int b_total = a.groups * a.N;
+                CUtensorMap map_a, map_b;
+                bool maps_ok = make_slab_map(&map_a, a.A, a.M, std::min<int64_t>(pw.a_col0 + pw.a_cols, a.lda), a.lda, 128, 32, false) &&
+                               make_slab_map(&map_b, a.B, a.M, std::min<int64_t>(pw.b_col0 + b_total, a.ldb), a.ldb, pw.n_t, 32, false);
+                if (maps_ok) {
+                    const bool want_bias = (a.dbias || a.dbias2) && scratch_bytes >= need_ts + need_cs;
+                    float* colsum = want_bias ? static_cast<float*>(scratch) + need_ts / sizeof(float) : nullptr;
+                    const int slot_b = 16384 + ((32 * pw.n_t * 4 + 1023) & ~1023);
+                    const int ts_smem = kWtStages * nbk * 8192 + kWtRing * slot_b + 4 * 128 * 4 + 256 + 1024;
+                    static bool ts_configured = false;
+                    if (!ts_configured) {
+                        SGCN_CUDA(cudaFuncSetAttribute(tc_wgrad_ts_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
+                        ts_configured = true;
+                    }
+                    dim3 tgrid(pw.n_chunks, pw.m_tiles);
+                    tc_wgrad_ts_kernel<<<tgrid, kWtThreads, ts_smem, st>>>(a, pw, static_cast<float*>(scratch), colsum, a.fault, map_a, map_b);
+                    SGCN_LAUNCH_CHECK();
+                    const int64_t total_w = (int64_t)a.groups * a.K * a.N;
+                    tc_wgrad_reduce_kernel<<<(unsigned)((total_w + 255) / 256), 256, 0, st>>>(static_cast<const float*>(scratch), pw,
+                                                                                             a.groups, a.K, a.N, gw, a.dW);
+                    SGCN_LAUNCH_CHECK();
+                    if (want_bias) {
+                        tc_wgrad_bias_reduce_kernel<<<(b_total + 127) / 128, 128, 0, st>>>(colsum, pw, a.groups, a.N, gw, a.dbias, a.dbias2);
+                        SGCN_LAUNCH_CHECK();
+                        if (bias_done) *bias_done = true;
+                    }
+                    count_launch(want_bias ? 3 : 2);
+                    return SLICEGCN_OK;
+                }
+            }
             const int stage_b = 32768 + 2 * 4 * nbk * 1024;
             int D = (220 * 1024) / stage_b;
             if (D > 3) D = 3;
