@@ -1890,14 +1890,15 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_wgrad_ws_kernel(const WgradA
 //   warp 4     MMA issuer: per 8 rows A_hi x [B_hi | B_lo] and A_lo x B_hi.
 // TMEM columns: accumulator [hi*hi + lo*hi | hi*lo] (64 nbk), then kWtStages x 64 (A hi | A lo).
 constexpr int kWtThreads = 192;
-constexpr int kWtRing = 4;
-constexpr int kWtStages = 2;
 
+// WIDE: B tiles of 129..256 columns -- no room for [hi | lo] in one operand (three chains per slab) nor
+// for a second operand stage.
+template <bool WIDE>
 __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradArgs a, const WgTcPlan pl, float* scratch, float* colsum,
                                                                     int* fault, const __grid_constant__ CUtensorMap map_a,
                                                                     const __grid_constant__ CUtensorMap map_b) {
     extern __shared__ __align__(1024) unsigned char smem[];
-    constexpr int R = kWtRing, S = kWtStages;
+    constexpr int R = WIDE ? 3 : 4, S = WIDE ? 1 : 2;   // raw slots; operand stages (TMEM A + shared-memory B)
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int mt = blockIdx.y, chunk = blockIdx.x;
     unsigned char* base = smem + ((1024u - (smem_u32(smem) & 1023u)) & 1023u);
@@ -1914,7 +1915,7 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
     uint64_t* rfree = rfull + R;                             // [R] raw slab read by the four producer warps
     uint64_t* tfull = rfree + R;                             // accumulator complete
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tfull + 1);
-    const uint32_t accw = 64u * (uint32_t)nbk;               // accumulator columns
+    const uint32_t accw = (WIDE ? 32u : 64u) * (uint32_t)nbk;   // accumulator columns
     if (tid == 0) {
         for (int i = 0; i < S; ++i) {
             mbar_init(&afull[i], 128);
@@ -1939,7 +1940,9 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
 
     if (warp < 4) {
         // ------------------------------------------------------------ producers (and, at the end, epilogue)
-        const int b_cc = tid & 31, b_r0 = tid >> 5;          // B: 16-byte column chunk b_cc of rows b_r0 + 4 i
+        // B: 16-byte column chunk b_cc of rows b_r0 + BSTEP i
+        const int b_cc = WIDE ? (tid & 63) : (tid & 31), b_r0 = WIDE ? (tid >> 6) : (tid >> 5);
+        constexpr int BI = WIDE ? 16 : 8, BSTEP = WIDE ? 2 : 4;
         const int nq = pl.n_t / 4;
         const bool b_mine = b_cc < nq;
         float4 csum = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -1973,8 +1976,8 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
                 const unsigned char* braw = slot + 16384 + b_cc * 16;
                 unsigned char* op = ops + ts * op_bytes;
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const int r = b_r0 + 4 * i;
+                for (int i = 0; i < BI; ++i) {
+                    const int r = b_r0 + BSTEP * i;
                     const float4 v = *reinterpret_cast<const float4*>(braw + r * (pl.n_t * 4));
                     const float h0 = tf32_hi(v.x), h1 = tf32_hi(v.y), h2 = tf32_hi(v.z), h3 = tf32_hi(v.w);
                     const uint32_t off = (uint32_t)((((r >> 2) * 2 * nbk + (b_cc >> 3)) << 9) + ((r & 3) << 7) +
@@ -2002,11 +2005,12 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
         if (!okp && lane == 0) atomicExch(fault, 8);
         // column sums of this chunk's rows: four row groups per column chunk, added in a fixed order
         if (colsum && (pl.b_cols_per_tile > 0 || mt == 0)) {
-            if (b_mine) *reinterpret_cast<float4*>(csum_s + b_r0 * 128 + b_cc * 4) = csum;
+            if (b_mine) *reinterpret_cast<float4*>(csum_s + b_r0 * (WIDE ? 256 : 128) + b_cc * 4) = csum;
             asm volatile("bar.sync 1, 128;" ::: "memory");
-            if (tid < pl.n_t) {
-                const float sum = ((csum_s[tid] + csum_s[128 + tid]) + csum_s[256 + tid]) + csum_s[384 + tid];
-                colsum[((int64_t)chunk * pl.m_tiles + mt) * pl.n_t + tid] = tid < pl.n_valid ? sum : 0.f;
+            for (int cidx = tid; cidx < pl.n_t; cidx += 128) {
+                const float sum = WIDE ? csum_s[cidx] + csum_s[256 + cidx]
+                                       : ((csum_s[cidx] + csum_s[128 + cidx]) + csum_s[256 + cidx]) + csum_s[384 + cidx];
+                colsum[((int64_t)chunk * pl.m_tiles + mt) * pl.n_t + cidx] = cidx < pl.n_valid ? sum : 0.f;
             }
         }
         // epilogue: partial tile -> scratch (row = A column 32 warp + lane of the tile)
@@ -2020,7 +2024,7 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
 #pragma unroll
                     for (int jx = 0; jx < 16; ++jx) x[jx] = 0.f;
                     tmem_ld16_add<0>(d_tmem + (uint32_t)c0, x);
-                    tmem_ld16_add<0>(d_tmem + (uint32_t)(32 * nbk + c0), x);
+                    if (!WIDE) tmem_ld16_add<0>(d_tmem + (uint32_t)(32 * nbk + c0), x);
 #pragma unroll
                     for (int jx = 0; jx < 16; jx += 4)
                         *reinterpret_cast<float4*>(out + c0 + jx) = make_float4(x[jx], x[jx + 1], x[jx + 2], x[jx + 3]);
@@ -2035,7 +2039,7 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             // M = 128 A-columns (K-major, from TMEM), N = B-columns (MN-major, from shared memory)
-            const uint32_t idesc_wide = idesc_f32acc(128, 64 * nbk, false) | (1u << 16);
+            const uint32_t idesc_wide = idesc_f32acc(128, WIDE ? 32 * nbk : 64 * nbk, false) | (1u << 16);
             const uint32_t idesc_hi = idesc_f32acc(128, 32 * nbk, false) | (1u << 16);
             bool okm = true;
             int ts = 0;
@@ -2050,8 +2054,15 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
                 for (int kb = 0; kb < 4; ++kb) {
                     // one MMA covers 8 rows = two K atoms; column blocks are 512 bytes apart
                     const uint64_t db = smem_desc_mn(op + kb * 2 * (2 * nbk * 512), 512, 2 * nbk * 512);
-                    umma_ts_tf32(tmem, a_hi + 8u * kb, db, idesc_wide, (j == 0 && kb == 0) ? 0u : 1u);
-                    umma_ts_tf32(tmem, a_lo + 8u * kb, db, idesc_hi, 1u);
+                    if (WIDE) {
+                        const uint64_t db_lo = smem_desc_mn(op + kb * 2 * (2 * nbk * 512) + nbk * 512, 512, 2 * nbk * 512);
+                        umma_ts_tf32(tmem, a_hi + 8u * kb, db, idesc_hi, (j == 0 && kb == 0) ? 0u : 1u);
+                        umma_ts_tf32(tmem, a_lo + 8u * kb, db, idesc_hi, 1u);
+                        umma_ts_tf32(tmem, a_hi + 8u * kb, db_lo, idesc_hi, 1u);
+                    } else {
+                        umma_ts_tf32(tmem, a_hi + 8u * kb, db, idesc_wide, (j == 0 && kb == 0) ? 0u : 1u);
+                        umma_ts_tf32(tmem, a_lo + 8u * kb, db, idesc_hi, 1u);
+                    }
                 }
                 umma_commit(&afree[ts]);
                 if (++ts == S) {
@@ -2236,8 +2247,9 @@ slicegcn_status_t tc_wgrad_run(const WgradArgs& a, void* scratch, int64_t scratc
             static const bool no_ts = getenv("SLICEGCN_NO_TS") != nullptr;
             const int64_t need_ts = (int64_t)pw.n_chunks * pw.m_tiles * 128 * pw.n_t * (int64_t)sizeof(float);
             const int64_t need_cs = (int64_t)pw.n_chunks * pw.m_tiles * pw.n_t * (int64_t)sizeof(float);
-            if (!no_ts && nbk <= 4 && scratch && scratch_bytes >= need_ts && a.M < ((int64_t)1 << 31)) {
-                // B tiles of at most 128 columns: the kernel that keeps A^T in TMEM (and sums B's columns on the way)
+            if (!no_ts && nbk <= 8 && scratch && scratch_bytes >= need_ts && a.M < ((int64_t)1 << 31)) {
+                // the kernel that keeps A^T in TMEM (and sums B's columns on the way)
+                const bool wide = nbk > 4;
                 const int b_total = a.groups * a.N;
                 CUtensorMap map_a, map_b;
                 bool maps_ok = make_slab_map(&map_a, a.A, a.M, std::min<int64_t>(pw.a_col0 + pw.a_cols, a.lda), a.lda, 128, 32, false) &&
@@ -2246,14 +2258,18 @@ slicegcn_status_t tc_wgrad_run(const WgradArgs& a, void* scratch, int64_t scratc
                     const bool want_bias = (a.dbias || a.dbias2) && scratch_bytes >= need_ts + need_cs;
                     float* colsum = want_bias ? static_cast<float*>(scratch) + need_ts / sizeof(float) : nullptr;
                     const int slot_b = 16384 + ((32 * pw.n_t * 4 + 1023) & ~1023);
-                    const int ts_smem = kWtStages * nbk * 8192 + kWtRing * slot_b + 4 * 128 * 4 + 256 + 1024;
+                    const int ts_smem = (wide ? 1 : 2) * nbk * 8192 + (wide ? 3 : 4) * slot_b + 4 * 128 * 4 + 256 + 1024;
                     static bool ts_configured = false;
                     if (!ts_configured) {
-                        SGCN_CUDA(cudaFuncSetAttribute(tc_wgrad_ts_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
+                        SGCN_CUDA(cudaFuncSetAttribute(tc_wgrad_ts_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
+                        SGCN_CUDA(cudaFuncSetAttribute(tc_wgrad_ts_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
                         ts_configured = true;
                     }
                     dim3 tgrid(pw.n_chunks, pw.m_tiles);
-                    tc_wgrad_ts_kernel<<<tgrid, kWtThreads, ts_smem, st>>>(a, pw, static_cast<float*>(scratch), colsum, a.fault, map_a, map_b);
+                    if (wide)
+                        tc_wgrad_ts_kernel<true><<<tgrid, kWtThreads, ts_smem, st>>>(a, pw, static_cast<float*>(scratch), colsum, a.fault, map_a, map_b);
+                    else
+                        tc_wgrad_ts_kernel<false><<<tgrid, kWtThreads, ts_smem, st>>>(a, pw, static_cast<float*>(scratch), colsum, a.fault, map_a, map_b);
                     SGCN_LAUNCH_CHECK();
                     const int64_t total_w = (int64_t)a.groups * a.K * a.N;
                     tc_wgrad_reduce_kernel<<<(unsigned)((total_w + 255) / 256), 256, 0, st>>>(static_cast<const float*>(scratch), pw,
