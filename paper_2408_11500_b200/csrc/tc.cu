@@ -969,12 +969,13 @@ constexpr int kTsRing = 6;     // raw slabs in flight or being read
 constexpr int kTsStages = 3;   // TMEM operand stages (with their weight images in shared memory)
 constexpr int kTsMaskPitch = 48;
 
-__global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArgs a, const int n_pad, const int n_tiles,
+__global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArgs a, const int n_pad, const int n_tiles, const int R,
                                                                    const unsigned char* image, const unsigned char* image2,
                                                                    int* fault, const __grid_constant__ CUtensorMap map_a,
                                                                    const __grid_constant__ CUtensorMap map_a2) {
     extern __shared__ __align__(1024) unsigned char smem[];
-    constexpr int R = kTsRing, S = kTsStages;
+    constexpr int S = kTsStages;
+    const bool concat = n_pad <= 64;   // [B_hi | B_lo] as one operand; wider tiles take three chains per slab
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     unsigned char* base = smem + ((1024u - (smem_u32(smem) & 1023u)) & 1023u);
     const uint32_t slab_bytes = 2u * (uint32_t)n_pad * 128u;                  // weight image [hi | lo]
@@ -992,7 +993,7 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
     uint64_t* rfull = tfree + 2;                                              // [R] raw slab landed (bytes)
     uint64_t* rfree = rfull + R;                                              // [R] raw slab read by the four producer warps
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(rfree + R);
-    const uint32_t prodw = 2u * (uint32_t)n_pad;            // columns of one product: [hi*hi + lo*hi | hi*lo]
+    const uint32_t prodw = (concat ? 2u : 1u) * (uint32_t)n_pad;   // columns of one product: [hi*hi + lo*hi | hi*lo]
     const uint32_t accw = fused ? 2 * prodw : prodw;        // columns of one accumulator
     const uint32_t a_col0 = 2 * accw;                       // first column of the operand stages
     if (tid == 0) {
@@ -1143,13 +1144,24 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
                     tc_fence_after();
                     const uint32_t a_hi = tmem + a_col0 + (uint32_t)ts * 64u, a_lo = a_hi + 32u;
                     const uint64_t db = smem_desc(wring + (uint32_t)ts * slab_bytes);
+                    if (concat) {
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks)
-                        umma_ts_tf32(d_tmem, a_hi + 8u * ks, db + (uint64_t)((ks * 32) >> 4), idesc_wide,
-                                     ((s == 0 || s == ns1) && ks == 0) ? 0u : 1u);
+                        for (int ks = 0; ks < 4; ++ks)
+                            umma_ts_tf32(d_tmem, a_hi + 8u * ks, db + (uint64_t)((ks * 32) >> 4), idesc_wide,
+                                         ((s == 0 || s == ns1) && ks == 0) ? 0u : 1u);
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks)
-                        umma_ts_tf32(d_tmem, a_lo + 8u * ks, db + (uint64_t)((ks * 32) >> 4), idesc_hi, 1u);
+                        for (int ks = 0; ks < 4; ++ks)
+                            umma_ts_tf32(d_tmem, a_lo + 8u * ks, db + (uint64_t)((ks * 32) >> 4), idesc_hi, 1u);
+                    } else {
+                        const uint64_t db_lo = smem_desc(wring + (uint32_t)ts * slab_bytes + n_pad * 128);
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks) {
+                            const uint64_t adv = (uint64_t)((ks * 32) >> 4);
+                            umma_ts_tf32(d_tmem, a_hi + 8u * ks, db + adv, idesc_hi, (s == 0 && ks == 0) ? 0u : 1u);
+                            umma_ts_tf32(d_tmem, a_lo + 8u * ks, db + adv, idesc_hi, 1u);
+                            umma_ts_tf32(d_tmem, a_hi + 8u * ks, db_lo + adv, idesc_hi, 1u);
+                        }
+                    }
                     umma_commit(&afree[ts]);
                     if (++ts == S) {
                         ts = 0;
@@ -1218,8 +1230,10 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
                 // ---- phase 1
                 float x[32];
                 tmem_ld32(d_tmem + (uint32_t)c0, x);
-                tmem_ld16_add<0>(d_tmem + (uint32_t)(n_pad + c0), x);
-                tmem_ld16_add<16>(d_tmem + (uint32_t)(n_pad + c0 + 16), x);
+                if (concat) {
+                    tmem_ld16_add<0>(d_tmem + (uint32_t)(n_pad + c0), x);
+                    tmem_ld16_add<16>(d_tmem + (uint32_t)(n_pad + c0 + 16), x);
+                }
                 const float* bvec = sbias + g * a.N + n0 + c0;
                 const float* pvec = spost + g * a.N + n0 + c0;
                 uint32_t mbits = 0;
@@ -1350,11 +1364,16 @@ template <typename TA, typename TC, bool BF16>
 slicegcn_status_t tc_gemm_launch(const GemmArgs& a, void* image, int64_t image_bytes, int* fault, cudaStream_t st) {
     constexpr int KS = BF16 ? 64 : 32;
     constexpr int EPC = BF16 ? 8 : 4;
-    const int n_pad = tc_n_pad(a.N);
+    int n_pad = tc_n_pad(a.N);
+    const bool fused = a.A2 != nullptr;
+    // N = 256 in fp32: two column tiles of 128 suit the kernel with the activation operand in TMEM
+    // (two accumulators and the operand stages have to share the 512 TMEM columns); same image bytes
+    if (!BF16 && std::is_same<TA, float>::value && std::is_same<TC, float>::value && !fused && a.N == 256 && a.groups * a.N <= kWsVecFloats &&
+        getenv("SLICEGCN_NO_TS") == nullptr)
+        n_pad = 128;
     const int n_tiles = (a.N + n_pad - 1) / n_pad;
     const int n_slabs = (a.K + KS - 1) / KS;
     const int64_t need = (int64_t)a.groups * n_tiles * n_slabs * 2 * n_pad * 128;
-    const bool fused = a.A2 != nullptr;
     const int n_slabs2 = fused ? (a.K2 + KS - 1) / KS : 0;
     const int64_t need2 = (int64_t)a.groups * n_tiles * n_slabs2 * 2 * n_pad * 128;
     if (!image || image_bytes < need + need2) {
@@ -1417,7 +1436,7 @@ slicegcn_status_t tc_gemm_launch(const GemmArgs& a, void* image, int64_t image_b
     if constexpr (!BF16 && std::is_same<TA, float>::value && std::is_same<TC, float>::value) {
         // narrow fp32 outputs (the sliced layers): the kernel that keeps the activation operand in TMEM
         static const bool no_ts = getenv("SLICEGCN_NO_TS") != nullptr;
-        if (vec && cvec && !a.a_mask && !no_ws && !no_ts && n_pad <= (fused ? 32 : 64) && a.groups * a.N <= kWsVecFloats &&
+        if (vec && cvec && !a.a_mask && !no_ws && !no_ts && n_pad <= (fused ? 32 : 128) && a.groups * a.N <= kWsVecFloats &&
             all_items < ((int64_t)1 << 31) && a.M < ((int64_t)1 << 31)) {
             // columns the slabs may touch: up to the end of the last group (the rest reads as zeros)
             int cols1 = 0, cols2 = 0;
@@ -1430,7 +1449,8 @@ slicegcn_status_t tc_gemm_launch(const GemmArgs& a, void* image, int64_t image_b
             if (maps_ok && fused) maps_ok = make_slab_map(&map_a2, a.A2, a.M, std::min<int64_t>(cols2, a.lda2), a.lda2);
             if (maps_ok && !fused) map_a2 = map_a;
             if (maps_ok) {
-            const int ts_smem = kTsStages * 2 * n_pad * 128 + 4 * kTsRing * 4096 + 8 * 32 * kStagePitch * 4 + 8 * 32 * kTsMaskPitch +
+            const int ring = n_pad > 64 ? 4 : kTsRing;   // the wider weight images leave room for fewer raw slabs
+            const int ts_smem = kTsStages * 2 * n_pad * 128 + 4 * ring * 4096 + 8 * 32 * kStagePitch * 4 + 8 * 32 * kTsMaskPitch +
                                 2 * (kWsVecFloats + 64) * 4 + 256 + 1024;
             static bool ts_configured = false;
             if (!ts_configured) {
@@ -1439,7 +1459,7 @@ slicegcn_status_t tc_gemm_launch(const GemmArgs& a, void* image, int64_t image_b
             }
             int64_t tgrid = 148;
             if (tgrid > all_items) tgrid = all_items;
-            tc_gemm_ts_kernel<<<(unsigned)tgrid, kTsThreads, ts_smem, st>>>(a, n_pad, n_tiles, static_cast<unsigned char*>(image), image2, fault,
+            tc_gemm_ts_kernel<<<(unsigned)tgrid, kTsThreads, ts_smem, st>>>(a, n_pad, n_tiles, ring, static_cast<unsigned char*>(image), image2, fault,
                                                                             map_a, map_a2);
             SGCN_LAUNCH_CHECK();
             count_launch(fused ? 3 : 2);
