@@ -160,7 +160,8 @@ def test_spmm_is_deterministic_and_identity_holds(B, torch):
 # ------------------------------------------------------------------------------ one layer
 
 @pytest.mark.parametrize("order", ["agg", "xform"])
-@pytest.mark.parametrize("case", ["plain_gcn", "sliced", "overlap_se_bself", "shared_input"])
+@pytest.mark.parametrize("case", ["plain_gcn", "sliced", "overlap_se_bself", "shared_input", "aligned_16", "aligned_tail_64",
+                                  "aligned_single_256"])
 def test_layer_forward_backward(B, torch, order, case):
     n = 1500
     src, dst = synth.chung_lu_powerlaw(n, 7000, 2.2, 500, seed=6)
@@ -173,9 +174,17 @@ def test_layer_forward_backward(B, torch, order, case):
         p, in_cols, starts, w_in, h_s, use_self, use_bs, use_e = 4, 48, [0, 12, 24, 36], 12, 8, True, False, False
     elif case == "overlap_se_bself":
         p, in_cols, starts, w_in, h_s, use_self, use_bs, use_e = 3, 10, [0, 4, 6], 4, 5, True, True, True
-    else:
+    elif case == "shared_input":
         p, in_cols, starts, w_in, h_s, use_self, use_bs, use_e = 3, 13, [0, 0, 0], 13, 6, True, False, True
-    in_ld, out_ld = in_cols + 3, p * h_s + 2
+    # 16-byte-aligned shapes (the ones the tensor-copy / TMEM-operand kernels take), ragged last row tile
+    elif case == "aligned_16":
+        p, in_cols, starts, w_in, h_s, use_self, use_bs, use_e = 4, 64, [0, 16, 32, 48], 16, 16, True, True, True
+    elif case == "aligned_tail_64":      # K = 40: the second K slab is mostly past the slice
+        p, in_cols, starts, w_in, h_s, use_self, use_bs, use_e = 2, 80, [0, 40], 40, 64, True, False, False
+    else:                                # one group, 256 outputs: two column tiles of 128
+        p, in_cols, starts, w_in, h_s, use_self, use_bs, use_e = 1, 96, [0], 96, 256, True, False, True
+    pad_in, pad_out = (4, 4) if case.startswith("aligned") else (3, 2)
+    in_ld, out_ld = in_cols + pad_in, p * h_s + pad_out
     H = rng.standard_normal((n, in_cols)).astype(np.float32)
     Wa = (rng.standard_normal((p, w_in, h_s)) * 0.3).astype(np.float32)
     Ws = (rng.standard_normal((p, w_in, h_s)) * 0.3).astype(np.float32)
@@ -278,6 +287,8 @@ def _compare_epoch(gp, od, og, X, y, params, train_idx, tol, rnd=orc.identity, o
     dict(p=4, use_b_self=True, use_se=True, order=2),
     dict(p=4, order=1, L=3),
     dict(p=2, in_d=301, hidden=40, use_ff=True),
+    dict(p=4, in_d=64, hidden=64, C=8, use_ff=True, use_se=True, n=1111),
+    dict(p=2, in_d=48, hidden=256, C=12, L=2, n=900),
 ])
 def test_epoch_gradients_fp32(B, kw):
     kw = dict(kw)
