@@ -167,12 +167,22 @@ __device__ __forceinline__ void finish_chunk(const SpmmParams& p, int64_t row, i
 // the column indices of the next batch are requested before the current batch is gathered.
 // Chunks that consist of one long row are left to the segment kernels.
 constexpr int kRowsWarps = 4;   // warps per CTA of the row kernel
+// Occupancy and neighbors gathered per round.  Measured on B200: for rows of 256 bytes and more what
+// pays is resident warps (32 per SM, i.e. at most 64 registers) rather than loads per lane -- they run
+// fastest with four 16-byte loads in flight per lane; narrower rows (several rows per warp) and the
+// widest ones (three or four chunks per lane) keep eight loads per lane at 20 warps per SM.
+template <int L, int C>
+constexpr bool kDenseWarps = L >= 16 && C <= 2;
+template <int L, int C>
+constexpr int kGatherRound = kDenseWarps<L, C> ? (C == 2 ? 2 : 4) : ((8 / C) < 2 ? 2 : (8 / C));
+template <int L, int C>
+constexpr int kRowsBlocksPerSm = (kDenseWarps<L, C> ? 32 : 20) / kRowsWarps;
 
 template <typename TI, typename TO, int L, int C, bool EPI>
 __device__ __forceinline__ void spmm_rows_block(const SpmmParams& p, const int64_t vblock) {
     constexpr int V = Vec<TI>::V;
     constexpr int RPW = 32 / L;
-    constexpr int U = (8 / C) < 2 ? 2 : (8 / C);   // neighbors gathered per round: U*C 16-byte loads per lane
+    constexpr int U = kGatherRound<L, C>;   // neighbors gathered per round: U*C 16-byte loads per lane
     // (column index, 1/sqrt(deg) bits) of the current batch, one slot per lane: read back as one
     // broadcast 8-byte load per neighbor
     __shared__ int2 nbuf[kRowsWarps][32];
@@ -309,7 +319,7 @@ __device__ __forceinline__ void spmm_segment_block(const SpmmParams& p, const in
     const int row = __ldg(p.long_rows + li);
     const int start = __ldg(p.rowptr + row) + (seg - __ldg(p.seg_ptr + li)) * kSegment;
     const int end = min(__ldg(p.rowptr + row + 1), start + kSegment);
-    constexpr int U = (8 / C) < 2 ? 2 : (8 / C);   // neighbors gathered per round
+    constexpr int U = kGatherRound<L, C>;   // neighbors gathered per round
     __shared__ int2 nbuf[kRowsWarps][32];          // (column index, 1/sqrt(deg) bits) of the current batch
     int2* nb = &nbuf[threadIdx.x >> 5][sub * L];
     const uint32_t row16 = (uint32_t)((p.ldx * (int64_t)sizeof(TI)) >> 4);
@@ -404,7 +414,7 @@ __device__ __forceinline__ void spmm_segment_block(const SpmmParams& p, const in
 // One launch for both kinds of work: the first seg_blocks CTAs reduce the segments of the long rows
 // (they are the heaviest items, so they start first), the others the row chunks.
 template <typename TI, typename TO, int L, int C, bool EPI>
-__global__ void __launch_bounds__(kRowsWarps * 32, 20 / kRowsWarps) spmm_rows_kernel(const SpmmParams p, const int seg_blocks) {
+__global__ void __launch_bounds__(kRowsWarps * 32, kRowsBlocksPerSm<L, C>) spmm_rows_kernel(const SpmmParams p, const int seg_blocks) {
     if ((int)blockIdx.x < seg_blocks)
         spmm_segment_block<TI, L, C>(p, blockIdx.x);
     else
