@@ -236,11 +236,10 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     params.copy_(params0); m1.zero_(); m2.zero_()
 
     def e2e_step(ep):
-        Xd.copy_(Xp, non_blocking=True)
-        yd.copy_(yp, non_blocking=True)
-        epoch(ep, Xd, yd)
-        loss_host.copy_(loss, non_blocking=True)
-        stream.synchronize()                   # the caller reads the loss of this step
+        # one C-ABI call: host X and labels in, loss out to host memory (copies and the wait are inside)
+        B.slicegcn_train_epoch_host(m, g, Xp, w["in_d"], yp, Xd, yd, None, 0, params, grads, m1, m2,
+                                    B.make_opt_desc(1e-3, ep, total_epochs), loss, loss_host, ws, ws_bytes,
+                                    stream.cuda_stream)
 
     for ep in range(max(args.warmup, 1)):
         e2e_step(ep)

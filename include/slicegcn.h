@@ -263,6 +263,25 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
                                        const slicegcn_opt_desc* opt, float* logits_out, float* loss_out,
                                        void* workspace, int64_t workspace_bytes, void* stream);
 
+/* The same iteration for callers whose inputs live in host memory (the paper's training loop,
+ * Algorithm 3, starts from the dataset in host memory): copies the feature matrix and the labels to
+ * the caller's device staging buffers, runs slicegcn_train_epoch on them, copies the loss back and
+ * waits for `stream`.
+ *   X_host      [host, n rows of in_d values of m's dtype, row pitch x_ld elements]
+ *   labels_host [host, int32 n]
+ *   X_stage     [device, n * x_ld elements of m's dtype], labels_stage [device, int32 n]: staging
+ *               owned by the caller, overwritten
+ *   loss_host   [host, one float] or NULL
+ *   loss_dev    [device, one float]: where the step leaves the loss before it is copied back
+ *   every other argument as for slicegcn_train_epoch (device memory).
+ * Host buffers should be page-locked: pageable memory works but the copies are slower and not
+ * asynchronous.  Synchronous: returns after the stream has drained.  Errors as above. */
+slicegcn_status_t slicegcn_train_epoch_host(const slicegcn_model* m, const slicegcn_graph* g, const void* X_host, int64_t x_ld,
+                                            const int32_t* labels_host, void* X_stage, int32_t* labels_stage,
+                                            const int32_t* train_idx, int64_t n_train, float* params, float* grads,
+                                            float* adam_m, float* adam_v, const slicegcn_opt_desc* opt, float* loss_dev,
+                                            float* loss_host, void* workspace, int64_t workspace_bytes, void* stream);
+
 /* ---------------------------------------------------------------------------------------------
  * Instrumentation for benchmarks (the paper reports only end-to-end epochs per second, Table IV;
  * this splits out the aggregation kernel).  Between profile_begin and profile_end every SpMM call

@@ -31,7 +31,7 @@ EXPORTS = [
     "slicegcn_spmm", "slicegcn_spmm_static_scratch", "slicegcn_layer_saved_bytes", "slicegcn_layer_workspace_bytes", "slicegcn_layer_forward",
     "slicegcn_layer_backward", "slicegcn_model_create", "slicegcn_model_destroy", "slicegcn_model_param_count",
     "slicegcn_model_param_elems", "slicegcn_model_num_tensors", "slicegcn_model_tensor_info", "slicegcn_model_slices",
-    "slicegcn_model_layer_order", "slicegcn_train_workspace_bytes", "slicegcn_train_epoch", "slicegcn_profile_begin",
+    "slicegcn_model_layer_order", "slicegcn_train_workspace_bytes", "slicegcn_train_epoch", "slicegcn_train_epoch_host", "slicegcn_profile_begin",
     "slicegcn_profile_end",
 ]
 
@@ -297,6 +297,15 @@ def slicegcn_train_epoch(m, g, X, x_ld: int, labels, train_idx, n_train: int, pa
                                      _vp(params), _vp(grads), _vp(adam_m), _vp(adam_v),
                                      byref(opt) if opt is not None else None, _vp(logits_out), _vp(loss_out),
                                      _vp(workspace), c_int64(workspace_bytes), _vp(stream)))
+
+
+def slicegcn_train_epoch_host(m, g, X_host, x_ld: int, labels_host, X_stage, labels_stage, train_idx, n_train: int, params,
+                              grads, adam_m, adam_v, opt: Optional[OptDesc], loss_dev, loss_host, workspace,
+                              workspace_bytes: int, stream=None) -> None:
+    _check(_lib.slicegcn_train_epoch_host(m, g, _vp(X_host), c_int64(x_ld), _vp(labels_host), _vp(X_stage), _vp(labels_stage),
+                                          _vp(train_idx), c_int64(n_train), _vp(params), _vp(grads), _vp(adam_m),
+                                          _vp(adam_v), byref(opt) if opt is not None else None, _vp(loss_dev),
+                                          _vp(loss_host), _vp(workspace), c_int64(workspace_bytes), _vp(stream)))
 
 
 def slicegcn_profile_begin() -> None:

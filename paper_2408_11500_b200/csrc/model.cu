@@ -1009,4 +1009,23 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
     return SLICEGCN_OK;
 }
 
+slicegcn_status_t slicegcn_train_epoch_host(const slicegcn_model* m, const slicegcn_graph* g, const void* X_host, int64_t x_ld,
+                                            const int32_t* labels_host, void* X_stage, int32_t* labels_stage,
+                                            const int32_t* train_idx, int64_t n_train, float* params, float* grads,
+                                            float* adam_m, float* adam_v, const slicegcn_opt_desc* opt, float* loss_dev,
+                                            float* loss_host, void* workspace, int64_t workspace_bytes, void* stream) {
+    if (!m || !g || !X_host || !labels_host || !X_stage || !labels_stage || !loss_dev)
+        SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "train_epoch_host: NULL argument");
+    if (x_ld < m->desc.in_d) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "train_epoch_host: x_ld < in_d");
+    cudaStream_t st = (cudaStream_t)stream;
+    const int64_t n = g->n;
+    SGCN_CUDA(cudaMemcpyAsync(X_stage, X_host, (size_t)(n * x_ld) * esize(m->desc.dtype), cudaMemcpyHostToDevice, st));
+    SGCN_CUDA(cudaMemcpyAsync(labels_stage, labels_host, (size_t)n * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    SGCN_TRY(slicegcn_train_epoch(m, g, X_stage, x_ld, labels_stage, train_idx, n_train, params, grads, adam_m, adam_v, opt, nullptr,
+                                  loss_dev, workspace, workspace_bytes, stream));
+    if (loss_host) SGCN_CUDA(cudaMemcpyAsync(loss_host, loss_dev, sizeof(float), cudaMemcpyDeviceToHost, st));
+    SGCN_CUDA(cudaStreamSynchronize(st));
+    return SLICEGCN_OK;
+}
+
 }  // extern "C"

@@ -420,3 +420,32 @@ def test_rmat_sweep_sampled_rows_and_identity(B, torch, relabel, dtype, width):
             np.testing.assert_allclose(idn, Xv, rtol=5e-6)
     finally:
         B.slicegcn_graph_destroy(g)
+
+
+def test_train_epoch_host_buffers_match_device_call(B, torch):
+    """The host-buffer entry point (copies inside the call) gives bit-identical loss, gradients and
+    updated parameters to the device-buffer call, from page-locked and from pageable memory."""
+    src, dst, X, y, mk, od, params = small_problem(p=4, in_d=64, hidden=64, C=8, n=1111)
+    gp = GpuProblem(len(X), src, dst, X, y, params, **mk)
+    try:
+        opt = B.make_opt_desc(1e-2, 3, 50)
+        p0 = gp.params.clone()
+        loss_dev = gp.epoch(opt)
+        want_g, want_p = gp.grads.clone(), gp.params.clone()
+        Xh = torch.from_numpy(np.ascontiguousarray(X, np.float32))
+        yh = torch.from_numpy(np.ascontiguousarray(y, np.int32))
+        for pinned in (True, False):
+            Xs, ys = (Xh.pin_memory(), yh.pin_memory()) if pinned else (Xh.clone(), yh.clone())
+            loss_host = torch.full((1,), float("nan")).pin_memory() if pinned else torch.full((1,), float("nan"))
+            Xd, yd = torch.full_like(gp.X, float("nan")), torch.zeros_like(gp.y)
+            gp.params.copy_(p0); gp.m1.zero_(); gp.m2.zero_(); gp.grads.fill_(float("nan")); gp.loss.zero_()
+            B.slicegcn_train_epoch_host(gp.m, gp.g, Xs, Xs.shape[1], ys, Xd, yd, None, 0, gp.params, gp.grads, gp.m1, gp.m2, opt,
+                                        gp.loss, loss_host, gp.ws, gp.ws_bytes, torch.cuda.current_stream().cuda_stream)
+            assert float(loss_host.item()) == loss_dev          # already there when the call returns
+            assert torch.equal(gp.grads, want_g) and torch.equal(gp.params, want_p)
+            assert torch.equal(Xd, gp.X) and torch.equal(yd, gp.y)
+        with pytest.raises(B.SliceGCNError):
+            B.slicegcn_train_epoch_host(gp.m, gp.g, None, 64, yh, Xd, yd, None, 0, gp.params, gp.grads, gp.m1, gp.m2, opt,
+                                        gp.loss, None, gp.ws, gp.ws_bytes, torch.cuda.current_stream().cuda_stream)
+    finally:
+        gp.close()
