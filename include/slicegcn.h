@@ -282,6 +282,23 @@ slicegcn_status_t slicegcn_train_epoch_host(const slicegcn_model* m, const slice
                                             float* adam_m, float* adam_v, const slicegcn_opt_desc* opt, float* loss_dev,
                                             float* loss_host, void* workspace, int64_t workspace_bytes, void* stream);
 
+/* num_epochs consecutive iterations of the loop of Algorithm 3 from host memory, epochs
+ * opt->epoch, opt->epoch + 1, ...  Every epoch copies the feature matrix and the labels from the
+ * host again (the caller may rewrite them between calls, not during one); the copy for epoch e+1
+ * runs on a second stream into the other staging buffer while epoch e computes, so in steady state
+ * the transfer is hidden behind the kernels.  Each epoch's loss is copied to losses_host[e] as
+ * soon as it exists.
+ *   X_stage0/1 [device, n * x_ld elements each], labels_stage0/1 [device, int32 n each]
+ *   losses_dev [device, num_epochs floats], losses_host [host, num_epochs floats] or NULL
+ *   opt        required (the epoch index advances inside the call)
+ * Creates and destroys one stream and four events per call.  Synchronous.  Errors as above. */
+slicegcn_status_t slicegcn_train_epochs_host(const slicegcn_model* m, const slicegcn_graph* g, const void* X_host, int64_t x_ld,
+                                             const int32_t* labels_host, void* X_stage0, void* X_stage1, int32_t* labels_stage0,
+                                             int32_t* labels_stage1, const int32_t* train_idx, int64_t n_train, float* params,
+                                             float* grads, float* adam_m, float* adam_v, const slicegcn_opt_desc* opt,
+                                             int32_t num_epochs, float* losses_dev, float* losses_host, void* workspace,
+                                             int64_t workspace_bytes, void* stream);
+
 /* ---------------------------------------------------------------------------------------------
  * Instrumentation for benchmarks (the paper reports only end-to-end epochs per second, Table IV;
  * this splits out the aggregation kernel).  Between profile_begin and profile_end every SpMM call

@@ -31,7 +31,7 @@ EXPORTS = [
     "slicegcn_spmm", "slicegcn_spmm_static_scratch", "slicegcn_layer_saved_bytes", "slicegcn_layer_workspace_bytes", "slicegcn_layer_forward",
     "slicegcn_layer_backward", "slicegcn_model_create", "slicegcn_model_destroy", "slicegcn_model_param_count",
     "slicegcn_model_param_elems", "slicegcn_model_num_tensors", "slicegcn_model_tensor_info", "slicegcn_model_slices",
-    "slicegcn_model_layer_order", "slicegcn_train_workspace_bytes", "slicegcn_train_epoch", "slicegcn_train_epoch_host", "slicegcn_profile_begin",
+    "slicegcn_model_layer_order", "slicegcn_train_workspace_bytes", "slicegcn_train_epoch", "slicegcn_train_epoch_host", "slicegcn_train_epochs_host", "slicegcn_profile_begin",
     "slicegcn_profile_end",
 ]
 
@@ -306,6 +306,16 @@ def slicegcn_train_epoch_host(m, g, X_host, x_ld: int, labels_host, X_stage, lab
                                           _vp(train_idx), c_int64(n_train), _vp(params), _vp(grads), _vp(adam_m),
                                           _vp(adam_v), byref(opt) if opt is not None else None, _vp(loss_dev),
                                           _vp(loss_host), _vp(workspace), c_int64(workspace_bytes), _vp(stream)))
+
+
+def slicegcn_train_epochs_host(m, g, X_host, x_ld: int, labels_host, X_stage0, X_stage1, labels_stage0, labels_stage1, train_idx,
+                               n_train: int, params, grads, adam_m, adam_v, opt: OptDesc, num_epochs: int, losses_dev,
+                               losses_host, workspace, workspace_bytes: int, stream=None) -> None:
+    _check(_lib.slicegcn_train_epochs_host(m, g, _vp(X_host), c_int64(x_ld), _vp(labels_host), _vp(X_stage0), _vp(X_stage1),
+                                           _vp(labels_stage0), _vp(labels_stage1), _vp(train_idx), c_int64(n_train),
+                                           _vp(params), _vp(grads), _vp(adam_m), _vp(adam_v), byref(opt), c_int32(num_epochs),
+                                           _vp(losses_dev), _vp(losses_host), _vp(workspace), c_int64(workspace_bytes),
+                                           _vp(stream)))
 
 
 def slicegcn_profile_begin() -> None:

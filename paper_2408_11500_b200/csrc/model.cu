@@ -1028,4 +1028,75 @@ slicegcn_status_t slicegcn_train_epoch_host(const slicegcn_model* m, const slice
     return SLICEGCN_OK;
 }
 
+slicegcn_status_t slicegcn_train_epochs_host(const slicegcn_model* m, const slicegcn_graph* g, const void* X_host, int64_t x_ld,
+                                             const int32_t* labels_host, void* X_stage0, void* X_stage1, int32_t* labels_stage0,
+                                             int32_t* labels_stage1, const int32_t* train_idx, int64_t n_train, float* params,
+                                             float* grads, float* adam_m, float* adam_v, const slicegcn_opt_desc* opt,
+                                             int32_t num_epochs, float* losses_dev, float* losses_host, void* workspace,
+                                             int64_t workspace_bytes, void* stream) {
+    if (!m || !g || !X_host || !labels_host || !X_stage0 || !X_stage1 || !labels_stage0 || !labels_stage1 || !losses_dev || !opt)
+        SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "train_epochs_host: NULL argument");
+    if (x_ld < m->desc.in_d) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "train_epochs_host: x_ld < in_d");
+    if (num_epochs < 1) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "train_epochs_host: num_epochs < 1");
+    cudaStream_t st = (cudaStream_t)stream;
+    const int64_t n = g->n;
+    const size_t x_bytes = (size_t)(n * x_ld) * esize(m->desc.dtype), y_bytes = (size_t)n * sizeof(int32_t);
+    void* xs[2] = {X_stage0, X_stage1};
+    int32_t* ys[2] = {labels_stage0, labels_stage1};
+    cudaStream_t copy = nullptr;
+    cudaEvent_t ready[2] = {nullptr, nullptr}, done[2] = {nullptr, nullptr};
+    slicegcn_status_t rc = SLICEGCN_OK;
+    auto cleanup = [&]() {
+        for (int i = 0; i < 2; ++i) {
+            if (ready[i]) cudaEventDestroy(ready[i]);
+            if (done[i]) cudaEventDestroy(done[i]);
+        }
+        if (copy) cudaStreamDestroy(copy);
+    };
+    auto run = [&]() -> slicegcn_status_t {
+        SGCN_CUDA(cudaStreamCreateWithFlags(&copy, cudaStreamNonBlocking));
+        for (int i = 0; i < 2; ++i) {
+            SGCN_CUDA(cudaEventCreateWithFlags(&ready[i], cudaEventDisableTiming));
+            SGCN_CUDA(cudaEventCreateWithFlags(&done[i], cudaEventDisableTiming));
+        }
+        // the copies may not start before work already queued on the caller's stream has finished
+        // with the staging buffers
+        SGCN_CUDA(cudaEventRecord(done[0], st));
+        SGCN_CUDA(cudaStreamWaitEvent(copy, done[0], 0));
+        auto stage = [&](int b) -> slicegcn_status_t {
+            SGCN_CUDA(cudaMemcpyAsync(xs[b], X_host, x_bytes, cudaMemcpyHostToDevice, copy));
+            SGCN_CUDA(cudaMemcpyAsync(ys[b], labels_host, y_bytes, cudaMemcpyHostToDevice, copy));
+            SGCN_CUDA(cudaEventRecord(ready[b], copy));
+            return SLICEGCN_OK;
+        };
+        SGCN_TRY(stage(0));
+        for (int e = 0; e < num_epochs; ++e) {
+            const int b = e & 1;
+            if (e + 1 < num_epochs) {
+                // buffer b^1 was read by epoch e-1, which the caller's stream has been told to mark as done
+                if (e >= 1) SGCN_CUDA(cudaStreamWaitEvent(copy, done[b ^ 1], 0));
+                SGCN_TRY(stage(b ^ 1));
+            }
+            SGCN_CUDA(cudaStreamWaitEvent(st, ready[b], 0));
+            slicegcn_opt_desc o = *opt;
+            o.epoch = opt->epoch + e;
+            SGCN_TRY(slicegcn_train_epoch(m, g, xs[b], x_ld, ys[b], train_idx, n_train, params, grads, adam_m, adam_v, &o, nullptr,
+                                          losses_dev + e, workspace, workspace_bytes, stream));
+            SGCN_CUDA(cudaEventRecord(done[b], st));
+            if (losses_host)
+                SGCN_CUDA(cudaMemcpyAsync(losses_host + e, losses_dev + e, sizeof(float), cudaMemcpyDeviceToHost, st));
+        }
+        SGCN_CUDA(cudaStreamSynchronize(st));
+        SGCN_CUDA(cudaStreamSynchronize(copy));
+        return SLICEGCN_OK;
+    };
+    rc = run();
+    if (rc != SLICEGCN_OK) {   // drain whatever was queued before the events and the stream go away
+        cudaStreamSynchronize(st);
+        if (copy) cudaStreamSynchronize(copy);
+    }
+    cleanup();
+    return rc;
+}
+
 }  // extern "C"

@@ -444,6 +444,19 @@ def test_train_epoch_host_buffers_match_device_call(B, torch):
             assert float(loss_host.item()) == loss_dev          # already there when the call returns
             assert torch.equal(gp.grads, want_g) and torch.equal(gp.params, want_p)
             assert torch.equal(Xd, gp.X) and torch.equal(yd, gp.y)
+        # three epochs in one call (the copy of the next epoch overlaps the kernels) == three device calls
+        gp.params.copy_(p0); gp.m1.zero_(); gp.m2.zero_()
+        want_losses = [gp.epoch(B.make_opt_desc(1e-2, 3 + e, 50)) for e in range(3)]
+        want_p3 = gp.params.clone()
+        gp.params.copy_(p0); gp.m1.zero_(); gp.m2.zero_()
+        Xs, ys = Xh.pin_memory(), yh.pin_memory()
+        stage = [torch.full_like(gp.X, float("nan")) for _ in range(2)], [torch.zeros_like(gp.y) for _ in range(2)]
+        ld, lh = torch.zeros(3, device="cuda"), torch.full((3,), float("nan")).pin_memory()
+        B.slicegcn_train_epochs_host(gp.m, gp.g, Xs, Xs.shape[1], ys, stage[0][0], stage[0][1], stage[1][0], stage[1][1], None, 0,
+                                     gp.params, gp.grads, gp.m1, gp.m2, opt, 3, ld, lh, gp.ws, gp.ws_bytes,
+                                     torch.cuda.current_stream().cuda_stream)
+        assert [float(v) for v in lh] == want_losses
+        assert torch.equal(gp.params, want_p3)
         with pytest.raises(B.SliceGCNError):
             B.slicegcn_train_epoch_host(gp.m, gp.g, None, 64, yh, Xd, yd, None, 0, gp.params, gp.grads, gp.m1, gp.m2, opt,
                                         gp.loss, None, gp.ws, gp.ws_bytes, torch.cuda.current_stream().cuda_stream)
