@@ -317,27 +317,32 @@ __global__ void mask_mul4_kernel(int64_t M, int N4, const float4* in, int64_t ld
     }
 }
 
-// one warp per training row
+// LG lanes per training row (a warp holds 32/LG rows): few classes would leave most of a warp idle
+template <int LG>
 __global__ void softmax_ce_kernel(int C, const float* logits, const int32_t* labels, const int32_t* train_idx,
                                   int64_t n_train, float inv_n, float* dlogits, int64_t ld_d, float* row_loss) {
     const int lane = threadIdx.x & 31;
-    const int64_t t = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
-    if (t >= n_train) return;
-    const int64_t r = train_idx ? train_idx[t] : t;
+    const int sub = lane / LG, sl = lane % LG;
+    const int64_t t = ((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5) * (32 / LG) + sub;
+    const bool live = t < n_train;   // idle groups stay for the shuffles
+    const int64_t r = live ? (train_idx ? train_idx[t] : t) : 0;
     const float* z = logits + r * C;
     float mx = -INFINITY;
-    for (int c = lane; c < C; c += 32) mx = fmaxf(mx, z[c]);
+    if (live)
+        for (int c = sl; c < C; c += LG) mx = fmaxf(mx, z[c]);
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    for (int o = LG / 2; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o, LG));
     float s = 0.f;
-    for (int c = lane; c < C; c += 32) s += expf(z[c] - mx);
+    if (live)
+        for (int c = sl; c < C; c += LG) s += expf(z[c] - mx);
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    for (int o = LG / 2; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o, LG);
+    if (!live) return;
     const int y = labels[r];
     const float lse = mx + logf(s);
-    if (lane == 0) row_loss[t] = lse - z[y];
+    if (sl == 0) row_loss[t] = lse - z[y];
     const float inv_s = 1.f / s;
-    for (int c = lane; c < ld_d; c += 32) {
+    for (int c = sl; c < ld_d; c += LG) {
         float v = 0.f;   // padding columns stay zero
         if (c < C) v = (expf(z[c] - mx) * inv_s - (c == y ? 1.f : 0.f)) * inv_n;
         dlogits[r * ld_d + c] = v;
@@ -485,8 +490,12 @@ slicegcn_status_t softmax_ce_run(int64_t n, int C, const float* logits, const in
     if (train_idx) SGCN_CUDA(cudaMemsetAsync(dlogits, 0, sizeof(float) * n * ld_d, st));
     const int64_t cnt = train_idx ? n_train : n;
     if (cnt < 1) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "empty training set");
-    softmax_ce_kernel<<<(unsigned)((cnt + 7) / 8), 256, 0, st>>>(C, logits, labels, train_idx, cnt, 1.0f / (float)cnt,
-                                                                  dlogits, ld_d, row_loss);
+    if (C <= 64)
+        softmax_ce_kernel<8><<<(unsigned)((cnt + 31) / 32), 256, 0, st>>>(C, logits, labels, train_idx, cnt, 1.0f / (float)cnt,
+                                                                          dlogits, ld_d, row_loss);
+    else
+        softmax_ce_kernel<32><<<(unsigned)((cnt + 7) / 8), 256, 0, st>>>(C, logits, labels, train_idx, cnt, 1.0f / (float)cnt,
+                                                                         dlogits, ld_d, row_loss);
     SGCN_LAUNCH_CHECK();
     count_launch();
     if (loss_out) {

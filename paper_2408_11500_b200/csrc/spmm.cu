@@ -306,8 +306,9 @@ __device__ __forceinline__ void spmm_rows_block(const SpmmParams& p, const int64
 }
 
 // One warp per segment of a long row; the 32/L lane groups interleave over the segment's
-// neighbors and are combined with a butterfly (fixed order).
-template <typename TI, int L, int C>
+// neighbors and are combined with a butterfly (fixed order).  A row that fits one segment is
+// finished here; the others leave partial rows for the finish kernel.
+template <typename TI, typename TO, int L, int C, bool EPI>
 __device__ __forceinline__ void spmm_segment_block(const SpmmParams& p, const int64_t vblock) {
     constexpr int V = Vec<TI>::V;
     const int lane = threadIdx.x & 31;
@@ -396,7 +397,17 @@ __device__ __forceinline__ void spmm_segment_block(const SpmmParams& p, const in
         for (int c = 0; c < C; ++c)
 #pragma unroll
             for (int e = 0; e < V; ++e) acc[c][e] += __shfl_xor_sync(0xffffffffu, acc[c][e], off);
-    if (sub == 0) {
+    const bool single = __ldg(p.seg_ptr + li + 1) - __ldg(p.seg_ptr + li) == 1;
+    if (single) {
+        if (sub == 0) {
+            const float di = __ldg(p.dinv + row);
+#pragma unroll
+            for (int c = 0; c < C; ++c) {
+                const int chunk = sl + c * L;
+                if (chunk < p.nch) finish_chunk<TO, V, EPI>(p, row, chunk, di, acc[c]);
+            }
+        }
+    } else if (sub == 0) {
         float* out = p.partial + (int64_t)seg * (p.nch * V);
 #pragma unroll
         for (int c = 0; c < C; ++c) {
@@ -416,22 +427,27 @@ __device__ __forceinline__ void spmm_segment_block(const SpmmParams& p, const in
 template <typename TI, typename TO, int L, int C, bool EPI>
 __global__ void __launch_bounds__(kRowsWarps * 32, kRowsBlocksPerSm<L, C>) spmm_rows_kernel(const SpmmParams p, const int seg_blocks) {
     if ((int)blockIdx.x < seg_blocks)
-        spmm_segment_block<TI, L, C>(p, blockIdx.x);
+        spmm_segment_block<TI, TO, L, C, EPI>(p, blockIdx.x);
     else
         spmm_rows_block<TI, TO, L, C, EPI>(p, (int64_t)blockIdx.x - seg_blocks);
 }
 
 // Sums the partial rows of each long row in segment order, then scales / applies the epilogue.
+// One warp per (long row, block of 32 columns): the hub rows with dozens of segments set the
+// kernel's duration, so their columns are spread over many warps.
 template <typename TO, bool EPI>
 __global__ void __launch_bounds__(256) spmm_long_finish_kernel(const SpmmParams p, int pstride) {
     const int lane = threadIdx.x & 31;
     const int li = (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5);
     if (li >= p.n_long) return;
+    const int col = blockIdx.y * 32 + lane;
+    if (col >= p.width) return;
     const int64_t row = __ldg(p.long_rows + li);
     const int s0 = __ldg(p.seg_ptr + li), s1 = __ldg(p.seg_ptr + li + 1);
+    if (s1 - s0 == 1) return;   // finished by its segment's warp
     const float di = __ldg(p.dinv + row);
     TO* Y = static_cast<TO*>(p.Y) + row * p.ldy;
-    for (int col = lane; col < p.width; col += 32) {
+    {
         float a = 0.f;
         int s = s0;
         for (; s + 8 <= s1; s += 8) {   // eight loads in flight, summed in segment order
@@ -500,9 +516,9 @@ slicegcn_status_t launch_lc(const SpmmParams& p, bool epi, cudaStream_t st) {
     if (p.n_seg > 0) {
         const int pstride = p.nch * Vec<TI>::V;
         if (epi)
-            spmm_long_finish_kernel<TO, true><<<(p.n_long + 7) / 8, 256, 0, st>>>(p, pstride);
+            spmm_long_finish_kernel<TO, true><<<dim3((p.n_long + 7) / 8, (p.width + 31) / 32), 256, 0, st>>>(p, pstride);
         else
-            spmm_long_finish_kernel<TO, false><<<(p.n_long + 7) / 8, 256, 0, st>>>(p, pstride);
+            spmm_long_finish_kernel<TO, false><<<dim3((p.n_long + 7) / 8, (p.width + 31) / 32), 256, 0, st>>>(p, pstride);
         SGCN_LAUNCH_CHECK();
         count_launch();
     }
