@@ -1898,7 +1898,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_wgrad_ws_kernel(const WgradA
 // partial-sum scratch as the kernels above; what changes is the path of the operands, along the lines
 // of the TS GEMM:
 //   warp 5     loader: per slab of 32 rows one tensor copy of the A tile (32 x 128 values) and one of
-//              the B tile (32 x n_t), unswizzled, into a ring of kWtRing raw slots; rows past the end
+//              the B tile (32 x n_t), unswizzled, into a ring of raw slots; rows past the end
 //              of the matrix and columns past its width arrive as zeros.
 //   warps 0-3  producers: lane m of warp w reads column 32w + m of the raw A slab (32 values down the
 //              rows -- consecutive lanes, consecutive words), splits them and writes hi and lo into a
@@ -1908,17 +1908,17 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_wgrad_ws_kernel(const WgradA
 //              2 n_t columns).  The producers also keep the column sums of B (the bias gradient) and,
 //              after the last slab, drain the accumulator into the scratch tile.
 //   warp 4     MMA issuer: per 8 rows A_hi x [B_hi | B_lo] and A_lo x B_hi.
-// TMEM columns: accumulator [hi*hi + lo*hi | hi*lo] (64 nbk), then kWtStages x 64 (A hi | A lo).
+// TMEM columns: accumulator [hi*hi + lo*hi | hi*lo] (64 nbk), then two stages of 64 (A hi | A lo).
 constexpr int kWtThreads = 192;
 
-// WIDE: B tiles of 129..256 columns -- no room for [hi | lo] in one operand (three chains per slab) nor
-// for a second operand stage.
+// WIDE: B tiles of 129..256 columns -- no room for [hi | lo] in one operand (three chains per slab) and
+// only two raw slots.
 template <bool WIDE>
 __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradArgs a, const WgTcPlan pl, float* scratch, float* colsum,
                                                                     int* fault, const __grid_constant__ CUtensorMap map_a,
                                                                     const __grid_constant__ CUtensorMap map_b) {
     extern __shared__ __align__(1024) unsigned char smem[];
-    constexpr int R = WIDE ? 3 : 4, S = WIDE ? 1 : 2;   // raw slots; operand stages (TMEM A + shared-memory B)
+    constexpr int R = WIDE ? 2 : 4, S = 2;   // raw slots; operand stages (TMEM A + shared-memory B)
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int mt = blockIdx.y, chunk = blockIdx.x;
     unsigned char* base = smem + ((1024u - (smem_u32(smem) & 1023u)) & 1023u);
@@ -1928,8 +1928,8 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
     const uint32_t op_bytes = (uint32_t)nbk * 8192u;         // B operand stage: 8 K atoms x (nbk hi + nbk lo) x 512 B
     unsigned char* ops = base;                               // [S]
     unsigned char* raw = ops + S * op_bytes;                 // [R]
-    float* csum_s = reinterpret_cast<float*>(raw + R * slot_bytes);   // [4][128] column-sum partials
-    uint64_t* afull = reinterpret_cast<uint64_t*>(csum_s + 4 * 128);  // [S] 128 producer arrivals
+    float* csum_s = reinterpret_cast<float*>(raw);           // [4][128] column-sum partials: reuse raw slot 0 after the last slab
+    uint64_t* afull = reinterpret_cast<uint64_t*>(raw + R * slot_bytes);   // [S] 128 producer arrivals
     uint64_t* afree = afull + S;                             // [S] MMAs of the stage completed
     uint64_t* rfull = afree + S;                             // [R] raw slab landed
     uint64_t* rfree = rfull + R;                             // [R] raw slab read by the four producer warps
@@ -2025,6 +2025,7 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
         if (!okp && lane == 0) atomicExch(fault, 8);
         // column sums of this chunk's rows: four row groups per column chunk, added in a fixed order
         if (colsum && (pl.b_cols_per_tile > 0 || mt == 0)) {
+            asm volatile("bar.sync 1, 128;" ::: "memory");   // every producer has read its last raw slab
             if (b_mine) *reinterpret_cast<float4*>(csum_s + b_r0 * (WIDE ? 256 : 128) + b_cc * 4) = csum;
             asm volatile("bar.sync 1, 128;" ::: "memory");
             for (int cidx = tid; cidx < pl.n_t; cidx += 128) {
@@ -2140,42 +2141,55 @@ __global__ void tc_wgrad_bias_reduce_kernel(const float* colsum, const WgTcPlan 
     if (dbias2) dbias2[i] = s;
 }
 
-// dW[g][k][n] = sum over chunks of the partial tiles (fixed order)
-__global__ void tc_wgrad_reduce_kernel(const float* scratch, const WgTcPlan pl, int groups, int K, int N, int groups_per_tile,
-                                       float* dW) {
+// dW[g][k][n] = sum over chunks of the partial tiles (fixed order).  A block owns 32 consecutive
+// elements; its eight warps each sum every eighth chunk (a handful of independent loads, so the
+// kernel is not one long dependent chain per element) and the eight partial sums are added in
+// warp order.
+__global__ void __launch_bounds__(256) tc_wgrad_reduce_kernel(const float* scratch, const WgTcPlan pl, int groups, int K, int N,
+                                                              int groups_per_tile, float* dW) {
+    __shared__ float part[8][32];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const int64_t total = (int64_t)groups * K * N;
-    const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-    if (i >= total) return;
-    const int g = (int)(i / ((int64_t)K * N));
-    const int k = (int)((i / N) % K), n = (int)(i % N);
-    int mt, f, c;
-    if (groups_per_tile > 0) {   // grouped: tile mt holds groups mt*gpt .. ; block (g % gpt)
-        mt = g / groups_per_tile;
-        const int gl = g % groups_per_tile;
-        f = gl * K + k;
-        c = gl * N + n;
-    } else if (groups_per_tile < 0) {   // all groups share A: tiles over K, group g in columns g*N ..
-        mt = k / 128;
-        f = k % 128;
-        c = g * N + n;
-    } else {                     // one group: tiles over K
-        mt = k / 128;
-        f = k % 128;
-        c = n;
-    }
+    const int64_t i = blockIdx.x * (int64_t)32 + lane;
     float s = 0.f;
-    const float* p = scratch + ((int64_t)mt * 128 + f) * pl.n_t + c;
-    const int64_t stride = (int64_t)pl.m_tiles * 128 * pl.n_t;
-    int ch = 0;
-    for (; ch + 8 <= pl.n_chunks; ch += 8) {   // eight loads in flight, summed in chunk order
-        float v[8];
+    if (i < total) {
+        const int g = (int)(i / ((int64_t)K * N));
+        const int k = (int)((i / N) % K), n = (int)(i % N);
+        int mt, f, c;
+        if (groups_per_tile > 0) {   // grouped: tile mt holds groups mt*gpt .. ; block (g % gpt)
+            mt = g / groups_per_tile;
+            const int gl = g % groups_per_tile;
+            f = gl * K + k;
+            c = gl * N + n;
+        } else if (groups_per_tile < 0) {   // all groups share A: tiles over K, group g in columns g*N ..
+            mt = k / 128;
+            f = k % 128;
+            c = g * N + n;
+        } else {                     // one group: tiles over K
+            mt = k / 128;
+            f = k % 128;
+            c = n;
+        }
+        const float* p = scratch + ((int64_t)mt * 128 + f) * pl.n_t + c;
+        const int64_t stride = (int64_t)pl.m_tiles * 128 * pl.n_t;
+        int ch = w;
+        for (; ch + 24 < pl.n_chunks; ch += 32) {   // four loads in flight, summed in chunk order
+            float v[4];
 #pragma unroll
-        for (int q = 0; q < 8; ++q) v[q] = __ldg(p + (ch + q) * stride);
+            for (int q = 0; q < 4; ++q) v[q] = __ldg(p + (ch + 8 * q) * stride);
 #pragma unroll
-        for (int q = 0; q < 8; ++q) s += v[q];
+            for (int q = 0; q < 4; ++q) s += v[q];
+        }
+        for (; ch < pl.n_chunks; ch += 8) s += __ldg(p + ch * stride);
     }
-    for (; ch < pl.n_chunks; ++ch) s += __ldg(p + ch * stride);
-    dW[i] = s;
+    part[w][lane] = s;
+    __syncthreads();
+    if (w == 0 && i < total) {
+        float t = part[0][lane];
+#pragma unroll
+        for (int q = 1; q < 8; ++q) t += part[q][lane];
+        dW[i] = t;
+    }
 }
 
 bool wgrad_tc_plan(const WgradArgs& a, WgTcPlan* pl, int* groups_per_tile, int force_per_sm = 0) {
@@ -2278,11 +2292,11 @@ slicegcn_status_t tc_wgrad_run(const WgradArgs& a, void* scratch, int64_t scratc
                     const bool want_bias = (a.dbias || a.dbias2) && scratch_bytes >= need_ts + need_cs;
                     float* colsum = want_bias ? static_cast<float*>(scratch) + need_ts / sizeof(float) : nullptr;
                     const int slot_b = 16384 + ((32 * pw.n_t * 4 + 1023) & ~1023);
-                    const int ts_smem = (wide ? 1 : 2) * nbk * 8192 + (wide ? 3 : 4) * slot_b + 4 * 128 * 4 + 256 + 1024;
+                    const int ts_smem = 2 * nbk * 8192 + (wide ? 2 : 4) * slot_b + 256 + 1024;
                     static bool ts_configured = false;
                     if (!ts_configured) {
-                        SGCN_CUDA(cudaFuncSetAttribute(tc_wgrad_ts_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
-                        SGCN_CUDA(cudaFuncSetAttribute(tc_wgrad_ts_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
+                        SGCN_CUDA(cudaFuncSetAttribute(tc_wgrad_ts_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+                        SGCN_CUDA(cudaFuncSetAttribute(tc_wgrad_ts_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
                         ts_configured = true;
                     }
                     dim3 tgrid(pw.n_chunks, pw.m_tiles);
@@ -2292,7 +2306,7 @@ slicegcn_status_t tc_wgrad_run(const WgradArgs& a, void* scratch, int64_t scratc
                         tc_wgrad_ts_kernel<false><<<tgrid, kWtThreads, ts_smem, st>>>(a, pw, static_cast<float*>(scratch), colsum, a.fault, map_a, map_b);
                     SGCN_LAUNCH_CHECK();
                     const int64_t total_w = (int64_t)a.groups * a.K * a.N;
-                    tc_wgrad_reduce_kernel<<<(unsigned)((total_w + 255) / 256), 256, 0, st>>>(static_cast<const float*>(scratch), pw,
+                    tc_wgrad_reduce_kernel<<<(unsigned)((total_w + 31) / 32), 256, 0, st>>>(static_cast<const float*>(scratch), pw,
                                                                                              a.groups, a.K, a.N, gw, a.dW);
                     SGCN_LAUNCH_CHECK();
                     if (want_bias) {
@@ -2323,7 +2337,7 @@ slicegcn_status_t tc_wgrad_run(const WgradArgs& a, void* scratch, int64_t scratc
                     tc_wgrad_ws_kernel<false><<<wgrid, kWsThreads, ws_smem, st>>>(a, pw, D, static_cast<float*>(scratch), a.fault);
                 SGCN_LAUNCH_CHECK();
                 const int64_t total_w = (int64_t)a.groups * a.K * a.N;
-                tc_wgrad_reduce_kernel<<<(unsigned)((total_w + 255) / 256), 256, 0, st>>>(static_cast<const float*>(scratch), pw,
+                tc_wgrad_reduce_kernel<<<(unsigned)((total_w + 31) / 32), 256, 0, st>>>(static_cast<const float*>(scratch), pw,
                                                                                          a.groups, a.K, a.N, gw, a.dW);
                 SGCN_LAUNCH_CHECK();
                 count_launch(2);
@@ -2348,7 +2362,7 @@ slicegcn_status_t tc_wgrad_run(const WgradArgs& a, void* scratch, int64_t scratc
         tc_wgrad_kernel<float, 1><<<grid, kWgThreads, smem_bytes, st>>>(a, pl, static_cast<float*>(scratch), a.fault);
     SGCN_LAUNCH_CHECK();
     const int64_t total = (int64_t)a.groups * a.K * a.N;
-    tc_wgrad_reduce_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(static_cast<const float*>(scratch), pl, a.groups,
+    tc_wgrad_reduce_kernel<<<(unsigned)((total + 31) / 32), 256, 0, st>>>(static_cast<const float*>(scratch), pl, a.groups,
                                                                            a.K, a.N, gpt, a.dW);
     SGCN_LAUNCH_CHECK();
     count_launch(2);
