@@ -369,7 +369,8 @@ slicegcn_status_t layer_backward_impl(const slicegcn_graph* g, const slicegcn_la
             SGCN_TRY(gemm_groups(dz, seq, st));
             SGCN_TRY(spmm_run(g, true, SLICEGCN_F32, SLICEGCN_F32, dZ, L.zt_ld, dH_in, din_ld, L.in_cols, nullptr, part,
                               part_bytes, st));
-            if (d->W_self) {
+            if (d->W_self) {   // added by the GEMM's epilogue (an accumulating epilogue in the SpMM measured slower:
+                               // its rows would wait for the old value at every row end)
                 dself.accumulate = 1;
                 SGCN_TRY(gemm_groups(dself, seq, st));
             }
@@ -424,10 +425,25 @@ slicegcn_status_t layer_backward_impl(const slicegcn_graph* g, const slicegcn_la
                 SGCN_CUDA(cudaMemset2DAsync(dH_in, din_ld * 4, 0, (size_t)L.in_cols * 4, L.n, st));
                 dt.accumulate = 1;
             }
-            SGCN_TRY(gemm_groups(dt, seq, st));
-            if (d->W_self) {
-                dself.accumulate = 1;
-                SGCN_TRY(gemm_groups(dself, seq, st));
+            bool done = false;
+            if (d->W_self && !seq) {   // both products in one pass: dH_in = dT W_agg^T + dH W_self^T
+                GemmArgs both = dt;
+                both.A2 = dH_out;
+                both.lda2 = dout_ld;
+                both.B2 = d->W_self;
+                both.b2_gstride = dself.b_gstride;
+                both.K2 = L.h_s;
+                for (int i = 0; i < L.p; ++i) both.a2_start[i] = i * L.h_s;
+                const slicegcn_status_t rc = gemm_run(both, st);
+                if (rc == SLICEGCN_OK) done = true;
+                else if (rc != SLICEGCN_ERR_UNSUPPORTED) return rc;
+            }
+            if (!done) {
+                SGCN_TRY(gemm_groups(dt, seq, st));
+                if (d->W_self) {
+                    dself.accumulate = 1;
+                    SGCN_TRY(gemm_groups(dself, seq, st));
+                }
             }
         }
     }

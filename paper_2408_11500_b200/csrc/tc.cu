@@ -166,6 +166,24 @@ __device__ __forceinline__ void tmem_ld16_add(uint32_t taddr, float (&x)[32]) {
 #pragma unroll
     for (int i = 0; i < 16; ++i) x[OFF + i] += __uint_as_float(r[i]);
 }
+// two loads of 32 lanes x 16 columns in flight, both added onto x[OFF..OFF+15]
+template <int OFF>
+__device__ __forceinline__ void tmem_ld16x2_add(uint32_t taddr0, uint32_t taddr1, float (&x)[32]) {
+    uint32_t r[16], q[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+          "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr0));
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(q[0]), "=r"(q[1]), "=r"(q[2]), "=r"(q[3]), "=r"(q[4]), "=r"(q[5]), "=r"(q[6]), "=r"(q[7]), "=r"(q[8]), "=r"(q[9]),
+          "=r"(q[10]), "=r"(q[11]), "=r"(q[12]), "=r"(q[13]), "=r"(q[14]), "=r"(q[15])
+        : "r"(taddr1));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) x[OFF + i] += __uint_as_float(r[i]) + __uint_as_float(q[i]);
+}
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 // D[tmem] (+)= A[tmem] * B[smem desc], tf32: A's row i sits in TMEM lane i, its K values in consecutive columns
 __device__ __forceinline__ void umma_ts_tf32(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
@@ -1186,6 +1204,7 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
         const int cq = lane & 7, sub = lane >> 3;
         float* Cf = static_cast<float*>(a.C);
         const bool wmask = a.relu && a.mask_out;
+        const bool has_vec = a.bias || a.post1 || a.post2;   // otherwise the staged vectors are all zero
         for (int i = tid - 256; i < a.groups * a.N; i += 256) {
             sbias[i] = a.bias ? __ldg(a.bias + i) : 0.f;
             float pv = a.post1 ? __ldg(a.post1 + i) : 0.f;
@@ -1229,14 +1248,40 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
                 const int col = cs + n;
                 // ---- phase 1
                 float x[32];
-                tmem_ld32(d_tmem + (uint32_t)c0, x);
-                if (concat) {
-                    tmem_ld16_add<0>(d_tmem + (uint32_t)(n_pad + c0), x);
-                    tmem_ld16_add<16>(d_tmem + (uint32_t)(n_pad + c0 + 16), x);
+                if (concat) {   // both halves requested before the one wait
+                    uint32_t u[32], v[32];
+                    tmem_ld32_issue(d_tmem + (uint32_t)c0, u);
+                    tmem_ld32_issue(d_tmem + (uint32_t)(n_pad + c0), v);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) x[j] = __uint_as_float(u[j]) + __uint_as_float(v[j]);
+                } else {
+                    tmem_ld32(d_tmem + (uint32_t)c0, x);
+                }
+                // gate values of phase 2: requested as soon as the accumulator halves are summed (their lines were
+                // asked into L2 an item earlier), used after the tile has been staged
+                float4 gate[8];
+                if (a.mul_pos) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        gate[i] = make_float4(1.f, 1.f, 1.f, 1.f);
+                        if (col_ok && 4 * i + sub < rows_here) {
+                            if (a.mul_pos_dtype == SLICEGCN_F32) {
+                                gate[i] = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(a.mul_pos) +
+                                                                                (rfirst + 4 * i) * a.mul_pos_ld + col));
+                            } else {
+                                const uint2 hq = __ldg(reinterpret_cast<const uint2*>(
+                                    static_cast<const __nv_bfloat16*>(a.mul_pos) + (rfirst + 4 * i) * a.mul_pos_ld + col));
+                                gate[i] = make_float4(__uint_as_float(hq.x << 16), __uint_as_float(hq.x & 0xffff0000u),
+                                                      __uint_as_float(hq.y << 16), __uint_as_float(hq.y & 0xffff0000u));
+                            }
+                        }
+                    }
                 }
                 const float* bvec = sbias + g * a.N + n0 + c0;
                 const float* pvec = spost + g * a.N + n0 + c0;
                 uint32_t mbits = 0;
+                if (has_vec || a.relu) {
 #pragma unroll
                 for (int j = 0; j < 32; j += 4) {
                     const float4 b4 = *reinterpret_cast<const float4*>(bvec + j);
@@ -1251,11 +1296,10 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
                     }
                     x[j] += p4.x; x[j + 1] += p4.y; x[j + 2] += p4.z; x[j + 3] += p4.w;
                 }
-                if (fused) {
-                    tmem_ld16_add<0>(d_tmem + prodw + (uint32_t)c0, x);
-                    tmem_ld16_add<16>(d_tmem + prodw + (uint32_t)(c0 + 16), x);
-                    tmem_ld16_add<0>(d_tmem + prodw + (uint32_t)(n_pad + c0), x);
-                    tmem_ld16_add<16>(d_tmem + prodw + (uint32_t)(n_pad + c0 + 16), x);
+                }
+                if (fused) {   // the second product's halves, 16 columns of each per wait
+                    tmem_ld16x2_add<0>(d_tmem + prodw + (uint32_t)c0, d_tmem + prodw + (uint32_t)(n_pad + c0), x);
+                    tmem_ld16x2_add<16>(d_tmem + prodw + (uint32_t)(c0 + 16), d_tmem + prodw + (uint32_t)(n_pad + c0 + 16), x);
                 }
                 if (c0 + 32 >= nn) {   // last read of this accumulator: hand it back to the MMA warp
                     tc_fence_before();
@@ -1276,52 +1320,30 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
                     }
                 }
                 __syncwarp();
-                // ---- phase 2, four rows at a time (the lines of the gate values were requested into L2 an
-                // item earlier)
-#pragma unroll 1
-                for (int hh = 0; hh < 8; hh += 4) {
-                    float4 gate[4];
+                // ---- phase 2
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int rr = 4 * i + sub;
+                    if (!col_ok || rr >= rows_here) continue;
+                    const int64_t row = rfirst + 4 * i;
+                    float4 t = *reinterpret_cast<const float4*>(stage + rr * kStagePitch + cq * 4);
+                    if (wmask)
+                        *reinterpret_cast<uint32_t*>(a.mask_out + row * a.mask_ld + col) =
+                            *reinterpret_cast<const uint32_t*>(mstage + rr * kTsMaskPitch + cq * 4);
                     if (a.mul_pos) {
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            gate[i] = make_float4(1.f, 1.f, 1.f, 1.f);
-                            if (col_ok && 4 * (hh + i) + sub < rows_here) {
-                                if (a.mul_pos_dtype == SLICEGCN_F32) {
-                                    gate[i] = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(a.mul_pos) +
-                                                                                    (rfirst + 4 * (hh + i)) * a.mul_pos_ld + col));
-                                } else {
-                                    const uint2 hq = __ldg(reinterpret_cast<const uint2*>(
-                                        static_cast<const __nv_bfloat16*>(a.mul_pos) + (rfirst + 4 * (hh + i)) * a.mul_pos_ld + col));
-                                    gate[i] = make_float4(__uint_as_float(hq.x << 16), __uint_as_float(hq.x & 0xffff0000u),
-                                                          __uint_as_float(hq.y << 16), __uint_as_float(hq.y & 0xffff0000u));
-                                }
-                            }
-                        }
+                        t.x = gate[i].x > 0.f ? t.x : 0.f;
+                        t.y = gate[i].y > 0.f ? t.y : 0.f;
+                        t.z = gate[i].z > 0.f ? t.z : 0.f;
+                        t.w = gate[i].w > 0.f ? t.w : 0.f;
                     }
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int rr = 4 * (hh + i) + sub;
-                        if (!col_ok || rr >= rows_here) continue;
-                        const int64_t row = rfirst + 4 * (hh + i);
-                        float4 t = *reinterpret_cast<const float4*>(stage + rr * kStagePitch + cq * 4);
-                        if (wmask)
-                            *reinterpret_cast<uint32_t*>(a.mask_out + row * a.mask_ld + col) =
-                                *reinterpret_cast<const uint32_t*>(mstage + rr * kTsMaskPitch + cq * 4);
-                        if (a.mul_pos) {
-                            t.x = gate[i].x > 0.f ? t.x : 0.f;
-                            t.y = gate[i].y > 0.f ? t.y : 0.f;
-                            t.z = gate[i].z > 0.f ? t.z : 0.f;
-                            t.w = gate[i].w > 0.f ? t.w : 0.f;
-                        }
-                        if (a.accumulate) {
-                            // C += t at the L2: every element receives exactly one addition per launch, so the
-                            // result does not depend on the order, and the old value never travels to the SM
-                            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(Cf + row * a.ldc + col), "f"(t.x),
-                                         "f"(t.y), "f"(t.z), "f"(t.w)
-                                         : "memory");
-                        } else {
-                            *reinterpret_cast<float4*>(Cf + row * a.ldc + col) = t;
-                        }
+                    if (a.accumulate) {
+                        // C += t at the L2: every element receives exactly one addition per launch, so the
+                        // result does not depend on the order, and the old value never travels to the SM
+                        asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(Cf + row * a.ldc + col), "f"(t.x),
+                                     "f"(t.y), "f"(t.z), "f"(t.w)
+                                     : "memory");
+                    } else {
+                        *reinterpret_cast<float4*>(Cf + row * a.ldc + col) = t;
                     }
                 }
                 __syncwarp();
