@@ -1,13 +1,19 @@
 // Tensor-core (tcgen05) versions of the dense kernels of the layer: the grouped row-panel GEMM with
 // the fused epilogues of Eq. 6-7 and the grouped weight gradient.
 //
-// Operands are staged in shared memory in the canonical K-major, 128-byte-swizzled layout that
-// tcgen05.mma reads through a matrix descriptor; accumulators live in tensor memory (TMEM) and come
-// back through tcgen05.ld for the epilogue.  fp32 operands use the tf32 path three times
-// (hi*hi + lo*hi + hi*lo with hi = the top 19 bits of the value, lo = value - hi), which keeps
-// ~21 mantissa bits -- single-pass tf32 (10 bits) would miss the 1e-4 parity bound.  bf16 operands use
-// one kind::f16 pass.  The hi/lo split needs a pass through registers anyway, so tiles are written
-// to shared memory with ordinary stores (swizzled by hand) followed by a proxy fence.
+// fp32 operands use the tf32 path three times (hi*hi + lo*hi + hi*lo with hi = the value rounded to
+// 10 mantissa bits, lo = value - hi), which keeps ~21 mantissa bits -- single-pass tf32 would miss the
+// 1e-4 parity bound.  bf16 operands use one kind::f16 pass per weight part.  Accumulators live in
+// tensor memory (TMEM) and come back through tcgen05.ld for the epilogue.
+//
+// Two generations of kernels share the contracts in kernels.cuh:
+//   * tc_gemm_ts_kernel / tc_wgrad_ts_kernel (fp32): slabs arrive by tensor copy (TMA), the split
+//     activation operand is written to TMEM with tcgen05.st and the MMAs read it from there; only the
+//     small weight operand (a prepared image) or the B slab of the weight gradient is an operand tile
+//     in shared memory.
+//   * tc_gemm_ws_kernel / tc_gemm_kernel / tc_wgrad_ws_kernel / tc_wgrad_kernel: both operands staged in
+//     shared memory in the canonical swizzled layouts that a tcgen05 matrix descriptor reads, written
+//     with ordinary stores followed by a proxy fence (bf16 activations, masked or unaligned operands).
 // Every wait on an mbarrier is bounded; a wait that runs out sets the caller's status word.
 #include <cuda.h>
 
