@@ -72,6 +72,9 @@ struct GemmArgs {
 slicegcn_status_t gemm_run(const GemmArgs& a, cudaStream_t st);
 slicegcn_status_t tc_gemm_run(const GemmArgs& a, cudaStream_t st);
 int64_t tc_image_bytes(int groups, int K, int N);
+// true when the tensor-core kernel that takes this product applies a.a_mask in its producer at no extra pass
+// (otherwise multiplying the operand once up front is cheaper than the masked fallback kernels)
+bool tc_gemm_masks_in_producer(const GemmArgs& a);
 
 // ---- grouped weight gradient  dW_g = A_g^T * B_g  (reduction over all rows) -------------------
 // A_g: K columns of A from a_start[g]; B_g: N columns of the fp32 matrix B from b_start[g], each
@@ -99,6 +102,7 @@ struct WgradArgs {
 };
 int64_t wgrad_scratch_bytes(int64_t M, int groups, int K, int N);
 int64_t tc_wgrad_scratch_bytes(const WgradArgs& a);
+bool tc_wgrad_masks_in_producer(const WgradArgs& a);   // the same question for a.b_mask
 // bias_done (optional): set when the column sums (dbias / dbias2) were produced as well
 slicegcn_status_t tc_wgrad_run(const WgradArgs& a, void* scratch, int64_t scratch_bytes, cudaStream_t st, bool* bias_done = nullptr);
 slicegcn_status_t wgrad_run(const WgradArgs& a, void* scratch, int64_t scratch_bytes, cudaStream_t st);

@@ -329,37 +329,55 @@ slicegcn_status_t layer_backward_impl(const slicegcn_graph* g, const slicegcn_la
     }
 
     if (L.order == SLICEGCN_AGG_FIRST) {
-        // dM = dH * mask, materialised once: it feeds the weight gradient, the bias gradient and dZ
+        // dM = dH * mask feeds the weight gradient, the bias gradient and dZ.  Where the tensor-core kernels
+        // apply the byte mask in their producers (a mask tile travels next to every slab), dM is never
+        // written; otherwise it is materialised once.
         const int64_t dm_ld = align_up(L.out_cols, 8);
         float* dM = static_cast<float*>(b.take(L.n * dm_ld * 4));
-        SGCN_TRY(mask_mul_run(L.n, L.out_cols, dH_out, dout_ld, mask, L.mask_ld, dM, dm_ld, st));
-        if (dW_agg || db) {   // dW_agg = Z^T dM, db = colsum(dM)
-            WgradArgs w;
-            w.fault = g->fault;
-            w.M = L.n;
-            w.groups = L.p;
-            w.K = dW_agg ? L.in_width : 0;
-            w.N = L.h_s;
-            w.A = zt;
-            w.lda = L.zt_ld;
-            w.a_dtype = L.dtype;
-            w.a_pad_zero = L.zt_pad_zero ? 1 : 0;
+        WgradArgs w;      // dW_agg = Z^T dM, db = colsum(dM)
+        w.fault = g->fault;
+        w.M = L.n;
+        w.groups = L.p;
+        w.K = dW_agg ? L.in_width : 0;
+        w.N = L.h_s;
+        w.A = zt;
+        w.lda = L.zt_ld;
+        w.a_dtype = L.dtype;
+        w.a_pad_zero = L.zt_pad_zero ? 1 : 0;
+        w.dW = dW_agg;
+        w.dbias = db;
+        for (int i = 0; i < L.p; ++i) {
+            w.a_start[i] = L.in_starts[i];
+            w.b_start[i] = i * L.h_s;
+        }
+        GemmArgs dz = dself;   // dZ = dM W_agg^T
+        dz.B = d->W_agg;
+        const bool need_w = dW_agg || db;
+        WgradArgs wm = w;
+        wm.B = dH_out;
+        wm.ldb = dout_ld;
+        wm.b_mask = mask;
+        wm.b_mask_ld = L.mask_ld;
+        GemmArgs dzm = dz;
+        dzm.A = dH_out;
+        dzm.lda = dout_ld;
+        dzm.a_mask = mask;
+        dzm.a_mask_ld = L.mask_ld;
+        const bool in_producers = !seq && (!need_w || (dW_agg && tc_wgrad_masks_in_producer(wm))) &&
+                                  (!dH_in || tc_gemm_masks_in_producer(dzm));
+        if (in_producers) {
+            w = wm;
+            dz = dzm;
+        } else {
+            SGCN_TRY(mask_mul_run(L.n, L.out_cols, dH_out, dout_ld, mask, L.mask_ld, dM, dm_ld, st));
             w.B = dM;
             w.ldb = dm_ld;
-            w.dW = dW_agg;
-            w.dbias = db;
-            for (int i = 0; i < L.p; ++i) {
-                w.a_start[i] = L.in_starts[i];
-                w.b_start[i] = i * L.h_s;
-            }
-            SGCN_TRY(wgrad_run(w, wg, wg_bytes, st));
-        }
-        if (dH_in) {
-            float* dZ = static_cast<float*>(b.take(L.n * L.zt_ld * 4));
-            GemmArgs dz = dself;   // dZ = dM W_agg^T
             dz.A = dM;
             dz.lda = dm_ld;
-            dz.B = d->W_agg;
+        }
+        if (need_w) SGCN_TRY(wgrad_run(w, wg, wg_bytes, st));
+        if (dH_in) {
+            float* dZ = static_cast<float*>(b.take(L.n * L.zt_ld * 4));
             dz.C = dZ;
             dz.ldc = L.zt_ld;
             if (seq) {

@@ -993,10 +993,12 @@ constexpr int kTsRing = 6;     // raw slabs in flight or being read
 constexpr int kTsStages = 3;   // TMEM operand stages (with their weight images in shared memory)
 constexpr int kTsMaskPitch = 48;
 
+template <bool MASKED>   // MASKED: the activation operand is multiplied by the byte mask a.a_mask on its way to TMEM
 __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArgs a, const int n_pad, const int n_tiles, const int R,
                                                                    const unsigned char* image, const unsigned char* image2,
                                                                    int* fault, const __grid_constant__ CUtensorMap map_a,
-                                                                   const __grid_constant__ CUtensorMap map_a2) {
+                                                                   const __grid_constant__ CUtensorMap map_a2,
+                                                                   const __grid_constant__ CUtensorMap map_m) {
     extern __shared__ __align__(1024) unsigned char smem[];
     constexpr int S = kTsStages;
     const bool concat = n_pad <= 64;   // [B_hi | B_lo] as one operand; wider tiles take three chains per slab
@@ -1005,8 +1007,12 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
     const uint32_t slab_bytes = 2u * (uint32_t)n_pad * 128u;                  // weight image [hi | lo]
     const bool fused = a.A2 != nullptr;
     unsigned char* wring = base;                                              // [S] weight images
-    unsigned char* raw = wring + (uint32_t)S * slab_bytes;                    // [R] raw activation slabs, 128 rows x 128 B, swizzled
-    float* stage_out = reinterpret_cast<float*>(raw + R * 16384);             // [8 warps] 32 x kStagePitch floats
+    // [R] raw activation slabs, 128 rows x 128 B, swizzled; with an operand mask (a.a_mask) each is followed by
+    // its 128 x 32 mask bytes
+    constexpr bool masked = MASKED;
+    constexpr uint32_t raw_slot = MASKED ? 16384u + 4096u : 16384u;
+    unsigned char* raw = wring + (uint32_t)S * slab_bytes;
+    float* stage_out = reinterpret_cast<float*>(raw + R * raw_slot);          // [8 warps] 32 x kStagePitch floats
     unsigned char* stage_mask = reinterpret_cast<unsigned char*>(stage_out + 8 * 32 * kStagePitch);   // [8] 32 x kTsMaskPitch
     float* sbias = reinterpret_cast<float*>(stage_mask + 8 * 32 * kTsMaskPitch);
     float* spost = sbias + kWsVecFloats + 64;
@@ -1078,15 +1084,29 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
             }
             __syncwarp();
             tc_fence_after();
-            const unsigned char* slot = raw + rs * 16384 + roff;
+            const unsigned char* slot = raw + rs * raw_slot + roff;
             const uint32_t t_hi = tmem + ((uint32_t)(32 * warp) << 16) + a_col0 + (uint32_t)ts * 64u;
+            uint32_t mw[8];
+            if (masked) {   // the row's 32 mask bytes: word ch covers the four values of 16-byte chunk ch
+                const uint4* mrow = reinterpret_cast<const uint4*>(raw + rs * raw_slot + 16384 + (32 * warp + lane) * 32);
+                const uint4 m0 = mrow[0], m1 = mrow[1];
+                mw[0] = m0.x; mw[1] = m0.y; mw[2] = m0.z; mw[3] = m0.w;
+                mw[4] = m1.x; mw[5] = m1.y; mw[6] = m1.z; mw[7] = m1.w;
+            }
 #pragma unroll
             for (int half = 0; half < 2; ++half) {   // 16 K values at a time keeps the register count down
                 uint32_t h[32];                      // [0,16): hi of K 16 half..; [16,32): lo of the same
 #pragma unroll
                 for (int cc = 0; cc < 4; ++cc) {
                     const int ch = half * 4 + cc;
-                    const float4 v = *reinterpret_cast<const float4*>(slot + ((ch ^ (lane & 7)) << 4));
+                    float4 v = *reinterpret_cast<const float4*>(slot + ((ch ^ (lane & 7)) << 4));
+                    if (masked) {
+                        const uint32_t m = mw[ch];
+                        v.x = (m & 0xffu) ? v.x : 0.f;
+                        v.y = (m & 0xff00u) ? v.y : 0.f;
+                        v.z = (m & 0xff0000u) ? v.z : 0.f;
+                        v.w = (m & 0xff000000u) ? v.w : 0.f;
+                    }
                     const float h0 = tf32_hi(v.x), h1 = tf32_hi(v.y), h2 = tf32_hi(v.z), h3 = tf32_hi(v.w);
                     h[4 * cc + 0] = __float_as_uint(h0);
                     h[4 * cc + 1] = __float_as_uint(h1);
@@ -1134,8 +1154,10 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
                 const bool second = s >= ns1;
                 if (second) s -= ns1;
                 const int x = (second ? a.a2_start[l_it.g] : a.a_start[l_it.g]) + s * 32;
-                mbar_expect_tx(&rfull[rs], 16384u);
-                tma_load_2d(raw + rs * 16384, second ? &map_a2 : &map_a, x, (int)l_it.row0(), &rfull[rs]);
+                const bool with_mask = masked && !second;
+                mbar_expect_tx(&rfull[rs], with_mask ? 16384u + 4096u : 16384u);
+                tma_load_2d(raw + rs * raw_slot, second ? &map_a2 : &map_a, x, (int)l_it.row0(), &rfull[rs]);
+                if (with_mask) tma_load_2d(raw + rs * raw_slot + 16384, &map_m, x, (int)l_it.row0(), &rfull[rs]);
                 if (++l_s == n_slabs) {
                     l_s = 0;
                     l_it.next();
@@ -1362,14 +1384,14 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
     if (warp == 4) tmem_dealloc(tmem, 512);
 }
 
-// Tensor map over a row-major fp32 matrix for boxes of box_rows x box_cols values (default: one
+// Tensor map over a row-major fp32 (or, elem_bytes = 1, byte) matrix for boxes of box_rows x box_cols values (default: one
 // activation slab of 128 rows x 32 columns), written to shared memory with the 128-byte swizzle or plain.  `cols` bounds the columns a box may read
 // (beyond it: zeros).  The encoder is a driver entry point, looked up once; false if unavailable.
 typedef CUresult (*TensorMapEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                       const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                       CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 bool make_slab_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int64_t ld, int box_cols = 32, int box_rows = 128,
-                   bool swizzle128 = true) {
+                   bool swizzle128 = true, int elem_bytes = 4) {
     static TensorMapEncodeFn encode = [] {
         void* fn = nullptr;
         cudaDriverEntryPointQueryResult q = cudaDriverEntryPointSymbolNotFound;
@@ -1379,11 +1401,32 @@ bool make_slab_map(CUtensorMap* map, const void* base, int64_t rows, int64_t col
     }();
     if (!encode || rows < 1 || cols < 1) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)ld * sizeof(float)};
+    const cuuint64_t strides[1] = {(cuuint64_t)ld * (cuuint64_t)elem_bytes};
     const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
-    return encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+    return encode(map, elem_bytes == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                   swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// fp32 products that tc_gemm_ts_kernel takes (n_pad as chosen by tc_gemm_launch): 16-byte aligned
+// operands and result, up to 128 output columns per tile (32 with the fused second product), bias /
+// post vectors that fit the staging arrays; an operand mask only without a second product and with
+// 16-byte aligned mask rows and slice starts (it travels by tensor copy next to the slab).
+bool ts_gemm_ok(const GemmArgs& a, int n_pad, int n_tiles) {
+    static const bool off = getenv("SLICEGCN_NO_TS") != nullptr || getenv("SLICEGCN_NO_WS") != nullptr;
+    if (off || a.a_dtype != SLICEGCN_F32 || a.c_dtype != SLICEGCN_F32) return false;
+    const bool fused = a.A2 != nullptr;
+    bool ok = ((uintptr_t)a.A % 16 == 0) && (a.lda % 4 == 0) && (a.K % 4 == 0 || a.a_pad_zero);
+    for (int g = 0; g < a.groups; ++g) ok = ok && (a.a_start[g] % 4 == 0) && (a.c_start[g] % 4 == 0);
+    ok = ok && (a.N % 4 == 0) && (a.ldc % 4 == 0) && ((uintptr_t)a.C % 16 == 0);
+    if (a.mask_out) ok = ok && (a.mask_ld % 4 == 0) && ((uintptr_t)a.mask_out % 4 == 0);
+    if (a.mul_pos) ok = ok && (a.mul_pos_ld % 4 == 0) && ((uintptr_t)a.mul_pos % 16 == 0);
+    if (a.a_mask) {
+        ok = ok && !fused && ((uintptr_t)a.a_mask % 16 == 0) && (a.a_mask_ld % 16 == 0);
+        for (int g = 0; g < a.groups; ++g) ok = ok && (a.a_start[g] % 16 == 0);
+    }
+    const int64_t items = ((a.M + 127) / 128) * a.groups * n_tiles;
+    return ok && n_pad <= (fused ? 32 : 128) && a.groups * a.N <= kWsVecFloats && items < ((int64_t)1 << 31) && a.M < ((int64_t)1 << 31);
 }
 
 int tc_n_pad(int N) { return N <= 256 ? ((N + 15) & ~15) : 256; }
@@ -1463,32 +1506,40 @@ slicegcn_status_t tc_gemm_launch(const GemmArgs& a, void* image, int64_t image_b
     const int64_t all_items = ((a.M + 127) / 128) * a.groups * n_tiles;
     if constexpr (!BF16 && std::is_same<TA, float>::value && std::is_same<TC, float>::value) {
         // narrow fp32 outputs (the sliced layers): the kernel that keeps the activation operand in TMEM
-        static const bool no_ts = getenv("SLICEGCN_NO_TS") != nullptr;
-        if (vec && cvec && !a.a_mask && !no_ws && !no_ts && n_pad <= (fused ? 32 : 128) && a.groups * a.N <= kWsVecFloats &&
-            all_items < ((int64_t)1 << 31) && a.M < ((int64_t)1 << 31)) {
+        if (ts_gemm_ok(a, n_pad, n_tiles)) {
             // columns the slabs may touch: up to the end of the last group (the rest reads as zeros)
             int cols1 = 0, cols2 = 0;
             for (int g = 0; g < a.groups; ++g) {
                 cols1 = std::max(cols1, a.a_start[g] + a.K);
                 if (fused) cols2 = std::max(cols2, a.a2_start[g] + a.K2);
             }
-            CUtensorMap map_a, map_a2;
+            CUtensorMap map_a, map_a2, map_m;
             bool maps_ok = make_slab_map(&map_a, a.A, a.M, std::min<int64_t>(cols1, a.lda), a.lda);
             if (maps_ok && fused) maps_ok = make_slab_map(&map_a2, a.A2, a.M, std::min<int64_t>(cols2, a.lda2), a.lda2);
             if (maps_ok && !fused) map_a2 = map_a;
+            if (maps_ok && a.a_mask)
+                maps_ok = make_slab_map(&map_m, a.a_mask, a.M, std::min<int64_t>(cols1, a.a_mask_ld), a.a_mask_ld, 32, 128, false, 1);
+            if (maps_ok && !a.a_mask) map_m = map_a;
             if (maps_ok) {
-            const int ring = n_pad > 64 ? 4 : kTsRing;   // the wider weight images leave room for fewer raw slabs
-            const int ts_smem = kTsStages * 2 * n_pad * 128 + 4 * ring * 4096 + 8 * 32 * kStagePitch * 4 + 8 * 32 * kTsMaskPitch +
-                                2 * (kWsVecFloats + 64) * 4 + 256 + 1024;
+            // as many raw slabs as fit next to the weight images and the staging tiles (wider images leave fewer)
+            const int raw_slot = a.a_mask ? 20480 : 16384;
+            const int ts_fixed = kTsStages * 2 * n_pad * 128 + 8 * 32 * kStagePitch * 4 + 8 * 32 * kTsMaskPitch + 2 * (kWsVecFloats + 64) * 4 + 256 + 1024;
+            const int ring = std::min(kTsRing, (225 * 1024 - ts_fixed) / raw_slot);
+            const int ts_smem = ts_fixed + ring * raw_slot;
             static bool ts_configured = false;
             if (!ts_configured) {
-                SGCN_CUDA(cudaFuncSetAttribute(tc_gemm_ts_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
+                SGCN_CUDA(cudaFuncSetAttribute(tc_gemm_ts_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
+                SGCN_CUDA(cudaFuncSetAttribute(tc_gemm_ts_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
                 ts_configured = true;
             }
             int64_t tgrid = 148;
             if (tgrid > all_items) tgrid = all_items;
-            tc_gemm_ts_kernel<<<(unsigned)tgrid, kTsThreads, ts_smem, st>>>(a, n_pad, n_tiles, ring, static_cast<unsigned char*>(image), image2, fault,
-                                                                            map_a, map_a2);
+            if (a.a_mask)
+                tc_gemm_ts_kernel<true><<<(unsigned)tgrid, kTsThreads, ts_smem, st>>>(a, n_pad, n_tiles, ring, static_cast<unsigned char*>(image), image2,
+                                                                                      fault, map_a, map_a2, map_m);
+            else
+                tc_gemm_ts_kernel<false><<<(unsigned)tgrid, kTsThreads, ts_smem, st>>>(a, n_pad, n_tiles, ring, static_cast<unsigned char*>(image), image2,
+                                                                                       fault, map_a, map_a2, map_m);
             SGCN_LAUNCH_CHECK();
             count_launch(fused ? 3 : 2);
             return SLICEGCN_OK;
@@ -1944,7 +1995,8 @@ constexpr int kWtThreads = 192;
 template <bool WIDE>
 __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradArgs a, const WgTcPlan pl, float* scratch, float* colsum,
                                                                     int* fault, const __grid_constant__ CUtensorMap map_a,
-                                                                    const __grid_constant__ CUtensorMap map_b) {
+                                                                    const __grid_constant__ CUtensorMap map_b,
+                                                                    const __grid_constant__ CUtensorMap map_bm) {
     extern __shared__ __align__(1024) unsigned char smem[];
     constexpr int R = WIDE ? 2 : 4, S = 2;   // raw slots; operand stages (TMEM A + shared-memory B)
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -1952,7 +2004,10 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
     unsigned char* base = smem + ((1024u - (smem_u32(smem) & 1023u)) & 1023u);
     const int nbk = (pl.n_t + 31) / 32;                      // column blocks of the B tile
     const uint32_t b_raw_bytes = 32u * (uint32_t)pl.n_t * 4u;
-    const uint32_t slot_bytes = 16384u + ((b_raw_bytes + 1023u) & ~1023u);   // raw A | raw B
+    const bool masked = a.b_mask != nullptr;                 // B is multiplied by a byte mask on the way
+    const uint32_t b_raw_pad = (b_raw_bytes + 1023u) & ~1023u;
+    const uint32_t m_raw_bytes = 32u * (uint32_t)pl.n_t;
+    const uint32_t slot_bytes = 16384u + b_raw_pad + (masked ? ((m_raw_bytes + 1023u) & ~1023u) : 0u);   // raw A | raw B | mask
     const uint32_t op_bytes = (uint32_t)nbk * 8192u;         // B operand stage: 8 K atoms x (nbk hi + nbk lo) x 512 B
     unsigned char* ops = base;                               // [S]
     unsigned char* raw = ops + S * op_bytes;                 // [R]
@@ -2022,11 +2077,19 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
             // ---- B: split into the operand tile
             if (b_mine) {
                 const unsigned char* braw = slot + 16384 + b_cc * 16;
+                const unsigned char* mraw = slot + 16384 + b_raw_pad + b_cc * 4;
                 unsigned char* op = ops + ts * op_bytes;
 #pragma unroll
                 for (int i = 0; i < BI; ++i) {
                     const int r = b_r0 + BSTEP * i;
-                    const float4 v = *reinterpret_cast<const float4*>(braw + r * (pl.n_t * 4));
+                    float4 v = *reinterpret_cast<const float4*>(braw + r * (pl.n_t * 4));
+                    if (masked) {
+                        const uint32_t m = *reinterpret_cast<const uint32_t*>(mraw + r * pl.n_t);
+                        v.x = (m & 0xffu) ? v.x : 0.f;
+                        v.y = (m & 0xff00u) ? v.y : 0.f;
+                        v.z = (m & 0xff0000u) ? v.z : 0.f;
+                        v.w = (m & 0xff000000u) ? v.w : 0.f;
+                    }
                     const float h0 = tf32_hi(v.x), h1 = tf32_hi(v.y), h2 = tf32_hi(v.z), h3 = tf32_hi(v.w);
                     const uint32_t off = (uint32_t)((((r >> 2) * 2 * nbk + (b_cc >> 3)) << 9) + ((r & 3) << 7) +
                                                     (((((b_cc & 7) >> 1) ^ (r & 3))) << 5) + ((b_cc & 1) << 4));
@@ -2135,9 +2198,10 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
                 }
                 unsigned char* slot = raw + rs * slot_bytes;
                 const int y = (int)(r_begin + (int64_t)j * 32);
-                mbar_expect_tx(&rfull[rs], 16384u + b_raw_bytes);
+                mbar_expect_tx(&rfull[rs], 16384u + b_raw_bytes + (masked ? m_raw_bytes : 0u));
                 tma_load_2d(slot, &map_a, ax, y, &rfull[rs]);
                 tma_load_2d(slot + 16384, &map_b, bx, y, &rfull[rs]);
+                if (masked) tma_load_2d(slot + 16384 + b_raw_pad, &map_bm, bx, y, &rfull[rs]);
                 if (++rs == R) {
                     rs = 0;
                     ++rpass;
@@ -2276,7 +2340,35 @@ bool wgrad_tc_plan(const WgradArgs& a, WgTcPlan* pl, int* groups_per_tile, int f
     return true;
 }
 
+// Weight gradients that tc_wgrad_ts_kernel takes under plan pl (fp32, one CTA per SM): B tiles of up to
+// 256 columns; a mask on B only for tiles of up to 128 columns (shared memory) with 16-byte aligned
+// mask rows and tile starts.
+bool wgrad_ts_ok(const WgradArgs& a, const WgTcPlan& pl) {
+    const int nbk = (pl.n_t + 31) / 32;
+    if (a.a_dtype != SLICEGCN_F32 || nbk > 8 || a.M >= ((int64_t)1 << 31)) return false;
+    if (a.b_mask) {
+        if (nbk > 4 || (uintptr_t)a.b_mask % 16 || a.b_mask_ld % 16 || pl.b_col0 % 16 || pl.b_cols_per_tile % 16) return false;
+    }
+    return true;
+}
+
 }  // namespace
+
+bool tc_wgrad_masks_in_producer(const WgradArgs& a) {
+    static const bool off = getenv("SLICEGCN_NO_TS") != nullptr || getenv("SLICEGCN_NO_WS") != nullptr;
+    WgTcPlan pl;
+    int gpt = 0;
+    if (off || !a.b_mask || !a.fault || !wgrad_tc_plan(a, &pl, &gpt, 1)) return false;
+    return wgrad_ts_ok(a, pl);
+}
+
+bool tc_gemm_masks_in_producer(const GemmArgs& a) {
+    if (!a.a_mask || !a.fault || !a.b_image || a.K < 1 || a.A2) return false;
+    int n_pad = tc_n_pad(a.N);
+    if (a.N == 256 && a.groups * a.N <= kWsVecFloats) n_pad = 128;
+    const int n_tiles = (a.N + n_pad - 1) / n_pad;
+    return ts_gemm_ok(a, n_pad, n_tiles) && a.b_image_bytes >= tc_image_bytes(a.groups, a.K, a.N);
+}
 
 int64_t tc_image_bytes(int groups, int K, int N) {
     const int n_pad = tc_n_pad(N);
@@ -2300,8 +2392,8 @@ slicegcn_status_t tc_wgrad_run(const WgradArgs& a, void* scratch, int64_t scratc
     if (bias_done) *bias_done = false;
     if (!a.fault || !wgrad_tc_plan(a, &pl, &gpt)) return SLICEGCN_ERR_UNSUPPORTED;
     static const bool no_ws = getenv("SLICEGCN_NO_WS") != nullptr;
-    if (!no_ws && a.a_dtype == SLICEGCN_F32 && !a.b_mask) {
-        // warp-specialised variant: one CTA per SM
+    if (!no_ws && a.a_dtype == SLICEGCN_F32) {
+        // warp-specialised variants: one CTA per SM
         WgTcPlan pw;
         int gw = 0;
         if (wgrad_tc_plan(a, &pw, &gw, 1)) {
@@ -2309,17 +2401,22 @@ slicegcn_status_t tc_wgrad_run(const WgradArgs& a, void* scratch, int64_t scratc
             static const bool no_ts = getenv("SLICEGCN_NO_TS") != nullptr;
             const int64_t need_ts = (int64_t)pw.n_chunks * pw.m_tiles * 128 * pw.n_t * (int64_t)sizeof(float);
             const int64_t need_cs = (int64_t)pw.n_chunks * pw.m_tiles * pw.n_t * (int64_t)sizeof(float);
-            if (!no_ts && nbk <= 8 && scratch && scratch_bytes >= need_ts && a.M < ((int64_t)1 << 31)) {
+            if (!no_ts && wgrad_ts_ok(a, pw) && scratch && scratch_bytes >= need_ts) {
                 // the kernel that keeps A^T in TMEM (and sums B's columns on the way)
                 const bool wide = nbk > 4;
                 const int b_total = a.groups * a.N;
                 CUtensorMap map_a, map_b;
+                CUtensorMap map_bm;
                 bool maps_ok = make_slab_map(&map_a, a.A, a.M, std::min<int64_t>(pw.a_col0 + pw.a_cols, a.lda), a.lda, 128, 32, false) &&
                                make_slab_map(&map_b, a.B, a.M, std::min<int64_t>(pw.b_col0 + b_total, a.ldb), a.ldb, pw.n_t, 32, false);
+                if (maps_ok && a.b_mask)
+                    maps_ok = make_slab_map(&map_bm, a.b_mask, a.M, std::min<int64_t>(pw.b_col0 + b_total, a.b_mask_ld), a.b_mask_ld, pw.n_t, 32,
+                                            false, 1);
+                if (maps_ok && !a.b_mask) map_bm = map_b;
                 if (maps_ok) {
                     const bool want_bias = (a.dbias || a.dbias2) && scratch_bytes >= need_ts + need_cs;
                     float* colsum = want_bias ? static_cast<float*>(scratch) + need_ts / sizeof(float) : nullptr;
-                    const int slot_b = 16384 + ((32 * pw.n_t * 4 + 1023) & ~1023);
+                    const int slot_b = 16384 + ((32 * pw.n_t * 4 + 1023) & ~1023) + (a.b_mask ? ((32 * pw.n_t + 1023) & ~1023) : 0);
                     const int ts_smem = 2 * nbk * 8192 + (wide ? 2 : 4) * slot_b + 256 + 1024;
                     static bool ts_configured = false;
                     if (!ts_configured) {
@@ -2329,9 +2426,9 @@ slicegcn_status_t tc_wgrad_run(const WgradArgs& a, void* scratch, int64_t scratc
                     }
                     dim3 tgrid(pw.n_chunks, pw.m_tiles);
                     if (wide)
-                        tc_wgrad_ts_kernel<true><<<tgrid, kWtThreads, ts_smem, st>>>(a, pw, static_cast<float*>(scratch), colsum, a.fault, map_a, map_b);
+                        tc_wgrad_ts_kernel<true><<<tgrid, kWtThreads, ts_smem, st>>>(a, pw, static_cast<float*>(scratch), colsum, a.fault, map_a, map_b, map_bm);
                     else
-                        tc_wgrad_ts_kernel<false><<<tgrid, kWtThreads, ts_smem, st>>>(a, pw, static_cast<float*>(scratch), colsum, a.fault, map_a, map_b);
+                        tc_wgrad_ts_kernel<false><<<tgrid, kWtThreads, ts_smem, st>>>(a, pw, static_cast<float*>(scratch), colsum, a.fault, map_a, map_b, map_bm);
                     SGCN_LAUNCH_CHECK();
                     const int64_t total_w = (int64_t)a.groups * a.K * a.N;
                     tc_wgrad_reduce_kernel<<<(unsigned)((total_w + 31) / 32), 256, 0, st>>>(static_cast<const float*>(scratch), pw,
@@ -2349,6 +2446,7 @@ slicegcn_status_t tc_wgrad_run(const WgradArgs& a, void* scratch, int64_t scratc
             const int stage_b = 32768 + 2 * 4 * nbk * 1024;
             int D = (220 * 1024) / stage_b;
             if (D > 3) D = 3;
+            if (a.b_mask) D = 0;   // the shared-memory-operand variant takes no mask
             const int64_t need_w = (int64_t)pw.n_chunks * pw.m_tiles * 128 * pw.n_t * (int64_t)sizeof(float);
             if (D >= 2 && scratch && scratch_bytes >= need_w) {
                 const int ws_smem = D * stage_b + 256 + 1024;
