@@ -1606,6 +1606,8 @@ struct WgTcPlan {
     int a_col0, b_col0; // first column of A / B
     int a_cols;         // total A columns (all groups)
     int b_cols_per_tile;
+    int a_tile_cols;    // A columns between consecutive tiles (128 unless the narrow grouped plan is used)
+    int a_box;          // A columns fetched per tile (multiple of 32, <= 128)
     int n_chunks;
     int64_t rows_per_chunk;
     int stages;
@@ -2059,14 +2061,15 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
             tc_fence_after();
             const unsigned char* slot = raw + rs * slot_bytes;
             // ---- A: column 32 warp + lane, 32 values down the rows
-            const float* acol = reinterpret_cast<const float*>(slot) + 32 * warp + lane;
+            const bool a_live = 32 * warp + lane < pl.a_box;   // columns past the fetched width stay zero
+            const float* acol = reinterpret_cast<const float*>(slot) + (a_live ? 32 * warp + lane : 0);
             const uint32_t t_hi = tmem + ((uint32_t)(32 * warp) << 16) + accw + (uint32_t)ts * 64u;
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
                 uint32_t h[32];   // [0,16): hi of rows 16 half ..; [16,32): lo of the same
 #pragma unroll
                 for (int k = 0; k < 16; ++k) {
-                    const float v = acol[(16 * half + k) * 128];
+                    const float v = a_live ? acol[(16 * half + k) * pl.a_box] : 0.f;
                     const float hv = tf32_hi(v);
                     h[k] = __float_as_uint(hv);
                     h[16 + k] = __float_as_uint(v - hv);
@@ -2190,7 +2193,7 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
         if (lane == 0) {
             int rs = 0;
             uint32_t rpass = 0;
-            const int ax = pl.a_col0 + mt * 128, bx = pl.b_col0 + mt * pl.b_cols_per_tile;
+            const int ax = pl.a_col0 + mt * pl.a_tile_cols, bx = pl.b_col0 + mt * pl.b_cols_per_tile;
             for (int j = 0; j < n_slabs; ++j) {
                 if (rpass >= 1 && !mbar_wait(&rfree[rs], (rpass - 1) & 1)) {
                     atomicExch(fault, 11);
@@ -2198,7 +2201,7 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
                 }
                 unsigned char* slot = raw + rs * slot_bytes;
                 const int y = (int)(r_begin + (int64_t)j * 32);
-                mbar_expect_tx(&rfull[rs], 16384u + b_raw_bytes + (masked ? m_raw_bytes : 0u));
+                mbar_expect_tx(&rfull[rs], 128u * (uint32_t)pl.a_box + b_raw_bytes + (masked ? m_raw_bytes : 0u));
                 tma_load_2d(slot, &map_a, ax, y, &rfull[rs]);
                 tma_load_2d(slot + 16384, &map_b, bx, y, &rfull[rs]);
                 if (masked) tma_load_2d(slot + 16384 + b_raw_pad, &map_bm, bx, y, &rfull[rs]);
@@ -2284,7 +2287,10 @@ __global__ void __launch_bounds__(256) tc_wgrad_reduce_kernel(const float* scrat
     }
 }
 
-bool wgrad_tc_plan(const WgradArgs& a, WgTcPlan* pl, int* groups_per_tile, int force_per_sm = 0) {
+// narrow: grouped layers take fewer groups per tile so that a tile's B columns stay within 128 (the TMEM-operand
+// kernel then runs its two-chain form with two operand stages, and may apply a mask); tiles of fewer than 128 A columns
+// follow each other at a_tile_cols.
+bool wgrad_tc_plan(const WgradArgs& a, WgTcPlan* pl, int* groups_per_tile, int force_per_sm = 0, bool narrow = false) {
     if (a.K < 1 || !a.dW) return false;
     bool shared_a = a.groups > 1;   // every group reads the same A columns (fused input feeding all slices)
     for (int g = 0; g < a.groups; ++g) shared_a = shared_a && (a.a_start[g] == a.a_start[0]);
@@ -2300,6 +2306,7 @@ bool wgrad_tc_plan(const WgradArgs& a, WgTcPlan* pl, int* groups_per_tile, int f
     if (a.N % 4 && !(a.b_pad_zero && a.groups == 1)) return false;
     if (a.b_mask && ((uintptr_t)a.b_mask % 4 || a.b_mask_ld % 4)) return false;
     WgTcPlan P{};
+    P.a_tile_cols = 128;
     P.a_col0 = a.a_start[0];
     P.b_col0 = a.b_start[0];
     P.a_cols = shared_a ? a.K : a.groups * a.K;
@@ -2314,7 +2321,10 @@ bool wgrad_tc_plan(const WgradArgs& a, WgTcPlan* pl, int* groups_per_tile, int f
         int gpt = 128 / a.K;
         if (gpt > a.groups) gpt = a.groups;
         if (a.groups % gpt != 0) return false;
+        if (narrow)
+            while (gpt * a.N > 128 && gpt % 2 == 0) gpt /= 2;
         if (gpt * a.N > 256) return false;
+        P.a_tile_cols = gpt * a.K;
         P.m_tiles = a.groups / gpt;
         P.n_valid = gpt * a.N;
         P.b_cols_per_tile = gpt * a.N;
@@ -2327,6 +2337,7 @@ bool wgrad_tc_plan(const WgradArgs& a, WgTcPlan* pl, int* groups_per_tile, int f
         *groups_per_tile = 0;
     }
     P.n_t = (P.n_valid + 15) & ~15;
+    P.a_box = std::min(128, (P.a_tile_cols + 31) & ~31);
     // single-stage CTAs are small enough for two or three per SM, which overlap each other
     P.stages = 1;
     const int per_sm = force_per_sm > 0 ? force_per_sm : (P.n_t <= 128 ? 3 : 2);
@@ -2358,7 +2369,7 @@ bool tc_wgrad_masks_in_producer(const WgradArgs& a) {
     static const bool off = getenv("SLICEGCN_NO_TS") != nullptr || getenv("SLICEGCN_NO_WS") != nullptr;
     WgTcPlan pl;
     int gpt = 0;
-    if (off || !a.b_mask || !a.fault || !wgrad_tc_plan(a, &pl, &gpt, 1)) return false;
+    if (off || !a.b_mask || !a.fault || !wgrad_tc_plan(a, &pl, &gpt, 1, true)) return false;
     return wgrad_ts_ok(a, pl);
 }
 
@@ -2396,27 +2407,30 @@ slicegcn_status_t tc_wgrad_run(const WgradArgs& a, void* scratch, int64_t scratc
         // warp-specialised variants: one CTA per SM
         WgTcPlan pw;
         int gw = 0;
-        if (wgrad_tc_plan(a, &pw, &gw, 1)) {
-            const int nbk = (pw.n_t + 31) / 32;
+        {   // first choice: the TMEM-operand kernel under the narrow plan
+            WgTcPlan pn;
+            int gn = 0;
+            if (wgrad_tc_plan(a, &pn, &gn, 1, true)) {
+            const int nbk = (pn.n_t + 31) / 32;
             static const bool no_ts = getenv("SLICEGCN_NO_TS") != nullptr;
-            const int64_t need_ts = (int64_t)pw.n_chunks * pw.m_tiles * 128 * pw.n_t * (int64_t)sizeof(float);
-            const int64_t need_cs = (int64_t)pw.n_chunks * pw.m_tiles * pw.n_t * (int64_t)sizeof(float);
-            if (!no_ts && wgrad_ts_ok(a, pw) && scratch && scratch_bytes >= need_ts) {
+            const int64_t need_ts = (int64_t)pn.n_chunks * pn.m_tiles * 128 * pn.n_t * (int64_t)sizeof(float);
+            const int64_t need_cs = (int64_t)pn.n_chunks * pn.m_tiles * pn.n_t * (int64_t)sizeof(float);
+            if (!no_ts && wgrad_ts_ok(a, pn) && scratch && scratch_bytes >= need_ts) {
                 // the kernel that keeps A^T in TMEM (and sums B's columns on the way)
                 const bool wide = nbk > 4;
                 const int b_total = a.groups * a.N;
                 CUtensorMap map_a, map_b;
                 CUtensorMap map_bm;
-                bool maps_ok = make_slab_map(&map_a, a.A, a.M, std::min<int64_t>(pw.a_col0 + pw.a_cols, a.lda), a.lda, 128, 32, false) &&
-                               make_slab_map(&map_b, a.B, a.M, std::min<int64_t>(pw.b_col0 + b_total, a.ldb), a.ldb, pw.n_t, 32, false);
+                bool maps_ok = make_slab_map(&map_a, a.A, a.M, std::min<int64_t>(pn.a_col0 + pn.a_cols, a.lda), a.lda, pn.a_box, 32, false) &&
+                               make_slab_map(&map_b, a.B, a.M, std::min<int64_t>(pn.b_col0 + b_total, a.ldb), a.ldb, pn.n_t, 32, false);
                 if (maps_ok && a.b_mask)
-                    maps_ok = make_slab_map(&map_bm, a.b_mask, a.M, std::min<int64_t>(pw.b_col0 + b_total, a.b_mask_ld), a.b_mask_ld, pw.n_t, 32,
+                    maps_ok = make_slab_map(&map_bm, a.b_mask, a.M, std::min<int64_t>(pn.b_col0 + b_total, a.b_mask_ld), a.b_mask_ld, pn.n_t, 32,
                                             false, 1);
                 if (maps_ok && !a.b_mask) map_bm = map_b;
                 if (maps_ok) {
                     const bool want_bias = (a.dbias || a.dbias2) && scratch_bytes >= need_ts + need_cs;
                     float* colsum = want_bias ? static_cast<float*>(scratch) + need_ts / sizeof(float) : nullptr;
-                    const int slot_b = 16384 + ((32 * pw.n_t * 4 + 1023) & ~1023) + (a.b_mask ? ((32 * pw.n_t + 1023) & ~1023) : 0);
+                    const int slot_b = 16384 + ((32 * pn.n_t * 4 + 1023) & ~1023) + (a.b_mask ? ((32 * pn.n_t + 1023) & ~1023) : 0);
                     const int ts_smem = 2 * nbk * 8192 + (wide ? 2 : 4) * slot_b + 256 + 1024;
                     static bool ts_configured = false;
                     if (!ts_configured) {
@@ -2424,18 +2438,18 @@ slicegcn_status_t tc_wgrad_run(const WgradArgs& a, void* scratch, int64_t scratc
                         SGCN_CUDA(cudaFuncSetAttribute(tc_wgrad_ts_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
                         ts_configured = true;
                     }
-                    dim3 tgrid(pw.n_chunks, pw.m_tiles);
+                    dim3 tgrid(pn.n_chunks, pn.m_tiles);
                     if (wide)
-                        tc_wgrad_ts_kernel<true><<<tgrid, kWtThreads, ts_smem, st>>>(a, pw, static_cast<float*>(scratch), colsum, a.fault, map_a, map_b, map_bm);
+                        tc_wgrad_ts_kernel<true><<<tgrid, kWtThreads, ts_smem, st>>>(a, pn, static_cast<float*>(scratch), colsum, a.fault, map_a, map_b, map_bm);
                     else
-                        tc_wgrad_ts_kernel<false><<<tgrid, kWtThreads, ts_smem, st>>>(a, pw, static_cast<float*>(scratch), colsum, a.fault, map_a, map_b, map_bm);
+                        tc_wgrad_ts_kernel<false><<<tgrid, kWtThreads, ts_smem, st>>>(a, pn, static_cast<float*>(scratch), colsum, a.fault, map_a, map_b, map_bm);
                     SGCN_LAUNCH_CHECK();
                     const int64_t total_w = (int64_t)a.groups * a.K * a.N;
-                    tc_wgrad_reduce_kernel<<<(unsigned)((total_w + 31) / 32), 256, 0, st>>>(static_cast<const float*>(scratch), pw,
-                                                                                             a.groups, a.K, a.N, gw, a.dW);
+                    tc_wgrad_reduce_kernel<<<(unsigned)((total_w + 31) / 32), 256, 0, st>>>(static_cast<const float*>(scratch), pn,
+                                                                                             a.groups, a.K, a.N, gn, a.dW);
                     SGCN_LAUNCH_CHECK();
                     if (want_bias) {
-                        tc_wgrad_bias_reduce_kernel<<<(b_total + 127) / 128, 128, 0, st>>>(colsum, pw, a.groups, a.N, gw, a.dbias, a.dbias2);
+                        tc_wgrad_bias_reduce_kernel<<<(b_total + 127) / 128, 128, 0, st>>>(colsum, pn, a.groups, a.N, gn, a.dbias, a.dbias2);
                         SGCN_LAUNCH_CHECK();
                         if (bias_done) *bias_done = true;
                     }
@@ -2443,6 +2457,10 @@ slicegcn_status_t tc_wgrad_run(const WgradArgs& a, void* scratch, int64_t scratc
                     return SLICEGCN_OK;
                 }
             }
+            }
+        }
+        if (wgrad_tc_plan(a, &pw, &gw, 1)) {
+            const int nbk = (pw.n_t + 31) / 32;
             const int stage_b = 32768 + 2 * 4 * nbk * 1024;
             int D = (220 * 1024) / stage_b;
             if (D > 3) D = 3;
