@@ -1981,16 +1981,17 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_wgrad_ws_kernel(const WgradA
 //   warp 5     loader: per slab of 32 rows one tensor copy of the A tile (32 x 128 values) and one of
 //              the B tile (32 x n_t), unswizzled, into a ring of raw slots; rows past the end
 //              of the matrix and columns past its width arrive as zeros.
-//   warps 0-3  producers: lane m of warp w reads column 32w + m of the raw A slab (32 values down the
+//   warps 0-3  A producers: lane m of warp w reads column 32w + m of the raw A slab (32 values down the
 //              rows -- consecutive lanes, consecutive words), splits them and writes hi and lo into a
-//              TMEM stage with tcgen05.st: A^T in the K-major form, M index = TMEM lane.  The B slab is
-//              split into the MN-major operand tile ("128-byte swizzle, 32-byte base"; per K atom the
-//              hi column blocks are followed by the lo column blocks, so [hi | lo] is one operand of
-//              2 n_t columns).  The producers also keep the column sums of B (the bias gradient) and,
-//              after the last slab, drain the accumulator into the scratch tile.
+//              TMEM stage with tcgen05.st: A^T in the K-major form, M index = TMEM lane.  After the last
+//              slab they drain the accumulator into the scratch tile.
+//   warps 8-11 B producers: split the B slab (times its byte mask, if any) into the MN-major operand
+//              tile ("128-byte swizzle, 32-byte base"; per K atom the hi column blocks are followed by
+//              the lo column blocks, so [hi | lo] is one operand of 2 n_t columns) and keep the column
+//              sums of B (the bias gradient).
 //   warp 4     MMA issuer: per 8 rows A_hi x [B_hi | B_lo] and A_lo x B_hi.
 // TMEM columns: accumulator [hi*hi + lo*hi | hi*lo] (64 nbk), then two stages of 64 (A hi | A lo).
-constexpr int kWtThreads = 192;
+constexpr int kWtThreads = 384;
 
 // WIDE: B tiles of 129..256 columns -- no room for [hi | lo] in one operand (three chains per slab) and
 // only two raw slots.
@@ -2013,7 +2014,7 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
     const uint32_t op_bytes = (uint32_t)nbk * 8192u;         // B operand stage: 8 K atoms x (nbk hi + nbk lo) x 512 B
     unsigned char* ops = base;                               // [S]
     unsigned char* raw = ops + S * op_bytes;                 // [R]
-    float* csum_s = reinterpret_cast<float*>(raw);           // [4][128] column-sum partials: reuse raw slot 0 after the last slab
+    float* csum_s = reinterpret_cast<float*>(raw + 16384);   // [4][128] column-sum partials: reuse the B part of raw slot 0 after the last slab
     uint64_t* afull = reinterpret_cast<uint64_t*>(raw + R * slot_bytes);   // [S] 128 producer arrivals
     uint64_t* afree = afull + S;                             // [S] MMAs of the stage completed
     uint64_t* rfull = afree + S;                             // [R] raw slab landed
@@ -2023,12 +2024,12 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
     const uint32_t accw = (WIDE ? 32u : 64u) * (uint32_t)nbk;   // accumulator columns
     if (tid == 0) {
         for (int i = 0; i < S; ++i) {
-            mbar_init(&afull[i], 128);
+            mbar_init(&afull[i], 256);
             mbar_init(&afree[i], 1);
         }
         for (int i = 0; i < R; ++i) {
             mbar_init(&rfull[i], 1);
-            mbar_init(&rfree[i], 4);
+            mbar_init(&rfree[i], 8);
         }
         mbar_init(tfull, 1);
     }
@@ -2044,13 +2045,7 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
     const int n_slabs = r_end > r_begin ? (int)((r_end - r_begin + 31) / 32) : 0;
 
     if (warp < 4) {
-        // ------------------------------------------------------------ producers (and, at the end, epilogue)
-        // B: 16-byte column chunk b_cc of rows b_r0 + BSTEP i
-        const int b_cc = WIDE ? (tid & 63) : (tid & 31), b_r0 = WIDE ? (tid >> 6) : (tid >> 5);
-        constexpr int BI = WIDE ? 16 : 8, BSTEP = WIDE ? 2 : 4;
-        const int nq = pl.n_t / 4;
-        const bool b_mine = b_cc < nq;
-        float4 csum = make_float4(0.f, 0.f, 0.f, 0.f);
+        // ------------------------------------------------------------ A producers (and, at the end, epilogue)
         int rs = 0, ts = 0;
         uint32_t pass = 0, rpass = 0;
         bool okp = true;
@@ -2060,7 +2055,7 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
             if (!okp) break;
             tc_fence_after();
             const unsigned char* slot = raw + rs * slot_bytes;
-            // ---- A: column 32 warp + lane, 32 values down the rows
+            // column 32 warp + lane of the slab, 32 values down the rows
             const bool a_live = 32 * warp + lane < pl.a_box;   // columns past the fetched width stay zero
             const float* acol = reinterpret_cast<const float*>(slot) + (a_live ? 32 * warp + lane : 0);
             const uint32_t t_hi = tmem + ((uint32_t)(32 * warp) << 16) + accw + (uint32_t)ts * 64u;
@@ -2074,10 +2069,66 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
                     h[k] = __float_as_uint(hv);
                     h[16 + k] = __float_as_uint(v - hv);
                 }
+                if (half == 1) {   // the slab is in registers: this warp is done with the raw slot
+                    __syncwarp();
+                    if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&rfree[rs])) : "memory");
+                    __syncwarp();
+                }
                 tmem_st16<0>(t_hi + 16u * half, h);
                 tmem_st16<16>(t_hi + 32u + 16u * half, h);
             }
-            // ---- B: split into the operand tile
+            tmem_st_wait();
+            tc_fence_before();
+            asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&afull[ts])) : "memory");
+            if (++rs == R) {
+                rs = 0;
+                ++rpass;
+            }
+            if (++ts == S) {
+                ts = 0;
+                ++pass;
+            }
+        }
+        if (!okp && lane == 0) atomicExch(fault, 8);
+        // epilogue: partial tile -> scratch (row = A column 32 warp + lane of the tile)
+        float* out = scratch + ((int64_t)chunk * pl.m_tiles + mt) * 128 * pl.n_t + (int64_t)(warp * 32 + lane) * pl.n_t;
+        if (n_slabs > 0 && okp) {
+            if (mbar_wait(tfull, 0)) {
+                tc_fence_after();
+                const uint32_t d_tmem = tmem + ((uint32_t)(warp * 32) << 16);
+                for (int c0 = 0; c0 < pl.n_t; c0 += 16) {
+                    float x[32];
+#pragma unroll
+                    for (int jx = 0; jx < 16; ++jx) x[jx] = 0.f;
+                    tmem_ld16_add<0>(d_tmem + (uint32_t)c0, x);
+                    if (!WIDE) tmem_ld16_add<0>(d_tmem + (uint32_t)(32 * nbk + c0), x);
+#pragma unroll
+                    for (int jx = 0; jx < 16; jx += 4)
+                        *reinterpret_cast<float4*>(out + c0 + jx) = make_float4(x[jx], x[jx + 1], x[jx + 2], x[jx + 3]);
+                }
+            } else if (lane == 0) {
+                atomicExch(fault, 10);
+            }
+        } else if (n_slabs == 0) {
+            for (int jx = 0; jx < pl.n_t; ++jx) out[jx] = 0.f;
+        }
+    } else if (warp >= 8) {
+        // ------------------------------------------------------------ B producers: split (and mask) the B slab into the
+        // operand tile, keep its column sums.  16-byte column chunk b_cc of rows b_r0 + BSTEP i.
+        const int tb = tid - 256;
+        const int b_cc = WIDE ? (tb & 63) : (tb & 31), b_r0 = WIDE ? (tb >> 6) : (tb >> 5);
+        constexpr int BI = WIDE ? 16 : 8, BSTEP = WIDE ? 2 : 4;
+        const int nq = pl.n_t / 4;
+        const bool b_mine = b_cc < nq;
+        float4 csum = make_float4(0.f, 0.f, 0.f, 0.f);
+        int rs = 0, ts = 0;
+        uint32_t pass = 0, rpass = 0;
+        bool okp = true;
+        for (int j = 0; j < n_slabs; ++j) {
+            okp = mbar_wait(&rfull[rs], rpass & 1);
+            if (okp && pass >= 1) okp = mbar_wait(&afree[ts], (pass - 1) & 1);
+            if (!okp) break;
+            const unsigned char* slot = raw + rs * slot_bytes;
             if (b_mine) {
                 const unsigned char* braw = slot + 16384 + b_cc * 16;
                 const unsigned char* mraw = slot + 16384 + b_raw_pad + b_cc * 4;
@@ -2103,8 +2154,6 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
             }
             __syncwarp();
             if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&rfree[rs])) : "memory");
-            tmem_st_wait();
-            tc_fence_before();
             proxy_fence();
             asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&afull[ts])) : "memory");
             if (++rs == R) {
@@ -2117,38 +2166,16 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
             }
         }
         if (!okp && lane == 0) atomicExch(fault, 8);
-        // column sums of this chunk's rows: four row groups per column chunk, added in a fixed order
+        // column sums of this chunk's rows: the row groups of each column chunk, added in a fixed order
         if (colsum && (pl.b_cols_per_tile > 0 || mt == 0)) {
-            asm volatile("bar.sync 1, 128;" ::: "memory");   // every producer has read its last raw slab
+            asm volatile("bar.sync 1, 128;" ::: "memory");   // every B producer has read its last raw slab
             if (b_mine) *reinterpret_cast<float4*>(csum_s + b_r0 * (WIDE ? 256 : 128) + b_cc * 4) = csum;
             asm volatile("bar.sync 1, 128;" ::: "memory");
-            for (int cidx = tid; cidx < pl.n_t; cidx += 128) {
+            for (int cidx = tb; cidx < pl.n_t; cidx += 128) {
                 const float sum = WIDE ? csum_s[cidx] + csum_s[256 + cidx]
                                        : ((csum_s[cidx] + csum_s[128 + cidx]) + csum_s[256 + cidx]) + csum_s[384 + cidx];
                 colsum[((int64_t)chunk * pl.m_tiles + mt) * pl.n_t + cidx] = cidx < pl.n_valid ? sum : 0.f;
             }
-        }
-        // epilogue: partial tile -> scratch (row = A column 32 warp + lane of the tile)
-        float* out = scratch + ((int64_t)chunk * pl.m_tiles + mt) * 128 * pl.n_t + (int64_t)(warp * 32 + lane) * pl.n_t;
-        if (n_slabs > 0 && okp) {
-            if (mbar_wait(tfull, 0)) {
-                tc_fence_after();
-                const uint32_t d_tmem = tmem + ((uint32_t)(warp * 32) << 16);
-                for (int c0 = 0; c0 < pl.n_t; c0 += 16) {
-                    float x[32];
-#pragma unroll
-                    for (int jx = 0; jx < 16; ++jx) x[jx] = 0.f;
-                    tmem_ld16_add<0>(d_tmem + (uint32_t)c0, x);
-                    if (!WIDE) tmem_ld16_add<0>(d_tmem + (uint32_t)(32 * nbk + c0), x);
-#pragma unroll
-                    for (int jx = 0; jx < 16; jx += 4)
-                        *reinterpret_cast<float4*>(out + c0 + jx) = make_float4(x[jx], x[jx + 1], x[jx + 2], x[jx + 3]);
-                }
-            } else if (lane == 0) {
-                atomicExch(fault, 10);
-            }
-        } else if (n_slabs == 0) {
-            for (int jx = 0; jx < pl.n_t; ++jx) out[jx] = 0.f;
         }
     } else if (warp == 4) {
         // ------------------------------------------------------------ MMA issuer
@@ -2188,7 +2215,7 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
             if (okm) umma_commit(tfull);
             else atomicExch(fault, 9);
         }
-    } else {
+    } else if (warp == 5) {
         // ------------------------------------------------------------ loader
         if (lane == 0) {
             int rs = 0;
