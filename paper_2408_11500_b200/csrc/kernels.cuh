@@ -72,6 +72,15 @@ struct GemmArgs {
 slicegcn_status_t gemm_run(const GemmArgs& a, cudaStream_t st);
 slicegcn_status_t tc_gemm_run(const GemmArgs& a, cudaStream_t st);
 int64_t tc_image_bytes(int groups, int K, int N);
+// Weight images kept across the GEMMs and epochs of a training run (see tc.cu).  Between begin and end the
+// tensor-core GEMMs of the calling thread take their images from the cache region; begin converts every image
+// recorded by earlier epochs in one launch.
+struct TcImageCache;
+TcImageCache* tc_image_cache_create();
+void tc_image_cache_destroy(TcImageCache* c);
+slicegcn_status_t tc_image_cache_begin(TcImageCache* c, void* region, int64_t bytes, const float* params, int64_t param_elems,
+                                       cudaStream_t st);
+void tc_image_cache_end();
 // true when the tensor-core kernel that takes this product applies a.a_mask in its producer at no extra pass
 // (otherwise multiplying the operand once up front is cheaper than the masked fallback kernels)
 bool tc_gemm_masks_in_producer(const GemmArgs& a);

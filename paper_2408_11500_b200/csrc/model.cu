@@ -487,6 +487,10 @@ struct slicegcn_model {
     int64_t ff_W1 = -1, ff_b1 = -1, ff_W2 = -1, ff_b2 = -1, E = -1, Wc1 = -1, bc1 = -1, Wc2 = -1, bc2 = -1;
     std::vector<int64_t> W_agg, W_self, b, b_self;
     std::vector<int> order;   // resolved per layer
+    // weight images of the tensor-core GEMMs, kept across the epochs of a training run (host bookkeeping only;
+    // the images live in the caller's workspace).  Makes training calls on one model non-reentrant.
+    mutable sgcn::TcImageCache* image_cache = nullptr;
+    ~slicegcn_model() { sgcn::tc_image_cache_destroy(image_cache); }
 
     int64_t add(const std::string& name, int d0, int d1, int d2) {
         const int64_t off = param_elems;
@@ -527,6 +531,8 @@ struct EpochLayout {
     int64_t ws_bytes = 0;
     void* tc_img = nullptr;      // weight images of the dense heads' tensor-core GEMMs
     int64_t tc_img_bytes = 0;
+    void* img_cache = nullptr;   // region of the epoch's image cache
+    int64_t img_cache_bytes = 0;
 };
 
 slicegcn_status_t layer_desc_for(const slicegcn_model* m, int l, const float* params, int64_t x_ld, int* starts_buf,
@@ -612,6 +618,16 @@ slicegcn_status_t build_layout(const slicegcn_model* m, const slicegcn_graph* g,
         }
         E.tc_img_bytes = align_up(img, 256);
         E.tc_img = b.take(E.tc_img_bytes);
+        // every distinct weight operand of an epoch once: two heads forward and backward, FF, and per layer the two
+        // forward and two backward operands (each at most one image of a layer's size)
+        int64_t cache = 4 * E.tc_img_bytes;
+        for (int l = 0; l < L; ++l) {
+            const int in_w = m->layer_in_width(l);
+            cache += 4 * align_up(std::max(tc_image_bytes(p, in_w, m->h_s), tc_image_bytes(p, m->h_s, in_w)), 256);
+        }
+        if (D.use_ff) cache += 4 * E.tc_img_bytes;
+        E.img_cache_bytes = cache;
+        E.img_cache = b.take(cache);
     }
     E.total = align_up(b.off, 256);
     return SLICEGCN_OK;
@@ -803,6 +819,12 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
         SGCN_FAIL(SLICEGCN_ERR_ALLOC, "train_epoch: workspace too small (%lld < %lld)", (long long)workspace_bytes,
                   (long long)E.total);
     SGCN_CUDA(cudaMemsetAsync(grads, 0, sizeof(float) * m->param_elems, st));
+    // weight images: everything recorded by earlier epochs of this run is converted now, in one launch
+    if (!m->image_cache) m->image_cache = tc_image_cache_create();
+    struct CacheScope {
+        ~CacheScope() { tc_image_cache_end(); }
+    } cache_scope;
+    SGCN_TRY(tc_image_cache_begin(m->image_cache, E.img_cache, E.img_cache_bytes, params, m->param_elems, st));
 
     // ---------------- forward
     const void* h0 = X;

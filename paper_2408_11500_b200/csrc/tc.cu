@@ -20,11 +20,39 @@
 #include <algorithm>
 #include <cstdlib>
 #include <type_traits>
+#include <vector>
 
 #include "common.cuh"
 #include "kernels.cuh"
 
 namespace sgcn {
+
+constexpr int kMaxPrepJobs = 40;
+struct PrepJob {            // one weight operand to convert: the B-side fields of a GemmArgs plus where the image goes
+    const float* B;
+    int64_t b_gstride;
+    int ldb, b_trans, K, N, n_pad, n_slabs, n_tiles, groups, bf16;
+    unsigned char* image;
+    int block0;             // first block of this job in a batched launch
+};
+
+
+// Weight images of one model, kept across the GEMMs and the epochs of a training run.  A GEMM that
+// finds its weight operand here skips the conversion; slicegcn_train_epoch converts every image
+// recorded so far in ONE launch when the epoch starts (the weights change once per epoch) instead of
+// one small launch in front of every GEMM.  Entries are keyed by the exact weight pointer and shape
+// and live in a region of the caller's workspace; a different region, or weights outside the
+// current parameter buffer, drop the entry.  Not thread-safe (one training run per model).
+struct TcImageCache {
+    unsigned char* region = nullptr;
+    int64_t region_bytes = 0, used = 0;
+    struct Entry {
+        PrepJob job;
+        bool fresh;
+    };
+    std::vector<Entry> entries;
+};
+
 namespace {
 
 constexpr int kWaitSpins = 1 << 22;
@@ -261,33 +289,58 @@ __device__ __forceinline__ void put_bf16x2(unsigned char* hi, unsigned char* lo,
 // GEMM into the exact bytes a shared-memory tile holds -- K-major rows of 128 bytes, swizzled, split
 // into hi and lo -- and every CTA then pulls a slab's image with one bulk copy.
 // Image of (group g, n tile nt, K slab s): [hi: n_pad rows x 128 B][lo: n_pad rows x 128 B].
+// One quarter (part) of the image of (group g, n tile nt, K slab s).
 template <bool BF16>
-__global__ void __launch_bounds__(128) tc_prep_b_kernel(const GemmArgs a, const int n_pad, unsigned char* image) {
+__device__ __forceinline__ void prep_image_block(const PrepJob& j, int s, int part, int nt, int g) {
     constexpr int KS = BF16 ? 64 : 32;
-    const int s = blockIdx.x / 4, part = blockIdx.x % 4, nt = blockIdx.y, g = blockIdx.z;
-    const int n_slabs = gridDim.x / 4, n_tiles = gridDim.y;
-    const float* B = a.B + (int64_t)g * a.b_gstride;
-    unsigned char* hi = image + ((((int64_t)g * n_tiles + nt) * n_slabs + s) * 2) * ((int64_t)n_pad * 128);
-    unsigned char* lo = hi + (int64_t)n_pad * 128;
-    const int n0 = nt * n_pad, k0 = s * KS;
-    const int per = (n_pad * KS + 3) / 4;   // this block's quarter of the tile's elements
-    for (int e = part * per + threadIdx.x; e < min((part + 1) * per, n_pad * KS); e += 128) {
+    const float* B = j.B + (int64_t)g * j.b_gstride;
+    unsigned char* hi = j.image + ((((int64_t)g * j.n_tiles + nt) * j.n_slabs + s) * 2) * ((int64_t)j.n_pad * 128);
+    unsigned char* lo = hi + (int64_t)j.n_pad * 128;
+    const int n0 = nt * j.n_pad, k0 = s * KS;
+    const int per = (j.n_pad * KS + 3) / 4;   // this block's quarter of the tile's elements
+    for (int e = part * per + threadIdx.x; e < min((part + 1) * per, j.n_pad * KS); e += 128) {
         int n, kk;
-        if (a.b_trans) {
+        if (j.b_trans) {
             kk = e % KS;
             n = e / KS;
         } else {
-            n = e % n_pad;
-            kk = e / n_pad;
+            n = e % j.n_pad;
+            kk = e / j.n_pad;
         }
         const int k = k0 + kk, col = n0 + n;
         float v = 0.f;
-        if (col < a.N && k < a.K) v = a.b_trans ? __ldg(B + (int64_t)col * a.ldb + k) : __ldg(B + (int64_t)k * a.ldb + col);
+        if (col < j.N && k < j.K) v = j.b_trans ? __ldg(B + (int64_t)col * j.ldb + k) : __ldg(B + (int64_t)k * j.ldb + col);
         if (BF16)
             put_bf16x2(hi, lo, n, kk, v);
         else
             put_f32(hi, lo, n, kk, v);
     }
+}
+
+template <bool BF16>
+__global__ void __launch_bounds__(128) tc_prep_b_kernel(const PrepJob j) {
+    prep_image_block<BF16>(j, blockIdx.x / 4, blockIdx.x % 4, blockIdx.y, blockIdx.z);
+}
+
+// All images of a training epoch in one launch: block b belongs to the job with block0 <= b < next block0.
+struct PrepBatch {
+    PrepJob job[kMaxPrepJobs];
+    int count;
+};
+__global__ void __launch_bounds__(128) tc_prep_batch_kernel(const __grid_constant__ PrepBatch batch) {
+    int ji = 0;
+    while (ji + 1 < batch.count && (int)blockIdx.x >= batch.job[ji + 1].block0) ++ji;
+    const PrepJob& j = batch.job[ji];
+    int b = (int)blockIdx.x - j.block0;
+    const int per_g = j.n_slabs * 4 * j.n_tiles;
+    const int g = b / per_g;
+    b -= g * per_g;
+    const int nt = b / (j.n_slabs * 4);
+    b -= nt * (j.n_slabs * 4);
+    if (j.bf16)
+        prep_image_block<true>(j, b / 4, b % 4, nt, g);
+    else
+        prep_image_block<false>(j, b / 4, b % 4, nt, g);
 }
 
 // ------------------------------------------------------------------------------ row-panel GEMM
@@ -1408,6 +1461,32 @@ bool make_slab_map(CUtensorMap* map, const void* base, int64_t rows, int64_t col
                   swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+thread_local TcImageCache* t_image_cache = nullptr;
+
+// The image for job j (image pointer filled in): from the cache when one is active, else nullptr.
+// *fresh tells whether it already holds this epoch's weights.
+unsigned char* cached_image(PrepJob& j, int64_t bytes, bool* fresh) {
+    TcImageCache* c = t_image_cache;
+    *fresh = false;
+    if (!c || !c->region) return nullptr;
+    for (auto& e : c->entries) {
+        const PrepJob& k = e.job;
+        if (k.B == j.B && k.b_gstride == j.b_gstride && k.ldb == j.ldb && k.b_trans == j.b_trans && k.K == j.K && k.N == j.N &&
+            k.n_pad == j.n_pad && k.groups == j.groups && k.bf16 == j.bf16) {
+            *fresh = e.fresh;
+            e.fresh = true;   // the caller converts it now if it was not
+            j.image = k.image;
+            return k.image;
+        }
+    }
+    const int64_t need = (bytes + 255) & ~(int64_t)255;
+    if ((int)c->entries.size() >= kMaxPrepJobs || c->used + need > c->region_bytes) return nullptr;
+    j.image = c->region + c->used;
+    c->used += need;
+    c->entries.push_back({j, true});
+    return j.image;
+}
+
 // fp32 products that tc_gemm_ts_kernel takes (n_pad as chosen by tc_gemm_launch): 16-byte aligned
 // operands and result, up to 128 output columns per tile (32 with the fused second product), bias /
 // post vectors that fit the staging arrays; an operand mask only without a second product and with
@@ -1476,17 +1555,31 @@ slicegcn_status_t tc_gemm_launch(const GemmArgs& a, void* image, int64_t image_b
         SGCN_CUDA(cudaFuncSetAttribute(tc_gemm_kernel<TA, TC, BF16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, mx));
         configured = true;
     }
-    dim3 pgrid(n_slabs * 4, n_tiles, a.groups);
-    tc_prep_b_kernel<BF16><<<pgrid, 128, 0, st>>>(a, n_pad, static_cast<unsigned char*>(image));
-    SGCN_LAUNCH_CHECK();
-    if (fused) {
-        GemmArgs b2 = a;
-        b2.B = a.B2;
-        b2.b_gstride = a.b2_gstride;
-        b2.K = a.K2;
-        dim3 pgrid2(n_slabs2 * 4, n_tiles, a.groups);
-        tc_prep_b_kernel<BF16><<<pgrid2, 128, 0, st>>>(b2, n_pad, image2);
-        SGCN_LAUNCH_CHECK();
+    {   // weight image(s): from the epoch's cache when there is one, else converted here into the scratch
+        PrepJob j{a.B, a.b_gstride, a.ldb, a.b_trans, a.K, a.N, n_pad, n_slabs, n_tiles, a.groups, BF16 ? 1 : 0, nullptr, 0};
+        bool fresh = false;
+        unsigned char* cimg = cached_image(j, need, &fresh);
+        if (cimg) image = cimg;
+        else j.image = static_cast<unsigned char*>(image);
+        if (!fresh) {
+            dim3 pgrid(n_slabs * 4, n_tiles, a.groups);
+            tc_prep_b_kernel<BF16><<<pgrid, 128, 0, st>>>(j);
+            SGCN_LAUNCH_CHECK();
+            count_launch();
+        }
+        if (fused) {
+            PrepJob j2{a.B2, a.b2_gstride, a.ldb, a.b_trans, a.K2, a.N, n_pad, n_slabs2, n_tiles, a.groups, BF16 ? 1 : 0, nullptr, 0};
+            bool fresh2 = false;
+            unsigned char* cimg2 = cached_image(j2, need2, &fresh2);
+            if (cimg2) image2 = cimg2;
+            else j2.image = image2;
+            if (!fresh2) {
+                dim3 pgrid2(n_slabs2 * 4, n_tiles, a.groups);
+                tc_prep_b_kernel<BF16><<<pgrid2, 128, 0, st>>>(j2);
+                SGCN_LAUNCH_CHECK();
+                count_launch();
+            }
+        }
     }
     // 16-byte loads of the activation need aligned slices
     bool vec = ((uintptr_t)a.A % 16 == 0) && (a.lda % EPC == 0) && (a.K % EPC == 0 || a.a_pad_zero);
@@ -1541,7 +1634,7 @@ slicegcn_status_t tc_gemm_launch(const GemmArgs& a, void* image, int64_t image_b
                 tc_gemm_ts_kernel<false><<<(unsigned)tgrid, kTsThreads, ts_smem, st>>>(a, n_pad, n_tiles, ring, static_cast<unsigned char*>(image), image2,
                                                                                        fault, map_a, map_a2, map_m);
             SGCN_LAUNCH_CHECK();
-            count_launch(fused ? 3 : 2);
+            count_launch();
             return SLICEGCN_OK;
             }
         }
@@ -1565,7 +1658,7 @@ slicegcn_status_t tc_gemm_launch(const GemmArgs& a, void* image, int64_t image_b
             if (wgrid > items) wgrid = items;
             tc_gemm_ws_kernel<TA, TC, BF16><<<(unsigned)wgrid, kWsThreads, ws_smem, st>>>(a, n_pad, n_tiles, D, static_cast<unsigned char*>(image), image2, fault);
             SGCN_LAUNCH_CHECK();
-            count_launch(fused ? 3 : 2);
+            count_launch();
             return SLICEGCN_OK;
         }
     }
@@ -1585,7 +1678,7 @@ slicegcn_status_t tc_gemm_launch(const GemmArgs& a, void* image, int64_t image_b
     else
         tc_gemm_kernel<TA, TC, BF16, false><<<(unsigned)grid, kTcThreads, smem_bytes, st>>>(a, n_pad, n_tiles, static_cast<unsigned char*>(image), fault);
     SGCN_LAUNCH_CHECK();
-    count_launch(2);
+    count_launch();
     return SLICEGCN_OK;
 }
 
@@ -2391,6 +2484,46 @@ bool wgrad_ts_ok(const WgradArgs& a, const WgTcPlan& pl) {
 }
 
 }  // namespace
+
+TcImageCache* tc_image_cache_create() { return new TcImageCache(); }
+void tc_image_cache_destroy(TcImageCache* c) { delete c; }
+
+slicegcn_status_t tc_image_cache_begin(TcImageCache* c, void* region, int64_t bytes, const float* params, int64_t param_elems,
+                                       cudaStream_t st) {
+    if (!c) return SLICEGCN_OK;
+    if (c->region != region || c->region_bytes != bytes) {   // another workspace: nothing recorded is valid
+        c->entries.clear();
+        c->used = 0;
+        c->region = static_cast<unsigned char*>(region);
+        c->region_bytes = bytes;
+    }
+    // keep what still points into this call's parameter buffer, convert all of it in one launch
+    std::vector<TcImageCache::Entry> keep;
+    for (auto& e : c->entries)
+        if (e.job.B >= params && e.job.B < params + param_elems) keep.push_back(e);
+    if (keep.size() != c->entries.size()) {   // a hole would waste space: start over
+        c->entries.clear();
+        c->used = 0;
+        keep.clear();
+    }
+    if (!keep.empty()) {
+        PrepBatch batch;
+        batch.count = (int)keep.size();
+        int blocks = 0;
+        for (int i = 0; i < batch.count; ++i) {
+            batch.job[i] = keep[i].job;
+            batch.job[i].block0 = blocks;
+            blocks += keep[i].job.n_slabs * 4 * keep[i].job.n_tiles * keep[i].job.groups;
+        }
+        tc_prep_batch_kernel<<<blocks, 128, 0, st>>>(batch);
+        SGCN_LAUNCH_CHECK();
+        count_launch();
+        for (auto& e : c->entries) e.fresh = true;
+    }
+    t_image_cache = c;
+    return SLICEGCN_OK;
+}
+void tc_image_cache_end() { t_image_cache = nullptr; }
 
 bool tc_wgrad_masks_in_producer(const WgradArgs& a) {
     static const bool off = getenv("SLICEGCN_NO_TS") != nullptr || getenv("SLICEGCN_NO_WS") != nullptr;
