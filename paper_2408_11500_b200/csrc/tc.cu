@@ -2337,34 +2337,45 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
     if (warp == 4) tmem_dealloc(tmem, 512);
 }
 
-// dbias[g][n] = sum over chunks of the column-sum partials (fixed order); same tile mapping as the dW reduce
-__global__ void tc_wgrad_bias_reduce_kernel(const float* colsum, const WgTcPlan pl, int groups, int N, int groups_per_tile, float* dbias,
-                                            float* dbias2) {
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= groups * N) return;
-    const int g = i / N, n = i % N;
-    int mt = 0, c = n;
-    if (groups_per_tile > 0) {
-        mt = g / groups_per_tile;
-        c = (g % groups_per_tile) * N + n;
-    } else if (groups_per_tile < 0) {
-        c = g * N + n;
-    }
-    float s = 0.f;
-    for (int ch = 0; ch < pl.n_chunks; ++ch) s += __ldg(colsum + ((int64_t)ch * pl.m_tiles + mt) * pl.n_t + c);
-    if (dbias) dbias[i] = s;
-    if (dbias2) dbias2[i] = s;
-}
-
 // dW[g][k][n] = sum over chunks of the partial tiles (fixed order).  A block owns 32 consecutive
 // elements; its eight warps each sum every eighth chunk (a handful of independent loads, so the
 // kernel is not one long dependent chain per element) and the eight partial sums are added in
 // warp order.
+// Blocks past the dW elements (when colsum != NULL) reduce the column-sum partials into dbias / dbias2 the same way.
 __global__ void __launch_bounds__(256) tc_wgrad_reduce_kernel(const float* scratch, const WgTcPlan pl, int groups, int K, int N,
-                                                              int groups_per_tile, float* dW) {
+                                                              int groups_per_tile, float* dW, const float* colsum = nullptr,
+                                                              float* dbias = nullptr, float* dbias2 = nullptr) {
     __shared__ float part[8][32];
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const int64_t total = (int64_t)groups * K * N;
+    const int64_t w_blocks = (total + 31) / 32;
+    if ((int64_t)blockIdx.x >= w_blocks) {   // bias part: element = (group, column)
+        const int i = (int)((blockIdx.x - w_blocks) * 32) + lane;
+        float s = 0.f;
+        if (i < groups * N) {
+            const int g = i / N, n = i % N;
+            int mt = 0, c = n;
+            if (groups_per_tile > 0) {
+                mt = g / groups_per_tile;
+                c = (g % groups_per_tile) * N + n;
+            } else if (groups_per_tile < 0) {
+                c = g * N + n;
+            }
+            const float* p = colsum + (int64_t)mt * pl.n_t + c;
+            const int64_t stride = (int64_t)pl.m_tiles * pl.n_t;
+            for (int ch = w; ch < pl.n_chunks; ch += 8) s += __ldg(p + ch * stride);
+        }
+        part[w][lane] = s;
+        __syncthreads();
+        if (w == 0 && i < groups * N) {
+            float t = part[0][lane];
+#pragma unroll
+            for (int q = 1; q < 8; ++q) t += part[q][lane];
+            if (dbias) dbias[i] = t;
+            if (dbias2) dbias2[i] = t;
+        }
+        return;
+    }
     const int64_t i = blockIdx.x * (int64_t)32 + lane;
     float s = 0.f;
     if (i < total) {
@@ -2605,15 +2616,12 @@ slicegcn_status_t tc_wgrad_run(const WgradArgs& a, void* scratch, int64_t scratc
                         tc_wgrad_ts_kernel<false><<<tgrid, kWtThreads, ts_smem, st>>>(a, pn, static_cast<float*>(scratch), colsum, a.fault, map_a, map_b, map_bm);
                     SGCN_LAUNCH_CHECK();
                     const int64_t total_w = (int64_t)a.groups * a.K * a.N;
-                    tc_wgrad_reduce_kernel<<<(unsigned)((total_w + 31) / 32), 256, 0, st>>>(static_cast<const float*>(scratch), pn,
-                                                                                             a.groups, a.K, a.N, gn, a.dW);
+                    const unsigned red_blocks = (unsigned)((total_w + 31) / 32) + (want_bias ? (unsigned)((b_total + 31) / 32) : 0u);
+                    tc_wgrad_reduce_kernel<<<red_blocks, 256, 0, st>>>(static_cast<const float*>(scratch), pn, a.groups, a.K, a.N, gn, a.dW,
+                                                                         colsum, a.dbias, a.dbias2);
                     SGCN_LAUNCH_CHECK();
-                    if (want_bias) {
-                        tc_wgrad_bias_reduce_kernel<<<(b_total + 127) / 128, 128, 0, st>>>(colsum, pn, a.groups, a.N, gn, a.dbias, a.dbias2);
-                        SGCN_LAUNCH_CHECK();
-                        if (bias_done) *bias_done = true;
-                    }
-                    count_launch(want_bias ? 3 : 2);
+                    if (want_bias && bias_done) *bias_done = true;
+                    count_launch(2);
                     return SLICEGCN_OK;
                 }
             }
