@@ -55,7 +55,7 @@ constexpr int kSegment = 256;
 // The remaining rows are dealt out in row-aligned chunks of about kChunk stored entries: chunk c
 // owns every row whose first entry index lies in [c*kChunk, (c+1)*kChunk), so each lane group gets
 // the same amount of gather work whatever the degree distribution.
-constexpr int kChunk = 128;
+constexpr int kChunk = 64;
 
 struct CsrView {
     const int32_t* rowptr = nullptr;   // [n+1]
