@@ -1,0 +1,83 @@
+"""Training throughput of the paper's model variants on one synthetic graph shape.
+
+The layout follows the paper's Table IV (methods x number of slices): plain GCN (one slice, no self
+branch), SliceGCN with p slices, and the -SE / -FF / -FFSE variants.  Accuracy columns need the
+paper's datasets and are not reproduced; this prints epochs/s of the CUDA path only.
+
+    python -m paper_2408_11500_b200.variant_grid --workload citation --epochs 20
+"""
+from __future__ import annotations
+
+import argparse
+
+import numpy as np
+
+
+def time_variant(B, torch, g, w, X, y, p, use_ff, use_se, use_self, epochs, warmup=3):
+    from . import synth
+    dev = X.device
+    m = B.slicegcn_model_create(in_d=w["in_d"], hidden=w["hidden"], num_layers=w["layers"], num_classes=w["classes"],
+                                num_slices=p, use_ff=use_ff, use_se=use_se, use_self=use_self,
+                                dtype=B.BF16 if X.dtype == torch.bfloat16 else B.F32)
+    try:
+        params = torch.from_numpy(B.pack_params(m, synth.init_params(B.named_param_shapes(m), 0))).to(dev)
+        grads, m1, m2 = torch.zeros_like(params), torch.zeros_like(params), torch.zeros_like(params)
+        ws_bytes = B.slicegcn_train_workspace_bytes(m, g)
+        ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+        loss = torch.zeros(1, dtype=torch.float32, device=dev)
+        st = torch.cuda.current_stream()
+
+        def epoch(ep):
+            B.slicegcn_train_epoch(m, g, X, w["in_d"], y, None, 0, params, grads, m1, m2, B.make_opt_desc(1e-3, ep, 500),
+                                   None, loss, ws, ws_bytes, st.cuda_stream)
+
+        for ep in range(warmup):
+            epoch(ep)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(st)
+        for ep in range(epochs):
+            epoch(warmup + ep)
+        e1.record(st)
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / epochs
+        count = B.slicegcn_model_param_count(m)
+        return ms, count, float(loss.item())
+    finally:
+        B.slicegcn_model_destroy(m)
+
+
+def main():
+    import torch
+    from . import binding as B, synth
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--workload", default="citation", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--epochs", type=int, default=20)
+    ap.add_argument("--slices", default="2,4,8")
+    args = ap.parse_args()
+    w = synth.WORKLOADS[args.workload]
+    src, dst = synth.make_graph(w, 0)
+    g = B.slicegcn_graph_create(w["n"], src, dst, B.SYMMETRIZE | B.ADD_SELF_LOOPS)
+    info = B.slicegcn_graph_info(g)
+    tdt = torch.bfloat16 if w["dtype"] == "bf16" else torch.float32
+    X = torch.from_numpy(synth.make_features(w, 0)).cuda().to(tdt).contiguous()
+    y = torch.from_numpy(synth.uniform_labels(w["n"], w["classes"], 0)).cuda()
+    ps = [int(v) for v in args.slices.split(",")]
+    print(f"workload `{args.workload}`: N={w['n']:,}, nnz={info['nnz']:,}, in_d={w['in_d']}, hidden={w['hidden']}, "
+          f"layers={w['layers']}, classes={w['classes']}, {w['dtype']}; {args.epochs} timed epochs per cell\n")
+    print("| method | " + " | ".join(f"p={p}: ms/epoch (epochs/s) [params]" for p in ps) + " |")
+    print("|---|" + "---|" * len(ps))
+    ms, cnt, _ = time_variant(B, torch, g, w, X, y, 1, False, False, False, args.epochs)
+    print(f"| GCN (one slice, no self branch) | {ms:.2f} ({1e3 / ms:.1f}) [{cnt:,}] |" + " |" * (len(ps) - 1))
+    for name, ff, se in (("SliceGCN", False, False), ("SliceGCN-SE", False, True), ("SliceGCN-FF", True, False),
+                         ("SliceGCN-FFSE", True, True)):
+        cells = []
+        for p in ps:
+            ms, cnt, _ = time_variant(B, torch, g, w, X, y, p, ff, se, True, args.epochs)
+            cells.append(f"{ms:.2f} ({1e3 / ms:.1f}) [{cnt:,}]")
+        print(f"| {name} | " + " | ".join(cells) + " |")
+    B.slicegcn_graph_destroy(g)
+
+
+if __name__ == "__main__":
+    main()
