@@ -1437,7 +1437,7 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
     if (warp == 4) tmem_dealloc(tmem, 512);
 }
 
-// Tensor map over a row-major fp32 (or, elem_bytes = 1, byte) matrix for boxes of box_rows x box_cols values (default: one
+// Tensor map over a row-major fp32 (elem_bytes = 2: bf16, 1: byte) matrix for boxes of box_rows x box_cols values (default: one
 // activation slab of 128 rows x 32 columns), written to shared memory with the 128-byte swizzle or plain.  `cols` bounds the columns a box may read
 // (beyond it: zeros).  The encoder is a driver entry point, looked up once; false if unavailable.
 typedef CUresult (*TensorMapEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -1457,7 +1457,7 @@ bool make_slab_map(CUtensorMap* map, const void* base, int64_t rows, int64_t col
     const cuuint64_t strides[1] = {(cuuint64_t)ld * (cuuint64_t)elem_bytes};
     const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
-    return encode(map, elem_bytes == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+    return encode(map, elem_bytes == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                   swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -2087,8 +2087,9 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_wgrad_ws_kernel(const WgradA
 constexpr int kWtThreads = 384;
 
 // WIDE: B tiles of 129..256 columns -- no room for [hi | lo] in one operand (three chains per slab) and
-// only two raw slots.
-template <bool WIDE>
+// only two raw slots.  ABF16: A is stored as bf16 -- exact in tf32, so it has no lo part and a slab takes
+// one chain less.
+template <bool WIDE, bool ABF16>
 __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradArgs a, const WgTcPlan pl, float* scratch, float* colsum,
                                                                     int* fault, const __grid_constant__ CUtensorMap map_a,
                                                                     const __grid_constant__ CUtensorMap map_b,
@@ -2151,16 +2152,22 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
             // column 32 warp + lane of the slab, 32 values down the rows
             const bool a_live = 32 * warp + lane < pl.a_box;   // columns past the fetched width stay zero
             const float* acol = reinterpret_cast<const float*>(slot) + (a_live ? 32 * warp + lane : 0);
+            const uint16_t* acol16 = reinterpret_cast<const uint16_t*>(slot) + (a_live ? 32 * warp + lane : 0);
             const uint32_t t_hi = tmem + ((uint32_t)(32 * warp) << 16) + accw + (uint32_t)ts * 64u;
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
                 uint32_t h[32];   // [0,16): hi of rows 16 half ..; [16,32): lo of the same
 #pragma unroll
                 for (int k = 0; k < 16; ++k) {
-                    const float v = a_live ? acol[(16 * half + k) * pl.a_box] : 0.f;
-                    const float hv = tf32_hi(v);
-                    h[k] = __float_as_uint(hv);
-                    h[16 + k] = __float_as_uint(v - hv);
+                    if (ABF16) {
+                        h[k] = a_live ? (uint32_t)acol16[(16 * half + k) * pl.a_box] << 16 : 0u;
+                        h[16 + k] = 0u;
+                    } else {
+                        const float v = a_live ? acol[(16 * half + k) * pl.a_box] : 0.f;
+                        const float hv = tf32_hi(v);
+                        h[k] = __float_as_uint(hv);
+                        h[16 + k] = __float_as_uint(v - hv);
+                    }
                 }
                 if (half == 1) {   // the slab is in registers: this warp is done with the raw slot
                     __syncwarp();
@@ -2168,7 +2175,7 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
                     __syncwarp();
                 }
                 tmem_st16<0>(t_hi + 16u * half, h);
-                tmem_st16<16>(t_hi + 32u + 16u * half, h);
+                if (!ABF16) tmem_st16<16>(t_hi + 32u + 16u * half, h);
             }
             tmem_st_wait();
             tc_fence_before();
@@ -2292,11 +2299,11 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
                     if (WIDE) {
                         const uint64_t db_lo = smem_desc_mn(op + kb * 2 * (2 * nbk * 512) + nbk * 512, 512, 2 * nbk * 512);
                         umma_ts_tf32(tmem, a_hi + 8u * kb, db, idesc_hi, (j == 0 && kb == 0) ? 0u : 1u);
-                        umma_ts_tf32(tmem, a_lo + 8u * kb, db, idesc_hi, 1u);
+                        if (!ABF16) umma_ts_tf32(tmem, a_lo + 8u * kb, db, idesc_hi, 1u);
                         umma_ts_tf32(tmem, a_hi + 8u * kb, db_lo, idesc_hi, 1u);
                     } else {
                         umma_ts_tf32(tmem, a_hi + 8u * kb, db, idesc_wide, (j == 0 && kb == 0) ? 0u : 1u);
-                        umma_ts_tf32(tmem, a_lo + 8u * kb, db, idesc_hi, 1u);
+                        if (!ABF16) umma_ts_tf32(tmem, a_lo + 8u * kb, db, idesc_hi, 1u);
                     }
                 }
                 umma_commit(&afree[ts]);
@@ -2321,7 +2328,7 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
                 }
                 unsigned char* slot = raw + rs * slot_bytes;
                 const int y = (int)(r_begin + (int64_t)j * 32);
-                mbar_expect_tx(&rfull[rs], 128u * (uint32_t)pl.a_box + b_raw_bytes + (masked ? m_raw_bytes : 0u));
+                mbar_expect_tx(&rfull[rs], (ABF16 ? 64u : 128u) * (uint32_t)pl.a_box + b_raw_bytes + (masked ? m_raw_bytes : 0u));
                 tma_load_2d(slot, &map_a, ax, y, &rfull[rs]);
                 tma_load_2d(slot + 16384, &map_b, bx, y, &rfull[rs]);
                 if (masked) tma_load_2d(slot + 16384 + b_raw_pad, &map_bm, bx, y, &rfull[rs]);
@@ -2487,7 +2494,8 @@ bool wgrad_tc_plan(const WgradArgs& a, WgTcPlan* pl, int* groups_per_tile, int f
 // mask rows and tile starts.
 bool wgrad_ts_ok(const WgradArgs& a, const WgTcPlan& pl) {
     const int nbk = (pl.n_t + 31) / 32;
-    if (a.a_dtype != SLICEGCN_F32 || nbk > 8 || a.M >= ((int64_t)1 << 31)) return false;
+    if (nbk > 8 || a.M >= ((int64_t)1 << 31)) return false;
+    if (a.a_dtype == SLICEGCN_BF16 && (a.lda % 8 || pl.a_col0 % 8 || pl.a_tile_cols % 8)) return false;   // 16-byte tensor copies
     if (a.b_mask) {
         if (nbk > 4 || (uintptr_t)a.b_mask % 16 || a.b_mask_ld % 16 || pl.b_col0 % 16 || pl.b_cols_per_tile % 16) return false;
     }
@@ -2574,7 +2582,7 @@ slicegcn_status_t tc_wgrad_run(const WgradArgs& a, void* scratch, int64_t scratc
     if (bias_done) *bias_done = false;
     if (!a.fault || !wgrad_tc_plan(a, &pl, &gpt)) return SLICEGCN_ERR_UNSUPPORTED;
     static const bool no_ws = getenv("SLICEGCN_NO_WS") != nullptr;
-    if (!no_ws && a.a_dtype == SLICEGCN_F32) {
+    if (!no_ws) {
         // warp-specialised variants: one CTA per SM
         WgTcPlan pw;
         int gw = 0;
@@ -2592,7 +2600,8 @@ slicegcn_status_t tc_wgrad_run(const WgradArgs& a, void* scratch, int64_t scratc
                 const int b_total = a.groups * a.N;
                 CUtensorMap map_a, map_b;
                 CUtensorMap map_bm;
-                bool maps_ok = make_slab_map(&map_a, a.A, a.M, std::min<int64_t>(pn.a_col0 + pn.a_cols, a.lda), a.lda, pn.a_box, 32, false) &&
+                bool maps_ok = make_slab_map(&map_a, a.A, a.M, std::min<int64_t>(pn.a_col0 + pn.a_cols, a.lda), a.lda, pn.a_box, 32, false,
+                                             a.a_dtype == SLICEGCN_BF16 ? 2 : 4) &&
                                make_slab_map(&map_b, a.B, a.M, std::min<int64_t>(pn.b_col0 + b_total, a.ldb), a.ldb, pn.n_t, 32, false);
                 if (maps_ok && a.b_mask)
                     maps_ok = make_slab_map(&map_bm, a.b_mask, a.M, std::min<int64_t>(pn.b_col0 + b_total, a.b_mask_ld), a.b_mask_ld, pn.n_t, 32,
@@ -2605,15 +2614,19 @@ slicegcn_status_t tc_wgrad_run(const WgradArgs& a, void* scratch, int64_t scratc
                     const int ts_smem = 2 * nbk * 8192 + (wide ? 2 : 4) * slot_b + 256 + 1024;
                     static bool ts_configured = false;
                     if (!ts_configured) {
-                        SGCN_CUDA(cudaFuncSetAttribute(tc_wgrad_ts_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-                        SGCN_CUDA(cudaFuncSetAttribute(tc_wgrad_ts_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+                        SGCN_CUDA(cudaFuncSetAttribute(tc_wgrad_ts_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+                        SGCN_CUDA(cudaFuncSetAttribute(tc_wgrad_ts_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+                        SGCN_CUDA(cudaFuncSetAttribute(tc_wgrad_ts_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+                        SGCN_CUDA(cudaFuncSetAttribute(tc_wgrad_ts_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
                         ts_configured = true;
                     }
                     dim3 tgrid(pn.n_chunks, pn.m_tiles);
-                    if (wide)
-                        tc_wgrad_ts_kernel<true><<<tgrid, kWtThreads, ts_smem, st>>>(a, pn, static_cast<float*>(scratch), colsum, a.fault, map_a, map_b, map_bm);
-                    else
-                        tc_wgrad_ts_kernel<false><<<tgrid, kWtThreads, ts_smem, st>>>(a, pn, static_cast<float*>(scratch), colsum, a.fault, map_a, map_b, map_bm);
+                    float* sc = static_cast<float*>(scratch);
+                    const bool abf = a.a_dtype == SLICEGCN_BF16;
+                    if (wide && abf) tc_wgrad_ts_kernel<true, true><<<tgrid, kWtThreads, ts_smem, st>>>(a, pn, sc, colsum, a.fault, map_a, map_b, map_bm);
+                    else if (wide) tc_wgrad_ts_kernel<true, false><<<tgrid, kWtThreads, ts_smem, st>>>(a, pn, sc, colsum, a.fault, map_a, map_b, map_bm);
+                    else if (abf) tc_wgrad_ts_kernel<false, true><<<tgrid, kWtThreads, ts_smem, st>>>(a, pn, sc, colsum, a.fault, map_a, map_b, map_bm);
+                    else tc_wgrad_ts_kernel<false, false><<<tgrid, kWtThreads, ts_smem, st>>>(a, pn, sc, colsum, a.fault, map_a, map_b, map_bm);
                     SGCN_LAUNCH_CHECK();
                     const int64_t total_w = (int64_t)a.groups * a.K * a.N;
                     const unsigned red_blocks = (unsigned)((total_w + 31) / 32) + (want_bias ? (unsigned)((b_total + 31) / 32) : 0u);
@@ -2632,7 +2645,7 @@ slicegcn_status_t tc_wgrad_run(const WgradArgs& a, void* scratch, int64_t scratc
             const int stage_b = 32768 + 2 * 4 * nbk * 1024;
             int D = (220 * 1024) / stage_b;
             if (D > 3) D = 3;
-            if (a.b_mask) D = 0;   // the shared-memory-operand variant takes no mask
+            if (a.b_mask || a.a_dtype != SLICEGCN_F32) D = 0;   // the shared-memory-operand variant takes fp32 operands without a mask
             const int64_t need_w = (int64_t)pw.n_chunks * pw.m_tiles * 128 * pw.n_t * (int64_t)sizeof(float);
             if (D >= 2 && scratch && scratch_bytes >= need_w) {
                 const int ws_smem = D * stage_b + 256 + 1024;
