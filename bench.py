@@ -29,7 +29,7 @@ from paper_2408_11500_b200 import synth  # noqa: E402
 
 # dram__bytes_read.sum + dram__bytes_write.sum per SpMM launch from the ncu capture summarised under
 # profiles/ (None until a capture of that workload exists)
-NCU_SPMM_TRAFFIC_BYTES = {"citation": 922e6}   # width-256 launches (4 of the 5 per epoch)
+NCU_SPMM_TRAFFIC_BYTES = {"citation": 919e6}   # width-256 launches (4 of the 5 per epoch)
 
 
 def measured_peak_gbs():
