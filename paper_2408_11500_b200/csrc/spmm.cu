@@ -166,7 +166,7 @@ __device__ __forceinline__ void finish_chunk(const SpmmParams& p, int64_t row, i
 // 1/sqrt(deg) of L consecutive rows are fetched by the L lanes at once and handed out by shuffles;
 // the column indices of the next batch are requested before the current batch is gathered.
 // Chunks that consist of one long row are left to the segment kernels.
-constexpr int kRowsWarps = 4;   // warps per CTA of the row kernel
+constexpr int kRowsWarps = 1;   // warps per CTA of the row kernel: a finished warp frees its slot at once (measured best)
 // Occupancy and neighbors gathered per round.  Measured on B200: for rows of 256 bytes and more what
 // pays is resident warps (32 per SM, i.e. at most 64 registers) rather than loads per lane -- they run
 // fastest with four 16-byte loads in flight per lane; narrower rows (several rows per warp) and the
