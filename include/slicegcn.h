@@ -308,6 +308,10 @@ slicegcn_status_t slicegcn_train_epochs_host(const slicegcn_model* m, const slic
  * number of kernels the library launched.  Any output pointer may be NULL.  Not thread-safe.
  */
 slicegcn_status_t slicegcn_profile_begin(void);
+/* The same, bracketing only every stride-th SpMM call (stride >= 1): an event pair costs the stream a few
+ * microseconds, which a benchmark that also reports whole-step time wants to keep small.  With a stride
+ * coprime to the number of SpMM calls per step every call site is sampled equally often. */
+slicegcn_status_t slicegcn_profile_begin_sampled(int32_t stride);
 slicegcn_status_t slicegcn_profile_end(double* spmm_ms, int64_t* spmm_calls, double* spmm_bytes,
                                        int64_t* kernel_launches);
 

@@ -31,7 +31,7 @@ EXPORTS = [
     "slicegcn_spmm", "slicegcn_spmm_static_scratch", "slicegcn_layer_saved_bytes", "slicegcn_layer_workspace_bytes", "slicegcn_layer_forward",
     "slicegcn_layer_backward", "slicegcn_model_create", "slicegcn_model_destroy", "slicegcn_model_param_count",
     "slicegcn_model_param_elems", "slicegcn_model_num_tensors", "slicegcn_model_tensor_info", "slicegcn_model_slices",
-    "slicegcn_model_layer_order", "slicegcn_train_workspace_bytes", "slicegcn_train_epoch", "slicegcn_train_epoch_host", "slicegcn_train_epochs_host", "slicegcn_profile_begin",
+    "slicegcn_model_layer_order", "slicegcn_train_workspace_bytes", "slicegcn_train_epoch", "slicegcn_train_epoch_host", "slicegcn_train_epochs_host", "slicegcn_profile_begin", "slicegcn_profile_begin_sampled",
     "slicegcn_profile_end",
 ]
 
@@ -320,6 +320,10 @@ def slicegcn_train_epochs_host(m, g, X_host, x_ld: int, labels_host, X_stage0, X
 
 def slicegcn_profile_begin() -> None:
     _check(_lib.slicegcn_profile_begin())
+
+
+def slicegcn_profile_begin_sampled(stride: int) -> None:
+    _check(_lib.slicegcn_profile_begin_sampled(c_int32(stride)))
 
 
 def slicegcn_profile_end() -> Dict[str, float]:

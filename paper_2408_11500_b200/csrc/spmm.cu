@@ -580,6 +580,8 @@ struct Profiler {
     size_t used = 0;
     int64_t calls = 0;
     double bytes = 0.0;
+    int64_t seen = 0;              // SpMM calls since begin
+    int stride = 1;                // every stride-th call is bracketed by events
 } g_prof;
 }  // namespace
 
@@ -627,7 +629,7 @@ slicegcn_status_t spmm_run(const slicegcn_graph* g, bool transpose, int in_dtype
                       (long long)spmm_partial_bytes(g, width));
     }
     cudaEvent_t ev_stop = nullptr;
-    if (g_prof.on && instrument) {
+    if (g_prof.on && instrument && (g_prof.seen++ % g_prof.stride) == 0) {
         if (g_prof.used + 2 > g_prof.ev.size()) {
             for (int i = 0; i < 2; ++i) {
                 cudaEvent_t e;
@@ -701,8 +703,11 @@ slicegcn_status_t slicegcn_spmm_static_scratch(const slicegcn_graph* g, int32_t 
                     (cudaStream_t)stream, /*instrument=*/false);
 }
 
-slicegcn_status_t slicegcn_profile_begin(void) {
+slicegcn_status_t slicegcn_profile_begin_sampled(int32_t stride) {
     using namespace sgcn;
+    if (stride < 1) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "profile_begin_sampled: stride < 1");
+    g_prof.stride = stride;
+    g_prof.seen = 0;
     g_prof.on = true;
     g_prof.used = 0;
     g_prof.calls = 0;
@@ -710,6 +715,8 @@ slicegcn_status_t slicegcn_profile_begin(void) {
     reset_launches();
     return SLICEGCN_OK;
 }
+
+slicegcn_status_t slicegcn_profile_begin(void) { return slicegcn_profile_begin_sampled(1); }
 
 slicegcn_status_t slicegcn_profile_end(double* spmm_ms, int64_t* spmm_calls, double* spmm_bytes,
                                        int64_t* kernel_launches) {

@@ -462,3 +462,33 @@ def test_train_epoch_host_buffers_match_device_call(B, torch):
                                         gp.loss, None, gp.ws, gp.ws_bytes, torch.cuda.current_stream().cuda_stream)
     finally:
         gp.close()
+
+
+def test_profile_counts_and_sampling(B, torch):
+    """The benchmark instrumentation: SpMM calls bracketed by events (all, or every stride-th), algorithmic
+    bytes per bracketed call, and the number of kernels launched in between."""
+    n = 3000
+    src, dst = synth.chung_lu_powerlaw(n, 12000, 2.2, 300, seed=3)
+    g = B.slicegcn_graph_create(n, src, dst, B.SYMMETRIZE | B.ADD_SELF_LOOPS)
+    try:
+        info = B.slicegcn_graph_info(g)
+        w = 64
+        X = torch.randn(n, w, device="cuda"); Y = torch.empty_like(X)
+        wsb = B.slicegcn_spmm_workspace_bytes(g, w); ws = torch.empty(max(wsb, 16), dtype=torch.uint8, device="cuda")
+        st = torch.cuda.current_stream().cuda_stream
+        per_call = 4 * info["nnz"] + 4 * (n + 1) + 4 * n + 2 * n * w * 4
+        for stride, want_calls in ((1, 10), (3, 4)):
+            if stride == 1:
+                B.slicegcn_profile_begin()
+            else:
+                B.slicegcn_profile_begin_sampled(stride)
+            for _ in range(10):
+                B.slicegcn_spmm(g, 0, B.F32, B.F32, X, w, Y, w, w, ws, wsb, st)
+            p = B.slicegcn_profile_end()
+            assert p["spmm_calls"] == want_calls                      # calls 0, 3, 6, 9 for stride 3
+            assert p["spmm_bytes"] == want_calls * per_call
+            assert p["spmm_ms"] > 0 and p["kernel_launches"] >= 10
+        with pytest.raises(B.SliceGCNError):
+            B.slicegcn_profile_begin_sampled(0)
+    finally:
+        B.slicegcn_graph_destroy(g)
