@@ -1,12 +1,14 @@
 // Normalised sparse aggregation  Y = A_hat X  (Eq. 1 / Eq. 6 neighbor sum; A_hat^T X in backward).
 //
-// Row-parallel CSR kernel.  A group of L lanes owns one row; each lane keeps C 16-byte chunks of
-// the output row in registers, so one 128-bit load per lane per chunk covers a neighbor's slice
-// row.  Column indices are read coalesced (L at a time) together with the neighbor's 1/sqrt(deg)
-// and handed around with shuffles; U neighbors are gathered before the FMAs so several rows are in
-// flight per lane.  No per-edge value array exists:  A_hat_ij = dinv_i * dinv_j.
-// Rows longer than kLongRow are cut into kSegment-entry segments, one warp each, whose partial
-// rows are summed afterwards in segment order -- deterministic, no floating-point atomics.
+// Row-parallel CSR kernel over row-aligned chunks of ~kChunk stored entries (common.cuh).  A group of
+// L lanes streams one chunk; each lane keeps C 16-byte chunks of the output row in registers, so one
+// 128-bit load per lane per chunk covers a neighbor's slice row.  Column indices are read coalesced
+// (L at a time) together with the neighbor's 1/sqrt(deg), parked in a per-warp shared-memory slot and
+// read back as one broadcast load per neighbor; a few neighbors are gathered before the FMAs so
+// several rows are in flight per lane.  No per-edge value array exists:  A_hat_ij = dinv_i * dinv_j.
+// Rows longer than kLongRow are cut into kSegment-entry segments, one warp each (same launch); a row
+// of one segment is finished by that warp, the others leave partial rows that a small second kernel
+// sums in segment order -- deterministic, no floating-point atomics.
 #include <vector>
 
 #include "common.cuh"
@@ -88,45 +90,6 @@ struct SpmmParams {
     int32_t relu;
     int32_t accumulate;
 };
-
-constexpr int kU = 4;   // neighbors gathered per lane before accumulating
-
-// Accumulate neighbors [base, base+cnt) of one row; lane `sl` of the group holds colidx[base+sl].
-template <typename TI, int L, int C>
-__device__ __forceinline__ void gather_block(const SpmmParams& p, unsigned gmask, int sl, int j, float dj, int cnt,
-                                             float (&acc)[C][Vec<TI>::V]) {
-    constexpr int V = Vec<TI>::V;
-    const TI* X = static_cast<const TI*>(p.X);
-    for (int t = 0; t < cnt; t += kU) {
-        uint4 raw[kU][C];
-        float dd[kU];
-#pragma unroll
-        for (int u = 0; u < kU; ++u) {
-            const int jj = __shfl_sync(gmask, j, (t + u) & (L - 1), L);
-            dd[u] = __shfl_sync(gmask, dj, (t + u) & (L - 1), L);
-            const bool live = (t + u) < cnt;
-            if (!live) dd[u] = 0.f;
-            const TI* xr = X + (int64_t)jj * p.ldx;
-#pragma unroll
-            for (int c = 0; c < C; ++c) {
-                const int chunk = sl + c * L;
-                if (live && chunk < p.nch)
-                    raw[u][c] = __ldg(reinterpret_cast<const uint4*>(xr + chunk * V));
-                else
-                    raw[u][c] = make_uint4(0, 0, 0, 0);
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < kU; ++u)
-#pragma unroll
-            for (int c = 0; c < C; ++c) {
-                float f[V];
-                Vec<TI>::unpack(raw[u][c], f);
-#pragma unroll
-                for (int e = 0; e < V; ++e) acc[c][e] = fmaf(dd[u], f[e], acc[c][e]);
-            }
-    }
-}
 
 template <typename TO, int V, bool EPI>
 __device__ __forceinline__ void finish_chunk(const SpmmParams& p, int64_t row, int chunk, float di, float (&o)[V]) {
