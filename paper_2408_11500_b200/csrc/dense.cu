@@ -376,6 +376,25 @@ __global__ void adam_kernel(int64_t count, float* theta, const float* grad, floa
     theta[i] = th - lr * (m / c1) / (sqrtf(v / c2) + eps);
 }
 
+// Slices of X copied side by side at aligned starts: out[r, i*w_pad + c] = X[r, start_i + c] for c < w, zero for the
+// padding columns (and for the columns between p*w_pad and out_ld).  Overlapping slices get their columns twice.
+struct RepackStarts {
+    int start[SLICEGCN_MAX_SLICES];
+};
+template <typename T>
+__global__ void repack_slices_kernel(int64_t n, int p, const RepackStarts st, int w, int w_pad, const T* X, int64_t x_ld, T* out,
+                                     int64_t out_ld) {
+    const int64_t total = n * out_ld;
+    for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = e / out_ld;
+        const int c = (int)(e - r * out_ld);
+        const int i = c / w_pad, cc = c - i * w_pad;
+        T v = T(0.f);
+        if (i < p && cc < w) v = X[r * x_ld + st.start[i] + cc];
+        out[e] = v;
+    }
+}
+
 }  // namespace
 
 slicegcn_status_t gemm_run(const GemmArgs& a, cudaStream_t st) {
@@ -446,6 +465,35 @@ slicegcn_status_t wgrad_run(const WgradArgs& a, void* scratch, int64_t scratch_b
             return wgrad_run(b, scratch, scratch_bytes, st);
         }
         if (rc != SLICEGCN_ERR_UNSUPPORTED) return rc;
+        // grouped shapes the tensor-core plan does not take as one launch (slices wider than a tile, widths that
+        // need their zero padding): one launch per group
+        if (a.groups > 1) {
+            bool all = true;
+            for (int g = 0; g < a.groups && all; ++g) {
+                WgradArgs s = a;
+                s.groups = 1;
+                s.a_start[0] = a.a_start[g];
+                s.b_start[0] = a.b_start[g];
+                s.dW = a.dW + (int64_t)g * a.K * a.N;
+                s.dbias = a.dbias ? a.dbias + g * a.N : nullptr;
+                s.dbias2 = a.dbias2 ? a.dbias2 + g * a.N : nullptr;
+                bool done_g = false;
+                const slicegcn_status_t rg = tc_wgrad_run(s, scratch, scratch_bytes, st, &done_g);
+                if (rg == SLICEGCN_ERR_UNSUPPORTED) {
+                    all = false;   // same shape for every group: the first one decides, nothing was launched
+                    break;
+                }
+                if (rg != SLICEGCN_OK) return rg;
+                if (bias && !done_g) {
+                    WgradArgs b = s;
+                    b.K = 0;
+                    b.dW = nullptr;
+                    b.fault = nullptr;
+                    SGCN_TRY(wgrad_run(b, scratch, scratch_bytes, st));
+                }
+            }
+            if (all) return SLICEGCN_OK;
+        }
     }
     int n_chunks, Kext;
     int64_t rpc;
@@ -464,6 +512,23 @@ slicegcn_status_t wgrad_run(const WgradArgs& a, void* scratch, int64_t scratch_b
                                                                       a.groups, a.K, Kext, a.N, a.dW, a.dbias, a.dbias2);
     SGCN_LAUNCH_CHECK();
     count_launch(2);
+    return SLICEGCN_OK;
+}
+
+slicegcn_status_t repack_slices_run(int64_t n, int p, const int* starts, int w, int w_pad, const void* X, int64_t x_ld, int dtype,
+                                    void* out, int64_t out_ld, cudaStream_t st) {
+    RepackStarts rs;
+    for (int i = 0; i < SLICEGCN_MAX_SLICES; ++i) rs.start[i] = i < p ? starts[i] : 0;
+    const int64_t total = n * out_ld;
+    const unsigned blocks = (unsigned)std::min<int64_t>((total + 255) / 256, 148 * 32);
+    if (dtype == SLICEGCN_BF16)
+        repack_slices_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(n, p, rs, w, w_pad, static_cast<const __nv_bfloat16*>(X), x_ld,
+                                                                    static_cast<__nv_bfloat16*>(out), out_ld);
+    else
+        repack_slices_kernel<float><<<blocks, 256, 0, st>>>(n, p, rs, w, w_pad, static_cast<const float*>(X), x_ld, static_cast<float*>(out),
+                                                            out_ld);
+    SGCN_LAUNCH_CHECK();
+    count_launch();
     return SLICEGCN_OK;
 }
 

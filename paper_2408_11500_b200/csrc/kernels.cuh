@@ -117,6 +117,9 @@ slicegcn_status_t tc_wgrad_run(const WgradArgs& a, void* scratch, int64_t scratc
 slicegcn_status_t wgrad_run(const WgradArgs& a, void* scratch, int64_t scratch_bytes, cudaStream_t st);
 
 // ---- small kernels ----------------------------------------------------------------------------
+// Slices of X (p column ranges of width w at starts[]) copied side by side at multiples of w_pad, padding zeroed
+slicegcn_status_t repack_slices_run(int64_t n, int p, const int* starts, int w, int w_pad, const void* X, int64_t x_ld, int dtype,
+                                    void* out, int64_t out_ld, cudaStream_t st);
 // out = in * mask (fp32, row-major with leading dimensions)
 slicegcn_status_t mask_mul_run(int64_t M, int N, const float* in, int64_t ld_in, const uint8_t* mask, int64_t ld_mask,
                                float* out, int64_t ld_out, cudaStream_t st);

@@ -363,8 +363,8 @@ slicegcn_status_t layer_backward_impl(const slicegcn_graph* g, const slicegcn_la
         dzm.lda = dout_ld;
         dzm.a_mask = mask;
         dzm.a_mask_ld = L.mask_ld;
-        const bool in_producers = !seq && (!need_w || (dW_agg && tc_wgrad_masks_in_producer(wm))) &&
-                                  (!dH_in || tc_gemm_masks_in_producer(dzm));
+        const bool in_producers = (!need_w || (dW_agg && tc_wgrad_masks_in_producer(wm))) &&
+                                  (!dH_in || (!seq && tc_gemm_masks_in_producer(dzm)));
         if (in_producers) {
             w = wm;
             dz = dzm;
@@ -502,6 +502,19 @@ struct slicegcn_model {
     }
     int layer_in_width(int l) const { return l == 0 ? (desc.use_ff ? slice_size : slice_width) : h_s; }
     int layer_in_cols(int l) const { return l == 0 ? (desc.use_ff ? slice_size : desc.in_d) : desc.num_slices * h_s; }
+    // Direct slicing with slices that are not 8-column aligned, or that overlap (Algorithm 1's shifted last slice):
+    // the first layer reads a repacked copy of X -- slices side by side at multiples of repack_pad(), zero padding --
+    // so that every kernel sees aligned, disjoint column blocks.  The copy is remade every epoch (X is an argument).
+    bool repack_input() const {
+        if (desc.use_ff) return false;
+        bool need = slice_width % 8 != 0;
+        for (int i = 0; i < desc.num_slices; ++i) {
+            need = need || starts[i] % 8 != 0;
+            if (i > 0) need = need || starts[i] < ends[i - 1];
+        }
+        return need;
+    }
+    int repack_pad() const { return (slice_width + 7) / 8 * 8; }
     void layer_in_starts(int l, int* out) const {
         for (int i = 0; i < desc.num_slices; ++i) out[i] = l == 0 ? (desc.use_ff ? 0 : starts[i]) : i * h_s;
     }
@@ -517,6 +530,8 @@ struct EpochLayout {
     // pointers (valid when built with a base)
     void* ff_act = nullptr;
     void* xff = nullptr;
+    void* xrep = nullptr;        // repacked first-layer input (see slicegcn_model::repack_input)
+    int64_t ld_xrep = 0;
     std::vector<void*> H;        // H[l+1], l = 0..L-1
     std::vector<void*> saved;
     std::vector<int64_t> saved_bytes;
@@ -544,6 +559,12 @@ slicegcn_status_t layer_desc_for(const slicegcn_model* m, int l, const float* pa
     d->in_width = m->layer_in_width(l);
     d->in_cols = m->layer_in_cols(l);
     d->in_ld = l == 0 ? (D.use_ff ? align_up(m->slice_size, 8) : x_ld) : align_up((int64_t)D.num_slices * m->h_s, 8);
+    if (l == 0 && m->repack_input()) {   // the first layer reads the repacked copy of X
+        const int pad = m->repack_pad();
+        for (int i = 0; i < D.num_slices; ++i) starts_buf[i] = i * pad;
+        d->in_cols = D.num_slices * pad;
+        d->in_ld = (int64_t)D.num_slices * pad;
+    }
     d->h_s = m->h_s;
     d->out_ld = align_up((int64_t)D.num_slices * m->h_s, 8);
     d->dtype = D.dtype;
@@ -575,6 +596,10 @@ slicegcn_status_t build_layout(const slicegcn_model* m, const slicegcn_graph* g,
     if (D.use_ff) {
         E.ff_act = b.take(n * E.ld_ffact * esz);
         E.xff = b.take(n * E.ld_x0 * esz);
+    }
+    if (m->repack_input()) {
+        E.ld_xrep = (int64_t)p * m->repack_pad();
+        E.xrep = b.take(n * E.ld_xrep * esz);
     }
     int64_t ws_need = 0;
     E.H.resize(L);
@@ -870,6 +895,12 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
         h0 = E.xff;
         ld0 = E.ld_x0;
     }
+    const bool repacked = m->repack_input();
+    if (repacked) {   // slicing (Algorithm 2) as a copy: slices side by side at aligned starts, zero padding
+        SGCN_TRY(repack_slices_run(n, p, m->starts, m->slice_width, m->repack_pad(), X, x_ld, D.dtype, E.xrep, E.ld_xrep, st));
+        h0 = E.xrep;
+        ld0 = E.ld_xrep;
+    }
     std::vector<slicegcn_layer_desc> descs(L);
     std::vector<LayerPlan> plans(L);
     std::vector<std::vector<int>> starts(L, std::vector<int>(SLICEGCN_MAX_SLICES));
@@ -878,6 +909,11 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
         layer_desc_for(m, l, params, x_ld, starts[l].data(), &descs[l]);
         if (l == 0) descs[l].in_ld = ld0;
         SGCN_TRY(make_plan(g, &descs[l], &plans[l]));
+        if (l == 0 && repacked) {
+            // padding columns of the copy are zero, and so are those of its aggregate
+            plans[l].in_pad_zero = true;
+            if (plans[l].order == SLICEGCN_AGG_FIRST) plans[l].zt_pad_zero = true;
+        }
         if (l == 0 && D.use_ff && (m->slice_size % 8) != 0) {
             // the fused input is narrower than its leading dimension: keep the padding columns of X_ff and of
             // the saved intermediate at zero (both buffers are fully rewritten below, padding excluded)
