@@ -60,7 +60,15 @@ __global__ void __launch_bounds__(256) gemm_kernel(const GemmArgs a) {
             const int kk = e / BN, nn = e % BN;
             const int k = k0 + kk, n = n0 + nn;
             float v = 0.f;
-            if (k < a.K && n < a.N) v = a.b_trans ? __ldg(B + (int64_t)n * a.ldb + k) : __ldg(B + (int64_t)k * a.ldb + n);
+            if (k < a.K && n < a.N) {
+                const float* Bq = B;
+                int kj = k;
+                if (a.b_kstack > 0) {
+                    Bq = B + (int64_t)(k / a.b_kstack) * a.b_gstride;
+                    kj = k % a.b_kstack;
+                }
+                v = a.b_trans ? __ldg(Bq + (int64_t)n * a.ldb + kj) : __ldg(Bq + (int64_t)kj * a.ldb + n);
+            }
             Bs[kk][nn] = v;
         }
         __syncthreads();

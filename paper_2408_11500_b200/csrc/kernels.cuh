@@ -39,6 +39,9 @@ struct GemmArgs {
     int64_t b_gstride = 0;
     int ldb = 0;
     int b_trans = 0;
+    // K index stacked over several weight blocks (groups == 1 only): k = q*b_kstack + j reads element j of block q at
+    // B + q*b_gstride -- the sum over slices of dM_i W_i^T as ONE product over the concatenated dM (0: plain B)
+    int b_kstack = 0;
     void* C = nullptr;
     int64_t ldc = 0;
     int c_dtype = SLICEGCN_F32;
@@ -53,6 +56,9 @@ struct GemmArgs {
     int64_t mul_pos_ld = 0;
     int mul_pos_dtype = SLICEGCN_F32;
     int accumulate = 0;
+    // N is not a multiple of 4 but C has room up to the next one and those padding columns may be written (with zeros:
+    // the weight image has none there); only without bias / post / ReLU.  Lets the aligned kernels take odd widths.
+    int c_pad_write = 0;
     // tensor-core path: device status word (set when a bounded wait runs out) and scratch for the
     // prepared weight image (tc_image_bytes()); without both the CUDA-core kernel runs
     int* fault = nullptr;

@@ -328,6 +328,20 @@ slicegcn_status_t layer_backward_impl(const slicegcn_graph* g, const slicegcn_la
         dself.c_start[i] = L.in_starts[i];
     }
 
+    // All slices read the same input columns (fused input): the input gradient sums over the slices, which is ONE
+    // product over the concatenated slice gradients with the slices' weight blocks stacked along K.
+    bool shared_in = L.p > 1;
+    for (int i = 1; i < L.p; ++i) shared_in = shared_in && L.in_starts[i] == L.in_starts[0];
+    auto stacked = [&](GemmArgs a) {   // a: grouped product with one K block per slice -> single group, K = p * h_s
+        a.groups = 1;
+        a.K = L.p * L.h_s;
+        a.b_kstack = L.h_s;
+        a.a_start[0] = 0;
+        a.c_start[0] = L.in_starts[0];
+        a.c_pad_write = 1;   // the gradient buffers keep their rows padded to 8 columns
+        return a;
+    };
+
     if (L.order == SLICEGCN_AGG_FIRST) {
         // dM = dH * mask feeds the weight gradient, the bias gradient and dZ.  Where the tensor-core kernels
         // apply the byte mask in their producers (a mask tile travels next to every slab), dM is never
@@ -380,17 +394,22 @@ slicegcn_status_t layer_backward_impl(const slicegcn_graph* g, const slicegcn_la
             float* dZ = static_cast<float*>(b.take(L.n * L.zt_ld * 4));
             dz.C = dZ;
             dz.ldc = L.zt_ld;
-            if (seq) {
-                SGCN_CUDA(cudaMemsetAsync(dZ, 0, L.n * L.zt_ld * 4, st));
-                dz.accumulate = 1;
+            if (shared_in) {
+                SGCN_TRY(gemm_run(stacked(dz), st));
+            } else {
+                if (seq) {
+                    SGCN_CUDA(cudaMemsetAsync(dZ, 0, L.n * L.zt_ld * 4, st));
+                    dz.accumulate = 1;
+                }
+                SGCN_TRY(gemm_groups(dz, seq, st));
             }
-            SGCN_TRY(gemm_groups(dz, seq, st));
             SGCN_TRY(spmm_run(g, true, SLICEGCN_F32, SLICEGCN_F32, dZ, L.zt_ld, dH_in, din_ld, L.in_cols, nullptr, part,
                               part_bytes, st));
             if (d->W_self) {   // added by the GEMM's epilogue (an accumulating epilogue in the SpMM measured slower:
                                // its rows would wait for the old value at every row end)
                 dself.accumulate = 1;
-                SGCN_TRY(gemm_groups(dself, seq, st));
+                if (shared_in) SGCN_TRY(gemm_run(stacked(dself), st));
+                else SGCN_TRY(gemm_groups(dself, seq, st));
             }
         }
     } else {

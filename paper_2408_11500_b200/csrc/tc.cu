@@ -31,7 +31,7 @@ constexpr int kMaxPrepJobs = 40;
 struct PrepJob {            // one weight operand to convert: the B-side fields of a GemmArgs plus where the image goes
     const float* B;
     int64_t b_gstride;
-    int ldb, b_trans, K, N, n_pad, n_slabs, n_tiles, groups, bf16;
+    int ldb, b_trans, K, N, n_pad, n_slabs, n_tiles, groups, bf16, kstack;
     unsigned char* image;
     int block0;             // first block of this job in a batched launch
 };
@@ -299,7 +299,15 @@ __device__ __forceinline__ void prep_image_block(const PrepJob& j, int s, int pa
         }
         const int k = k0 + kk, col = n0 + n;
         float v = 0.f;
-        if (col < j.N && k < j.K) v = j.b_trans ? __ldg(B + (int64_t)col * j.ldb + k) : __ldg(B + (int64_t)k * j.ldb + col);
+        if (col < j.N && k < j.K) {
+            const float* Bq = B;
+            int kj = k;
+            if (j.kstack > 0) {   // K stacked over weight blocks
+                Bq = B + (int64_t)(k / j.kstack) * j.b_gstride;
+                kj = k % j.kstack;
+            }
+            v = j.b_trans ? __ldg(Bq + (int64_t)col * j.ldb + kj) : __ldg(Bq + (int64_t)kj * j.ldb + col);
+        }
         if (BF16)
             put_bf16x2(hi, lo, n, kk, v);
         else
@@ -1291,7 +1299,8 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
             const int g = e_it.g, nt = e_it.nt;
             e_it.next();
             const int n0 = nt * n_pad;
-            const int nn = min(n_pad, a.N - n0);
+            const int n_all = a.c_pad_write ? ((a.N + 3) & ~3) : a.N;   // padding columns of C are written too (zeros)
+            const int nn = min(n_pad, n_all - n0);
             const int cs = a.c_start[g] + n0;
             const int rows_here = (int)min((int64_t)32, a.M - (row0 + q * 32));   // valid rows of this warp's quarter
             const int64_t rfirst = row0 + q * 32 + sub;
@@ -1462,7 +1471,7 @@ unsigned char* cached_image(PrepJob& j, int64_t bytes, bool* fresh) {
     for (auto& e : c->entries) {
         const PrepJob& k = e.job;
         if (k.B == j.B && k.b_gstride == j.b_gstride && k.ldb == j.ldb && k.b_trans == j.b_trans && k.K == j.K && k.N == j.N &&
-            k.n_pad == j.n_pad && k.groups == j.groups && k.bf16 == j.bf16) {
+            k.n_pad == j.n_pad && k.groups == j.groups && k.bf16 == j.bf16 && k.kstack == j.kstack) {
             *fresh = e.fresh;
             e.fresh = true;   // the caller converts it now if it was not
             j.image = k.image;
@@ -1487,7 +1496,9 @@ bool ts_gemm_ok(const GemmArgs& a, int n_pad, int n_tiles) {
     const bool fused = a.A2 != nullptr;
     bool ok = ((uintptr_t)a.A % 16 == 0) && (a.lda % 4 == 0) && (a.K % 4 == 0 || a.a_pad_zero);
     for (int g = 0; g < a.groups; ++g) ok = ok && (a.a_start[g] % 4 == 0) && (a.c_start[g] % 4 == 0);
-    ok = ok && (a.N % 4 == 0) && (a.ldc % 4 == 0) && ((uintptr_t)a.C % 16 == 0);
+    const bool pad_write = a.c_pad_write && !a.bias && !a.post1 && !a.post2 && !a.relu && !a.mul_pos && a.groups == 1 &&
+                           a.c_start[0] + ((a.N + 3) & ~3) <= a.ldc;
+    ok = ok && (a.N % 4 == 0 || pad_write) && (a.ldc % 4 == 0) && ((uintptr_t)a.C % 16 == 0);
     if (a.mask_out) ok = ok && (a.mask_ld % 4 == 0) && ((uintptr_t)a.mask_out % 4 == 0);
     if (a.mul_pos) ok = ok && (a.mul_pos_ld % 4 == 0) && ((uintptr_t)a.mul_pos % 16 == 0);
     if (a.a_mask) {
@@ -1546,7 +1557,7 @@ slicegcn_status_t tc_gemm_launch(const GemmArgs& a, void* image, int64_t image_b
         configured = true;
     }
     {   // weight image(s): from the epoch's cache when there is one, else converted here into the scratch
-        PrepJob j{a.B, a.b_gstride, a.ldb, a.b_trans, a.K, a.N, n_pad, n_slabs, n_tiles, a.groups, BF16 ? 1 : 0, nullptr, 0};
+        PrepJob j{a.B, a.b_gstride, a.ldb, a.b_trans, a.K, a.N, n_pad, n_slabs, n_tiles, a.groups, BF16 ? 1 : 0, a.b_kstack, nullptr, 0};
         bool fresh = false;
         unsigned char* cimg = cached_image(j, need, &fresh);
         if (cimg) image = cimg;
@@ -1558,7 +1569,7 @@ slicegcn_status_t tc_gemm_launch(const GemmArgs& a, void* image, int64_t image_b
             count_launch();
         }
         if (fused) {
-            PrepJob j2{a.B2, a.b2_gstride, a.ldb, a.b_trans, a.K2, a.N, n_pad, n_slabs2, n_tiles, a.groups, BF16 ? 1 : 0, nullptr, 0};
+            PrepJob j2{a.B2, a.b2_gstride, a.ldb, a.b_trans, a.K2, a.N, n_pad, n_slabs2, n_tiles, a.groups, BF16 ? 1 : 0, 0, nullptr, 0};
             bool fresh2 = false;
             unsigned char* cimg2 = cached_image(j2, need2, &fresh2);
             if (cimg2) image2 = cimg2;
