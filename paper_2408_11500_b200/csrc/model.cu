@@ -71,6 +71,9 @@ struct LayerPlan {
     // set by callers that keep the padding columns (up to the leading dimension) of H_in / the saved
     // intermediate at zero: lets 16-byte loads run over widths that are not multiples of 8
     bool in_pad_zero = false, zt_pad_zero = false;
+    // backward may write zeros into the columns of dH_in between in_cols and the next multiple of 4 (internal buffers
+    // of the training step only; never set for the layer-level calls, whose dH_in belongs to the caller)
+    bool din_pad_write = false;
 };
 
 slicegcn_status_t make_plan(const slicegcn_graph* g, const slicegcn_layer_desc* d, LayerPlan* pl) {
@@ -395,6 +398,8 @@ slicegcn_status_t layer_backward_impl(const slicegcn_graph* g, const slicegcn_la
             dz.C = dZ;
             dz.ldc = L.zt_ld;
             if (shared_in) {
+                // whatever kernel takes the product, dZ's padding columns must be zero when they are aggregated below
+                if (L.din_pad_write) SGCN_CUDA(cudaMemsetAsync(dZ, 0, L.n * L.zt_ld * 4, st));
                 SGCN_TRY(gemm_run(stacked(dz), st));
             } else {
                 if (seq) {
@@ -403,7 +408,10 @@ slicegcn_status_t layer_backward_impl(const slicegcn_graph* g, const slicegcn_la
                 }
                 SGCN_TRY(gemm_groups(dz, seq, st));
             }
-            SGCN_TRY(spmm_run(g, true, SLICEGCN_F32, SLICEGCN_F32, dZ, L.zt_ld, dH_in, din_ld, L.in_cols, nullptr, part,
+            // the stacked product left zeros in dZ's padding columns: aggregating them too keeps dH_in's padding at zero
+            int sp_w = L.in_cols;
+            if (shared_in && L.din_pad_write && align_up(L.in_cols, 4) <= std::min(L.zt_ld, din_ld)) sp_w = (int)align_up(L.in_cols, 4);
+            SGCN_TRY(spmm_run(g, true, SLICEGCN_F32, SLICEGCN_F32, dZ, L.zt_ld, dH_in, din_ld, sp_w, nullptr, part,
                               part_bytes, st));
             if (d->W_self) {   // added by the GEMM's epilogue (an accumulating epilogue in the SpMM measured slower:
                                // its rows would wait for the old value at every row end)
@@ -534,6 +542,12 @@ struct slicegcn_model {
         return need;
     }
     int repack_pad() const { return (slice_width + 7) / 8 * 8; }
+    // Feature fusion reads all of X: when its rows are not 16-byte aligned (or in_d is no multiple of 8) the fusion
+    // MLP reads a copy with rows padded to 8 columns, zero padding.
+    bool repack_ff_input(int64_t x_ld) const {
+        const int64_t esz = desc.dtype == SLICEGCN_BF16 ? 2 : 4;
+        return desc.use_ff && ((x_ld * esz) % 16 != 0 || desc.in_d % 8 != 0);
+    }
     void layer_in_starts(int l, int* out) const {
         for (int i = 0; i < desc.num_slices; ++i) out[i] = l == 0 ? (desc.use_ff ? 0 : starts[i]) : i * h_s;
     }
@@ -618,6 +632,9 @@ slicegcn_status_t build_layout(const slicegcn_model* m, const slicegcn_graph* g,
     }
     if (m->repack_input()) {
         E.ld_xrep = (int64_t)p * m->repack_pad();
+        E.xrep = b.take(n * E.ld_xrep * esz);
+    } else if (m->repack_ff_input(x_ld)) {
+        E.ld_xrep = align_up(D.in_d, 8);
         E.xrep = b.take(n * E.ld_xrep * esz);
     }
     int64_t ws_need = 0;
@@ -875,6 +892,19 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
     int64_t ld0 = x_ld;
     if (D.use_ff && (m->slice_size % 8) != 0)
         SGCN_CUDA(cudaMemsetAsync(E.xff, 0, n * E.ld_x0 * esize(D.dtype), st));
+    // the hidden activation of the fusion MLP is narrower than its rows: keep the padding columns at zero so that the
+    // aligned kernels can read it (it is rewritten below, padding excluded)
+    const bool ffact_pad = D.use_ff && (D.in_d % 8) != 0;
+    if (ffact_pad) SGCN_CUDA(cudaMemsetAsync(E.ff_act, 0, n * E.ld_ffact * esize(D.dtype), st));
+    const void* xin = X;          // what the fusion MLP reads
+    int64_t xin_ld = x_ld;
+    const bool ff_repacked = m->repack_ff_input(x_ld);
+    if (ff_repacked) {
+        const int zero = 0;
+        SGCN_TRY(repack_slices_run(n, 1, &zero, D.in_d, (int)E.ld_xrep, X, x_ld, D.dtype, E.xrep, E.ld_xrep, st));
+        xin = E.xrep;
+        xin_ld = E.ld_xrep;
+    }
     if (D.use_ff) {   // X_ff = ReLU(X W1 + b1) W2 + b2  (Eq. 4 / Algorithm 3)
         GemmArgs a;
         a.fault = g->fault;
@@ -883,8 +913,9 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
         a.M = n;
         a.K = D.in_d;
         a.N = D.in_d;
-        a.A = X;
-        a.lda = x_ld;
+        a.A = xin;
+        a.lda = xin_ld;
+        a.a_pad_zero = ff_repacked ? 1 : 0;
         a.a_dtype = D.dtype;
         a.B = params + m->ff_W1;
         a.ldb = D.in_d;
@@ -903,6 +934,7 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
         c.N = m->slice_size;
         c.A = E.ff_act;
         c.lda = E.ld_ffact;
+        c.a_pad_zero = ffact_pad ? 1 : 0;
         c.a_dtype = D.dtype;
         c.B = params + m->ff_W2;
         c.ldb = m->slice_size;
@@ -933,6 +965,7 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
             plans[l].in_pad_zero = true;
             if (plans[l].order == SLICEGCN_AGG_FIRST) plans[l].zt_pad_zero = true;
         }
+        if (l == 0 && D.use_ff) plans[l].din_pad_write = true;   // dX_ff lives in the step's own gradient buffer
         if (l == 0 && D.use_ff && (m->slice_size % 8) != 0) {
             // the fused input is narrower than its leading dimension: keep the padding columns of X_ff and of
             // the saved intermediate at zero (both buffers are fully rewritten below, padding excluded)
@@ -1064,6 +1097,9 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
     }
     if (D.use_ff) {   // backward of the fusion MLP from dX_ff (sum over slices already formed)
         float* dxff = E.dH[cur];
+        // aggregate-first first layer: its backward kept the padding columns of dX_ff at zero (see din_pad_write)
+        const bool dxff_pad = plans[0].order == SLICEGCN_AGG_FIRST && p > 1 && align_up(m->slice_size, 4) <= E.ld_grad &&
+                              align_up(m->slice_size, 4) <= plans[0].zt_ld;
         WgradArgs w;
         w.fault = g->fault;
         w.M = n;
@@ -1071,9 +1107,11 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
         w.N = m->slice_size;
         w.A = E.ff_act;
         w.lda = E.ld_ffact;
+        w.a_pad_zero = ffact_pad ? 1 : 0;
         w.a_dtype = D.dtype;
         w.B = dxff;
         w.ldb = E.ld_grad;
+        w.b_pad_zero = dxff_pad ? 1 : 0;
         w.dW = grads + m->ff_W2;
         w.dbias = grads + m->ff_b2;
         SGCN_TRY(wgrad_run(w, E.ws, E.ws_bytes, st));
@@ -1087,6 +1125,7 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
         a.N = D.in_d;
         a.A = dxff;
         a.lda = E.ld_grad;
+        a.a_pad_zero = dxff_pad ? 1 : 0;
         a.B = params + m->ff_W2;
         a.ldb = m->slice_size;
         a.b_trans = 1;
@@ -1101,8 +1140,9 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
         w1.M = n;
         w1.K = D.in_d;
         w1.N = D.in_d;
-        w1.A = X;
-        w1.lda = x_ld;
+        w1.A = xin;
+        w1.lda = xin_ld;
+        w1.a_pad_zero = ff_repacked ? 1 : 0;
         w1.a_dtype = D.dtype;
         w1.B = dact;
         w1.ldb = E.ld_grad;
