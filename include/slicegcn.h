@@ -263,6 +263,13 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
                                        const slicegcn_opt_desc* opt, float* logits_out, float* loss_out,
                                        void* workspace, int64_t workspace_bytes, void* stream);
 
+/* Evaluation pass: the forward half of the iteration above (Eq. 4-9) with the current parameters; writes the logits
+ * [device, fp32 n x num_classes, dense] and nothing else a caller can see.  Same workspace as slicegcn_train_epoch.
+ * Asynchronous on `stream`.  Errors: INVALID_ARG, ALLOC, UNSUPPORTED, CUDA. */
+slicegcn_status_t slicegcn_forward_logits(const slicegcn_model* m, const slicegcn_graph* g, const void* X, int64_t x_ld,
+                                          const float* params, float* logits_out, void* workspace, int64_t workspace_bytes,
+                                          void* stream);
+
 /* The same iteration for callers whose inputs live in host memory (the paper's training loop,
  * Algorithm 3, starts from the dataset in host memory): copies the feature matrix and the labels to
  * the caller's device staging buffers, runs slicegcn_train_epoch on them, copies the loss back and

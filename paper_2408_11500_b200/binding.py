@@ -31,7 +31,7 @@ EXPORTS = [
     "slicegcn_spmm", "slicegcn_spmm_static_scratch", "slicegcn_layer_saved_bytes", "slicegcn_layer_workspace_bytes", "slicegcn_layer_forward",
     "slicegcn_layer_backward", "slicegcn_model_create", "slicegcn_model_destroy", "slicegcn_model_param_count",
     "slicegcn_model_param_elems", "slicegcn_model_num_tensors", "slicegcn_model_tensor_info", "slicegcn_model_slices",
-    "slicegcn_model_layer_order", "slicegcn_train_workspace_bytes", "slicegcn_train_epoch", "slicegcn_train_epoch_host", "slicegcn_train_epochs_host", "slicegcn_profile_begin", "slicegcn_profile_begin_sampled",
+    "slicegcn_model_layer_order", "slicegcn_train_workspace_bytes", "slicegcn_train_epoch", "slicegcn_forward_logits", "slicegcn_train_epoch_host", "slicegcn_train_epochs_host", "slicegcn_profile_begin", "slicegcn_profile_begin_sampled",
     "slicegcn_profile_end",
 ]
 
@@ -297,6 +297,11 @@ def slicegcn_train_epoch(m, g, X, x_ld: int, labels, train_idx, n_train: int, pa
                                      _vp(params), _vp(grads), _vp(adam_m), _vp(adam_v),
                                      byref(opt) if opt is not None else None, _vp(logits_out), _vp(loss_out),
                                      _vp(workspace), c_int64(workspace_bytes), _vp(stream)))
+
+
+def slicegcn_forward_logits(m, g, X, x_ld: int, params, logits_out, workspace, workspace_bytes: int, stream=None) -> None:
+    _check(_lib.slicegcn_forward_logits(m, g, _vp(X), c_int64(x_ld), _vp(params), _vp(logits_out), _vp(workspace),
+                                        c_int64(workspace_bytes), _vp(stream)))
 
 
 def slicegcn_train_epoch_host(m, g, X_host, x_ld: int, labels_host, X_stage, labels_stage, train_idx, n_train: int, params,

@@ -859,12 +859,13 @@ slicegcn_status_t slicegcn_train_workspace_bytes(const slicegcn_model* m, const 
     return SLICEGCN_OK;
 }
 
-slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_graph* g, const void* X, int64_t x_ld,
-                                       const int32_t* labels, const int32_t* train_idx, int64_t n_train, float* params,
-                                       float* grads, float* adam_m, float* adam_v, const slicegcn_opt_desc* opt,
-                                       float* logits_out, float* loss_out, void* workspace, int64_t workspace_bytes,
-                                       void* stream) {
-    if (!m || !g || !X || !labels || !params || !grads || !workspace)
+// forward_only: stops after the logits (evaluation pass); labels, grads and the optimiser arguments are not used.
+static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, const slicegcn_graph* g, const void* X, int64_t x_ld,
+                                    const int32_t* labels, const int32_t* train_idx, int64_t n_train, float* params,
+                                    float* grads, float* adam_m, float* adam_v, const slicegcn_opt_desc* opt,
+                                    float* logits_out, float* loss_out, void* workspace, int64_t workspace_bytes,
+                                    void* stream) {
+    if (!m || !g || !X || !params || !workspace || (!forward_only && (!labels || !grads)))
         SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "train_epoch: NULL argument");
     const slicegcn_model_desc& D = m->desc;
     if (x_ld < D.in_d) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "train_epoch: x_ld < in_d");
@@ -879,7 +880,7 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
     if (workspace_bytes < E.total)
         SGCN_FAIL(SLICEGCN_ERR_ALLOC, "train_epoch: workspace too small (%lld < %lld)", (long long)workspace_bytes,
                   (long long)E.total);
-    SGCN_CUDA(cudaMemsetAsync(grads, 0, sizeof(float) * m->param_elems, st));
+    if (!forward_only) SGCN_CUDA(cudaMemsetAsync(grads, 0, sizeof(float) * m->param_elems, st));
     // weight images: everything recorded by earlier epochs of this run is converted now, in one launch
     if (!m->image_cache) m->image_cache = tc_image_cache_create();
     struct CacheScope {
@@ -1017,6 +1018,7 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
         c.c_dtype = SLICEGCN_F32;
         SGCN_TRY(gemm_run(c, st));
     }
+    if (forward_only) return SLICEGCN_OK;
     // ---------------- loss (Eq. 10) and its gradient
     SGCN_TRY(softmax_ce_run(n, C, logits, labels, train_idx, n_train, E.dlogits, E.ld_dlog, E.row_loss, loss_out, st));
 
@@ -1158,6 +1160,23 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
                           (float)opt->eps, (float)opt->weight_decay, opt->epoch + 1, st));
     }
     return SLICEGCN_OK;
+}
+
+slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_graph* g, const void* X, int64_t x_ld,
+                                       const int32_t* labels, const int32_t* train_idx, int64_t n_train, float* params,
+                                       float* grads, float* adam_m, float* adam_v, const slicegcn_opt_desc* opt,
+                                       float* logits_out, float* loss_out, void* workspace, int64_t workspace_bytes,
+                                       void* stream) {
+    return epoch_impl(false, m, g, X, x_ld, labels, train_idx, n_train, params, grads, adam_m, adam_v, opt, logits_out, loss_out,
+                      workspace, workspace_bytes, stream);
+}
+
+slicegcn_status_t slicegcn_forward_logits(const slicegcn_model* m, const slicegcn_graph* g, const void* X, int64_t x_ld,
+                                          const float* params, float* logits_out, void* workspace, int64_t workspace_bytes,
+                                          void* stream) {
+    if (!logits_out) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "forward_logits: logits_out is NULL");
+    return epoch_impl(true, m, g, X, x_ld, nullptr, nullptr, 0, const_cast<float*>(params), nullptr, nullptr, nullptr, nullptr,
+                      logits_out, nullptr, workspace, workspace_bytes, stream);
 }
 
 slicegcn_status_t slicegcn_train_epoch_host(const slicegcn_model* m, const slicegcn_graph* g, const void* X_host, int64_t x_ld,

@@ -492,3 +492,29 @@ def test_profile_counts_and_sampling(B, torch):
             B.slicegcn_profile_begin_sampled(0)
     finally:
         B.slicegcn_graph_destroy(g)
+
+
+def test_forward_logits_is_the_forward_half_of_the_epoch(B, torch):
+    """The evaluation pass writes exactly the logits a training step computes before its update, touches
+    neither gradients nor parameters, and matches the oracle."""
+    src, dst, X, y, mk, od, params = small_problem(p=4, in_d=64, hidden=64, C=8, n=1111, use_ff=True, use_se=True)
+    og = orc.build_graph(len(X), src, dst, True, True)
+    gp = GpuProblem(len(X), src, dst, X, y, params, **mk)
+    try:
+        gp.epoch(None)                                   # no update: parameters stay as given
+        want = gp.logits.clone()
+        p0, g0 = gp.params.clone(), gp.grads.clone()
+        got = torch.full_like(gp.logits, float("nan"))
+        B.slicegcn_forward_logits(gp.m, gp.g, gp.X, gp.X.shape[1], gp.params, got, gp.ws, gp.ws_bytes,
+                                  torch.cuda.current_stream().cuda_stream)
+        torch.cuda.synchronize()
+        assert torch.equal(got, want)
+        assert torch.equal(gp.params, p0) and torch.equal(gp.grads, g0)
+        P = {k: v.astype(np.float64) for k, v in params.items()}
+        cache = orc.forward(od, og, X.astype(np.float64), P, y, None)
+        assert rel_inf(got.cpu().numpy(), cache["logits"]) <= TOL_F32
+        with pytest.raises(B.SliceGCNError):
+            B.slicegcn_forward_logits(gp.m, gp.g, gp.X, gp.X.shape[1], gp.params, None, gp.ws, gp.ws_bytes,
+                                      torch.cuda.current_stream().cuda_stream)
+    finally:
+        gp.close()
