@@ -209,6 +209,14 @@ __device__ __forceinline__ void tmem_ld16x2_add(uint32_t taddr0, uint32_t taddr1
     for (int i = 0; i < 16; ++i) x[OFF + i] += __uint_as_float(r[i]) + __uint_as_float(q[i]);
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+// the same for 16-bit operands (bf16): two K values per TMEM column
+__device__ __forceinline__ void umma_ts_f16(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
 // D[tmem] (+)= A[tmem] * B[smem desc], tf32: A's row i sits in TMEM lane i, its K values in consecutive columns
 __device__ __forceinline__ void umma_ts_tf32(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
     asm volatile(
@@ -1044,7 +1052,10 @@ constexpr int kTsRing = 6;     // raw slabs in flight or being read
 constexpr int kTsStages = 3;   // TMEM operand stages (with their weight images in shared memory)
 constexpr int kTsMaskPitch = 48;
 
-template <bool MASKED>   // MASKED: the activation operand is multiplied by the byte mask a.a_mask on its way to TMEM
+// MASKED: the activation operand is multiplied by the byte mask a.a_mask on its way to TMEM (fp32 only).
+// ABF16: activations stored as bf16 -- a K slab is 64 values, they go to TMEM as they are (two per column) and the
+// MMAs are kind::f16 against the bf16 hi / lo weight image: A x [B_hi | B_lo], one chain.  TC: float or bf16 result.
+template <bool MASKED, bool ABF16, typename TC>
 __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArgs a, const int n_pad, const int n_tiles, const int R,
                                                                    const unsigned char* image, const unsigned char* image2,
                                                                    int* fault, const __grid_constant__ CUtensorMap map_a,
@@ -1098,8 +1109,9 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
-    const int ns1 = (a.K + 31) / 32;                         // K slabs of the first product
-    const int ns2 = fused ? (a.K2 + 31) / 32 : 0;            // and of the second
+    constexpr int KS = ABF16 ? 64 : 32;                      // K values per slab (one 128-byte row)
+    const int ns1 = (a.K + KS - 1) / KS;                     // K slabs of the first product
+    const int ns2 = fused ? (a.K2 + KS - 1) / KS : 0;        // and of the second
     const int n_slabs = ns1 + ns2;
     const int64_t row_tiles = (a.M + 127) / 128;
     const int64_t n_items = row_tiles * a.groups * n_tiles;
@@ -1144,8 +1156,24 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
                 mw[0] = m0.x; mw[1] = m0.y; mw[2] = m0.z; mw[3] = m0.w;
                 mw[4] = m1.x; mw[5] = m1.y; mw[6] = m1.z; mw[7] = m1.w;
             }
+            if (ABF16) {   // 64 bf16 values of the row, unchanged, into 32 columns
+                uint32_t u[32];
 #pragma unroll
-            for (int half = 0; half < 2; ++half) {   // 16 K values at a time keeps the register count down
+                for (int ch = 0; ch < 8; ++ch) {
+                    const uint4 v = *reinterpret_cast<const uint4*>(slot + ((ch ^ (lane & 7)) << 4));
+                    u[4 * ch + 0] = v.x;
+                    u[4 * ch + 1] = v.y;
+                    u[4 * ch + 2] = v.z;
+                    u[4 * ch + 3] = v.w;
+                }
+                __syncwarp();
+                if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&rfree[rs])) : "memory");
+                __syncwarp();
+                tmem_st16<0>(t_hi, u);
+                tmem_st16<16>(t_hi + 16u, u);
+            }
+#pragma unroll
+            for (int half = 0; half < (ABF16 ? 0 : 2); ++half) {   // 16 K values at a time keeps the register count down
                 uint32_t h[32];                      // [0,16): hi of K 16 half..; [16,32): lo of the same
 #pragma unroll
                 for (int cc = 0; cc < 4; ++cc) {
@@ -1204,7 +1232,7 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
                 int s = l_s;
                 const bool second = s >= ns1;
                 if (second) s -= ns1;
-                const int x = (second ? a.a2_start[l_it.g] : a.a_start[l_it.g]) + s * 32;
+                const int x = (second ? a.a2_start[l_it.g] : a.a_start[l_it.g]) + s * KS;
                 const bool with_mask = masked && !second;
                 mbar_expect_tx(&rfull[rs], with_mask ? 16384u + 4096u : 16384u);
                 tma_load_2d(raw + rs * raw_slot, second ? &map_a2 : &map_a, x, (int)l_it.row0(), &rfull[rs]);
@@ -1223,8 +1251,8 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             bool okm = true;
-            const uint32_t idesc_wide = idesc_f32acc(128, 2 * n_pad, false);   // A_hi x [B_hi | B_lo]
-            const uint32_t idesc_hi = idesc_f32acc(128, n_pad, false);         // A_lo x B_hi
+            const uint32_t idesc_wide = idesc_f32acc(128, 2 * n_pad, ABF16);   // A_hi x [B_hi | B_lo]
+            const uint32_t idesc_hi = idesc_f32acc(128, n_pad, ABF16);         // A_lo x B_hi
             int ts = 0;
             uint32_t pass = 0;
             for (int64_t it = 0; it < my_items && okm; ++it) {
@@ -1241,7 +1269,20 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
                     tc_fence_after();
                     const uint32_t a_hi = tmem + a_col0 + (uint32_t)ts * 64u, a_lo = a_hi + 32u;
                     const uint64_t db = smem_desc(wring + (uint32_t)ts * slab_bytes);
-                    if (concat) {
+                    if (ABF16) {   // bf16 activations: exact, so only the weight has a lo part
+                        const uint64_t db_lo = smem_desc(wring + (uint32_t)ts * slab_bytes + n_pad * 128);
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks) {
+                            const uint64_t adv = (uint64_t)((ks * 32) >> 4);
+                            const uint32_t first = ((s == 0 || s == ns1) && ks == 0) ? 0u : 1u;
+                            if (concat) {
+                                umma_ts_f16(d_tmem, a_hi + 8u * ks, db + adv, idesc_wide, first);
+                            } else {
+                                umma_ts_f16(d_tmem, a_hi + 8u * ks, db + adv, idesc_hi, first);
+                                umma_ts_f16(d_tmem, a_hi + 8u * ks, db_lo + adv, idesc_hi, 1u);
+                            }
+                        }
+                    } else if (concat) {
 #pragma unroll
                         for (int ks = 0; ks < 4; ++ks)
                             umma_ts_tf32(d_tmem, a_hi + 8u * ks, db + (uint64_t)((ks * 32) >> 4), idesc_wide,
@@ -1281,7 +1322,8 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
         float* stage = stage_out + ew * (32 * kStagePitch);
         unsigned char* mstage = stage_mask + ew * (32 * kTsMaskPitch);
         const int cq = lane & 7, sub = lane >> 3;
-        float* Cf = static_cast<float*>(a.C);
+        float* Cf = static_cast<float*>(a.C);               // fp32 result
+        unsigned char* Cb = static_cast<unsigned char*>(a.C);   // bf16 result (no accumulation, no gate)
         const bool wmask = a.relu && a.mask_out;
         const bool has_vec = a.bias || a.post1 || a.post2;   // otherwise the staged vectors are all zero
         for (int i = tid - 256; i < a.groups * a.N; i += 256) {
@@ -1422,8 +1464,14 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
                         asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(Cf + row * a.ldc + col), "f"(t.x),
                                      "f"(t.y), "f"(t.z), "f"(t.w)
                                      : "memory");
-                    } else {
+                    } else if (sizeof(TC) == 4) {
                         *reinterpret_cast<float4*>(Cf + row * a.ldc + col) = t;
+                    } else {
+                        const __nv_bfloat162 lo2 = __floats2bfloat162_rn(t.x, t.y), hi2 = __floats2bfloat162_rn(t.z, t.w);
+                        uint2 pk;
+                        pk.x = *reinterpret_cast<const uint32_t*>(&lo2);
+                        pk.y = *reinterpret_cast<const uint32_t*>(&hi2);
+                        *reinterpret_cast<uint2*>(Cb + (row * a.ldc + col) * 2) = pk;
                     }
                 }
                 __syncwarp();
@@ -1492,10 +1540,17 @@ unsigned char* cached_image(PrepJob& j, int64_t bytes, bool* fresh) {
 // 16-byte aligned mask rows and slice starts (it travels by tensor copy next to the slab).
 bool ts_gemm_ok(const GemmArgs& a, int n_pad, int n_tiles) {
     static const bool off = getenv("SLICEGCN_NO_TS") != nullptr || getenv("SLICEGCN_NO_WS") != nullptr;
-    if (off || a.a_dtype != SLICEGCN_F32 || a.c_dtype != SLICEGCN_F32) return false;
+    const bool abf = a.a_dtype == SLICEGCN_BF16, cbf = a.c_dtype == SLICEGCN_BF16;
+    if (off || (!abf && cbf)) return false;
+    if (abf && (a.a_mask || a.accumulate || a.mul_pos || a.c_pad_write)) return false;   // forward products only
     const bool fused = a.A2 != nullptr;
-    bool ok = ((uintptr_t)a.A % 16 == 0) && (a.lda % 4 == 0) && (a.K % 4 == 0 || a.a_pad_zero);
-    for (int g = 0; g < a.groups; ++g) ok = ok && (a.a_start[g] % 4 == 0) && (a.c_start[g] % 4 == 0);
+    const int epc = abf ? 8 : 4;   // elements per 16 bytes of the activation operand
+    bool ok = ((uintptr_t)a.A % 16 == 0) && (a.lda % epc == 0) && (a.K % epc == 0 || a.a_pad_zero);
+    if (fused) ok = ok && ((uintptr_t)a.A2 % 16 == 0) && (a.lda2 % epc == 0) && (a.K2 % epc == 0 || a.a2_pad_zero);
+    for (int g = 0; g < a.groups; ++g) {
+        ok = ok && (a.a_start[g] % epc == 0) && (a.c_start[g] % 4 == 0);
+        if (fused) ok = ok && (a.a2_start[g] % epc == 0);
+    }
     const bool pad_write = a.c_pad_write && !a.bias && !a.post1 && !a.post2 && !a.relu && !a.mul_pos && a.groups == 1 &&
                            a.c_start[0] + ((a.N + 3) & ~3) <= a.ldc;
     ok = ok && (a.N % 4 == 0 || pad_write) && (a.ldc % 4 == 0) && ((uintptr_t)a.C % 16 == 0);
@@ -1519,8 +1574,7 @@ slicegcn_status_t tc_gemm_launch(const GemmArgs& a, void* image, int64_t image_b
     const bool fused = a.A2 != nullptr;
     // N = 256 in fp32: two column tiles of 128 suit the kernel with the activation operand in TMEM
     // (two accumulators and the operand stages have to share the 512 TMEM columns); same image bytes
-    if (!BF16 && std::is_same<TA, float>::value && std::is_same<TC, float>::value && !fused && a.N == 256 && a.groups * a.N <= kWsVecFloats &&
-        getenv("SLICEGCN_NO_TS") == nullptr)
+    if ((BF16 || std::is_same<TC, float>::value) && !fused && a.N == 256 && a.groups * a.N <= kWsVecFloats && getenv("SLICEGCN_NO_TS") == nullptr)
         n_pad = 128;
     const int n_tiles = (a.N + n_pad - 1) / n_pad;
     const int n_slabs = (a.K + KS - 1) / KS;
@@ -1598,9 +1652,10 @@ slicegcn_status_t tc_gemm_launch(const GemmArgs& a, void* image, int64_t image_b
     if (a.post2) cvec = cvec && ((uintptr_t)a.post2 % 16 == 0);
     (void)ces;
     const int64_t all_items = ((a.M + 127) / 128) * a.groups * n_tiles;
-    if constexpr (!BF16 && std::is_same<TA, float>::value && std::is_same<TC, float>::value) {
-        // narrow fp32 outputs (the sliced layers): the kernel that keeps the activation operand in TMEM
+    if constexpr (BF16 || std::is_same<TC, float>::value) {
+        // the kernel that keeps the activation operand in TMEM (fp32 -> fp32, bf16 -> bf16 / fp32)
         if (ts_gemm_ok(a, n_pad, n_tiles)) {
+            constexpr int eb = BF16 ? 2 : 4;       // bytes per activation element; a slab row is 128 bytes either way
             // columns the slabs may touch: up to the end of the last group (the rest reads as zeros)
             int cols1 = 0, cols2 = 0;
             for (int g = 0; g < a.groups; ++g) {
@@ -1608,8 +1663,9 @@ slicegcn_status_t tc_gemm_launch(const GemmArgs& a, void* image, int64_t image_b
                 if (fused) cols2 = std::max(cols2, a.a2_start[g] + a.K2);
             }
             CUtensorMap map_a, map_a2, map_m;
-            bool maps_ok = make_slab_map(&map_a, a.A, a.M, std::min<int64_t>(cols1, a.lda), a.lda);
-            if (maps_ok && fused) maps_ok = make_slab_map(&map_a2, a.A2, a.M, std::min<int64_t>(cols2, a.lda2), a.lda2);
+            bool maps_ok = make_slab_map(&map_a, a.A, a.M, std::min<int64_t>(cols1, a.lda), a.lda, 128 / eb, 128, true, eb);
+            if (maps_ok && fused)
+                maps_ok = make_slab_map(&map_a2, a.A2, a.M, std::min<int64_t>(cols2, a.lda2), a.lda2, 128 / eb, 128, true, eb);
             if (maps_ok && !fused) map_a2 = map_a;
             if (maps_ok && a.a_mask)
                 maps_ok = make_slab_map(&map_m, a.a_mask, a.M, std::min<int64_t>(cols1, a.a_mask_ld), a.a_mask_ld, 32, 128, false, 1);
@@ -1622,18 +1678,19 @@ slicegcn_status_t tc_gemm_launch(const GemmArgs& a, void* image, int64_t image_b
             const int ts_smem = ts_fixed + ring * raw_slot;
             static bool ts_configured = false;
             if (!ts_configured) {
-                SGCN_CUDA(cudaFuncSetAttribute(tc_gemm_ts_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
-                SGCN_CUDA(cudaFuncSetAttribute(tc_gemm_ts_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
+                SGCN_CUDA(cudaFuncSetAttribute(tc_gemm_ts_kernel<false, BF16, TC>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
+                if (!BF16)
+                    SGCN_CUDA(cudaFuncSetAttribute(tc_gemm_ts_kernel<!BF16, BF16, TC>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
                 ts_configured = true;
             }
             int64_t tgrid = 148;
             if (tgrid > all_items) tgrid = all_items;
-            if (a.a_mask)
-                tc_gemm_ts_kernel<true><<<(unsigned)tgrid, kTsThreads, ts_smem, st>>>(a, n_pad, n_tiles, ring, static_cast<unsigned char*>(image), image2,
-                                                                                      fault, map_a, map_a2, map_m);
+            if (!BF16 && a.a_mask)
+                tc_gemm_ts_kernel<!BF16, BF16, TC><<<(unsigned)tgrid, kTsThreads, ts_smem, st>>>(a, n_pad, n_tiles, ring, static_cast<unsigned char*>(image),
+                                                                                                 image2, fault, map_a, map_a2, map_m);
             else
-                tc_gemm_ts_kernel<false><<<(unsigned)tgrid, kTsThreads, ts_smem, st>>>(a, n_pad, n_tiles, ring, static_cast<unsigned char*>(image), image2,
-                                                                                       fault, map_a, map_a2, map_m);
+                tc_gemm_ts_kernel<false, BF16, TC><<<(unsigned)tgrid, kTsThreads, ts_smem, st>>>(a, n_pad, n_tiles, ring, static_cast<unsigned char*>(image),
+                                                                                                 image2, fault, map_a, map_a2, map_m);
             SGCN_LAUNCH_CHECK();
             count_launch();
             return SLICEGCN_OK;
