@@ -7,13 +7,14 @@
 // tensor memory (TMEM) and come back through tcgen05.ld for the epilogue.
 //
 // Two generations of kernels share the contracts in kernels.cuh:
-//   * tc_gemm_ts_kernel / tc_wgrad_ts_kernel (fp32): slabs arrive by tensor copy (TMA), the split
-//     activation operand is written to TMEM with tcgen05.st and the MMAs read it from there; only the
-//     small weight operand (a prepared image) or the B slab of the weight gradient is an operand tile
-//     in shared memory.
+//   * tc_gemm_ts_kernel / tc_wgrad_ts_kernel (fp32 and bf16 activations): slabs arrive by tensor copy
+//     (TMA), the activation operand (split into hi / lo when fp32) is written to TMEM with tcgen05.st
+//     and the MMAs read it from there; only the small weight operand (a prepared image) or the B slab
+//     of the weight gradient is an operand tile in shared memory.
 //   * tc_gemm_ws_kernel / tc_gemm_kernel / tc_wgrad_ws_kernel / tc_wgrad_kernel: both operands staged in
 //     shared memory in the canonical swizzled layouts that a tcgen05 matrix descriptor reads, written
-//     with ordinary stores followed by a proxy fence (bf16 activations, masked or unaligned operands).
+//     with ordinary stores followed by a proxy fence (unaligned operands, odd output widths, masks
+//     the first generation does not take).
 // Every wait on an mbarrier is bounded; a wait that runs out sets the caller's status word.
 #include <cuda.h>
 
