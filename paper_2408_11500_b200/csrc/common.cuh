@@ -65,6 +65,7 @@ struct CsrView {
     const int32_t* seg_ptr = nullptr;    // [n_long+1] first segment of each long row
     int32_t n_seg = 0;
     const int32_t* seg_row = nullptr;    // [n_seg] index into long_rows
+    const int32_t* seg_order = nullptr;  // [n_seg] segments sorted by their first column index (processing order)
     int32_t n_chunks = 0;
     const int32_t* chunk_row = nullptr;  // [n_chunks+1] first row of each chunk
 };
@@ -87,6 +88,7 @@ struct slicegcn_graph {
     int32_t* long_rows[2] = {nullptr, nullptr};
     int32_t* seg_ptr[2] = {nullptr, nullptr};
     int32_t* seg_row[2] = {nullptr, nullptr};
+    int32_t* seg_order[2] = {nullptr, nullptr};
     int32_t n_long[2] = {0, 0};
     int32_t n_seg[2] = {0, 0};
     int32_t* chunk_row[2] = {nullptr, nullptr};
@@ -102,6 +104,7 @@ struct slicegcn_graph {
         v.seg_ptr = seg_ptr[t];
         v.n_seg = n_seg[t];
         v.seg_row = seg_row[t];
+        v.seg_order = seg_order[t];
         v.n_chunks = n_chunks[t];
         v.chunk_row = chunk_row[t];
         return v;

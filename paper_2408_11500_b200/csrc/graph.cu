@@ -179,7 +179,17 @@ slicegcn_status_t rowptr_from_deg(const int32_t* deg, int64_t n, int32_t* rowptr
 }
 
 // Builds the long-row tables of one CSR pattern.
-slicegcn_status_t build_long_tables(slicegcn_graph* g, int t, const int32_t* rowptr, cudaStream_t st) {
+// key of a segment = the column index of its first entry
+__global__ void seg_first_col_kernel(const int32_t* rowptr, const int32_t* colidx, const int32_t* long_rows, const int32_t* seg_ptr,
+                                     const int32_t* seg_row, int32_t n_seg, int32_t* key, int32_t* id) {
+    const int32_t s = blockIdx.x * blockDim.x + threadIdx.x;
+    if (s >= n_seg) return;
+    const int32_t li = seg_row[s];
+    key[s] = colidx[rowptr[long_rows[li]] + (s - seg_ptr[li]) * kSegment];
+    id[s] = s;
+}
+
+slicegcn_status_t build_long_tables(slicegcn_graph* g, int t, const int32_t* rowptr, const int32_t* colidx, cudaStream_t st) {
     int64_t n = g->n;
     DevBuf ids, sel, cnt, tmp;
     SGCN_CUDA(ids.alloc(sizeof(int32_t) * n));
@@ -236,8 +246,26 @@ slicegcn_status_t build_long_tables(slicegcn_graph* g, int t, const int32_t* row
     SGCN_CUDA(sr.alloc(sizeof(int32_t) * n_seg));
     seg_fill_kernel<<<n_long, 128, 0, st>>>(sp.as<int32_t>(), n_long, sr.as<int32_t>());
     SGCN_LAUNCH_CHECK();
+    // Processing order of the segments: by first column index.  Columns are sorted inside a row, so segments that
+    // start at similar columns gather from the same stretch of the operand; run next to each other they find it in L2
+    // (in row order every long row sweeps the whole operand again).
+    DevBuf key, id, key2, so, stmp;
+    SGCN_CUDA(key.alloc(sizeof(int32_t) * n_seg));
+    SGCN_CUDA(id.alloc(sizeof(int32_t) * n_seg));
+    SGCN_CUDA(key2.alloc(sizeof(int32_t) * n_seg));
+    SGCN_CUDA(so.alloc(sizeof(int32_t) * n_seg));
+    seg_first_col_kernel<<<(n_seg + 255) / 256, 256, 0, st>>>(rowptr, colidx, lr.as<int32_t>(), sp.as<int32_t>(), sr.as<int32_t>(), n_seg,
+                                                             key.as<int32_t>(), id.as<int32_t>());
+    SGCN_LAUNCH_CHECK();
+    size_t stb = 0;
+    SGCN_CUDA(cub::DeviceRadixSort::SortPairs(nullptr, stb, key.as<int32_t>(), key2.as<int32_t>(), id.as<int32_t>(), so.as<int32_t>(), n_seg,
+                                              0, 32, st));
+    SGCN_CUDA(stmp.alloc(stb));
+    SGCN_CUDA(cub::DeviceRadixSort::SortPairs(stmp.p, stb, key.as<int32_t>(), key2.as<int32_t>(), id.as<int32_t>(), so.as<int32_t>(), n_seg,
+                                              0, 32, st));
     SGCN_CUDA(cudaStreamSynchronize(st));
     g->n_seg[t] = n_seg;
+    g->seg_order[t] = so.release<int32_t>();
     g->long_rows[t] = lr.release<int32_t>();
     g->seg_ptr[t] = sp.release<int32_t>();
     g->seg_row[t] = sr.release<int32_t>();
@@ -365,8 +393,8 @@ slicegcn_status_t create_impl(int64_t n, int64_t m, const int32_t* d_src, const 
     g->colidx = colidx.release<int32_t>();
     g->deg = deg.release<int32_t>();
     g->dinv = dinv.release<float>();
-    SGCN_TRY(build_long_tables(g, 0, g->rowptr, st));
-    if (!symmetric) SGCN_TRY(build_long_tables(g, 1, g->rowptr_t, st));
+    SGCN_TRY(build_long_tables(g, 0, g->rowptr, g->colidx, st));
+    if (!symmetric) SGCN_TRY(build_long_tables(g, 1, g->rowptr_t, g->colidx_t, st));
     SGCN_CUDA(cudaStreamSynchronize(st));
     guard.g = nullptr;
     *out = g;
@@ -487,6 +515,7 @@ slicegcn_status_t slicegcn_graph_destroy(slicegcn_graph* g) {
         cudaFree(g->long_rows[t]);
         cudaFree(g->seg_ptr[t]);
         cudaFree(g->seg_row[t]);
+        cudaFree(g->seg_order[t]);
         cudaFree(g->chunk_row[t]);
     }
     delete g;

@@ -80,6 +80,7 @@ struct SpmmParams {
     const int32_t* long_rows;
     const int32_t* seg_ptr;
     const int32_t* seg_row;
+    const int32_t* seg_order;   // processing order of the segments (by first column index)
     float* partial;  // [n_seg][nch*V]
     int32_t n_chunks;
     const int32_t* chunk_row;
@@ -276,8 +277,9 @@ __device__ __forceinline__ void spmm_segment_block(const SpmmParams& p, const in
     constexpr int V = Vec<TI>::V;
     const int lane = threadIdx.x & 31;
     const int sub = lane / L, sl = lane % L;
-    const int seg = (int)((vblock * (int64_t)blockDim.x + threadIdx.x) >> 5);
-    if (seg >= p.n_seg) return;
+    const int vseg = (int)((vblock * (int64_t)blockDim.x + threadIdx.x) >> 5);
+    if (vseg >= p.n_seg) return;
+    const int seg = __ldg(p.seg_order + vseg);
     const unsigned gmask = (L == 32) ? 0xffffffffu : (((1u << L) - 1u) << (sub * L));
     const int li = __ldg(p.seg_row + seg);
     const int row = __ldg(p.long_rows + li);
@@ -586,6 +588,7 @@ slicegcn_status_t spmm_run(const slicegcn_graph* g, bool transpose, int in_dtype
         p.long_rows = v.long_rows;
         p.seg_ptr = v.seg_ptr;
         p.seg_row = v.seg_row;
+        p.seg_order = v.seg_order;
         p.partial = static_cast<float*>(ws);
         if (v.n_seg > 0 && (!ws || ws_bytes < spmm_partial_bytes(g, width)))
             SGCN_FAIL(SLICEGCN_ERR_ALLOC, "spmm: workspace too small (%lld < %lld bytes)", (long long)ws_bytes,
