@@ -51,7 +51,7 @@ void reset_launches();
 // segment is reduced by one warp into a partial row, and the partial rows of a long row are summed
 // in a fixed order afterwards (deterministic, no floating-point atomics).
 constexpr int kLongRow = 64;
-constexpr int kSegment = 256;
+constexpr int kSegment = 128;
 // The remaining rows are dealt out in row-aligned chunks of about kChunk stored entries: chunk c
 // owns every row whose first entry index lies in [c*kChunk, (c+1)*kChunk), so each lane group gets
 // the same amount of gather work whatever the degree distribution.
