@@ -289,6 +289,8 @@ def _compare_epoch(gp, od, og, X, y, params, train_idx, tol, rnd=orc.identity, o
     dict(p=2, in_d=301, hidden=40, use_ff=True),
     dict(p=4, in_d=64, hidden=64, C=8, use_ff=True, use_se=True, n=1111),
     dict(p=2, in_d=48, hidden=256, C=12, L=2, n=900),
+    dict(p=4, in_d=64, hidden=64, C=8, n=70, m_edges=120, max_degree=30, use_ff=True, use_se=True),   # less than one tile
+    dict(p=4, in_d=64, hidden=128, C=8, n=129, m_edges=300, max_degree=60),                    # one full tile and one row
 ])
 def test_epoch_gradients_fp32(B, kw):
     kw = dict(kw)
