@@ -33,7 +33,7 @@ from paper_2408_11500_b200 import synth  # noqa: E402
 # stream ~10 us; bracketing all five calls of an epoch would add ~4 % to the step time).  7 is coprime to the 4-6 SpMM
 # calls of an epoch, so every call site is sampled equally often.
 SPMM_SAMPLE_STRIDE = 7
-NCU_SPMM_TRAFFIC_BYTES = {"citation": 920e6}   # width-256 launches (4 of the 5 per epoch)
+NCU_SPMM_TRAFFIC_BYTES = {"citation": 891e6}   # width-256 launches (4 of the 5 per epoch)
 
 
 def measured_peak_gbs():
