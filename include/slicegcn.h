@@ -256,7 +256,10 @@ slicegcn_status_t slicegcn_train_workspace_bytes(const slicegcn_model* m, const 
  *   logits_out [device, fp32 n x num_classes, dense] or NULL
  *   loss_out [device, one float] or NULL: mean cross entropy BEFORE the update
  *   workspace [device], workspace_bytes >= slicegcn_train_workspace_bytes()
- * Asynchronous on `stream`.  Errors: INVALID_ARG, ALLOC, UNSUPPORTED, CUDA. */
+ * Asynchronous on `stream`.  The model object keeps host-side bookkeeping of the converted weight operands it
+ * has placed in `workspace` (they are converted again, in one launch, at the start of every call): calls on ONE model
+ * must not run concurrently, and the contents of `workspace` are only meaningful to the library.
+ * Errors: INVALID_ARG, ALLOC, UNSUPPORTED, CUDA. */
 slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_graph* g, const void* X, int64_t x_ld,
                                        const int32_t* labels, const int32_t* train_idx, int64_t n_train,
                                        float* params, float* grads, float* adam_m, float* adam_v,
