@@ -396,3 +396,11 @@ def unpack_params(m, flat: np.ndarray) -> Dict[str, np.ndarray]:
         else:
             out[name] = data.reshape(dims[0], dims[1]).copy()
     return out
+
+
+def slicegcn_graph_degrees(g) -> np.ndarray:
+    """deg [n] alone (the CSR arrays of a large graph stay on the device)."""
+    info = slicegcn_graph_info(g)
+    deg = np.empty(info["n"], np.int32)
+    _check(_lib.slicegcn_graph_export(g, None, None, _vp(deg), None))
+    return deg

@@ -3,8 +3,8 @@
 // Row-parallel CSR kernel over row-aligned chunks of ~kChunk stored entries (common.cuh).  A group of
 // L lanes streams one chunk; each lane keeps C 16-byte chunks of the output row in registers, so one
 // 128-bit load per lane per chunk covers a neighbor's slice row.  Column indices are read coalesced
-// (L at a time) together with the neighbor's 1/sqrt(deg), parked in a per-warp shared-memory slot and
-// read back as one broadcast load per neighbor; a few neighbors are gathered before the FMAs so
+// (a batch of L or 2 L at a time) together with the neighbor's 1/sqrt(deg), parked in a per-warp shared-memory
+// slot and read back as one broadcast load per neighbor; a few neighbors are gathered before the FMAs so
 // several rows are in flight per lane.  No per-edge value array exists:  A_hat_ij = dinv_i * dinv_j.
 // Rows longer than kLongRow are cut into kSegment-entry segments, one warp each (same launch); a row
 // of one segment is finished by that warp, the others leave partial rows that a small second kernel
@@ -123,33 +123,45 @@ __device__ __forceinline__ void finish_chunk(const SpmmParams& p, int64_t row, i
 }
 
 // One lane group per row-aligned chunk of about kChunk stored entries (see common.cuh): a run of
-// short rows whose entries are contiguous.  The group streams the chunk's entries L at a time; a row
-// ends where the running entry index meets the row's end, at which point the accumulators are
-// scaled, stored and cleared.  Short rows therefore share one stream of gathers (many loads in
-// flight even for degree-1 rows) and every group does the same amount of work.  Row ends and
-// 1/sqrt(deg) of L consecutive rows are fetched by the L lanes at once and handed out by shuffles;
-// the column indices of the next batch are requested before the current batch is gathered.
+// short rows whose entries are contiguous.  The group streams the chunk's entries a batch (L or 2 L
+// entries) at a time; a row ends where the running entry index meets the row's end, at which point the
+// accumulators are scaled, stored and cleared.  Short rows therefore share one stream of gathers (many
+// loads in flight even for degree-1 rows) and every group does the same amount of work.  Row ends and
+// 1/sqrt(deg) of a batch of consecutive rows are fetched by the L lanes at once and handed out by
+// shuffles; the column indices of the next batch are requested before the current batch is gathered.
 // Chunks that consist of one long row are left to the segment kernels.
 constexpr int kRowsWarps = 1;   // warps per CTA of the row kernel: a finished warp frees its slot at once (measured best)
 // Occupancy and neighbors gathered per round.  Measured on B200: for rows of 256 bytes and more what
 // pays is resident warps (32 per SM, i.e. at most 64 registers) rather than loads per lane -- they run
-// fastest with four 16-byte loads in flight per lane; narrower rows (several rows per warp) and the
-// widest ones (three or four chunks per lane) keep eight loads per lane at 20 warps per SM.
+// fastest with four 16-byte loads in flight per lane; the widest ones (three or four chunks per lane)
+// keep eight loads per lane at 20 warps per SM.
 template <int L, int C>
-constexpr bool kDenseWarps = L >= 16 && C <= 2;
+constexpr bool kDenseWarps = C <= 2;
 template <int L, int C>
 constexpr int kGatherRound = kDenseWarps<L, C> ? (C == 2 ? 2 : 4) : ((8 / C) < 2 ? 2 : (8 / C));
 template <int L, int C>
 constexpr int kRowsBlocksPerSm = (kDenseWarps<L, C> ? 32 : 20) / kRowsWarps;
+// Column indices a lane fetches per batch: a lane group of L < 32 lanes works on batches of 2 L entries,
+// so that narrow rows (few lanes per row, several rows per warp) see full gather rounds.  (Four or
+// eight indices per lane measured 3-5x slower: the unrolled body no longer fits the instruction cache.)
+template <int L>
+constexpr int kIdxPerLane = L >= 32 ? 1 : 2;
+template <int L>
+constexpr int kBatch = kIdxPerLane<L> * L;
+// shared-memory slots per warp: (column index, 1/sqrt(deg) bits) of every group's current batch; one
+// slot of padding per group keeps the groups' broadcast reads on different banks
+template <int L>
+constexpr int kSlotStride = kBatch<L> + (L < 32 ? 1 : 0);
+template <int L>
+constexpr int kSlotsPerWarp = (32 / L) * kSlotStride<L>;
 
 template <typename TI, typename TO, int L, int C, bool EPI>
 __device__ __forceinline__ void spmm_rows_block(const SpmmParams& p, const int64_t vblock) {
     constexpr int V = Vec<TI>::V;
     constexpr int RPW = 32 / L;
+    constexpr int NB = kIdxPerLane<L>;
+    constexpr int BT = kBatch<L>;
     constexpr int U = kGatherRound<L, C>;   // neighbors gathered per round: U*C 16-byte loads per lane
-    // (column index, 1/sqrt(deg) bits) of the current batch, one slot per lane: read back as one
-    // broadcast 8-byte load per neighbor
-    __shared__ int2 nbuf[kRowsWarps][32];
     const int lane = threadIdx.x & 31;
     const int sub = lane / L, sl = lane % L;
     const int64_t warp = (vblock * (int64_t)blockDim.x + threadIdx.x) >> 5;
@@ -161,29 +173,55 @@ __device__ __forceinline__ void spmm_rows_block(const SpmmParams& p, const int64
     if (r0 >= r1) return;
     int kk = __ldg(p.rowptr + r0);             // next entry to consume
     const int k1 = __ldg(p.rowptr + r1);       // end of the chunk's entries
-    // row metadata of L rows at a time
+    // row metadata (row end, 1/sqrt(deg)) of BT rows at a time: lane sl holds rows rbase + sl + i*L
     int rbase = r0;
-    int rp_l = (r0 + sl < r1) ? __ldg(p.rowptr + r0 + sl + 1) : k1;
-    float di_l = (r0 + sl < r1) ? __ldg(p.dinv + r0 + sl) : 0.f;
+    int rp_l[NB];
+    float di_l[NB];
+    auto load_meta = [&]() {
+#pragma unroll
+        for (int i = 0; i < NB; ++i) {
+            const int r = rbase + sl + i * L;
+            rp_l[i] = (r < r1) ? __ldg(p.rowptr + r + 1) : k1;
+            di_l[i] = (r < r1) ? __ldg(p.dinv + r) : 0.f;
+        }
+    };
+    auto meta_end = [&](int idx) {   // idx is the same in every lane of the group
+        int v = rp_l[0];
+#pragma unroll
+        for (int i = 1; i < NB; ++i) v = (idx / L == i) ? rp_l[i] : v;
+        return __shfl_sync(gmask, v, idx % L, L);
+    };
+    auto meta_dinv = [&](int idx) {
+        float v = di_l[0];
+#pragma unroll
+        for (int i = 1; i < NB; ++i) v = (idx / L == i) ? di_l[i] : v;
+        return __shfl_sync(gmask, v, idx % L, L);
+    };
+    load_meta();
     int row = r0;
-    int row_end = __shfl_sync(gmask, rp_l, 0, L);
+    int row_end = meta_end(0);
     if (row_end - kk > kLongRow) return;       // a long row sits alone in its chunk
     // per-lane column pointers (lanes past the last chunk re-read it; they never store)
     const uint32_t row16 = (uint32_t)((p.ldx * (int64_t)sizeof(TI)) >> 4);
     const uint4* xl[C];
 #pragma unroll
     for (int c = 0; c < C; ++c) xl[c] = static_cast<const uint4*>(p.X) + min(sl + c * L, p.nch - 1);
-    int2* nb = &nbuf[threadIdx.x >> 5][sub * L];
+    __shared__ int2 slots[kRowsWarps][kSlotsPerWarp<L>];
+    int2* nb = &slots[threadIdx.x >> 5][sub * kSlotStride<L>];
     float acc[C][V];
 #pragma unroll
     for (int c = 0; c < C; ++c)
 #pragma unroll
         for (int e = 0; e < V; ++e) acc[c][e] = 0.f;
-    int jn = (kk + sl < k1) ? __ldg(p.colidx + kk + sl) : 0;
-    float djn = (kk + sl < k1) ? __ldg(p.dinv + jn) : 0.f;
+    int jn[NB];
+    float djn[NB];
+#pragma unroll
+    for (int i = 0; i < NB; ++i) jn[i] = (kk + sl + i * L < k1) ? __ldg(p.colidx + kk + sl + i * L) : 0;
+#pragma unroll
+    for (int i = 0; i < NB; ++i) djn[i] = (kk + sl + i * L < k1) ? __ldg(p.dinv + jn[i]) : 0.f;
 
     auto close_row = [&]() {   // scale, store and clear the finished row; step to the next one
-        const float di = __shfl_sync(gmask, di_l, row - rbase, L);
+        const float di = meta_dinv(row - rbase);
 #pragma unroll
         for (int c = 0; c < C; ++c) {
             const int ch = sl + c * L;
@@ -193,12 +231,11 @@ __device__ __forceinline__ void spmm_rows_block(const SpmmParams& p, const int64
         }
         ++row;
         if (row < r1) {
-            if (row - rbase == L) {
+            if (row - rbase == BT) {
                 rbase = row;
-                rp_l = (row + sl < r1) ? __ldg(p.rowptr + row + sl + 1) : k1;
-                di_l = (row + sl < r1) ? __ldg(p.dinv + row + sl) : 0.f;
+                load_meta();
             }
-            row_end = __shfl_sync(gmask, rp_l, row - rbase, L);
+            row_end = meta_end(row - rbase);
         } else {
             row_end = -1;   // no further row: never matches an entry index
         }
@@ -207,13 +244,16 @@ __device__ __forceinline__ void spmm_rows_block(const SpmmParams& p, const int64
     for (;;) {
         while (kk == row_end) close_row();   // rows ending here, rows without entries included
         if (row >= r1) return;
-        // one batch of up to L entries starting at kk
-        const int cnt = min(L, k1 - kk);
+        // one batch of up to BT entries starting at kk
+        const int cnt = min(BT, k1 - kk);
         __syncwarp(gmask);
-        nb[sl] = make_int2(jn, __float_as_int(djn));
+#pragma unroll
+        for (int i = 0; i < NB; ++i) nb[sl + i * L] = make_int2(jn[i], __float_as_int(djn[i]));
         __syncwarp(gmask);
         const int nk = kk + cnt;
-        if (nk + sl < k1) jn = __ldg(p.colidx + nk + sl);   // requested now, used by the next batch
+#pragma unroll
+        for (int i = 0; i < NB; ++i)   // requested now, used by the next batch
+            if (nk + sl + i * L < k1) jn[i] = __ldg(p.colidx + nk + sl + i * L);
         for (int t = 0; t < cnt;) {
             uint4 raw[U][C];
             int2 meta[U];
@@ -265,16 +305,23 @@ __device__ __forceinline__ void spmm_rows_block(const SpmmParams& p, const int64
             }
             t += U;
         }
-        if (nk + sl < k1) djn = __ldg(p.dinv + jn);   // its index has arrived by now
+#pragma unroll
+        for (int i = 0; i < NB; ++i)   // the indices have arrived by now
+            if (nk + sl + i * L < k1) djn[i] = __ldg(p.dinv + jn[i]);
     }
 }
 
-// One warp per segment of a long row; the 32/L lane groups interleave over the segment's
-// neighbors and are combined with a butterfly (fixed order).  A row that fits one segment is
+// One warp per segment of a long row; each of the 32/L lane groups takes a contiguous part of the
+// segment and the groups are combined with a butterfly (fixed order).  A row that fits one segment is
 // finished here; the others leave partial rows for the finish kernel.
 template <typename TI, typename TO, int L, int C, bool EPI>
 __device__ __forceinline__ void spmm_segment_block(const SpmmParams& p, const int64_t vblock) {
     constexpr int V = Vec<TI>::V;
+    constexpr int RPW = 32 / L;
+    constexpr int GS = kSegment / RPW;                               // entries of a segment per lane group
+    constexpr int BT = kBatch<L> < GS ? kBatch<L> : GS;              // entries per batch
+    constexpr int NB = BT / L;
+    static_assert(GS % L == 0 && BT % L == 0 && NB >= 1, "segment split");
     const int lane = threadIdx.x & 31;
     const int sub = lane / L, sl = lane % L;
     const int vseg = (int)((vblock * (int64_t)blockDim.x + threadIdx.x) >> 5);
@@ -284,10 +331,12 @@ __device__ __forceinline__ void spmm_segment_block(const SpmmParams& p, const in
     const int li = __ldg(p.seg_row + seg);
     const int row = __ldg(p.long_rows + li);
     const int start = __ldg(p.rowptr + row) + (seg - __ldg(p.seg_ptr + li)) * kSegment;
-    const int end = min(__ldg(p.rowptr + row + 1), start + kSegment);
+    const int end_seg = min(__ldg(p.rowptr + row + 1), start + kSegment);
+    int base = start + sub * GS;                                      // this group's part: [base, end)
+    const int end = min(end_seg, base + GS);
     constexpr int U = kGatherRound<L, C>;   // neighbors gathered per round
-    __shared__ int2 nbuf[kRowsWarps][32];          // (column index, 1/sqrt(deg) bits) of the current batch
-    int2* nb = &nbuf[threadIdx.x >> 5][sub * L];
+    __shared__ int2 slots[kRowsWarps][kSlotsPerWarp<L>];
+    int2* nb = &slots[threadIdx.x >> 5][sub * kSlotStride<L>];
     const uint32_t row16 = (uint32_t)((p.ldx * (int64_t)sizeof(TI)) >> 4);
     const uint4* xl[C];
 #pragma unroll
@@ -297,16 +346,22 @@ __device__ __forceinline__ void spmm_segment_block(const SpmmParams& p, const in
     for (int c = 0; c < C; ++c)
 #pragma unroll
         for (int e = 0; e < V; ++e) acc[c][e] = 0.f;
-    int base = start + sub * L;
-    int jn = (base + sl < end) ? __ldg(p.colidx + base + sl) : 0;
-    float djn = (base + sl < end) ? __ldg(p.dinv + jn) : 0.f;
-    for (; base < end; base += 32) {
-        const int cnt = min(L, end - base);
+    int jn[NB];
+    float djn[NB];
+#pragma unroll
+    for (int i = 0; i < NB; ++i) jn[i] = (base + sl + i * L < end) ? __ldg(p.colidx + base + sl + i * L) : 0;
+#pragma unroll
+    for (int i = 0; i < NB; ++i) djn[i] = (base + sl + i * L < end) ? __ldg(p.dinv + jn[i]) : 0.f;
+    for (; base < end; base += BT) {
+        const int cnt = min(BT, end - base);
         __syncwarp(gmask);
-        nb[sl] = make_int2(jn, __float_as_int(djn));
+#pragma unroll
+        for (int i = 0; i < NB; ++i) nb[sl + i * L] = make_int2(jn[i], __float_as_int(djn[i]));
         __syncwarp(gmask);
-        const int nbase = base + 32;
-        if (nbase + sl < end) jn = __ldg(p.colidx + nbase + sl);   // requested now, used by the next batch
+        const int nbase = base + BT;
+#pragma unroll
+        for (int i = 0; i < NB; ++i)   // requested now, used by the next batch
+            if (nbase + sl + i * L < end) jn[i] = __ldg(p.colidx + nbase + sl + i * L);
         int t = 0;
         for (; t + U <= cnt; t += U) {   // no row ends inside a segment: plain rounds
             uint4 raw[U][C];
@@ -353,7 +408,9 @@ __device__ __forceinline__ void spmm_segment_block(const SpmmParams& p, const in
                 }
             }
         }
-        if (nbase + sl < end) djn = __ldg(p.dinv + jn);   // its index has arrived by now
+#pragma unroll
+        for (int i = 0; i < NB; ++i)   // the indices have arrived by now
+            if (nbase + sl + i * L < end) djn[i] = __ldg(p.dinv + jn[i]);
     }
     __syncwarp();
 #pragma unroll

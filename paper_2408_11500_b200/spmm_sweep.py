@@ -1,0 +1,124 @@
+"""SpMM kernel sweep on R-MAT graphs: rates per feature width against the HBM copy peak.
+
+R-MAT (a, b, c) = (0.57, 0.19, 0.19), edge factor 16, self pairs dropped, repeats merged, symmetrized,
+self-loops added, int32 CSR; node ids as generated ("natural": hubs at low ids) and under a seeded random
+relabeling.  For every (graph, dtype, width) the aggregation Y = A_hat X runs `reps` times between CUDA
+events and three rates are printed:
+
+    algorithmic   (4 nnz + 4 (N+1) + 4 N + 2 N w e) / t     each array once -- the roofline numerator
+    gathered      nnz w e / t                                what the SMs request from L2
+    fraction      algorithmic / measured copy peak
+
+Every case is also checked at full size without a reference run: with X = sqrt(deg) in every column the
+normalized aggregation returns sqrt(deg) again (row i sums deg_i terms sqrt(deg_j) / (sqrt(deg_i) sqrt(deg_j))),
+so max |Y / sqrt(deg) - 1| must stay at rounding level.  The pattern is symmetric, so the transposed pass of
+the backward runs the same launch.
+
+    python -m paper_2408_11500_b200.spmm_sweep --scales 20,22 --widths 16,32,64,128,256,512 --dtypes f32,bf16
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import time
+
+import numpy as np
+
+
+def copy_peak_gbs() -> float:
+    path = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        return float(json.load(open(path))["hbm_gbs"])
+    return 6650.0
+
+
+def run_case(B, torch, g, info, deg_dev, width, dtype_name, reps, budget_bytes):
+    n, nnz = info["n"], info["nnz"]
+    tdt, bdt, e = (torch.float32, B.F32, 4) if dtype_name == "f32" else (torch.bfloat16, B.BF16, 2)
+    if 2 * n * width * e > budget_bytes:
+        return None
+    st = torch.cuda.current_stream()
+    wsb = B.slicegcn_spmm_workspace_bytes(g, width)
+    ws = torch.empty(max(wsb, 16), dtype=torch.uint8, device="cuda")
+    X = torch.empty(n, width, dtype=tdt, device="cuda")
+    Y = torch.empty_like(X)
+
+    def spmm():
+        B.slicegcn_spmm(g, 0, bdt, bdt, X, width, Y, width, width, ws, wsb, st.cuda_stream)
+
+    # identity check at full size
+    root = deg_dev.to(torch.float32).sqrt()
+    X.copy_(root.to(tdt)[:, None].expand(n, width))
+    spmm()
+    torch.cuda.synchronize()
+    # compare with what the kernel was given (sqrt(deg) after rounding to the storage type)
+    err = float(((Y.to(torch.float32) / X.to(torch.float32)) - 1.0).abs().max().item())
+    # timing on Gaussian features
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(width)
+    X.normal_(generator=gen)
+    for _ in range(2):
+        spmm()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(st)
+    for _ in range(reps):
+        spmm()
+    e1.record(st)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    alg = 4.0 * nnz + 4.0 * (n + 1) + 4.0 * n + 2.0 * n * width * e
+    return {"ms": ms, "alg_gbs": alg / ms / 1e6, "gather_gbs": float(nnz) * width * e / ms / 1e6, "identity_err": err}
+
+
+def main():
+    import torch
+    from . import binding as B, synth
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--scales", default="20")
+    ap.add_argument("--widths", default="16,32,64,128,256,512")
+    ap.add_argument("--dtypes", default="f32,bf16")
+    ap.add_argument("--ids", default="natural,relabeled")
+    ap.add_argument("--reps", type=int, default=10)
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--max-gb", type=float, default=100.0, help="skip cases whose X and Y together exceed this")
+    args = ap.parse_args()
+    if not torch.cuda.is_available():
+        raise SystemExit("the sweep needs a CUDA device (there is no CPU path)")
+    peak = copy_peak_gbs()
+    widths = [int(v) for v in args.widths.split(",")]
+    print(f"copy peak {peak:,.0f} GB/s; {args.reps} timed launches per case\n")
+    print("| scale | ids | N | nnz | long-row segments | dtype | width | us | algorithmic GB/s | of copy peak | gathered GB/s "
+          "| identity err |")
+    print("|---|---|---|---|---|---|---|---|---|---|---|---|")
+    for scale in (int(v) for v in args.scales.split(",")):
+        t0 = time.time()
+        n, src, dst = synth.rmat(scale, 16, seed=args.seed)
+        gen_s = time.time() - t0
+        for ids in args.ids.split(","):
+            s, d = (src, dst) if ids == "natural" else synth.random_relabel(n, src, dst, args.seed)
+            g = B.slicegcn_graph_create(n, np.ascontiguousarray(s), np.ascontiguousarray(d),
+                                        B.SYMMETRIZE | B.ADD_SELF_LOOPS)
+            try:
+                info = B.slicegcn_graph_info(g)
+                deg_dev = torch.from_numpy(B.slicegcn_graph_degrees(g)).cuda()
+                for dtype_name in args.dtypes.split(","):
+                    for width in widths:
+                        r = run_case(B, torch, g, info, deg_dev, width, dtype_name, args.reps, args.max_gb * 1e9)
+                        if r is None:
+                            continue
+                        tol = 1e-5 if dtype_name == "f32" else 1e-2
+                        flag = "" if r["identity_err"] <= tol else " (ABOVE TOLERANCE)"
+                        print(f"| {scale} | {ids} | {n:,} | {info['nnz']:,} | {info['n_segments']:,} | {dtype_name} | {width} | "
+                              f"{r['ms'] * 1e3:,.0f} | {r['alg_gbs']:,.0f} | {r['alg_gbs'] / peak:.3f} | "
+                              f"{r['gather_gbs']:,.0f} | {r['identity_err']:.1e}{flag} |", flush=True)
+                if B.slicegcn_graph_device_status(g) != 0:
+                    raise SystemExit("a bounded wait in a kernel ran out (device status word set)")
+            finally:
+                B.slicegcn_graph_destroy(g)
+        print(f"<!-- scale {scale}: edge list generated in {gen_s:.0f} s on the host -->", flush=True)
+
+
+if __name__ == "__main__":
+    main()

@@ -112,9 +112,15 @@ def rmat(scale: int, edge_factor: int = 16, a: float = 0.57, b: float = 0.19, c:
         dsts.append(v[ok].astype(np.int32))
     src, dst = np.concatenate(srcs), np.concatenate(dsts)
     if relabel:
-        perm = _rng(seed, 6).permutation(n).astype(np.int32)
-        src, dst = perm[src], perm[dst]
+        src, dst = random_relabel(n, src, dst, seed)
     return n, src, dst
+
+
+def random_relabel(n: int, src: np.ndarray, dst: np.ndarray, seed: int = 0) -> Tuple[np.ndarray, np.ndarray]:
+    """The same edge list under a seeded random permutation of the node ids (R-MAT's natural ids put the
+    hubs at low ids, which flatters locality)."""
+    perm = _rng(seed, 6).permutation(n).astype(np.int32)
+    return perm[src], perm[dst]
 
 
 # --------------------------------------------------------------------------
