@@ -134,7 +134,10 @@ constexpr int kRowsWarps = 1;   // warps per CTA of the row kernel: a finished w
 // Occupancy and neighbors gathered per round.  Measured on B200: for rows of 256 bytes and more what
 // pays is resident warps (32 per SM, i.e. at most 64 registers) rather than loads per lane -- they run
 // fastest with four 16-byte loads in flight per lane; the widest ones (three or four chunks per lane)
-// keep eight loads per lane at 20 warps per SM.
+// keep eight loads per lane at 20 warps per SM.  (One-warp CTAs cap an SM at 32 warps; two-warp CTAs
+// at 40-48 warps per SM need 40-48 registers, which this loop only reaches with spills: -5 % for
+// 512-byte fp32 rows, +4..12 % for bf16 rows -- not adopted.  Five to eight loads per lane at 28-20
+// warps per SM: 8-37 % slower.)
 template <int L, int C>
 constexpr bool kDenseWarps = C <= 2;
 template <int L, int C>

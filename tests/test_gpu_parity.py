@@ -396,7 +396,8 @@ def test_social_shape_transform_first_fp32(B):
 
 
 @pytest.mark.parametrize("relabel", [False, True])
-@pytest.mark.parametrize("dtype,width", [("f32", 16), ("f32", 64), ("f32", 512), ("bf16", 32), ("bf16", 256)])
+@pytest.mark.parametrize("dtype,width", [("f32", 8), ("f32", 16), ("f32", 32), ("f32", 64), ("f32", 128), ("f32", 512),
+                                         ("bf16", 16), ("bf16", 32), ("bf16", 64), ("bf16", 128), ("bf16", 256)])
 def test_rmat_sweep_sampled_rows_and_identity(B, torch, relabel, dtype, width):
     """SpMM sweep on an R-MAT graph (a, b, c = 0.57, 0.19, 0.19; edge factor 16): exact oracle values on a
     seeded sample of rows that includes the 100 longest, and A_hat sqrt(deg) = sqrt(deg) on every row."""
@@ -420,6 +421,24 @@ def test_rmat_sweep_sampled_rows_and_identity(B, torch, relabel, dtype, width):
             Xv = np.repeat(v[:, None], width, axis=1).astype(np.float32)
             idn, _ = _gpu_spmm(B, torch, g, Xv, width, dt)
             np.testing.assert_allclose(idn, Xv, rtol=5e-6)
+    finally:
+        B.slicegcn_graph_destroy(g)
+
+
+def test_sweep_module_case_runs_and_checks_identity(B, torch):
+    """The sweep tool's per-case routine: rates are positive and the full-size identity holds."""
+    from paper_2408_11500_b200 import spmm_sweep
+    n, src, dst = synth.rmat(14, 16, seed=1)
+    g = B.slicegcn_graph_create(n, src, dst, B.SYMMETRIZE | B.ADD_SELF_LOOPS)
+    try:
+        info = B.slicegcn_graph_info(g)
+        deg = B.slicegcn_graph_degrees(g)
+        assert deg.sum() == info["nnz"] and deg.min() >= 1
+        deg_dev = torch.from_numpy(deg).cuda()
+        for dtype, width, tol in (("f32", 32, 1e-5), ("bf16", 64, 1e-2)):
+            r = spmm_sweep.run_case(B, torch, g, info, deg_dev, width, dtype, 2, 1e9)
+            assert r["ms"] > 0 and r["alg_gbs"] > 0 and r["identity_err"] <= tol
+        assert spmm_sweep.run_case(B, torch, g, info, deg_dev, 512, "f32", 1, 1e3) is None   # over the memory budget
     finally:
         B.slicegcn_graph_destroy(g)
 
