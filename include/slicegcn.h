@@ -114,10 +114,11 @@ slicegcn_status_t slicegcn_graph_destroy(slicegcn_graph* g);
  *   Y[i, 0:width] = sum_{j in N(v_i)} X[j, 0:width] / c_ij          (transpose = 0)
  *   Y = A_hat^T X                                                    (transpose = 1, backward pass)
  * X [device, n x width, leading dimension ldx], Y [device, n x width, ldy]; X and Y must not
- * overlap.  in_dtype / out_dtype: SLICEGCN_F32 or SLICEGCN_BF16 (fp32 accumulation).
+ * overlap.  in_dtype / out_dtype: SLICEGCN_F32 or SLICEGCN_BF16 (fp32 accumulation); the pairs fp32 -> fp32,
+ * bf16 -> bf16 and bf16 -> fp32 are supported (fp32 -> bf16: UNSUPPORTED).
  * workspace [device]: at least slicegcn_spmm_workspace_bytes(g, width) bytes (partial sums of the
  * split hub rows; may be NULL when that size is 0).  Deterministic: no floating-point atomics.
- * Errors: INVALID_ARG, ALLOC (workspace too small), CUDA.
+ * Errors: INVALID_ARG, UNSUPPORTED, ALLOC (workspace too small), CUDA.
  */
 slicegcn_status_t slicegcn_spmm_workspace_bytes(const slicegcn_graph* g, int32_t width, int64_t* bytes);
 slicegcn_status_t slicegcn_spmm(const slicegcn_graph* g, int32_t transpose, int32_t in_dtype, int32_t out_dtype,

@@ -367,9 +367,15 @@ def forward(m: ModelDesc, g: Graph, x: np.ndarray, params: Dict[str, np.ndarray]
 
 
 def backward(m: ModelDesc, g: Graph, x: np.ndarray, params: Dict[str, np.ndarray], labels: np.ndarray,
-             cache: Dict[str, object], threads: int = 0, relu_margin: float = 0.0) -> Dict[str, np.ndarray]:
+             cache: Dict[str, object], threads: int = 0, relu_margin: float = 0.0,
+             rnd: Callable[[np.ndarray], np.ndarray] = identity) -> Dict[str, np.ndarray]:
     """Reverse-mode gradient of the mean cross-entropy w.r.t. every parameter
-    (storage rounding treated as identity).  ReLU'(0) = 0.
+    (the forward pass's storage rounding treated as identity).  ReLU'(0) = 0.
+
+    rnd (identity for fp32 storage, round_bf16 for bf16 storage) is applied at the one point where a
+    bf16 schedule stores an activation gradient in the storage type: dZ = dM W_agg^T of an
+    aggregate-first layer whose slices read disjoint input columns, i.e. the operand of the transposed
+    aggregation.  Every other gradient tensor stays in full precision.
 
     relu_margin (default 0 = the definition) moves the ReLU decision threshold to
     relu_margin * max|pre-activation| of each ReLU: a positive / negative margin switches every
@@ -405,6 +411,7 @@ def backward(m: ModelDesc, g: Graph, x: np.ndarray, params: Dict[str, np.ndarray
         if m.use_se and l == m.num_layers - 1:
             G["E"] = np.stack([dh[:, i * m.h_s:(i + 1) * m.h_s].sum(axis=0) for i in range(m.p)])
         m_scale = max(np.abs(c[f"M.{l}.{i}"]).max() for i in range(m.p))
+        disjoint = all(ranges[i][1] <= ranges[i + 1][0] for i in range(len(ranges) - 1))
         for i, (s, e) in enumerate(ranges):
             dhi = dh[:, i * m.h_s:(i + 1) * m.h_s]
             hin = hprev[:, s:e]
@@ -420,6 +427,8 @@ def backward(m: ModelDesc, g: Graph, x: np.ndarray, params: Dict[str, np.ndarray
             if c["order"][l] == "agg":
                 G[f"W_agg.{l}.{i}"] = c[f"Z.{l}.{i}"].T @ dm
                 dz = dm @ W.T
+                if disjoint:
+                    dz = rnd(dz)
                 dhin = dhin + spmm(g, dz, transpose=True)
             else:
                 dt = spmm(g, dm, transpose=True)
@@ -468,7 +477,7 @@ def train_epoch(m: ModelDesc, g: Graph, x, params: Dict[str, np.ndarray], labels
     opt_state holds {"m1": {...}, "m2": {...}}; params are updated in place.
     Returns (loss, logits, grads)."""
     cache = forward(m, g, x, params, labels, train_idx, rnd, order, threads)
-    grads = backward(m, g, x, params, labels, cache, threads)
+    grads = backward(m, g, x, params, labels, cache, threads, rnd=rnd)
     lr = cosine_lr(lr0, epoch, total_epochs)
     for k in params:
         m1 = opt_state["m1"].setdefault(k, np.zeros_like(params[k], dtype=np.float64))

@@ -369,6 +369,10 @@ slicegcn_status_t layer_backward_impl(const slicegcn_graph* g, const slicegcn_la
         }
         GemmArgs dz = dself;   // dZ = dM W_agg^T
         dz.B = d->W_agg;
+        // bf16 models store dZ -- the operand of the transposed aggregation, gathered deg times -- in bf16 like the
+        // activations (fp32 accumulation on both sides); the fused input's narrow dZ stays fp32
+        const bool dz_bf16 = L.dtype == SLICEGCN_BF16 && !shared_in && !seq && L.zt_ld % 8 == 0;
+        if (dz_bf16) dz.c_dtype = SLICEGCN_BF16;
         const bool need_w = dW_agg || db;
         WgradArgs wm = w;
         wm.B = dH_out;
@@ -411,8 +415,8 @@ slicegcn_status_t layer_backward_impl(const slicegcn_graph* g, const slicegcn_la
             // the stacked product left zeros in dZ's padding columns: aggregating them too keeps dH_in's padding at zero
             int sp_w = L.in_cols;
             if (shared_in && L.din_pad_write && align_up(L.in_cols, 4) <= std::min(L.zt_ld, din_ld)) sp_w = (int)align_up(L.in_cols, 4);
-            SGCN_TRY(spmm_run(g, true, SLICEGCN_F32, SLICEGCN_F32, dZ, L.zt_ld, dH_in, din_ld, sp_w, nullptr, part,
-                              part_bytes, st));
+            SGCN_TRY(spmm_run(g, true, dz_bf16 ? SLICEGCN_BF16 : SLICEGCN_F32, SLICEGCN_F32, dZ, L.zt_ld, dH_in, din_ld, sp_w,
+                              nullptr, part, part_bytes, st));
             if (d->W_self) {   // added by the GEMM's epilogue (an accumulating epilogue in the SpMM measured slower:
                                // its rows would wait for the old value at every row end)
                 dself.accumulate = 1;

@@ -113,9 +113,21 @@ __device__ __forceinline__ void finish_chunk(const SpmmParams& p, int64_t row, i
             }
         }
     }
-    if (col0 + V <= p.width && V == Vec<TO>::V) {
-        Vec<TO>::store(Y + col0, reinterpret_cast<float(&)[Vec<TO>::V]>(o));
-    } else {
+    bool stored = false;
+    if constexpr (V == Vec<TO>::V) {
+        if (col0 + V <= p.width) {
+            Vec<TO>::store(Y + col0, o);
+            stored = true;
+        }
+    } else if constexpr (V == 8 && Vec<TO>::V == 4) {   // bf16 operand, fp32 result: two 16-byte stores
+        if (col0 + V <= p.width) {
+            const float lo[4] = {o[0], o[1], o[2], o[3]}, hi[4] = {o[4], o[5], o[6], o[7]};
+            Vec<TO>::store(Y + col0, lo);
+            Vec<TO>::store(Y + col0 + 4, hi);
+            stored = true;
+        }
+    }
+    if (!stored) {
 #pragma unroll
         for (int e = 0; e < V; ++e)
             if (col0 + e < p.width) Y[col0 + e] = from_f<TO>(o[e]);
@@ -622,8 +634,10 @@ slicegcn_status_t spmm_run(const slicegcn_graph* g, bool transpose, int in_dtype
                            int64_t ws_bytes, cudaStream_t st, bool instrument) {
     if (!g || !X || !Y) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "spmm: NULL argument");
     if (width < 1 || ldx < width || ldy < width) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "spmm: bad width / leading dimension");
-    if (in_dtype != out_dtype) SGCN_FAIL(SLICEGCN_ERR_UNSUPPORTED, "spmm: input and output dtype must match");
     if (in_dtype != SLICEGCN_F32 && in_dtype != SLICEGCN_BF16) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "spmm: bad dtype");
+    if (out_dtype != SLICEGCN_F32 && out_dtype != SLICEGCN_BF16) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "spmm: bad dtype");
+    if (in_dtype == SLICEGCN_F32 && out_dtype == SLICEGCN_BF16)
+        SGCN_FAIL(SLICEGCN_ERR_UNSUPPORTED, "spmm: an fp32 operand with a bf16 result is not supported");
     const CsrView v = g->view(transpose);
     SpmmParams p{};
     p.n = g->n;
@@ -637,9 +651,10 @@ slicegcn_status_t spmm_run(const slicegcn_graph* g, bool transpose, int in_dtype
     p.width = width;
     const int V = in_dtype == SLICEGCN_F32 ? 4 : 8;
     const int64_t esz = in_dtype == SLICEGCN_F32 ? 4 : 2;
+    const int64_t osz = out_dtype == SLICEGCN_F32 ? 4 : 2;
     p.nch = (width + V - 1) / V;
     const bool vec_ok = ((uintptr_t)X % 16 == 0) && ((uintptr_t)Y % 16 == 0) && (ldx * esz) % 16 == 0 &&
-                        (ldy * esz) % 16 == 0 && (int64_t)p.nch * V <= ldx;
+                        (ldy * osz) % 16 == 0 && (int64_t)p.nch * V <= ldx;
     p.n_chunks = v.n_chunks;
     p.chunk_row = v.chunk_row;
     if (vec_ok) {
@@ -668,7 +683,7 @@ slicegcn_status_t spmm_run(const slicegcn_graph* g, bool transpose, int in_dtype
         g_prof.used += 2;
         g_prof.calls += 1;
         g_prof.bytes += 4.0 * (double)g->nnz + 4.0 * (double)(g->n + 1) + 4.0 * (double)g->n +
-                        2.0 * (double)g->n * (double)width * (double)esz;
+                        (double)g->n * (double)width * (double)(esz + osz);
     }
     bool has_epi = false;
     if (epi) {
@@ -681,7 +696,9 @@ slicegcn_status_t spmm_run(const slicegcn_graph* g, bool transpose, int in_dtype
     }
     slicegcn_status_t rc = in_dtype == SLICEGCN_F32
                                ? launch_typed<float, float>(p, vec_ok, has_epi, g->fault, st)
-                               : launch_typed<__nv_bfloat16, __nv_bfloat16>(p, vec_ok, has_epi, g->fault, st);
+                               : out_dtype == SLICEGCN_BF16
+                                     ? launch_typed<__nv_bfloat16, __nv_bfloat16>(p, vec_ok, has_epi, g->fault, st)
+                                     : launch_typed<__nv_bfloat16, float>(p, vec_ok, has_epi, g->fault, st);
     if (ev_stop) SGCN_CUDA(cudaEventRecord(ev_stop, st));
     return rc;
 }

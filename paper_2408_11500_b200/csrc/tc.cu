@@ -1542,8 +1542,9 @@ unsigned char* cached_image(PrepJob& j, int64_t bytes, bool* fresh) {
 bool ts_gemm_ok(const GemmArgs& a, int n_pad, int n_tiles) {
     static const bool off = getenv("SLICEGCN_NO_TS") != nullptr || getenv("SLICEGCN_NO_WS") != nullptr;
     const bool abf = a.a_dtype == SLICEGCN_BF16, cbf = a.c_dtype == SLICEGCN_BF16;
-    if (off || (!abf && cbf)) return false;
+    if (off) return false;
     if (abf && (a.a_mask || a.accumulate || a.mul_pos || a.c_pad_write)) return false;   // forward products only
+    if (!abf && cbf && (a.accumulate || a.mul_pos || a.c_pad_write || a.A2)) return false;   // a bf16 result is stored, never added to
     const bool fused = a.A2 != nullptr;
     const int epc = abf ? 8 : 4;   // elements per 16 bytes of the activation operand
     bool ok = ((uintptr_t)a.A % 16 == 0) && (a.lda % epc == 0) && (a.K % epc == 0 || a.a_pad_zero);
@@ -1575,7 +1576,7 @@ slicegcn_status_t tc_gemm_launch(const GemmArgs& a, void* image, int64_t image_b
     const bool fused = a.A2 != nullptr;
     // N = 256 in fp32: two column tiles of 128 suit the kernel with the activation operand in TMEM
     // (two accumulators and the operand stages have to share the 512 TMEM columns); same image bytes
-    if ((BF16 || std::is_same<TC, float>::value) && !fused && a.N == 256 && a.groups * a.N <= kWsVecFloats && getenv("SLICEGCN_NO_TS") == nullptr)
+    if (!fused && a.N == 256 && a.groups * a.N <= kWsVecFloats && getenv("SLICEGCN_NO_TS") == nullptr)
         n_pad = 128;
     const int n_tiles = (a.N + n_pad - 1) / n_pad;
     const int n_slabs = (a.K + KS - 1) / KS;
@@ -1653,8 +1654,8 @@ slicegcn_status_t tc_gemm_launch(const GemmArgs& a, void* image, int64_t image_b
     if (a.post2) cvec = cvec && ((uintptr_t)a.post2 % 16 == 0);
     (void)ces;
     const int64_t all_items = ((a.M + 127) / 128) * a.groups * n_tiles;
-    if constexpr (BF16 || std::is_same<TC, float>::value) {
-        // the kernel that keeps the activation operand in TMEM (fp32 -> fp32, bf16 -> bf16 / fp32)
+    {
+        // the kernel that keeps the activation operand in TMEM (fp32 -> fp32 / bf16, bf16 -> bf16 / fp32)
         if (ts_gemm_ok(a, n_pad, n_tiles)) {
             constexpr int eb = BF16 ? 2 : 4;       // bytes per activation element; a slab row is 128 bytes either way
             // columns the slabs may touch: up to the end of the last group (the rest reads as zeros)

@@ -123,6 +123,37 @@ def test_spmm_matches_oracle(B, torch, width, ld_pad, dtype):
         B.slicegcn_graph_destroy(g)
 
 
+@pytest.mark.parametrize("width,ld_pad", [(8, 0), (13, 3), (64, 0), (100, 4), (256, 0), (300, 4), (1100, 4)])
+def test_spmm_bf16_operand_fp32_result(B, torch, width, ld_pad):
+    """The pair the backward pass of bf16 models uses: bf16 operand gathered, fp32 result (no rounding of
+    the result); fp32 operand with bf16 result is refused."""
+    n = 5000
+    src, dst = synth.chung_lu_powerlaw(n, 30000, 2.2, 1500, seed=1)
+    og = orc.build_graph(n, src, dst, True, True)
+    g = B.slicegcn_graph_create(n, src, dst, B.SYMMETRIZE | B.ADD_SELF_LOOPS)
+    try:
+        X = synth.gaussian_features(n, width, seed=width)
+        ldx = width + ld_pad + (-(width + ld_pad)) % 8
+        ldy = width + ld_pad
+        xd = torch.zeros((n, ldx), dtype=torch.bfloat16, device="cuda")
+        xd[:, :width] = torch.from_numpy(X).cuda().to(torch.bfloat16)
+        yd = torch.full((n, ldy), float("nan"), dtype=torch.float32, device="cuda")
+        wsb = B.slicegcn_spmm_workspace_bytes(g, width)
+        ws = torch.empty(max(wsb, 16), dtype=torch.uint8, device="cuda")
+        st = torch.cuda.current_stream().cuda_stream
+        B.slicegcn_spmm(g, 1, B.BF16, B.F32, xd, ldx, yd, ldy, width, ws, wsb, st)
+        torch.cuda.synchronize()
+        out = yd.cpu().numpy()
+        assert np.isnan(out[:, width:]).all() if ld_pad else True
+        want = orc.spmm(og, xd[:, :width].float().cpu().numpy().astype(np.float64), transpose=True)
+        assert rel_inf(out[:, :width], want) <= 2e-6
+        with pytest.raises(B.SliceGCNError) as e:
+            B.slicegcn_spmm(g, 0, B.F32, B.BF16, yd, ldy, xd, ldx, width, ws, wsb, st)
+        assert e.value.status == B.ERR_UNSUPPORTED
+    finally:
+        B.slicegcn_graph_destroy(g)
+
+
 def test_spmm_transposed_on_directed_graph(B, torch):
     rng = np.random.default_rng(3)
     n = 4000
@@ -258,11 +289,11 @@ def _compare_epoch(gp, od, og, X, y, params, train_idx, tol, rnd=orc.identity, o
     do not depend on any such decision and keep the plain tolerance."""
     P = {k: v.astype(np.float64) for k, v in params.items()}
     cache = orc.forward(od, og, X, P, y, train_idx, rnd=rnd, order=orders)
-    G = orc.backward(od, og, X, P, y, cache)
+    G = orc.backward(od, og, X, P, y, cache, rnd=rnd)
     spread = None
     if relu_margin > 0:
-        lo = orc.backward(od, og, X, P, y, cache, relu_margin=relu_margin)
-        hi = orc.backward(od, og, X, P, y, cache, relu_margin=-relu_margin)
+        lo = orc.backward(od, og, X, P, y, cache, relu_margin=relu_margin, rnd=rnd)
+        hi = orc.backward(od, og, X, P, y, cache, relu_margin=-relu_margin, rnd=rnd)
         spread = {k: np.abs(hi[k] - lo[k]) for k in P}
     loss = gp.epoch(None)
     errs = {"logits": rel_inf(gp.logits.cpu().numpy(), cache["logits"]), "loss": abs(loss - cache["loss"]) / abs(cache["loss"])}

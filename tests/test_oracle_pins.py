@@ -360,6 +360,33 @@ def test_backward_matches_finite_differences(kw, order):
             assert abs(fd - an) <= 1e-6 * max(1.0, abs(fd)) + 1e-8, (name, k, fd, an)
 
 
+def test_backward_storage_rounding_acts_only_on_disjoint_aggregate_first_layers():
+    """The bf16 rounding point of the backward pass (dZ of aggregate-first layers with disjoint slices):
+    it changes nothing where it must not apply (transform-first layers, a shared fused input, the layers
+    above it), and where it applies the change is bounded by the rounding (2^-8 relative per element)."""
+    g, m, X, y, P = _tiny_problem(p=2, L=2)
+    c = orc.forward(m, g, X, P, y, order=["agg", "agg"])
+    ref = orc.backward(m, g, X, P, y, c)
+    rb = orc.backward(m, g, X, P, y, c, rnd=orc.round_bf16)
+    # only what lies below the rounded dZ of layer 1 (the gradients of layer 0) may move
+    for k in ref:
+        if k.endswith(".1.0") or k.endswith(".1.1") or k in ("Wc1", "bc1", "Wc2", "bc2"):
+            assert np.array_equal(ref[k], rb[k]), k
+    moved = [k for k in ref if not np.array_equal(ref[k], rb[k])]
+    assert any(k.startswith("W_agg.0") for k in moved) and "H0" in moved
+    for k in moved:
+        assert np.abs(rb[k] - ref[k]).max() <= 2.0 ** -7 * np.abs(ref[k]).max(), k
+    # transform-first: no dZ exists, nothing is rounded
+    cx = orc.forward(m, g, X, P, y, order=["xform", "xform"])
+    gx, gxr = orc.backward(m, g, X, P, y, cx), orc.backward(m, g, X, P, y, cx, rnd=orc.round_bf16)
+    assert all(np.array_equal(gx[k], gxr[k]) for k in gx)
+    # shared fused input: layer 0 is excluded, layer 1 (disjoint slices of H1) is not
+    g2, m2, X2, y2, P2 = _tiny_problem(p=3, in_d=10, hidden=6, use_ff=True, L=1)
+    c2 = orc.forward(m2, g2, X2, P2, y2, order=["agg"])
+    a, b = orc.backward(m2, g2, X2, P2, y2, c2), orc.backward(m2, g2, X2, P2, y2, c2, rnd=orc.round_bf16)
+    assert all(np.array_equal(a[k], b[k]) for k in a)
+
+
 def test_order_of_aggregate_and_transform_is_immaterial():
     g, m, X, y, P = _tiny_problem(p=2, use_se=True)
     a = orc.forward(m, g, X, P, y, order=["agg", "agg"])
