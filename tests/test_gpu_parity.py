@@ -380,6 +380,27 @@ def test_epoch_bf16_storage(B):
         gp.close()
 
 
+def test_epoch_bf16_copurchase_shape(B):
+    """The co-purchase configuration's own widths at reduced node count (100 bf16 features, fusion MLP and
+    slice encoding on, hidden 256 in 8 slices of 32, 47 classes): the slices start on 32-column boundaries, so
+    the tensor-core kernels apply the ReLU byte mask in their producers and dZ is stored in bf16 by the
+    masked product -- the launch configuration of the full-size workload."""
+    src, dst, X, y, mk, od, params = small_problem(n=2600, m_edges=40000, max_degree=900, in_d=100, hidden=256, L=3,
+                                                   C=47, p=8, use_ff=True, use_se=True)
+    mk["dtype"] = B.BF16
+    Xr = orc.round_bf16(X)
+    og = orc.build_graph(len(X), src, dst, True, True)
+    assert (og.deg > 128).sum() >= 3          # rows of several segments
+    gp = GpuProblem(len(X), src, dst, X, y, params, **mk)
+    try:
+        orders = [{1: "agg", 2: "xform"}[B.slicegcn_model_layer_order(gp.m, l)] for l in range(3)]
+        assert orders == ["agg", "agg", "agg"]
+        _compare_epoch(gp, od, og, Xr, y, params, None, TOL_BF16, rnd=orc.round_bf16, orders=orders)
+        assert B.slicegcn_graph_device_status(gp.g) == 0
+    finally:
+        gp.close()
+
+
 def test_citation_workload_full_size_fp32(B):
     """The benchmark workload at full size (169,343 nodes, 3 layers, hidden 256, 8 slices), in the
     launch configuration bench.py times: one epoch, every logit and gradient against the oracle."""
