@@ -461,6 +461,34 @@ slicegcn_status_t wgrad_run(const WgradArgs& a, void* scratch, int64_t scratch_b
             return SLICEGCN_OK;
         }
     }
+    // one group wider than a tensor-core tile (256 result columns): column blocks of dW, one launch each
+    if (!no_tc && a.fault && a.K >= 1 && a.dW && a.groups == 1 && a.N > 256 && a.N % 4 == 0 && a.ldw == 0) {
+        bool all = true;
+        for (int c0 = 0; c0 < a.N; c0 += 256) {
+            WgradArgs s = a;
+            s.N = std::min(256, a.N - c0);
+            s.b_start[0] = a.b_start[0] + c0;
+            s.dW = a.dW + c0;
+            s.ldw = a.N;
+            s.dbias = a.dbias ? a.dbias + c0 : nullptr;
+            s.dbias2 = a.dbias2 ? a.dbias2 + c0 : nullptr;
+            bool done_c = false;
+            const slicegcn_status_t rc = tc_wgrad_run(s, scratch, scratch_bytes, st, &done_c);
+            if (rc == SLICEGCN_ERR_UNSUPPORTED && c0 == 0) {
+                all = false;   // nothing was launched: the general path below takes the whole product
+                break;
+            }
+            if (rc != SLICEGCN_OK) return rc;
+            if (bias && !done_c) {
+                WgradArgs b = s;
+                b.K = 0;
+                b.dW = nullptr;
+                b.fault = nullptr;
+                SGCN_TRY(wgrad_run(b, scratch, scratch_bytes, st));
+            }
+        }
+        if (all) return SLICEGCN_OK;
+    }
     if (!no_tc && a.fault && a.K >= 1 && a.dW) {
         bool bias_done = false;
         const slicegcn_status_t rc = tc_wgrad_run(a, scratch, scratch_bytes, st, &bias_done);
@@ -503,6 +531,7 @@ slicegcn_status_t wgrad_run(const WgradArgs& a, void* scratch, int64_t scratch_b
             if (all) return SLICEGCN_OK;
         }
     }
+    if (a.ldw != 0 && a.ldw != a.N) SGCN_FAIL(SLICEGCN_ERR_UNSUPPORTED, "wgrad: a column block of dW needs the tensor-core path");
     int n_chunks, Kext;
     int64_t rpc;
     wgrad_plan(a.M, a.groups, a.K, a.N, bias, &n_chunks, &rpc, &Kext);

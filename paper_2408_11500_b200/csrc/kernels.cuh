@@ -111,6 +111,7 @@ struct WgradArgs {
     int a_pad_zero = 0;        // A / B columns up to the next multiple of 4 past the last group exist and hold zeros
     int b_pad_zero = 0;
     float* dW = nullptr;       // may be NULL when K == 0
+    int64_t ldw = 0;           // leading dimension of a group's K x N block of dW (0: N, dense)
     float* dbias = nullptr;    // may be NULL
     float* dbias2 = nullptr;   // optional second copy of the column sums (slice-encoding gradient)
     int* fault = nullptr;      // device status word; NULL: CUDA-core path

@@ -2411,7 +2411,7 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
 // Blocks past the dW elements (when colsum != NULL) reduce the column-sum partials into dbias / dbias2 the same way.
 __global__ void __launch_bounds__(256) tc_wgrad_reduce_kernel(const float* scratch, const WgTcPlan pl, int groups, int K, int N,
                                                               int groups_per_tile, float* dW, const float* colsum = nullptr,
-                                                              float* dbias = nullptr, float* dbias2 = nullptr) {
+                                                              float* dbias = nullptr, float* dbias2 = nullptr, int64_t ldw = 0) {
     __shared__ float part[8][32];
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const int64_t total = (int64_t)groups * K * N;
@@ -2445,9 +2445,11 @@ __global__ void __launch_bounds__(256) tc_wgrad_reduce_kernel(const float* scrat
     }
     const int64_t i = blockIdx.x * (int64_t)32 + lane;
     float s = 0.f;
+    int64_t o = i;                  // where element i goes: rows of ldw floats when dW is a column block of a wider matrix
     if (i < total) {
         const int g = (int)(i / ((int64_t)K * N));
         const int k = (int)((i / N) % K), n = (int)(i % N);
+        if (ldw > 0) o = ((int64_t)g * K + k) * ldw + n;
         int mt, f, c;
         if (groups_per_tile > 0) {   // grouped: tile mt holds groups mt*gpt .. ; block (g % gpt)
             mt = g / groups_per_tile;
@@ -2481,7 +2483,7 @@ __global__ void __launch_bounds__(256) tc_wgrad_reduce_kernel(const float* scrat
         float t = part[0][lane];
 #pragma unroll
         for (int q = 1; q < 8; ++q) t += part[q][lane];
-        dW[i] = t;
+        dW[o] = t;
     }
 }
 
@@ -2691,7 +2693,7 @@ slicegcn_status_t tc_wgrad_run(const WgradArgs& a, void* scratch, int64_t scratc
                     const int64_t total_w = (int64_t)a.groups * a.K * a.N;
                     const unsigned red_blocks = (unsigned)((total_w + 31) / 32) + (want_bias ? (unsigned)((b_total + 31) / 32) : 0u);
                     tc_wgrad_reduce_kernel<<<red_blocks, 256, 0, st>>>(static_cast<const float*>(scratch), pn, a.groups, a.K, a.N, gn, a.dW,
-                                                                         colsum, a.dbias, a.dbias2);
+                                                                         colsum, a.dbias, a.dbias2, a.ldw);
                     SGCN_LAUNCH_CHECK();
                     if (want_bias && bias_done) *bias_done = true;
                     count_launch(2);
@@ -2723,7 +2725,7 @@ slicegcn_status_t tc_wgrad_run(const WgradArgs& a, void* scratch, int64_t scratc
                 SGCN_LAUNCH_CHECK();
                 const int64_t total_w = (int64_t)a.groups * a.K * a.N;
                 tc_wgrad_reduce_kernel<<<(unsigned)((total_w + 31) / 32), 256, 0, st>>>(static_cast<const float*>(scratch), pw,
-                                                                                         a.groups, a.K, a.N, gw, a.dW);
+                                                                                         a.groups, a.K, a.N, gw, a.dW, nullptr, nullptr, nullptr, a.ldw);
                 SGCN_LAUNCH_CHECK();
                 count_launch(2);
                 return SLICEGCN_OK;
@@ -2748,7 +2750,7 @@ slicegcn_status_t tc_wgrad_run(const WgradArgs& a, void* scratch, int64_t scratc
     SGCN_LAUNCH_CHECK();
     const int64_t total = (int64_t)a.groups * a.K * a.N;
     tc_wgrad_reduce_kernel<<<(unsigned)((total + 31) / 32), 256, 0, st>>>(static_cast<const float*>(scratch), pl, a.groups,
-                                                                           a.K, a.N, gpt, a.dW);
+                                                                           a.K, a.N, gpt, a.dW, nullptr, nullptr, nullptr, a.ldw);
     SGCN_LAUNCH_CHECK();
     count_launch(2);
     return SLICEGCN_OK;

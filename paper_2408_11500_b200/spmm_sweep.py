@@ -2,8 +2,9 @@
 
 R-MAT (a, b, c) = (0.57, 0.19, 0.19), edge factor 16, self pairs dropped, repeats merged, symmetrized,
 self-loops added, int32 CSR; node ids as generated ("natural": hubs at low ids) and under a seeded random
-relabeling.  For every (graph, dtype, width) the aggregation Y = A_hat X runs `reps` times between CUDA
-events and three rates are printed:
+relabeling.  For every (graph, dtype, width) the aggregation Y = A_hat X runs `reps` times, each launch between
+its own pair of CUDA events, back to back and with L2 flushed before every launch; the median, the minimum and the
+flushed median are printed, and three rates from the median:
 
     algorithmic   (4 nnz + 4 (N+1) + 4 N + 2 N w e) / t     each array once -- the roofline numerator
     gathered      nnz w e / t                                what the SMs request from L2
@@ -33,7 +34,7 @@ def copy_peak_gbs() -> float:
     return 6650.0
 
 
-def run_case(B, torch, g, info, deg_dev, width, dtype_name, reps, budget_bytes):
+def run_case(B, torch, g, info, deg_dev, width, dtype_name, reps, budget_bytes, flush_buf=None):
     n, nnz = info["n"], info["nnz"]
     tdt, bdt, e = (torch.float32, B.F32, 4) if dtype_name == "f32" else (torch.bfloat16, B.BF16, 2)
     if 2 * n * width * e > budget_bytes:
@@ -58,22 +59,32 @@ def run_case(B, torch, g, info, deg_dev, width, dtype_name, reps, budget_bytes):
     for r in range(0, n, step):
         q = Y[r:r + step].to(torch.float32) / X[r:r + step].to(torch.float32) - 1.0
         err = max(err, float(q.abs().max().item()))
-    # timing on Gaussian features
+    # timing on Gaussian features: every launch between its own pair of events; back to back ("warm": whatever
+    # the previous launch left in L2 stays) and with L2 flushed before each launch (a write larger than L2)
     gen = torch.Generator(device="cuda")
     gen.manual_seed(width)
     X.normal_(generator=gen)
-    for _ in range(2):
+    for _ in range(3):
         spmm()
     torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(st)
-    for _ in range(reps):
-        spmm()
-    e1.record(st)
-    torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1) / reps
+
+    def timed(flush):
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+        for a, b in ev:
+            if flush is not None:
+                flush.zero_()
+            a.record(st)
+            spmm()
+            b.record(st)
+        torch.cuda.synchronize()
+        return sorted(a.elapsed_time(b) for a, b in ev)
+
+    warm = timed(None)
+    cold = timed(flush_buf) if flush_buf is not None else warm
+    ms = warm[len(warm) // 2]
     alg = 4.0 * nnz + 4.0 * (n + 1) + 4.0 * n + 2.0 * n * width * e
-    return {"ms": ms, "alg_gbs": alg / ms / 1e6, "gather_gbs": float(nnz) * width * e / ms / 1e6, "identity_err": err}
+    return {"ms": ms, "ms_min": warm[0], "ms_flushed": cold[len(cold) // 2], "alg_gbs": alg / ms / 1e6,
+            "gather_gbs": float(nnz) * width * e / ms / 1e6, "identity_err": err}
 
 
 def main():
@@ -84,7 +95,7 @@ def main():
     ap.add_argument("--widths", default="16,32,64,128,256,512")
     ap.add_argument("--dtypes", default="f32,bf16")
     ap.add_argument("--ids", default="natural,relabeled")
-    ap.add_argument("--reps", type=int, default=10)
+    ap.add_argument("--reps", type=int, default=10, help="timed launches per case (median reported)")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--max-gb", type=float, default=100.0, help="skip cases whose X and Y together exceed this")
     args = ap.parse_args()
@@ -92,10 +103,11 @@ def main():
         raise SystemExit("the sweep needs a CUDA device (there is no CPU path)")
     peak = copy_peak_gbs()
     widths = [int(v) for v in args.widths.split(",")]
-    print(f"copy peak {peak:,.0f} GB/s; {args.reps} timed launches per case\n")
-    print("| scale | ids | N | nnz | long-row segments | dtype | width | us | algorithmic GB/s | of copy peak | gathered GB/s "
-          "| identity err |")
-    print("|---|---|---|---|---|---|---|---|---|---|---|---|")
+    flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")     # twice the L2
+    print(f"copy peak {peak:,.0f} GB/s; 3 warm-up and {args.reps} timed launches per case (median; rates from the median)\n")
+    print("| scale | ids | N | nnz | long-row segments | dtype | width | us (median) | us (min) | us (L2 flushed) | "
+          "algorithmic GB/s | of copy peak | gathered GB/s | identity err |")
+    print("|---|---|---|---|---|---|---|---|---|---|---|---|---|---|")
     for scale in (int(v) for v in args.scales.split(",")):
         t0 = time.time()
         n, src, dst = synth.rmat(scale, 16, seed=args.seed)
@@ -109,13 +121,14 @@ def main():
                 deg_dev = torch.from_numpy(B.slicegcn_graph_degrees(g)).cuda()
                 for dtype_name in args.dtypes.split(","):
                     for width in widths:
-                        r = run_case(B, torch, g, info, deg_dev, width, dtype_name, args.reps, args.max_gb * 1e9)
+                        r = run_case(B, torch, g, info, deg_dev, width, dtype_name, args.reps, args.max_gb * 1e9, flush_buf)
                         if r is None:
                             continue
                         tol = 1e-5 if dtype_name == "f32" else 1e-2
                         flag = "" if r["identity_err"] <= tol else " (ABOVE TOLERANCE)"
                         print(f"| {scale} | {ids} | {n:,} | {info['nnz']:,} | {info['n_segments']:,} | {dtype_name} | {width} | "
-                              f"{r['ms'] * 1e3:,.0f} | {r['alg_gbs']:,.0f} | {r['alg_gbs'] / peak:.3f} | "
+                              f"{r['ms'] * 1e3:,.0f} | {r['ms_min'] * 1e3:,.0f} | {r['ms_flushed'] * 1e3:,.0f} | "
+                              f"{r['alg_gbs']:,.0f} | {r['alg_gbs'] / peak:.3f} | "
                               f"{r['gather_gbs']:,.0f} | {r['identity_err']:.1e}{flag} |", flush=True)
                 if B.slicegcn_graph_device_status(g) != 0:
                     raise SystemExit("a bounded wait in a kernel ran out (device status word set)")

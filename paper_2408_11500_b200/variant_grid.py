@@ -13,11 +13,15 @@ import argparse
 import numpy as np
 
 
-def time_variant(B, torch, g, w, X, y, p, use_ff, use_se, use_self, epochs, warmup=3):
+def time_variant(B, torch, g, w, X, y, p, use_ff, use_se, use_self, epochs, warmup=3, table3=False):
     from . import synth
     dev = X.device
+    # table3: the shapes behind the paper's parameter counts (Table III): slices of floor(d'/p) + 1 columns and a
+    # second bias vector per layer
     m = B.slicegcn_model_create(in_d=w["in_d"], hidden=w["hidden"], num_layers=w["layers"], num_classes=w["classes"],
                                 num_slices=p, use_ff=use_ff, use_se=use_se, use_self=use_self,
+                                slice_rule=B.RULE_FLOOR_PLUS_1 if (table3 and p > 1) else B.RULE_CEIL,
+                                use_b_self=bool(table3 and use_self),
                                 dtype=B.BF16 if X.dtype == torch.bfloat16 else B.F32)
     try:
         params = torch.from_numpy(B.pack_params(m, synth.init_params(B.named_param_shapes(m), 0))).to(dev)
@@ -54,8 +58,16 @@ def main():
     ap.add_argument("--workload", default="citation", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--epochs", type=int, default=20)
     ap.add_argument("--slices", default="2,4,8")
+    ap.add_argument("--hidden", type=int, default=0, help="override the workload's hidden width (the paper's Table III uses 512)")
+    ap.add_argument("--layers", type=int, default=0, help="override the number of layers (the paper goes up to 7)")
+    ap.add_argument("--table3-shapes", action="store_true",
+                    help="slices of floor(d'/p) + 1 columns and two bias vectors per layer, as the paper's parameter counts imply")
     args = ap.parse_args()
-    w = synth.WORKLOADS[args.workload]
+    w = dict(synth.WORKLOADS[args.workload])
+    if args.hidden:
+        w["hidden"] = args.hidden
+    if args.layers:
+        w["layers"] = args.layers
     src, dst = synth.make_graph(w, 0)
     g = B.slicegcn_graph_create(w["n"], src, dst, B.SYMMETRIZE | B.ADD_SELF_LOOPS)
     info = B.slicegcn_graph_info(g)
@@ -67,13 +79,17 @@ def main():
           f"layers={w['layers']}, classes={w['classes']}, {w['dtype']}; {args.epochs} timed epochs per cell\n")
     print("| method | " + " | ".join(f"p={p}: ms/epoch (epochs/s) [params]" for p in ps) + " |")
     print("|---|" + "---|" * len(ps))
-    ms, cnt, _ = time_variant(B, torch, g, w, X, y, 1, False, False, False, args.epochs)
-    print(f"| GCN (one slice, no self branch) | {ms:.2f} ({1e3 / ms:.1f}) [{cnt:,}] |" + " |" * (len(ps) - 1))
+    t3 = args.table3_shapes
+    # Table III counts two weight matrices and two bias vectors per GCN layer: with --table3-shapes the one-slice row
+    # keeps the self branch so that the parameter count printed here is the table's
+    ms, cnt, _ = time_variant(B, torch, g, w, X, y, 1, False, False, t3, args.epochs, table3=t3)
+    label = "GCN (one slice, self branch as in Table III)" if t3 else "GCN (one slice, no self branch)"
+    print(f"| {label} | {ms:.2f} ({1e3 / ms:.1f}) [{cnt:,}] |" + " |" * (len(ps) - 1))
     for name, ff, se in (("SliceGCN", False, False), ("SliceGCN-SE", False, True), ("SliceGCN-FF", True, False),
                          ("SliceGCN-FFSE", True, True)):
         cells = []
         for p in ps:
-            ms, cnt, _ = time_variant(B, torch, g, w, X, y, p, ff, se, True, args.epochs)
+            ms, cnt, _ = time_variant(B, torch, g, w, X, y, p, ff, se, True, args.epochs, table3=t3)
             cells.append(f"{ms:.2f} ({1e3 / ms:.1f}) [{cnt:,}]")
         print(f"| {name} | " + " | ".join(cells) + " |")
     B.slicegcn_graph_destroy(g)
