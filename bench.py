@@ -304,7 +304,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         "e2e": {"value": world * args.steps / (e2e_ms / 1e3), "unit": "epochs/s",
                 "h2d_bytes_per_step": Xp.numel() * Xp.element_size() + yp.numel() * 4, "d2h_bytes_per_step": 4},
         "gpu_launches": int(prof["kernel_launches"]),
-        "roofline": {"bound": "hbm", "kernel": "spmm_rows_kernel (+ spmm_long_finish_kernel)",
+        "roofline": {"bound": "hbm", "kernel": "spmm_rows_kernel",
                      "achieved": achieved, "peak": peak, "peak_source": f"of {peak_src}", "unit": "GB/s",
                      "frac": achieved / peak, "traffic": NCU_SPMM_TRAFFIC_BYTES.get(args.workload),
                      "launches": int(prof["spmm_calls"]), "sampled_every": SPMM_SAMPLE_STRIDE, "avg_ms": spmm_avg_ms,

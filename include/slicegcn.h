@@ -117,7 +117,8 @@ slicegcn_status_t slicegcn_graph_destroy(slicegcn_graph* g);
  * overlap.  in_dtype / out_dtype: SLICEGCN_F32 or SLICEGCN_BF16 (fp32 accumulation); the pairs fp32 -> fp32,
  * bf16 -> bf16 and bf16 -> fp32 are supported (fp32 -> bf16: UNSUPPORTED).
  * workspace [device]: at least slicegcn_spmm_workspace_bytes(g, width) bytes (partial sums of the
- * split hub rows; may be NULL when that size is 0).  Deterministic: no floating-point atomics.
+ * split hub rows and one counter per such row; may be NULL when that size is 0; two calls that may
+ * overlap on the GPU need separate workspaces).  Deterministic: no floating-point atomics.
  * Errors: INVALID_ARG, UNSUPPORTED, ALLOC (workspace too small), CUDA.
  */
 slicegcn_status_t slicegcn_spmm_workspace_bytes(const slicegcn_graph* g, int32_t width, int64_t* bytes);

@@ -7,8 +7,9 @@
 // slot and read back as one broadcast load per neighbor; a few neighbors are gathered before the FMAs so
 // several rows are in flight per lane.  No per-edge value array exists:  A_hat_ij = dinv_i * dinv_j.
 // Rows longer than kLongRow are cut into kSegment-entry segments, one warp each (same launch); a row
-// of one segment is finished by that warp, the others leave partial rows that a small second kernel
-// sums in segment order -- deterministic, no floating-point atomics.
+// of one segment is finished by that warp, the others leave partial rows, and the warp that arrives
+// last at the row's counter (an integer atomic) sums them in segment order -- deterministic, no
+// floating-point atomics, no second launch.
 #include <vector>
 
 #include "common.cuh"
@@ -82,6 +83,7 @@ struct SpmmParams {
     const int32_t* seg_row;
     const int32_t* seg_order;   // processing order of the segments (by first column index)
     float* partial;  // [n_seg][nch*V]
+    int32_t* seg_done;   // [n_long] segments of each long row that have left their partial row (zeroed before the launch)
     int32_t n_chunks;
     const int32_t* chunk_row;
     // epilogue (transform-first layers):  y = act(dinv_i*acc + bias) (+ previous y)
@@ -329,7 +331,7 @@ __device__ __forceinline__ void spmm_rows_block(const SpmmParams& p, const int64
 
 // One warp per segment of a long row; each of the 32/L lane groups takes a contiguous part of the
 // segment and the groups are combined with a butterfly (fixed order).  A row that fits one segment is
-// finished here; the others leave partial rows for the finish kernel.
+// finished here; of the others the last warp to arrive sums the partial rows.
 template <typename TI, typename TO, int L, int C, bool EPI>
 __device__ __forceinline__ void spmm_segment_block(const SpmmParams& p, const int64_t vblock) {
     constexpr int V = Vec<TI>::V;
@@ -445,16 +447,56 @@ __device__ __forceinline__ void spmm_segment_block(const SpmmParams& p, const in
                 if (chunk < p.nch) finish_chunk<TO, V, EPI>(p, row, chunk, di, acc[c]);
             }
         }
-    } else if (sub == 0) {
-        float* out = p.partial + (int64_t)seg * (p.nch * V);
+    } else {
+        // several segments: leave the partial row; the warp that arrives last at the row's counter sums the row's
+        // partial rows in segment order (whichever warp that is, the order of the additions is the same)
+        const int pstride = p.nch * V;
+        if (sub == 0) {
+            float* out = p.partial + (int64_t)seg * pstride;
 #pragma unroll
-        for (int c = 0; c < C; ++c) {
-            const int chunk = sl + c * L;
-            if (chunk < p.nch) {
+            for (int c = 0; c < C; ++c) {
+                const int chunk = sl + c * L;
+                if (chunk < p.nch) {
 #pragma unroll
-                for (int e = 0; e < V; e += 4)
-                    *reinterpret_cast<float4*>(out + chunk * V + e) =
-                        make_float4(acc[c][e], acc[c][e + 1], acc[c][e + 2], acc[c][e + 3]);
+                    for (int e = 0; e < V; e += 4)
+                        *reinterpret_cast<float4*>(out + chunk * V + e) =
+                            make_float4(acc[c][e], acc[c][e + 1], acc[c][e + 2], acc[c][e + 3]);
+                }
+            }
+        }
+        __threadfence();   // the partial row is visible device-wide before the counter moves
+        __syncwarp();
+        const int s0 = __ldg(p.seg_ptr + li), s1 = __ldg(p.seg_ptr + li + 1);
+        int last = 0;
+        if (lane == 0) last = atomicAdd(p.seg_done + li, 1) == s1 - s0 - 1;
+        last = __shfl_sync(0xffffffffu, last, 0);
+        if (last && sub == 0) {
+            __threadfence();
+#pragma unroll
+            for (int c = 0; c < C; ++c)
+#pragma unroll
+                for (int e = 0; e < V; ++e) acc[c][e] = 0.f;
+#pragma unroll 4
+            for (int s = s0; s < s1; ++s) {
+                const float* src = p.partial + (int64_t)s * pstride;
+#pragma unroll
+                for (int c = 0; c < C; ++c) {
+                    const int chunk = min(sl + c * L, p.nch - 1);
+#pragma unroll
+                    for (int e = 0; e < V; e += 4) {
+                        const float4 v = __ldcg(reinterpret_cast<const float4*>(src + chunk * V + e));   // written by other SMs
+                        acc[c][e] += v.x;
+                        acc[c][e + 1] += v.y;
+                        acc[c][e + 2] += v.z;
+                        acc[c][e + 3] += v.w;
+                    }
+                }
+            }
+            const float di = __ldg(p.dinv + row);
+#pragma unroll
+            for (int c = 0; c < C; ++c) {
+                const int chunk = sl + c * L;
+                if (chunk < p.nch) finish_chunk<TO, V, EPI>(p, row, chunk, di, acc[c]);
             }
         }
     }
@@ -468,45 +510,6 @@ __global__ void __launch_bounds__(kRowsWarps * 32, kRowsBlocksPerSm<L, C>) spmm_
         spmm_segment_block<TI, TO, L, C, EPI>(p, blockIdx.x);
     else
         spmm_rows_block<TI, TO, L, C, EPI>(p, (int64_t)blockIdx.x - seg_blocks);
-}
-
-// Sums the partial rows of each long row in segment order, then scales / applies the epilogue.
-// One warp per (long row, block of 32 columns): the hub rows with dozens of segments set the
-// kernel's duration, so their columns are spread over many warps.
-template <typename TO, bool EPI>
-__global__ void __launch_bounds__(256) spmm_long_finish_kernel(const SpmmParams p, int pstride) {
-    const int lane = threadIdx.x & 31;
-    const int li = (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5);
-    if (li >= p.n_long) return;
-    const int col = blockIdx.y * 32 + lane;
-    if (col >= p.width) return;
-    const int64_t row = __ldg(p.long_rows + li);
-    const int s0 = __ldg(p.seg_ptr + li), s1 = __ldg(p.seg_ptr + li + 1);
-    if (s1 - s0 == 1) return;   // finished by its segment's warp
-    const float di = __ldg(p.dinv + row);
-    TO* Y = static_cast<TO*>(p.Y) + row * p.ldy;
-    {
-        float a = 0.f;
-        int s = s0;
-        for (; s + 8 <= s1; s += 8) {   // eight loads in flight, summed in segment order
-            float v[8];
-#pragma unroll
-            for (int q = 0; q < 8; ++q) v[q] = p.partial[(int64_t)(s + q) * pstride + col];
-#pragma unroll
-            for (int q = 0; q < 8; ++q) a += v[q];
-        }
-        for (; s < s1; ++s) a += p.partial[(int64_t)s * pstride + col];
-        float x = a * di;
-        if (EPI) {
-            x += p.bias ? __ldg(p.bias + col) : 0.f;
-            if (p.relu) {
-                if (p.mask) p.mask[row * p.mask_ld + col] = x > 0.f ? 1 : 0;
-                x = fmaxf(x, 0.f);
-            }
-            if (p.accumulate) x += to_f(Y[col]);
-        }
-        Y[col] = from_f<TO>(x);
-    }
 }
 
 // Fallback for operands that do not allow 128-bit access (odd leading dimension / alignment):
@@ -545,21 +548,13 @@ slicegcn_status_t launch_lc(const SpmmParams& p, bool epi, cudaStream_t st) {
     const int64_t warps = ((int64_t)p.n_chunks + RPW - 1) / RPW;
     const int64_t blocks = (warps + kRowsWarps - 1) / kRowsWarps;
     const int seg_blocks = (p.n_seg + kRowsWarps - 1) / kRowsWarps;
+    if (p.n_seg > 0) SGCN_CUDA(cudaMemsetAsync(p.seg_done, 0, sizeof(int32_t) * (size_t)p.n_long, st));
     if (epi)
         spmm_rows_kernel<TI, TO, L, C, true><<<(unsigned)(blocks + seg_blocks), kRowsWarps * 32, 0, st>>>(p, seg_blocks);
     else
         spmm_rows_kernel<TI, TO, L, C, false><<<(unsigned)(blocks + seg_blocks), kRowsWarps * 32, 0, st>>>(p, seg_blocks);
     SGCN_LAUNCH_CHECK();
     count_launch();
-    if (p.n_seg > 0) {
-        const int pstride = p.nch * Vec<TI>::V;
-        if (epi)
-            spmm_long_finish_kernel<TO, true><<<dim3((p.n_long + 7) / 8, (p.width + 31) / 32), 256, 0, st>>>(p, pstride);
-        else
-            spmm_long_finish_kernel<TO, false><<<dim3((p.n_long + 7) / 8, (p.width + 31) / 32), 256, 0, st>>>(p, pstride);
-        SGCN_LAUNCH_CHECK();
-        count_launch();
-    }
     return SLICEGCN_OK;
 }
 
@@ -623,11 +618,18 @@ struct Profiler {
 } g_prof;
 }  // namespace
 
-int64_t spmm_partial_bytes(const slicegcn_graph* g, int width) {
+static int64_t partial_rows_bytes(const slicegcn_graph* g, int width) {
     // enough for either dtype: chunks of 8 elements, at most 128 chunks per column block
     int64_t w = width < 1024 ? width : 1024;
     int64_t padded = (w + 7) / 8 * 8;
     return (int64_t)g->max_segments() * padded * (int64_t)sizeof(float);
+}
+
+int64_t spmm_partial_bytes(const slicegcn_graph* g, int width) {
+    // partial rows of the segments, then one counter per long row
+    if (g->max_segments() == 0) return 0;
+    const int64_t n_long = g->n_long[0] > g->n_long[1] ? g->n_long[0] : g->n_long[1];
+    return partial_rows_bytes(g, width) + (n_long * (int64_t)sizeof(int32_t) + 15) / 16 * 16;
 }
 
 slicegcn_status_t spmm_run(const slicegcn_graph* g, bool transpose, int in_dtype, int out_dtype, const void* X,
@@ -666,6 +668,7 @@ slicegcn_status_t spmm_run(const slicegcn_graph* g, bool transpose, int in_dtype
         p.seg_row = v.seg_row;
         p.seg_order = v.seg_order;
         p.partial = static_cast<float*>(ws);
+        p.seg_done = ws ? reinterpret_cast<int32_t*>(static_cast<unsigned char*>(ws) + partial_rows_bytes(g, width)) : nullptr;
         if (v.n_seg > 0 && (!ws || ws_bytes < spmm_partial_bytes(g, width)))
             SGCN_FAIL(SLICEGCN_ERR_ALLOC, "spmm: workspace too small (%lld < %lld bytes)", (long long)ws_bytes,
                       (long long)spmm_partial_bytes(g, width));
