@@ -9,7 +9,7 @@
 // Rows longer than kLongRow are cut into kSegment-entry segments, one warp each (same launch); a row
 // of one segment is finished by that warp, the others leave partial rows, and the warp that arrives
 // last at the row's counter (an integer atomic) sums them in segment order -- deterministic, no
-// floating-point atomics, no second launch.
+// floating-point atomics, no second launch (rows narrower than 512 bytes keep a small second kernel).
 #include <vector>
 
 #include "common.cuh"
@@ -464,20 +464,23 @@ __device__ __forceinline__ void spmm_segment_block(const SpmmParams& p, const in
                 }
             }
         }
+        if (p.seg_done == nullptr) return;   // narrow rows: a second launch sums the partial rows
         __threadfence();   // the partial row is visible device-wide before the counter moves
         __syncwarp();
         const int s0 = __ldg(p.seg_ptr + li), s1 = __ldg(p.seg_ptr + li + 1);
         int last = 0;
         if (lane == 0) last = atomicAdd(p.seg_done + li, 1) == s1 - s0 - 1;
         last = __shfl_sync(0xffffffffu, last, 0);
-        if (last && sub == 0) {
+        if (last) {
+            // lane group g sums segments s0 + g, s0 + g + 32/L, ... in that order; the groups are then combined
+            // with the same butterfly as above
             __threadfence();
 #pragma unroll
             for (int c = 0; c < C; ++c)
 #pragma unroll
                 for (int e = 0; e < V; ++e) acc[c][e] = 0.f;
 #pragma unroll 4
-            for (int s = s0; s < s1; ++s) {
+            for (int s = s0 + sub; s < s1; s += RPW) {
                 const float* src = p.partial + (int64_t)s * pstride;
 #pragma unroll
                 for (int c = 0; c < C; ++c) {
@@ -492,11 +495,20 @@ __device__ __forceinline__ void spmm_segment_block(const SpmmParams& p, const in
                     }
                 }
             }
-            const float di = __ldg(p.dinv + row);
+            __syncwarp();
 #pragma unroll
-            for (int c = 0; c < C; ++c) {
-                const int chunk = sl + c * L;
-                if (chunk < p.nch) finish_chunk<TO, V, EPI>(p, row, chunk, di, acc[c]);
+            for (int off = L; off < 32; off <<= 1)
+#pragma unroll
+                for (int c = 0; c < C; ++c)
+#pragma unroll
+                    for (int e = 0; e < V; ++e) acc[c][e] += __shfl_xor_sync(0xffffffffu, acc[c][e], off);
+            if (sub == 0) {
+                const float di = __ldg(p.dinv + row);
+#pragma unroll
+                for (int c = 0; c < C; ++c) {
+                    const int chunk = sl + c * L;
+                    if (chunk < p.nch) finish_chunk<TO, V, EPI>(p, row, chunk, di, acc[c]);
+                }
             }
         }
     }
@@ -510,6 +522,46 @@ __global__ void __launch_bounds__(kRowsWarps * 32, kRowsBlocksPerSm<L, C>) spmm_
         spmm_segment_block<TI, TO, L, C, EPI>(p, blockIdx.x);
     else
         spmm_rows_block<TI, TO, L, C, EPI>(p, (int64_t)blockIdx.x - seg_blocks);
+}
+
+// Narrow rows only (see launch_lc): sums the partial rows of each long row in segment order, then scales / applies
+// the epilogue.
+// One warp per (long row, block of 32 columns): the hub rows with dozens of segments set the
+// kernel's duration, so their columns are spread over many warps.
+template <typename TO, bool EPI>
+__global__ void __launch_bounds__(256) spmm_long_finish_kernel(const SpmmParams p, int pstride) {
+    const int lane = threadIdx.x & 31;
+    const int li = (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5);
+    if (li >= p.n_long) return;
+    const int col = blockIdx.y * 32 + lane;
+    if (col >= p.width) return;
+    const int64_t row = __ldg(p.long_rows + li);
+    const int s0 = __ldg(p.seg_ptr + li), s1 = __ldg(p.seg_ptr + li + 1);
+    if (s1 - s0 == 1) return;   // finished by its segment's warp
+    const float di = __ldg(p.dinv + row);
+    TO* Y = static_cast<TO*>(p.Y) + row * p.ldy;
+    {
+        float a = 0.f;
+        int s = s0;
+        for (; s + 8 <= s1; s += 8) {   // eight loads in flight, summed in segment order
+            float v[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) v[q] = p.partial[(int64_t)(s + q) * pstride + col];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) a += v[q];
+        }
+        for (; s < s1; ++s) a += p.partial[(int64_t)s * pstride + col];
+        float x = a * di;
+        if (EPI) {
+            x += p.bias ? __ldg(p.bias + col) : 0.f;
+            if (p.relu) {
+                if (p.mask) p.mask[row * p.mask_ld + col] = x > 0.f ? 1 : 0;
+                x = fmaxf(x, 0.f);
+            }
+            if (p.accumulate) x += to_f(Y[col]);
+        }
+        Y[col] = from_f<TO>(x);
+    }
 }
 
 // Fallback for operands that do not allow 128-bit access (odd leading dimension / alignment):
@@ -548,13 +600,28 @@ slicegcn_status_t launch_lc(const SpmmParams& p, bool epi, cudaStream_t st) {
     const int64_t warps = ((int64_t)p.n_chunks + RPW - 1) / RPW;
     const int64_t blocks = (warps + kRowsWarps - 1) / kRowsWarps;
     const int seg_blocks = (p.n_seg + kRowsWarps - 1) / kRowsWarps;
-    if (p.n_seg > 0) SGCN_CUDA(cudaMemsetAsync(p.seg_done, 0, sizeof(int32_t) * (size_t)p.n_long, st));
+    // Rows with several segments: for rows of 512 bytes and more the last segment warp to arrive sums the partial
+    // rows (its fence and counter update, ~1 us, are small next to a segment's gathers); for narrower rows that
+    // latency costs more than a second launch (R-MAT scale 20, 238 K segments: +50 us per call), so they keep one.
+    const bool in_kernel = L >= 32;
+    SpmmParams q = p;
+    if (!in_kernel) q.seg_done = nullptr;
+    if (q.n_seg > 0 && in_kernel) SGCN_CUDA(cudaMemsetAsync(q.seg_done, 0, sizeof(int32_t) * (size_t)q.n_long, st));
     if (epi)
-        spmm_rows_kernel<TI, TO, L, C, true><<<(unsigned)(blocks + seg_blocks), kRowsWarps * 32, 0, st>>>(p, seg_blocks);
+        spmm_rows_kernel<TI, TO, L, C, true><<<(unsigned)(blocks + seg_blocks), kRowsWarps * 32, 0, st>>>(q, seg_blocks);
     else
-        spmm_rows_kernel<TI, TO, L, C, false><<<(unsigned)(blocks + seg_blocks), kRowsWarps * 32, 0, st>>>(p, seg_blocks);
+        spmm_rows_kernel<TI, TO, L, C, false><<<(unsigned)(blocks + seg_blocks), kRowsWarps * 32, 0, st>>>(q, seg_blocks);
     SGCN_LAUNCH_CHECK();
     count_launch();
+    if (q.n_seg > 0 && !in_kernel) {
+        const int pstride = q.nch * Vec<TI>::V;
+        if (epi)
+            spmm_long_finish_kernel<TO, true><<<dim3((q.n_long + 7) / 8, (q.width + 31) / 32), 256, 0, st>>>(q, pstride);
+        else
+            spmm_long_finish_kernel<TO, false><<<dim3((q.n_long + 7) / 8, (q.width + 31) / 32), 256, 0, st>>>(q, pstride);
+        SGCN_LAUNCH_CHECK();
+        count_launch();
+    }
     return SLICEGCN_OK;
 }
 
