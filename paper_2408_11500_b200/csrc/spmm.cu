@@ -465,11 +465,13 @@ __device__ __forceinline__ void spmm_segment_block(const SpmmParams& p, const in
             }
         }
         if (p.seg_done == nullptr) return;   // narrow rows: a second launch sums the partial rows
-        __threadfence();   // the partial row is visible device-wide before the counter moves
-        __syncwarp();
         const int s0 = __ldg(p.seg_ptr + li), s1 = __ldg(p.seg_ptr + li + 1);
         int last = 0;
-        if (lane == 0) last = atomicAdd(p.seg_done + li, 1) == s1 - s0 - 1;
+        __syncwarp();          // every lane's stores are ordered before lane 0's fence ...
+        if (lane == 0) {
+            __threadfence();   // ... which makes the whole partial row visible device-wide before the counter moves
+            last = atomicAdd(p.seg_done + li, 1) == s1 - s0 - 1;
+        }
         last = __shfl_sync(0xffffffffu, last, 0);
         if (last) {
             // lane group g sums segments s0 + g, s0 + g + 32/L, ... in that order; the groups are then combined
