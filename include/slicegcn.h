@@ -187,7 +187,9 @@ slicegcn_status_t slicegcn_layer_forward(const slicegcn_graph* g, const slicegcn
  * loss w.r.t. H_out and is not modified.  Outputs (all fp32, OVERWRITTEN, each may be NULL to skip):
  *   dH_in  [device, n x in_cols, leading dimension din_ld] -- contributions of overlapping slices add;
  *   dW_agg, dW_self [p x in_width x h_s]; db, db_self, dE [p x h_s].
- * ReLU'(0) = 0. */
+ * ReLU'(0) = 0.  With dtype SLICEGCN_BF16 one intermediate gradient is kept in bf16 as well: dZ = dM W_agg^T of an
+ * aggregate-first layer whose slices read disjoint columns (the operand of the transposed aggregation); sums are
+ * accumulated in fp32 on both sides of it. */
 slicegcn_status_t slicegcn_layer_backward(const slicegcn_graph* g, const slicegcn_layer_desc* d, const void* H_in,
                                           const void* saved, const float* dH_out, int64_t dout_ld, float* dH_in,
                                           int64_t din_ld, float* dW_agg, float* dW_self, float* db, float* db_self,
@@ -213,7 +215,8 @@ typedef struct slicegcn_model_desc {
     int32_t use_se;            /* slice encoding on/off */
     int32_t use_self;          /* W_self term of Eq. 6 (0: plain GCN, Eq. 1) */
     int32_t use_b_self;        /* second bias per layer */
-    int32_t dtype;             /* storage type of X and of every activation */
+    int32_t dtype;             /* storage type of X and of every activation (bf16: also of dZ, see slicegcn_layer_backward);
+                                  parameters, their gradients, logits and loss are always fp32 */
     int32_t order;             /* SLICEGCN_ORDER_AUTO or a forced order for every layer */
 } slicegcn_model_desc;
 
