@@ -112,7 +112,9 @@ __global__ void __launch_bounds__(256) gemm_kernel(const GemmArgs a) {
             if (a.mul_pos) {
                 const float pv = a.mul_pos_dtype == SLICEGCN_F32
                                      ? static_cast<const float*>(a.mul_pos)[row * a.mul_pos_ld + col]
-                                     : __bfloat162float(static_cast<const __nv_bfloat16*>(a.mul_pos)[row * a.mul_pos_ld + col]);
+                                     : a.mul_pos_dtype == kGateBytes
+                                           ? (float)static_cast<const uint8_t*>(a.mul_pos)[row * a.mul_pos_ld + col]
+                                           : __bfloat162float(static_cast<const __nv_bfloat16*>(a.mul_pos)[row * a.mul_pos_ld + col]);
                 x = pv > 0.f ? x : 0.f;
             }
             if (a.accumulate) x += ldf(C + row * a.ldc + col);

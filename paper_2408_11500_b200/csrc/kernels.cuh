@@ -25,6 +25,8 @@ slicegcn_status_t spmm_run(const slicegcn_graph* g, bool transpose, int in_dtype
 // block of B and writes N columns of C starting at c_start[g].  Epilogue, in this order:
 //   x = acc + bias[g][n];  if relu: (mask_out = x > 0), x = max(x, 0);  x += post1[g][n] + post2[g][n];
 //   if mul_pos: x *= (P[r, c] > 0);  if accumulate: x += C_old;  C = x
+constexpr int kGateBytes = 2;   // GemmArgs::mul_pos_dtype: one byte per element (a ReLU mask)
+
 struct GemmArgs {
     int64_t M = 0;
     int groups = 1, K = 0, N = 0;
@@ -52,7 +54,8 @@ struct GemmArgs {
     int relu = 0;
     uint8_t* mask_out = nullptr;       // mask_out[r*mask_ld + c] = pre-activation > 0 (c = column of C)
     int64_t mask_ld = 0;
-    const void* mul_pos = nullptr;     // tensor P indexed like C (own dtype / leading dimension): x *= (P > 0)
+    const void* mul_pos = nullptr;     // tensor P indexed like C (own dtype / leading dimension): x *= (P > 0);
+                                       // mul_pos_dtype kGateBytes: P is a byte mask (non-zero lets x pass)
     int64_t mul_pos_ld = 0;
     int mul_pos_dtype = SLICEGCN_F32;
     int accumulate = 0;

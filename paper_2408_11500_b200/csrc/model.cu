@@ -573,6 +573,13 @@ struct EpochLayout {
     std::vector<void*> saved;
     std::vector<int64_t> saved_bytes;
     void* cls_act = nullptr;
+    // ReLU byte masks of the two MLP hidden layers, used as the gates of their backward products when the
+    // activations are far larger than L2 (on smaller problems the activation itself was just read by the preceding
+    // weight gradient and gates from L2: measured faster than the mask from DRAM)
+    uint8_t* cls_mask = nullptr;
+    uint8_t* ff_mask = nullptr;
+    int64_t ld_clsm = 0, ld_ffm = 0;
+    bool gate_masks = false;
     float* logits = nullptr;
     float* dlogits = nullptr;
     float* row_loss = nullptr;
@@ -630,8 +637,13 @@ slicegcn_status_t build_layout(const slicegcn_model* m, const slicegcn_graph* g,
     int64_t gw = E.ld_h;
     if (D.use_ff) gw = std::max(gw, std::max(E.ld_x0, E.ld_ffact));
     E.ld_grad = gw;
+    E.ld_clsm = align_up(D.hidden, 16);
+    E.ld_ffm = align_up(D.in_d, 16);
+    E.gate_masks = n * E.ld_cls * esz >= ((int64_t)512 << 20);
+    if (const char* force = getenv("SLICEGCN_GATE_MASKS")) E.gate_masks = atoi(force) != 0;   // tests reach both forms at small sizes
     if (D.use_ff) {
         E.ff_act = b.take(n * E.ld_ffact * esz);
+        if (E.gate_masks) E.ff_mask = static_cast<uint8_t*>(b.take(n * E.ld_ffm));
         E.xff = b.take(n * E.ld_x0 * esz);
     }
     if (m->repack_input()) {
@@ -657,6 +669,7 @@ slicegcn_status_t build_layout(const slicegcn_model* m, const slicegcn_graph* g,
         ws_need = std::max(ws_need, std::max(layer_fwd_ws_bytes(g, pl), layer_bwd_ws_bytes(g, pl)));
     }
     E.cls_act = b.take(n * E.ld_cls * esz);
+    if (E.gate_masks) E.cls_mask = static_cast<uint8_t*>(b.take(n * E.ld_clsm));
     E.logits = static_cast<float*>(b.take(n * (int64_t)D.num_classes * 4));
     E.ld_dlog = align_up(D.num_classes, 4);
     E.dlogits = static_cast<float*>(b.take(n * E.ld_dlog * 4));
@@ -926,6 +939,10 @@ static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, 
         a.ldb = D.in_d;
         a.bias = params + m->ff_b1;
         a.relu = 1;
+        if (E.gate_masks) {
+            a.mask_out = E.ff_mask;
+            a.mask_ld = E.ld_ffm;
+        }
         a.C = E.ff_act;
         a.ldc = E.ld_ffact;
         a.c_dtype = D.dtype;
@@ -1000,6 +1017,10 @@ static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, 
         a.ldb = D.hidden;
         a.bias = params + m->bc1;
         a.relu = 1;
+        if (E.gate_masks) {
+            a.mask_out = E.cls_mask;
+            a.mask_ld = E.ld_clsm;
+        }
         a.C = E.cls_act;
         a.ldc = E.ld_cls;
         a.c_dtype = D.dtype;
@@ -1060,6 +1081,11 @@ static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, 
         a.mul_pos = E.cls_act;
         a.mul_pos_ld = E.ld_cls;
         a.mul_pos_dtype = D.dtype;
+        if (E.gate_masks) {   // the byte mask of the forward ReLU: a quarter (bf16: half) of the activation's bytes
+            a.mul_pos = E.cls_mask;
+            a.mul_pos_ld = E.ld_clsm;
+            a.mul_pos_dtype = kGateBytes;
+        }
         SGCN_TRY(gemm_run(a, st));
         WgradArgs w1;
         w1.fault = g->fault;
@@ -1140,6 +1166,11 @@ static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, 
         a.mul_pos = E.ff_act;
         a.mul_pos_ld = E.ld_ffact;
         a.mul_pos_dtype = D.dtype;
+        if (E.gate_masks) {
+            a.mul_pos = E.ff_mask;
+            a.mul_pos_ld = E.ld_ffm;
+            a.mul_pos_dtype = kGateBytes;
+        }
         SGCN_TRY(gemm_run(a, st));
         WgradArgs w1;
         w1.fault = g->fault;

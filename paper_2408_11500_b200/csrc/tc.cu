@@ -599,7 +599,9 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const GemmArgs a, c
                     if (row < a.M && col_ok)
                         pv = a.mul_pos_dtype == SLICEGCN_F32
                                  ? __ldg(static_cast<const float*>(a.mul_pos) + row * a.mul_pos_ld + col)
-                                 : __bfloat162float(static_cast<const __nv_bfloat16*>(a.mul_pos)[row * a.mul_pos_ld + col]);
+                                 : a.mul_pos_dtype == kGateBytes
+                                       ? (float)__ldg(static_cast<const uint8_t*>(a.mul_pos) + row * a.mul_pos_ld + col)
+                                       : __bfloat162float(static_cast<const __nv_bfloat16*>(a.mul_pos)[row * a.mul_pos_ld + col]);
                     gate[r] = pv;
                 }
             }
@@ -966,6 +968,13 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_gemm_ws_kernel(const GemmArg
                             if (a.mul_pos_dtype == SLICEGCN_F32) {
                                 gate[i] = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(a.mul_pos) +
                                                                                 (rfirst + 4 * i) * a.mul_pos_ld + col));
+                            } else if (a.mul_pos_dtype == kGateBytes) {   // four mask bytes
+                                const uint32_t mb = __ldg(reinterpret_cast<const uint32_t*>(
+                                    static_cast<const uint8_t*>(a.mul_pos) + (rfirst + 4 * i) * a.mul_pos_ld + col));
+                                // the bytes as float BIT PATTERNS (1 -> a positive denormal): the test below is "> 0", and an
+                                // integer-to-float conversion per element would cost more than the load saves
+                                gate[i] = make_float4(__uint_as_float(mb & 0xffu), __uint_as_float((mb >> 8) & 0xffu),
+                                                      __uint_as_float((mb >> 16) & 0xffu), __uint_as_float(mb >> 24));
                             } else {
                                 const uint2 h = __ldg(reinterpret_cast<const uint2*>(
                                     static_cast<const __nv_bfloat16*>(a.mul_pos) + (rfirst + 4 * i) * a.mul_pos_ld + col));
@@ -1357,7 +1366,7 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
                     for (int cc = 0; cc < nnn; cc += 32) {
                         asm volatile("prefetch.global.L2 [%0];" ::"l"(static_cast<const char*>(a.mul_pos) +
                                                                           ((nrow + 4 * i) * a.mul_pos_ld + ncol0 + cc) *
-                                                                              (a.mul_pos_dtype == SLICEGCN_F32 ? 4 : 2)));
+                                                                              (a.mul_pos_dtype == SLICEGCN_F32 ? 4 : a.mul_pos_dtype == kGateBytes ? 1 : 2)));
                     }
                 }
             }
@@ -1392,6 +1401,13 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
                             if (a.mul_pos_dtype == SLICEGCN_F32) {
                                 gate[i] = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(a.mul_pos) +
                                                                                 (rfirst + 4 * i) * a.mul_pos_ld + col));
+                            } else if (a.mul_pos_dtype == kGateBytes) {   // four mask bytes
+                                const uint32_t mb = __ldg(reinterpret_cast<const uint32_t*>(
+                                    static_cast<const uint8_t*>(a.mul_pos) + (rfirst + 4 * i) * a.mul_pos_ld + col));
+                                // the bytes as float BIT PATTERNS (1 -> a positive denormal): the test below is "> 0", and an
+                                // integer-to-float conversion per element would cost more than the load saves
+                                gate[i] = make_float4(__uint_as_float(mb & 0xffu), __uint_as_float((mb >> 8) & 0xffu),
+                                                      __uint_as_float((mb >> 16) & 0xffu), __uint_as_float(mb >> 24));
                             } else {
                                 const uint2 hq = __ldg(reinterpret_cast<const uint2*>(
                                     static_cast<const __nv_bfloat16*>(a.mul_pos) + (rfirst + 4 * i) * a.mul_pos_ld + col));
@@ -1557,7 +1573,7 @@ bool ts_gemm_ok(const GemmArgs& a, int n_pad, int n_tiles) {
                            a.c_start[0] + ((a.N + 3) & ~3) <= a.ldc;
     ok = ok && (a.N % 4 == 0 || pad_write) && (a.ldc % 4 == 0) && ((uintptr_t)a.C % 16 == 0);
     if (a.mask_out) ok = ok && (a.mask_ld % 4 == 0) && ((uintptr_t)a.mask_out % 4 == 0);
-    if (a.mul_pos) ok = ok && (a.mul_pos_ld % 4 == 0) && ((uintptr_t)a.mul_pos % 16 == 0);
+    if (a.mul_pos) ok = ok && (a.mul_pos_ld % 4 == 0) && ((uintptr_t)a.mul_pos % 16 == 0);   // (a byte mask would do with 4)
     if (a.a_mask) {
         ok = ok && !fused && ((uintptr_t)a.a_mask % 16 == 0) && (a.a_mask_ld % 16 == 0);
         for (int g = 0; g < a.groups; ++g) ok = ok && (a.a_start[g] % 16 == 0);

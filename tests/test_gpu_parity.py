@@ -354,6 +354,28 @@ def test_epoch_gradients_fp32(B, kw):
         gp.close()
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_epoch_with_byte_mask_gates(B, dtype, monkeypatch):
+    """Large problems gate the backward products of the classifier and of the fusion MLP by the forward ReLU's
+    byte mask instead of the activation; SLICEGCN_GATE_MASKS=1 selects that form at test size."""
+    monkeypatch.setenv("SLICEGCN_GATE_MASKS", "1")
+    src, dst, X, y, mk, od, params = small_problem(n=1500, m_edges=9000, in_d=100, hidden=128, L=2, C=11, p=4,
+                                                   use_ff=True, use_se=True)
+    og = orc.build_graph(len(X), src, dst, True, True)
+    rnd = orc.identity
+    if dtype == "bf16":
+        mk["dtype"] = B.BF16
+        X = orc.round_bf16(X)
+        rnd = orc.round_bf16
+    gp = GpuProblem(len(X), src, dst, X, y, params, **mk)
+    try:
+        orders = [{1: "agg", 2: "xform"}[B.slicegcn_model_layer_order(gp.m, l)] for l in range(2)]
+        _compare_epoch(gp, od, og, np.asarray(X, np.float64), y, params, None, TOL_F32 if dtype == "f32" else TOL_BF16,
+                       rnd=rnd, orders=orders)
+    finally:
+        gp.close()
+
+
 def test_tiny_workload_ten_epochs_fp32(B):
     """The tiny workload (2,708 nodes, 1,433 binary features, 4 overlapping slices, hidden 16):
     ten training epochs, loss / logits / parameters tracked against the oracle."""
