@@ -47,6 +47,7 @@ struct GemmArgs {
     void* C = nullptr;
     int64_t ldc = 0;
     int c_dtype = SLICEGCN_F32;
+    int reverse = 0;                   // visit the row tiles from the last one down (L2 reuse across consecutive kernels)
     int c_start[SLICEGCN_MAX_SLICES] = {0};
     const float* bias = nullptr;       // [groups][N] (stride N), added before the activation
     const float* post1 = nullptr;      // [groups][N], added after the activation

@@ -642,6 +642,7 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const GemmArgs a, c
 struct ItemCursor {
     uint32_t rt, rem, dq, dr, per_row;
     int n_tiles, g, nt;
+    int flip = -1;   // >= 0: row tiles are visited from the last one (index flip) down
     __device__ void init(uint32_t first, uint32_t stride, int groups, int n_tiles_) {
         n_tiles = n_tiles_;
         per_row = (uint32_t)(n_tiles * groups);
@@ -669,7 +670,7 @@ struct ItemCursor {
         }
         split();
     }
-    __device__ int64_t row0() const { return (int64_t)rt * 128; }
+    __device__ int64_t row0() const { return (int64_t)(flip >= 0 ? (uint32_t)flip - rt : rt) * 128; }
 };
 
 
@@ -1136,6 +1137,7 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
         uint32_t pass = 0, rpass = 0;
         ItemCursor c_it;
         c_it.init(blockIdx.x, gridDim.x, a.groups, n_tiles);
+        c_it.flip = a.reverse ? (int)((a.M + 127) / 128) - 1 : -1;
         bool okp = true;
         for (int64_t j = 0; j < my_steps; ++j) {
             okp = mbar_wait(&rfull[rs], rpass & 1);
@@ -1234,6 +1236,7 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
             uint32_t rpass = 0;
             ItemCursor l_it;
             l_it.init(blockIdx.x, gridDim.x, a.groups, n_tiles);
+            l_it.flip = a.reverse ? (int)((a.M + 127) / 128) - 1 : -1;
             for (int64_t j = 0; j < my_steps; ++j) {
                 if (rpass >= 1 && !mbar_wait(&rfree[rs], (rpass - 1) & 1)) {
                     atomicExch(fault, 8);
@@ -1346,6 +1349,7 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
         bool oke = true;
         ItemCursor e_it;
         e_it.init(blockIdx.x + (uint32_t)e * gridDim.x, 2 * gridDim.x, a.groups, n_tiles);
+        e_it.flip = a.reverse ? (int)((a.M + 127) / 128) - 1 : -1;
         for (int64_t it = e; it < my_items && oke; it += 2) {
             const int64_t row0 = e_it.row0();
             const int g = e_it.g, nt = e_it.nt;
