@@ -16,8 +16,12 @@ What is pinned (see tests/test_oracle_*.py) and what is not:
   * backward                          -- central finite differences of the loss
   * cross entropy (Eq. 10)            -- uniform logits => ln C
   * Adam / cosine schedule            -- first-step closed form, lr(T/2), lr(T)
+  * epoch loop (Algorithm 3)          -- two epochs of a three-parameter problem worked by
+                                          hand: which index feeds the rate, which the step
+  * storage rounding (bf16 configs)   -- which tensors are representable afterwards, call counts
   * parity unpinned: the activation inside MLP_FF and MLP_CLS (ReLU is a choice;
-    the paper prints none), Adam's beta/eps constants, dropout (not modelled).
+    the paper prints none), Adam's beta/eps constants, the placement of dropout
+    (Table II lists a rate, the text never says where it acts).
 
 Array conventions: row-major numpy float64 unless stated; node features are
 n x d'; slices are column ranges [start, end) (0-based, half-open, as in
@@ -84,20 +88,13 @@ def slice_strategy(in_d: int, p: int, scale: float = 1.0, rule: str = "ceil") ->
         slice_size = in_d // p + 1
     else:
         raise ValueError(rule)
-    width = int(slice_size * scale)          # int(): truncation toward zero
+    width = int(slice_size * scale)          # Algorithm 1 truncates the scaled width toward zero
     if width < 1 or width > in_d:
         raise ValueError("scaled slice width outside [1, in_d]")
-    in_sizes = []
-    for i in range(p):
-        slice_start = i * slice_size
-        slice_end = slice_start + width
-        if slice_end > in_d:                 # the last slice(s): shift left
-            slice_start = slice_start - (slice_end - in_d)
-            slice_end = in_d
-        if slice_start < 0:
-            raise ValueError("slice does not fit")
-        in_sizes.append((slice_start, slice_end))
-    return in_sizes, slice_size
+    # Slice i would start at i * slice_size; one that would run past the last column is moved
+    # left until it ends there (Algorithm 1's correction step; Eq. 3's second case).
+    starts = [min(i * slice_size, in_d - width) for i in range(p)]
+    return [(s0, s0 + width) for s0 in starts], slice_size
 
 
 def slice_bounds_eq3(d_in: int, p: int, i: int) -> Tuple[int, int]:
@@ -157,15 +154,6 @@ def build_graph(n: int, src: np.ndarray, dst: np.ndarray, symmetrize: bool = Tru
     if rowptr[-1] >= 2 ** 31:
         raise OverflowError("nnz does not fit int32")
     g = Graph(n, rowptr.astype(np.int32), cols.astype(np.int32), deg.astype(np.int32), False)
-    g.symmetric = is_symmetric(g)
-    return g
-
-
-def graph_from_csr(n: int, rowptr: np.ndarray, colidx: np.ndarray) -> Graph:
-    rowptr = np.asarray(rowptr, dtype=np.int32)
-    colidx = np.asarray(colidx, dtype=np.int32)
-    deg = np.diff(rowptr).astype(np.int32)
-    g = Graph(n, rowptr, colidx, deg, False)
     g.symmetric = is_symmetric(g)
     return g
 
@@ -308,23 +296,57 @@ def relu(x):
     return np.maximum(x, 0.0)
 
 
+# Names of the places where a bf16-stored schedule keeps a tensor in the storage type.  Which of them a
+# given run uses is an INPUT of forward() / backward() (`rnd_at`), never derived here:
+#   forward : "ff_act", "X_ff", "Z.<l>" (aggregate-first layer l), "T.<l>" (transform-first), "H.<l>"
+#             (output of layer l, l = 1..L), "cls_act"
+#   backward: "dZ.<l>" (dM W_agg^T of aggregate-first layer l, the operand of the transposed aggregation)
+def forward_rounding_points(m: "ModelDesc", order: Sequence[str]) -> frozenset:
+    """Every forward point of a model with the given per-layer orders (what a schedule that stores
+    all activations in the storage type uses)."""
+    pts = {"cls_act"} | {f"H.{l + 1}" for l in range(m.num_layers)}
+    pts |= {("Z" if order[l] == "agg" else "T") + f".{l}" for l in range(m.num_layers)}
+    if m.use_ff:
+        pts |= {"ff_act", "X_ff"}
+    return frozenset(pts)
+
+
+def _check_points(rnd_at, allowed):
+    unknown = set(rnd_at) - set(allowed)
+    if unknown:
+        raise ValueError(f"no such rounding point in this model / schedule: {sorted(unknown)}")
+
+
 def forward(m: ModelDesc, g: Graph, x: np.ndarray, params: Dict[str, np.ndarray],
             labels: Optional[np.ndarray] = None, train_idx: Optional[np.ndarray] = None,
             rnd: Callable[[np.ndarray], np.ndarray] = identity,
-            order: Optional[Sequence[str]] = None, threads: int = 0) -> Dict[str, object]:
-    """One forward pass.  rnd is applied wherever the evaluated schedule stores
-    an activation (identity for fp32 storage, round_bf16 for bf16 storage);
-    order[l] in {"agg", "xform"} says which intermediate layer l stores
-    (A_hat*H or H*W_agg) -- the two are the same mathematics.
-    Returns every intermediate needed by backward()."""
+            order: Optional[Sequence[str]] = None, threads: int = 0,
+            rnd_at: Optional[Sequence[str]] = None,
+            dropout: Optional[Dict[int, np.ndarray]] = None, drop_rate: float = 0.0) -> Dict[str, object]:
+    """One forward pass (Eq. 4-10).
+
+    order[l] in {"agg", "xform"} says which intermediate layer l stores (A_hat*H or H*W_agg) -- the
+    two are the same mathematics.  rnd (identity for fp32 storage, round_bf16 for bf16 storage) is
+    applied at the stores named in rnd_at (see forward_rounding_points; None = all of them).
+    dropout: {l: 0/1 mask of shape n x (p*h_s)} for l in 1..L-1 -- the output of layer l is multiplied
+    by the mask and by 1/(1 - drop_rate) before the next layer reads it (placement is a choice: the
+    paper lists only a rate).  Returns every intermediate needed by backward()."""
     P = {k: np.asarray(v, dtype=np.float64) for k, v in params.items()}
     x = np.asarray(x, dtype=np.float64)
     order = list(order) if order is not None else ["agg"] * m.num_layers
-    c: Dict[str, object] = {"order": order}
+    allowed = forward_rounding_points(m, order)
+    if rnd_at is None:
+        rnd_at = allowed
+    _check_points(rnd_at, allowed)
+    r = lambda name, v: rnd(v) if name in rnd_at else v
+    dropout = dropout or {}
+    if any(l < 1 or l >= m.num_layers for l in dropout):
+        raise ValueError("dropout masks act between layers: keys 1..L-1")
+    c: Dict[str, object] = {"order": order, "dropout": dropout, "drop_rate": drop_rate}
     if m.use_ff:
         c["ff_pre"] = x @ P["ff_W1"] + P["ff_b1"]
-        c["ff_act"] = rnd(relu(c["ff_pre"]))
-        h = rnd(c["ff_act"] @ P["ff_W2"] + P["ff_b2"])
+        c["ff_act"] = r("ff_act", relu(c["ff_pre"]))
+        h = r("X_ff", c["ff_act"] @ P["ff_W2"] + P["ff_b2"])
     else:
         h = x
     c["H0"] = h
@@ -335,11 +357,11 @@ def forward(m: ModelDesc, g: Graph, x: np.ndarray, params: Dict[str, np.ndarray]
             hin = h[:, s:e]                                   # Eq. 2 / Eq. 5
             W = P[f"W_agg.{l}.{i}"]
             if order[l] == "agg":
-                z = rnd(spmm(g, hin, threads=threads))        # sum_u h_u / c_uv
+                z = r(f"Z.{l}", spmm(g, hin, threads=threads))   # sum_u h_u / c_uv
                 c[f"Z.{l}.{i}"] = z
                 mm = z @ W + P[f"b.{l}.{i}"]
             else:
-                t = rnd(hin @ W)
+                t = r(f"T.{l}", hin @ W)
                 c[f"T.{l}.{i}"] = t
                 mm = spmm(g, t, threads=threads) + P[f"b.{l}.{i}"]
             c[f"M.{l}.{i}"] = mm
@@ -351,10 +373,12 @@ def forward(m: ModelDesc, g: Graph, x: np.ndarray, params: Dict[str, np.ndarray]
             if m.use_se and l == m.num_layers - 1:
                 hi = hi + P["E"][i]                           # Eq. 7, row i of E for slice i
             out[:, i * m.h_s:(i + 1) * m.h_s] = hi            # Eq. 8: concat = adjacent columns
-        h = rnd(out)
+        if (l + 1) in dropout:
+            out = out * np.asarray(dropout[l + 1], dtype=np.float64) / (1.0 - drop_rate)
+        h = r(f"H.{l + 1}", out)
         c[f"H{l + 1}"] = h
     c["cls_pre"] = h @ P["Wc1"] + P["bc1"]                    # Eq. 9
-    c["cls_act"] = rnd(relu(c["cls_pre"]))
+    c["cls_act"] = r("cls_act", relu(c["cls_pre"]))
     logits = c["cls_act"] @ P["Wc2"] + P["bc2"]
     c["logits"] = logits
     if labels is not None:
@@ -368,14 +392,13 @@ def forward(m: ModelDesc, g: Graph, x: np.ndarray, params: Dict[str, np.ndarray]
 
 def backward(m: ModelDesc, g: Graph, x: np.ndarray, params: Dict[str, np.ndarray], labels: np.ndarray,
              cache: Dict[str, object], threads: int = 0, relu_margin: float = 0.0,
-             rnd: Callable[[np.ndarray], np.ndarray] = identity) -> Dict[str, np.ndarray]:
+             rnd: Callable[[np.ndarray], np.ndarray] = identity, rnd_at: Sequence[str] = ()) -> Dict[str, np.ndarray]:
     """Reverse-mode gradient of the mean cross-entropy w.r.t. every parameter
     (the forward pass's storage rounding treated as identity).  ReLU'(0) = 0.
 
-    rnd (identity for fp32 storage, round_bf16 for bf16 storage) is applied at the one point where a
-    bf16 schedule stores an activation gradient in the storage type: dZ = dM W_agg^T of an
-    aggregate-first layer whose slices read disjoint input columns, i.e. the operand of the transposed
-    aggregation.  Every other gradient tensor stays in full precision.
+    rnd is applied to the activation gradients named in rnd_at ("dZ.<l>": dM W_agg^T of the
+    aggregate-first layer l, the operand of the transposed aggregation); nothing is rounded unless
+    named.  Every other gradient tensor stays in full precision.
 
     relu_margin (default 0 = the definition) moves the ReLU decision threshold to
     relu_margin * max|pre-activation| of each ReLU: a positive / negative margin switches every
@@ -385,6 +408,8 @@ def backward(m: ModelDesc, g: Graph, x: np.ndarray, params: Dict[str, np.ndarray
     x = np.asarray(x, dtype=np.float64)
     idx = cache["train_idx"]
     logits = cache["logits"]
+    order = cache["order"]
+    _check_points(rnd_at, {f"dZ.{l}" for l in range(m.num_layers) if order[l] == "agg"})
     G: Dict[str, np.ndarray] = {}
     dlog = np.zeros_like(logits)
     z = logits[idx] - logits[idx].max(axis=1, keepdims=True)
@@ -394,6 +419,7 @@ def backward(m: ModelDesc, g: Graph, x: np.ndarray, params: Dict[str, np.ndarray
     dlog[idx] = sm / idx.size
     G["Wc2"] = cache["cls_act"].T @ dlog
     G["bc2"] = dlog.sum(axis=0)
+
     def on(pre, scale=None):
         sc = np.abs(pre).max() if scale is None else scale
         return pre > relu_margin * sc
@@ -408,12 +434,14 @@ def backward(m: ModelDesc, g: Graph, x: np.ndarray, params: Dict[str, np.ndarray
         ranges = m.layer_in_ranges(l)
         hprev = c[f"H{l}"]
         dprev = np.zeros_like(hprev)
+        if (l + 1) in c.get("dropout", {}):                   # the layer's output passed through a dropout mask
+            dh = dh * np.asarray(c["dropout"][l + 1], dtype=np.float64) / (1.0 - c["drop_rate"])
         if m.use_se and l == m.num_layers - 1:
             G["E"] = np.stack([dh[:, i * m.h_s:(i + 1) * m.h_s].sum(axis=0) for i in range(m.p)])
         m_scale = max(np.abs(c[f"M.{l}.{i}"]).max() for i in range(m.p))
-        disjoint = all(ranges[i][1] <= ranges[i + 1][0] for i in range(len(ranges) - 1))
         for i, (s, e) in enumerate(ranges):
-            dhi = dh[:, i * m.h_s:(i + 1) * m.h_s]
+            cols = slice(i * m.h_s, (i + 1) * m.h_s)
+            dhi = dh[:, cols]
             hin = hprev[:, s:e]
             dm = dhi * on(c[f"M.{l}.{i}"], m_scale)
             G[f"b.{l}.{i}"] = dm.sum(axis=0)
@@ -424,10 +452,10 @@ def backward(m: ModelDesc, g: Graph, x: np.ndarray, params: Dict[str, np.ndarray
                 G[f"W_self.{l}.{i}"] = hin.T @ dhi
                 dhin = dhin + dhi @ P[f"W_self.{l}.{i}"].T
             W = P[f"W_agg.{l}.{i}"]
-            if c["order"][l] == "agg":
+            if order[l] == "agg":
                 G[f"W_agg.{l}.{i}"] = c[f"Z.{l}.{i}"].T @ dm
                 dz = dm @ W.T
-                if disjoint:
+                if f"dZ.{l}" in rnd_at:
                     dz = rnd(dz)
                 dhin = dhin + spmm(g, dz, transpose=True)
             else:
@@ -470,18 +498,26 @@ def adam_step(theta: np.ndarray, grad: np.ndarray, m1: np.ndarray, m2: np.ndarra
     return theta - lr * mh / (np.sqrt(vh) + eps), m1, m2
 
 
-def train_epoch(m: ModelDesc, g: Graph, x, params: Dict[str, np.ndarray], labels, opt_state: Dict[str, object],
-                lr0: float, epoch: int, total_epochs: int, train_idx=None, rnd=identity, order=None,
-                threads: int = 0):
-    """Algorithm 3, one iteration of the epoch loop: forward, loss, backward, update.
-    opt_state holds {"m1": {...}, "m2": {...}}; params are updated in place.
-    Returns (loss, logits, grads)."""
-    cache = forward(m, g, x, params, labels, train_idx, rnd, order, threads)
-    grads = backward(m, g, x, params, labels, cache, threads, rnd=rnd)
+def apply_update(params: Dict[str, np.ndarray], grads: Dict[str, np.ndarray], opt_state: Dict[str, object],
+                 lr0: float, epoch: int, total_epochs: int) -> None:
+    """The update at the end of one iteration of Algorithm 3's epoch loop: the 0-based epoch index
+    sets the cosine-annealed rate, the number of updates made so far plus one (epoch + 1) is Adam's
+    step count.  params and opt_state ({"m1": {...}, "m2": {...}}) are updated in place."""
     lr = cosine_lr(lr0, epoch, total_epochs)
     for k in params:
         m1 = opt_state["m1"].setdefault(k, np.zeros_like(params[k], dtype=np.float64))
         m2 = opt_state["m2"].setdefault(k, np.zeros_like(params[k], dtype=np.float64))
         params[k], opt_state["m1"][k], opt_state["m2"][k] = adam_step(
             np.asarray(params[k], dtype=np.float64), grads[k], m1, m2, epoch + 1, lr)
+
+
+def train_epoch(m: ModelDesc, g: Graph, x, params: Dict[str, np.ndarray], labels, opt_state: Dict[str, object],
+                lr0: float, epoch: int, total_epochs: int, train_idx=None, rnd=identity, order=None,
+                threads: int = 0, rnd_at=None, rnd_at_bwd=(), dropout=None, drop_rate: float = 0.0):
+    """Algorithm 3, one iteration of the epoch loop: forward, loss, backward, update.
+    opt_state holds {"m1": {...}, "m2": {...}}; params are updated in place.
+    Returns (loss, logits, grads)."""
+    cache = forward(m, g, x, params, labels, train_idx, rnd, order, threads, rnd_at, dropout, drop_rate)
+    grads = backward(m, g, x, params, labels, cache, threads, rnd=rnd, rnd_at=rnd_at_bwd)
+    apply_update(params, {k: grads[k] for k in params}, opt_state, lr0, epoch, total_epochs)
     return cache["loss"], cache["logits"], grads

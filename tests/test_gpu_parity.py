@@ -289,7 +289,19 @@ def test_layer_forward_backward(B, torch, order, case):
 
 # ------------------------------------------------------------------------------ whole epoch
 
-def _compare_epoch(gp, od, og, X, y, params, train_idx, tol, rnd=orc.identity, orders=None, relu_margin=0.0):
+def _bf16_backward_points(od, orders):
+    """The activation gradients a bf16 model keeps in bf16, as the library documents them (slicegcn_layer_backward):
+    dZ = dM W_agg^T of an aggregate-first layer whose slices read disjoint columns.  Layers above the first read
+    the p disjoint blocks of the previous layer's output; the first layer computes a dZ only under feature fusion,
+    where all slices share one input (not disjoint) unless there is a single slice."""
+    pts = {f"dZ.{l}" for l in range(1, od.num_layers) if orders[l] == "agg"}
+    if od.use_ff and od.p == 1 and orders[0] == "agg":
+        pts.add("dZ.0")
+    return frozenset(pts)
+
+
+def _compare_epoch(gp, od, og, X, y, params, train_idx, tol, rnd=orc.identity, orders=None, relu_margin=0.0,
+                   report=None):
     """Logits, loss and every gradient against the oracle, per tensor in max|a-b|/max|b|.
     With relu_margin > 0 (full-size runs): of ~10^8 ReLU pre-activations a handful lie within fp32
     rounding noise of zero, and the fp32 kernel may take their sign differently from the fp64
@@ -297,28 +309,44 @@ def _compare_epoch(gp, od, og, X, y, params, train_idx, tol, rnd=orc.identity, o
     i.e. by ~1/sqrt(n) of its size, which is above 1e-4 at these sizes.  Each tensor may therefore
     also differ by twice the largest change the oracle's own gradient shows when every borderline
     unit is switched off versus on.  Logits, loss and the gradients above the last ReLU (Wc2, bc2)
-    do not depend on any such decision and keep the plain tolerance."""
+    do not depend on any such decision and keep the plain tolerance.
+    bf16 storage (rnd = round_bf16): the oracle rounds at the stores the schedule keeps in bf16 -- all forward
+    activations, and the backward points of _bf16_backward_points -- and the gradients must ALSO hold the
+    tolerance against the oracle's backward pass with no gradient rounded at all."""
     P = {k: v.astype(np.float64) for k, v in params.items()}
+    bf16 = rnd is not orc.identity
+    orders = list(orders) if orders is not None else ["agg"] * od.num_layers
+    bwd_pts = _bf16_backward_points(od, orders) if bf16 else frozenset()
     cache = orc.forward(od, og, X, P, y, train_idx, rnd=rnd, order=orders)
-    G = orc.backward(od, og, X, P, y, cache, rnd=rnd)
+    G = orc.backward(od, og, X, P, y, cache, rnd=rnd, rnd_at=bwd_pts)
+    G_plain = orc.backward(od, og, X, P, y, cache) if bwd_pts else None
     spread = None
     if relu_margin > 0:
-        lo = orc.backward(od, og, X, P, y, cache, relu_margin=relu_margin, rnd=rnd)
-        hi = orc.backward(od, og, X, P, y, cache, relu_margin=-relu_margin, rnd=rnd)
+        lo = orc.backward(od, og, X, P, y, cache, relu_margin=relu_margin, rnd=rnd, rnd_at=bwd_pts)
+        hi = orc.backward(od, og, X, P, y, cache, relu_margin=-relu_margin, rnd=rnd, rnd_at=bwd_pts)
         spread = {k: np.abs(hi[k] - lo[k]) for k in P}
     loss = gp.epoch(None)
     errs = {"logits": rel_inf(gp.logits.cpu().numpy(), cache["logits"]), "loss": abs(loss - cache["loss"]) / abs(cache["loss"])}
     bad = {k: v for k, v in errs.items() if not v <= tol}
     got = gp.named_grads()
+    rows = [("logits", errs["logits"], tol, 0.0), ("loss", errs["loss"], tol, 0.0)]
     for k in P:
         errs["d" + k] = rel_inf(got[k], G[k])
-        allowed = tol
+        allowed, sp = tol, 0.0
         if spread is not None and k not in ("Wc2", "bc2"):
-            allowed += 2.0 * spread[k].max() / np.abs(G[k]).max()
+            sp = float(spread[k].max() / np.abs(G[k]).max())
+            allowed += 2.0 * sp
         if not errs["d" + k] <= allowed:
             bad["d" + k] = (errs["d" + k], allowed)
+        if G_plain is not None and not rel_inf(got[k], G_plain[k]) <= tol:
+            bad["d" + k + " vs unrounded backward"] = rel_inf(got[k], G_plain[k])
+        rows.append(("d" + k, errs["d" + k], allowed, sp))
+    text = "\n".join(f"  {name:<12} err {e:.3e}  allowed {a:.3e}  relu-spread {sp:.3e}" for name, e, a, sp in rows)
+    print(text)
+    if report is not None:
+        report.extend(rows)
     assert not bad, bad
-    return errs
+    return errs, cache
 
 
 @pytest.mark.parametrize("kw", [
@@ -453,7 +481,7 @@ def test_citation_workload_full_size_fp32(B):
     try:
         ex = B.slicegcn_graph_export(gp.g)
         assert np.array_equal(ex["rowptr"], og.rowptr) and np.array_equal(ex["colidx"], og.colidx)
-        errs = _compare_epoch(gp, od, og, X.astype(np.float64), y, params, None, TOL_F32, relu_margin=1e-6)
+        errs, cache = _compare_epoch(gp, od, og, X.astype(np.float64), y, params, None, TOL_F32, relu_margin=1e-6)
         assert max(errs.values()) <= 1e-3 and errs["logits"] <= 2e-5
     finally:
         gp.close()
@@ -477,8 +505,8 @@ def test_social_shape_transform_first_fp32(B):
     try:
         assert [B.slicegcn_model_layer_order(gp.m, l) for l in range(2)] == [B.XFORM_FIRST, B.AGG_FIRST]
         # ~3 M ReLU units: a borderline sign decision is likely, so the oracle's own spread is allowed for
-        errs = _compare_epoch(gp, od, og, X.astype(np.float64), y, params, None, TOL_F32, orders=["xform", "agg"],
-                              relu_margin=1e-6)
+        errs, _ = _compare_epoch(gp, od, og, X.astype(np.float64), y, params, None, TOL_F32, orders=["xform", "agg"],
+                                 relu_margin=1e-6)
         assert max(errs.values()) <= 2e-3 and errs["logits"] <= 2e-5
         assert B.slicegcn_graph_device_status(gp.g) == 0
     finally:

@@ -360,14 +360,17 @@ def test_backward_matches_finite_differences(kw, order):
             assert abs(fd - an) <= 1e-6 * max(1.0, abs(fd)) + 1e-8, (name, k, fd, an)
 
 
-def test_backward_storage_rounding_acts_only_on_disjoint_aggregate_first_layers():
-    """The bf16 rounding point of the backward pass (dZ of aggregate-first layers with disjoint slices):
-    it changes nothing where it must not apply (transform-first layers, a shared fused input, the layers
-    above it), and where it applies the change is bounded by the rounding (2^-8 relative per element)."""
+def test_backward_storage_rounding_acts_only_where_named():
+    """The bf16 rounding point of the backward pass (dZ of an aggregate-first layer) is an explicit input: nothing is
+    rounded unless named; naming layer 1's dZ moves only what lies below it, by no more than the rounding
+    (2^-8 relative per element); a name that does not exist in the schedule is an error."""
     g, m, X, y, P = _tiny_problem(p=2, L=2)
     c = orc.forward(m, g, X, P, y, order=["agg", "agg"])
     ref = orc.backward(m, g, X, P, y, c)
-    rb = orc.backward(m, g, X, P, y, c, rnd=orc.round_bf16)
+    # rnd alone rounds nothing
+    quiet = orc.backward(m, g, X, P, y, c, rnd=orc.round_bf16)
+    assert all(np.array_equal(ref[k], quiet[k]) for k in ref)
+    rb = orc.backward(m, g, X, P, y, c, rnd=orc.round_bf16, rnd_at={"dZ.1"})
     # only what lies below the rounded dZ of layer 1 (the gradients of layer 0) may move
     for k in ref:
         if k.endswith(".1.0") or k.endswith(".1.1") or k in ("Wc1", "bc1", "Wc2", "bc2"):
@@ -376,15 +379,53 @@ def test_backward_storage_rounding_acts_only_on_disjoint_aggregate_first_layers(
     assert any(k.startswith("W_agg.0") for k in moved) and "H0" in moved
     for k in moved:
         assert np.abs(rb[k] - ref[k]).max() <= 2.0 ** -7 * np.abs(ref[k]).max(), k
-    # transform-first: no dZ exists, nothing is rounded
+    # layer 0's dZ only reaches the input gradient
+    r0 = orc.backward(m, g, X, P, y, c, rnd=orc.round_bf16, rnd_at={"dZ.0"})
+    assert [k for k in ref if not np.array_equal(ref[k], r0[k])] == ["H0"]
+    # transform-first: no dZ exists
     cx = orc.forward(m, g, X, P, y, order=["xform", "xform"])
-    gx, gxr = orc.backward(m, g, X, P, y, cx), orc.backward(m, g, X, P, y, cx, rnd=orc.round_bf16)
-    assert all(np.array_equal(gx[k], gxr[k]) for k in gx)
-    # shared fused input: layer 0 is excluded, layer 1 (disjoint slices of H1) is not
-    g2, m2, X2, y2, P2 = _tiny_problem(p=3, in_d=10, hidden=6, use_ff=True, L=1)
-    c2 = orc.forward(m2, g2, X2, P2, y2, order=["agg"])
-    a, b = orc.backward(m2, g2, X2, P2, y2, c2), orc.backward(m2, g2, X2, P2, y2, c2, rnd=orc.round_bf16)
-    assert all(np.array_equal(a[k], b[k]) for k in a)
+    with pytest.raises(ValueError):
+        orc.backward(m, g, X, P, y, cx, rnd=orc.round_bf16, rnd_at={"dZ.0"})
+    with pytest.raises(ValueError):
+        orc.backward(m, g, X, P, y, c, rnd=orc.round_bf16, rnd_at={"dH.1"})
+
+
+def _is_bf16(a):
+    return np.array_equal(orc.round_bf16(a), np.asarray(a, np.float64))
+
+
+def test_forward_storage_rounding_points():
+    """Which tensors a bf16-stored forward pass keeps in the storage type: exactly the named ones are
+    bf16-representable afterwards, pre-activations and logits never are, and the rounding function is called once
+    per named store."""
+    g, m, X, y, P = _tiny_problem(p=2, L=2, use_ff=True, use_se=True)
+    order = ["agg", "xform"]
+    pts = orc.forward_rounding_points(m, order)
+    assert pts == {"ff_act", "X_ff", "Z.0", "T.1", "H.1", "H.2", "cls_act"}
+    calls = []
+
+    def counting(v):
+        calls.append(v.shape)
+        return orc.round_bf16(v)
+
+    Xr = orc.round_bf16(X)
+    c = orc.forward(m, g, Xr, P, y, rnd=counting, order=order)          # default: every point of the schedule
+    # ff_act, X_ff, Z.0 and T.1 once per slice (2 each), H.1, H.2, cls_act
+    assert len(calls) == 2 + 2 + 2 + 3
+    stored = ["ff_act", "H0", "Z.0.0", "Z.0.1", "T.1.0", "T.1.1", "H1", "H2", "cls_act"]
+    full = ["ff_pre", "M.0.0", "M.1.1", "cls_pre", "logits"]
+    assert all(_is_bf16(c[k]) for k in stored)
+    assert not any(_is_bf16(c[k]) for k in full)
+    # a subset: only H.1 is rounded, everything else keeps full precision
+    c1 = orc.forward(m, g, Xr, P, y, rnd=orc.round_bf16, order=order, rnd_at={"H.1"})
+    assert _is_bf16(c1["H1"]) and not any(_is_bf16(c1[k]) for k in ["ff_act", "H0", "Z.0.0", "T.1.0", "H2", "cls_act"])
+    # no point named = the fp64 pass; a rounded pass differs from it by no more than a few roundings
+    c0 = orc.forward(m, g, Xr, P, y, rnd=orc.round_bf16, order=order, rnd_at=())
+    cf = orc.forward(m, g, Xr, P, y, order=order)
+    assert np.array_equal(c0["logits"], cf["logits"])
+    assert 0 < np.abs(c["logits"] - cf["logits"]).max() <= 0.05 * np.abs(cf["logits"]).max()
+    with pytest.raises(ValueError):
+        orc.forward(m, g, Xr, P, y, rnd=orc.round_bf16, order=order, rnd_at={"Z.1"})   # layer 1 stores T, not Z
 
 
 def test_order_of_aggregate_and_transform_is_immaterial():
@@ -411,6 +452,82 @@ def test_adam_first_step_and_cosine():
     # weight decay enters as an L2 term added to the gradient
     new_wd, _, _ = orc.adam_step(th, np.zeros(3), np.zeros(3), np.zeros(3), 1, lr=0.01, weight_decay=0.1)
     np.testing.assert_allclose(new_wd - th, -0.01 * 0.1 / (0.1 + 1e-8), rtol=1e-12)
+
+
+def _read_update_golden():
+    d = {}
+    for line in open(os.path.join(GOLDEN, "two_epoch_update.txt")):
+        t = line.split()
+        if t and not t[0].startswith("#"):
+            d[t[0]] = [float(v) for v in t[1:]]
+    return d
+
+
+def test_epoch_update_two_epochs_worked_by_hand():
+    """Which index feeds the rate and which the step count (hand-worked values): a rate taken at epoch + 1 or a step
+    count taken at epoch would both miss them."""
+    d = _read_update_golden()
+    P = {"theta": np.array(d["theta0"])}
+    st = {"m1": {}, "m2": {}}
+    T = int(d["total_epochs"][0])
+    assert abs(orc.cosine_lr(d["lr0"][0], 0, T) - d["lr_epoch0"][0]) < 1e-12
+    assert abs(orc.cosine_lr(d["lr0"][0], 1, T) - d["lr_epoch1"][0]) < 1e-8
+    orc.apply_update(P, {"theta": np.array(d["g0"])}, st, d["lr0"][0], 0, T)
+    np.testing.assert_allclose(P["theta"], d["theta1"], atol=1e-7)
+    orc.apply_update(P, {"theta": np.array(d["g1"])}, st, d["lr0"][0], 1, T)
+    np.testing.assert_allclose(P["theta"], d["theta2"], atol=1e-7)
+
+
+def test_train_epoch_is_forward_backward_update():
+    """train_epoch = forward, backward, then the update pinned above, on the parameters as they were before it:
+    epoch 0's step is the first-step closed form at the FULL rate lr0; epoch 1 (of 2) uses lr0/2 and step 2."""
+    g, m, X, y, P = _tiny_problem(n=30, m_edges=80, p=2, use_se=True)
+    P0 = {k: v.copy() for k, v in P.items()}
+    st = {"m1": {}, "m2": {}}
+    lr0 = 0.05
+    loss0, logits0, G0 = orc.train_epoch(m, g, X, P, y, st, lr0, 0, 2)
+    c = orc.forward(m, g, X, P0, y)
+    assert loss0 == c["loss"] and np.array_equal(logits0, c["logits"])      # loss and logits BEFORE the update
+    Gref = orc.backward(m, g, X, P0, y, c)
+    for k in P0:
+        assert np.array_equal(G0[k], Gref[k])
+        np.testing.assert_allclose(P[k], P0[k] - lr0 * Gref[k] / (np.abs(Gref[k]) + 1e-8), rtol=0, atol=1e-12)
+    P1 = {k: v.copy() for k, v in P.items()}
+    _, _, G1 = orc.train_epoch(m, g, X, P, y, st, lr0, 1, 2)
+    for k in P0:    # step 2 written out: 1 - 0.9^2 = 0.19, 1 - 0.999^2 = 0.001999; rate lr0/2 (cos(pi/2) = 0)
+        mh = (0.09 * G0[k] + 0.1 * G1[k]) / 0.19
+        vh = (0.000999 * G0[k] ** 2 + 0.001 * G1[k] ** 2) / 0.001999
+        np.testing.assert_allclose(P[k], P1[k] - 0.5 * lr0 * mh / (np.sqrt(vh) + 1e-8), rtol=0, atol=1e-12)
+
+
+def test_dropout_mask_between_layers():
+    """Dropout as an explicit 0/1 mask on the output of layer l < L, kept units scaled by 1/(1 - rate): a mask of
+    ones at rate 0 changes nothing; dropped units pass neither value nor gradient; finite differences hold."""
+    g, m, X, y, P = _tiny_problem(n=24, m_edges=60, p=2, L=3, seed=4)
+    base = orc.forward(m, g, X, P, y)
+    ones = {1: np.ones((g.n, m.p * m.h_s), np.uint8), 2: np.ones((g.n, m.p * m.h_s), np.uint8)}
+    same = orc.forward(m, g, X, P, y, dropout=ones, drop_rate=0.0)
+    assert np.array_equal(same["logits"], base["logits"])
+    rng = np.random.default_rng(0)
+    masks = {1: (rng.random((g.n, m.p * m.h_s)) >= 0.5).astype(np.uint8), 2: (rng.random((g.n, m.p * m.h_s)) >= 0.5).astype(np.uint8)}
+    c = orc.forward(m, g, X, P, y, dropout=masks, drop_rate=0.5)
+    assert np.all(c["H1"][masks[1] == 0] == 0) and np.all(c["H2"][masks[2] == 0] == 0)
+    kept = masks[1] == 1
+    # kept units are the undropped layer output times 1/(1 - 0.5)
+    np.testing.assert_allclose(c["H1"][kept], 2.0 * base["H1"][kept], rtol=1e-13)
+    G = orc.backward(m, g, X, P, y, c)
+    eps = 1e-6
+    for name in ("W_agg.0.1", "W_self.1.0", "b.0.0", "Wc1"):
+        flat = P[name].reshape(-1)
+        for k in (0, flat.size // 2):
+            old = flat[k]
+            flat[k] = old + eps; lp = orc.forward(m, g, X, P, y, dropout=masks, drop_rate=0.5)["loss"]
+            flat[k] = old - eps; lm = orc.forward(m, g, X, P, y, dropout=masks, drop_rate=0.5)["loss"]
+            flat[k] = old
+            fd = (lp - lm) / (2 * eps)
+            assert abs(fd - G[name].reshape(-1)[k]) <= 1e-6 * max(1.0, abs(fd)) + 1e-8, (name, k)
+    with pytest.raises(ValueError):
+        orc.forward(m, g, X, P, y, dropout={3: ones[1]}, drop_rate=0.5)     # no layer reads the last layer's output
 
 
 def test_train_epoch_decreases_loss():
