@@ -19,7 +19,8 @@
  *     calls are asynchronous on that stream; graph construction and the export calls
  *     synchronise it.
  *   - Compute calls (spmm, layer_forward/backward, train_epoch) allocate nothing; scratch
- *     memory comes from the caller, sized by the *_bytes queries.
+ *     memory comes from the caller, sized by the *_bytes queries.  (One exception takes no scratch
+ *     argument at all: slicegcn_spmm_static_scratch uses a buffer compiled into the library.)
  *   - dtype: storage type of features / activations.  Accumulation is always fp32;
  *     parameters, gradients and logits are always fp32.
  *   - There is no CPU fallback: without a CUDA device every compute call fails with
@@ -103,8 +104,12 @@ slicegcn_status_t slicegcn_graph_info(const slicegcn_graph* g, int64_t* n, int64
 slicegcn_status_t slicegcn_graph_export(const slicegcn_graph* g, int32_t* rowptr, int32_t* colidx, int32_t* deg,
                                         float* dinv);
 /* Device-side status word of the graph.  Kernels that wait on asynchronous copies bound every wait;
- * a wait that runs out sets this word instead of hanging.  Synchronises the device; *status is 0
- * when no kernel working on this graph ever gave up.  Errors: INVALID_ARG, CUDA. */
+ * a wait that runs out sets this word instead of hanging (values 1..31), and the loss kernel sets it to
+ * SLICEGCN_DEVSTATUS_BAD_LABEL when it meets a label or a training index outside its range (that node is
+ * skipped: it adds nothing to the loss or the gradients, and nothing is read through the bad value).
+ * Synchronises the device; *status is 0 when no kernel working on this graph ever reported anything.
+ * Errors: INVALID_ARG, CUDA. */
+enum { SLICEGCN_DEVSTATUS_BAD_LABEL = 32 };
 slicegcn_status_t slicegcn_graph_device_status(const slicegcn_graph* g, int32_t* status);
 /* Frees the handle and its device memory (NULL is accepted). */
 slicegcn_status_t slicegcn_graph_destroy(slicegcn_graph* g);
@@ -182,8 +187,8 @@ slicegcn_status_t slicegcn_layer_workspace_bytes(const slicegcn_graph* g, const 
 slicegcn_status_t slicegcn_layer_forward(const slicegcn_graph* g, const slicegcn_layer_desc* d, const void* H_in,
                                          void* H_out, void* saved, int64_t saved_bytes, void* workspace,
                                          int64_t workspace_bytes, void* stream);
-/* Backward of the same layer (the paper leaves it implicit: "Backpropagation to update parameters",
- * Algorithm 3).  dH_out [device, fp32, n x p*h_s, leading dimension dout_ld] is the gradient of the
+/* Backward of the same layer (the paper leaves it implicit: the last step of the epoch loop of
+ * Algorithm 3 only names it).  dH_out [device, fp32, n x p*h_s, leading dimension dout_ld] is the gradient of the
  * loss w.r.t. H_out and is not modified.  Outputs (all fp32, OVERWRITTEN, each may be NULL to skip):
  *   dH_in  [device, n x in_cols, leading dimension din_ld] -- contributions of overlapping slices add;
  *   dW_agg, dW_self [p x in_width x h_s]; db, db_self, dE [p x h_s].
@@ -252,8 +257,10 @@ slicegcn_status_t slicegcn_train_workspace_bytes(const slicegcn_model* m, const 
 /* One iteration of the epoch loop of Algorithm 3: forward, loss, backward and (if opt != NULL)
  * one Adam update with the cosine-annealed rate of epoch opt->epoch.
  *   X        [device, n x in_d of m's dtype, leading dimension x_ld]   (not modified)
- *   labels   [device, int32 n], each in [0, num_classes)                (not validated on device)
- *   train_idx[device, int32 n_train] or NULL = every node is a training node (then n_train is ignored)
+ *   labels   [device, int32 n], each in [0, num_classes); a training node whose label is outside that range is
+ *            skipped and reported through slicegcn_graph_device_status (SLICEGCN_DEVSTATUS_BAD_LABEL)
+ *   train_idx[device, int32 n_train] or NULL = every node is a training node (then n_train is ignored); an index
+ *            outside [0, n) is skipped and reported the same way
  *   params   [device, fp32 param_elems]  updated in place when opt != NULL
  *   grads    [device, fp32 param_elems]  overwritten with dLoss/dparams
  *   adam_m, adam_v [device, fp32 param_elems]  optimiser state (zero before the first epoch); may be
@@ -290,7 +297,8 @@ slicegcn_status_t slicegcn_forward_logits(const slicegcn_model* m, const slicegc
  *   loss_dev    [device, one float]: where the step leaves the loss before it is copied back
  *   every other argument as for slicegcn_train_epoch (device memory).
  * Host buffers should be page-locked: pageable memory works but the copies are slower and not
- * asynchronous.  Synchronous: returns after the stream has drained.  Errors as above. */
+ * asynchronous.  Synchronous: returns after the stream has drained.  The labels are checked on the host before
+ * anything is copied: OUT_OF_RANGE if one is outside [0, num_classes).  Other errors as above. */
 slicegcn_status_t slicegcn_train_epoch_host(const slicegcn_model* m, const slicegcn_graph* g, const void* X_host, int64_t x_ld,
                                             const int32_t* labels_host, void* X_stage, int32_t* labels_stage,
                                             const int32_t* train_idx, int64_t n_train, float* params, float* grads,
@@ -306,7 +314,8 @@ slicegcn_status_t slicegcn_train_epoch_host(const slicegcn_model* m, const slice
  *   X_stage0/1 [device, n * x_ld elements each], labels_stage0/1 [device, int32 n each]
  *   losses_dev [device, num_epochs floats], losses_host [host, num_epochs floats] or NULL
  *   opt        required (the epoch index advances inside the call)
- * Creates and destroys one stream and four events per call.  Synchronous.  Errors as above. */
+ * Creates and destroys one stream and four events per call.  Synchronous.  OUT_OF_RANGE for a label outside
+ * [0, num_classes) (checked on the host before the first copy); other errors as above. */
 slicegcn_status_t slicegcn_train_epochs_host(const slicegcn_model* m, const slicegcn_graph* g, const void* X_host, int64_t x_ld,
                                              const int32_t* labels_host, void* X_stage0, void* X_stage1, int32_t* labels_stage0,
                                              int32_t* labels_stage1, const int32_t* train_idx, int64_t n_train, float* params,

@@ -24,6 +24,7 @@ ORDER_AUTO, AGG_FIRST, XFORM_FIRST = 0, 1, 2
 RULE_CEIL, RULE_FLOOR_PLUS_1 = 0, 1
 SYMMETRIZE, ADD_SELF_LOOPS, INPUT_ON_DEVICE = 1, 2, 4
 MAX_SLICES = 64
+DEVSTATUS_BAD_LABEL = 32
 
 EXPORTS = [
     "slicegcn_last_error", "slicegcn_slice_strategy", "slicegcn_graph_create", "slicegcn_graph_create_from_csr",

@@ -327,15 +327,25 @@ __global__ void mask_mul4_kernel(int64_t M, int N4, const float4* in, int64_t ld
     }
 }
 
-// LG lanes per training row (a warp holds 32/LG rows): few classes would leave most of a warp idle
+// LG lanes per training row (a warp holds 32/LG rows): few classes would leave most of a warp idle.
+// A training index outside [0, n) or a label outside [0, C) is never dereferenced: the row is skipped (loss 0, zero
+// gradient) and the status word receives kStatusBadLabel.
 template <int LG>
-__global__ void softmax_ce_kernel(int C, const float* logits, const int32_t* labels, const int32_t* train_idx,
-                                  int64_t n_train, float inv_n, float* dlogits, int64_t ld_d, float* row_loss) {
+__global__ void softmax_ce_kernel(int64_t n, int C, const float* logits, const int32_t* labels, const int32_t* train_idx,
+                                  int64_t n_train, float inv_n, float* dlogits, int64_t ld_d, float* row_loss, int* fault) {
     const int lane = threadIdx.x & 31;
     const int sub = lane / LG, sl = lane % LG;
     const int64_t t = ((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5) * (32 / LG) + sub;
-    const bool live = t < n_train;   // idle groups stay for the shuffles
-    const int64_t r = live ? (train_idx ? train_idx[t] : t) : 0;
+    const bool in_set = t < n_train;   // idle groups stay for the shuffles
+    int64_t r = in_set ? (train_idx ? (int64_t)train_idx[t] : t) : 0;
+    const bool row_ok = r >= 0 && r < n;
+    if (!row_ok) r = 0;
+    const int y = (in_set && row_ok) ? labels[r] : 0;
+    const bool live = in_set && row_ok && y >= 0 && y < C;
+    if (in_set && !live && sl == 0) {
+        if (fault) atomicExch(fault, kStatusBadLabel);
+        row_loss[t] = 0.f;
+    }
     const float* z = logits + r * C;
     float mx = -INFINITY;
     if (live)
@@ -347,8 +357,11 @@ __global__ void softmax_ce_kernel(int C, const float* logits, const int32_t* lab
         for (int c = sl; c < C; c += LG) s += expf(z[c] - mx);
 #pragma unroll
     for (int o = LG / 2; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o, LG);
-    if (!live) return;
-    const int y = labels[r];
+    if (!in_set || !row_ok) return;
+    if (!live) {   // a bad label on a valid row: the row contributes nothing
+        for (int c = sl; c < ld_d; c += LG) dlogits[r * ld_d + c] = 0.f;
+        return;
+    }
     const float lse = mx + logf(s);
     if (sl == 0) row_loss[t] = lse - z[y];
     const float inv_s = 1.f / s;
@@ -590,16 +603,16 @@ slicegcn_status_t mask_mul_run(int64_t M, int N, const float* in, int64_t ld_in,
 
 slicegcn_status_t softmax_ce_run(int64_t n, int C, const float* logits, const int32_t* labels, const int32_t* train_idx,
                                  int64_t n_train, float* dlogits, int64_t ld_d, float* row_loss, float* loss_out,
-                                 cudaStream_t st) {
+                                 int* fault, cudaStream_t st) {
     if (train_idx) SGCN_CUDA(cudaMemsetAsync(dlogits, 0, sizeof(float) * n * ld_d, st));
     const int64_t cnt = train_idx ? n_train : n;
     if (cnt < 1) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "empty training set");
     if (C <= 64)
-        softmax_ce_kernel<8><<<(unsigned)((cnt + 31) / 32), 256, 0, st>>>(C, logits, labels, train_idx, cnt, 1.0f / (float)cnt,
-                                                                          dlogits, ld_d, row_loss);
+        softmax_ce_kernel<8><<<(unsigned)((cnt + 31) / 32), 256, 0, st>>>(n, C, logits, labels, train_idx, cnt, 1.0f / (float)cnt,
+                                                                          dlogits, ld_d, row_loss, fault);
     else
-        softmax_ce_kernel<32><<<(unsigned)((cnt + 7) / 8), 256, 0, st>>>(C, logits, labels, train_idx, cnt, 1.0f / (float)cnt,
-                                                                         dlogits, ld_d, row_loss);
+        softmax_ce_kernel<32><<<(unsigned)((cnt + 7) / 8), 256, 0, st>>>(n, C, logits, labels, train_idx, cnt, 1.0f / (float)cnt,
+                                                                         dlogits, ld_d, row_loss, fault);
     SGCN_LAUNCH_CHECK();
     count_launch();
     if (loss_out) {

@@ -137,9 +137,12 @@ slicegcn_status_t mask_mul_run(int64_t M, int N, const float* in, int64_t ld_in,
 // Softmax cross entropy (Eq. 10) over the training rows: writes dlogits = (softmax - onehot)/n_train
 // (rows outside the training set are zeroed) and the mean loss.  row_loss: scratch [n_train] floats.
 // dlogits has leading dimension ld_d >= C; columns C..ld_d-1 of every row are written as zeros.
+// A label outside [0, C) or a training index outside [0, n) is skipped, never dereferenced; `fault` (the graph's status
+// word, may be NULL) then receives kStatusBadLabel.
+constexpr int kStatusBadLabel = SLICEGCN_DEVSTATUS_BAD_LABEL;
 slicegcn_status_t softmax_ce_run(int64_t n, int C, const float* logits, const int32_t* labels, const int32_t* train_idx,
                                  int64_t n_train, float* dlogits, int64_t ld_d, float* row_loss, float* loss_out,
-                                 cudaStream_t st);
+                                 int* fault, cudaStream_t st);
 // Adam with bias correction; `step` is 1-based.
 slicegcn_status_t adam_run(int64_t count, float* theta, const float* grad, float* m1, float* m2, float lr, float beta1,
                            float beta2, float eps, float weight_decay, int step, cudaStream_t st);

@@ -1056,7 +1056,7 @@ static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, 
     }
     if (forward_only) return SLICEGCN_OK;
     // ---------------- loss (Eq. 10) and its gradient
-    SGCN_TRY(softmax_ce_run(n, C, logits, labels, train_idx, n_train, E.dlogits, E.ld_dlog, E.row_loss, loss_out, st));
+    SGCN_TRY(softmax_ce_run(n, C, logits, labels, train_idx, n_train, E.dlogits, E.ld_dlog, E.row_loss, loss_out, g->fault, st));
 
     // ---------------- backward
     {
@@ -1226,6 +1226,14 @@ slicegcn_status_t slicegcn_forward_logits(const slicegcn_model* m, const slicegc
                       logits_out, nullptr, workspace, workspace_bytes, stream);
 }
 
+// The labels of the host-buffer entry points are readable here: every one must name a class.
+static slicegcn_status_t check_labels_host(const int32_t* labels, int64_t n, int C, const char* who) {
+    for (int64_t i = 0; i < n; ++i)
+        if (labels[i] < 0 || labels[i] >= C)
+            SGCN_FAIL(SLICEGCN_ERR_OUT_OF_RANGE, "%s: label %d of node %lld is outside [0, %d)", who, labels[i], (long long)i, C);
+    return SLICEGCN_OK;
+}
+
 slicegcn_status_t slicegcn_train_epoch_host(const slicegcn_model* m, const slicegcn_graph* g, const void* X_host, int64_t x_ld,
                                             const int32_t* labels_host, void* X_stage, int32_t* labels_stage,
                                             const int32_t* train_idx, int64_t n_train, float* params, float* grads,
@@ -1236,6 +1244,7 @@ slicegcn_status_t slicegcn_train_epoch_host(const slicegcn_model* m, const slice
     if (x_ld < m->desc.in_d) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "train_epoch_host: x_ld < in_d");
     cudaStream_t st = (cudaStream_t)stream;
     const int64_t n = g->n;
+    SGCN_TRY(check_labels_host(labels_host, n, m->desc.num_classes, "train_epoch_host"));
     SGCN_CUDA(cudaMemcpyAsync(X_stage, X_host, (size_t)(n * x_ld) * esize(m->desc.dtype), cudaMemcpyHostToDevice, st));
     SGCN_CUDA(cudaMemcpyAsync(labels_stage, labels_host, (size_t)n * sizeof(int32_t), cudaMemcpyHostToDevice, st));
     SGCN_TRY(slicegcn_train_epoch(m, g, X_stage, x_ld, labels_stage, train_idx, n_train, params, grads, adam_m, adam_v, opt, nullptr,
@@ -1257,6 +1266,7 @@ slicegcn_status_t slicegcn_train_epochs_host(const slicegcn_model* m, const slic
     if (num_epochs < 1) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "train_epochs_host: num_epochs < 1");
     cudaStream_t st = (cudaStream_t)stream;
     const int64_t n = g->n;
+    SGCN_TRY(check_labels_host(labels_host, n, m->desc.num_classes, "train_epochs_host"));
     const size_t x_bytes = (size_t)(n * x_ld) * esize(m->desc.dtype), y_bytes = (size_t)n * sizeof(int32_t);
     void* xs[2] = {X_stage0, X_stage1};
     int32_t* ys[2] = {labels_stage0, labels_stage1};

@@ -627,6 +627,41 @@ def test_train_epoch_host_buffers_match_device_call(B, torch):
         gp.close()
 
 
+def test_bad_label_is_skipped_and_reported_not_dereferenced(B, torch):
+    """A label outside [0, C) or a training index outside [0, n): the loss kernel skips that node (it adds nothing
+    to loss or gradients), sets the graph's status word and reads nothing through the bad value; the host-buffer
+    entry points refuse such labels before copying anything."""
+    src, dst, X, y, mk, od, params = small_problem(p=4, in_d=64, hidden=64, C=8, n=1111)
+    og = orc.build_graph(len(X), src, dst, True, True)
+    train_idx = np.arange(0, len(X), 2).astype(np.int32)
+    bad_y = y.copy(); bad_y[10] = 2 ** 30; bad_y[12] = -5          # both are training nodes
+    bad_idx = train_idx.copy(); bad_idx[7] = 2 ** 30; bad_idx[9] = -1
+    keep = np.array([i for k, i in enumerate(train_idx) if i not in (10, 12) and k not in (7, 9)], np.int32)
+    gp = GpuProblem(len(X), src, dst, X, bad_y, params, train_idx=bad_idx, **mk)
+    try:
+        loss = gp.epoch(None)
+        assert B.slicegcn_graph_device_status(gp.g) == B.DEVSTATUS_BAD_LABEL
+        # the surviving nodes give the oracle's sums over `keep`, still divided by the full |V_L| the caller named
+        P = {k: v.astype(np.float64) for k, v in params.items()}
+        c = orc.forward(od, og, X.astype(np.float64), P, y, keep)
+        G = orc.backward(od, og, X.astype(np.float64), P, y, c)
+        scale = keep.size / train_idx.size
+        assert abs(loss - c["loss"] * scale) <= 1e-4 * abs(c["loss"])
+        got = gp.named_grads()
+        for k in P:
+            assert rel_inf(got[k], G[k] * scale) <= TOL_F32, k
+        # host-buffer entry points see the labels on the host and refuse
+        Xh = torch.from_numpy(np.ascontiguousarray(X, np.float32)).pin_memory()
+        yh = torch.from_numpy(bad_y).pin_memory()
+        Xd, yd = torch.empty_like(gp.X), torch.full_like(gp.y, 3)
+        with pytest.raises(B.SliceGCNError) as e:
+            B.slicegcn_train_epoch_host(gp.m, gp.g, Xh, Xh.shape[1], yh, Xd, yd, None, 0, gp.params, gp.grads, gp.m1, gp.m2,
+                                        None, gp.loss, None, gp.ws, gp.ws_bytes, torch.cuda.current_stream().cuda_stream)
+        assert e.value.status == B.ERR_OUT_OF_RANGE and bool((yd == 3).all())       # nothing was copied
+    finally:
+        gp.close()
+
+
 def test_profile_counts_and_sampling(B, torch):
     """The benchmark instrumentation: SpMM calls bracketed by events (all, or every stride-th), algorithmic
     bytes per bracketed call, and the number of kernels launched in between."""
