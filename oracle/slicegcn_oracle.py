@@ -133,36 +133,42 @@ def build_graph(n: int, src: np.ndarray, dst: np.ndarray, symmetrize: bool = Tru
     of i; an input pair (src, dst) = (u, v) makes v a neighbor of u (row u,
     column v).  A is 0/1: repeated pairs are merged; with self_loops every
     diagonal entry is stored exactly once."""
-    src = np.asarray(src, dtype=np.int64)
-    dst = np.asarray(dst, dtype=np.int64)
+    src = np.asarray(src)
+    dst = np.asarray(dst)
     if src.shape != dst.shape:
         raise ValueError("src/dst length mismatch")
     if src.size and (src.min() < 0 or dst.min() < 0 or src.max() >= n or dst.max() >= n):
         raise ValueError("node id out of range")
-    r, c = src, dst
+    # one key row * n + col per candidate entry: the input pairs, their reverses, the diagonal
+    m = src.size
+    key = np.empty(m * (2 if symmetrize else 1) + (n if self_loops else 0), dtype=np.int64)
+    key[:m] = src
+    key[:m] *= n
+    key[:m] += dst
     if symmetrize:
-        r, c = np.concatenate([src, dst]), np.concatenate([dst, src])
+        key[m:2 * m] = dst
+        key[m:2 * m] *= n
+        key[m:2 * m] += src
     if self_loops:
-        d = np.arange(n, dtype=np.int64)
-        r, c = np.concatenate([r, d]), np.concatenate([c, d])
-    key = np.unique(r * n + c)               # sorted by (row, col), duplicates merged
+        key[key.size - n:] = np.arange(n, dtype=np.int64) * (n + 1)
+    key.sort()                               # sorted by (row, col) ...
+    if key.size:
+        key = key[np.concatenate(([True], key[1:] != key[:-1]))]   # ... repeated pairs merged (A is 0/1)
     rows = key // n
-    cols = key % n
+    cols = (key - rows * n).astype(np.int32)
     deg = np.bincount(rows, minlength=n).astype(np.int64)
     rowptr = np.zeros(n + 1, dtype=np.int64)
     np.cumsum(deg, out=rowptr[1:])
     if rowptr[-1] >= 2 ** 31:
         raise OverflowError("nnz does not fit int32")
-    g = Graph(n, rowptr.astype(np.int32), cols.astype(np.int32), deg.astype(np.int32), False)
-    g.symmetric = is_symmetric(g)
+    g = Graph(n, rowptr.astype(np.int32), cols, deg.astype(np.int32), False)
+    # symmetric pattern: the transposed keys, sorted, are the keys
+    key_t = cols.astype(np.int64)
+    key_t *= n
+    key_t += rows
+    key_t.sort()
+    g.symmetric = bool(np.array_equal(key, key_t))
     return g
-
-
-def is_symmetric(g: Graph) -> bool:
-    rows = np.repeat(np.arange(g.n, dtype=np.int64), np.diff(g.rowptr.astype(np.int64)))
-    a = np.sort(rows * g.n + g.colidx.astype(np.int64))
-    b = np.sort(g.colidx.astype(np.int64) * g.n + rows)
-    return bool(np.array_equal(a, b))
 
 
 def dinv_f32(deg: np.ndarray) -> np.ndarray:

@@ -22,6 +22,25 @@ def _rng(seed: int, stream: int) -> np.random.Generator:
 # graphs (undirected edge lists without self pairs or repeats)
 # --------------------------------------------------------------------------
 
+def _inverse_cdf(cdf: np.ndarray, q: np.ndarray) -> np.ndarray:
+    """searchsorted(cdf, q, side="right") as int64, through a table of the answers at 2^20 evenly spaced points:
+    the answer for q starts at the table entry of q's bucket and moves up while cdf[answer] <= q (a few vector
+    passes instead of one cache-missing binary search per query; identical results)."""
+    nb = 1 << 20
+    table = np.searchsorted(cdf, np.arange(nb, dtype=np.float64) / nb, side="right").astype(np.int64)
+    out = table[np.minimum((q * nb).astype(np.int64), nb - 1)]
+    n = cdf.size
+    todo = np.flatnonzero(cdf[np.minimum(out, n - 1)] <= q)
+    todo = todo[out[todo] < n]
+    while todo.size:
+        out[todo] += 1
+        nxt = out[todo]
+        more = nxt < n
+        more[more] = cdf[nxt[more]] <= q[todo[more]]
+        todo = todo[more]
+    return out
+
+
 def _sample_pairs(n: int, weights: np.ndarray, m: int, rng: np.random.Generator) -> Tuple[np.ndarray, np.ndarray]:
     """m distinct unordered pairs {u, v}, u != v, endpoints drawn in proportion to weights."""
     cdf = np.cumsum(weights, dtype=np.float64)
@@ -31,14 +50,15 @@ def _sample_pairs(n: int, weights: np.ndarray, m: int, rng: np.random.Generator)
     while keys.size < m:
         need = m - keys.size
         batch = int(need * 1.15) + 1024
-        u = np.searchsorted(cdf, rng.random(batch), side="right").astype(np.int64)
-        v = np.searchsorted(cdf, rng.random(batch), side="right").astype(np.int64)
+        u = _inverse_cdf(cdf, rng.random(batch))
+        v = _inverse_cdf(cdf, rng.random(batch))
         np.minimum(u, n - 1, out=u)
         np.minimum(v, n - 1, out=v)
         ok = u != v
         lo = np.minimum(u[ok], v[ok])
         hi = np.maximum(u[ok], v[ok])
-        keys = np.union1d(keys, lo * n + hi)
+        keys = np.sort(np.concatenate([keys, lo * n + hi]))       # sorted union of the distinct pairs so far
+        keys = keys[np.concatenate(([True], keys[1:] != keys[:-1]))]
         rounds += 1
         if rounds > 200:
             raise RuntimeError("edge sampler did not reach the requested edge count")
