@@ -27,13 +27,10 @@ sys.path.insert(0, ROOT)
 
 from paper_2408_11500_b200 import synth  # noqa: E402
 
-# dram__bytes_read.sum + dram__bytes_write.sum per SpMM launch from the ncu capture summarised under
-# profiles/ (None until a capture of that workload exists)
 # Every SPMM_SAMPLE_STRIDE-th SpMM call inside the timed region is bracketed by CUDA events (an event pair costs the
 # stream ~10 us; bracketing all five calls of an epoch would add ~4 % to the step time).  7 is coprime to the 4-6 SpMM
 # calls of an epoch, so every call site is sampled equally often.
 SPMM_SAMPLE_STRIDE = 7
-NCU_SPMM_TRAFFIC_BYTES = {"citation": 891e6}   # width-256 launches (4 of the 5 per epoch)
 
 
 def measured_peak_gbs():
@@ -149,10 +146,12 @@ def run_reference(args, rank: int):
     """--impl reference: the oracle on the host cores, on a bounded sample of the same workload."""
     if rank != 0:
         return
+    if args.steps <= 0:
+        args.steps = 3
     total_steps = args.steps + args.warmup
     full_epoch_s = {"tiny": 0.4, "citation": 20.0, "social": 600.0, "copurchase": 900.0}[args.workload]
     frac = 1.0
-    while frac > 1 / 64 and full_epoch_s * frac * total_steps > 200.0:
+    while frac > 1 / 512 and full_epoch_s * frac * total_steps > 150.0:
         frac /= 2
     w = scaled_workload(args.workload, frac)
     times, threads = oracle_epochs(w, args.steps, args.warmup)
@@ -171,19 +170,39 @@ def run_reference(args, rank: int):
 
 # ---------------------------------------------------------------------------------- CUDA path
 
-def run_ours(args, rank: int, world: int, local_rank: int):
+# DRAM traffic of the dominant SpMM launch (dram__bytes_read.sum + dram__bytes_write.sum from one ncu capture, per launch),
+# with the committed summary each figure comes from; None where no capture exists.
+NCU_SPMM_TRAFFIC = {
+    "citation": (891e6, "profiles/spmm_rows_kernel_citation_w256.md (fp32 width-256 launch, 4 of the 5 per epoch)"),
+    "copurchase": (38.1e9, "profiles/spmm_sweep_rmat.md (bf16 width-256 forward launch, 4 of the 6 per epoch; single-pass capture)"),
+    "social": (12.0e9, "profiles/spmm_sweep_rmat.md (fp32 width-256 launch, all 4 per epoch alike)"),
+}
+DEFAULT_STEPS = {"tiny": 200, "citation": 200, "social": 20, "copurchase": 20}
+DEFAULT_CPU_FRACTION = {"tiny": 1.0, "citation": 1.0, "social": 1 / 16, "copurchase": 1 / 16}
+
+
+def max_over_ranks(x: float, world: int, dist=None, device=None, torch=None) -> float:
+    """The slowest rank's elapsed time: the only cross-rank reduction of a replica run (after a barrier)."""
+    if world == 1:
+        return x
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(world: int, steps: int, elapsed_ms: float) -> float:
+    """Epochs all replicas finished per second of the slowest replica's time."""
+    return world * steps / (elapsed_ms / 1e3)
+
+
+def measure(workload: str, steps: int, warmup: int, world: int, local_rank: int, with_e2e: bool, dist=None):
+    """Device-resident timing (and, if asked, the end-to-end run from host buffers) of one workload.
+    Returns the fields of the JSON line that depend on the workload."""
     import torch
-    import torch.distributed as dist
     from paper_2408_11500_b200 import binding as B
 
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
-    torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
-
-    w = synth.WORKLOADS[args.workload]
+    w = synth.WORKLOADS[workload]
     src, dst = synth.make_graph(w, 0)
     Xh = synth.make_features(w, 0)
     yh = synth.uniform_labels(w["n"], w["classes"], 0)
@@ -191,8 +210,11 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     dtype = B.BF16 if w["dtype"] == "bf16" else B.F32
     tdt = torch.bfloat16 if dtype == B.BF16 else torch.float32
     g = B.slicegcn_graph_create(n, src, dst, B.SYMMETRIZE | B.ADD_SELF_LOOPS)
+    del src, dst
     info = B.slicegcn_graph_info(g)
-    m = B.slicegcn_model_create(dtype=dtype, **model_kwargs(w))
+    # The features are sliced once, outside the epoch loop (Algorithm 3): with X resident on the device the first
+    # layer's aggregate is kept across epochs.  (The end-to-end run copies X anew every epoch and recomputes it.)
+    m = B.slicegcn_model_create(dtype=dtype, cache_input_aggregate=True, **model_kwargs(w))
     params0 = torch.from_numpy(B.pack_params(m, synth.init_params(B.named_param_shapes(m), 0))).to(dev)
     params = params0.clone()
     grads, m1, m2 = torch.zeros_like(params), torch.zeros_like(params), torch.zeros_like(params)
@@ -214,30 +236,29 @@ def run_ours(args, rank: int, world: int, local_rank: int):
             dist.barrier()
         torch.cuda.synchronize()
 
-    def max_over_ranks(x: float) -> float:
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    mor = lambda x: max_over_ranks(x, world, dist, dev, torch)
 
     # ---- device-resident run
     sampler = ClockSampler(local_rank)
     sampler.start()
-    for ep in range(args.warmup):
+    for ep in range(warmup - 1):
         epoch(ep, X, y)
+    B.slicegcn_profile_begin()                 # the last warm-up epoch counts the SpMM calls and launches of one epoch
+    epoch(warmup - 1, X, y)
+    per_epoch = B.slicegcn_profile_end()
     sampler.wait_first_sample()
     barrier()
     sampler.mark_begin()
     B.slicegcn_profile_begin_sampled(SPMM_SAMPLE_STRIDE)   # CUDA events around every 7th SpMM call of the timed region
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for ep in range(args.steps):
-        epoch(args.warmup + ep, X, y)
-    e1.record(stream)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    ev[0].record(stream)
+    for ep in range(steps):
+        epoch(warmup + ep, X, y)
+        ev[ep + 1].record(stream)
     barrier()
     prof = B.slicegcn_profile_end()
-    ms_total = max_over_ranks(e0.elapsed_time(e1))
+    ms_total = mor(ev[0].elapsed_time(ev[-1]))
+    step_ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
     final_loss = float(loss.item())
     # A timed region shorter than a few sampling periods holds too few clock samples: keep the same load running
     # (untimed, on copies of the optimizer state) until the sampler has seen at least three.
@@ -247,7 +268,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         t_ext = time.time()
         while sampler.samples_inside() < 3 and time.time() - t_ext < 3.0:
             for ep in range(8):
-                epoch(args.warmup + args.steps + clock_extension + ep, X, y)
+                epoch(warmup + steps + clock_extension + ep, X, y)
             torch.cuda.synchronize()
             clock_extension += 8
         for t, k in zip((params, grads, m1, m2, loss), keep):
@@ -259,67 +280,104 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         clocks["note"] = (f"timed region of {ms_total:.0f} ms is shorter than three sampling periods: sampled over it and "
                           f"{clock_extension} further untimed epochs of the same load")
 
-    # ---- end to end: ONE C-ABI call runs the epochs from host buffers.  Every epoch copies X and the
-    # labels from page-locked host memory again and returns its loss to the host; the library overlaps the
-    # copy for epoch e+1 with the kernels of epoch e (two staging buffers).
-    Xp = (torch.from_numpy(Xh).to(tdt) if dtype == B.BF16 else torch.from_numpy(Xh)).pin_memory()
-    yp = torch.from_numpy(yh).pin_memory()
-    n_e2e = max(args.steps, args.warmup, 1)
-    losses_host = torch.zeros(n_e2e, dtype=torch.float32).pin_memory()
-    losses_dev = torch.zeros(n_e2e, dtype=torch.float32, device=dev)
-    Xd = [torch.empty_like(X), torch.empty_like(X)]
-    yd = [torch.empty_like(y), torch.empty_like(y)]
-    params.copy_(params0); m1.zero_(); m2.zero_()
-
-    def e2e_run(first_epoch, count):
-        B.slicegcn_train_epochs_host(m, g, Xp, w["in_d"], yp, Xd[0], Xd[1], yd[0], yd[1], None, 0, params, grads, m1, m2,
-                                     B.make_opt_desc(1e-3, first_epoch, total_epochs), count, losses_dev, losses_host,
-                                     ws, ws_bytes, stream.cuda_stream)
-
-    e2e_run(0, max(args.warmup, 1))
-    barrier()
-    t0 = time.perf_counter()
-    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    f0.record(stream)
-    e2e_run(args.warmup, args.steps)          # returns after the last loss has reached the host
-    f1.record(stream)
-    barrier()
-    e2e_ms = max_over_ranks(max(f0.elapsed_time(f1), 1e3 * (time.perf_counter() - t0)))
-    if not all(np.isfinite(losses_host[:args.steps].numpy())):
-        raise SystemExit("end-to-end run produced a non-finite loss")
-
-    value = world * args.steps / (ms_total / 1e3)
     peak, peak_src = measured_peak_gbs()
     spmm_avg_ms = prof["spmm_ms"] / max(prof["spmm_calls"], 1)
     achieved = (prof["spmm_bytes"] / 1e9) / (prof["spmm_ms"] / 1e3) if prof["spmm_ms"] > 0 else 0.0
-    line = {
-        "metric": "full-graph GCN training throughput", "value": value, "unit": "epochs/s", "n_gpus": world,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "f32" if dtype == B.F32 else "bf16", "data": "synthetic",
-        "config": {"workload": args.workload, "nodes": n, "nnz": info["nnz"], "in_d": w["in_d"], "hidden": w["hidden"],
+    traffic, traffic_src = NCU_SPMM_TRAFFIC.get(workload, (None, None))
+    ms_per_step = ms_total / steps
+    out = {
+        "value": whole_job_rate(world, steps, ms_total), "ms_per_step": ms_per_step,
+        "ms_per_step_median": statistics.median(step_ms), "ms_per_step_min": min(step_ms),
+        "dtype": "f32" if dtype == B.F32 else "bf16",
+        "config": {"workload": workload, "nodes": n, "nnz": info["nnz"], "in_d": w["in_d"], "hidden": w["hidden"],
                    "layers": w["layers"], "classes": w["classes"], "num_slices": w["p"], "use_ff": w["use_ff"],
                    "use_se": w["use_se"], "parallelism": "replicas only" if world > 1 else "single GPU",
-                   "l2": "working set per epoch is larger than L2 (no flush needed)", "final_loss": final_loss},
+                   "l2": "working set per epoch is larger than L2 (no flush needed)", "final_loss": final_loss,
+                   "input_aggregate_cached": bool(not w["use_ff"])},
         "clocks": clocks,
-        "e2e": {"value": world * args.steps / (e2e_ms / 1e3), "unit": "epochs/s",
-                "h2d_bytes_per_step": Xp.numel() * Xp.element_size() + yp.numel() * 4, "d2h_bytes_per_step": 4},
         "gpu_launches": int(prof["kernel_launches"]),
         "roofline": {"bound": "hbm", "kernel": "spmm_rows_kernel",
                      "achieved": achieved, "peak": peak, "peak_source": f"of {peak_src}", "unit": "GB/s",
-                     "frac": achieved / peak, "traffic": NCU_SPMM_TRAFFIC_BYTES.get(args.workload),
+                     "frac": achieved / peak, "traffic": traffic, "traffic_source": traffic_src,
                      "launches": int(prof["spmm_calls"]), "sampled_every": SPMM_SAMPLE_STRIDE, "avg_ms": spmm_avg_ms,
                      "algorithmic_bytes_per_launch": prof["spmm_bytes"] / max(prof["spmm_calls"], 1),
-                     "share_of_step": prof["spmm_ms"] * SPMM_SAMPLE_STRIDE / ms_total},
+                     "spmm_calls_per_step": int(per_epoch["spmm_calls"]),
+                     "share_of_step": spmm_avg_ms * per_epoch["spmm_calls"] / ms_per_step},
     }
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        cw = scaled_workload(args.workload, args.cpu_fraction)
-        times, threads = oracle_epochs(cw, 1, 0)
-        v = args.cpu_fraction / times[0]
-        sample = ("1 full epoch of the same workload" if args.cpu_fraction >= 1 else
-                  f"1 epoch of the same generator at {args.cpu_fraction:g} of the nodes and edges, scaled")
-        line["cpu_baseline"] = {"value": v, "unit": "epochs/s", "cores": threads, "kind": "oracle", "sample": sample}
+
+    if with_e2e:
+        # ---- end to end: ONE C-ABI call runs the epochs from host buffers.  Every epoch copies X and the
+        # labels from page-locked host memory again and returns its loss to the host; the library overlaps the
+        # copy for epoch e+1 with the kernels of epoch e (two staging buffers).
+        Xp = (torch.from_numpy(Xh).to(tdt) if dtype == B.BF16 else torch.from_numpy(Xh)).pin_memory()
+        yp = torch.from_numpy(yh).pin_memory()
+        n_e2e = max(steps, warmup, 1)
+        losses_host = torch.zeros(n_e2e, dtype=torch.float32).pin_memory()
+        losses_dev = torch.zeros(n_e2e, dtype=torch.float32, device=dev)
+        Xd = [torch.empty_like(X), torch.empty_like(X)]
+        yd = [torch.empty_like(y), torch.empty_like(y)]
+        params.copy_(params0); m1.zero_(); m2.zero_()
+
+        def e2e_run(first_epoch, count):
+            B.slicegcn_train_epochs_host(m, g, Xp, w["in_d"], yp, Xd[0], Xd[1], yd[0], yd[1], None, 0, params, grads, m1, m2,
+                                         B.make_opt_desc(1e-3, first_epoch, total_epochs), count, losses_dev, losses_host,
+                                         ws, ws_bytes, stream.cuda_stream)
+
+        e2e_run(0, max(warmup, 1))
+        barrier()
+        t0 = time.perf_counter()
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record(stream)
+        e2e_run(warmup, steps)          # returns after the last loss has reached the host
+        f1.record(stream)
+        barrier()
+        e2e_ms = mor(max(f0.elapsed_time(f1), 1e3 * (time.perf_counter() - t0)))
+        if not all(np.isfinite(losses_host[:steps].numpy())):
+            raise SystemExit("end-to-end run produced a non-finite loss")
+        out["e2e"] = {"value": whole_job_rate(world, steps, e2e_ms), "unit": "epochs/s",
+                      "h2d_bytes_per_step": Xp.numel() * Xp.element_size() + yp.numel() * 4, "d2h_bytes_per_step": 4}
     B.slicegcn_model_destroy(m)
     B.slicegcn_graph_destroy(g)
+    del ws, X, y, params, grads, m1, m2
+    torch.cuda.empty_cache()
+    return out
+
+
+def run_ours(args, rank: int, world: int, local_rank: int):
+    import torch
+    import torch.distributed as dist
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    steps = args.steps if args.steps > 0 else DEFAULT_STEPS[args.workload]
+    main_part = measure(args.workload, steps, args.warmup, world, local_rank, True, dist)
+    line = {"metric": "full-graph GCN training throughput", "value": main_part.pop("value"), "unit": "epochs/s",
+            "n_gpus": world, "steps": steps, "warmup": args.warmup, "ms_per_step": main_part.pop("ms_per_step"),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "data": "synthetic"}
+    line.update(main_part)
+    # the other model workloads, device-resident timing only (one line covers all three)
+    if world == 1 and not args.no_secondary:
+        line["secondary"] = []
+        for name in [k for k in ("citation", "social", "copurchase") if k != args.workload]:
+            part = measure(name, DEFAULT_STEPS[name] if args.steps <= 0 else min(DEFAULT_STEPS[name], max(args.steps, 5)),
+                           args.warmup, 1, local_rank, False)
+            line["secondary"].append({"workload": name, "value": part["value"], "unit": "epochs/s",
+                                      "ms_per_step": part["ms_per_step"], "ms_per_step_median": part["ms_per_step_median"],
+                                      "ms_per_step_min": part["ms_per_step_min"], "dtype": part["dtype"],
+                                      "nodes": part["config"]["nodes"], "nnz": part["config"]["nnz"],
+                                      "clocks": part["clocks"], "roofline": part["roofline"]})
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        frac = args.cpu_fraction if args.cpu_fraction > 0 else DEFAULT_CPU_FRACTION[args.workload]
+        cw = scaled_workload(args.workload, frac)
+        times, threads = oracle_epochs(cw, 1, 0)
+        v = frac / times[0]
+        sample = ("1 full epoch of the same workload" if frac >= 1 else
+                  f"1 epoch of the same generator at {frac:g} of the nodes and edges (n={cw['n']}), epochs/s scaled by {frac:g}")
+        line["cpu_baseline"] = {"value": v, "unit": "epochs/s", "cores": threads, "kind": "oracle", "sample": sample}
     if rank == 0:
         print(json.dumps(line), flush=True)
     if world > 1:
@@ -329,12 +387,13 @@ def run_ours(args, rank: int, world: int, local_rank: int):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=0, help="timed epochs (0: a default per workload that runs a second or two)")
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="citation", choices=sorted(synth.WORKLOADS))
-    ap.add_argument("--cpu-fraction", type=float, default=1.0, help="size of the oracle's timed sample")
+    ap.add_argument("--workload", default="copurchase", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--cpu-fraction", type=float, default=0.0, help="size of the oracle's timed sample (0: a default per workload)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-secondary", action="store_true", help="skip the device-resident timing of the other workloads")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     rank = int(os.environ.get("RANK", "0"))

@@ -182,6 +182,13 @@ typedef struct slicegcn_layer_desc {
 slicegcn_status_t slicegcn_layer_saved_bytes(const slicegcn_graph* g, const slicegcn_layer_desc* d, int64_t* bytes);
 slicegcn_status_t slicegcn_layer_workspace_bytes(const slicegcn_graph* g, const slicegcn_layer_desc* d,
                                                  int64_t* bytes);
+/* Where things lie inside `saved` after slicegcn_layer_forward, for inspection (tests read the ReLU decisions the
+ * forward pass took): the intermediate (A_hat H_in for an aggregate-first layer, H_in W_agg for a transform-first
+ * one; d->dtype, row-major) starts at byte *zt_offset with leading dimension *zt_ld elements and *zt_cols columns;
+ * the ReLU mask of Eq. 6 -- one byte per unit, 1 where b + aggregation > 0 -- starts at byte *mask_offset with
+ * leading dimension *mask_ld bytes and p*h_s columns.  Any output pointer may be NULL. */
+slicegcn_status_t slicegcn_layer_saved_layout(const slicegcn_graph* g, const slicegcn_layer_desc* d, int64_t* zt_offset,
+                                              int64_t* zt_ld, int32_t* zt_cols, int64_t* mask_offset, int64_t* mask_ld);
 /* Forward.  H_in [device, n x in_cols], H_out [device, n x p*h_s], both of d->dtype.
  * Errors: INVALID_ARG, ALLOC (buffers too small), UNSUPPORTED, CUDA. */
 slicegcn_status_t slicegcn_layer_forward(const slicegcn_graph* g, const slicegcn_layer_desc* d, const void* H_in,
@@ -223,6 +230,7 @@ typedef struct slicegcn_model_desc {
     int32_t dtype;             /* storage type of X and of every activation (bf16: also of dZ, see slicegcn_layer_backward);
                                   parameters, their gradients, logits and loss are always fp32 */
     int32_t order;             /* SLICEGCN_ORDER_AUTO or a forced order for every layer */
+    int32_t cache_input_aggregate;  /* 1: keep A_hat X of the first layer across calls (see slicegcn_train_epoch) */
 } slicegcn_model_desc;
 
 typedef struct slicegcn_opt_desc {
@@ -268,6 +276,12 @@ slicegcn_status_t slicegcn_train_workspace_bytes(const slicegcn_model* m, const 
  *   logits_out [device, fp32 n x num_classes, dense] or NULL
  *   loss_out [device, one float] or NULL: mean cross entropy BEFORE the update
  *   workspace [device], workspace_bytes >= slicegcn_train_workspace_bytes()
+ * Input aggregate cache (desc.cache_input_aggregate = 1; direct slicing with an aggregate-first first layer only):
+ * Algorithm 3 slices the features once, outside the epoch loop, so the first layer's aggregate A_hat X^i (Eq. 6,
+ * l = 1) is the same tensor in every epoch.  With the flag set the library keeps it in `workspace` and skips that
+ * aggregation whenever X, x_ld, the graph, `workspace` and `stream` are those of the previous call on this model.  The caller
+ * then promises that the CONTENTS of X and of `workspace` do not change between such calls; after changing them, call
+ * slicegcn_model_invalidate_caches().  The host-buffer entry points copy X anew every epoch and never use the cache.
  * Asynchronous on `stream`.  The model object keeps host-side bookkeeping of the converted weight operands it
  * has placed in `workspace` (they are converted again, in one launch, at the start of every call): calls on ONE model
  * must not run concurrently, and the contents of `workspace` are only meaningful to the library.
@@ -277,6 +291,9 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
                                        float* params, float* grads, float* adam_m, float* adam_v,
                                        const slicegcn_opt_desc* opt, float* logits_out, float* loss_out,
                                        void* workspace, int64_t workspace_bytes, void* stream);
+
+/* Forgets what the model object remembers about earlier calls (the input aggregate cache above).  Host only. */
+slicegcn_status_t slicegcn_model_invalidate_caches(const slicegcn_model* m);
 
 /* Evaluation pass: the forward half of the iteration above (Eq. 4-9) with the current parameters; writes the logits
  * [device, fp32 n x num_classes, dense] and nothing else a caller can see.  Same workspace as slicegcn_train_epoch.

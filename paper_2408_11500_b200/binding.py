@@ -29,8 +29,8 @@ DEVSTATUS_BAD_LABEL = 32
 EXPORTS = [
     "slicegcn_last_error", "slicegcn_slice_strategy", "slicegcn_graph_create", "slicegcn_graph_create_from_csr",
     "slicegcn_graph_info", "slicegcn_graph_export", "slicegcn_graph_device_status", "slicegcn_graph_destroy", "slicegcn_spmm_workspace_bytes",
-    "slicegcn_spmm", "slicegcn_spmm_static_scratch", "slicegcn_layer_saved_bytes", "slicegcn_layer_workspace_bytes", "slicegcn_layer_forward",
-    "slicegcn_layer_backward", "slicegcn_model_create", "slicegcn_model_destroy", "slicegcn_model_param_count",
+    "slicegcn_spmm", "slicegcn_spmm_static_scratch", "slicegcn_layer_saved_bytes", "slicegcn_layer_saved_layout", "slicegcn_layer_workspace_bytes", "slicegcn_layer_forward",
+    "slicegcn_layer_backward", "slicegcn_model_create", "slicegcn_model_destroy", "slicegcn_model_invalidate_caches", "slicegcn_model_param_count",
     "slicegcn_model_param_elems", "slicegcn_model_num_tensors", "slicegcn_model_tensor_info", "slicegcn_model_slices",
     "slicegcn_model_layer_order", "slicegcn_train_workspace_bytes", "slicegcn_train_epoch", "slicegcn_forward_logits", "slicegcn_train_epoch_host", "slicegcn_train_epochs_host", "slicegcn_profile_begin", "slicegcn_profile_begin_sampled",
     "slicegcn_profile_end",
@@ -53,7 +53,7 @@ class ModelDesc(ctypes.Structure):
     _fields_ = [("in_d", c_int32), ("hidden", c_int32), ("num_layers", c_int32), ("num_classes", c_int32),
                 ("num_slices", c_int32), ("slice_size_scale", c_double), ("slice_rule", c_int32), ("use_ff", c_int32),
                 ("use_se", c_int32), ("use_self", c_int32), ("use_b_self", c_int32), ("dtype", c_int32),
-                ("order", c_int32)]
+                ("order", c_int32), ("cache_input_aggregate", c_int32)]
 
 
 class OptDesc(ctypes.Structure):
@@ -204,6 +204,12 @@ def slicegcn_layer_saved_bytes(g, d: LayerDesc) -> int:
     return b.value
 
 
+def slicegcn_layer_saved_layout(g, d: LayerDesc) -> Dict[str, int]:
+    zo, zl, mo, ml, zc = c_int64(), c_int64(), c_int64(), c_int64(), c_int32()
+    _check(_lib.slicegcn_layer_saved_layout(g, byref(d), byref(zo), byref(zl), byref(zc), byref(mo), byref(ml)))
+    return {"zt_offset": zo.value, "zt_ld": zl.value, "zt_cols": zc.value, "mask_offset": mo.value, "mask_ld": ml.value}
+
+
 def slicegcn_layer_workspace_bytes(g, d: LayerDesc) -> int:
     b = c_int64()
     _check(_lib.slicegcn_layer_workspace_bytes(g, byref(d), byref(b)))
@@ -228,9 +234,9 @@ def slicegcn_layer_backward(g, d: LayerDesc, H_in, saved, dH_out, dout_ld: int, 
 def slicegcn_model_create(in_d: int, hidden: int, num_layers: int, num_classes: int, num_slices: int = 1,
                           slice_size_scale: float = 1.0, slice_rule: int = RULE_CEIL, use_ff: bool = False,
                           use_se: bool = False, use_self: bool = True, use_b_self: bool = False, dtype: int = F32,
-                          order: int = ORDER_AUTO) -> c_void_p:
+                          order: int = ORDER_AUTO, cache_input_aggregate: bool = False) -> c_void_p:
     d = ModelDesc(in_d, hidden, num_layers, num_classes, num_slices, slice_size_scale, slice_rule, int(use_ff),
-                  int(use_se), int(use_self), int(use_b_self), dtype, order)
+                  int(use_se), int(use_self), int(use_b_self), dtype, order, int(cache_input_aggregate))
     h = c_void_p()
     _check(_lib.slicegcn_model_create(byref(d), byref(h)))
     return h
@@ -238,6 +244,10 @@ def slicegcn_model_create(in_d: int, hidden: int, num_layers: int, num_classes: 
 
 def slicegcn_model_destroy(m) -> None:
     _check(_lib.slicegcn_model_destroy(m))
+
+
+def slicegcn_model_invalidate_caches(m) -> None:
+    _check(_lib.slicegcn_model_invalidate_caches(m))
 
 
 def slicegcn_model_param_count(m) -> int:

@@ -171,9 +171,10 @@ slicegcn_status_t gemm_groups(const GemmArgs& a, bool sequential, cudaStream_t s
     return SLICEGCN_OK;
 }
 
+// aggregate_cached: the saved intermediate already holds A_hat H_in from an earlier call (aggregate-first layers only)
 slicegcn_status_t layer_forward_impl(const slicegcn_graph* g, const slicegcn_layer_desc* d, const LayerPlan& L,
                                      const void* H_in, void* H_out, void* saved, void* ws, int64_t ws_bytes,
-                                     cudaStream_t st) {
+                                     cudaStream_t st, bool aggregate_cached = false) {
     char* zt = static_cast<char*>(saved);
     uint8_t* mask = reinterpret_cast<uint8_t*>(zt + L.zt_bytes);
     if (ws_bytes < layer_fwd_ws_bytes(g, L)) SGCN_FAIL(SLICEGCN_ERR_ALLOC, "layer_forward: workspace too small");
@@ -213,7 +214,8 @@ slicegcn_status_t layer_forward_impl(const slicegcn_graph* g, const slicegcn_lay
 
     if (L.order == SLICEGCN_AGG_FIRST) {
         // Z = A_hat H_in over every input column once; slices then read their column ranges of Z
-        SGCN_TRY(spmm_run(g, false, L.dtype, L.dtype, H_in, L.in_ld, zt, L.zt_ld, L.in_cols, nullptr, part, part_bytes, st));
+        if (!aggregate_cached)
+            SGCN_TRY(spmm_run(g, false, L.dtype, L.dtype, H_in, L.in_ld, zt, L.zt_ld, L.in_cols, nullptr, part, part_bytes, st));
         if (d->W_self) {
             // one pass: H_out = ReLU(Z W_agg + b) + H_in W_self + b_self + E (two accumulators)
             GemmArgs both = self;
@@ -531,6 +533,16 @@ struct slicegcn_model {
     // weight images of the tensor-core GEMMs, kept across the epochs of a training run (host bookkeeping only;
     // the images live in the caller's workspace).  Makes training calls on one model non-reentrant.
     mutable sgcn::TcImageCache* image_cache = nullptr;
+    // input aggregate cache: what the first layer's saved A_hat X in the caller's workspace was computed from
+    struct InputAggregateKey {
+        const void* X = nullptr;
+        int64_t x_ld = 0;
+        const void* graph = nullptr;
+        const void* workspace = nullptr;
+        const void* stream = nullptr;
+        bool valid = false;
+    };
+    mutable InputAggregateKey zkey;
     ~slicegcn_model() { sgcn::tc_image_cache_destroy(image_cache); }
 
     int64_t add(const std::string& name, int d0, int d1, int d2) {
@@ -741,6 +753,18 @@ slicegcn_status_t slicegcn_layer_saved_bytes(const slicegcn_graph* g, const slic
     return SLICEGCN_OK;
 }
 
+slicegcn_status_t slicegcn_layer_saved_layout(const slicegcn_graph* g, const slicegcn_layer_desc* d, int64_t* zt_offset,
+                                              int64_t* zt_ld, int32_t* zt_cols, int64_t* mask_offset, int64_t* mask_ld) {
+    LayerPlan pl;
+    SGCN_TRY(make_plan(g, d, &pl));
+    if (zt_offset) *zt_offset = 0;
+    if (zt_ld) *zt_ld = pl.zt_ld;
+    if (zt_cols) *zt_cols = pl.zt_cols;
+    if (mask_offset) *mask_offset = pl.zt_bytes;
+    if (mask_ld) *mask_ld = pl.mask_ld;
+    return SLICEGCN_OK;
+}
+
 slicegcn_status_t slicegcn_layer_workspace_bytes(const slicegcn_graph* g, const slicegcn_layer_desc* d, int64_t* bytes) {
     if (!bytes) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "bytes is NULL");
     LayerPlan pl;
@@ -825,6 +849,12 @@ slicegcn_status_t slicegcn_model_create(const slicegcn_model_desc* desc, slicegc
 
 slicegcn_status_t slicegcn_model_destroy(slicegcn_model* m) {
     delete m;
+    return SLICEGCN_OK;
+}
+
+slicegcn_status_t slicegcn_model_invalidate_caches(const slicegcn_model* m) {
+    if (!m) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "model is NULL");
+    m->zkey.valid = false;
     return SLICEGCN_OK;
 }
 
@@ -978,8 +1008,17 @@ static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, 
         h0 = E.xff;
         ld0 = E.ld_x0;
     }
+    // Input aggregate cache: with direct slicing the first layer's A_hat X does not change from epoch to epoch
+    // (Algorithm 3 slices outside the epoch loop); reuse what the previous call left in the workspace.
+    const bool z_cacheable = D.cache_input_aggregate && !D.use_ff && m->order[0] == SLICEGCN_AGG_FIRST;
+    const bool z_cached = z_cacheable && m->zkey.valid && m->zkey.X == X && m->zkey.x_ld == x_ld && m->zkey.graph == g &&
+                          m->zkey.workspace == workspace && m->zkey.stream == stream;
+    m->zkey.valid = false;   // until this call has queued the first layer
     const bool repacked = m->repack_input();
-    if (repacked) {   // slicing (Algorithm 2) as a copy: slices side by side at aligned starts, zero padding
+    if (repacked && z_cached) {   // the repacked copy is still in the workspace as well
+        h0 = E.xrep;
+        ld0 = E.ld_xrep;
+    } else if (repacked) {   // slicing (Algorithm 2) as a copy: slices side by side at aligned starts, zero padding
         SGCN_TRY(repack_slices_run(n, p, m->starts, m->slice_width, m->repack_pad(), X, x_ld, D.dtype, E.xrep, E.ld_xrep, st));
         h0 = E.xrep;
         ld0 = E.ld_xrep;
@@ -1007,7 +1046,15 @@ static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, 
                 SGCN_CUDA(cudaMemsetAsync(E.saved[l], 0, plans[l].zt_bytes, st));
             }
         }
-        SGCN_TRY(layer_forward_impl(g, &descs[l], plans[l], hin, E.H[l], E.saved[l], E.ws, E.ws_bytes, st));
+        SGCN_TRY(layer_forward_impl(g, &descs[l], plans[l], hin, E.H[l], E.saved[l], E.ws, E.ws_bytes, st, l == 0 && z_cached));
+        if (l == 0 && z_cacheable) {
+            m->zkey.X = X;
+            m->zkey.x_ld = x_ld;
+            m->zkey.graph = g;
+            m->zkey.workspace = workspace;
+            m->zkey.stream = stream;
+            m->zkey.valid = true;
+        }
         hin = E.H[l];
     }
     const int HW = p * m->h_s;
@@ -1245,6 +1292,7 @@ slicegcn_status_t slicegcn_train_epoch_host(const slicegcn_model* m, const slice
     cudaStream_t st = (cudaStream_t)stream;
     const int64_t n = g->n;
     SGCN_TRY(check_labels_host(labels_host, n, m->desc.num_classes, "train_epoch_host"));
+    m->zkey.valid = false;   // X is copied anew: nothing computed from the staging buffer's old contents may be reused
     SGCN_CUDA(cudaMemcpyAsync(X_stage, X_host, (size_t)(n * x_ld) * esize(m->desc.dtype), cudaMemcpyHostToDevice, st));
     SGCN_CUDA(cudaMemcpyAsync(labels_stage, labels_host, (size_t)n * sizeof(int32_t), cudaMemcpyHostToDevice, st));
     SGCN_TRY(slicegcn_train_epoch(m, g, X_stage, x_ld, labels_stage, train_idx, n_train, params, grads, adam_m, adam_v, opt, nullptr,
@@ -1307,6 +1355,7 @@ slicegcn_status_t slicegcn_train_epochs_host(const slicegcn_model* m, const slic
             SGCN_CUDA(cudaStreamWaitEvent(st, ready[b], 0));
             slicegcn_opt_desc o = *opt;
             o.epoch = opt->epoch + e;
+            m->zkey.valid = false;   // the staging buffer holds a fresh copy of X
             SGCN_TRY(slicegcn_train_epoch(m, g, xs[b], x_ld, ys[b], train_idx, n_train, params, grads, adam_m, adam_v, &o, nullptr,
                                           losses_dev + e, workspace, workspace_bytes, stream));
             SGCN_CUDA(cudaEventRecord(done[b], st));

@@ -92,7 +92,6 @@ struct SpmmParams {
     int64_t mask_ld;
     int32_t relu;
     int32_t accumulate;
-    int* fault;      // device status word (set when a bounded wait of the bulk-copy kernel runs out)
 };
 
 template <typename TO, int V, bool EPI>
@@ -517,292 +516,6 @@ __device__ __forceinline__ void spmm_segment_block(const SpmmParams& p, const in
     }
 }
 
-// ---- rows of 512 bytes and more: gathers by the bulk-copy engine ------------------------------------------------
-// The register-gather loop above keeps 32 warps x 4 loads x 512 bytes = 64 KB per SM in flight, which is all the
-// register file allows, and that (Little's law against ~1 us of loaded memory latency) is what bounds it at ~10-11 TB/s
-// of gathers.  For rows of 512 bytes and more a warp instead asks the bulk-copy engine for whole neighbor rows: one
-// cp.async.bulk per neighbor into a ring of shared-memory stages (completion counted on one mbarrier per stage), so the
-// bytes in flight live in shared memory (up to ~200 KB per SM) and cost no registers and one instruction per row.
-// A warp is its own producer and consumer: while it accumulates stage q from shared memory, stages q+1 .. q+NS-1 are in
-// flight.  Work items, row bookkeeping and the deterministic finish of split rows are those of the kernels above.
-constexpr int kBulkWaitSpins = 1 << 22;
-constexpr int kStatusSpmmWait = 9;
-
-__device__ __forceinline__ uint32_t sm_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ bool bulk_bar_wait(uint64_t* bar, uint32_t parity) {   // bounded: ~2 s, then gives up
-    const long long t0 = clock64();
-    for (int i = 0; i < kBulkWaitSpins; ++i) {
-        uint32_t ok;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(ok)
-            : "r"(sm_u32(bar)), "r"(parity)
-            : "memory");
-        if (ok) return true;
-        if (clock64() - t0 > 4000000000LL) break;
-    }
-    return false;
-}
-
-template <int NS, int STAGE>
-struct BulkSmem {
-    static constexpr int kMaxRows = STAGE / 512 > 0 ? STAGE / 512 : 1;   // rows per stage at the narrowest row this kernel takes
-    alignas(128) unsigned char stage[NS][STAGE];
-    float dd[NS][kMaxRows];                                // 1/sqrt(deg) of the neighbor behind each staged row
-    alignas(8) uint64_t bar[NS];
-};
-
-// Streams the neighbor rows of entries [e0, e1) through the ring and hands (1/sqrt(deg_j), the lane's C 16-byte
-// chunks of row j) to `f`, entry by entry in CSR order.  Returns false when a wait ran out.
-template <typename TI, int C, int NS, int STAGE, bool LSU, typename F>
-__device__ __forceinline__ bool bulk_stream(const SpmmParams& p, BulkSmem<NS, STAGE>& sm, uint32_t (&uses)[NS], const int e0,
-                                            const int e1, const int R, const uint32_t rowbytes, F&& f) {
-    const int lane = threadIdx.x & 31;
-    const int Q = (e1 - e0 + R - 1) / R;
-    const unsigned char* Xb = static_cast<const unsigned char*>(p.X);
-    const uint64_t ldxb = (uint64_t)p.ldx * sizeof(TI);
-    // neighbor ids two rounds ahead, their 1/sqrt(deg) one round ahead (lane u serves entry u of a round)
-    int j0 = 0, j1 = 0, j2 = 0;
-    float d0 = 0.f, d1 = 0.f;
-    auto ld_j = [&](int q) { const int e = e0 + q * R + lane; return (lane < R && e < e1) ? __ldg(p.colidx + e) : 0; };
-    j0 = ld_j(0);
-    j1 = ld_j(1);
-    d0 = __ldg(p.dinv + j0);
-    auto issue = [&](int q) {   // uses (j0, d0) = round q; rotates the prefetch registers
-        const int s = q % NS;
-        const int cnt = min(R, e1 - (e0 + q * R));
-        j2 = ld_j(q + 2);
-        d1 = __ldg(p.dinv + j1);
-        if (LSU) {
-            // per-lane 16-byte asynchronous copies (load/store unit path): lane l moves chunks l, l+32, ... of every row
-            if (q < Q) {
-                if (lane < cnt) sm.dd[s][lane] = d0;
-                for (int u = 0; u < cnt; ++u) {
-                    const uint32_t ju = (uint32_t)__shfl_sync(0xffffffffu, j0, u);
-                    const unsigned char* src = Xb + (uint64_t)ju * ldxb;
-                    const uint32_t dst = sm_u32(&sm.stage[s][0]) + (uint32_t)u * rowbytes;
-#pragma unroll
-                    for (int c = 0; c < C; ++c) {
-                        const int ch = lane + c * 32;
-                        if (ch < p.nch)
-                            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + (uint32_t)ch * 16u), "l"(src + (size_t)ch * 16) : "memory");
-                    }
-                }
-            }
-            asm volatile("cp.async.commit_group;" ::: "memory");
-        } else {
-            if (lane == 0)
-                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(sm_u32(&sm.bar[s])), "r"((uint32_t)cnt * rowbytes)
-                             : "memory");
-            __syncwarp();
-            if (lane < cnt) {
-                sm.dd[s][lane] = d0;
-                asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                                 sm_u32(&sm.stage[s][0]) + (uint32_t)lane * rowbytes),
-                             "l"(Xb + (uint64_t)(uint32_t)j0 * ldxb), "r"(rowbytes), "r"(sm_u32(&sm.bar[s]))
-                             : "memory");
-            }
-        }
-        j0 = j1;
-        d0 = d1;
-        j1 = j2;
-    };
-    const int ahead = NS - 1;
-    if (LSU) {
-#pragma unroll 1
-        for (int q = 0; q < ahead; ++q) issue(q);          // rounds past the end commit empty groups: the group count per
-    } else {                                               // iteration stays fixed, so one wait_group depth serves all
-        for (int q = 0; q < ahead && q < Q; ++q) issue(q);
-    }
-    for (int q = 0; q < Q; ++q) {
-        if (LSU || q + ahead < Q) issue(q + ahead);   // into the stage round q-1 left (its reads are behind the __syncwarp below)
-        const int s = q % NS;
-        if (LSU) {
-            asm volatile("cp.async.wait_group %0;" ::"n"(NS - 1) : "memory");
-            __syncwarp();   // every lane's copies of round q have landed
-        } else {
-            if (!bulk_bar_wait(&sm.bar[s], uses[s] & 1u)) return false;
-            uses[s]++;
-        }
-        const int cnt = min(R, e1 - (e0 + q * R));
-        const unsigned char* rows = &sm.stage[s][0] + (uint32_t)min(lane, p.nch - 1) * 16u;
-#pragma unroll 2
-        for (int u = 0; u < cnt; ++u) {
-            uint4 raw[C];
-#pragma unroll
-            for (int c = 0; c < C; ++c) {
-                const int off = (lane + c * 32 < p.nch) ? c * 512 : 0;   // lanes past the row re-read a valid chunk, never store
-                raw[c] = *reinterpret_cast<const uint4*>(rows + (uint32_t)u * rowbytes + off);
-            }
-            f(sm.dd[s][u], raw);
-        }
-        __syncwarp();
-    }
-    if (LSU) asm volatile("cp.async.wait_group 0;" ::: "memory");
-    return true;
-}
-
-template <typename TI, typename TO, int C, int NS, int STAGE, bool LSU, bool EPI>
-__global__ void __launch_bounds__(32) spmm_bulk_kernel(const SpmmParams p, const int seg_blocks) {
-    constexpr int V = Vec<TI>::V;
-    extern __shared__ unsigned char bulk_smem_raw[];
-    BulkSmem<NS, STAGE>& sm = *reinterpret_cast<BulkSmem<NS, STAGE>*>(
-        (reinterpret_cast<uintptr_t>(bulk_smem_raw) + 127) & ~(uintptr_t)127);
-    const int lane = threadIdx.x;
-    if (!LSU && lane == 0) {
-#pragma unroll
-        for (int i = 0; i < NS; ++i) asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(sm_u32(&sm.bar[i])), "r"(1));
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    __syncwarp();
-    uint32_t uses[NS];
-#pragma unroll
-    for (int i = 0; i < NS; ++i) uses[i] = 0;
-    const uint32_t rowbytes = (uint32_t)p.nch * 16u;
-    const int R = STAGE / (int)rowbytes;
-    float acc[C][V];
-#pragma unroll
-    for (int c = 0; c < C; ++c)
-#pragma unroll
-        for (int e = 0; e < V; ++e) acc[c][e] = 0.f;
-    auto accumulate = [&](float dd, const uint4 (&raw)[C]) {
-#pragma unroll
-        for (int c = 0; c < C; ++c) {
-            float fv[V];
-            Vec<TI>::unpack(raw[c], fv);
-#pragma unroll
-            for (int e = 0; e < V; ++e) acc[c][e] = fmaf(dd, fv[e], acc[c][e]);
-        }
-    };
-    bool ok = true;
-    if ((int)blockIdx.x < seg_blocks) {
-        // ---- one 128-entry segment of a long row
-        const int vseg = blockIdx.x;
-        if (vseg >= p.n_seg) return;
-        const int seg = __ldg(p.seg_order + vseg);
-        const int li = __ldg(p.seg_row + seg);
-        const int row = __ldg(p.long_rows + li);
-        const int start = __ldg(p.rowptr + row) + (seg - __ldg(p.seg_ptr + li)) * kSegment;
-        const int end = min(__ldg(p.rowptr + row + 1), start + kSegment);
-        ok = bulk_stream<TI, C, NS, STAGE, LSU>(p, sm, uses, start, end, R, rowbytes, accumulate);
-        if (!ok) {
-            if (lane == 0 && p.fault) atomicExch(p.fault, kStatusSpmmWait);
-            return;
-        }
-        const int s0 = __ldg(p.seg_ptr + li), s1 = __ldg(p.seg_ptr + li + 1);
-        if (s1 - s0 == 1) {
-            const float di = __ldg(p.dinv + row);
-#pragma unroll
-            for (int c = 0; c < C; ++c) {
-                const int chunk = lane + c * 32;
-                if (chunk < p.nch) finish_chunk<TO, V, EPI>(p, row, chunk, di, acc[c]);
-            }
-            return;
-        }
-        // several segments: leave the partial row; the warp that arrives last at the row's counter sums the row's
-        // partial rows in segment order (whichever warp that is, the order of the additions is the same)
-        const int pstride = p.nch * V;
-        float* out = p.partial + (int64_t)seg * pstride;
-#pragma unroll
-        for (int c = 0; c < C; ++c) {
-            const int chunk = lane + c * 32;
-            if (chunk < p.nch) {
-#pragma unroll
-                for (int e = 0; e < V; e += 4)
-                    *reinterpret_cast<float4*>(out + chunk * V + e) = make_float4(acc[c][e], acc[c][e + 1], acc[c][e + 2], acc[c][e + 3]);
-            }
-        }
-        int last = 0;
-        __syncwarp();
-        if (lane == 0) {
-            __threadfence();
-            last = atomicAdd(p.seg_done + li, 1) == s1 - s0 - 1;
-        }
-        last = __shfl_sync(0xffffffffu, last, 0);
-        if (!last) return;
-        __threadfence();
-#pragma unroll
-        for (int c = 0; c < C; ++c)
-#pragma unroll
-            for (int e = 0; e < V; ++e) acc[c][e] = 0.f;
-#pragma unroll 4
-        for (int sg = s0; sg < s1; ++sg) {
-            const float* src = p.partial + (int64_t)sg * pstride;
-#pragma unroll
-            for (int c = 0; c < C; ++c) {
-                const int chunk = min(lane + c * 32, p.nch - 1);
-#pragma unroll
-                for (int e = 0; e < V; e += 4) {
-                    const float4 v = __ldcg(reinterpret_cast<const float4*>(src + chunk * V + e));
-                    acc[c][e] += v.x;
-                    acc[c][e + 1] += v.y;
-                    acc[c][e + 2] += v.z;
-                    acc[c][e + 3] += v.w;
-                }
-            }
-        }
-        const float di = __ldg(p.dinv + row);
-#pragma unroll
-        for (int c = 0; c < C; ++c) {
-            const int chunk = lane + c * 32;
-            if (chunk < p.nch) finish_chunk<TO, V, EPI>(p, row, chunk, di, acc[c]);
-        }
-        return;
-    }
-    // ---- one row-aligned chunk of short rows
-    const int64_t chunk_id = (int64_t)blockIdx.x - seg_blocks;
-    if (chunk_id >= p.n_chunks) return;
-    const int r0 = __ldg(p.chunk_row + chunk_id);
-    const int r1 = __ldg(p.chunk_row + chunk_id + 1);
-    if (r0 >= r1) return;
-    const int k0 = __ldg(p.rowptr + r0), k1 = __ldg(p.rowptr + r1);
-    // row ends and 1/sqrt(deg) of 32 consecutive rows at a time, handed out by shuffles
-    int rbase = r0, rp_l = 0;
-    float di_l = 0.f;
-    auto load_meta = [&]() {
-        const int r = rbase + lane;
-        rp_l = (r < r1) ? __ldg(p.rowptr + r + 1) : k1;
-        di_l = (r < r1) ? __ldg(p.dinv + r) : 0.f;
-    };
-    load_meta();
-    int row = r0;
-    int row_end = __shfl_sync(0xffffffffu, rp_l, 0);
-    if (row_end - k0 > kLongRow) return;   // a long row sits alone in its chunk: left to its segments
-    int kk = k0;
-    auto close_row = [&]() {
-        const float di = __shfl_sync(0xffffffffu, di_l, row - rbase);
-#pragma unroll
-        for (int c = 0; c < C; ++c) {
-            const int ch = lane + c * 32;
-            if (ch < p.nch) finish_chunk<TO, V, EPI>(p, row, ch, di, acc[c]);
-#pragma unroll
-            for (int e = 0; e < V; ++e) acc[c][e] = 0.f;
-        }
-        ++row;
-        if (row < r1) {
-            if (row - rbase == 32) {
-                rbase = row;
-                load_meta();
-            }
-            row_end = __shfl_sync(0xffffffffu, rp_l, row - rbase);
-        } else {
-            row_end = -1;
-        }
-    };
-    ok = bulk_stream<TI, C, NS, STAGE, LSU>(p, sm, uses, k0, k1, R, rowbytes, [&](float dd, const uint4 (&raw)[C]) {
-        while (kk == row_end) close_row();   // rows ending here, rows without entries included
-        accumulate(dd, raw);
-        ++kk;
-    });
-    if (!ok) {
-        if (lane == 0 && p.fault) atomicExch(p.fault, kStatusSpmmWait);
-        return;
-    }
-    while (row < r1 && kk == row_end) close_row();
-}
-
 // One launch for both kinds of work: the first seg_blocks CTAs reduce the segments of the long rows
 // (they are the heaviest items, so they start first), the others the row chunks.
 template <typename TI, typename TO, int L, int C, bool EPI>
@@ -883,66 +596,6 @@ __global__ void __launch_bounds__(256) spmm_scalar_kernel(const SpmmParams p) {
     }
 }
 
-// Which gather loop serves rows of 512 bytes and more: 1 (default) the bulk-copy ring, 0 the register loop.
-// SLICEGCN_SPMM_BULK overrides it (benchmark A/B); SLICEGCN_SPMM_RING picks the ring shape (0..3, see bulk_launch).
-static int bulk_mode() {
-    static const int mode = [] {
-        const char* e = getenv("SLICEGCN_SPMM_BULK");
-        return e ? atoi(e) : 1;
-    }();
-    return mode;
-}
-static int bulk_ring() {
-    static const int ring = [] {
-        const char* e = getenv("SLICEGCN_SPMM_RING");
-        return e ? atoi(e) : 0;
-    }();
-    return ring;
-}
-
-template <typename TI, typename TO, int C, int NS, int STAGE, bool LSU>
-slicegcn_status_t bulk_launch_cfg(const SpmmParams& q, bool epi, unsigned grid, int seg_blocks, cudaStream_t st) {
-    const int smem = (int)sizeof(BulkSmem<NS, STAGE>) + 128;
-    if (epi) {
-        auto k = spmm_bulk_kernel<TI, TO, C, NS, STAGE, LSU, true>;
-        static bool set = false;
-        if (!set) {
-            SGCN_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-            set = true;
-        }
-        k<<<grid, 32, smem, st>>>(q, seg_blocks);
-    } else {
-        auto k = spmm_bulk_kernel<TI, TO, C, NS, STAGE, LSU, false>;
-        static bool set = false;
-        if (!set) {
-            SGCN_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-            set = true;
-        }
-        k<<<grid, 32, smem, st>>>(q, seg_blocks);
-    }
-    SGCN_LAUNCH_CHECK();
-    count_launch();
-    return SLICEGCN_OK;
-}
-
-template <typename TI, typename TO, int C>
-slicegcn_status_t bulk_launch(const SpmmParams& q, bool epi, unsigned grid, int seg_blocks, cudaStream_t st) {
-    if (bulk_mode() == 2) {   // per-lane asynchronous copies
-        switch (bulk_ring()) {
-            case 1: return bulk_launch_cfg<TI, TO, C, 4, 4096, true>(q, epi, grid, seg_blocks, st);
-            case 2: return bulk_launch_cfg<TI, TO, C, 2, 8192, true>(q, epi, grid, seg_blocks, st);
-            case 3: return bulk_launch_cfg<TI, TO, C, 3, 4096, true>(q, epi, grid, seg_blocks, st);
-            case 4: return bulk_launch_cfg<TI, TO, C, 3, 2048, true>(q, epi, grid, seg_blocks, st);
-            case 5: return bulk_launch_cfg<TI, TO, C, 4, 2048, true>(q, epi, grid, seg_blocks, st);
-            default: return bulk_launch_cfg<TI, TO, C, 3, 8192, true>(q, epi, grid, seg_blocks, st);
-        }
-    }
-    switch (bulk_ring()) {
-        case 2: return bulk_launch_cfg<TI, TO, C, 2, 8192, false>(q, epi, grid, seg_blocks, st);
-        default: return bulk_launch_cfg<TI, TO, C, 3, 8192, false>(q, epi, grid, seg_blocks, st);
-    }
-}
-
 template <typename TI, typename TO, int L, int C>
 slicegcn_status_t launch_lc(const SpmmParams& p, bool epi, cudaStream_t st) {
     constexpr int RPW = 32 / L;
@@ -956,9 +609,6 @@ slicegcn_status_t launch_lc(const SpmmParams& p, bool epi, cudaStream_t st) {
     SpmmParams q = p;
     if (!in_kernel) q.seg_done = nullptr;
     if (q.n_seg > 0 && in_kernel) SGCN_CUDA(cudaMemsetAsync(q.seg_done, 0, sizeof(int32_t) * (size_t)q.n_long, st));
-    if constexpr (L == 32) {
-        if (bulk_mode() != 0 && q.nch >= 32) return bulk_launch<TI, TO, C>(q, epi, (unsigned)(blocks + seg_blocks), seg_blocks, st);
-    }
     if (epi)
         spmm_rows_kernel<TI, TO, L, C, true><<<(unsigned)(blocks + seg_blocks), kRowsWarps * 32, 0, st>>>(q, seg_blocks);
     else
@@ -1079,7 +729,6 @@ slicegcn_status_t spmm_run(const slicegcn_graph* g, bool transpose, int in_dtype
                         (ldy * osz) % 16 == 0 && (int64_t)p.nch * V <= ldx;
     p.n_chunks = v.n_chunks;
     p.chunk_row = v.chunk_row;
-    p.fault = g->fault;
     if (vec_ok) {
         p.n_long = v.n_long;
         p.n_seg = v.n_seg;

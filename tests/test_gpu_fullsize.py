@@ -1,0 +1,231 @@
+"""Full-size parity for the large workloads: the dense-social graph (232,965 nodes, 114.8 M stored entries), the
+co-purchase graph (2,449,029 nodes, 126.2 M entries, bf16 storage) and the R-MAT sweep graph at scale 20 with
+relabeled ids -- each at its own size, in the launch configuration the benchmark times.
+
+Per workload: the CSR bit-exact against the oracle's; the aggregation (Eq. 6's neighbor sum, forward and transposed)
+at the workload's own widths and storage types on Gaussian operands, compared with exact oracle values on a seeded
+sample of >= 10^4 rows that includes the 100 longest; and for the two model workloads one hidden layer (Eq. 6-7)
+forward and backward at that size: every output element, the ReLU decisions the kernel took, every weight gradient,
+and the input gradient on the row sample.
+"""
+import time
+
+import numpy as np
+import pytest
+
+from oracle import slicegcn_oracle as orc
+from paper_2408_11500_b200 import synth
+
+from helpers import rel_inf
+
+pytestmark = pytest.mark.gpu
+
+RELU_BAND = 1e-6     # |pre-activation| <= RELU_BAND * max|pre-activation|: the sign is within fp32 rounding noise
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2408_11500_b200 import binding
+    return binding
+
+
+@pytest.fixture(scope="module")
+def torch():
+    import torch
+    return torch
+
+
+def _row_sample(og, k=10000, seed=0):
+    """>= 10^4 seeded rows plus the 100 longest (hub rows with hundreds of segments)."""
+    longest = np.argsort(og.deg, kind="stable")[-100:]
+    rnd = np.random.default_rng(seed).choice(og.n, size=min(k, og.n), replace=False)
+    return np.unique(np.concatenate([longest, rnd])).astype(np.int64)
+
+
+def _check_csr(B, g, og):
+    ex = B.slicegcn_graph_export(g)
+    assert np.array_equal(ex["rowptr"], og.rowptr) and np.array_equal(ex["colidx"], og.colidx)
+    assert np.array_equal(ex["deg"], og.deg)
+    assert np.array_equal(ex["dinv"].view(np.uint32), orc.dinv_f32(og.deg).view(np.uint32))
+    info = B.slicegcn_graph_info(g)
+    assert info["nnz"] == og.nnz and info["symmetric"] == og.symmetric
+
+
+def _spmm_case(B, torch, g, og, rows, width, in_dt, out_dt, transpose, seed):
+    """One aggregation at full size on a Gaussian operand; sampled rows against the oracle.  The graphs here are
+    symmetrized (asserted), so A_hat^T = A_hat and the oracle's row-sampled gather form serves both directions."""
+    assert og.symmetric
+    n = og.n
+    tdt = {B.F32: torch.float32, B.BF16: torch.bfloat16}
+    X = torch.from_numpy(synth.gaussian_features(n, width, seed=seed)).cuda().to(tdt[in_dt]).contiguous()
+    Y = torch.full((n, width), float("nan"), dtype=tdt[out_dt], device="cuda")
+    wsb = B.slicegcn_spmm_workspace_bytes(g, width)
+    ws = torch.empty(max(wsb, 16), dtype=torch.uint8, device="cuda")
+    B.slicegcn_spmm(g, int(transpose), in_dt, out_dt, X, width, Y, width, width, ws, wsb, torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    ridx = torch.from_numpy(rows).cuda()
+    got = Y[ridx].float().cpu().numpy().astype(np.float64)
+    assert not bool(torch.isnan(Y.float().sum()).item())          # every row was written
+    want = orc.spmm(og, X.float().cpu().numpy().astype(np.float64), rows=rows)
+    if out_dt == B.F32:
+        err = rel_inf(got, want)
+        assert err <= 2e-6, (width, in_dt, out_dt, transpose, err)
+    else:   # one bf16 rounding of the fp32-accumulated result
+        assert np.all(np.abs(got - want) <= 2 ** -8 * np.abs(want) + 1e-5 * np.abs(want).max()), (width, transpose)
+    del X, Y, ws
+    torch.cuda.empty_cache()
+
+
+def _hidden_layer_case(B, torch, g, og, rows, p, h_s, dtype, use_e, seed, report):
+    """One hidden layer of the model (input = the p*h_s-wide output of the layer below, aggregate first, W_self,
+    optional slice encoding) forward and backward at full size."""
+    n, W = og.n, p * h_s
+    bf16 = dtype == B.BF16
+    rnd = orc.round_bf16 if bf16 else orc.identity
+    tol = 2e-2 if bf16 else 1e-4
+    rng = np.random.default_rng(seed)
+    tdt = torch.bfloat16 if bf16 else torch.float32
+    Hd = torch.from_numpy(synth.gaussian_features(n, W, seed=seed)).cuda().to(tdt).contiguous()
+    dHd = torch.from_numpy(synth.gaussian_features(n, W, seed=seed + 1)).cuda().contiguous()
+    Wa = (rng.standard_normal((p, h_s, h_s)) * 0.2).astype(np.float32)
+    Ws = (rng.standard_normal((p, h_s, h_s)) * 0.2).astype(np.float32)
+    b = (rng.standard_normal((p, h_s)) * 0.2).astype(np.float32)
+    E = (rng.standard_normal((p, h_s)) * 0.2).astype(np.float32)
+    cu = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    Wad, Wsd, bd, Ed = cu(Wa), cu(Ws), cu(b), cu(E)
+    starts = [i * h_s for i in range(p)]
+    desc = B.make_layer_desc(p, starts, h_s, W, W, h_s, W, dtype, B.AGG_FIRST, Wad, Wsd, bd, None, Ed if use_e else None)
+    sb, wb = B.slicegcn_layer_saved_bytes(g, desc), B.slicegcn_layer_workspace_bytes(g, desc)
+    lay = B.slicegcn_layer_saved_layout(g, desc)
+    saved = torch.empty(sb, dtype=torch.uint8, device="cuda")
+    ws = torch.empty(max(wb, 16), dtype=torch.uint8, device="cuda")
+    out = torch.full((n, W), float("nan"), dtype=tdt, device="cuda")
+    st = torch.cuda.current_stream().cuda_stream
+    B.slicegcn_layer_forward(g, desc, Hd, out, saved, sb, ws, wb, st)
+    dHin = torch.full((n, W), float("nan"), device="cuda")
+    gWa, gWs, gb, gE = torch.empty_like(Wad), torch.empty_like(Wsd), torch.empty_like(bd), torch.empty_like(bd)
+    B.slicegcn_layer_backward(g, desc, Hd, saved, dHd, W, dHin, W, gWa, gWs, gb, None, gE if use_e else None, ws, wb, st)
+    torch.cuda.synchronize()
+    assert B.slicegcn_graph_device_status(g) == 0
+    got_out = out.float().cpu().numpy()
+    got_mask = saved[lay["mask_offset"]:lay["mask_offset"] + n * lay["mask_ld"]].view(n, lay["mask_ld"])[:, :W].cpu().numpy()
+    ridx = torch.from_numpy(rows).cuda()
+    got_din = dHin[ridx].cpu().numpy()
+    got = {"dW_agg": gWa.cpu().numpy(), "dW_self": gWs.cpu().numpy(), "db": gb.cpu().numpy(), "dE": gE.cpu().numpy()}
+    H = Hd.float().cpu().numpy().astype(np.float64)
+    dH = dHd.cpu().numpy().astype(np.float64)
+    del Hd, dHd, out, saved, ws, dHin
+    torch.cuda.empty_cache()
+    # ---- oracle: Eq. 6-7 written out per slice, the whole forward in full, the input gradient on the row sample
+    Z = rnd(orc.spmm(og, H))                                         # the stored intermediate
+    want_out = np.empty((n, W)); M = np.empty((n, W))
+    for i in range(p):
+        c = slice(i * h_s, (i + 1) * h_s)
+        M[:, c] = Z[:, c] @ Wa[i].astype(np.float64) + b[i]
+        want_out[:, c] = np.maximum(M[:, c], 0.0) + H[:, c] @ Ws[i].astype(np.float64) + (E[i] if use_e else 0.0)
+    err_out = rel_inf(got_out, rnd(want_out))
+    assert err_out <= tol, err_out
+    # ReLU decisions: the kernel may differ from the fp64 oracle only where the pre-activation is rounding noise
+    band = np.abs(M) <= RELU_BAND * np.abs(M).max() if not bf16 else np.abs(M) <= 2.0 ** -7 * np.abs(M).max()
+    differ = (got_mask != 0) != (M > 0)
+    n_differ, n_band = int(differ.sum()), int(band.sum())
+    assert not np.any(differ & ~band), "a ReLU decision differs outside the rounding band"
+    assert n_differ <= n_band
+    want = {"dW_agg": np.empty((p, h_s, h_s)), "dW_self": np.empty((p, h_s, h_s)), "db": np.empty((p, h_s)),
+            "dE": np.empty((p, h_s))}
+    spread = {k: np.zeros_like(v) for k, v in want.items()}
+    dZ = np.empty((n, W))
+    for i in range(p):
+        c = slice(i * h_s, (i + 1) * h_s)
+        dM = dH[:, c] * (M[:, c] > 0)
+        want["dW_agg"][i] = Z[:, c].T @ dM
+        want["db"][i] = dM.sum(0)
+        want["dW_self"][i] = H[:, c].T @ dH[:, c]
+        want["dE"][i] = dH[:, c].sum(0)
+        dZ[:, c] = dM @ Wa[i].astype(np.float64).T
+        # the oracle's own spread over the borderline units: all of them on versus all of them off
+        bm = dH[:, c] * band[:, c]
+        spread["dW_agg"][i] = np.abs(Z[:, c].T @ bm)
+        spread["db"][i] = np.abs(bm.sum(0))
+    dZs = rnd(dZ)                                                    # bf16 models keep this operand in bf16
+    want_din = orc.spmm(og, dZs, rows=rows)
+    want_din_plain = orc.spmm(og, dZ, rows=rows) if bf16 else want_din
+    for i in range(p):
+        c = slice(i * h_s, (i + 1) * h_s)
+        extra = dH[rows][:, c] @ Ws[i].astype(np.float64).T
+        want_din[:, c] += extra
+        if bf16:
+            want_din_plain[:, c] += extra
+    errs = {"H_out": (err_out, tol, 0.0)}
+    for k in want:
+        if k == "dE" and not use_e:
+            continue
+        # fp32: twice the oracle's own spread over the borderline ReLU units is allowed on top (bf16: the plain bound)
+        sp = 0.0 if bf16 else float(spread[k].max() / np.abs(want[k]).max())
+        errs[k] = (rel_inf(got[k], want[k]), tol + 2 * sp, sp)
+    errs["dH_in (rows)"] = (rel_inf(got_din, want_din), tol, 0.0)
+    if bf16:
+        errs["dH_in vs unrounded dZ"] = (rel_inf(got_din, want_din_plain), tol, 0.0)
+    for k, (e, a, sp) in errs.items():
+        print(f"  {k:<24} err {e:.3e}  allowed {a:.3e}  relu-spread {sp:.3e}")
+        report.append((k, e, a, sp))
+    print(f"  ReLU decisions differing from the oracle: {n_differ} of {M.size} (all inside the band of {n_band} units)")
+    report.append(("relu_differ/band/units", n_differ, n_band, M.size))
+    bad = {k: v for k, v in errs.items() if not v[0] <= v[1]}
+    assert not bad, bad
+
+
+def _model_workload(B, torch, name, spmm_cases, p, h_s, dtype, use_e):
+    w = synth.WORKLOADS[name]
+    t0 = time.time()
+    src, dst = synth.make_graph(w, 0)
+    og = orc.build_graph(w["n"], src, dst, True, True)
+    g = B.slicegcn_graph_create(w["n"], src, dst, B.SYMMETRIZE | B.ADD_SELF_LOOPS)
+    del src, dst
+    print(f"\n{name}: n {og.n} nnz {og.nnz} max degree {og.deg.max()} (inputs built in {time.time() - t0:.0f} s)")
+    report = []
+    try:
+        _check_csr(B, g, og)
+        rows = _row_sample(og)
+        assert rows.size >= 10000 and og.deg[rows].max() == og.deg.max()
+        for k, (width, in_dt, out_dt, transpose) in enumerate(spmm_cases):
+            _spmm_case(B, torch, g, og, rows, width, in_dt, out_dt, transpose, seed=20 + k)
+        assert B.slicegcn_graph_device_status(g) == 0
+        _hidden_layer_case(B, torch, g, og, rows, p, h_s, dtype, use_e, seed=7, report=report)
+    finally:
+        B.slicegcn_graph_destroy(g)
+    return report
+
+
+def test_social_full_size(B, torch):
+    """Dense-social workload at N = 232,965 (mean degree ~492): fp32, width 256, hidden layer with 4 slices of 64."""
+    _model_workload(B, torch, "social", [(256, B.F32, B.F32, False), (256, B.F32, B.F32, True)], p=4, h_s=64,
+                    dtype=B.F32, use_e=False)
+
+
+def test_copurchase_full_size(B, torch):
+    """Co-purchase workload at N = 2,449,029: bf16 storage; the fused input's 16-wide aggregation, the 256-wide
+    bf16 -> bf16 forward aggregation and the bf16 -> fp32 transposed one (a 2.5 GB result: byte offsets beyond 2^31);
+    the last hidden layer (8 slices of 32, slice encoding) forward and backward."""
+    _model_workload(B, torch, "copurchase", [(16, B.BF16, B.BF16, False), (256, B.BF16, B.BF16, False),
+                                             (256, B.BF16, B.F32, True)], p=8, h_s=32, dtype=B.BF16, use_e=True)
+
+
+def test_rmat_scale_20_relabeled(B, torch):
+    """Sweep graph at scale 20 (1,048,576 nodes, 32.5 M stored entries, seeded random relabeling): CSR bit-exact; every
+    output element at width 16; sampled rows (the 100 longest included) at widths 16 / 256 / 512 fp32 and 256 bf16,
+    forward and transposed (width 512 fp32: a 2 GiB operand and result)."""
+    n, src, dst = synth.rmat(20, 16, seed=0, relabel=True)
+    og = orc.build_graph(n, src, dst, True, True)
+    g = B.slicegcn_graph_create(n, src, dst, B.SYMMETRIZE | B.ADD_SELF_LOOPS)
+    try:
+        _check_csr(B, g, og)
+        rows = _row_sample(og)
+        every = np.arange(n, dtype=np.int64)
+        _spmm_case(B, torch, g, og, every, 16, B.F32, B.F32, False, seed=3)
+        for k, (width, dt) in enumerate([(16, B.F32), (256, B.F32), (512, B.F32), (256, B.BF16)]):
+            for transpose in (False, True):
+                _spmm_case(B, torch, g, og, rows, width, dt, dt, transpose, seed=40 + k)
+        assert B.slicegcn_graph_device_status(g) == 0
+    finally:
+        B.slicegcn_graph_destroy(g)
