@@ -292,6 +292,27 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
                                        const slicegcn_opt_desc* opt, float* logits_out, float* loss_out,
                                        void* workspace, int64_t workspace_bytes, void* stream);
 
+/* The same iteration with dropout between the layers.  Table II of the paper lists a dropout rate per dataset; the
+ * text never says where it acts, so the placement is this library's choice (and the oracle's): the output of every
+ * sliced layer but the last is multiplied by a 0/1 mask and by 1/(1 - rate) before the next layer reads it, forward
+ * and backward.  The masks are the caller's: the library draws no random numbers.
+ *   rate      in [0, 1)
+ *   masks     [host array of num_layers - 1 pointers]; masks[l] [device, n x (p*h_s) bytes, leading dimension mask_ld
+ *             bytes]: 0 drops the unit, anything else keeps it; it acts on the output of layer l (0-based)
+ * drop == NULL is slicegcn_train_epoch.  Errors: INVALID_ARG (rate outside [0,1), NULL mask, mask_ld < p*h_s), and
+ * those of slicegcn_train_epoch. */
+typedef struct slicegcn_dropout_desc {
+    double rate;
+    const uint8_t* const* masks;
+    int64_t mask_ld;
+} slicegcn_dropout_desc;
+slicegcn_status_t slicegcn_train_epoch_dropout(const slicegcn_model* m, const slicegcn_graph* g, const void* X, int64_t x_ld,
+                                               const int32_t* labels, const int32_t* train_idx, int64_t n_train,
+                                               float* params, float* grads, float* adam_m, float* adam_v,
+                                               const slicegcn_opt_desc* opt, const slicegcn_dropout_desc* drop,
+                                               float* logits_out, float* loss_out, void* workspace, int64_t workspace_bytes,
+                                               void* stream);
+
 /* Forgets what the model object remembers about earlier calls (the input aggregate cache above).  Host only. */
 slicegcn_status_t slicegcn_model_invalidate_caches(const slicegcn_model* m);
 

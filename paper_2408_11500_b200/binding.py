@@ -32,7 +32,7 @@ EXPORTS = [
     "slicegcn_spmm", "slicegcn_spmm_static_scratch", "slicegcn_layer_saved_bytes", "slicegcn_layer_saved_layout", "slicegcn_layer_workspace_bytes", "slicegcn_layer_forward",
     "slicegcn_layer_backward", "slicegcn_model_create", "slicegcn_model_destroy", "slicegcn_model_invalidate_caches", "slicegcn_model_param_count",
     "slicegcn_model_param_elems", "slicegcn_model_num_tensors", "slicegcn_model_tensor_info", "slicegcn_model_slices",
-    "slicegcn_model_layer_order", "slicegcn_train_workspace_bytes", "slicegcn_train_epoch", "slicegcn_forward_logits", "slicegcn_train_epoch_host", "slicegcn_train_epochs_host", "slicegcn_profile_begin", "slicegcn_profile_begin_sampled",
+    "slicegcn_model_layer_order", "slicegcn_train_workspace_bytes", "slicegcn_train_epoch", "slicegcn_train_epoch_dropout", "slicegcn_forward_logits", "slicegcn_train_epoch_host", "slicegcn_train_epochs_host", "slicegcn_profile_begin", "slicegcn_profile_begin_sampled",
     "slicegcn_profile_end",
 ]
 
@@ -59,6 +59,19 @@ class ModelDesc(ctypes.Structure):
 class OptDesc(ctypes.Structure):
     _fields_ = [("lr0", c_double), ("beta1", c_double), ("beta2", c_double), ("eps", c_double),
                 ("weight_decay", c_double), ("epoch", c_int32), ("total_epochs", c_int32)]
+
+
+class DropoutDesc(ctypes.Structure):
+    _fields_ = [("rate", c_double), ("masks", POINTER(c_void_p)), ("mask_ld", c_int64)]
+
+
+def make_dropout_desc(rate: float, masks: Sequence, mask_ld: int) -> DropoutDesc:
+    """masks: one device tensor (bytes, n x mask_ld) per layer but the last."""
+    d = DropoutDesc()
+    arr = (c_void_p * max(len(masks), 1))(*[_ptr(t) for t in masks])
+    d._keep = (arr, list(masks))       # keep the pointer array and the tensors alive with the struct
+    d.rate, d.masks, d.mask_ld = rate, ctypes.cast(arr, POINTER(c_void_p)), mask_ld
+    return d
 
 
 def _load() -> ctypes.CDLL:
@@ -308,6 +321,16 @@ def slicegcn_train_epoch(m, g, X, x_ld: int, labels, train_idx, n_train: int, pa
                                      _vp(params), _vp(grads), _vp(adam_m), _vp(adam_v),
                                      byref(opt) if opt is not None else None, _vp(logits_out), _vp(loss_out),
                                      _vp(workspace), c_int64(workspace_bytes), _vp(stream)))
+
+
+def slicegcn_train_epoch_dropout(m, g, X, x_ld: int, labels, train_idx, n_train: int, params, grads, adam_m, adam_v,
+                                 opt: Optional[OptDesc], drop: Optional[DropoutDesc], logits_out, loss_out, workspace,
+                                 workspace_bytes: int, stream=None) -> None:
+    _check(_lib.slicegcn_train_epoch_dropout(m, g, _vp(X), c_int64(x_ld), _vp(labels), _vp(train_idx), c_int64(n_train),
+                                             _vp(params), _vp(grads), _vp(adam_m), _vp(adam_v),
+                                             byref(opt) if opt is not None else None,
+                                             byref(drop) if drop is not None else None, _vp(logits_out), _vp(loss_out),
+                                             _vp(workspace), c_int64(workspace_bytes), _vp(stream)))
 
 
 def slicegcn_forward_logits(m, g, X, x_ld: int, params, logits_out, workspace, workspace_bytes: int, stream=None) -> None:

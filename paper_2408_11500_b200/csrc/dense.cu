@@ -584,6 +584,67 @@ slicegcn_status_t repack_slices_run(int64_t n, int p, const int* starts, int w, 
     return SLICEGCN_OK;
 }
 
+// Parameter tensors between the caller's layout (blocks of r x c) and the padded internal one (blocks of rp x cp, the
+// extra rows and columns zero).  One launch covers every tensor: blockIdx.y picks the table entry.
+template <bool PAD>
+__global__ void pad_params_kernel(const PadTable t, const float* src, float* dst) {
+    const PadEntry e = t.e[blockIdx.y];
+    // PAD: every element of the padded tensor is written (padding as zero); else: every element of the caller's tensor
+    const int64_t total = (int64_t)e.blocks * (PAD ? (int64_t)e.rp * e.cp : (int64_t)e.r * e.c);
+    for (int64_t k = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; k < total; k += (int64_t)gridDim.x * blockDim.x) {
+        const int cols = PAD ? e.cp : e.c, rows = PAD ? e.rp : e.r;
+        const int64_t per = (int64_t)rows * cols;
+        const int64_t blk = k / per, rem = k - blk * per;
+        const int i = (int)(rem / cols), j = (int)(rem - (int64_t)i * cols);
+        if (PAD) {
+            float v = 0.f;
+            if (i < e.r && j < e.c) v = src[e.outer + (blk * e.r + i) * e.c + j];
+            dst[e.inner + k] = v;
+        } else {
+            dst[e.outer + k] = src[e.inner + (blk * e.rp + i) * e.cp + j];
+        }
+    }
+}
+
+slicegcn_status_t pad_params_run(const PadTable& t, bool pad, const float* src, float* dst, cudaStream_t st) {
+    if (t.count < 1) return SLICEGCN_OK;
+    dim3 grid(64, t.count);
+    if (pad)
+        pad_params_kernel<true><<<grid, 256, 0, st>>>(t, src, dst);
+    else
+        pad_params_kernel<false><<<grid, 256, 0, st>>>(t, src, dst);
+    SGCN_LAUNCH_CHECK();
+    count_launch();
+    return SLICEGCN_OK;
+}
+
+template <typename T>
+__global__ void dropout_apply_kernel(int64_t n, int cols, T* data, int64_t ld, const uint8_t* mask, int64_t mask_ld, int h_s,
+                                     int hp, float scale) {
+    const int64_t total = n * cols;
+    for (int64_t k = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; k < total; k += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = k / cols;
+        const int c = (int)(k - r * cols);
+        const int blk = c / hp, j = c - blk * hp;
+        if (j >= h_s) continue;   // padding column of the internal layout
+        T* d = data + r * ld + c;
+        const float v = mask[r * mask_ld + blk * h_s + j] ? (float)*d * scale : 0.f;
+        *d = (T)v;
+    }
+}
+
+slicegcn_status_t dropout_apply_run(int64_t n, int cols, void* data, int64_t ld, int dtype, const uint8_t* mask, int64_t mask_ld,
+                                    int h_s, int hp, float scale, cudaStream_t st) {
+    const unsigned blocks = (unsigned)std::min<int64_t>((n * cols + 255) / 256, 148 * 32);
+    if (dtype == SLICEGCN_BF16)
+        dropout_apply_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(n, cols, static_cast<__nv_bfloat16*>(data), ld, mask, mask_ld, h_s, hp, scale);
+    else
+        dropout_apply_kernel<float><<<blocks, 256, 0, st>>>(n, cols, static_cast<float*>(data), ld, mask, mask_ld, h_s, hp, scale);
+    SGCN_LAUNCH_CHECK();
+    count_launch();
+    return SLICEGCN_OK;
+}
+
 slicegcn_status_t mask_mul_run(int64_t M, int N, const float* in, int64_t ld_in, const uint8_t* mask, int64_t ld_mask,
                                float* out, int64_t ld_out, cudaStream_t st) {
     int64_t blocks = (M * N + 255) / 256;

@@ -131,6 +131,22 @@ slicegcn_status_t wgrad_run(const WgradArgs& a, void* scratch, int64_t scratch_b
 // Slices of X (p column ranges of width w at starts[]) copied side by side at multiples of w_pad, padding zeroed
 slicegcn_status_t repack_slices_run(int64_t n, int p, const int* starts, int w, int w_pad, const void* X, int64_t x_ld, int dtype,
                                     void* out, int64_t out_ld, cudaStream_t st);
+// Parameter (or gradient) tensors copied between the caller's layout and the padded internal one: tensor e is
+// `blocks` blocks of r x c floats at element offset `outer` of the caller's buffer and of rp x cp (rp >= r, cp >= c) at
+// offset `inner` of the internal buffer.  pad: caller -> internal, padding written as zeros; else internal -> caller.
+struct PadEntry {
+    int64_t outer, inner;
+    int blocks, r, c, rp, cp;
+};
+struct PadTable {
+    int count = 0;
+    PadEntry e[48];
+};
+slicegcn_status_t pad_params_run(const PadTable& t, bool pad, const float* src, float* dst, cudaStream_t st);
+// Dropout in place: data[r, c] = mask[r, mc] ? data[r, c] * scale : 0 over n x cols (fp32 or bf16).  The data may keep
+// every block of h_s columns padded to hp columns (hp >= h_s; padding untouched); the mask is dense in blocks of h_s.
+slicegcn_status_t dropout_apply_run(int64_t n, int cols, void* data, int64_t ld, int dtype, const uint8_t* mask, int64_t mask_ld,
+                                    int h_s, int hp, float scale, cudaStream_t st);
 // out = in * mask (fp32, row-major with leading dimensions)
 slicegcn_status_t mask_mul_run(int64_t M, int N, const float* in, int64_t ld_in, const uint8_t* mask, int64_t ld_mask,
                                float* out, int64_t ld_out, cudaStream_t st);

@@ -543,7 +543,17 @@ struct slicegcn_model {
         bool valid = false;
     };
     mutable InputAggregateKey zkey;
-    ~slicegcn_model() { sgcn::tc_image_cache_destroy(image_cache); }
+    // Per-slice hidden widths that are not a multiple of 4 (fp32) / 8 (bf16) columns -- the paper's own p = 3:
+    // ceil(512/3) = 171 -- run on an internal copy of the model whose slices are padded to the next multiple of 8.
+    // The padded units have zero weights and biases, so they stay zero through every layer and take no gradient; the
+    // caller's parameter layout is unchanged (parameters are copied in, gradients copied out, once per epoch each).
+    slicegcn_model* inner = nullptr;
+    sgcn::PadTable pad_table;
+    int caller_h_s = 0;   // per-slice width of the caller's layout (= h_s unless this is a padded internal model)
+    ~slicegcn_model() {
+        sgcn::tc_image_cache_destroy(image_cache);
+        delete inner;
+    }
 
     int64_t add(const std::string& name, int d0, int d1, int d2) {
         const int64_t off = param_elems;
@@ -797,7 +807,47 @@ slicegcn_status_t slicegcn_layer_backward(const slicegcn_graph* g, const slicegc
                                workspace, workspace_bytes, (cudaStream_t)stream);
 }
 
+static slicegcn_status_t model_create_impl(const slicegcn_model_desc* desc, int h_s_override, slicegcn_model** out);
+
 slicegcn_status_t slicegcn_model_create(const slicegcn_model_desc* desc, slicegcn_model** out) {
+    SGCN_TRY(model_create_impl(desc, 0, out));
+    slicegcn_model* m = *out;
+    const int unit = m->desc.dtype == SLICEGCN_BF16 ? 8 : 4;
+    if (m->h_s % unit == 0) return SLICEGCN_OK;
+    // padded internal model: same tensors in the same order, every h_s-sized dimension widened to a multiple of 8
+    const int hp = (m->h_s + 7) / 8 * 8;
+    slicegcn_model* in = nullptr;
+    slicegcn_status_t s = model_create_impl(desc, hp, &in);
+    if (s != SLICEGCN_OK || in->tensors.size() != m->tensors.size() || m->tensors.size() > 48) {
+        delete in;
+        delete m;
+        *out = nullptr;
+        if (s == SLICEGCN_OK) SGCN_FAIL(SLICEGCN_ERR_UNSUPPORTED, "model: too many parameter tensors for the padded layout");
+        return s;
+    }
+    m->inner = in;
+    const int p = m->desc.num_slices;
+    for (size_t t = 0; t < m->tensors.size(); ++t) {
+        const auto& a = m->tensors[t];
+        const auto& b = in->tensors[t];
+        sgcn::PadEntry e;
+        e.outer = a.offset;
+        e.inner = b.offset;
+        if (a.name == "Wc1") {   // (p*h_s) x hidden: p blocks of h_s rows
+            e.blocks = p; e.r = m->h_s; e.c = a.dims[1]; e.rp = hp; e.cp = b.dims[1];
+        } else {                 // d0 blocks (slices, or 1) of d1 x d2
+            e.blocks = a.dims[0]; e.r = a.dims[1]; e.c = a.dims[2]; e.rp = b.dims[1]; e.cp = b.dims[2];
+            if (a.dims[2] == 1 && b.dims[2] == 1 && a.dims[0] == p && b.dims[0] == p && a.name != "ff_b1" && a.name != "ff_b2" &&
+                a.name != "bc1" && a.name != "bc2") {   // per-slice vectors p x h_s: one row of h_s columns per slice
+                e.r = 1; e.rp = 1; e.c = a.dims[1]; e.cp = b.dims[1];
+            }
+        }
+        m->pad_table.e[m->pad_table.count++] = e;
+    }
+    return SLICEGCN_OK;
+}
+
+static slicegcn_status_t model_create_impl(const slicegcn_model_desc* desc, int h_s_override, slicegcn_model** out) {
     if (!out) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "out is NULL");
     *out = nullptr;
     if (!desc) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "desc is NULL");
@@ -819,6 +869,8 @@ slicegcn_status_t slicegcn_model_create(const slicegcn_model_desc* desc, slicegc
     }
     m->slice_width = m->ends[0] - m->starts[0];
     m->h_s = (D.hidden + D.num_slices - 1) / D.num_slices;   // each layer scaled down in proportion to p
+    m->caller_h_s = m->h_s;
+    if (h_s_override > 0) m->h_s = h_s_override;
     const int p = D.num_slices;
     if (D.use_ff) {
         m->ff_W1 = m->add("ff_W1", D.in_d, D.in_d, 1);
@@ -855,6 +907,7 @@ slicegcn_status_t slicegcn_model_destroy(slicegcn_model* m) {
 slicegcn_status_t slicegcn_model_invalidate_caches(const slicegcn_model* m) {
     if (!m) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "model is NULL");
     m->zkey.valid = false;
+    if (m->inner) m->inner->zkey.valid = false;
     return SLICEGCN_OK;
 }
 
@@ -904,15 +957,16 @@ slicegcn_status_t slicegcn_model_slices(const slicegcn_model* m, int32_t* starts
 
 slicegcn_status_t slicegcn_model_layer_order(const slicegcn_model* m, int32_t layer, int32_t* order) {
     if (!m || !order || layer < 0 || layer >= m->desc.num_layers) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "bad argument");
-    *order = m->order[layer];
+    *order = (m->inner ? m->inner : m)->order[layer];   // the order that actually runs
     return SLICEGCN_OK;
 }
 
 slicegcn_status_t slicegcn_train_workspace_bytes(const slicegcn_model* m, const slicegcn_graph* g, int64_t* bytes) {
     if (!m || !g || !bytes) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "NULL argument");
     EpochLayout E;
-    SGCN_TRY(build_layout(m, g, m->desc.in_d, nullptr, &E));
+    SGCN_TRY(build_layout(m->inner ? m->inner : m, g, m->desc.in_d, nullptr, &E));
     *bytes = E.total;
+    if (m->inner) *bytes += 2 * align_up(m->inner->param_elems * (int64_t)sizeof(float), 256);   // padded parameters and gradients
     return SLICEGCN_OK;
 }
 
@@ -921,14 +975,48 @@ static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, 
                                     const int32_t* labels, const int32_t* train_idx, int64_t n_train, float* params,
                                     float* grads, float* adam_m, float* adam_v, const slicegcn_opt_desc* opt,
                                     float* logits_out, float* loss_out, void* workspace, int64_t workspace_bytes,
-                                    void* stream) {
+                                    void* stream, const slicegcn_dropout_desc* drop = nullptr) {
     if (!m || !g || !X || !params || !workspace || (!forward_only && (!labels || !grads)))
         SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "train_epoch: NULL argument");
+    if (m->inner) {
+        // padded internal model: parameters in, the whole iteration on the padded shapes, gradients out, then the update
+        // on the caller's buffers
+        if (opt && (!adam_m || !adam_v)) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "train_epoch: optimiser state is NULL");
+        if (opt && (opt->total_epochs < 1 || opt->epoch < 0)) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "train_epoch: bad epoch");
+        cudaStream_t st = (cudaStream_t)stream;
+        const int64_t pbytes = align_up(m->inner->param_elems * (int64_t)sizeof(float), 256);
+        if (workspace_bytes < 2 * pbytes) SGCN_FAIL(SLICEGCN_ERR_ALLOC, "train_epoch: workspace too small");
+        float* pin = static_cast<float*>(workspace);
+        float* gin = reinterpret_cast<float*>(static_cast<char*>(workspace) + pbytes);
+        void* iws = static_cast<char*>(workspace) + 2 * pbytes;
+        SGCN_TRY(pad_params_run(m->pad_table, true, params, pin, st));
+        SGCN_TRY(epoch_impl(forward_only, m->inner, g, X, x_ld, labels, train_idx, n_train, pin, gin, nullptr, nullptr, nullptr,
+                            logits_out, loss_out, iws, workspace_bytes - 2 * pbytes, stream, drop));
+        if (forward_only) return SLICEGCN_OK;
+        SGCN_CUDA(cudaMemsetAsync(grads, 0, sizeof(float) * m->param_elems, st));
+        SGCN_TRY(pad_params_run(m->pad_table, false, gin, grads, st));
+        if (opt) {
+            const double kPi = 3.14159265358979323846;
+            const double lr = opt->lr0 * 0.5 * (1.0 + std::cos(kPi * (double)opt->epoch / (double)opt->total_epochs));
+            SGCN_TRY(adam_run(m->param_elems, params, grads, adam_m, adam_v, (float)lr, (float)opt->beta1, (float)opt->beta2,
+                              (float)opt->eps, (float)opt->weight_decay, opt->epoch + 1, st));
+        }
+        return SLICEGCN_OK;
+    }
     const slicegcn_model_desc& D = m->desc;
     if (x_ld < D.in_d) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "train_epoch: x_ld < in_d");
     if (opt && (!adam_m || !adam_v)) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "train_epoch: optimiser state is NULL");
     if (opt && (opt->total_epochs < 1 || opt->epoch < 0)) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "train_epoch: bad epoch");
     if (train_idx && n_train < 1) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "train_epoch: empty training set");
+    float drop_scale = 1.f;
+    if (drop) {
+        if (!(drop->rate >= 0.0 && drop->rate < 1.0)) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "train_epoch: dropout rate outside [0, 1)");
+        if (D.num_layers > 1 && (!drop->masks || drop->mask_ld < (int64_t)D.num_slices * m->caller_h_s))
+            SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "train_epoch: dropout masks missing or mask_ld too small");
+        for (int l = 0; l + 1 < D.num_layers; ++l)
+            if (!drop->masks[l]) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "train_epoch: dropout mask %d is NULL", l);
+        drop_scale = (float)(1.0 / (1.0 - drop->rate));
+    }
     cudaStream_t st = (cudaStream_t)stream;
     const int64_t n = g->n;
     const int p = D.num_slices, L = D.num_layers, C = D.num_classes;
@@ -1055,6 +1143,9 @@ static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, 
             m->zkey.stream = stream;
             m->zkey.valid = true;
         }
+        if (drop && l + 1 < L)   // dropout on what the next layer reads (placement: see slicegcn_train_epoch_dropout)
+            SGCN_TRY(dropout_apply_run(n, p * m->h_s, E.H[l], E.ld_h, D.dtype, drop->masks[l], drop->mask_ld, m->caller_h_s, m->h_s,
+                                       drop_scale, st));
         hin = E.H[l];
     }
     const int HW = p * m->h_s;
@@ -1179,6 +1270,9 @@ static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, 
     for (int l = L - 1; l >= 0; --l) {
         const void* lin = l == 0 ? h0 : E.H[l - 1];
         const bool need_din = l > 0 || D.use_ff;
+        if (drop && l + 1 < L)   // the gradient passes the same mask and scale on its way into the layer
+            SGCN_TRY(dropout_apply_run(n, p * m->h_s, E.dH[cur], E.ld_grad, SLICEGCN_F32, drop->masks[l], drop->mask_ld, m->caller_h_s,
+                                       m->h_s, drop_scale, st));
         SGCN_TRY(layer_backward_impl(g, &descs[l], plans[l], lin, E.saved[l], E.dH[cur], E.ld_grad,
                                      need_din ? E.dH[cur ^ 1] : nullptr, E.ld_grad, grads + m->W_agg[l],
                                      D.use_self ? grads + m->W_self[l] : nullptr, grads + m->b[l],
@@ -1265,6 +1359,16 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
                       workspace, workspace_bytes, stream);
 }
 
+slicegcn_status_t slicegcn_train_epoch_dropout(const slicegcn_model* m, const slicegcn_graph* g, const void* X, int64_t x_ld,
+                                               const int32_t* labels, const int32_t* train_idx, int64_t n_train,
+                                               float* params, float* grads, float* adam_m, float* adam_v,
+                                               const slicegcn_opt_desc* opt, const slicegcn_dropout_desc* drop,
+                                               float* logits_out, float* loss_out, void* workspace, int64_t workspace_bytes,
+                                               void* stream) {
+    return epoch_impl(false, m, g, X, x_ld, labels, train_idx, n_train, params, grads, adam_m, adam_v, opt, logits_out, loss_out,
+                      workspace, workspace_bytes, stream, drop);
+}
+
 slicegcn_status_t slicegcn_forward_logits(const slicegcn_model* m, const slicegcn_graph* g, const void* X, int64_t x_ld,
                                           const float* params, float* logits_out, void* workspace, int64_t workspace_bytes,
                                           void* stream) {
@@ -1292,7 +1396,7 @@ slicegcn_status_t slicegcn_train_epoch_host(const slicegcn_model* m, const slice
     cudaStream_t st = (cudaStream_t)stream;
     const int64_t n = g->n;
     SGCN_TRY(check_labels_host(labels_host, n, m->desc.num_classes, "train_epoch_host"));
-    m->zkey.valid = false;   // X is copied anew: nothing computed from the staging buffer's old contents may be reused
+    slicegcn_model_invalidate_caches(m);   // X is copied anew: nothing computed from the staging buffer's old contents may be reused
     SGCN_CUDA(cudaMemcpyAsync(X_stage, X_host, (size_t)(n * x_ld) * esize(m->desc.dtype), cudaMemcpyHostToDevice, st));
     SGCN_CUDA(cudaMemcpyAsync(labels_stage, labels_host, (size_t)n * sizeof(int32_t), cudaMemcpyHostToDevice, st));
     SGCN_TRY(slicegcn_train_epoch(m, g, X_stage, x_ld, labels_stage, train_idx, n_train, params, grads, adam_m, adam_v, opt, nullptr,
@@ -1355,7 +1459,7 @@ slicegcn_status_t slicegcn_train_epochs_host(const slicegcn_model* m, const slic
             SGCN_CUDA(cudaStreamWaitEvent(st, ready[b], 0));
             slicegcn_opt_desc o = *opt;
             o.epoch = opt->epoch + e;
-            m->zkey.valid = false;   // the staging buffer holds a fresh copy of X
+            slicegcn_model_invalidate_caches(m);   // the staging buffer holds a fresh copy of X
             SGCN_TRY(slicegcn_train_epoch(m, g, xs[b], x_ld, ys[b], train_idx, n_train, params, grads, adam_m, adam_v, &o, nullptr,
                                           losses_dev + e, workspace, workspace_bytes, stream));
             SGCN_CUDA(cudaEventRecord(done[b], st));
