@@ -142,6 +142,35 @@ def oracle_epochs(w: dict, epochs: int, warm: int):
     return times, orc.max_threads()
 
 
+class SweepOracleLeg:
+    """CPU-baseline leg of the SpMM sweep (`--sweep`): exact oracle values on a seeded sample of rows that includes the
+    100 longest, and the oracle's own time on that sample scaled by (stored entries of the graph) / (entries of the
+    sampled rows) -- an extrapolation, labelled as such in the table."""
+
+    def __init__(self, n, src, dst, rows_wanted):
+        from oracle import slicegcn_oracle as orc
+        self.orc = orc
+        self.g = orc.build_graph(n, src, dst, True, True)
+        longest = np.argsort(self.g.deg, kind="stable")[-100:]
+        rnd = np.random.default_rng(0).choice(n, size=min(rows_wanted, n), replace=False)
+        self.rows = np.unique(np.concatenate([longest, rnd])).astype(np.int64)
+        self.entries = int(self.g.deg[self.rows].astype(np.int64).sum())
+
+    def check(self, X_dev, Y_rows, dtype_name):
+        X = X_dev.float().cpu().numpy().astype(np.float64)
+        t0 = time.perf_counter()
+        want = self.orc.spmm(self.g, X, rows=self.rows)
+        dt = time.perf_counter() - t0
+        if dtype_name == "f32":
+            err = float(np.abs(Y_rows - want).max() / np.abs(want).max())
+            ok = err <= 2e-6
+        else:   # one bf16 rounding of the fp32-accumulated result
+            err = float((np.abs(Y_rows - want) / (np.abs(want) + 1e-5 * np.abs(want).max())).max())
+            ok = bool(np.all(np.abs(Y_rows - want) <= 2 ** -8 * np.abs(want) + 1e-5 * np.abs(want).max()))
+        return {"err": err, "ok": ok, "rows": int(self.rows.size), "threads": self.orc.max_threads(),
+                "cpu_ms": 1e3 * dt * self.g.nnz / max(self.entries, 1)}
+
+
 def run_reference(args, rank: int):
     """--impl reference: the oracle on the host cores, on a bounded sample of the same workload."""
     if rank != 0:
@@ -394,7 +423,15 @@ def main():
     ap.add_argument("--cpu-fraction", type=float, default=0.0, help="size of the oracle's timed sample (0: a default per workload)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-secondary", action="store_true", help="skip the device-resident timing of the other workloads")
-    args = ap.parse_args()
+    ap.add_argument("--sweep", action="store_true",
+                    help="the SpMM kernel sweep on R-MAT graphs with the oracle's leg; the remaining arguments are spmm_sweep.py's")
+    args, rest = ap.parse_known_args()
+    if args.sweep:
+        import spmm_sweep
+        spmm_sweep.main(rest, oracle_leg=SweepOracleLeg)
+        return
+    if rest:
+        ap.error("unrecognised arguments: " + " ".join(rest))
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

@@ -193,6 +193,27 @@ WORKLOADS = {
 }
 
 
+# Seeded graphs with the sizes of the paper's Table I (nodes, undirected edges, features, classes) and the layer
+# count and dropout rate of its Table II; width 512 as its Table III implies.  Only the sizes are the paper's: the
+# edges are Chung-Lu power-law draws like the other workloads, the features Gaussian, the labels uniform.
+TABLE1_SHAPES = {
+    "t1_22662": dict(n=22662, m=32927, in_d=300, classes=18, layers=3, dropout=0.5),
+    "t1_24492": dict(n=24492, m=93050, in_d=300, classes=5, layers=4, dropout=0.5),
+    "t1_10000": dict(n=10000, m=39402, in_d=7, classes=2, layers=7, dropout=0.5),
+    "t1_11758": dict(n=11758, m=519000, in_d=10, classes=2, layers=4, dropout=0.5),
+    "t1_48921": dict(n=48921, m=153540, in_d=301, classes=2, layers=6, dropout=0.5),
+    "t1_169343": dict(n=169343, m=1166243, in_d=128, classes=40, layers=4, dropout=0.0),
+}
+
+
+def table1_workload(name: str) -> dict:
+    t = TABLE1_SHAPES[name]
+    mean_deg = 2.0 * t["m"] / t["n"]
+    return dict(n=t["n"], m=t["m"], gen="powerlaw", gamma=2.2, max_degree=min(t["n"] / 8.0, max(64.0, 60.0 * mean_deg)),
+                in_d=t["in_d"], feat="gauss", classes=t["classes"], layers=t["layers"], hidden=512, p=2, dtype="f32",
+                use_ff=False, use_se=False, dropout=t["dropout"])
+
+
 def make_graph(w: dict, seed: int = 0) -> Tuple[np.ndarray, np.ndarray]:
     if w["gen"] == "powerlaw":
         return chung_lu_powerlaw(w["n"], w["m"], w["gamma"], w["max_degree"], seed)

@@ -1,5 +1,6 @@
 """bench.py at N > 1 runs independent replicas; the only cross-rank steps are a barrier and the
-max-over-ranks of the elapsed time.  This checks that reduction with two gloo ranks on CPU."""
+max-over-ranks of the elapsed time.  This runs bench.py's own reduction (max_over_ranks, whole_job_rate) in two
+gloo ranks on CPU."""
 import os
 import socket
 import subprocess
@@ -22,16 +23,18 @@ def test_max_over_ranks_two_gloo_processes(tmp_path):
     script.write_text(textwrap.dedent("""
         import os, sys, json
         import torch, torch.distributed as dist
+        sys.path.insert(0, os.getcwd())
+        import bench                                # the functions under test are the benchmark's own
         rank, world = int(os.environ["RANK"]), int(os.environ["WORLD_SIZE"])
         dist.init_process_group("gloo", rank=rank, world_size=world)
         elapsed_ms = [12.5, 20.25][rank]            # what each replica measured for K steps
-        t = torch.tensor([elapsed_ms], dtype=torch.float64)
         dist.barrier()
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        slowest = bench.max_over_ranks(elapsed_ms, world, dist, torch.device("cpu"), torch)
         steps = 5
-        value = world * steps / (t.item() / 1e3)    # whole-job epochs/s: all replicas' steps over the slowest time
+        value = bench.whole_job_rate(world, steps, slowest)   # all replicas' steps over the slowest replica's time
+        alone = bench.max_over_ranks(elapsed_ms, 1)           # a single replica needs no reduction
         if rank == 0:
-            print(json.dumps({"max_ms": t.item(), "value": value}))
+            print(json.dumps({"max_ms": slowest, "value": value, "alone": alone}))
         dist.destroy_process_group()
     """))
     port = _free_port()
@@ -44,5 +47,5 @@ def test_max_over_ranks_two_gloo_processes(tmp_path):
     assert all(p.returncode == 0 for p in procs), outs
     import json
     line = json.loads(outs[0][0].strip().splitlines()[-1])
-    assert line["max_ms"] == 20.25
+    assert line["max_ms"] == 20.25 and line["alone"] == 12.5
     assert abs(line["value"] - 2 * 5 / 0.02025) < 1e-9

@@ -657,7 +657,7 @@ def test_rmat_scale_20_whole_output(B, torch):
 
 def test_sweep_module_case_runs_and_checks_identity(B, torch):
     """The sweep tool's per-case routine: rates are positive and the full-size identity holds."""
-    from paper_2408_11500_b200 import spmm_sweep
+    import spmm_sweep
     n, src, dst = synth.rmat(14, 16, seed=1)
     g = B.slicegcn_graph_create(n, src, dst, B.SYMMETRIZE | B.ADD_SELF_LOOPS)
     try:

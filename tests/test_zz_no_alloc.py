@@ -9,6 +9,7 @@ Collected last on purpose: a failure here must not hide the results of the other
 import numpy as np
 import pytest
 
+from oracle import slicegcn_oracle as orc
 from paper_2408_11500_b200 import synth
 
 pytestmark = pytest.mark.gpu
@@ -18,14 +19,14 @@ def _graph_with_hubs(B, n=6000, m=40000, max_degree=2500, seed=7):
     src, dst = synth.chung_lu_powerlaw(n, m, 2.2, max_degree, seed=seed)
     g = B.slicegcn_graph_create(n, src, dst, B.SYMMETRIZE | B.ADD_SELF_LOOPS)
     assert B.slicegcn_graph_info(g)["n_segments"] > 0        # the path that needs scratch is exercised
-    return g, n
+    return g, n, orc.build_graph(n, src, dst, True, True)
 
 
 @pytest.mark.parametrize("dtype,width", [("f32", 128), ("f32", 72), ("bf16", 256)])
 def test_static_scratch_matches_workspace_entry_point_twice(dtype, width):
     import torch
     from paper_2408_11500_b200 import binding as B
-    g, n = _graph_with_hubs(B)
+    g, n, og = _graph_with_hubs(B)
     try:
         tdt, bdt = (torch.float32, B.F32) if dtype == "f32" else (torch.bfloat16, B.BF16)
         st = torch.cuda.current_stream().cuda_stream
@@ -42,7 +43,42 @@ def test_static_scratch_matches_workspace_entry_point_twice(dtype, width):
             assert not torch.isnan(got.float()).any()
             a, b = got.float().cpu().numpy(), want.float().cpu().numpy()
             assert np.abs(a - b).max() <= 2e-6 * np.abs(b).max()   # same kernels, same order: in practice identical
+            # and against the definition itself (the CPU oracle), not only against the sibling entry point
+            ref = orc.spmm(og, X.float().cpu().numpy().astype(np.float64))
+            if dtype == "f32":
+                assert np.abs(a - ref).max() <= 2e-6 * np.abs(ref).max()
+            else:
+                assert np.all(np.abs(a - ref) <= 2 ** -8 * np.abs(ref) + 1e-5 * np.abs(ref).max())
         assert B.slicegcn_graph_device_status(g) == 0
+    finally:
+        B.slicegcn_graph_destroy(g)
+
+
+def test_static_scratch_transposed_directed_graph_and_no_allocation():
+    """A directed graph (its transpose has its own hub rows): the transposed aggregation through the built-in buffer
+    matches the oracle, and the calls leave the device's free memory and torch's allocator exactly as they were."""
+    import torch
+    from paper_2408_11500_b200 import binding as B
+    rng = np.random.default_rng(3)
+    n = 4000
+    src = rng.integers(0, n, 40000).astype(np.int32); dst = rng.integers(0, n, 40000).astype(np.int32)
+    dst[:900] = 11                                           # a long column -> a long row of the transpose
+    og = orc.build_graph(n, src, dst, False, False)
+    g = B.slicegcn_graph_create(n, src, dst, 0)
+    try:
+        assert not B.slicegcn_graph_info(g)["symmetric"]
+        X = torch.from_numpy(synth.gaussian_features(n, 64, seed=9)).cuda()
+        Y = torch.empty_like(X)
+        B.slicegcn_spmm_static_scratch(g, 1, B.F32, B.F32, X, 64, Y, 64, 64, None)   # the first call looks the buffer up
+        torch.cuda.synchronize()
+        free0, alloc0, reserved0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+        for transpose in (1, 0, 1):
+            B.slicegcn_spmm_static_scratch(g, transpose, B.F32, B.F32, X, 64, Y, 64, 64, None)
+            torch.cuda.synchronize()
+            ref = orc.spmm(og, X.cpu().numpy().astype(np.float64), transpose=bool(transpose))
+            assert np.abs(Y.cpu().numpy() - ref).max() <= 2e-6 * np.abs(ref).max()
+        assert torch.cuda.mem_get_info()[0] == free0
+        assert torch.cuda.memory_allocated() == alloc0 and torch.cuda.memory_reserved() == reserved0
     finally:
         B.slicegcn_graph_destroy(g)
 
