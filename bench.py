@@ -202,7 +202,7 @@ def run_reference(args, rank: int):
 # DRAM traffic of the dominant SpMM launch (dram__bytes_read.sum + dram__bytes_write.sum from one ncu capture, per launch),
 # with the committed summary each figure comes from; None where no capture exists.
 NCU_SPMM_TRAFFIC = {
-    "citation": (891e6, "profiles/spmm_rows_kernel_citation_w256.md (fp32 width-256 launch, 4 of the 5 per epoch)"),
+    "citation": (897e6, "profiles/spmm_rows_kernel_citation_w256.md (fp32 width-256 launch: every SpMM of a steady-state epoch)"),
     "copurchase": (38.1e9, "profiles/spmm_sweep_rmat.md (bf16 width-256 forward launch, 4 of the 6 per epoch; single-pass capture)"),
     "social": (12.0e9, "profiles/spmm_sweep_rmat.md (fp32 width-256 launch, all 4 per epoch alike)"),
 }
