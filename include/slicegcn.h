@@ -52,7 +52,12 @@ enum { SLICEGCN_RULE_CEIL = 0, SLICEGCN_RULE_FLOOR_PLUS_1 = 1 };
 enum {                                                          /* graph_create flags */
     SLICEGCN_SYMMETRIZE = 1u,       /* also store (v,u) for every input pair (u,v) */
     SLICEGCN_ADD_SELF_LOOPS = 2u,   /* set every diagonal entry (an input self-loop is not doubled) */
-    SLICEGCN_INPUT_ON_DEVICE = 4u   /* src/dst (or rowptr/colidx) are device pointers */
+    SLICEGCN_INPUT_ON_DEVICE = 4u,  /* src/dst (or rowptr/colidx) are device pointers */
+    /* Aggregator.  Default (neither flag): the normalisation of Eq. 1, A_hat = D^-1/2 A D^-1/2.  The paper defines
+     * only that one; its closing section points at other GNN layers, whose aggregators share every kernel here:
+     * mean over the neighbor set, A_hat = D^-1 A, and plain sum, A_hat = A.  At most one of the two. */
+    SLICEGCN_NORM_MEAN = 8u,
+    SLICEGCN_NORM_SUM = 16u
 };
 #define SLICEGCN_MAX_SLICES 64
 
@@ -88,7 +93,7 @@ slicegcn_status_t slicegcn_slice_strategy(int32_t in_d, int32_t p, double scale,
  *   SLICEGCN_INPUT_ON_DEVICE; never modified.  *out receives a handle owned by the library.
  * slicegcn_graph_create_from_csr: same from rowptr int32 [n+1] / colidx int32 [rowptr[n]]
  *   (columns need not be sorted or unique); the same flags apply.
- * Errors: INVALID_ARG, OUT_OF_RANGE (an id outside [0,n)), OVERFLOW (stored entries >= 2^31),
+ * Errors: INVALID_ARG (also: both NORM flags), OUT_OF_RANGE (an id outside [0,n)), OVERFLOW (stored entries >= 2^31),
  *   ALLOC, CUDA.  On error *out is NULL.  Both calls synchronise `stream`.
  */
 slicegcn_status_t slicegcn_graph_create(int64_t n, int64_t n_edges, const int32_t* src, const int32_t* dst,
@@ -118,6 +123,7 @@ slicegcn_status_t slicegcn_graph_destroy(slicegcn_graph* g);
  * Normalised sparse aggregation -- the neighbor sum of Eq. 1 / Eq. 6:
  *   Y[i, 0:width] = sum_{j in N(v_i)} X[j, 0:width] / c_ij          (transpose = 0)
  *   Y = A_hat^T X                                                    (transpose = 1, backward pass)
+ * (A_hat as fixed at graph creation: Eq. 1's normalisation unless a NORM flag chose the mean or the sum.)
  * X [device, n x width, leading dimension ldx], Y [device, n x width, ldy]; X and Y must not
  * overlap.  in_dtype / out_dtype: SLICEGCN_F32 or SLICEGCN_BF16 (fp32 accumulation); the pairs fp32 -> fp32,
  * bf16 -> bf16 and bf16 -> fp32 are supported (fp32 -> bf16: UNSUPPORTED).

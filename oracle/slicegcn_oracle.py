@@ -56,9 +56,9 @@ def _lib():
     if _LIB is None:
         lib = ctypes.CDLL(build_c())
         i64, p = ctypes.c_int64, ctypes.c_void_p
-        lib.oracle_spmm_gather.argtypes = [i64, p, p, p, p, i64, i64, p, i64, p, i64, ctypes.c_int]
+        lib.oracle_spmm_gather.argtypes = [i64, p, p, p, p, i64, i64, p, i64, p, i64, ctypes.c_int, ctypes.c_int]
         lib.oracle_spmm_gather.restype = None
-        lib.oracle_spmm_scatter_t.argtypes = [i64, p, p, p, p, i64, i64, p, i64]
+        lib.oracle_spmm_scatter_t.argtypes = [i64, p, p, p, p, i64, i64, p, i64, ctypes.c_int]
         lib.oracle_spmm_scatter_t.restype = None
         lib.oracle_max_threads.restype = ctypes.c_int
         _LIB = lib
@@ -182,14 +182,19 @@ def dinv_f32(deg: np.ndarray) -> np.ndarray:
     return out
 
 
+AGGREGATORS = {"sym": 0, "mean": 1, "sum": 2}
+
+
 def spmm(g: Graph, x: np.ndarray, transpose: bool = False, rows: Optional[np.ndarray] = None,
-         threads: int = 0) -> np.ndarray:
-    """A_hat @ x (or A_hat^T @ x): the normalised neighbor sum of Eq. 1 / Eq. 6,
-    1/c_ij = 1/(sqrt|N(v_i)| sqrt|N(v_j)|).  rows= limits the gather form to a
-    list of output rows (used for sampled checks on large graphs)."""
+         threads: int = 0, norm: str = "sym") -> np.ndarray:
+    """A_hat @ x (or A_hat^T @ x).  norm="sym" (the paper's): the normalised neighbor sum of Eq. 1 / Eq. 6,
+    1/c_ij = 1/(sqrt|N(v_i)| sqrt|N(v_j)|).  The two other aggregators of message-passing layers the paper's
+    closing section alludes to: "mean" (A_hat = D^-1 A, the mean over N(v_i)) and "sum" (A_hat = A).
+    rows= limits the gather form to a list of output rows (used for sampled checks on large graphs)."""
+    code = AGGREGATORS[norm]
     x = np.ascontiguousarray(x, dtype=np.float64)
     if x.ndim == 1:
-        return spmm(g, x[:, None], transpose, rows, threads)[:, 0]
+        return spmm(g, x[:, None], transpose, rows, threads, norm)[:, 0]
     n, w = x.shape
     assert n == g.n
     lib = _lib()
@@ -199,15 +204,15 @@ def spmm(g: Graph, x: np.ndarray, transpose: bool = False, rows: Optional[np.nda
             rows = np.ascontiguousarray(rows, dtype=np.int64)
             out = np.empty((rows.size, w), dtype=np.float64)
             lib.oracle_spmm_gather(n, vp(g.rowptr), vp(g.colidx), vp(g.deg), vp(x), w, w, vp(out), w,
-                                   vp(rows), rows.size, threads)
+                                   vp(rows), rows.size, threads, code)
         else:
             out = np.empty((n, w), dtype=np.float64)
             lib.oracle_spmm_gather(n, vp(g.rowptr), vp(g.colidx), vp(g.deg), vp(x), w, w, vp(out), w,
-                                   None, 0, threads)
+                                   None, 0, threads, code)
         return out
     assert rows is None
     out = np.empty((n, w), dtype=np.float64)
-    lib.oracle_spmm_scatter_t(n, vp(g.rowptr), vp(g.colidx), vp(g.deg), vp(x), w, w, vp(out), w)
+    lib.oracle_spmm_scatter_t(n, vp(g.rowptr), vp(g.colidx), vp(g.deg), vp(x), w, w, vp(out), w, code)
     return out
 
 
@@ -246,6 +251,7 @@ class ModelDesc:
     use_self: bool = True           # W_self term of Eq. 6 (False: Eq. 1, plain GCN)
     use_b_self: bool = False        # second bias per layer (needed by Table III only)
     slice_rule: str = "ceil"
+    aggregator: str = "sym"         # "sym" = Eq. 1 / Eq. 6 as printed; "mean" / "sum": other message-passing aggregators
     slices: List[Tuple[int, int]] = field(default_factory=list)
     slice_size: int = 0
     h_s: int = 0
@@ -363,13 +369,13 @@ def forward(m: ModelDesc, g: Graph, x: np.ndarray, params: Dict[str, np.ndarray]
             hin = h[:, s:e]                                   # Eq. 2 / Eq. 5
             W = P[f"W_agg.{l}.{i}"]
             if order[l] == "agg":
-                z = r(f"Z.{l}", spmm(g, hin, threads=threads))   # sum_u h_u / c_uv
+                z = r(f"Z.{l}", spmm(g, hin, threads=threads, norm=m.aggregator))   # sum_u h_u / c_uv
                 c[f"Z.{l}.{i}"] = z
                 mm = z @ W + P[f"b.{l}.{i}"]
             else:
                 t = r(f"T.{l}", hin @ W)
                 c[f"T.{l}.{i}"] = t
-                mm = spmm(g, t, threads=threads) + P[f"b.{l}.{i}"]
+                mm = spmm(g, t, threads=threads, norm=m.aggregator) + P[f"b.{l}.{i}"]
             c[f"M.{l}.{i}"] = mm
             hi = relu(mm)                                     # Eq. 6: ReLU covers the aggregation only
             if m.use_self:
@@ -463,9 +469,9 @@ def backward(m: ModelDesc, g: Graph, x: np.ndarray, params: Dict[str, np.ndarray
                 dz = dm @ W.T
                 if f"dZ.{l}" in rnd_at:
                     dz = rnd(dz)
-                dhin = dhin + spmm(g, dz, transpose=True)
+                dhin = dhin + spmm(g, dz, transpose=True, norm=m.aggregator)
             else:
-                dt = spmm(g, dm, transpose=True)
+                dt = spmm(g, dm, transpose=True, norm=m.aggregator)
                 G[f"W_agg.{l}.{i}"] = hin.T @ dt
                 dhin = dhin + dt @ W.T
             dprev[:, s:e] += dhin            # overlapping slices / shared X_ff: contributions add

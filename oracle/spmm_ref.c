@@ -6,7 +6,10 @@
  *
  *     out[i, :] = sum_{j in N(v_i)}  x[j, :] / ( sqrt|N(v_i)| * sqrt|N(v_j)| )
  *
- * with N(v) = the stored entries of row v of the adjacency matrix.  No blocking,
+ * with N(v) = the stored entries of row v of the adjacency matrix.  Two other aggregators
+ * of message-passing layers (the paper's closing section points at "a broader range of GNN
+ * methods"; it defines only the one above) share the loops: the mean over the neighbor set,
+ * weight 1/|N(v_i)| (norm 1), and the plain sum, weight 1 (norm 2).  No blocking,
  * no reordering: one loop over rows, one over the row's neighbors, one over
  * feature columns, in storage order.  Shares no code with the CUDA library.
  *
@@ -21,8 +24,11 @@
 #include <omp.h>
 #endif
 
-/* 1/c_ij of Eq. 1; a node with an empty neighbor set contributes / receives 0. */
-static double inv_c(int32_t deg_i, int32_t deg_j) {
+/* Weight of stored entry (i, j).  norm 0: 1/c_ij of Eq. 1 (a node with an empty neighbor set
+ * contributes / receives 0); norm 1: 1/|N(v_i)| (mean over the neighbors of i); norm 2: 1 (sum). */
+static double weight(int norm, int32_t deg_i, int32_t deg_j) {
+    if (norm == 2) return 1.0;
+    if (norm == 1) return deg_i > 0 ? 1.0 / (double)deg_i : 0.0;
     if (deg_i <= 0 || deg_j <= 0) return 0.0;
     return 1.0 / (sqrt((double)deg_i) * sqrt((double)deg_j));
 }
@@ -34,7 +40,7 @@ static double inv_c(int32_t deg_i, int32_t deg_j) {
 void oracle_spmm_gather(int64_t n, const int32_t* rowptr, const int32_t* colidx,
                         const int32_t* deg, const double* x, int64_t ldx,
                         int64_t w, double* out, int64_t ldo,
-                        const int64_t* rows, int64_t n_rows, int threads) {
+                        const int64_t* rows, int64_t n_rows, int threads, int norm) {
     int64_t count = rows ? n_rows : n;
 #ifdef _OPENMP
     if (threads > 0) omp_set_num_threads(threads);
@@ -48,7 +54,7 @@ void oracle_spmm_gather(int64_t n, const int32_t* rowptr, const int32_t* colidx,
         for (int64_t c = 0; c < w; ++c) o[c] = 0.0;
         for (int32_t k = rowptr[i]; k < rowptr[i + 1]; ++k) {
             int32_t j = colidx[k];
-            double a = inv_c(deg[i], deg[j]);
+            double a = weight(norm, deg[i], deg[j]);
             const double* xj = x + (int64_t)j * ldx;
             for (int64_t c = 0; c < w; ++c) o[c] += a * xj[c];
         }
@@ -59,14 +65,14 @@ void oracle_spmm_gather(int64_t n, const int32_t* rowptr, const int32_t* colidx,
  * entry (i, j) of A_hat sends y[i, :] to out[j, :].  Single-threaded. */
 void oracle_spmm_scatter_t(int64_t n, const int32_t* rowptr, const int32_t* colidx,
                            const int32_t* deg, const double* y, int64_t ldy,
-                           int64_t w, double* out, int64_t ldo) {
+                           int64_t w, double* out, int64_t ldo, int norm) {
     for (int64_t i = 0; i < n; ++i)
         for (int64_t c = 0; c < w; ++c) out[i * ldo + c] = 0.0;
     for (int64_t i = 0; i < n; ++i) {
         const double* yi = y + i * ldy;
         for (int32_t k = rowptr[i]; k < rowptr[i + 1]; ++k) {
             int32_t j = colidx[k];
-            double a = inv_c(deg[i], deg[j]);
+            double a = weight(norm, deg[i], deg[j]);
             double* o = out + (int64_t)j * ldo;
             for (int64_t c = 0; c < w; ++c) o[c] += a * yi[c];
         }

@@ -22,7 +22,7 @@ OK, ERR_INVALID_ARG, ERR_OUT_OF_RANGE, ERR_OVERFLOW, ERR_ALLOC, ERR_CUDA, ERR_UN
 F32, BF16 = 0, 1
 ORDER_AUTO, AGG_FIRST, XFORM_FIRST = 0, 1, 2
 RULE_CEIL, RULE_FLOOR_PLUS_1 = 0, 1
-SYMMETRIZE, ADD_SELF_LOOPS, INPUT_ON_DEVICE = 1, 2, 4
+SYMMETRIZE, ADD_SELF_LOOPS, INPUT_ON_DEVICE, NORM_MEAN, NORM_SUM = 1, 2, 4, 8, 16
 MAX_SLICES = 64
 DEVSTATUS_BAD_LABEL = 32
 

@@ -68,6 +68,9 @@ struct CsrView {
     const int32_t* seg_order = nullptr;  // [n_seg] segments sorted by their first column index (processing order)
     int32_t n_chunks = 0;
     const int32_t* chunk_row = nullptr;  // [n_chunks+1] first row of each chunk
+    // A_hat_ij = row_scale[i] * col_scale[j] for every stored entry (no per-entry value array)
+    const float* row_scale = nullptr;
+    const float* col_scale = nullptr;
 };
 
 }  // namespace sgcn
@@ -80,6 +83,10 @@ struct slicegcn_graph {
     int32_t* colidx = nullptr;
     int32_t* deg = nullptr;
     float* dinv = nullptr;
+    // aggregators other than Eq. 1's: 1/deg (0 for an empty row) and a vector of ones; norm 0 sym, 1 mean, 2 sum
+    float* invdeg = nullptr;
+    float* ones = nullptr;
+    int norm = 0;
     int* fault = nullptr;   // device status word: non-zero once a bounded wait in a kernel ran out
     // transpose pattern (only when !symmetric)
     int32_t* rowptr_t = nullptr;
@@ -107,6 +114,9 @@ struct slicegcn_graph {
         v.seg_order = seg_order[t];
         v.n_chunks = n_chunks[t];
         v.chunk_row = chunk_row[t];
+        // sym: D^-1/2 A D^-1/2 either way; mean: D^-1 A forward, A^T D^-1 transposed; sum: A
+        v.row_scale = norm == 0 ? dinv : (norm == 1 && !transpose ? invdeg : ones);
+        v.col_scale = norm == 0 ? dinv : (norm == 1 && transpose ? invdeg : ones);
         return v;
     }
     int32_t max_segments() const { return n_seg[0] > n_seg[1] ? n_seg[0] : n_seg[1]; }

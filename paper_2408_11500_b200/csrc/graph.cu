@@ -112,6 +112,15 @@ __global__ void dinv_kernel(const int32_t* deg, int64_t n, float* dinv) {
     }
 }
 
+__global__ void invdeg_ones_kernel(const int32_t* deg, int64_t n, float* invdeg, float* ones) {
+    int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (i < n) {
+        int32_t d = deg[i];
+        invdeg[i] = d > 0 ? __fdiv_rn(1.0f, (float)d) : 0.0f;
+        ones[i] = 1.0f;
+    }
+}
+
 __global__ void expand_rows_kernel(const int32_t* rowptr, int64_t n, int32_t* rows) {
     // one warp per row
     int64_t warp = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
@@ -303,6 +312,8 @@ slicegcn_status_t sort_unique(DevBuf& keys, int64_t total, int end_bit, int64_t*
 slicegcn_status_t create_impl(int64_t n, int64_t m, const int32_t* d_src, const int32_t* d_dst, uint32_t flags,
                               cudaStream_t st, slicegcn_graph** out) {
     const bool sym = flags & SLICEGCN_SYMMETRIZE, loops = flags & SLICEGCN_ADD_SELF_LOOPS;
+    if ((flags & SLICEGCN_NORM_MEAN) && (flags & SLICEGCN_NORM_SUM))
+        SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "graph_create: NORM_MEAN and NORM_SUM exclude each other");
     DevBuf flag;
     SGCN_CUDA(flag.alloc(sizeof(int)));
     SGCN_CUDA(cudaMemsetAsync(flag.p, 0, sizeof(int), st));
@@ -393,6 +404,16 @@ slicegcn_status_t create_impl(int64_t n, int64_t m, const int32_t* d_src, const 
     g->colidx = colidx.release<int32_t>();
     g->deg = deg.release<int32_t>();
     g->dinv = dinv.release<float>();
+    g->norm = (flags & SLICEGCN_NORM_MEAN) ? 1 : (flags & SLICEGCN_NORM_SUM) ? 2 : 0;
+    if (g->norm != 0) {
+        DevBuf inv, one;
+        SGCN_CUDA(inv.alloc(sizeof(float) * n));
+        SGCN_CUDA(one.alloc(sizeof(float) * n));
+        invdeg_ones_kernel<<<(int)((n + 255) / 256), 256, 0, st>>>(g->deg, n, inv.as<float>(), one.as<float>());
+        SGCN_LAUNCH_CHECK();
+        g->invdeg = inv.release<float>();
+        g->ones = one.release<float>();
+    }
     SGCN_TRY(build_long_tables(g, 0, g->rowptr, g->colidx, st));
     if (!symmetric) SGCN_TRY(build_long_tables(g, 1, g->rowptr_t, g->colidx_t, st));
     SGCN_CUDA(cudaStreamSynchronize(st));
@@ -508,6 +529,8 @@ slicegcn_status_t slicegcn_graph_destroy(slicegcn_graph* g) {
     cudaFree(g->colidx);
     cudaFree(g->deg);
     cudaFree(g->dinv);
+    cudaFree(g->invdeg);
+    cudaFree(g->ones);
     cudaFree(g->fault);
     cudaFree(g->rowptr_t);
     cudaFree(g->colidx_t);

@@ -69,7 +69,8 @@ struct SpmmParams {
     int64_t n;
     const int32_t* rowptr;
     const int32_t* colidx;
-    const float* dinv;
+    const float* rs;   // row scale (1/sqrt(deg_i) for Eq. 1's normalisation)
+    const float* cs;   // column scale (1/sqrt(deg_j))
     const void* X;
     int64_t ldx;
     void* Y;
@@ -199,7 +200,7 @@ __device__ __forceinline__ void spmm_rows_block(const SpmmParams& p, const int64
         for (int i = 0; i < NB; ++i) {
             const int r = rbase + sl + i * L;
             rp_l[i] = (r < r1) ? __ldg(p.rowptr + r + 1) : k1;
-            di_l[i] = (r < r1) ? __ldg(p.dinv + r) : 0.f;
+            di_l[i] = (r < r1) ? __ldg(p.rs + r) : 0.f;
         }
     };
     auto meta_end = [&](int idx) {   // idx is the same in every lane of the group
@@ -235,7 +236,7 @@ __device__ __forceinline__ void spmm_rows_block(const SpmmParams& p, const int64
 #pragma unroll
     for (int i = 0; i < NB; ++i) jn[i] = (kk + sl + i * L < k1) ? __ldg(p.colidx + kk + sl + i * L) : 0;
 #pragma unroll
-    for (int i = 0; i < NB; ++i) djn[i] = (kk + sl + i * L < k1) ? __ldg(p.dinv + jn[i]) : 0.f;
+    for (int i = 0; i < NB; ++i) djn[i] = (kk + sl + i * L < k1) ? __ldg(p.cs + jn[i]) : 0.f;
 
     auto close_row = [&]() {   // scale, store and clear the finished row; step to the next one
         const float di = meta_dinv(row - rbase);
@@ -325,7 +326,7 @@ __device__ __forceinline__ void spmm_rows_block(const SpmmParams& p, const int64
         }
 #pragma unroll
         for (int i = 0; i < NB; ++i)   // the indices have arrived by now
-            if (nk + sl + i * L < k1) djn[i] = __ldg(p.dinv + jn[i]);
+            if (nk + sl + i * L < k1) djn[i] = __ldg(p.cs + jn[i]);
     }
 }
 
@@ -369,7 +370,7 @@ __device__ __forceinline__ void spmm_segment_block(const SpmmParams& p, const in
 #pragma unroll
     for (int i = 0; i < NB; ++i) jn[i] = (base + sl + i * L < end) ? __ldg(p.colidx + base + sl + i * L) : 0;
 #pragma unroll
-    for (int i = 0; i < NB; ++i) djn[i] = (base + sl + i * L < end) ? __ldg(p.dinv + jn[i]) : 0.f;
+    for (int i = 0; i < NB; ++i) djn[i] = (base + sl + i * L < end) ? __ldg(p.cs + jn[i]) : 0.f;
     for (; base < end; base += BT) {
         const int cnt = min(BT, end - base);
         __syncwarp(gmask);
@@ -428,7 +429,7 @@ __device__ __forceinline__ void spmm_segment_block(const SpmmParams& p, const in
         }
 #pragma unroll
         for (int i = 0; i < NB; ++i)   // the indices have arrived by now
-            if (nbase + sl + i * L < end) djn[i] = __ldg(p.dinv + jn[i]);
+            if (nbase + sl + i * L < end) djn[i] = __ldg(p.cs + jn[i]);
     }
     __syncwarp();
 #pragma unroll
@@ -440,7 +441,7 @@ __device__ __forceinline__ void spmm_segment_block(const SpmmParams& p, const in
     const bool single = __ldg(p.seg_ptr + li + 1) - __ldg(p.seg_ptr + li) == 1;
     if (single) {
         if (sub == 0) {
-            const float di = __ldg(p.dinv + row);
+            const float di = __ldg(p.rs + row);
 #pragma unroll
             for (int c = 0; c < C; ++c) {
                 const int chunk = sl + c * L;
@@ -505,7 +506,7 @@ __device__ __forceinline__ void spmm_segment_block(const SpmmParams& p, const in
 #pragma unroll
                     for (int e = 0; e < V; ++e) acc[c][e] += __shfl_xor_sync(0xffffffffu, acc[c][e], off);
             if (sub == 0) {
-                const float di = __ldg(p.dinv + row);
+                const float di = __ldg(p.rs + row);
 #pragma unroll
                 for (int c = 0; c < C; ++c) {
                     const int chunk = sl + c * L;
@@ -540,7 +541,7 @@ __global__ void __launch_bounds__(256) spmm_long_finish_kernel(const SpmmParams 
     const int64_t row = __ldg(p.long_rows + li);
     const int s0 = __ldg(p.seg_ptr + li), s1 = __ldg(p.seg_ptr + li + 1);
     if (s1 - s0 == 1) return;   // finished by its segment's warp
-    const float di = __ldg(p.dinv + row);
+    const float di = __ldg(p.rs + row);
     TO* Y = static_cast<TO*>(p.Y) + row * p.ldy;
     {
         float a = 0.f;
@@ -576,12 +577,12 @@ __global__ void __launch_bounds__(256) spmm_scalar_kernel(const SpmmParams p) {
     const TI* X = static_cast<const TI*>(p.X);
     TO* Y = static_cast<TO*>(p.Y) + row * p.ldy;
     const int start = __ldg(p.rowptr + row), end = __ldg(p.rowptr + row + 1);
-    const float di = __ldg(p.dinv + row);
+    const float di = __ldg(p.rs + row);
     for (int col = lane; col < p.width; col += 32) {
         float a = 0.f;
         for (int k = start; k < end; ++k) {
             const int j = __ldg(p.colidx + k);
-            a = fmaf(__ldg(p.dinv + j), to_f(X[(int64_t)j * p.ldx + col]), a);
+            a = fmaf(__ldg(p.cs + j), to_f(X[(int64_t)j * p.ldx + col]), a);
         }
         float x = a * di;
         if (EPI) {
@@ -715,7 +716,8 @@ slicegcn_status_t spmm_run(const slicegcn_graph* g, bool transpose, int in_dtype
     p.n = g->n;
     p.rowptr = v.rowptr;
     p.colidx = v.colidx;
-    p.dinv = g->dinv;
+    p.rs = v.row_scale;
+    p.cs = v.col_scale;
     p.X = X;
     p.ldx = ldx;
     p.Y = Y;

@@ -20,18 +20,21 @@ def oracle_desc(**kw):
                          scale=kw.get("slice_size_scale", 1.0), use_ff=kw.get("use_ff", False),
                          use_se=kw.get("use_se", False), use_self=kw.get("use_self", True),
                          use_b_self=kw.get("use_b_self", False),
-                         slice_rule="floor_plus_1" if kw.get("slice_rule", 0) == 1 else "ceil")
+                         slice_rule="floor_plus_1" if kw.get("slice_rule", 0) == 1 else "ceil",
+                         aggregator=kw.get("aggregator", "sym"))
 
 
 class GpuProblem:
     """Device-side state of one model on one graph (torch is used for memory only)."""
 
-    def __init__(self, n, src, dst, X, y, named_params, self_loops=True, symmetrize=True, train_idx=None, **model_kw):
+    def __init__(self, n, src, dst, X, y, named_params, self_loops=True, symmetrize=True, train_idx=None, aggregator="sym",
+                 **model_kw):
         import torch
         from paper_2408_11500_b200 import binding as B
         self.B, self.torch = B, torch
         dev = torch.device("cuda:0")
         flags = (B.SYMMETRIZE if symmetrize else 0) | (B.ADD_SELF_LOOPS if self_loops else 0)
+        flags |= {"sym": 0, "mean": B.NORM_MEAN, "sum": B.NORM_SUM}[aggregator]      # the aggregator is a property of the graph object
         self.g = B.slicegcn_graph_create(n, np.ascontiguousarray(src, np.int32), np.ascontiguousarray(dst, np.int32), flags)
         self.m = B.slicegcn_model_create(**model_kw)
         self.kw = model_kw

@@ -174,6 +174,38 @@ def test_spmm_transposed_on_directed_graph(B, torch):
         B.slicegcn_graph_destroy(g)
 
 
+@pytest.mark.parametrize("norm", ["mean", "sum"])
+def test_spmm_mean_and_sum_aggregators(B, torch, norm):
+    """The other aggregators (graph flags NORM_MEAN: D^-1 A, NORM_SUM: A) through the same kernels: forward and
+    transposed, on a symmetrized graph with hub rows and on a directed one (the mean's transpose scales the SOURCE
+    rows, A^T D^-1), fp32 and bf16."""
+    flag = B.NORM_MEAN if norm == "mean" else B.NORM_SUM
+    n = 5000
+    src, dst = synth.chung_lu_powerlaw(n, 30000, 2.2, 1500, seed=1)
+    rng = np.random.default_rng(3)
+    dsrc = rng.integers(0, n, 40000).astype(np.int32); ddst = rng.integers(0, n, 40000).astype(np.int32)
+    ddst[:900] = 11
+    for (s_, d_, sym, loops) in ((src, dst, True, True), (dsrc, ddst, False, False)):
+        og = orc.build_graph(n, s_, d_, sym, loops)
+        g = B.slicegcn_graph_create(n, s_, d_, (B.SYMMETRIZE if sym else 0) | (B.ADD_SELF_LOOPS if loops else 0) | flag)
+        try:
+            for width, dt in ((64, B.F32), (256, B.F32), (256, B.BF16), (13, B.F32)):
+                X = synth.gaussian_features(n, width, seed=width)
+                for transpose in (False, True):
+                    got, x_used = _gpu_spmm(B, torch, g, X, width, dt, transpose=transpose, ld_pad=3 if width == 13 else 0)
+                    want = orc.spmm(og, x_used.astype(np.float64), transpose=transpose, norm=norm)
+                    if dt == B.F32:
+                        assert rel_inf(got, want) <= 2e-6, (norm, sym, width, transpose)
+                    else:
+                        assert np.all(np.abs(got - want) <= 2 ** -8 * np.abs(want) + 1e-5 * np.abs(want).max())
+            assert B.slicegcn_graph_device_status(g) == 0
+        finally:
+            B.slicegcn_graph_destroy(g)
+    with pytest.raises(B.SliceGCNError) as e:
+        B.slicegcn_graph_create(n, src, dst, B.NORM_MEAN | B.NORM_SUM)
+    assert e.value.status == B.ERR_INVALID_ARG
+
+
 def test_spmm_is_deterministic_and_identity_holds(B, torch):
     n = 20000
     src, dst = synth.chung_lu_powerlaw(n, 150000, 2.2, 3000, seed=4)
@@ -419,6 +451,11 @@ def _compare_epoch(gp, od, og, X, y, params, train_idx, tol, rnd=orc.identity, o
     dict(p=8, in_d=128, hidden=64, C=8, n=900, slice_size_scale=0.5),
     dict(p=8, in_d=128, hidden=64, C=8, n=900, slice_size_scale=1.5, use_se=True),
     dict(p=8, in_d=128, hidden=64, C=8, n=900, slice_size_scale=1.5, order=2),
+    # other aggregators (mean / sum over the neighbor set instead of Eq. 1's normalisation): the backward pass runs the
+    # transposed aggregation with the scales swapped
+    dict(p=4, in_d=64, hidden=64, C=8, n=1111, aggregator="mean", use_se=True),
+    dict(p=4, in_d=64, hidden=64, C=8, n=1111, aggregator="mean", order=2),
+    dict(p=2, in_d=40, hidden=32, C=5, n=700, L=3, aggregator="sum"),
     # the paper's own slice counts: p = 3 gives per-slice widths that are no multiple of 4 (ceil(512/3) = 171,
     # ceil(128/3) = 43; input slices of floor(128/3) + 1 = 43 columns) -- these run on the padded internal model
     dict(p=3, in_d=48, hidden=512, C=12, L=2, n=700, use_se=True, relu_margin=5e-5),
@@ -433,7 +470,7 @@ def test_epoch_gradients_fp32(B, kw):
     mk["order"] = order
     og = orc.build_graph(len(X), src, dst, True, True)
     train_idx = np.arange(0, len(X), 3).astype(np.int32)
-    gp = GpuProblem(len(X), src, dst, X, y, params, train_idx=train_idx, **mk)
+    gp = GpuProblem(len(X), src, dst, X, y, params, train_idx=train_idx, **mk)   # (takes `aggregator` as a graph flag)
     try:
         orders = [{1: "agg", 2: "xform"}[B.slicegcn_model_layer_order(gp.m, l)] for l in range(mk["num_layers"])]
         _compare_epoch(gp, od, og, X.astype(np.float64), y, params, train_idx, TOL_F32, orders=orders, relu_margin=relu_margin)
@@ -567,6 +604,34 @@ def test_citation_workload_full_size_fp32(B):
         print(f"  ReLU decisions of layer 1 differing from the oracle: {int(differ.sum())} of {M.size}; "
               f"oracle units inside the 1e-6 band: {int(band.sum())}")
         assert not np.any(differ & ~band) and differ.sum() <= band.sum()
+    finally:
+        gp.close()
+
+
+def test_citation_workload_ten_epochs_loss_trajectory(B):
+    """The citation workload's own protocol: ten full-batch training epochs (Adam, cosine schedule) with the loss of
+    every epoch against the oracle's, the first layer's aggregate kept across epochs as the benchmark keeps it."""
+    w = synth.WORKLOADS["citation"]
+    src, dst = synth.make_graph(w, 0)
+    X = synth.make_features(w, 0); y = synth.uniform_labels(w["n"], w["classes"], 0)
+    mk = dict(in_d=w["in_d"], hidden=w["hidden"], num_layers=w["layers"], num_classes=w["classes"], num_slices=w["p"])
+    od = oracle_desc(**mk)
+    params = synth.init_params(orc.param_shapes(od), seed=0)
+    og = orc.build_graph(w["n"], src, dst, True, True)
+    gp = GpuProblem(w["n"], src, dst, X, y, params, cache_input_aggregate=True, **mk)
+    try:
+        P = {k: v.astype(np.float64) for k, v in params.items()}
+        st = {"m1": {}, "m2": {}}
+        X64 = X.astype(np.float64)
+        rows = []
+        for ep in range(10):
+            loss_o, logits_o, _ = orc.train_epoch(od, og, X64, P, y, st, 1e-3, ep, 10)
+            loss_g = gp.epoch(B.make_opt_desc(lr0=1e-3, epoch=ep, total_epochs=10))
+            rows.append((ep, loss_o, loss_g))
+            assert abs(loss_g - loss_o) <= 1e-4 * abs(loss_o), (ep, loss_g, loss_o)
+        print("\n".join(f"  epoch {ep}: oracle {lo:.7f}  gpu {lg:.7f}  rel {abs(lg - lo) / lo:.1e}" for ep, lo, lg in rows))
+        assert rows[-1][1] < rows[0][1]                       # and it trains
+        assert rel_inf(gp.logits.cpu().numpy(), logits_o) <= 5e-4     # Adam amplifies rounding over epochs
     finally:
         gp.close()
 

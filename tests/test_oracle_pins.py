@@ -153,6 +153,48 @@ def test_spmm_vs_dense_bruteforce(n, m, sym, loops, seed):
     assert g.symmetric == np.array_equal(ah != 0, (ah != 0).T)
 
 
+@pytest.mark.parametrize("norm", ["mean", "sum"])
+@pytest.mark.parametrize("n,m,sym,loops,seed", [(17, 40, True, False, 1), (33, 90, False, True, 3), (48, 200, False, False, 4)])
+def test_other_aggregators_vs_dense_bruteforce(norm, n, m, sym, loops, seed):
+    """Mean (D^-1 A) and sum (A) aggregation, forward and transposed, against dense matrices built with python loops;
+    closed forms: the mean of a constant is that constant on every node with a neighbor, the sum of ones is the degree."""
+    rng = np.random.default_rng(seed)
+    g = orc.build_graph(n, rng.integers(0, n, m), rng.integers(0, n, m), sym, loops)
+    A = np.zeros((n, n))
+    for i in range(n):
+        for k in range(g.rowptr[i], g.rowptr[i + 1]):
+            A[i, g.colidx[k]] = 1.0
+    if norm == "mean":
+        for i in range(n):
+            if A[i].sum() > 0:
+                A[i] /= A[i].sum()
+    X = rng.standard_normal((n, 5))
+    np.testing.assert_allclose(orc.spmm(g, X, norm=norm), A @ X, rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(orc.spmm(g, X, transpose=True, norm=norm), A.T @ X, rtol=1e-12, atol=1e-12)
+    rows = np.array([0, n - 1, 3], dtype=np.int64)
+    assert np.array_equal(orc.spmm(g, X, rows=rows, norm=norm), orc.spmm(g, X, norm=norm)[rows])
+    ones = np.ones(n)
+    if norm == "mean":
+        np.testing.assert_allclose(orc.spmm(g, 7.0 * ones, norm=norm), 7.0 * (g.deg > 0), rtol=1e-13)
+    else:
+        np.testing.assert_allclose(orc.spmm(g, ones, norm=norm), g.deg.astype(np.float64), rtol=1e-13)
+    # and the model's backward under these aggregators: finite differences
+    m_ = orc.ModelDesc(6, 4, 2, 3, p=2, aggregator=norm)
+    P = {k: v.astype(np.float64) for k, v in synth.init_params(orc.param_shapes(m_), seed=seed, bias_scale=0.3).items()}
+    Xf = rng.standard_normal((n, 6)); y = rng.integers(0, 3, n)
+    for order in (["agg", "agg"], ["xform", "agg"]):
+        c = orc.forward(m_, g, Xf, P, y, order=order)
+        G = orc.backward(m_, g, Xf, P, y, c)
+        for name in ("W_agg.0.1", "W_self.1.0", "b.0.0"):
+            flat = P[name].reshape(-1)
+            old = flat[0]
+            flat[0] = old + 1e-6; lp = orc.loss_only(m_, g, Xf, P, y, None, order)
+            flat[0] = old - 1e-6; lm = orc.loss_only(m_, g, Xf, P, y, None, order)
+            flat[0] = old
+            fd = (lp - lm) / 2e-6
+            assert abs(fd - G[name].reshape(-1)[0]) <= 1e-6 * max(1.0, abs(fd)) + 1e-8, (norm, order, name)
+
+
 def test_spmm_closed_form_sqrt_degree():
     # row i of A_hat * sqrt(deg): sum_j sqrt(d_j)/(sqrt d_i sqrt d_j) = d_i/sqrt(d_i) = sqrt(d_i)
     src, dst = synth.chung_lu_powerlaw(3000, 9000, 2.2, 200, seed=3)
