@@ -282,10 +282,11 @@ slicegcn_status_t slicegcn_train_workspace_bytes(const slicegcn_model* m, const 
  *   logits_out [device, fp32 n x num_classes, dense] or NULL
  *   loss_out [device, one float] or NULL: mean cross entropy BEFORE the update
  *   workspace [device], workspace_bytes >= slicegcn_train_workspace_bytes()
- * Input aggregate cache (desc.cache_input_aggregate = 1; direct slicing with an aggregate-first first layer only):
- * Algorithm 3 slices the features once, outside the epoch loop, so the first layer's aggregate A_hat X^i (Eq. 6,
- * l = 1) is the same tensor in every epoch.  With the flag set the library keeps it in `workspace` and skips that
- * aggregation whenever X, x_ld, the graph, `workspace` and `stream` are those of the previous call on this model.  The caller
+ * Input aggregate cache (desc.cache_input_aggregate = 1): Algorithm 3 slices the features once, outside the epoch
+ * loop, so what depends on X alone is the same in every epoch: with direct slicing and an aggregate-first first layer
+ * its aggregate A_hat X^i (Eq. 6, l = 1), and any aligned / padded copy of X the kernels work from.  With the flag set
+ * the library keeps these in `workspace` and skips recomputing them whenever X, x_ld, the graph, `workspace` and
+ * `stream` are those of the previous call on this model.  The caller
  * then promises that the CONTENTS of X and of `workspace` do not change between such calls; after changing them, call
  * slicegcn_model_invalidate_caches().  The host-buffer entry points copy X anew every epoch and never use the cache.
  * Asynchronous on `stream`.  The model object keeps host-side bookkeeping of the converted weight operands it

@@ -1044,10 +1044,17 @@ static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, 
     if (ffact_pad) SGCN_CUDA(cudaMemsetAsync(E.ff_act, 0, n * E.ld_ffact * esize(D.dtype), st));
     const void* xin = X;          // what the fusion MLP reads
     int64_t xin_ld = x_ld;
+    // What a caller who set cache_input_aggregate promises not to change between calls: X (and the workspace).  When
+    // this call sees the X, graph, workspace and stream of the previous one, everything computed from X alone is still
+    // in the workspace: the padded copy of X below, the repacked slices and the first layer's aggregate further down.
+    const bool x_unchanged = D.cache_input_aggregate && m->zkey.valid && m->zkey.X == X && m->zkey.x_ld == x_ld && m->zkey.graph == g &&
+                             m->zkey.workspace == workspace && m->zkey.stream == stream;
+    m->zkey.valid = false;   // until this call has queued the first layer
     const bool ff_repacked = m->repack_ff_input(x_ld);
     if (ff_repacked) {
         const int zero = 0;
-        SGCN_TRY(repack_slices_run(n, 1, &zero, D.in_d, (int)E.ld_xrep, X, x_ld, D.dtype, E.xrep, E.ld_xrep, st));
+        if (!x_unchanged)
+            SGCN_TRY(repack_slices_run(n, 1, &zero, D.in_d, (int)E.ld_xrep, X, x_ld, D.dtype, E.xrep, E.ld_xrep, st));
         xin = E.xrep;
         xin_ld = E.ld_xrep;
     }
@@ -1099,11 +1106,9 @@ static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, 
     // Input aggregate cache: with direct slicing the first layer's A_hat X does not change from epoch to epoch
     // (Algorithm 3 slices outside the epoch loop); reuse what the previous call left in the workspace.
     const bool z_cacheable = D.cache_input_aggregate && !D.use_ff && m->order[0] == SLICEGCN_AGG_FIRST;
-    const bool z_cached = z_cacheable && m->zkey.valid && m->zkey.X == X && m->zkey.x_ld == x_ld && m->zkey.graph == g &&
-                          m->zkey.workspace == workspace && m->zkey.stream == stream;
-    m->zkey.valid = false;   // until this call has queued the first layer
+    const bool z_cached = z_cacheable && x_unchanged;
     const bool repacked = m->repack_input();
-    if (repacked && z_cached) {   // the repacked copy is still in the workspace as well
+    if (repacked && x_unchanged) {   // the repacked copy is still in the workspace as well
         h0 = E.xrep;
         ld0 = E.ld_xrep;
     } else if (repacked) {   // slicing (Algorithm 2) as a copy: slices side by side at aligned starts, zero padding
@@ -1135,7 +1140,7 @@ static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, 
             }
         }
         SGCN_TRY(layer_forward_impl(g, &descs[l], plans[l], hin, E.H[l], E.saved[l], E.ws, E.ws_bytes, st, l == 0 && z_cached));
-        if (l == 0 && z_cacheable) {
+        if (l == 0 && D.cache_input_aggregate) {
             m->zkey.X = X;
             m->zkey.x_ld = x_ld;
             m->zkey.graph = g;

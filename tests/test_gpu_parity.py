@@ -631,7 +631,10 @@ def test_citation_workload_ten_epochs_loss_trajectory(B):
             assert abs(loss_g - loss_o) <= 1e-4 * abs(loss_o), (ep, loss_g, loss_o)
         print("\n".join(f"  epoch {ep}: oracle {lo:.7f}  gpu {lg:.7f}  rel {abs(lg - lo) / lo:.1e}" for ep, lo, lg in rows))
         assert rows[-1][1] < rows[0][1]                       # and it trains
-        assert rel_inf(gp.logits.cpu().numpy(), logits_o) <= 5e-4     # Adam amplifies rounding over epochs
+        # Adam's first steps move every parameter by ~lr * sign(gradient): an entry whose gradient is rounding noise gets
+        # a different step in fp32 and fp64, so parameters (and through them the logits) drift apart by a few lr per
+        # epoch while the loss stays together to 1e-6 (the ten-epoch test of the tiny workload allows the same 2e-3)
+        assert rel_inf(gp.logits.cpu().numpy(), logits_o) <= 2e-3
     finally:
         gp.close()
 
@@ -780,7 +783,8 @@ def test_train_epoch_host_buffers_match_device_call(B, torch):
         gp.close()
 
 
-@pytest.mark.parametrize("kw", [dict(p=4, in_d=64, hidden=64, C=8, n=1111), dict(p=4, in_d=37, hidden=48, C=5, n=900)])
+@pytest.mark.parametrize("kw", [dict(p=4, in_d=64, hidden=64, C=8, n=1111), dict(p=4, in_d=37, hidden=48, C=5, n=900),
+                                dict(p=4, in_d=100, hidden=64, C=8, n=1111, use_ff=True)])   # feature fusion: only the padded copy of X is kept
 def test_input_aggregate_cache(B, torch, kw):
     """Algorithm 3 slices X once, outside the epoch loop, so the first layer's A_hat X is the same in every epoch.  With
     cache_input_aggregate the library skips that aggregation from the second call on: every epoch's loss, gradients
