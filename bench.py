@@ -120,9 +120,19 @@ def model_kwargs(w: dict) -> dict:
 
 # ---------------------------------------------------------------------------------- oracle timing
 
-def oracle_epochs(w: dict, epochs: int, warm: int):
-    """Times the CPU oracle, as it stands, on workload w.  Returns (seconds per epoch list, threads)."""
+def oracle_epochs(w: dict, epochs: int, warm: int, single_thread: bool = False):
+    """Times the CPU oracle, as it stands, on workload w.  Returns (seconds per epoch list, threads).
+    single_thread: one OpenMP thread in the neighbor sum and one BLAS thread in the dense products."""
     from oracle import slicegcn_oracle as orc
+    if single_thread:
+        from threadpoolctl import threadpool_limits
+        with threadpool_limits(limits=1):
+            times, _ = oracle_epochs_impl(orc, w, epochs, warm, 1)
+        return times, 1
+    return oracle_epochs_impl(orc, w, epochs, warm, len(os.sched_getaffinity(0)))   # every core this process may use
+
+
+def oracle_epochs_impl(orc, w: dict, epochs: int, warm: int, threads: int):
     src, dst = synth.make_graph(w, 0)
     X = synth.make_features(w, 0).astype(np.float64)
     y = synth.uniform_labels(w["n"], w["classes"], 0)
@@ -136,10 +146,10 @@ def oracle_epochs(w: dict, epochs: int, warm: int):
     times = []
     for ep in range(warm + epochs):
         t0 = time.perf_counter()
-        orc.train_epoch(od, g, X, P, y, st, 1e-3, ep, max(warm + epochs, 2), rnd=rnd)
+        orc.train_epoch(od, g, X, P, y, st, 1e-3, ep, max(warm + epochs, 2), rnd=rnd, threads=threads)
         if ep >= warm:
             times.append(time.perf_counter() - t0)
-    return times, orc.max_threads()
+    return times, (threads if threads > 0 else orc.max_threads())
 
 
 class SweepOracleLeg:
@@ -407,6 +417,12 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         sample = ("1 full epoch of the same workload" if frac >= 1 else
                   f"1 epoch of the same generator at {frac:g} of the nodes and edges (n={cw['n']}), epochs/s scaled by {frac:g}")
         line["cpu_baseline"] = {"value": v, "unit": "epochs/s", "cores": threads, "kind": "oracle", "sample": sample}
+        # the same oracle on ONE thread, on a quarter of that sample (it is ~10x slower)
+        f1 = frac / 4
+        c1 = scaled_workload(args.workload, f1)
+        t1, _ = oracle_epochs(c1, 1, 0, single_thread=True)
+        line["cpu_baseline"]["single_thread"] = {"value": f1 / t1[0], "unit": "epochs/s", "cores": 1,
+                                                 "sample": f"1 epoch at {f1:g} of the nodes and edges (n={c1['n']}), scaled"}
     if rank == 0:
         print(json.dumps(line), flush=True)
     if world > 1:

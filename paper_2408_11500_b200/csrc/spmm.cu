@@ -517,6 +517,69 @@ __device__ __forceinline__ void spmm_segment_block(const SpmmParams& p, const in
     }
 }
 
+// Rows of at most 128 bytes (one to eight 16-byte chunks): L lanes per row-aligned chunk, 32/L chunks per warp, and NO
+// cooperation between the lanes of a warp -- every lane group walks its own chunk with plain loads (the L lanes of a
+// group read the same index and scale, which the load unit broadcasts), four neighbors requested before they are
+// accumulated, rows closed where the running entry index meets the row's end.  The general kernel above stages indices
+// in shared memory and hands row metadata around by shuffles, which pays for wide rows; for these narrow ones its
+// per-batch bookkeeping (a batch is 2 L entries) is most of the instructions.  Long rows stay with the segment path.
+template <typename TI, typename TO, int L, bool EPI>
+__global__ void __launch_bounds__(128) spmm_narrow_kernel(const SpmmParams p) {
+    constexpr int V = Vec<TI>::V;
+    constexpr int U = 4;
+    const int lane = threadIdx.x & 31;
+    const int sub = lane / L, sl = lane % L;
+    const int64_t chunk = ((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5) * (32 / L) + sub;
+    if (chunk >= p.n_chunks) return;
+    const int r0 = __ldg(p.chunk_row + chunk);
+    const int r1 = __ldg(p.chunk_row + chunk + 1);
+    if (r0 >= r1) return;
+    int k = __ldg(p.rowptr + r0);
+    const int k1 = __ldg(p.rowptr + r1);
+    int row = r0;
+    int row_end = __ldg(p.rowptr + r0 + 1);
+    if (row_end - k > kLongRow) return;   // a long row sits alone in its chunk: left to its segments
+    const bool live = sl < p.nch;
+    const uint32_t row16 = (uint32_t)((p.ldx * (int64_t)sizeof(TI)) >> 4);
+    const uint4* xl = static_cast<const uint4*>(p.X) + min(sl, p.nch - 1);
+    float acc[V];
+#pragma unroll
+    for (int e = 0; e < V; ++e) acc[e] = 0.f;
+    auto close_row = [&]() {
+        const float di = __ldg(p.rs + row);
+        if (live) finish_chunk<TO, V, EPI>(p, row, sl, di, acc);
+#pragma unroll
+        for (int e = 0; e < V; ++e) acc[e] = 0.f;
+        ++row;
+        row_end = row < r1 ? __ldg(p.rowptr + row + 1) : -1;
+    };
+    while (k < k1) {
+        const int cnt = min(U, k1 - k);
+        int j[U];
+        float d[U];
+        uint4 raw[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) j[u] = u < cnt ? __ldg(p.colidx + k + u) : 0;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            d[u] = u < cnt ? __ldg(p.cs + j[u]) : 0.f;
+            raw[u] = __ldg(xl + (uint64_t)(uint32_t)j[u] * row16);
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (u < cnt) {
+                while (k == row_end) close_row();   // rows ending here, rows without entries included
+                float f[V];
+                Vec<TI>::unpack(raw[u], f);
+#pragma unroll
+                for (int e = 0; e < V; ++e) acc[e] = fmaf(d[u], f[e], acc[e]);
+                ++k;
+            }
+        }
+    }
+    while (row < r1 && k == row_end) close_row();
+}
+
 // One launch for both kinds of work: the first seg_blocks CTAs reduce the segments of the long rows
 // (they are the heaviest items, so they start first), the others the row chunks.
 template <typename TI, typename TO, int L, int C, bool EPI>
@@ -610,12 +673,33 @@ slicegcn_status_t launch_lc(const SpmmParams& p, bool epi, cudaStream_t st) {
     SpmmParams q = p;
     if (!in_kernel) q.seg_done = nullptr;
     if (q.n_seg > 0 && in_kernel) SGCN_CUDA(cudaMemsetAsync(q.seg_done, 0, sizeof(int32_t) * (size_t)q.n_long, st));
-    if (epi)
-        spmm_rows_kernel<TI, TO, L, C, true><<<(unsigned)(blocks + seg_blocks), kRowsWarps * 32, 0, st>>>(q, seg_blocks);
-    else
-        spmm_rows_kernel<TI, TO, L, C, false><<<(unsigned)(blocks + seg_blocks), kRowsWarps * 32, 0, st>>>(q, seg_blocks);
-    SGCN_LAUNCH_CHECK();
-    count_launch();
+    bool narrow = false;
+    if constexpr (L <= 8 && C == 1) {
+        static const bool use_narrow = [] {
+            const char* e = getenv("SLICEGCN_SPMM_NARROW");   // 0: the general kernel for every width (A/B checks)
+            return e ? atoi(e) != 0 : true;
+        }();
+        narrow = use_narrow;
+        if (narrow) {
+            const unsigned nblocks = (unsigned)((warps + 3) / 4);
+            if (epi)
+                spmm_narrow_kernel<TI, TO, L, true><<<nblocks, 128, 0, st>>>(q);
+            else
+                spmm_narrow_kernel<TI, TO, L, false><<<nblocks, 128, 0, st>>>(q);
+            SGCN_LAUNCH_CHECK();
+            count_launch();
+        }
+    }
+    // (with the narrow kernel above only the segment CTAs of this one are launched)
+    const unsigned rows_grid = (unsigned)((narrow ? 0 : blocks) + seg_blocks);
+    if (rows_grid > 0) {
+        if (epi)
+            spmm_rows_kernel<TI, TO, L, C, true><<<rows_grid, kRowsWarps * 32, 0, st>>>(q, seg_blocks);
+        else
+            spmm_rows_kernel<TI, TO, L, C, false><<<rows_grid, kRowsWarps * 32, 0, st>>>(q, seg_blocks);
+        SGCN_LAUNCH_CHECK();
+        count_launch();
+    }
     if (q.n_seg > 0 && !in_kernel) {
         const int pstride = q.nch * Vec<TI>::V;
         if (epi)
