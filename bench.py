@@ -234,14 +234,15 @@ def whole_job_rate(world: int, steps: int, elapsed_ms: float) -> float:
     return world * steps / (elapsed_ms / 1e3)
 
 
-def measure(workload: str, steps: int, warmup: int, world: int, local_rank: int, with_e2e: bool, dist=None):
+def measure(workload: str, steps: int, warmup: int, world: int, local_rank: int, with_e2e: bool, dist=None, fraction: float = 1.0):
     """Device-resident timing (and, if asked, the end-to-end run from host buffers) of one workload.
-    Returns the fields of the JSON line that depend on the workload."""
+    Returns the fields of the JSON line that depend on the workload.  fraction < 1 shrinks the graph (same generator,
+    that share of the nodes and edges): a profiling aid for counter captures, which must stay on small cases."""
     import torch
     from paper_2408_11500_b200 import binding as B
 
     dev = torch.device("cuda", local_rank)
-    w = synth.WORKLOADS[workload]
+    w = scaled_workload(workload, fraction)
     src, dst = synth.make_graph(w, 0)
     Xh = synth.make_features(w, 0)
     yh = synth.uniform_labels(w["n"], w["classes"], 0)
@@ -322,7 +323,7 @@ def measure(workload: str, steps: int, warmup: int, world: int, local_rank: int,
     peak, peak_src = measured_peak_gbs()
     spmm_avg_ms = prof["spmm_ms"] / max(prof["spmm_calls"], 1)
     achieved = (prof["spmm_bytes"] / 1e9) / (prof["spmm_ms"] / 1e3) if prof["spmm_ms"] > 0 else 0.0
-    traffic, traffic_src = NCU_SPMM_TRAFFIC.get(workload, (None, None))
+    traffic, traffic_src = NCU_SPMM_TRAFFIC.get(workload, (None, None)) if fraction >= 1.0 else (None, None)
     ms_per_step = ms_total / steps
     out = {
         "value": whole_job_rate(world, steps, ms_total), "ms_per_step": ms_per_step,
@@ -332,7 +333,7 @@ def measure(workload: str, steps: int, warmup: int, world: int, local_rank: int,
                    "layers": w["layers"], "classes": w["classes"], "num_slices": w["p"], "use_ff": w["use_ff"],
                    "use_se": w["use_se"], "parallelism": "replicas only" if world > 1 else "single GPU",
                    "l2": "working set per epoch is larger than L2 (no flush needed)", "final_loss": final_loss,
-                   "input_aggregate_cached": bool(not w["use_ff"])},
+                   "input_aggregate_cached": bool(not w["use_ff"]), "fraction_of_workload": fraction},
         "clocks": clocks,
         "gpu_launches": int(prof["kernel_launches"]),
         "roofline": {"bound": "hbm", "kernel": "spmm_rows_kernel",
@@ -393,13 +394,13 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
     steps = args.steps if args.steps > 0 else DEFAULT_STEPS[args.workload]
-    main_part = measure(args.workload, steps, args.warmup, world, local_rank, True, dist)
+    main_part = measure(args.workload, steps, args.warmup, world, local_rank, True, dist, args.fraction)
     line = {"metric": "full-graph GCN training throughput", "value": main_part.pop("value"), "unit": "epochs/s",
             "n_gpus": world, "steps": steps, "warmup": args.warmup, "ms_per_step": main_part.pop("ms_per_step"),
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "data": "synthetic"}
     line.update(main_part)
     # the other model workloads, device-resident timing only (one line covers all three)
-    if world == 1 and not args.no_secondary:
+    if world == 1 and not args.no_secondary and args.fraction >= 1.0:
         line["secondary"] = []
         for name in [k for k in ("citation", "social", "copurchase") if k != args.workload]:
             part = measure(name, DEFAULT_STEPS[name] if args.steps <= 0 else min(DEFAULT_STEPS[name], max(args.steps, 5)),
@@ -439,6 +440,8 @@ def main():
     ap.add_argument("--cpu-fraction", type=float, default=0.0, help="size of the oracle's timed sample (0: a default per workload)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-secondary", action="store_true", help="skip the device-resident timing of the other workloads")
+    ap.add_argument("--fraction", type=float, default=1.0,
+                    help="shrink the workload to this share of its nodes and edges (profiling aid: not the benchmark configuration)")
     ap.add_argument("--sweep", action="store_true",
                     help="the SpMM kernel sweep on R-MAT graphs with the oracle's leg; the remaining arguments are spmm_sweep.py's")
     args, rest = ap.parse_known_args()

@@ -881,6 +881,12 @@ def test_epoch_with_dropout_masks(B, torch, kw, rate):
         with_ones = gp.grads.clone()
         gp.epoch(None)
         assert torch.equal(with_ones, gp.grads)
+        # the evaluation pass (no dropout) on the same model object, padded internal layout included
+        want = gp.logits.clone()
+        got_l = torch.full_like(gp.logits, float("nan"))
+        B.slicegcn_forward_logits(gp.m, gp.g, gp.X, gp.X.shape[1], gp.params, got_l, gp.ws, gp.ws_bytes, st)
+        torch.cuda.synchronize()
+        assert torch.equal(got_l, want)
         with pytest.raises(B.SliceGCNError):
             run(1.0)
     finally:
