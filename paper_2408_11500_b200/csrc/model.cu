@@ -394,8 +394,19 @@ slicegcn_status_t layer_backward_impl(const slicegcn_graph* g, const slicegcn_la
         dzm.lda = dout_ld;
         dzm.a_mask = mask;
         dzm.a_mask_ld = L.mask_ld;
-        const bool in_producers = (!need_w || (dW_agg && tc_wgrad_masks_in_producer(wm))) &&
-                                  (!dH_in || (!seq && tc_gemm_masks_in_producer(dzm)));
+        // (a fused input shared by all slices: its dZ is ONE product over the stacked weight blocks, which takes the mask
+        // like any other single-group product)
+        bool dz_masked_ok = true;
+        if (dH_in) {
+            if (shared_in) {
+                GemmArgs probe = stacked(dzm);
+                probe.ldc = L.zt_ld;
+                dz_masked_ok = tc_gemm_masks_in_producer(probe);
+            } else {
+                dz_masked_ok = !seq && tc_gemm_masks_in_producer(dzm);
+            }
+        }
+        const bool in_producers = (!need_w || (dW_agg && tc_wgrad_masks_in_producer(wm))) && dz_masked_ok;
         if (in_producers) {
             w = wm;
             dz = dzm;

@@ -1,15 +1,17 @@
 // Normalised sparse aggregation  Y = A_hat X  (Eq. 1 / Eq. 6 neighbor sum; A_hat^T X in backward).
 //
-// Row-parallel CSR kernel over row-aligned chunks of ~kChunk stored entries (common.cuh).  A group of
-// L lanes streams one chunk; each lane keeps C 16-byte chunks of the output row in registers, so one
-// 128-bit load per lane per chunk covers a neighbor's slice row.  Column indices are read coalesced
-// (a batch of L or 2 L at a time) together with the neighbor's 1/sqrt(deg), parked in a per-warp shared-memory
-// slot and read back as one broadcast load per neighbor; a few neighbors are gathered before the FMAs so
-// several rows are in flight per lane.  No per-edge value array exists:  A_hat_ij = dinv_i * dinv_j.
-// Rows longer than kLongRow are cut into kSegment-entry segments, one warp each (same launch); a row
-// of one segment is finished by that warp, the others leave partial rows, and the warp that arrives
-// last at the row's counter (an integer atomic) sums them in segment order -- deterministic, no
-// floating-point atomics, no second launch (rows narrower than 512 bytes keep a small second kernel).
+// Row-parallel CSR over row-aligned chunks of ~kChunk stored entries (common.cuh).  A group of L lanes streams one
+// chunk; each lane keeps C 16-byte chunks of the output row in registers, so one 128-bit load per lane per chunk covers
+// a neighbor's slice row.  No per-edge value array exists:  A_hat_ij = row_scale_i * col_scale_j.  Rows longer than
+// kLongRow are cut into kSegment-entry segments, one warp each (same launch); a row of one segment is finished by that
+// warp, the others leave partial rows that are summed in segment order -- deterministic, no floating-point atomics.
+// Two gather loops share this structure:
+//   - the staged kernel (rows of 512 bytes and more, a whole warp per chunk): column indices and the neighbor's scale
+//     are read coalesced a batch at a time, parked in a per-warp shared-memory slot and read back as one broadcast
+//     load per neighbor, row metadata handed out by shuffles; the warp that arrives last at a split row's counter
+//     (an integer atomic) sums its partial rows, so there is no second launch;
+//   - the direct kernel (rows of at most 256 bytes, 32/L chunks per warp): every lane group walks its chunk with plain
+//     loads and no cooperation inside the warp; a small second launch sums the partial rows.
 #include <vector>
 
 #include "common.cuh"
@@ -159,9 +161,8 @@ template <int L, int C>
 constexpr int kGatherRound = kDenseWarps<L, C> ? (C == 2 ? 2 : 4) : ((8 / C) < 2 ? 2 : (8 / C));
 template <int L, int C>
 constexpr int kRowsBlocksPerSm = (kDenseWarps<L, C> ? 32 : 20) / kRowsWarps;
-// Column indices a lane fetches per batch: a lane group of L < 32 lanes works on batches of 2 L entries,
-// so that narrow rows (few lanes per row, several rows per warp) see full gather rounds.  (Four or
-// eight indices per lane measured 3-5x slower: the unrolled body no longer fits the instruction cache.)
+// Column indices a lane fetches per batch.  (The loop is written for any lane-group width L; only L = 32 is
+// instantiated -- rows narrower than 512 bytes take the direct kernel -- so a batch is 32 entries, one per lane.)
 template <int L>
 constexpr int kIdxPerLane = L >= 32 ? 1 : 2;
 template <int L>
@@ -275,7 +276,6 @@ __device__ __forceinline__ void spmm_rows_block(const SpmmParams& p, const int64
         for (int t = 0; t < cnt;) {
             uint4 raw[U][C];
             int2 meta[U];
-            // (narrow rows skip this branch: their lane groups stay converged on the general round, 3-6 % faster)
             if (L >= 16 && t + U <= cnt && row_end - kk >= U) {
                 // fast round: U entries of the current row, no row end among them
 #pragma unroll
@@ -465,7 +465,7 @@ __device__ __forceinline__ void spmm_segment_block(const SpmmParams& p, const in
                 }
             }
         }
-        if (p.seg_done == nullptr) return;   // narrow rows: a second launch sums the partial rows
+        if (p.seg_done == nullptr) return;   // (no counters given: a second launch sums the partial rows)
         const int s0 = __ldg(p.seg_ptr + li), s1 = __ldg(p.seg_ptr + li + 1);
         int last = 0;
         __syncwarp();          // every lane's stores are ordered before lane 0's fence ...
@@ -517,19 +517,105 @@ __device__ __forceinline__ void spmm_segment_block(const SpmmParams& p, const in
     }
 }
 
-// Rows of at most 128 bytes (one to eight 16-byte chunks): L lanes per row-aligned chunk, 32/L chunks per warp, and NO
-// cooperation between the lanes of a warp -- every lane group walks its own chunk with plain loads (the L lanes of a
-// group read the same index and scale, which the load unit broadcasts), four neighbors requested before they are
-// accumulated, rows closed where the running entry index meets the row's end.  The general kernel above stages indices
-// in shared memory and hands row metadata around by shuffles, which pays for wide rows; for these narrow ones its
-// per-batch bookkeeping (a batch is 2 L entries) is most of the instructions.  Long rows stay with the segment path.
-template <typename TI, typename TO, int L, bool EPI>
-__global__ void __launch_bounds__(128) spmm_narrow_kernel(const SpmmParams p) {
+// The direct kernel: L lanes per row-aligned chunk (32/L chunks per warp), each lane C 16-byte chunks of the row, and NO
+// cooperation between the lane groups of a warp -- every group walks its own chunk with plain loads (the lanes of a
+// group read the same index and scale, which the load unit broadcasts), a few neighbors requested before they are
+// accumulated, rows closed where the running entry index meets the row's end.  The staged kernel above parks indices
+// in shared memory and hands row metadata around by shuffles; measured, its per-batch bookkeeping costs more than it
+// saves wherever this kernel is used (see launch_direct).
+template <int C>
+constexpr int kDirectRound = C == 1 ? 4 : 2;   // neighbors requested per round: four 16-byte loads per lane in flight
+
+// The 128-entry segments of the long rows: the 32/L lane groups of a warp take consecutive parts of the segment, each
+// with plain loads as above, and are combined by a butterfly in a fixed order; a row of one segment is finished here,
+// the others leave their partial row to spmm_long_finish_kernel.
+template <typename TI, typename TO, int L, int C, bool EPI>
+__device__ __forceinline__ void spmm_direct_segment(const SpmmParams& p, const int vseg) {
     constexpr int V = Vec<TI>::V;
-    constexpr int U = 4;
+    constexpr int U = kDirectRound<C>;
+    constexpr int GS = kSegment / (32 / L);   // entries of a segment per lane group
     const int lane = threadIdx.x & 31;
     const int sub = lane / L, sl = lane % L;
-    const int64_t chunk = ((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5) * (32 / L) + sub;
+    const int seg = __ldg(p.seg_order + vseg);
+    const int li = __ldg(p.seg_row + seg);
+    const int row = __ldg(p.long_rows + li);
+    const int start = __ldg(p.rowptr + row) + (seg - __ldg(p.seg_ptr + li)) * kSegment;
+    const int end_seg = min(__ldg(p.rowptr + row + 1), start + kSegment);
+    const int base = start + sub * GS;
+    const int end = min(end_seg, base + GS);
+    const uint32_t row16 = (uint32_t)((p.ldx * (int64_t)sizeof(TI)) >> 4);
+    const uint4* xl[C];
+#pragma unroll
+    for (int c = 0; c < C; ++c) xl[c] = static_cast<const uint4*>(p.X) + min(sl + c * L, p.nch - 1);
+    float acc[C][V];
+#pragma unroll
+    for (int c = 0; c < C; ++c)
+#pragma unroll
+        for (int e = 0; e < V; ++e) acc[c][e] = 0.f;
+    for (int k = base; k < end; k += U) {
+        const int cnt = min(U, end - k);
+        int j[U];
+        float d[U];
+        uint4 raw[U][C];
+#pragma unroll
+        for (int u = 0; u < U; ++u) j[u] = u < cnt ? __ldg(p.colidx + k + u) : 0;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            d[u] = u < cnt ? __ldg(p.cs + j[u]) : 0.f;
+#pragma unroll
+            for (int c = 0; c < C; ++c) raw[u][c] = __ldg(xl[c] + (uint64_t)(uint32_t)j[u] * row16);
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (u < cnt) {   // (slots past the end loaded row 0: never accumulated, whatever it holds)
+#pragma unroll
+                for (int c = 0; c < C; ++c) {
+                    float f[V];
+                    Vec<TI>::unpack(raw[u][c], f);
+#pragma unroll
+                    for (int e = 0; e < V; ++e) acc[c][e] = fmaf(d[u], f[e], acc[c][e]);
+                }
+            }
+        }
+    }
+    __syncwarp();
+#pragma unroll
+    for (int off = L; off < 32; off <<= 1)
+#pragma unroll
+        for (int c = 0; c < C; ++c)
+#pragma unroll
+            for (int e = 0; e < V; ++e) acc[c][e] += __shfl_xor_sync(0xffffffffu, acc[c][e], off);
+    if (sub != 0) return;
+    const bool single = __ldg(p.seg_ptr + li + 1) - __ldg(p.seg_ptr + li) == 1;
+    const float di = single ? __ldg(p.rs + row) : 0.f;
+#pragma unroll
+    for (int c = 0; c < C; ++c) {
+        const int ch = sl + c * L;
+        if (ch >= p.nch) continue;
+        if (single) {
+            finish_chunk<TO, V, EPI>(p, row, ch, di, acc[c]);
+        } else {
+            float* out = p.partial + (int64_t)seg * (p.nch * V) + ch * V;
+#pragma unroll
+            for (int e = 0; e < V; e += 4)
+                *reinterpret_cast<float4*>(out + e) = make_float4(acc[c][e], acc[c][e + 1], acc[c][e + 2], acc[c][e + 3]);
+        }
+    }
+}
+
+// One launch: the first seg_blocks CTAs (four warps, one segment each) take the long rows' segments, the others the chunks.
+template <typename TI, typename TO, int L, int C, bool EPI>
+__global__ void __launch_bounds__(128, 8) spmm_direct_kernel(const SpmmParams p, const int seg_blocks) {
+    constexpr int V = Vec<TI>::V;
+    constexpr int U = kDirectRound<C>;
+    const int lane = threadIdx.x & 31;
+    const int sub = lane / L, sl = lane % L;
+    if ((int)blockIdx.x < seg_blocks) {
+        const int vseg = (int)blockIdx.x * 4 + (threadIdx.x >> 5);
+        if (vseg < p.n_seg) spmm_direct_segment<TI, TO, L, C, EPI>(p, vseg);
+        return;
+    }
+    const int64_t chunk = ((((int64_t)blockIdx.x - seg_blocks) * (int64_t)blockDim.x + threadIdx.x) >> 5) * (32 / L) + sub;
     if (chunk >= p.n_chunks) return;
     const int r0 = __ldg(p.chunk_row + chunk);
     const int r1 = __ldg(p.chunk_row + chunk + 1);
@@ -539,17 +625,24 @@ __global__ void __launch_bounds__(128) spmm_narrow_kernel(const SpmmParams p) {
     int row = r0;
     int row_end = __ldg(p.rowptr + r0 + 1);
     if (row_end - k > kLongRow) return;   // a long row sits alone in its chunk: left to its segments
-    const bool live = sl < p.nch;
     const uint32_t row16 = (uint32_t)((p.ldx * (int64_t)sizeof(TI)) >> 4);
-    const uint4* xl = static_cast<const uint4*>(p.X) + min(sl, p.nch - 1);
-    float acc[V];
+    const uint4* xl[C];
 #pragma unroll
-    for (int e = 0; e < V; ++e) acc[e] = 0.f;
+    for (int c = 0; c < C; ++c) xl[c] = static_cast<const uint4*>(p.X) + min(sl + c * L, p.nch - 1);
+    float acc[C][V];
+#pragma unroll
+    for (int c = 0; c < C; ++c)
+#pragma unroll
+        for (int e = 0; e < V; ++e) acc[c][e] = 0.f;
     auto close_row = [&]() {
         const float di = __ldg(p.rs + row);
-        if (live) finish_chunk<TO, V, EPI>(p, row, sl, di, acc);
 #pragma unroll
-        for (int e = 0; e < V; ++e) acc[e] = 0.f;
+        for (int c = 0; c < C; ++c) {
+            const int ch = sl + c * L;
+            if (ch < p.nch) finish_chunk<TO, V, EPI>(p, row, ch, di, acc[c]);
+#pragma unroll
+            for (int e = 0; e < V; ++e) acc[c][e] = 0.f;
+        }
         ++row;
         row_end = row < r1 ? __ldg(p.rowptr + row + 1) : -1;
     };
@@ -557,22 +650,26 @@ __global__ void __launch_bounds__(128) spmm_narrow_kernel(const SpmmParams p) {
         const int cnt = min(U, k1 - k);
         int j[U];
         float d[U];
-        uint4 raw[U];
+        uint4 raw[U][C];
 #pragma unroll
         for (int u = 0; u < U; ++u) j[u] = u < cnt ? __ldg(p.colidx + k + u) : 0;
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             d[u] = u < cnt ? __ldg(p.cs + j[u]) : 0.f;
-            raw[u] = __ldg(xl + (uint64_t)(uint32_t)j[u] * row16);
+#pragma unroll
+            for (int c = 0; c < C; ++c) raw[u][c] = __ldg(xl[c] + (uint64_t)(uint32_t)j[u] * row16);
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             if (u < cnt) {
                 while (k == row_end) close_row();   // rows ending here, rows without entries included
-                float f[V];
-                Vec<TI>::unpack(raw[u], f);
 #pragma unroll
-                for (int e = 0; e < V; ++e) acc[e] = fmaf(d[u], f[e], acc[e]);
+                for (int c = 0; c < C; ++c) {
+                    float f[V];
+                    Vec<TI>::unpack(raw[u][c], f);
+#pragma unroll
+                    for (int e = 0; e < V; ++e) acc[c][e] = fmaf(d[u], f[e], acc[c][e]);
+                }
                 ++k;
             }
         }
@@ -590,7 +687,7 @@ __global__ void __launch_bounds__(kRowsWarps * 32, kRowsBlocksPerSm<L, C>) spmm_
         spmm_rows_block<TI, TO, L, C, EPI>(p, (int64_t)blockIdx.x - seg_blocks);
 }
 
-// Narrow rows only (see launch_lc): sums the partial rows of each long row in segment order, then scales / applies
+// After the direct kernel (see launch_direct): sums the partial rows of each long row in segment order, then scales / applies
 // the epilogue.
 // One warp per (long row, block of 32 columns): the hub rows with dozens of segments set the
 // kernel's duration, so their columns are spread over many warps.
@@ -660,47 +757,26 @@ __global__ void __launch_bounds__(256) spmm_scalar_kernel(const SpmmParams p) {
     }
 }
 
-template <typename TI, typename TO, int L, int C>
-slicegcn_status_t launch_lc(const SpmmParams& p, bool epi, cudaStream_t st) {
+// Rows of at most 256 bytes (up to sixteen 16-byte chunks): the direct kernel, then one small launch that sums the
+// partial rows of the split long rows.  Measured against the staged kernel at the same widths: 9-27 % faster
+// (co-purchase graph: 16-wide bf16 1.62 -> 1.35 ms, 16-wide fp32 2.21 -> 1.62 ms, 64-wide fp32 4.59 -> 4.01 ms), with
+// bit-identical results.  At 512 bytes and more the staged kernel wins where the operand is near the L2's size
+// (citation graph, 256 bf16: 167 us against 178 us) and loses 2-4 % where DRAM binds anyway; it keeps those widths.
+template <typename TI, typename TO, int L>
+slicegcn_status_t launch_direct(const SpmmParams& p, bool epi, cudaStream_t st) {
     constexpr int RPW = 32 / L;
     const int64_t warps = ((int64_t)p.n_chunks + RPW - 1) / RPW;
-    const int64_t blocks = (warps + kRowsWarps - 1) / kRowsWarps;
-    const int seg_blocks = (p.n_seg + kRowsWarps - 1) / kRowsWarps;
-    // Rows with several segments: for rows of 512 bytes and more the last segment warp to arrive sums the partial
-    // rows (its fence and counter update, ~1 us, are small next to a segment's gathers); for narrower rows that
-    // latency costs more than a second launch (R-MAT scale 20, 238 K segments: +50 us per call), so they keep one.
-    const bool in_kernel = L >= 32;
     SpmmParams q = p;
-    if (!in_kernel) q.seg_done = nullptr;
-    if (q.n_seg > 0 && in_kernel) SGCN_CUDA(cudaMemsetAsync(q.seg_done, 0, sizeof(int32_t) * (size_t)q.n_long, st));
-    bool narrow = false;
-    if constexpr (L <= 8 && C == 1) {
-        static const bool use_narrow = [] {
-            const char* e = getenv("SLICEGCN_SPMM_NARROW");   // 0: the general kernel for every width (A/B checks)
-            return e ? atoi(e) != 0 : true;
-        }();
-        narrow = use_narrow;
-        if (narrow) {
-            const unsigned nblocks = (unsigned)((warps + 3) / 4);
-            if (epi)
-                spmm_narrow_kernel<TI, TO, L, true><<<nblocks, 128, 0, st>>>(q);
-            else
-                spmm_narrow_kernel<TI, TO, L, false><<<nblocks, 128, 0, st>>>(q);
-            SGCN_LAUNCH_CHECK();
-            count_launch();
-        }
-    }
-    // (with the narrow kernel above only the segment CTAs of this one are launched)
-    const unsigned rows_grid = (unsigned)((narrow ? 0 : blocks) + seg_blocks);
-    if (rows_grid > 0) {
-        if (epi)
-            spmm_rows_kernel<TI, TO, L, C, true><<<rows_grid, kRowsWarps * 32, 0, st>>>(q, seg_blocks);
-        else
-            spmm_rows_kernel<TI, TO, L, C, false><<<rows_grid, kRowsWarps * 32, 0, st>>>(q, seg_blocks);
-        SGCN_LAUNCH_CHECK();
-        count_launch();
-    }
-    if (q.n_seg > 0 && !in_kernel) {
+    q.seg_done = nullptr;   // split rows are summed by the second launch
+    const int seg_blocks = (q.n_seg + 3) / 4;
+    const unsigned blocks = (unsigned)((warps + 3) / 4) + (unsigned)seg_blocks;
+    if (epi)
+        spmm_direct_kernel<TI, TO, L, 1, true><<<blocks, 128, 0, st>>>(q, seg_blocks);
+    else
+        spmm_direct_kernel<TI, TO, L, 1, false><<<blocks, 128, 0, st>>>(q, seg_blocks);
+    SGCN_LAUNCH_CHECK();
+    count_launch();
+    if (q.n_seg > 0) {
         const int pstride = q.nch * Vec<TI>::V;
         if (epi)
             spmm_long_finish_kernel<TO, true><<<dim3((q.n_long + 7) / 8, (q.width + 31) / 32), 256, 0, st>>>(q, pstride);
@@ -712,18 +788,35 @@ slicegcn_status_t launch_lc(const SpmmParams& p, bool epi, cudaStream_t st) {
     return SLICEGCN_OK;
 }
 
+// Rows of 512 bytes and more: the staged kernel, a whole warp per chunk (L = 32), C chunks per lane.  Rows with several
+// segments are finished by the last of their segment warps to arrive (its fence and counter update, ~1 us, are small
+// next to a segment's gathers at these widths): no second launch.
+template <typename TI, typename TO, int C>
+slicegcn_status_t launch_staged(const SpmmParams& p, bool epi, cudaStream_t st) {
+    const int64_t blocks = ((int64_t)p.n_chunks + kRowsWarps - 1) / kRowsWarps;
+    const int seg_blocks = (p.n_seg + kRowsWarps - 1) / kRowsWarps;
+    if (p.n_seg > 0) SGCN_CUDA(cudaMemsetAsync(p.seg_done, 0, sizeof(int32_t) * (size_t)p.n_long, st));
+    if (epi)
+        spmm_rows_kernel<TI, TO, 32, C, true><<<(unsigned)(blocks + seg_blocks), kRowsWarps * 32, 0, st>>>(p, seg_blocks);
+    else
+        spmm_rows_kernel<TI, TO, 32, C, false><<<(unsigned)(blocks + seg_blocks), kRowsWarps * 32, 0, st>>>(p, seg_blocks);
+    SGCN_LAUNCH_CHECK();
+    count_launch();
+    return SLICEGCN_OK;
+}
+
 template <typename TI, typename TO>
 slicegcn_status_t launch_vec(const SpmmParams& p, bool epi, int* fault, cudaStream_t st) {
     const int nch = p.nch;
     (void)fault;
-    if (nch <= 2) return launch_lc<TI, TO, 2, 1>(p, epi, st);
-    if (nch <= 4) return launch_lc<TI, TO, 4, 1>(p, epi, st);
-    if (nch <= 8) return launch_lc<TI, TO, 8, 1>(p, epi, st);
-    if (nch <= 16) return launch_lc<TI, TO, 16, 1>(p, epi, st);
-    if (nch <= 32) return launch_lc<TI, TO, 32, 1>(p, epi, st);
-    if (nch <= 64) return launch_lc<TI, TO, 32, 2>(p, epi, st);
-    if (nch <= 96) return launch_lc<TI, TO, 32, 3>(p, epi, st);
-    return launch_lc<TI, TO, 32, 4>(p, epi, st);
+    if (nch <= 2) return launch_direct<TI, TO, 2>(p, epi, st);
+    if (nch <= 4) return launch_direct<TI, TO, 4>(p, epi, st);
+    if (nch <= 8) return launch_direct<TI, TO, 8>(p, epi, st);
+    if (nch <= 16) return launch_direct<TI, TO, 16>(p, epi, st);
+    if (nch <= 32) return launch_staged<TI, TO, 1>(p, epi, st);
+    if (nch <= 64) return launch_staged<TI, TO, 2>(p, epi, st);
+    if (nch <= 96) return launch_staged<TI, TO, 3>(p, epi, st);
+    return launch_staged<TI, TO, 4>(p, epi, st);
 }
 
 template <typename TI, typename TO>
