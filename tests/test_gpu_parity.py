@@ -174,6 +174,58 @@ def test_spmm_transposed_on_directed_graph(B, torch):
         B.slicegcn_graph_destroy(g)
 
 
+def _degenerate_graphs():
+    """(name, n, src, dst, symmetrize, add_self_loops): the shapes where a row-partitioned SpMM has special cases."""
+    e = np.zeros(0, np.int32)
+    ar = lambda *v: np.array(v, np.int32)
+    star_n = 3000
+    spokes = np.arange(1, star_n, dtype=np.int32)
+    hub = np.zeros(star_n - 1, np.int32)
+    chain = np.arange(0, 199, dtype=np.int32)
+    return [
+        ("one node, its loop only", 1, e, e, False, True),
+        ("one node, no entry at all", 1, e, e, False, False),
+        ("two nodes, one directed edge, empty row and empty column", 2, ar(0), ar(1), False, False),
+        ("isolated nodes between edges, no loops (empty rows, dinv = 0)", 40, ar(3, 3, 17, 38), ar(4, 38, 4, 39), True, False),
+        ("star: one row of n entries cut into segments, n-1 rows of two", star_n, hub, spokes, True, True),
+        ("directed star, no loops: one full row, every other row empty", star_n, hub, spokes, False, False),
+        ("path of 200 nodes: every row shorter than a chunk", 200, chain, chain + 1, True, True),
+        ("exactly 64 and 65 entries in a row (the split threshold)", 200,
+         np.concatenate([np.full(63, 0, np.int32), np.full(64, 100, np.int32)]),
+         np.concatenate([np.arange(1, 64, dtype=np.int32), np.arange(101, 165, dtype=np.int32)]), False, True),
+    ]
+
+
+@pytest.mark.parametrize("idx", range(8))
+def test_spmm_degenerate_graphs(B, torch, idx):
+    """Empty rows and columns, a single node, one row holding almost every entry, rows right at the length where
+    they are cut into segments: forward and transposed, on the narrow-row kernel (widths 3, 16) and the wide-row one
+    (256, 300), fp32 and bf16, against the oracle."""
+    name, n, src, dst, sym, loops = _degenerate_graphs()[idx]
+    og = orc.build_graph(n, src, dst, sym, loops)
+    g = B.slicegcn_graph_create(n, src, dst, (B.SYMMETRIZE if sym else 0) | (B.ADD_SELF_LOOPS if loops else 0))
+    try:
+        info = B.slicegcn_graph_info(g)
+        assert info["nnz"] == og.nnz, name
+        if "split threshold" in name:
+            assert sorted(og.deg.tolist())[-2:] == [64, 65]
+        for width, dt in ((3, B.F32), (16, B.F32), (16, B.BF16), (256, B.F32), (256, B.BF16), (300, B.F32)):
+            X = synth.gaussian_features(n, width, seed=7 + width)
+            for transpose in (False, True):
+                got, x_used = _gpu_spmm(B, torch, g, X, width, dt, transpose=transpose, ld_pad=1 if width == 3 else 0)
+                want = orc.spmm(og, x_used.astype(np.float64), transpose=transpose)
+                assert np.isfinite(got).all(), (name, width, transpose)
+                if dt == B.F32:
+                    assert np.abs(got - want).max() <= 2e-6 * np.abs(want).max(), (name, width, transpose)
+                else:
+                    assert np.all(np.abs(got - want) <= 2 ** -8 * np.abs(want) + 1e-5 * np.abs(want).max()), (name, width)
+                empty = (np.bincount(og.colidx, minlength=n) if transpose else np.diff(og.rowptr)) == 0
+                assert not got[empty].any(), (name, "rows without entries are written as zeros")
+        assert B.slicegcn_graph_device_status(g) == 0
+    finally:
+        B.slicegcn_graph_destroy(g)
+
+
 @pytest.mark.parametrize("norm", ["mean", "sum"])
 def test_spmm_mean_and_sum_aggregators(B, torch, norm):
     """The other aggregators (graph flags NORM_MEAN: D^-1 A, NORM_SUM: A) through the same kernels: forward and
