@@ -451,6 +451,52 @@ int64_t wgrad_scratch_bytes(int64_t M, int groups, int K, int N) {
     return best;
 }
 
+// Width of the column blocks wgrad_run cuts a single group's dW into (0: it is not cut).
+static int wgrad_col_block(const WgradArgs& a) {
+    if (!a.fault || a.K < 1 || !a.dW || a.groups != 1 || a.N % 4 != 0 || a.ldw != 0) return 0;
+    if (a.N > 256) return 256;
+    if (a.b_mask && a.N > 128 && a.N % 16 == 0 && !tc_wgrad_masks_in_producer(a)) {
+        WgradArgs s = a;
+        s.N = 128;
+        s.ldw = a.N;
+        if (tc_wgrad_masks_in_producer(s)) return 128;
+    }
+    return 0;
+}
+
+// Groups per launch when a masked grouped product is too wide for one launch with the mask in the producer but
+// fits as several launches over runs of consecutive groups (0: no such split).
+static WgradArgs wgrad_group_run(const WgradArgs& a, int g0, int gb) {
+    WgradArgs s = a;
+    s.groups = gb;
+    for (int g = 0; g < gb; ++g) {
+        s.a_start[g] = a.a_start[g0 + g];
+        s.b_start[g] = a.b_start[g0 + g];
+    }
+    s.dW = a.dW + (int64_t)g0 * a.K * a.N;
+    s.dbias = a.dbias ? a.dbias + g0 * a.N : nullptr;
+    s.dbias2 = a.dbias2 ? a.dbias2 + g0 * a.N : nullptr;
+    return s;
+}
+
+static int wgrad_mask_group_block(const WgradArgs& a) {
+    if (!a.fault || !a.b_mask || a.K < 1 || !a.dW || a.groups < 2 || a.ldw != 0 || tc_wgrad_masks_in_producer(a)) return 0;
+    for (int gb = a.groups / 2; gb >= 1; gb /= 2) {
+        if (a.groups % gb) continue;
+        bool ok = true;
+        for (int g0 = 0; g0 < a.groups && ok; g0 += gb) ok = tc_wgrad_masks_in_producer(wgrad_group_run(a, g0, gb));
+        if (ok) return gb;
+    }
+    return 0;
+}
+
+bool wgrad_masks_in_producer(const WgradArgs& a) {
+    if (tc_wgrad_masks_in_producer(a)) return true;
+    static const bool no_tc = getenv("SLICEGCN_NO_TC") != nullptr;
+    if (no_tc || !a.b_mask) return false;
+    return (a.N <= 256 && wgrad_col_block(a) == 128) || wgrad_mask_group_block(a) > 0;
+}
+
 slicegcn_status_t wgrad_run(const WgradArgs& a, void* scratch, int64_t scratch_bytes, cudaStream_t st) {
     if (a.M < 1 || a.groups < 1 || a.groups > SLICEGCN_MAX_SLICES || a.N < 1 || a.K < 0)
         SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "wgrad: bad shape");
@@ -476,12 +522,14 @@ slicegcn_status_t wgrad_run(const WgradArgs& a, void* scratch, int64_t scratch_b
             return SLICEGCN_OK;
         }
     }
-    // one group wider than a tensor-core tile (256 result columns): column blocks of dW, one launch each
-    if (!no_tc && a.fault && a.K >= 1 && a.dW && a.groups == 1 && a.N > 256 && a.N % 4 == 0 && a.ldw == 0) {
+    // one group wider than a tensor-core tile (256 result columns; 128 when B carries a byte mask, whose tiles share
+    // the kernel's shared memory): column blocks of dW, one launch each
+    const int col_block = wgrad_col_block(a);
+    if (!no_tc && col_block > 0) {
         bool all = true;
-        for (int c0 = 0; c0 < a.N; c0 += 256) {
+        for (int c0 = 0; c0 < a.N; c0 += col_block) {
             WgradArgs s = a;
-            s.N = std::min(256, a.N - c0);
+            s.N = std::min(col_block, a.N - c0);
             s.b_start[0] = a.b_start[0] + c0;
             s.dW = a.dW + c0;
             s.ldw = a.N;
@@ -503,6 +551,21 @@ slicegcn_status_t wgrad_run(const WgradArgs& a, void* scratch, int64_t scratch_b
             }
         }
         if (all) return SLICEGCN_OK;
+    }
+    if (const int gb = no_tc ? 0 : wgrad_mask_group_block(a)) {   // masked, too wide for one launch: runs of gb groups
+        for (int g0 = 0; g0 < a.groups; g0 += gb) {
+            const WgradArgs s = wgrad_group_run(a, g0, gb);
+            bool done_g = false;
+            SGCN_TRY(tc_wgrad_run(s, scratch, scratch_bytes, st, &done_g));
+            if (bias && !done_g) {
+                WgradArgs b = s;
+                b.K = 0;
+                b.dW = nullptr;
+                b.fault = nullptr;
+                SGCN_TRY(wgrad_run(b, scratch, scratch_bytes, st));
+            }
+        }
+        return SLICEGCN_OK;
     }
     if (!no_tc && a.fault && a.K >= 1 && a.dW) {
         bool bias_done = false;

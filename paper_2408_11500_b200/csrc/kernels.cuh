@@ -122,7 +122,8 @@ struct WgradArgs {
 };
 int64_t wgrad_scratch_bytes(int64_t M, int groups, int K, int N);
 int64_t tc_wgrad_scratch_bytes(const WgradArgs& a);
-bool tc_wgrad_masks_in_producer(const WgradArgs& a);   // the same question for a.b_mask
+bool tc_wgrad_masks_in_producer(const WgradArgs& a);   // the same question for a.b_mask, one launch
+bool wgrad_masks_in_producer(const WgradArgs& a);      // ... for wgrad_run, which may cut dW into column blocks
 // bias_done (optional): set when the column sums (dbias / dbias2) were produced as well
 slicegcn_status_t tc_wgrad_run(const WgradArgs& a, void* scratch, int64_t scratch_bytes, cudaStream_t st, bool* bias_done = nullptr);
 slicegcn_status_t wgrad_run(const WgradArgs& a, void* scratch, int64_t scratch_bytes, cudaStream_t st);

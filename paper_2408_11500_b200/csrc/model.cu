@@ -406,7 +406,7 @@ slicegcn_status_t layer_backward_impl(const slicegcn_graph* g, const slicegcn_la
                 dz_masked_ok = !seq && tc_gemm_masks_in_producer(dzm);
             }
         }
-        const bool in_producers = (!need_w || (dW_agg && tc_wgrad_masks_in_producer(wm))) && dz_masked_ok;
+        const bool in_producers = (!need_w || (dW_agg && wgrad_masks_in_producer(wm))) && dz_masked_ok;
         if (in_producers) {
             w = wm;
             dz = dzm;
@@ -682,8 +682,11 @@ slicegcn_status_t build_layout(const slicegcn_model* m, const slicegcn_graph* g,
     E.ld_grad = gw;
     E.ld_clsm = align_up(D.hidden, 16);
     E.ld_ffm = align_up(D.in_d, 16);
-    E.gate_masks = n * E.ld_cls * esz >= ((int64_t)512 << 20);
-    if (const char* force = getenv("SLICEGCN_GATE_MASKS")) E.gate_masks = atoi(force) != 0;   // tests reach both forms at small sizes
+    // The ReLUs of the classifier and of the fusion MLP leave a byte mask; their backward products are stored ungated
+    // and the consumers multiply by the mask in their producers (see the classifier's backward below).  Without the
+    // masks (SLICEGCN_GATE_MASKS=0: the tests reach both forms) the products are gated by the activation in their epilogue.
+    E.gate_masks = true;
+    if (const char* force = getenv("SLICEGCN_GATE_MASKS")) E.gate_masks = atoi(force) != 0;
     if (D.use_ff) {
         E.ff_act = b.take(n * E.ld_ffact * esz);
         if (E.gate_masks) E.ff_mask = static_cast<uint8_t*>(b.take(n * E.ld_ffm));
@@ -1252,7 +1255,6 @@ static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, 
             a.mul_pos_dtype = kGateBytes;
         }
         a.reverse = 1;
-        SGCN_TRY(gemm_run(a, st));
         WgradArgs w1;
         w1.fault = g->fault;
         w1.M = n;
@@ -1265,7 +1267,6 @@ static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, 
         w1.ldb = E.ld_cls;
         w1.dW = grads + m->Wc1;
         w1.dbias = grads + m->bc1;
-        SGCN_TRY(wgrad_run(w1, E.ws, E.ws_bytes, st));
         GemmArgs h;   // dH = dA Wc1^T
         h.fault = g->fault;
         h.b_image = E.tc_img;
@@ -1280,6 +1281,25 @@ static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, 
         h.b_trans = 1;
         h.C = E.dH[0];
         h.ldc = E.ld_grad;
+        if (E.gate_masks) {
+            // A gate read in the epilogue costs that product two thirds of its time (its loads queue behind the
+            // epilogue's own stores: 421 us with the gate against 140 us without, on a fifth of the largest
+            // workload).  Both consumers of dA can multiply by the byte mask on their operand's way to the tensor
+            // cores instead (a mask tile travels next to every slab), so dA is stored ungated.
+            WgradArgs w1m = w1;
+            w1m.b_mask = E.cls_mask;
+            w1m.b_mask_ld = E.ld_clsm;
+            GemmArgs hm = h;
+            hm.a_mask = E.cls_mask;
+            hm.a_mask_ld = E.ld_clsm;
+            if (wgrad_masks_in_producer(w1m) && tc_gemm_masks_in_producer(hm)) {
+                a.mul_pos = nullptr;
+                w1 = w1m;
+                h = hm;
+            }
+        }
+        SGCN_TRY(gemm_run(a, st));
+        SGCN_TRY(wgrad_run(w1, E.ws, E.ws_bytes, st));
         SGCN_TRY(gemm_run(h, st));
     }
     int cur = 0;
@@ -1340,7 +1360,6 @@ static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, 
             a.mul_pos_ld = E.ld_ffm;
             a.mul_pos_dtype = kGateBytes;
         }
-        SGCN_TRY(gemm_run(a, st));
         WgradArgs w1;
         w1.fault = g->fault;
         w1.M = n;
@@ -1354,6 +1373,16 @@ static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, 
         w1.ldb = E.ld_grad;
         w1.dW = grads + m->ff_W1;
         w1.dbias = grads + m->ff_b1;
+        if (E.gate_masks) {   // as for the classifier: the one consumer of this gradient applies the mask itself
+            WgradArgs w1m = w1;
+            w1m.b_mask = E.ff_mask;
+            w1m.b_mask_ld = E.ld_ffm;
+            if (wgrad_masks_in_producer(w1m)) {
+                a.mul_pos = nullptr;
+                w1 = w1m;
+            }
+        }
+        SGCN_TRY(gemm_run(a, st));
         SGCN_TRY(wgrad_run(w1, E.ws, E.ws_bytes, st));
     }
     // ---------------- update: Adam, cosine-annealed learning rate, one step per epoch

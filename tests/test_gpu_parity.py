@@ -530,11 +530,13 @@ def test_epoch_gradients_fp32(B, kw):
         gp.close()
 
 
+@pytest.mark.parametrize("masks", ["0", "1"])
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-def test_epoch_with_byte_mask_gates(B, dtype, monkeypatch):
-    """Large problems gate the backward products of the classifier and of the fusion MLP by the forward ReLU's
-    byte mask instead of the activation; SLICEGCN_GATE_MASKS=1 selects that form at test size."""
-    monkeypatch.setenv("SLICEGCN_GATE_MASKS", "1")
+def test_epoch_with_byte_mask_gates(B, dtype, masks, monkeypatch):
+    """Both forms of the ReLU gates in the backward products of the classifier and of the fusion MLP: the forward
+    pass's byte masks applied by the consumers of those gradients (the default), and the activation itself read in
+    the products' epilogue (SLICEGCN_GATE_MASKS=0)."""
+    monkeypatch.setenv("SLICEGCN_GATE_MASKS", masks)
     src, dst, X, y, mk, od, params = small_problem(n=1500, m_edges=9000, in_d=100, hidden=128, L=2, C=11, p=4,
                                                    use_ff=True, use_se=True)
     og = orc.build_graph(len(X), src, dst, True, True)
