@@ -2176,6 +2176,7 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
                                                                     const __grid_constant__ CUtensorMap map_bm) {
     extern __shared__ __align__(1024) unsigned char smem[];
     constexpr int R = WIDE ? 2 : 4, S = 2;   // raw slots; operand stages (TMEM A + shared-memory B)
+    constexpr uint32_t kARaw = ABF16 ? 8192u : 16384u;   // raw A slab: 32 rows x 128 columns
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int mt = blockIdx.y, chunk = blockIdx.x;
     unsigned char* base = smem + ((1024u - (smem_u32(smem) & 1023u)) & 1023u);
@@ -2184,11 +2185,11 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
     const bool masked = a.b_mask != nullptr;                 // B is multiplied by a byte mask on the way
     const uint32_t b_raw_pad = (b_raw_bytes + 1023u) & ~1023u;
     const uint32_t m_raw_bytes = 32u * (uint32_t)pl.n_t;
-    const uint32_t slot_bytes = 16384u + b_raw_pad + (masked ? ((m_raw_bytes + 1023u) & ~1023u) : 0u);   // raw A | raw B | mask
+    const uint32_t slot_bytes = kARaw + b_raw_pad + (masked ? ((m_raw_bytes + 1023u) & ~1023u) : 0u);   // raw A | raw B | mask
     const uint32_t op_bytes = (uint32_t)nbk * 8192u;         // B operand stage: 8 K atoms x (nbk hi + nbk lo) x 512 B
     unsigned char* ops = base;                               // [S]
     unsigned char* raw = ops + S * op_bytes;                 // [R]
-    float* csum_s = reinterpret_cast<float*>(raw + 16384);   // [4][128] column-sum partials: reuse the B part of raw slot 0 after the last slab
+    float* csum_s = reinterpret_cast<float*>(raw + kARaw);   // [4][128] column-sum partials: reuse the B part of raw slot 0 after the last slab
     uint64_t* afull = reinterpret_cast<uint64_t*>(raw + R * slot_bytes);   // [S] 128 producer arrivals
     uint64_t* afree = afull + S;                             // [S] MMAs of the stage completed
     uint64_t* rfull = afree + S;                             // [R] raw slab landed
@@ -2310,8 +2311,8 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
             if (!okp) break;
             const unsigned char* slot = raw + rs * slot_bytes;
             if (b_mine) {
-                const unsigned char* braw = slot + 16384 + b_cc * 16;
-                const unsigned char* mraw = slot + 16384 + b_raw_pad + b_cc * 4;
+                const unsigned char* braw = slot + kARaw + b_cc * 16;
+                const unsigned char* mraw = slot + kARaw + b_raw_pad + b_cc * 4;
                 unsigned char* op = ops + ts * op_bytes;
 #pragma unroll
                 for (int i = 0; i < BI; ++i) {
@@ -2410,8 +2411,8 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
                 const int y = (int)(r_begin + (int64_t)j * 32);
                 mbar_expect_tx(&rfull[rs], (ABF16 ? 64u : 128u) * (uint32_t)pl.a_box + b_raw_bytes + (masked ? m_raw_bytes : 0u));
                 tma_load_2d(slot, &map_a, ax, y, &rfull[rs]);
-                tma_load_2d(slot + 16384, &map_b, bx, y, &rfull[rs]);
-                if (masked) tma_load_2d(slot + 16384 + b_raw_pad, &map_bm, bx, y, &rfull[rs]);
+                tma_load_2d(slot + kARaw, &map_b, bx, y, &rfull[rs]);
+                if (masked) tma_load_2d(slot + kARaw + b_raw_pad, &map_bm, bx, y, &rfull[rs]);
                 if (++rs == R) {
                     rs = 0;
                     ++rpass;
@@ -2578,8 +2579,10 @@ bool wgrad_ts_ok(const WgradArgs& a, const WgTcPlan& pl) {
     const int nbk = (pl.n_t + 31) / 32;
     if (nbk > 8 || a.M >= ((int64_t)1 << 31)) return false;
     if (a.a_dtype == SLICEGCN_BF16 && (a.lda % 8 || pl.a_col0 % 8 || pl.a_tile_cols % 8)) return false;   // 16-byte tensor copies
-    if (a.b_mask) {
-        if (nbk > 4 || (uintptr_t)a.b_mask % 16 || a.b_mask_ld % 16 || pl.b_col0 % 16 || pl.b_cols_per_tile % 16) return false;
+    if (a.b_mask) {   // (the mask tiles of a wide B fit the shared memory only next to the half-size raw slabs of a bf16 A)
+        if (nbk > (a.a_dtype == SLICEGCN_BF16 ? 8 : 4) || (uintptr_t)a.b_mask % 16 || a.b_mask_ld % 16 || pl.b_col0 % 16 ||
+            pl.b_cols_per_tile % 16)
+            return false;
     }
     return true;
 }
@@ -2692,8 +2695,10 @@ slicegcn_status_t tc_wgrad_run(const WgradArgs& a, void* scratch, int64_t scratc
                 if (maps_ok) {
                     const bool want_bias = (a.dbias || a.dbias2) && scratch_bytes >= need_ts + need_cs;
                     float* colsum = want_bias ? static_cast<float*>(scratch) + need_ts / sizeof(float) : nullptr;
-                    const int slot_b = 16384 + ((32 * pn.n_t * 4 + 1023) & ~1023) + (a.b_mask ? ((32 * pn.n_t + 1023) & ~1023) : 0);
+                    const int slot_b = (a.a_dtype == SLICEGCN_BF16 ? 8192 : 16384) + ((32 * pn.n_t * 4 + 1023) & ~1023) +
+                                       (a.b_mask ? ((32 * pn.n_t + 1023) & ~1023) : 0);
                     const int ts_smem = 2 * nbk * 8192 + (wide ? 2 : 4) * slot_b + 256 + 1024;
+                    if (ts_smem > 227 * 1024) return SLICEGCN_ERR_UNSUPPORTED;   // (wgrad_ts_ok rules these shapes out)
                     static bool ts_configured = false;
                     if (!ts_configured) {
                         SGCN_CUDA(cudaFuncSetAttribute(tc_wgrad_ts_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
