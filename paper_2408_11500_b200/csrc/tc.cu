@@ -1275,10 +1275,12 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
                 if (!okm) break;
                 tc_fence_after();
                 const uint32_t d_tmem0 = tmem + (uint32_t)acc * accw;
-                if (ABF16 && fused && concat && ns1 == 1 && ns2 == 1) {
+                if (fused && concat && ns1 == 1 && ns2 == 1) {
                     // One slab per product (the sliced layers' 32-wide blocks): MMAs into one accumulator range depend
                     // on each other and such small ones are bound by that latency, so the two products' chains -- they
-                    // fill different column ranges -- are issued alternately (measured: 14 % off the kernel's time).
+                    // fill different column ranges -- are issued alternately (measured: 12-14 % off the kernel's time).  (Pairing two
+                    // consecutive one-slab items the same way measured slower: the second item's producers and the first
+                    // item's epilogue then wait for each other.)
                     const int ts2 = (ts + 1 == S) ? 0 : ts + 1;
                     const uint32_t pass2 = (ts + 1 == S) ? pass + 1 : pass;
                     okm = mbar_wait(&afull[ts], pass & 1);
@@ -1287,11 +1289,26 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
                     tc_fence_after();
                     const uint32_t a1 = tmem + a_col0 + (uint32_t)ts * 64u, a2 = tmem + a_col0 + (uint32_t)ts2 * 64u;
                     const uint64_t db1 = smem_desc(wring + (uint32_t)ts * slab_bytes), db2 = smem_desc(wring + (uint32_t)ts2 * slab_bytes);
+                    if (ABF16) {
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks) {
-                        const uint64_t adv = (uint64_t)((ks * 32) >> 4);
-                        umma_ts_f16(d_tmem0, a1 + 8u * ks, db1 + adv, idesc_wide, ks == 0 ? 0u : 1u);
-                        umma_ts_f16(d_tmem0 + prodw, a2 + 8u * ks, db2 + adv, idesc_wide, ks == 0 ? 0u : 1u);
+                        for (int ks = 0; ks < 4; ++ks) {
+                            const uint64_t adv = (uint64_t)((ks * 32) >> 4);
+                            umma_ts_f16(d_tmem0, a1 + 8u * ks, db1 + adv, idesc_wide, ks == 0 ? 0u : 1u);
+                            umma_ts_f16(d_tmem0 + prodw, a2 + 8u * ks, db2 + adv, idesc_wide, ks == 0 ? 0u : 1u);
+                        }
+                    } else {   // fp32: A_hi x [B_hi | B_lo] of both products, then A_lo x B_hi of both
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks) {
+                            const uint64_t adv = (uint64_t)((ks * 32) >> 4);
+                            umma_ts_tf32(d_tmem0, a1 + 8u * ks, db1 + adv, idesc_wide, ks == 0 ? 0u : 1u);
+                            umma_ts_tf32(d_tmem0 + prodw, a2 + 8u * ks, db2 + adv, idesc_wide, ks == 0 ? 0u : 1u);
+                        }
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks) {
+                            const uint64_t adv = (uint64_t)((ks * 32) >> 4);
+                            umma_ts_tf32(d_tmem0, a1 + 32u + 8u * ks, db1 + adv, idesc_hi, 1u);
+                            umma_ts_tf32(d_tmem0 + prodw, a2 + 32u + 8u * ks, db2 + adv, idesc_hi, 1u);
+                        }
                     }
                     umma_commit(&afree[ts]);
                     umma_commit(&afree[ts2]);
