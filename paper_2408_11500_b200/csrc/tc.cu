@@ -91,7 +91,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
     const long long t0 = clock64();
     for (int i = 0; i < kWaitSpins; ++i) {
         if (mbar_try(bar, parity)) return true;
-        if (clock64() - t0 > 4000000000LL) break;
+        if ((i & 63) == 63 && clock64() - t0 > 4000000000LL) break;   // (a spinning warp shares its issue slots with working ones)
     }
     return false;
 }
@@ -1465,22 +1465,30 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
                 }
                 const float* bvec = sbias + g * a.N + n0 + c0;
                 const float* pvec = spost + g * a.N + n0 + c0;
-                uint32_t mbits = 0;
-                if (has_vec || a.relu) {
+                uint32_t mword[8];   // the ReLU mask bytes of columns 4q .. 4q+3, one word per column quad
+                if (a.relu) {
 #pragma unroll
-                for (int j = 0; j < 32; j += 4) {
-                    const float4 b4 = *reinterpret_cast<const float4*>(bvec + j);
-                    const float4 p4 = *reinterpret_cast<const float4*>(pvec + j);
-                    x[j] += b4.x; x[j + 1] += b4.y; x[j + 2] += b4.z; x[j + 3] += b4.w;
-                    if (a.relu) {
-#pragma unroll
-                        for (int t = 0; t < 4; ++t) {
-                            mbits |= (x[j + t] > 0.f ? 1u : 0u) << (j + t);
-                            x[j + t] = fmaxf(x[j + t], 0.f);
-                        }
+                    for (int j = 0; j < 32; j += 4) {
+                        const float4 b4 = *reinterpret_cast<const float4*>(bvec + j);
+                        const float4 p4 = *reinterpret_cast<const float4*>(pvec + j);
+                        x[j] += b4.x; x[j + 1] += b4.y; x[j + 2] += b4.z; x[j + 3] += b4.w;
+                        mword[j >> 2] = (x[j] > 0.f ? 1u : 0u) | (x[j + 1] > 0.f ? 0x100u : 0u) | (x[j + 2] > 0.f ? 0x10000u : 0u) |
+                                        (x[j + 3] > 0.f ? 0x1000000u : 0u);
+                        x[j] = fmaxf(x[j], 0.f) + p4.x;
+                        x[j + 1] = fmaxf(x[j + 1], 0.f) + p4.y;
+                        x[j + 2] = fmaxf(x[j + 2], 0.f) + p4.z;
+                        x[j + 3] = fmaxf(x[j + 3], 0.f) + p4.w;
                     }
-                    x[j] += p4.x; x[j + 1] += p4.y; x[j + 2] += p4.z; x[j + 3] += p4.w;
-                }
+                } else if (has_vec) {
+#pragma unroll
+                    for (int j = 0; j < 32; j += 4) {
+                        const float4 b4 = *reinterpret_cast<const float4*>(bvec + j);
+                        const float4 p4 = *reinterpret_cast<const float4*>(pvec + j);
+                        x[j] = (x[j] + b4.x) + p4.x;
+                        x[j + 1] = (x[j + 1] + b4.y) + p4.y;
+                        x[j + 2] = (x[j + 2] + b4.z) + p4.z;
+                        x[j + 3] = (x[j + 3] + b4.w) + p4.w;
+                    }
                 }
                 if (fused) {   // the second product's halves, 16 columns of each per wait
                     tmem_ld16x2_add<0>(d_tmem + prodw + (uint32_t)c0, d_tmem + prodw + (uint32_t)(n_pad + c0), x);
@@ -1493,19 +1501,40 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
 #pragma unroll
                 for (int j = 0; j < 32; j += 4)
                     *reinterpret_cast<float4*>(stage + lane * kStagePitch + j) = make_float4(x[j], x[j + 1], x[j + 2], x[j + 3]);
-                if (wmask) {
-#pragma unroll
-                    for (int j = 0; j < 32; j += 16) {
-                        uint4 mb;
-                        mb.x = ((mbits >> (j + 0)) & 1u) | (((mbits >> (j + 1)) & 1u) << 8) | (((mbits >> (j + 2)) & 1u) << 16) | (((mbits >> (j + 3)) & 1u) << 24);
-                        mb.y = ((mbits >> (j + 4)) & 1u) | (((mbits >> (j + 5)) & 1u) << 8) | (((mbits >> (j + 6)) & 1u) << 16) | (((mbits >> (j + 7)) & 1u) << 24);
-                        mb.z = ((mbits >> (j + 8)) & 1u) | (((mbits >> (j + 9)) & 1u) << 8) | (((mbits >> (j + 10)) & 1u) << 16) | (((mbits >> (j + 11)) & 1u) << 24);
-                        mb.w = ((mbits >> (j + 12)) & 1u) | (((mbits >> (j + 13)) & 1u) << 8) | (((mbits >> (j + 14)) & 1u) << 16) | (((mbits >> (j + 15)) & 1u) << 24);
-                        *reinterpret_cast<uint4*>(mstage + lane * kTsMaskPitch + j) = mb;
-                    }
+                if (wmask) {   // (wmask implies a.relu: mword is set)
+                    *reinterpret_cast<uint4*>(mstage + lane * kTsMaskPitch) = make_uint4(mword[0], mword[1], mword[2], mword[3]);
+                    *reinterpret_cast<uint4*>(mstage + lane * kTsMaskPitch + 16) = make_uint4(mword[4], mword[5], mword[6], mword[7]);
                 }
                 __syncwarp();
                 // ---- phase 2
+                if (rows_here == 32 && col_ok && !a.mul_pos && !a.accumulate) {
+                    // whole tile, plain store (every forward product): no per-row tests, addresses by repeated addition
+                    unsigned char* cp = Cb + (rfirst * a.ldc + col) * (int64_t)sizeof(TC);
+                    uint8_t* mp = wmask ? a.mask_out + rfirst * a.mask_ld + col : nullptr;
+                    const int64_t cstep = 4 * a.ldc * (int64_t)sizeof(TC), mstep = 4 * a.mask_ld;
+                    const float* sp = stage + sub * kStagePitch + cq * 4;
+                    const unsigned char* msp = mstage + sub * kTsMaskPitch + cq * 4;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const float4 t = *reinterpret_cast<const float4*>(sp + 4 * i * kStagePitch);
+                        if (wmask) {
+                            *reinterpret_cast<uint32_t*>(mp) = *reinterpret_cast<const uint32_t*>(msp + 4 * i * kTsMaskPitch);
+                            mp += mstep;
+                        }
+                        if (sizeof(TC) == 4) {
+                            *reinterpret_cast<float4*>(cp) = t;
+                        } else {
+                            const __nv_bfloat162 lo2 = __floats2bfloat162_rn(t.x, t.y), hi2 = __floats2bfloat162_rn(t.z, t.w);
+                            uint2 pk;
+                            pk.x = *reinterpret_cast<const uint32_t*>(&lo2);
+                            pk.y = *reinterpret_cast<const uint32_t*>(&hi2);
+                            *reinterpret_cast<uint2*>(cp) = pk;
+                        }
+                        cp += cstep;
+                    }
+                    __syncwarp();
+                    continue;
+                }
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
                     const int rr = 4 * i + sub;
