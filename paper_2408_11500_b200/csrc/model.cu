@@ -1113,6 +1113,7 @@ static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, 
         c.C = E.xff;
         c.ldc = E.ld_x0;
         c.c_dtype = D.dtype;
+        c.c_pad_write = 1;   // an odd slice width (13 columns): the tile's padding columns are stored too, as zeros
         SGCN_TRY(gemm_run(c, st));
         h0 = E.xff;
         ld0 = E.ld_x0;

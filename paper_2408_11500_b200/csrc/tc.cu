@@ -1381,12 +1381,16 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
         unsigned char* Cb = static_cast<unsigned char*>(a.C);   // bf16 result (no accumulation, no gate)
         const bool wmask = a.relu && a.mask_out;
         const bool has_vec = a.bias || a.post1 || a.post2;   // otherwise the staged vectors are all zero
-        for (int i = tid - 256; i < a.groups * a.N; i += 256) {
-            sbias[i] = a.bias ? __ldg(a.bias + i) : 0.f;
-            float pv = a.post1 ? __ldg(a.post1 + i) : 0.f;
-            if (a.post2) pv += __ldg(a.post2 + i);
+        const int nvec = a.groups * a.N;   // (with padding columns written: zeros up to the padded width)
+        for (int i = tid - 256; i < (a.c_pad_write ? ((nvec + 3) & ~3) : nvec); i += 256) {
+            const bool in = i < nvec;
+            sbias[i] = (in && a.bias) ? __ldg(a.bias + i) : 0.f;
+            float pv = (in && a.post1) ? __ldg(a.post1 + i) : 0.f;
+            if (in && a.post2) pv += __ldg(a.post2 + i);
             spost[i] = pv;
         }
+        // an fp32 result whose rows do not allow 16-byte stores (47 classes): element-wise stores, every other step alike
+        const bool ragged = ((a.N & 3) && !a.c_pad_write) || (a.ldc & 3) || ((uintptr_t)a.C & 15);
         asm volatile("bar.sync 1, 256;" ::: "memory");
         bool oke = true;
         ItemCursor e_it;
@@ -1422,7 +1426,7 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
             const uint32_t d_tmem = tmem + (uint32_t)e * accw + ((uint32_t)(q * 32) << 16);
             for (int c0 = 0; c0 < nn; c0 += 32) {
                 const int n = c0 + cq * 4;            // first of this lane's four columns in phase 2
-                const bool col_ok = n < nn;           // nn is a multiple of 4 on this path
+                const bool col_ok = n < nn;           // (nn is a multiple of 4 unless the result is ragged)
                 const int col = cs + n;
                 // ---- phase 1
                 float x[32];
@@ -1507,7 +1511,7 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
                 }
                 __syncwarp();
                 // ---- phase 2
-                if (rows_here == 32 && col_ok && !a.mul_pos && !a.accumulate) {
+                if (rows_here == 32 && col_ok && !a.mul_pos && !a.accumulate && !ragged) {
                     // whole tile, plain store (every forward product): no per-row tests, addresses by repeated addition
                     unsigned char* cp = Cb + (rfirst * a.ldc + col) * (int64_t)sizeof(TC);
                     uint8_t* mp = wmask ? a.mask_out + rfirst * a.mask_ld + col : nullptr;
@@ -1556,6 +1560,12 @@ __global__ void __launch_bounds__(kTsThreads, 1) tc_gemm_ts_kernel(const GemmArg
                         asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(Cf + row * a.ldc + col), "f"(t.x),
                                      "f"(t.y), "f"(t.z), "f"(t.w)
                                      : "memory");
+                    } else if (ragged) {
+                        float* cp = Cf + row * a.ldc + col;
+                        cp[0] = t.x;
+                        if (n + 1 < nn) cp[1] = t.y;
+                        if (n + 2 < nn) cp[2] = t.z;
+                        if (n + 3 < nn) cp[3] = t.w;
                     } else if (sizeof(TC) == 4) {
                         *reinterpret_cast<float4*>(Cf + row * a.ldc + col) = t;
                     } else {
@@ -1634,7 +1644,7 @@ bool ts_gemm_ok(const GemmArgs& a, int n_pad, int n_tiles) {
     static const bool off = getenv("SLICEGCN_NO_TS") != nullptr || getenv("SLICEGCN_NO_WS") != nullptr;
     const bool abf = a.a_dtype == SLICEGCN_BF16, cbf = a.c_dtype == SLICEGCN_BF16;
     if (off) return false;
-    if (abf && (a.a_mask || a.accumulate || a.mul_pos || a.c_pad_write)) return false;   // forward products only
+    if (abf && (a.a_mask || a.accumulate || a.mul_pos)) return false;   // forward products only
     if (!abf && cbf && (a.accumulate || a.mul_pos || a.c_pad_write || a.A2)) return false;   // a bf16 result is stored, never added to
     const bool fused = a.A2 != nullptr;
     const int epc = abf ? 8 : 4;   // elements per 16 bytes of the activation operand
@@ -1644,9 +1654,10 @@ bool ts_gemm_ok(const GemmArgs& a, int n_pad, int n_tiles) {
         ok = ok && (a.a_start[g] % epc == 0) && (a.c_start[g] % 4 == 0);
         if (fused) ok = ok && (a.a2_start[g] % epc == 0);
     }
-    const bool pad_write = a.c_pad_write && !a.bias && !a.post1 && !a.post2 && !a.relu && !a.mul_pos && a.groups == 1 &&
-                           a.c_start[0] + ((a.N + 3) & ~3) <= a.ldc;
-    ok = ok && (a.N % 4 == 0 || pad_write) && (a.ldc % 4 == 0) && ((uintptr_t)a.C % 16 == 0);
+    const bool pad_write = a.c_pad_write && !a.mask_out && !a.mul_pos && a.groups == 1 && a.c_start[0] + ((a.N + 3) & ~3) <= a.ldc;
+    // an fp32 result with rows that do not allow 16-byte stores is written element by element (one group, plain store)
+    const bool ragged_ok = !cbf && !a.c_pad_write && a.groups == 1 && !a.mask_out && !a.mul_pos && !a.accumulate && !fused;
+    ok = ok && (((a.N % 4 == 0 || pad_write) && (a.ldc % 4 == 0) && ((uintptr_t)a.C % 16 == 0)) || ragged_ok);
     if (a.mask_out) ok = ok && (a.mask_ld % 4 == 0) && ((uintptr_t)a.mask_out % 4 == 0);
     if (a.mul_pos) ok = ok && (a.mul_pos_ld % 4 == 0) && ((uintptr_t)a.mul_pos % 16 == 0);   // (a byte mask would do with 4)
     if (a.a_mask) {
