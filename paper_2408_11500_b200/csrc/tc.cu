@@ -2240,13 +2240,14 @@ __global__ void __launch_bounds__(kWsThreads, 1) tc_wgrad_ws_kernel(const WgradA
 //              rows -- consecutive lanes, consecutive words), splits them and writes hi and lo into a
 //              TMEM stage with tcgen05.st: A^T in the K-major form, M index = TMEM lane.  After the last
 //              slab they drain the accumulator into the scratch tile.
-//   warps 8-11 B producers: split the B slab (times its byte mask, if any) into the MN-major operand
+//   warps 8-15 B producers (they carry the most work per slab -- measured, they set the kernel's pace -- hence eight
+//              warps): split the B slab (times its byte mask, if any) into the MN-major operand
 //              tile ("128-byte swizzle, 32-byte base"; per K atom the hi column blocks are followed by
 //              the lo column blocks, so [hi | lo] is one operand of 2 n_t columns) and keep the column
 //              sums of B (the bias gradient).
 //   warp 4     MMA issuer: per 8 rows A_hi x [B_hi | B_lo] and A_lo x B_hi.
 // TMEM columns: accumulator [hi*hi + lo*hi | hi*lo] (64 nbk), then two stages of 64 (A hi | A lo).
-constexpr int kWtThreads = 384;
+constexpr int kWtThreads = 512;
 
 // WIDE: B tiles of 129..256 columns -- no room for [hi | lo] in one operand (three chains per slab) and
 // only two raw slots.  ABF16: A is stored as bf16 -- exact in tf32, so it has no lo part and a slab takes
@@ -2271,7 +2272,7 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
     const uint32_t op_bytes = (uint32_t)nbk * 8192u;         // B operand stage: 8 K atoms x (nbk hi + nbk lo) x 512 B
     unsigned char* ops = base;                               // [S]
     unsigned char* raw = ops + S * op_bytes;                 // [R]
-    float* csum_s = reinterpret_cast<float*>(raw + kARaw);   // [4][128] column-sum partials: reuse the B part of raw slot 0 after the last slab
+    float* csum_s = reinterpret_cast<float*>(raw + kARaw);   // [8][n_t] (wide: [4][n_t]) column-sum partials: reuse the B part of raw slot 0 after the last slab
     uint64_t* afull = reinterpret_cast<uint64_t*>(raw + R * slot_bytes);   // [S] 128 producer arrivals
     uint64_t* afree = afull + S;                             // [S] MMAs of the stage completed
     uint64_t* rfull = afree + S;                             // [R] raw slab landed
@@ -2281,12 +2282,12 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
     const uint32_t accw = (WIDE ? 32u : 64u) * (uint32_t)nbk;   // accumulator columns
     if (tid == 0) {
         for (int i = 0; i < S; ++i) {
-            mbar_init(&afull[i], 256);
+            mbar_init(&afull[i], 128 + 256);
             mbar_init(&afree[i], 1);
         }
         for (int i = 0; i < R; ++i) {
             mbar_init(&rfull[i], 1);
-            mbar_init(&rfree[i], 8);
+            mbar_init(&rfree[i], 4 + 8);
         }
         mbar_init(tfull, 1);
     }
@@ -2379,8 +2380,8 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
         // ------------------------------------------------------------ B producers: split (and mask) the B slab into the
         // operand tile, keep its column sums.  16-byte column chunk b_cc of rows b_r0 + BSTEP i.
         const int tb = tid - 256;
-        const int b_cc = WIDE ? (tb & 63) : (tb & 31), b_r0 = WIDE ? (tb >> 6) : (tb >> 5);
-        constexpr int BI = WIDE ? 16 : 8, BSTEP = WIDE ? 2 : 4;
+        const int b_cc = WIDE ? (tb & 63) : (tb & 31), b_r0 = WIDE ? (tb >> 6) : (tb >> 5);   // 256 threads
+        constexpr int BI = WIDE ? 8 : 4, BSTEP = WIDE ? 4 : 8;
         const int nq = pl.n_t / 4;
         const bool b_mine = b_cc < nq;
         float4 csum = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -2431,12 +2432,13 @@ __global__ void __launch_bounds__(kWtThreads, 1) tc_wgrad_ts_kernel(const WgradA
         if (!okp && lane == 0) atomicExch(fault, 8);
         // column sums of this chunk's rows: the row groups of each column chunk, added in a fixed order
         if (colsum && (pl.b_cols_per_tile > 0 || mt == 0)) {
-            asm volatile("bar.sync 1, 128;" ::: "memory");   // every B producer has read its last raw slab
-            if (b_mine) *reinterpret_cast<float4*>(csum_s + b_r0 * (WIDE ? 256 : 128) + b_cc * 4) = csum;
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            for (int cidx = tb; cidx < pl.n_t; cidx += 128) {
-                const float sum = WIDE ? csum_s[cidx] + csum_s[256 + cidx]
-                                       : ((csum_s[cidx] + csum_s[128 + cidx]) + csum_s[256 + cidx]) + csum_s[384 + cidx];
+            asm volatile("bar.sync 1, 256;" ::: "memory");   // every B producer has read its last raw slab
+            if (b_mine) *reinterpret_cast<float4*>(csum_s + b_r0 * pl.n_t + b_cc * 4) = csum;   // (inside the slot's B part: 128 n_t bytes)
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            for (int cidx = tb; cidx < pl.n_t; cidx += 256) {
+                float sum = 0.f;   // the row groups' partial sums in a fixed order
+#pragma unroll
+                for (int rg = 0; rg < (WIDE ? 4 : 8); ++rg) sum += csum_s[rg * pl.n_t + cidx];
                 colsum[((int64_t)chunk * pl.m_tiles + mt) * pl.n_t + cidx] = cidx < pl.n_valid ? sum : 0.f;
             }
         }
