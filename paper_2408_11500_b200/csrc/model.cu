@@ -622,7 +622,7 @@ struct EpochLayout {
     uint8_t* cls_mask = nullptr;
     uint8_t* ff_mask = nullptr;
     int64_t ld_clsm = 0, ld_ffm = 0;
-    bool gate_masks = false;
+    bool cls_masks = false, ff_masks = false;   // the ReLU of the classifier / of the fusion MLP leaves a byte mask
     float* logits = nullptr;
     float* dlogits = nullptr;
     float* row_loss = nullptr;
@@ -685,11 +685,63 @@ slicegcn_status_t build_layout(const slicegcn_model* m, const slicegcn_graph* g,
     // The ReLUs of the classifier and of the fusion MLP leave a byte mask; their backward products are stored ungated
     // and the consumers multiply by the mask in their producers (see the classifier's backward below).  Without the
     // masks (SLICEGCN_GATE_MASKS=0: the tests reach both forms) the products are gated by the activation in their epilogue.
-    E.gate_masks = true;
-    if (const char* force = getenv("SLICEGCN_GATE_MASKS")) E.gate_masks = atoi(force) != 0;
+    // That pays where the consumers' kernels take a mask (probed here with the shapes and leading dimensions of this
+    // model; the pointers are aligned stand-ins that nothing dereferences); elsewhere a byte mask is still cheaper
+    // to read back than the activation once the activation is far larger than the L2.
+    {
+        void* const fake = reinterpret_cast<void*>(static_cast<uintptr_t>(1) << 20);
+        const bool big = n * E.ld_cls * esz >= ((int64_t)512 << 20);
+        WgradArgs w1;   // dWc1 = H^T (dA * mask)
+        w1.fault = static_cast<int*>(fake);
+        w1.M = n;
+        w1.K = p * m->h_s;
+        w1.N = D.hidden;
+        w1.A = fake;
+        w1.lda = E.ld_h;
+        w1.a_dtype = D.dtype;
+        w1.B = static_cast<const float*>(fake);
+        w1.ldb = E.ld_cls;
+        w1.dW = static_cast<float*>(fake);
+        w1.dbias = static_cast<float*>(fake);
+        w1.b_mask = static_cast<const uint8_t*>(fake);
+        w1.b_mask_ld = E.ld_clsm;
+        GemmArgs h;     // dH = (dA * mask) Wc1^T
+        h.fault = static_cast<int*>(fake);
+        h.b_image = fake;
+        h.b_image_bytes = (int64_t)1 << 60;
+        h.M = n;
+        h.K = D.hidden;
+        h.N = p * m->h_s;
+        h.A = fake;
+        h.lda = E.ld_cls;
+        h.B = static_cast<const float*>(fake);
+        h.ldb = D.hidden;
+        h.b_trans = 1;
+        h.C = fake;
+        h.ldc = gw;
+        h.a_mask = static_cast<const uint8_t*>(fake);
+        h.a_mask_ld = E.ld_clsm;
+        E.cls_masks = big || (wgrad_masks_in_producer(w1) && tc_gemm_masks_in_producer(h));
+        WgradArgs f1;   // dW1 = X^T (dact * mask) of the fusion MLP
+        f1.fault = static_cast<int*>(fake);
+        f1.M = n;
+        f1.K = D.in_d;
+        f1.N = D.in_d;
+        f1.A = fake;
+        f1.lda = m->repack_ff_input(x_ld) ? align_up(D.in_d, 8) : x_ld;
+        f1.a_dtype = D.dtype;
+        f1.B = static_cast<const float*>(fake);
+        f1.ldb = gw;
+        f1.dW = static_cast<float*>(fake);
+        f1.dbias = static_cast<float*>(fake);
+        f1.b_mask = static_cast<const uint8_t*>(fake);
+        f1.b_mask_ld = E.ld_ffm;
+        E.ff_masks = D.use_ff && (big || wgrad_masks_in_producer(f1));
+        if (const char* force = getenv("SLICEGCN_GATE_MASKS")) E.cls_masks = E.ff_masks = atoi(force) != 0;
+    }
     if (D.use_ff) {
         E.ff_act = b.take(n * E.ld_ffact * esz);
-        if (E.gate_masks) E.ff_mask = static_cast<uint8_t*>(b.take(n * E.ld_ffm));
+        if (E.ff_masks) E.ff_mask = static_cast<uint8_t*>(b.take(n * E.ld_ffm));
         E.xff = b.take(n * E.ld_x0 * esz);
     }
     if (m->repack_input()) {
@@ -715,7 +767,7 @@ slicegcn_status_t build_layout(const slicegcn_model* m, const slicegcn_graph* g,
         ws_need = std::max(ws_need, std::max(layer_fwd_ws_bytes(g, pl), layer_bwd_ws_bytes(g, pl)));
     }
     E.cls_act = b.take(n * E.ld_cls * esz);
-    if (E.gate_masks) E.cls_mask = static_cast<uint8_t*>(b.take(n * E.ld_clsm));
+    if (E.cls_masks) E.cls_mask = static_cast<uint8_t*>(b.take(n * E.ld_clsm));
     E.logits = static_cast<float*>(b.take(n * (int64_t)D.num_classes * 4));
     E.ld_dlog = align_up(D.num_classes, 4);
     E.dlogits = static_cast<float*>(b.take(n * E.ld_dlog * 4));
@@ -1088,7 +1140,7 @@ static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, 
         a.ldb = D.in_d;
         a.bias = params + m->ff_b1;
         a.relu = 1;
-        if (E.gate_masks) {
+        if (E.ff_masks) {
             a.mask_out = E.ff_mask;
             a.mask_ld = E.ld_ffm;
         }
@@ -1185,7 +1237,7 @@ static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, 
         a.ldb = D.hidden;
         a.bias = params + m->bc1;
         a.relu = 1;
-        if (E.gate_masks) {
+        if (E.cls_masks) {
             a.mask_out = E.cls_mask;
             a.mask_ld = E.ld_clsm;
         }
@@ -1250,7 +1302,7 @@ static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, 
         a.mul_pos = E.cls_act;
         a.mul_pos_ld = E.ld_cls;
         a.mul_pos_dtype = D.dtype;
-        if (E.gate_masks) {   // the byte mask of the forward ReLU: a quarter (bf16: half) of the activation's bytes
+        if (E.cls_masks) {   // the byte mask of the forward ReLU: a quarter (bf16: half) of the activation's bytes
             a.mul_pos = E.cls_mask;
             a.mul_pos_ld = E.ld_clsm;
             a.mul_pos_dtype = kGateBytes;
@@ -1282,7 +1334,7 @@ static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, 
         h.b_trans = 1;
         h.C = E.dH[0];
         h.ldc = E.ld_grad;
-        if (E.gate_masks) {
+        if (E.cls_masks) {
             // A gate read in the epilogue costs that product two thirds of its time (its loads queue behind the
             // epilogue's own stores: 421 us with the gate against 140 us without, on a fifth of the largest
             // workload).  Both consumers of dA can multiply by the byte mask on their operand's way to the tensor
@@ -1356,7 +1408,7 @@ static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, 
         a.mul_pos = E.ff_act;
         a.mul_pos_ld = E.ld_ffact;
         a.mul_pos_dtype = D.dtype;
-        if (E.gate_masks) {
+        if (E.ff_masks) {
             a.mul_pos = E.ff_mask;
             a.mul_pos_ld = E.ld_ffm;
             a.mul_pos_dtype = kGateBytes;
@@ -1374,7 +1426,7 @@ static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, 
         w1.ldb = E.ld_grad;
         w1.dW = grads + m->ff_W1;
         w1.dbias = grads + m->ff_b1;
-        if (E.gate_masks) {   // as for the classifier: the one consumer of this gradient applies the mask itself
+        if (E.ff_masks) {   // as for the classifier: the one consumer of this gradient applies the mask itself
             WgradArgs w1m = w1;
             w1m.b_mask = E.ff_mask;
             w1m.b_mask_ld = E.ld_ffm;

@@ -513,6 +513,11 @@ def _compare_epoch(gp, od, og, X, y, params, train_idx, tol, rnd=orc.identity, o
     dict(p=3, in_d=48, hidden=512, C=12, L=2, n=700, use_se=True, relu_margin=5e-5),
     dict(p=3, in_d=128, hidden=128, C=10, L=3, n=1500, slice_rule=1, use_se=True, use_b_self=True),
     dict(p=3, in_d=128, hidden=128, C=10, L=2, n=1500, slice_rule=1, use_ff=True, use_se=True),
+    # the co-purchase model's shapes in fp32: 13-wide fused input shared by 8 slices of 32 (its masked weight gradient
+    # runs as two launches over runs of four groups), 256-wide classifier (masked dWc1 as two column blocks of 128),
+    # 47 classes (logits rows without 16-byte alignment: element-wise stores)
+    dict(p=8, in_d=100, hidden=256, C=47, L=2, n=900, use_ff=True, use_se=True),
+    dict(p=8, in_d=100, hidden=256, C=47, L=3, n=1400, use_ff=True, order=1),
 ])
 def test_epoch_gradients_fp32(B, kw):
     kw = dict(kw)
