@@ -320,6 +320,40 @@ slicegcn_status_t slicegcn_train_epoch_dropout(const slicegcn_model* m, const sl
                                                float* logits_out, float* loss_out, void* workspace, int64_t workspace_bytes,
                                                void* stream);
 
+/* The paper's own placement (Section IV-A, Eq. 8): slice i of the features lives on its own device, the graph is
+ * replicated, nothing is exchanged during message passing, and the slices' outputs H^i meet once, for the
+ * concatenation in front of the classifier.  One process per GPU calls this entry point with the SAME model, graph,
+ * X, labels and parameter buffers' contents, and its own range [slice_begin, slice_end) of the p slices: the sliced
+ * layers (Eq. 6, 7) run for those slices only; the fusion MLP (Eq. 4), the classifier (Eq. 9), the loss and the Adam
+ * step run on every rank with identical inputs, so the parameters stay replicas without being sent.  The library
+ * does no communication itself; at three points it calls `exchange` (on the host, work queued on `stream` so far is
+ * the caller's to order against):
+ *   SLICEGCN_EXCHANGE_GATHER_H   buf [device, m's dtype, rows x (p*h_s), leading dimension ld]: columns
+ *                                [col0, col0 + cols) hold this rank's slice outputs; on return every column must
+ *                                hold its owner's values (an all-gather of column blocks: Eq. 8)
+ *   SLICEGCN_EXCHANGE_SUM_DXFF   (feature-fusion models) buf [device, fp32, rows x cols, leading dimension ld]: this
+ *                                rank's part of the gradient of the fused input X_ff, which every slice reads; on
+ *                                return the sum over ranks
+ *   SLICEGCN_EXCHANGE_SUM_GRADS  buf = grads [device, fp32, `rows` elements, ld = cols = 1]: per-slice tensors hold
+ *                                this rank's slices (zeros elsewhere), replicated tensors are non-zero on the rank with
+ *                                slice_begin == 0 only; on return the sum over ranks
+ * `exchange` returns SLICEGCN_OK or an error code, which ends the call with that code (nothing is updated then).
+ * With slice_begin = 0, slice_end = p and exchange = NULL this is slicegcn_train_epoch.  Not combined with dropout,
+ * the input aggregate cache or per-slice widths that need the padded internal layout (UNSUPPORTED).
+ * Errors: INVALID_ARG (empty or out-of-range slice range, exchange NULL for a partial range), and those of
+ * slicegcn_train_epoch. */
+#define SLICEGCN_EXCHANGE_GATHER_H 1
+#define SLICEGCN_EXCHANGE_SUM_DXFF 2
+#define SLICEGCN_EXCHANGE_SUM_GRADS 3
+typedef slicegcn_status_t (*slicegcn_exchange_fn)(void* ctx, int32_t what, void* buf, int64_t rows, int64_t ld, int32_t col0,
+                                                  int32_t cols, int32_t dtype, void* stream);
+slicegcn_status_t slicegcn_train_epoch_sliced(const slicegcn_model* m, const slicegcn_graph* g, const void* X, int64_t x_ld,
+                                              const int32_t* labels, const int32_t* train_idx, int64_t n_train,
+                                              float* params, float* grads, float* adam_m, float* adam_v,
+                                              const slicegcn_opt_desc* opt, int32_t slice_begin, int32_t slice_end,
+                                              slicegcn_exchange_fn exchange, void* exchange_ctx, float* logits_out,
+                                              float* loss_out, void* workspace, int64_t workspace_bytes, void* stream);
+
 /* Forgets what the model object remembers about earlier calls (the input aggregate cache above).  Host only. */
 slicegcn_status_t slicegcn_model_invalidate_caches(const slicegcn_model* m);
 

@@ -32,7 +32,7 @@ EXPORTS = [
     "slicegcn_spmm", "slicegcn_spmm_static_scratch", "slicegcn_layer_saved_bytes", "slicegcn_layer_saved_layout", "slicegcn_layer_workspace_bytes", "slicegcn_layer_forward",
     "slicegcn_layer_backward", "slicegcn_model_create", "slicegcn_model_destroy", "slicegcn_model_invalidate_caches", "slicegcn_model_param_count",
     "slicegcn_model_param_elems", "slicegcn_model_num_tensors", "slicegcn_model_tensor_info", "slicegcn_model_slices",
-    "slicegcn_model_layer_order", "slicegcn_train_workspace_bytes", "slicegcn_train_epoch", "slicegcn_train_epoch_dropout", "slicegcn_forward_logits", "slicegcn_train_epoch_host", "slicegcn_train_epochs_host", "slicegcn_profile_begin", "slicegcn_profile_begin_sampled",
+    "slicegcn_model_layer_order", "slicegcn_train_workspace_bytes", "slicegcn_train_epoch", "slicegcn_train_epoch_dropout", "slicegcn_train_epoch_sliced", "slicegcn_forward_logits", "slicegcn_train_epoch_host", "slicegcn_train_epochs_host", "slicegcn_profile_begin", "slicegcn_profile_begin_sampled",
     "slicegcn_profile_end",
 ]
 
@@ -331,6 +331,27 @@ def slicegcn_train_epoch_dropout(m, g, X, x_ld: int, labels, train_idx, n_train:
                                              byref(opt) if opt is not None else None,
                                              byref(drop) if drop is not None else None, _vp(logits_out), _vp(loss_out),
                                              _vp(workspace), c_int64(workspace_bytes), _vp(stream)))
+
+
+EXCHANGE_GATHER_H, EXCHANGE_SUM_DXFF, EXCHANGE_SUM_GRADS = 1, 2, 3
+ExchangeFn = ctypes.CFUNCTYPE(c_int32, c_void_p, c_int32, c_void_p, c_int64, c_int64, c_int32, c_int32, c_int32, c_void_p)
+
+
+def slicegcn_train_epoch_sliced(m, g, X, x_ld: int, labels, train_idx, n_train: int, params, grads, adam_m, adam_v,
+                                opt: Optional[OptDesc], slice_begin: int, slice_end: int, exchange, logits_out, loss_out,
+                                workspace, workspace_bytes: int, stream=None) -> None:
+    """exchange(what, buf_address, rows, ld, col0, cols, dtype, stream_address) -> status (0 = OK), or None."""
+    def trampoline(_ctx, what, buf, rows, ld, col0, cols, dtype, st):
+        try:
+            return int(exchange(what, buf, rows, ld, col0, cols, dtype, st) or 0)
+        except Exception:          # an exception must not cross the C frames
+            return ERR_INVALID_ARG
+    fn = ExchangeFn(trampoline) if exchange is not None else ctypes.cast(None, ExchangeFn)
+    _check(_lib.slicegcn_train_epoch_sliced(m, g, _vp(X), c_int64(x_ld), _vp(labels), _vp(train_idx), c_int64(n_train),
+                                            _vp(params), _vp(grads), _vp(adam_m), _vp(adam_v),
+                                            byref(opt) if opt is not None else None, c_int32(slice_begin), c_int32(slice_end),
+                                            fn, None, _vp(logits_out), _vp(loss_out), _vp(workspace), c_int64(workspace_bytes),
+                                            _vp(stream)))
 
 
 def slicegcn_forward_logits(m, g, X, x_ld: int, params, logits_out, workspace, workspace_bytes: int, stream=None) -> None:

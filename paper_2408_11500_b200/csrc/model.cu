@@ -1036,14 +1036,23 @@ slicegcn_status_t slicegcn_train_workspace_bytes(const slicegcn_model* m, const 
     return SLICEGCN_OK;
 }
 
+// The slices this process computes and how their outputs meet the other processes' (slicegcn_train_epoch_sliced).
+struct SliceRange {
+    int begin, end;
+    slicegcn_exchange_fn exchange;
+    void* ctx;
+};
+
 // forward_only: stops after the logits (evaluation pass); labels, grads and the optimiser arguments are not used.
 static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, const slicegcn_graph* g, const void* X, int64_t x_ld,
                                     const int32_t* labels, const int32_t* train_idx, int64_t n_train, float* params,
                                     float* grads, float* adam_m, float* adam_v, const slicegcn_opt_desc* opt,
                                     float* logits_out, float* loss_out, void* workspace, int64_t workspace_bytes,
-                                    void* stream, const slicegcn_dropout_desc* drop = nullptr) {
+                                    void* stream, const slicegcn_dropout_desc* drop = nullptr, const SliceRange* sr = nullptr) {
     if (!m || !g || !X || !params || !workspace || (!forward_only && (!labels || !grads)))
         SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "train_epoch: NULL argument");
+    if (sr && (m->inner || drop || forward_only))
+        SGCN_FAIL(SLICEGCN_ERR_UNSUPPORTED, "train_epoch_sliced: not with dropout or per-slice widths that need the padded layout");
     if (m->inner) {
         // padded internal model: parameters in, the whole iteration on the padded shapes, gradients out, then the update
         // on the caller's buffers
@@ -1086,6 +1095,11 @@ static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, 
     cudaStream_t st = (cudaStream_t)stream;
     const int64_t n = g->n;
     const int p = D.num_slices, L = D.num_layers, C = D.num_classes;
+    // the slices computed here: all of them, or this process's range (Section IV-A's placement)
+    const int s0 = sr ? sr->begin : 0, s1 = sr ? sr->end : p, pl = s1 - s0;
+    if (s0 < 0 || s1 > p || pl < 1) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "train_epoch_sliced: slice range outside [0, p)");
+    const bool partial = pl != p;
+    if (partial && !sr->exchange) SGCN_FAIL(SLICEGCN_ERR_INVALID_ARG, "train_epoch_sliced: a partial range needs an exchange function");
     EpochLayout E;
     SGCN_TRY(build_layout(m, g, x_ld, static_cast<char*>(workspace), &E));
     if (workspace_bytes < E.total)
@@ -1113,7 +1127,7 @@ static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, 
     // What a caller who set cache_input_aggregate promises not to change between calls: X (and the workspace).  When
     // this call sees the X, graph, workspace and stream of the previous one, everything computed from X alone is still
     // in the workspace: the padded copy of X below, the repacked slices and the first layer's aggregate further down.
-    const bool x_unchanged = D.cache_input_aggregate && m->zkey.valid && m->zkey.X == X && m->zkey.x_ld == x_ld && m->zkey.graph == g &&
+    const bool x_unchanged = !sr && D.cache_input_aggregate && m->zkey.valid && m->zkey.X == X && m->zkey.x_ld == x_ld && m->zkey.graph == g &&
                              m->zkey.workspace == workspace && m->zkey.stream == stream;
     m->zkey.valid = false;   // until this call has queued the first layer
     const bool ff_repacked = m->repack_ff_input(x_ld);
@@ -1190,6 +1204,17 @@ static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, 
     for (int l = 0; l < L; ++l) {
         layer_desc_for(m, l, params, x_ld, starts[l].data(), &descs[l]);
         if (l == 0) descs[l].in_ld = ld0;
+        if (partial) {   // this process's slices: their input ranges, their blocks of the per-slice tensors
+            slicegcn_layer_desc& d = descs[l];
+            const int64_t wblock = (int64_t)d.in_width * d.h_s;
+            d.num_slices = pl;
+            d.in_starts += s0;
+            d.W_agg += s0 * wblock;
+            if (d.W_self) d.W_self += s0 * wblock;
+            if (d.b) d.b += s0 * d.h_s;
+            if (d.b_self) d.b_self += s0 * d.h_s;
+            if (d.E) d.E += s0 * d.h_s;
+        }
         SGCN_TRY(make_plan(g, &descs[l], &plans[l]));
         if (l == 0 && repacked) {
             // padding columns of the copy are zero, and so are those of its aggregate
@@ -1206,8 +1231,11 @@ static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, 
                 SGCN_CUDA(cudaMemsetAsync(E.saved[l], 0, plans[l].zt_bytes, st));
             }
         }
-        SGCN_TRY(layer_forward_impl(g, &descs[l], plans[l], hin, E.H[l], E.saved[l], E.ws, E.ws_bytes, st, l == 0 && z_cached));
-        if (l == 0 && D.cache_input_aggregate) {
+        // (a partial range writes its own column block of the layer's output; the layers below the last never read
+        // another process's columns)
+        SGCN_TRY(layer_forward_impl(g, &descs[l], plans[l], hin, static_cast<char*>(E.H[l]) + (int64_t)s0 * m->h_s * esize(D.dtype),
+                                    E.saved[l], E.ws, E.ws_bytes, st, l == 0 && z_cached));
+        if (l == 0 && D.cache_input_aggregate && !sr) {
             m->zkey.X = X;
             m->zkey.x_ld = x_ld;
             m->zkey.graph = g;
@@ -1221,6 +1249,8 @@ static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, 
         hin = E.H[l];
     }
     const int HW = p * m->h_s;
+    if (partial)   // Eq. 8: the one exchange of the forward pass -- every process ends up with all slices' outputs
+        SGCN_TRY(sr->exchange(sr->ctx, SLICEGCN_EXCHANGE_GATHER_H, E.H[L - 1], n, E.ld_h, s0 * m->h_s, pl * m->h_s, D.dtype, stream));
     float* logits = logits_out ? logits_out : E.logits;
     {   // classifier (Eq. 9)
         GemmArgs a;
@@ -1362,17 +1392,22 @@ static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, 
         if (drop && l + 1 < L)   // the gradient passes the same mask and scale on its way into the layer
             SGCN_TRY(dropout_apply_run(n, p * m->h_s, E.dH[cur], E.ld_grad, SLICEGCN_F32, drop->masks[l], drop->mask_ld, m->caller_h_s,
                                        m->h_s, drop_scale, st));
-        SGCN_TRY(layer_backward_impl(g, &descs[l], plans[l], lin, E.saved[l], E.dH[cur], E.ld_grad,
-                                     need_din ? E.dH[cur ^ 1] : nullptr, E.ld_grad, grads + m->W_agg[l],
-                                     D.use_self ? grads + m->W_self[l] : nullptr, grads + m->b[l],
-                                     D.use_b_self ? grads + m->b_self[l] : nullptr,
-                                     (D.use_se && l == L - 1) ? grads + m->E : nullptr, E.ws, E.ws_bytes, st));
+        // (s0 = 0 unless this process computes a range of the slices: then its column block of the incoming
+        // gradient and its blocks of the per-slice gradient tensors)
+        const int64_t wb = (int64_t)s0 * descs[l].in_width * m->h_s, vb = (int64_t)s0 * m->h_s;
+        SGCN_TRY(layer_backward_impl(g, &descs[l], plans[l], lin, E.saved[l], E.dH[cur] + vb, E.ld_grad,
+                                     need_din ? E.dH[cur ^ 1] : nullptr, E.ld_grad, grads + m->W_agg[l] + wb,
+                                     D.use_self ? grads + m->W_self[l] + wb : nullptr, grads + m->b[l] + vb,
+                                     D.use_b_self ? grads + m->b_self[l] + vb : nullptr,
+                                     (D.use_se && l == L - 1) ? grads + m->E + vb : nullptr, E.ws, E.ws_bytes, st));
         cur ^= 1;
     }
     if (D.use_ff) {   // backward of the fusion MLP from dX_ff (sum over slices already formed)
         float* dxff = E.dH[cur];
+        if (partial)   // every slice reads X_ff: the other processes' slices contribute too
+            SGCN_TRY(sr->exchange(sr->ctx, SLICEGCN_EXCHANGE_SUM_DXFF, dxff, n, E.ld_grad, 0, m->slice_size, SLICEGCN_F32, stream));
         // aggregate-first first layer: its backward kept the padding columns of dX_ff at zero (see din_pad_write)
-        const bool dxff_pad = plans[0].order == SLICEGCN_AGG_FIRST && p > 1 && align_up(m->slice_size, 4) <= E.ld_grad &&
+        const bool dxff_pad = plans[0].order == SLICEGCN_AGG_FIRST && pl > 1 && align_up(m->slice_size, 4) <= E.ld_grad &&
                               align_up(m->slice_size, 4) <= plans[0].zt_ld;
         WgradArgs w;
         w.fault = g->fault;
@@ -1438,6 +1473,15 @@ static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, 
         SGCN_TRY(gemm_run(a, st));
         SGCN_TRY(wgrad_run(w1, E.ws, E.ws_bytes, st));
     }
+    if (partial) {
+        // The replicated tensors (fusion MLP, classifier) got the same gradient on every process: all but the one with
+        // the first slice clear theirs, so that the sum over processes is the full gradient everywhere.
+        if (s0 != 0)
+            for (const auto& t : m->tensors)
+                if (t.name.rfind("ff_", 0) == 0 || t.name == "Wc1" || t.name == "bc1" || t.name == "Wc2" || t.name == "bc2")
+                    SGCN_CUDA(cudaMemsetAsync(grads + t.offset, 0, sizeof(float) * (size_t)t.dims[0] * t.dims[1] * t.dims[2], st));
+        SGCN_TRY(sr->exchange(sr->ctx, SLICEGCN_EXCHANGE_SUM_GRADS, grads, m->param_elems, 1, 0, 1, SLICEGCN_F32, stream));
+    }
     // ---------------- update: Adam, cosine-annealed learning rate, one step per epoch
     if (opt) {
         const double kPi = 3.14159265358979323846;
@@ -1455,6 +1499,17 @@ slicegcn_status_t slicegcn_train_epoch(const slicegcn_model* m, const slicegcn_g
                                        void* stream) {
     return epoch_impl(false, m, g, X, x_ld, labels, train_idx, n_train, params, grads, adam_m, adam_v, opt, logits_out, loss_out,
                       workspace, workspace_bytes, stream);
+}
+
+slicegcn_status_t slicegcn_train_epoch_sliced(const slicegcn_model* m, const slicegcn_graph* g, const void* X, int64_t x_ld,
+                                              const int32_t* labels, const int32_t* train_idx, int64_t n_train,
+                                              float* params, float* grads, float* adam_m, float* adam_v,
+                                              const slicegcn_opt_desc* opt, int32_t slice_begin, int32_t slice_end,
+                                              slicegcn_exchange_fn exchange, void* exchange_ctx, float* logits_out,
+                                              float* loss_out, void* workspace, int64_t workspace_bytes, void* stream) {
+    const SliceRange sr{slice_begin, slice_end, exchange, exchange_ctx};
+    return epoch_impl(false, m, g, X, x_ld, labels, train_idx, n_train, params, grads, adam_m, adam_v, opt, logits_out, loss_out,
+                      workspace, workspace_bytes, stream, nullptr, &sr);
 }
 
 slicegcn_status_t slicegcn_train_epoch_dropout(const slicegcn_model* m, const slicegcn_graph* g, const void* X, int64_t x_ld,
