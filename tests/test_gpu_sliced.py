@@ -154,3 +154,31 @@ def test_sliced_epoch_argument_errors(B):
         assert e.value.status == B.ERR_UNSUPPORTED
     finally:
         gp.close()
+
+
+def test_exchange_on_device_buffers_single_process_group(B):
+    """`slice_exchange.make_exchange` on device memory: the address views (fp32 and bf16), the stream hand-over and the
+    NCCL calls, in a process group of one (the only size one GPU allows): every step must leave the data as it is."""
+    import socket
+    import torch
+    import torch.distributed as dist
+    s = socket.socket(); s.bind(("127.0.0.1", 0)); port = s.getsockname()[1]; s.close()
+    dist.init_process_group("nccl", init_method=f"tcp://127.0.0.1:{port}", rank=0, world_size=1)
+    try:
+        ex = sx.make_exchange(None, device="cuda")
+        st = torch.cuda.Stream()
+        with torch.cuda.stream(st):
+            H = torch.randn(300, 40, device="cuda")
+            Hb = torch.randn(300, 40, device="cuda").to(torch.bfloat16)
+            d = torch.randn(300, 16, device="cuda")
+            gvec = torch.randn(5000, device="cuda")
+            keep = [t.clone() for t in (H, Hb, d, gvec)]
+            assert ex(B.EXCHANGE_GATHER_H, H.data_ptr(), 300, 40, 0, 32, B.F32, st.cuda_stream) == B.OK
+            assert ex(B.EXCHANGE_GATHER_H, Hb.data_ptr(), 300, 40, 0, 32, B.BF16, st.cuda_stream) == B.OK
+            assert ex(B.EXCHANGE_SUM_DXFF, d.data_ptr(), 300, 16, 0, 13, B.F32, st.cuda_stream) == B.OK
+            assert ex(B.EXCHANGE_SUM_GRADS, gvec.data_ptr(), 5000, 1, 0, 1, B.F32, st.cuda_stream) == B.OK
+        st.synchronize()
+        for a, b in zip((H, Hb, d, gvec), keep):
+            assert torch.equal(a, b)
+    finally:
+        dist.destroy_process_group()
