@@ -71,6 +71,8 @@ def test_static_scratch_transposed_directed_graph_and_no_allocation():
         Y = torch.empty_like(X)
         B.slicegcn_spmm_static_scratch(g, 1, B.F32, B.F32, X, 64, Y, 64, 64, None)   # the first call looks the buffer up
         torch.cuda.synchronize()
+        import gc
+        gc.collect()                # tensors of earlier tests that only a reference cycle keeps alive go now, not mid-measurement
         free0, alloc0, reserved0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
         for transpose in (1, 0, 1):
             B.slicegcn_spmm_static_scratch(g, transpose, B.F32, B.F32, X, 64, Y, 64, 64, None)
