@@ -1200,15 +1200,24 @@ static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, 
     std::vector<slicegcn_layer_desc> descs(L);
     std::vector<LayerPlan> plans(L);
     std::vector<std::vector<int>> starts(L, std::vector<int>(SLICEGCN_MAX_SLICES));
+    std::vector<int> win(L, 0);   // first input column of each layer's window (0 unless this process computes a range of the slices)
     const void* hin = h0;
     for (int l = 0; l < L; ++l) {
         layer_desc_for(m, l, params, x_ld, starts[l].data(), &descs[l]);
         if (l == 0) descs[l].in_ld = ld0;
-        if (partial) {   // this process's slices: their input ranges, their blocks of the per-slice tensors
+        if (partial) {   // this process's slices: their blocks of the per-slice tensors, and as the layer's input the
+                         // window of columns they read (so that the layer sees slices tiling its input, as always)
             slicegcn_layer_desc& d = descs[l];
             const int64_t wblock = (int64_t)d.in_width * d.h_s;
+            int lo = starts[l][s0], hi = starts[l][s0] + d.in_width;
+            for (int i = s0; i < s1; ++i) {
+                lo = std::min(lo, starts[l][i]);
+                hi = std::max(hi, starts[l][i] + d.in_width);
+            }
+            for (int i = 0; i < pl; ++i) starts[l][i] = starts[l][s0 + i] - lo;
+            win[l] = lo;
+            d.in_cols = hi - lo;
             d.num_slices = pl;
-            d.in_starts += s0;
             d.W_agg += s0 * wblock;
             if (d.W_self) d.W_self += s0 * wblock;
             if (d.b) d.b += s0 * d.h_s;
@@ -1233,7 +1242,8 @@ static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, 
         }
         // (a partial range writes its own column block of the layer's output; the layers below the last never read
         // another process's columns)
-        SGCN_TRY(layer_forward_impl(g, &descs[l], plans[l], hin, static_cast<char*>(E.H[l]) + (int64_t)s0 * m->h_s * esize(D.dtype),
+        SGCN_TRY(layer_forward_impl(g, &descs[l], plans[l], static_cast<const char*>(hin) + (int64_t)win[l] * esize(D.dtype),
+                                    static_cast<char*>(E.H[l]) + (int64_t)s0 * m->h_s * esize(D.dtype),
                                     E.saved[l], E.ws, E.ws_bytes, st, l == 0 && z_cached));
         if (l == 0 && D.cache_input_aggregate && !sr) {
             m->zkey.X = X;
@@ -1395,8 +1405,9 @@ static slicegcn_status_t epoch_impl(bool forward_only, const slicegcn_model* m, 
         // (s0 = 0 unless this process computes a range of the slices: then its column block of the incoming
         // gradient and its blocks of the per-slice gradient tensors)
         const int64_t wb = (int64_t)s0 * descs[l].in_width * m->h_s, vb = (int64_t)s0 * m->h_s;
-        SGCN_TRY(layer_backward_impl(g, &descs[l], plans[l], lin, E.saved[l], E.dH[cur] + vb, E.ld_grad,
-                                     need_din ? E.dH[cur ^ 1] : nullptr, E.ld_grad, grads + m->W_agg[l] + wb,
+        SGCN_TRY(layer_backward_impl(g, &descs[l], plans[l], static_cast<const char*>(lin) + (int64_t)win[l] * esize(D.dtype), E.saved[l],
+                                     E.dH[cur] + vb, E.ld_grad, need_din ? E.dH[cur ^ 1] + win[l] : nullptr, E.ld_grad,
+                                     grads + m->W_agg[l] + wb,
                                      D.use_self ? grads + m->W_self[l] + wb : nullptr, grads + m->b[l] + vb,
                                      D.use_b_self ? grads + m->b_self[l] + vb : nullptr,
                                      (D.use_se && l == L - 1) ? grads + m->E + vb : nullptr, E.ws, E.ws_bytes, st));
